@@ -1,0 +1,558 @@
+"""CPU oracle for the HAC / sHAC formats and their compressed-domain product.
+
+TEST INFRASTRUCTURE ONLY: the slow, plain fp64 reference that the CUDA library
+is compared with.  It shares no code with that library; only tests, the smoke
+check and the CPU-baseline leg of the benchmark may import it.
+
+Each function states the passage of the paper it follows (Marino, Petrini,
+Malchiodi, Frasca, "Compact representations of convolutional neural networks
+via weight pruning and quantization").  Where the paper leaves a choice open
+(ties, initialisation, bit order, which optimal Huffman code) the rule taken is
+written in the docstring.  The loops that would be too slow in Python live in
+hac_oracle.c (k-means sweeps, bit-by-bit packing, Algorithms 1-3).
+
+Parity unpinned: `kmeans_share` has no value printed by the paper to compare
+with; it is held by invariants only (see tests/test_oracle_quantizers.py).
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+import subprocess
+from collections import deque
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_SRC = os.path.join(_HERE, "hac_oracle.c")
+_LIB = os.path.join(_HERE, "libhac_oracle.so")
+
+B_WORD = 32          # b: bits of one memory word (FP32 weights), Sect. IV-A
+MAX_SYMBOLS = 2048   # larger alphabets are rejected by both implementations
+
+
+def build_native(force: bool = False) -> str:
+    """Compile hac_oracle.c with gcc (plain C, no fast-math, no FMA contraction)."""
+    if force or not os.path.exists(_LIB) or os.path.getmtime(_LIB) < os.path.getmtime(_SRC):
+        tmp = _LIB + f".tmp{os.getpid()}"
+        subprocess.check_call(["gcc", "-O2", "-std=c11", "-fPIC", "-shared", "-ffp-contract=off",
+                               "-fno-fast-math", "-pthread", _SRC, "-o", tmp, "-lm"])
+        os.replace(tmp, _LIB)
+    return _LIB
+
+
+_lib = None
+
+
+def _native():
+    global _lib
+    if _lib is None:
+        _lib = ctypes.CDLL(build_native())
+        _lib.orc_pack.restype = ctypes.c_int64
+        _lib.orc_decode.restype = ctypes.c_int64
+    return _lib
+
+
+def _p(a):
+    return a.ctypes.data_as(ctypes.c_void_p)
+
+
+# ----------------------------------------------------------------------------
+# Sect. III-B  weight pruning
+# ----------------------------------------------------------------------------
+def prune(W: np.ndarray, sparsity: float) -> np.ndarray:
+    """Magnitude pruning (Sect. III-B): fix a percentile w_p of the magnitudes
+    and keep w only where |w| > w_p.
+
+    Reading: z = floor(sparsity * n*m) entries are to go; w_p is the z-th
+    smallest magnitude itself (an order statistic, no interpolation); every
+    entry with |w| <= w_p becomes 0, so ties at w_p are all pruned.  z = 0
+    leaves W unchanged.  Non-finite inputs are rejected; -0.0 becomes +0.0.
+    """
+    W = np.asarray(W, dtype=np.float32)
+    if not np.all(np.isfinite(W)):
+        raise ValueError("non-finite weight")
+    out = W.copy()
+    out[out == 0] = np.float32(0.0)
+    if not (0.0 <= sparsity < 1.0):
+        raise ValueError("sparsity must be in [0, 1)")
+    z = int(np.floor(np.float64(sparsity) * np.float64(W.size)))
+    if z == 0:
+        return out
+    mag = np.abs(out).ravel()
+    w_p = np.sort(mag)[z - 1]
+    out[np.abs(out) <= w_p] = np.float32(0.0)
+    return out
+
+
+# ----------------------------------------------------------------------------
+# SplitMix64 (Steele, Lea, Flood, "Fast splittable pseudorandom number
+# generators", OOPSLA 2014), used as a counter-based generator: the i-th draw
+# mixes seed + (i + 1) * gamma.  Only the k-means initialisation draws numbers.
+# ----------------------------------------------------------------------------
+_M64 = (1 << 64) - 1
+
+
+def splitmix64(seed: int, i: int) -> int:
+    z = (seed + (i + 1) * 0x9E3779B97F4A7C15) & _M64
+    z = ((z ^ (z >> 30)) * 0xBF58476D1CE4E5B9) & _M64
+    z = ((z ^ (z >> 27)) * 0x94D049BB133111EB) & _M64
+    return z ^ (z >> 31)
+
+
+def kmeans_init(u: np.ndarray, k: int, seed: int) -> np.ndarray:
+    """k distinct starting centroids: a partial Fisher-Yates shuffle of the
+    sorted distinct values u, draw i swapping position i with position
+    i + (r_i mod (len(u) - i)); the first k entries, sorted ascending."""
+    idx = np.arange(len(u), dtype=np.int64)
+    for i in range(k):
+        j = i + splitmix64(seed, i) % (len(u) - i)
+        idx[i], idx[j] = idx[j], idx[i]
+    return np.sort(u[idx[:k]])
+
+
+# ----------------------------------------------------------------------------
+# Sect. III-C  weight sharing
+# ----------------------------------------------------------------------------
+def _nonnull_colmajor(Wp: np.ndarray):
+    """Non-null weights of the pruned matrix listed by columns (the order of
+    the CSC vector nz, Sect. IV-A), and the boolean mask they come from."""
+    mask = Wp != 0
+    return Wp.T[mask.T].astype(np.float64), mask
+
+
+def _scatter_colmajor(mask: np.ndarray, values32: np.ndarray) -> np.ndarray:
+    Wq = np.zeros(mask.shape, dtype=np.float32)
+    WqT = Wq.T                      # view: assignment in column-major order
+    WqT[mask.T] = values32
+    Wq[Wq == 0] = np.float32(0.0)   # a centroid that rounds to -0.0 is stored as +0.0
+    return Wq
+
+
+def kmeans_share(Wp: np.ndarray, k: int, iters: int, seed: int, return_trace: bool = False):
+    """CWS (Sect. III-C.1): k-means over the non-null weights (pruning and CWS
+    in chain cluster only the weights that survived pruning), every weight
+    replaced by its centroid.
+
+    Reading (the paper only says "k-means"): Lloyd iterations, exactly `iters`
+    of them, in fp64, on the weights in column-major storage order; seeded
+    start from k distinct data values (kmeans_init); nearest centroid through
+    midpoints, ties to the lower centroid; empty clusters keep their centroid;
+    after the last update one more assignment.  If the data has at most k
+    distinct values they are the codebook.  Centroids are rounded to fp32 when
+    they replace the weights, so fewer than k shared values may remain.
+    Returns (Wq, mask) with mask the positions of the non-null weights.
+    """
+    data, mask = _nonnull_colmajor(Wp)
+    if k < 1:
+        raise ValueError("k must be >= 1")
+    if data.size == 0:
+        return (np.zeros_like(Wp), mask) if not return_trace else (np.zeros_like(Wp), mask, None, None)
+    u = np.unique(data)
+    if len(u) <= k:
+        Wq = _scatter_colmajor(mask, data.astype(np.float32))
+        return (Wq, mask) if not return_trace else (Wq, mask, u, None)
+    c = np.ascontiguousarray(kmeans_init(u, k, seed), dtype=np.float64)
+    assign = np.empty(data.size, dtype=np.int32)
+    sse = np.zeros(iters + 1, dtype=np.float64)
+    data = np.ascontiguousarray(data)
+    rc = _native().orc_kmeans(_p(data), ctypes.c_int64(data.size), _p(c), ctypes.c_int32(k),
+                              ctypes.c_int32(iters), _p(assign), _p(sse))
+    if rc != 0:
+        raise RuntimeError(f"orc_kmeans failed: {rc}")
+    Wq = _scatter_colmajor(mask, c.astype(np.float32)[assign])
+    if return_trace:
+        return Wq, mask, c, sse
+    return Wq, mask
+
+
+def uniform_share(Wp: np.ndarray, k: int):
+    """UQ (Sect. III-C.3): representatives spaced uniformly in the weight domain,
+    w = delta * round(w0 / delta) with the grid laid over the range of the
+    non-null weights so that it has exactly k levels:
+    lo = min, hi = max, delta = (hi - lo) / (k - 1),
+    level(w) = floor((w - lo) / delta + 1/2) clamped to [0, k-1] (round half up),
+    value = fp32(lo + level * delta).  Levels nobody falls in are not part of
+    the codebook.  Returns (Wq, mask)."""
+    data, mask = _nonnull_colmajor(Wp)
+    if k < 2:
+        raise ValueError("uniform quantization needs k >= 2")
+    if data.size == 0:
+        return np.zeros_like(Wp), mask
+    lo = data.min()
+    hi = data.max()
+    if hi == lo:
+        return _scatter_colmajor(mask, data.astype(np.float32)), mask
+    delta = (hi - lo) / np.float64(k - 1)
+    level = np.floor((data - lo) / delta + 0.5)
+    level = np.clip(level, 0.0, np.float64(k - 1))
+    values = (lo + level * delta).astype(np.float32)
+    return _scatter_colmajor(mask, values), mask
+
+
+def share_none(Wp: np.ndarray):
+    """No weight sharing: the matrix already holds few distinct values."""
+    Wq = Wp.copy()
+    Wq[Wq == 0] = np.float32(0.0)
+    return Wq, Wq != 0
+
+
+def quantize(W: np.ndarray, sparsity: float, k: int, quantizer: int, iters: int = 20, seed: int = 0):
+    """Pruning then weight sharing, as chained in Sect. III-C.1.  quantizer:
+    0 none, 1 k-means (CWS), 2 uniform (UQ).  Returns (Wq, mask)."""
+    Wp = prune(W, sparsity)
+    if quantizer == 0:
+        return share_none(Wp)
+    if quantizer == 1:
+        return kmeans_share(Wp, k, iters, seed)
+    if quantizer == 2:
+        return uniform_share(Wp, k)
+    raise ValueError("unknown quantizer")
+
+
+# ----------------------------------------------------------------------------
+# Sect. IV-B  Huffman code
+# ----------------------------------------------------------------------------
+def huffman_lengths(counts) -> np.ndarray:
+    """Code word length of every symbol of a Huffman code for `counts`.
+
+    Huffman's construction: repeatedly merge the two least frequent nodes.
+    Which optimal code results depends on how ties are broken; the rule here:
+    leaves sorted by (count, symbol id); merged nodes queue up in creation
+    order; of two candidates with the same weight the leaf is taken before the
+    merged node.  A single-symbol alphabet gets a 1-bit code word (a prefix
+    code needs at least one bit per symbol to be countable in a stream).
+    """
+    counts = [int(c) for c in counts]
+    k = len(counts)
+    if k == 0:
+        return np.zeros(0, dtype=np.uint8)
+    if any(c <= 0 for c in counts):
+        raise ValueError("every symbol of the alphabet must occur")
+    if k == 1:
+        return np.array([1], dtype=np.uint8)
+    parent = {}
+    leaves = deque(sorted(range(k), key=lambda s: (counts[s], s)))
+    weight = {s: counts[s] for s in range(k)}
+    merged = deque()
+    nxt = k
+
+    def take():
+        if leaves and (not merged or weight[leaves[0]] <= weight[merged[0]]):
+            return leaves.popleft()
+        return merged.popleft()
+
+    while len(leaves) + len(merged) > 1:
+        a = take()
+        b = take()
+        weight[nxt] = weight[a] + weight[b]
+        parent[a] = nxt
+        parent[b] = nxt
+        merged.append(nxt)
+        nxt += 1
+    lengths = np.zeros(k, dtype=np.int64)
+    for s in range(k):
+        v, d = s, 0
+        while v in parent:
+            v = parent[v]
+            d += 1
+        lengths[s] = d
+    if lengths.max() > 32:
+        raise ValueError("code word longer than 32 bits")
+    return lengths.astype(np.uint8)
+
+
+def canonical_codes(lengths) -> np.ndarray:
+    """Code words for given lengths: symbols ordered by (length, id); the first
+    gets 0...0, each next one the previous code word plus one, shifted left by
+    the growth in length.  Code words are read most significant bit first.
+    (The paper keeps the dictionaries H and H^-1 as B-trees; any prefix code
+    with Huffman's lengths is an equally valid H.)"""
+    lengths = np.asarray(lengths, dtype=np.int64)
+    order = sorted(range(len(lengths)), key=lambda s: (int(lengths[s]), s))
+    codes = np.zeros(len(lengths), dtype=np.uint32)
+    code = 0
+    prev = None
+    for s in order:
+        if prev is not None:
+            code = (code + 1) << (int(lengths[s]) - prev)
+        codes[s] = code
+        prev = int(lengths[s])
+    return codes
+
+
+def entropy_bits(counts) -> float:
+    p = np.asarray(counts, dtype=np.float64)
+    p = p / p.sum()
+    return float(-(p * np.log2(p)).sum())
+
+
+# ----------------------------------------------------------------------------
+# Sect. IV-A / IV-B / IV-C  the formats
+# ----------------------------------------------------------------------------
+def csc(Wq: np.ndarray, mask: np.ndarray):
+    """CSC of Sect. IV-A: nz (stored values by column, rows ascending), ri (row
+    of each), cb (cb[j] = number of stored entries in columns before j; the
+    paper's cb is this plus one).  Stored entries are those of `mask`."""
+    cols, rows = np.nonzero(mask.T)
+    nz = Wq.T[mask.T].astype(np.float32)
+    cb = np.zeros(mask.shape[1] + 1, dtype=np.int64)
+    np.cumsum(np.bincount(cols, minlength=mask.shape[1]), out=cb[1:])
+    return nz, rows.astype(np.int32), cb
+
+
+def _pack(sym: np.ndarray, codes: np.ndarray, lengths: np.ndarray):
+    total_bits = int(lengths.astype(np.int64)[sym].sum())
+    nwords = (total_bits + B_WORD - 1) // B_WORD
+    words = np.zeros(max(nwords, 1), dtype=np.uint32)
+    sym = np.ascontiguousarray(sym, dtype=np.int32)
+    codes = np.ascontiguousarray(codes, dtype=np.uint32)
+    lengths = np.ascontiguousarray(lengths, dtype=np.uint8)
+    written = _native().orc_pack(_p(sym), ctypes.c_int64(sym.size), _p(codes), _p(lengths),
+                                 _p(words), ctypes.c_int64(nwords))
+    if written != total_bits:
+        raise RuntimeError("orc_pack failed")
+    return words[:nwords], total_bits
+
+
+def _alphabet(values_in_stream_order: np.ndarray):
+    codebook, sym, counts = np.unique(values_in_stream_order, return_inverse=True, return_counts=True)
+    if len(codebook) > MAX_SYMBOLS:
+        raise ValueError("too many distinct values")
+    return codebook.astype(np.float32), sym.astype(np.int32).ravel(), counts.astype(np.int64)
+
+
+def hac_encode(Wq: np.ndarray) -> dict:
+    """HAC (Sect. IV-B): the address map of W in column order with a(z) the
+    Huffman code word of z and the null entries coded like any other value;
+    the bit string is cut into N = ceil(bits / 32) words, the last zero padded.
+    Symbol id = rank of the value among the distinct values (ascending)."""
+    n, m = Wq.shape
+    seq = np.ascontiguousarray(Wq.T).ravel()          # column after column
+    codebook, sym, counts = _alphabet(seq)
+    lengths = huffman_lengths(counts)
+    codes = canonical_codes(lengths)
+    words, bits = _pack(sym, codes, lengths)
+    return dict(kind="hac", n=n, m=m, codebook=codebook, counts=counts, code_len=lengths,
+                codes=codes, sym=sym, words=words, bits=bits)
+
+
+def shac_encode(Wq: np.ndarray, mask: np.ndarray) -> dict:
+    """sHAC (Sect. IV-C): the CSC vectors of W with nz Huffman coded (code built
+    on the stored values only, no code word for the null entries) and ri, cb
+    kept as they are."""
+    n, m = Wq.shape
+    nz, ri, cb = csc(Wq, mask)
+    if nz.size:
+        codebook, sym, counts = _alphabet(nz)
+        lengths = huffman_lengths(counts)
+        codes = canonical_codes(lengths)
+        words, bits = _pack(sym, codes, lengths)
+    else:
+        codebook = np.zeros(0, np.float32); sym = np.zeros(0, np.int32)
+        counts = np.zeros(0, np.int64); lengths = np.zeros(0, np.uint8)
+        codes = np.zeros(0, np.uint32); words = np.zeros(0, np.uint32); bits = 0
+    return dict(kind="shac", n=n, m=m, codebook=codebook, counts=counts, code_len=lengths,
+                codes=codes, sym=sym, words=words, bits=bits, nz=nz, ri=ri, cb=cb)
+
+
+def decode_symbols(fmt: dict, bit0: int, count: int) -> tuple:
+    """Read `count` symbols starting at bit `bit0` of the stream (tree walk)."""
+    out = np.empty(max(count, 1), dtype=np.int32)
+    words = np.ascontiguousarray(fmt["words"], dtype=np.uint32)
+    end = _native().orc_decode(_p(words), ctypes.c_int64(words.size), ctypes.c_int64(bit0),
+                               _p(np.ascontiguousarray(fmt["codes"])),
+                               _p(np.ascontiguousarray(fmt["code_len"])),
+                               ctypes.c_int32(len(fmt["codebook"])), ctypes.c_int64(count), _p(out))
+    if end < 0:
+        raise RuntimeError(f"orc_decode failed: {end}")
+    return out[:count], int(end)
+
+
+def hac_decode(fmt: dict) -> np.ndarray:
+    """Rebuild the quantized matrix from a HAC stream (the format is lossless)."""
+    sym, _ = decode_symbols(fmt, 0, fmt["n"] * fmt["m"])
+    return fmt["codebook"][sym].reshape(fmt["m"], fmt["n"]).T.copy()
+
+
+def shac_decode(fmt: dict) -> np.ndarray:
+    sym, _ = decode_symbols(fmt, 0, int(fmt["cb"][-1]))
+    W = np.zeros((fmt["n"], fmt["m"]), dtype=np.float32)
+    cols = np.repeat(np.arange(fmt["m"]), np.diff(fmt["cb"]))
+    W[fmt["ri"], cols] = fmt["codebook"][sym]
+    return W
+
+
+# ----------------------------------------------------------------------------
+# Offset index (the column-offset vector the paper's conclusions propose for a
+# finer parallelism, refined to sub-segments of S symbols)
+# ----------------------------------------------------------------------------
+def hac_offset_index(fmt: dict, S: int) -> dict:
+    """Every column is cut into sub-segments of S symbols (the last shorter);
+    32 consecutive sub-segments of a column form a segment.  seg_bit_off[u] is
+    the bit at which segment u = j*G + g starts, sub_bits[u*32 + l] the bit
+    length of its l-th sub-segment (0 where the column has ended)."""
+    n, m = fmt["n"], fmt["m"]
+    T = -(-n // S)
+    G = -(-T // 32)
+    lens = fmt["code_len"].astype(np.int64)[fmt["sym"]].reshape(m, n)
+    padded = np.zeros((m, G * 32 * S), dtype=np.int64)
+    padded[:, :n] = lens
+    sub_bits = padded.reshape(m, G * 32, S).sum(axis=2)
+    seg_bits = sub_bits.reshape(m * G, 32).sum(axis=1)
+    seg_bit_off = np.concatenate(([0], np.cumsum(seg_bits)[:-1])).astype(np.uint64)
+    return dict(S=S, T=T, G=G, seg_bit_off=seg_bit_off,
+                sub_bits=sub_bits.reshape(-1).astype(np.uint16))
+
+
+def shac_offset_index(fmt: dict, S: int) -> dict:
+    """As for HAC, over each column's run of stored entries: column j with q_j
+    entries has ceil(q_j / S) sub-segments and ceil(that / 32) segments.
+    seg_first[j] = number of segments in columns before j, seg_col[u] = column
+    of segment u."""
+    m = fmt["m"]
+    cb = fmt["cb"]
+    lens = fmt["code_len"].astype(np.int64)[fmt["sym"]] if fmt["sym"].size else np.zeros(0, np.int64)
+    seg_first = np.zeros(m + 1, dtype=np.uint32)
+    seg_col, seg_bits_all, sub_all = [], [], []
+    for j in range(m):
+        l = lens[cb[j]:cb[j + 1]]
+        T = -(-len(l) // S)
+        G = -(-T // 32)
+        seg_first[j + 1] = seg_first[j] + G
+        if G == 0:
+            continue
+        padded = np.zeros(G * 32 * S, dtype=np.int64)
+        padded[:len(l)] = l
+        sb = padded.reshape(G * 32, S).sum(axis=1)
+        sub_all.append(sb)
+        seg_bits_all.append(sb.reshape(G, 32).sum(axis=1))
+        seg_col.extend([j] * G)
+    if seg_col:
+        seg_bits = np.concatenate(seg_bits_all)
+        seg_bit_off = np.concatenate(([0], np.cumsum(seg_bits)[:-1])).astype(np.uint64)
+        sub_bits = np.concatenate(sub_all).astype(np.uint16)
+    else:
+        seg_bit_off = np.zeros(0, np.uint64); sub_bits = np.zeros(0, np.uint16)
+    return dict(S=S, seg_first=seg_first, seg_col=np.asarray(seg_col, dtype=np.uint32),
+                seg_bit_off=seg_bit_off, sub_bits=sub_bits)
+
+
+# ----------------------------------------------------------------------------
+# Space bounds (Corollaries 1 and 2) with the paper's accounting
+# ----------------------------------------------------------------------------
+def hac_paper_bits(fmt: dict) -> int:
+    """|HAC(W)| as the paper counts it: stream words plus 6*k*b bits for the two
+    dictionaries held as B-trees (proof of Theorem 1)."""
+    return len(fmt["words"]) * B_WORD + 6 * len(fmt["codebook"]) * B_WORD
+
+
+def cor1_bound_bits(n: int, m: int, k: int) -> float:
+    """Corollary 1: |HAC(W)| <= nm (1 + log k) + 6 k b."""
+    return n * m * (1.0 + np.log2(k)) + 6 * k * B_WORD
+
+
+def shac_paper_bits(fmt: dict) -> int:
+    """|sHAC(W)|: stream words, dictionaries, and ri, cb at b bits per entry."""
+    q = int(fmt["cb"][-1])
+    return (len(fmt["words"]) * B_WORD + 6 * len(fmt["codebook"]) * B_WORD
+            + B_WORD * (q + fmt["m"] + 1))
+
+
+def cor2_bound_bits(n: int, m: int, q: int, k: int) -> float:
+    """Corollary 2 with s*n*m = q stored entries:
+    |sHAC(W)| <= q (1 + log k) + b (6k + q + m + 1)."""
+    return q * (1.0 + np.log2(max(k, 1))) + B_WORD * (6 * k + q + m + 1)
+
+
+def shac_smaller_than_hac_threshold(n: int, m: int, k: int) -> float:
+    """Non-zero ratio s below which the sHAC bound is under the HAC bound
+    (the inequality after Algorithm 2)."""
+    a = (1.0 + np.log2(k)) / B_WORD
+    return (a - (m + 1) / (n * m)) / (1.0 + a)
+
+
+# ----------------------------------------------------------------------------
+# Sect. IV-B / IV-C / IV-D  the dot procedures
+# ----------------------------------------------------------------------------
+def _c32(a):
+    return np.ascontiguousarray(a, dtype=np.float32)
+
+
+def dot_hac(fmt: dict, x: np.ndarray) -> np.ndarray:
+    """Algorithm 1 (Dot_HAC): sequential scan of the words, NCW pulling one code
+    word at a time.  x has n entries; the result has m (one per column)."""
+    out = np.zeros(fmt["m"], dtype=np.float64)
+    words = np.ascontiguousarray(fmt["words"], dtype=np.uint32)
+    rc = _native().orc_dot_hac(_p(words), ctypes.c_int64(words.size),
+                               _p(np.ascontiguousarray(fmt["codes"])), _p(np.ascontiguousarray(fmt["code_len"])),
+                               _p(_c32(fmt["codebook"])), ctypes.c_int32(len(fmt["codebook"])),
+                               _p(_c32(x)), ctypes.c_int64(fmt["n"]), ctypes.c_int64(fmt["m"]), _p(out))
+    if rc:
+        raise RuntimeError(f"orc_dot_hac failed: {rc}")
+    return out
+
+
+def dot_shac(fmt: dict, x: np.ndarray) -> np.ndarray:
+    """Algorithm 2 (Dot_sHAC)."""
+    out = np.zeros(fmt["m"], dtype=np.float64)
+    if fmt["cb"][-1] == 0:
+        return out
+    words = np.ascontiguousarray(fmt["words"], dtype=np.uint32)
+    rc = _native().orc_dot_shac(_p(words), ctypes.c_int64(words.size),
+                                _p(np.ascontiguousarray(fmt["codes"])), _p(np.ascontiguousarray(fmt["code_len"])),
+                                _p(_c32(fmt["codebook"])), ctypes.c_int32(len(fmt["codebook"])),
+                                _p(np.ascontiguousarray(fmt["ri"], dtype=np.int32)),
+                                _p(np.ascontiguousarray(fmt["cb"], dtype=np.int64)),
+                                _p(_c32(x)), ctypes.c_int64(fmt["m"]), _p(out))
+    if rc:
+        raise RuntimeError(f"orc_dot_shac failed: {rc}")
+    return out
+
+
+def pardot(fmt: dict, X: np.ndarray, q: int) -> np.ndarray:
+    """Algorithm 3 (ParDot): X is B x n, one input per row; its rows are split
+    into q chunks, each handled by one thread running Algorithm 1 or 2 once per
+    row.  Returns B x m."""
+    X = _c32(X)
+    B = X.shape[0]
+    out = np.zeros((B, fmt["m"]), dtype=np.float64)
+    words = np.ascontiguousarray(fmt["words"], dtype=np.uint32)
+    common = (_p(words), ctypes.c_int64(words.size), _p(np.ascontiguousarray(fmt["codes"])),
+              _p(np.ascontiguousarray(fmt["code_len"])), _p(_c32(fmt["codebook"])),
+              ctypes.c_int32(len(fmt["codebook"])))
+    tail = (_p(X), ctypes.c_int64(B), ctypes.c_int64(fmt["n"]), ctypes.c_int64(fmt["m"]),
+            ctypes.c_int32(q), _p(out))
+    if fmt["kind"] == "hac":
+        rc = _native().orc_pardot_hac(*common, *tail)
+    else:
+        if fmt["cb"][-1] == 0:
+            return out
+        rc = _native().orc_pardot_shac(*common, _p(np.ascontiguousarray(fmt["ri"], dtype=np.int32)),
+                                       _p(np.ascontiguousarray(fmt["cb"], dtype=np.int64)), *tail)
+    if rc:
+        raise RuntimeError(f"pardot failed: {rc}")
+    return out
+
+
+def dot_definition(Wq: np.ndarray, X: np.ndarray, cols=None):
+    """What the dot procedures output, written out: y[b, j] = sum_i Wq[i, j] X[b, i]
+    in fp64 with i ascending, and a[b, j] = sum_i |Wq[i, j] X[b, i]|, the scale of the
+    output tolerance.  With `cols`, only those columns (full-size spot checks)."""
+    Wq = _c32(Wq)
+    X = _c32(np.atleast_2d(X))
+    n, m = Wq.shape
+    B = X.shape[0]
+    if cols is None:
+        y = np.zeros((B, m)); a = np.zeros((B, m))
+        _native().orc_dot_definition(_p(Wq), ctypes.c_int64(n), ctypes.c_int64(m), _p(X),
+                                     ctypes.c_int64(B), _p(y), _p(a))
+    else:
+        cols = np.ascontiguousarray(cols, dtype=np.int64)
+        y = np.zeros((B, cols.size)); a = np.zeros((B, cols.size))
+        rc = _native().orc_dot_definition_cols(_p(Wq), ctypes.c_int64(n), ctypes.c_int64(m), _p(X),
+                                               ctypes.c_int64(B), _p(cols), ctypes.c_int64(cols.size),
+                                               _p(y), _p(a))
+        if rc:
+            raise RuntimeError("bad column index")
+    return y, a

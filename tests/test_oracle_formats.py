@@ -1,0 +1,185 @@
+"""Pins of the oracle's format code: the examples the paper prints (Sect. IV-A Example 2,
+Sect. IV-B address map), a stream worked out by hand from them, and the properties the
+paper states for the formats (lossless, N = ceil(bits / b) words, Corollaries 1 and 2)."""
+import numpy as np
+import pytest
+
+from oracle import hac_oracle as orc
+from golden_io import golden, read_sections
+
+
+def example2():
+    g = read_sections(golden("example2_csc.txt"))
+    W = np.array(g["W"], dtype=np.float32)
+    nz = np.array(g["nz"][0], dtype=np.float32)
+    ri = np.array(g["ri"][0], dtype=np.int64)
+    cb = np.array(g["cb"][0], dtype=np.int64)
+    return W, nz, ri, cb
+
+
+def test_csc_matches_paper_example2():
+    W, nz, ri, cb = example2()
+    got_nz, got_ri, got_cb = orc.csc(W, W != 0)
+    assert np.array_equal(got_nz, nz)
+    assert np.array_equal(got_ri + 1, ri)          # the paper counts from 1
+    assert np.array_equal(got_cb + 1, cb)
+
+
+def test_hac_symbol_order_matches_paper_address_map():
+    W, *_ = example2()
+    tokens = read_sections(golden("example_address_map.txt"))[None][0]
+    assert len(tokens) == 25
+    fmt = orc.hac_encode(W)
+    values = fmt["codebook"][fmt["sym"]]
+    for tok, v in zip(tokens, values):
+        want = 0.0 if tok == "0" else float(tok[2:-1])
+        assert v == want
+    # one code word per entry, zeros included: "q + 1 code words" for q distinct non-null values
+    assert len(fmt["codebook"]) == len(np.unique(W[W != 0])) + 1
+
+
+def test_hand_coded_example_hac():
+    W, *_ = example2()
+    g = read_sections(golden("example2_hand_coded.txt"))
+    fmt = orc.hac_encode(W)
+    assert np.array_equal(fmt["codebook"], np.array(g["hac_values"][0], dtype=np.float32))
+    assert fmt["code_len"].tolist() == [int(t) for t in g["hac_lengths"][0]]
+    assert [format(int(c), f"0{l}b") for c, l in zip(fmt["codes"], fmt["code_len"])] == g["hac_codes"][0]
+    assert fmt["bits"] == int(g["hac_bits"][0][0])
+    assert [f"{int(w):08X}" for w in fmt["words"]] == g["hac_words"][0]
+    # one sub-segment per column (S = n): segment offsets are the column offsets
+    idx = orc.hac_offset_index(fmt, S=5)
+    want = [int(t) for t in g["hac_column_bit_offsets"][0]]
+    assert idx["seg_bit_off"].tolist() == want[:-1]
+    assert int(idx["seg_bit_off"][-1]) + int(idx["sub_bits"].reshape(-1, 32)[-1].sum()) == want[-1]
+
+
+def test_hand_coded_example_shac_and_dot():
+    W, *_ = example2()
+    g = read_sections(golden("example2_hand_coded.txt"))
+    fmt = orc.shac_encode(W, W != 0)
+    assert np.array_equal(fmt["codebook"], np.array(g["shac_values"][0], dtype=np.float32))
+    assert fmt["code_len"].tolist() == [int(t) for t in g["shac_lengths"][0]]
+    assert [format(int(c), f"0{l}b") for c, l in zip(fmt["codes"], fmt["code_len"])] == g["shac_codes"][0]
+    assert fmt["bits"] == int(g["shac_bits"][0][0])
+    assert [f"{int(w):08X}" for w in fmt["words"]] == g["shac_words"][0]
+    x = np.array(g["x"][0], dtype=np.float32)
+    want = np.array(g["xTW"][0], dtype=np.float64)
+    assert np.array_equal(orc.dot_shac(fmt, x), want)
+    assert np.array_equal(orc.dot_hac(orc.hac_encode(W), x), want)
+    assert np.array_equal(orc.dot_definition(W, x)[0][0], want)
+
+
+def _random_quantized(rng, n, m, k, zero_frac):
+    values = np.sort(rng.standard_normal(k).astype(np.float32))
+    p = rng.dirichlet(np.ones(k) * 0.5)
+    W = values[rng.choice(k, size=(n, m), p=p)]
+    W[rng.random((n, m)) < zero_frac] = 0.0
+    return W.astype(np.float32)
+
+
+@pytest.mark.parametrize("n,m,k,zf", [(7, 5, 3, 0.5), (64, 33, 17, 0.0), (130, 70, 40, 0.9), (33, 9, 1, 0.0)])
+def test_round_trip_is_lossless(n, m, k, zf):
+    rng = np.random.default_rng(n * 1000 + m)
+    W = _random_quantized(rng, n, m, k, zf)
+    fh = orc.hac_encode(W)
+    assert np.array_equal(orc.hac_decode(fh).view(np.uint32), W.view(np.uint32))
+    fs = orc.shac_encode(W, W != 0)
+    assert np.array_equal(orc.shac_decode(fs).view(np.uint32), W.view(np.uint32))
+
+
+@pytest.mark.parametrize("n,m,k,zf", [(50, 20, 9, 0.3), (64, 64, 32, 0.8)])
+def test_stream_length_and_padding(n, m, k, zf):
+    rng = np.random.default_rng(5)
+    W = _random_quantized(rng, n, m, k, zf)
+    for fmt in (orc.hac_encode(W), orc.shac_encode(W, W != 0)):
+        bits = int((fmt["counts"] * fmt["code_len"].astype(np.int64)).sum())
+        assert fmt["bits"] == bits
+        assert len(fmt["words"]) == -(-bits // 32)                       # N = ceil(|HAC| / b)
+        pad = len(fmt["words"]) * 32 - bits
+        if pad:
+            assert int(fmt["words"][-1]) & ((1 << pad) - 1) == 0         # zero padding
+
+
+def test_offset_index_segments_decode_alone():
+    rng = np.random.default_rng(11)
+    W = _random_quantized(rng, 300, 7, 12, 0.4)
+    fmt = orc.hac_encode(W)
+    S = 4
+    idx = orc.hac_offset_index(fmt, S)
+    n, m, G = fmt["n"], fmt["m"], idx["G"]
+    assert idx["T"] == 75 and G == 3
+    sym = fmt["sym"].reshape(m, n)
+    for j in range(m):
+        for g in range(G):
+            u = j * G + g
+            bit = int(idx["seg_bit_off"][u])
+            for l in range(32):
+                r0 = (g * 32 + l) * S
+                cnt = max(0, min(S, n - r0))
+                got, end = orc.decode_symbols(fmt, bit, cnt)
+                assert np.array_equal(got, sym[j, r0:r0 + cnt])
+                assert end - bit == int(idx["sub_bits"][u * 32 + l])
+                bit = end
+    last = len(idx["seg_bit_off"]) - 1
+    assert int(idx["seg_bit_off"][last]) + int(idx["sub_bits"][last * 32:].sum()) == fmt["bits"]
+
+
+def test_shac_offset_index_segments_decode_alone():
+    rng = np.random.default_rng(12)
+    W = _random_quantized(rng, 500, 9, 10, 0.6)
+    W[:, 3] = 0.0                                       # an empty column
+    fmt = orc.shac_encode(W, W != 0)
+    S = 3
+    idx = orc.shac_offset_index(fmt, S)
+    cb = fmt["cb"]
+    assert idx["seg_first"][3] == idx["seg_first"][4]
+    for j in range(fmt["m"]):
+        for u in range(int(idx["seg_first"][j]), int(idx["seg_first"][j + 1])):
+            assert idx["seg_col"][u] == j
+            g = u - int(idx["seg_first"][j])
+            bit = int(idx["seg_bit_off"][u])
+            for l in range(32):
+                p0 = int(cb[j]) + (g * 32 + l) * S
+                cnt = max(0, min(S, int(cb[j + 1]) - p0))
+                got, end = orc.decode_symbols(fmt, bit, cnt)
+                assert np.array_equal(got, fmt["sym"][p0:p0 + cnt])
+                assert end - bit == int(idx["sub_bits"][u * 32 + l])
+                bit = end
+    assert len(idx["seg_col"]) == int(idx["seg_first"][-1])
+
+
+@pytest.mark.parametrize("k", [2, 8, 32])
+@pytest.mark.parametrize("zf", [0.0, 0.5, 0.9, 0.99])
+def test_sizes_within_corollaries(k, zf):
+    rng = np.random.default_rng(k * 100 + int(zf * 100))
+    n, m = 256, 96
+    W = _random_quantized(rng, n, m, k, zf)
+    fh = orc.hac_encode(W)
+    kk = len(fh["codebook"])
+    assert orc.hac_paper_bits(fh) <= orc.cor1_bound_bits(n, m, kk) + 31      # + word padding
+    fs = orc.shac_encode(W, W != 0)
+    q = int(fs["cb"][-1])
+    assert orc.shac_paper_bits(fs) <= orc.cor2_bound_bits(n, m, q, len(fs["codebook"])) + 31
+    # occupancy bounds, Eq. (1) and Eq. (2), are the corollaries divided by b*n*m
+    psi_hac = orc.hac_paper_bits(fh) / (32.0 * n * m)
+    assert psi_hac <= (1 + np.log2(kk)) / 32 + 6 * kk / (n * m) + 31 / (32.0 * n * m)
+
+
+def test_two_values_dense_is_one_bit_per_weight():
+    # Table III of the paper: k = 2 on a dense matrix gives psi = 0.0313 = 1/32
+    rng = np.random.default_rng(3)
+    W = np.where(rng.random((128, 64)) < 0.3, np.float32(-0.5), np.float32(0.25)).astype(np.float32)
+    fmt = orc.hac_encode(W)
+    assert fmt["bits"] == W.size
+    assert abs(fmt["bits"] / (32.0 * W.size)- 0.0313) <= 5.001e-5      # the printed value is 1/32 rounded
+
+
+def test_crossover_formula_consistent_with_bounds():
+    n, m, k = 4096, 4096, 32
+    s_star = orc.shac_smaller_than_hac_threshold(n, m, k)
+    for s in (s_star * 0.98, s_star * 1.02):
+        q = int(s * n * m)
+        shac_b = orc.cor2_bound_bits(n, m, q, k) - 6 * k * 32
+        hac_b = orc.cor1_bound_bits(n, m, k) - 6 * k * 32
+        assert (shac_b < hac_b) == (s < s_star)
