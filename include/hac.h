@@ -1,0 +1,236 @@
+/*
+ * hac.h - C ABI of the HAC / sHAC compressed-domain product library for NVIDIA B200 (sm_100a).
+ *
+ * The formats and the product are those of Marino, Petrini, Malchiodi, Frasca, "Compact
+ * representations of convolutional neural networks via weight pruning and quantization":
+ *   HAC  (Sect. IV-B): the matrix as a column-order address map whose entries, zeros included,
+ *        are replaced by Huffman code words; the bit string is stored in 32-bit words.
+ *   sHAC (Sect. IV-C): the CSC vectors nz, ri, cb of the matrix with nz Huffman coded.
+ *   Dot  (Algorithms 1-3): x^T W computed on the compressed representation, one output per
+ *        column of W, for one input vector or a batch of them.
+ *
+ * Conventions
+ *   - Every call returns an int status: HAC_OK (0) or a negative HAC_ERR_* code; nothing throws.
+ *     hac_status_string() gives the text.  On error, outputs are left untouched unless stated.
+ *   - "host" pointers are ordinary CPU memory, "device" pointers are CUDA global memory of the
+ *     current device.  The library never allocates device memory: the caller provides the buffer a
+ *     format is uploaded to, the inputs, the outputs and the workspace.  `cuda_stream` is a
+ *     cudaStream_t passed as void* (NULL = the legacy default stream); device work is enqueued on
+ *     it and the call returns without waiting, unless stated.
+ *   - Handles are opaque, created by *_build, owned by the caller, released by *_free.  A handle
+ *     may be used from one thread at a time.
+ *   - Indices are 0-based (the paper counts from 1).  W is n x m: n inputs (rows), m outputs
+ *     (columns).  b = 32 bits per memory word.
+ */
+#ifndef HAC_H_
+#define HAC_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define HAC_OK                    0
+#define HAC_ERR_INVALID_ARG      -1   /* null pointer, bad size, bad parameter                    */
+#define HAC_ERR_ALLOC            -2   /* host allocation failed                                   */
+#define HAC_ERR_NONFINITE_INPUT  -3   /* W holds NaN or Inf                                       */
+#define HAC_ERR_K_TOO_LARGE      -4   /* more than HAC_MAX_SYMBOLS distinct values after sharing  */
+#define HAC_ERR_CODE_TOO_LONG    -5   /* a Huffman code word longer than 32 bits                  */
+#define HAC_ERR_OFFSET_OVERFLOW  -6   /* a size or offset does not fit its field                  */
+#define HAC_ERR_NOT_UPLOADED     -7   /* device call on a format that was not uploaded            */
+#define HAC_ERR_BUFFER_TOO_SMALL -8   /* caller's buffer or workspace too small                   */
+#define HAC_ERR_CUDA             -9   /* a CUDA runtime call failed                               */
+#define HAC_ERR_CORRUPT          -10  /* serialized data fails validation                         */
+
+#define HAC_MAX_SYMBOLS        2048   /* largest alphabet (distinct values, zero included)        */
+#define HAC_MAX_SEG_SYMBOLS    1024   /* largest sub-segment length of the offset index           */
+
+#define HAC_QUANT_NONE     0u   /* W already holds few distinct values                            */
+#define HAC_QUANT_KMEANS   1u   /* CWS, Sect. III-C.1                                             */
+#define HAC_QUANT_UNIFORM  2u   /* UQ,  Sect. III-C.3, grid over [min, max] of the non-null weights */
+
+typedef struct hac_format  hac_format;    /* HAC : stream, codebook, code lengths, offset index          */
+typedef struct shac_format shac_format;   /* sHAC: stream of nz, ri, cb, codebook, lengths, offset index */
+
+/* Build parameters (Sect. III-B, III-C).  Zero-initialise, then set what is needed. */
+typedef struct hac_build_params {
+    double   sparsity;      /* target fraction of zeros in [0,1); 0 = no pruning (Sect. III-B)          */
+    uint32_t k;             /* number of shared values for the non-null weights (Sect. III-C)           */
+    uint32_t quantizer;     /* HAC_QUANT_*                                                              */
+    uint32_t kmeans_iters;  /* Lloyd iterations, run in full (no early stop)                            */
+    uint32_t seg_symbols;   /* S: symbols per sub-segment of the offset index, 1..HAC_MAX_SEG_SYMBOLS;
+                               0 = default (64 for HAC, 32 for sHAC)                                    */
+    uint64_t seed;          /* seed of the k-means initialisation                                       */
+    uint32_t ri_bits;       /* sHAC: width of a stored row index, 16 or 32; 0 = 16 if n <= 65536 else 32
+                               (the footnote of Sect. IV-A: ri needs only ceil(log n) bits)             */
+    uint32_t reserved;      /* must be 0                                                                */
+} hac_build_params;
+
+/* Sizes of a built format.  "paper_bits" follows the paper's accounting (stream words, 6*k*b bits
+ * for the two dictionaries kept as B-trees, and for sHAC ri and cb at b bits per entry); the
+ * *_bytes fields are what this library really stores.  bound_bits is Corollary 1 (HAC) or
+ * Corollary 2 (sHAC) evaluated at the format's own k and number of stored entries. */
+typedef struct hac_size_report {
+    int64_t n, m;               /* shape of W                                                     */
+    int64_t nnz;                /* entries that survived pruning (stored entries of sHAC)         */
+    int64_t symbols;            /* code words in the stream: n*m (HAC) or nnz (sHAC)              */
+    int64_t stream_bits;        /* |HAC(W)| or |HAC(nz)|: sum of code word lengths                */
+    int64_t stream_words;       /* N = ceil(stream_bits / 32)                                     */
+    int64_t stream_bytes;       /* 4 * N                                                          */
+    int64_t pad_bytes;          /* zero words appended after word N (alignment + over-read slack)  */
+    int64_t codebook_bytes;     /* 4 * k_eff                                                      */
+    int64_t code_len_bytes;     /* k_eff                                                          */
+    int64_t ri_bytes;           /* sHAC: nnz * ri_bits / 8                                        */
+    int64_t cb_bytes;           /* sHAC: 4 * (m + 1)                                              */
+    int64_t offset_index_bytes; /* all arrays of the offset index                                 */
+    int64_t total_bytes;        /* sum of the *_bytes fields above                                */
+    int64_t paper_bits;         /* size by the paper's accounting                                 */
+    double  bound_bits;         /* Corollary 1 / Corollary 2                                      */
+    double  entropy;            /* source entropy H, bits per symbol                              */
+    double  avg_code_len;       /* stream_bits / symbols                                          */
+    uint32_t k_eff;             /* alphabet size                                                  */
+    uint32_t max_code_len;
+    uint32_t min_code_len;
+    uint32_t seg_symbols;       /* S                                                              */
+    uint32_t ri_bits;
+    uint32_t units;             /* segments (warp work units) in the offset index                 */
+} hac_size_report;
+
+/* Borrowed host pointers to every array of a format; valid until the handle is freed.
+ * Symbol id = rank of the value in `codebook` (ascending).  `stream` has stream_words data
+ * words followed by stream_pad_words zero words.  Offset index: see hac_build. */
+typedef struct hac_host_view {
+    int64_t n, m;
+    uint32_t k_eff, seg_symbols;
+    const float*    codebook;      /* [k_eff] shared values, ascending                            */
+    const uint8_t*  code_len;      /* [k_eff] code word length of each symbol                     */
+    const uint32_t* codes;         /* [k_eff] canonical code word of each symbol (right aligned)  */
+    const int64_t*  counts;        /* [k_eff] occurrences of each symbol                          */
+    const uint32_t* stream;        /* [stream_words + stream_pad_words]                           */
+    int64_t stream_bits, stream_words, stream_pad_words;
+    uint32_t units;                /* U                                                           */
+    uint32_t segs_per_col;         /* HAC: G; sHAC: 0                                             */
+    const uint64_t* seg_bit_off;   /* [U]                                                         */
+    const uint16_t* sub_bits;      /* [U * 32]                                                    */
+} hac_host_view;
+
+typedef struct shac_host_view {
+    hac_host_view   base;          /* stream etc. of nz                                           */
+    int64_t nnz;
+    uint32_t ri_bits;
+    const void*     ri;            /* [nnz] uint16_t or uint32_t row indices                      */
+    const uint32_t* cb;            /* [m + 1] cb[j] = stored entries in columns before j          */
+    const uint32_t* seg_first;     /* [m + 1] segments in columns before j                        */
+    const uint32_t* seg_col;       /* [U] column of each segment                                  */
+} shac_host_view;
+
+/* ---------------------------------------------------------------------------------------------
+ * hac_build / shac_build - Sect. III-B (pruning), III-C.1 / III-C.3 (weight sharing), IV-B / IV-C
+ * (formats).  Host only, synchronous.
+ *   W      host, row-major n x m fp32 with leading dimension ldw >= m (elements); borrowed for the
+ *          duration of the call.  NaN / Inf -> HAC_ERR_NONFINITE_INPUT.  -0.0 counts as 0.
+ *   params see hac_build_params.
+ *   out    receives the new handle.
+ * Steps: entries with |w| <= the floor(sparsity*n*m)-th smallest magnitude become 0; the others are
+ * replaced by one of k shared values (k-means over them in column-major order, or a uniform grid
+ * over their range); distinct values sorted ascending form the codebook; a Huffman code over the
+ * symbol counts (HAC: every entry, zeros included; sHAC: stored entries only) is made canonical;
+ * code words are concatenated column by column, most significant bit first, into 32-bit words.
+ * Offset index (the column-offset vector suggested in the paper's conclusions, refined): each column
+ * (HAC: its n entries; sHAC: its stored entries) is cut into sub-segments of S symbols, 32
+ * consecutive sub-segments form a segment; seg_bit_off[u] is the bit where segment u starts and
+ * sub_bits[u*32 + l] the bit length of its l-th sub-segment.  HAC numbers segments u = j*G + g with
+ * G = ceil(ceil(n/S)/32); sHAC numbers them column after column and adds seg_first, seg_col.
+ * ------------------------------------------------------------------------------------------- */
+int hac_build (const float* W, int64_t n, int64_t m, int64_t ldw, const hac_build_params* params,
+               hac_format** out);
+int shac_build(const float* W, int64_t n, int64_t m, int64_t ldw, const hac_build_params* params,
+               shac_format** out);
+
+/* Sizes (Corollaries 1 and 2 for bound_bits) and borrowed views of the built arrays. Host only. */
+int hac_sizes  (const hac_format*  f, hac_size_report* out);
+int shac_sizes (const shac_format* f, hac_size_report* out);
+int hac_export (const hac_format*  f, hac_host_view*  out);
+int shac_export(const shac_format* f, shac_host_view* out);
+
+/* The pruned and quantized matrix the format encodes, written to a host buffer Wq (row-major n x m,
+ * leading dimension ldq >= m), reconstructed on the host from the stream (lossless, Sect. IV-B). */
+int hac_decode_host (const hac_format*  f, float* Wq, int64_t ldq);
+int shac_decode_host(const shac_format* f, float* Wq, int64_t ldq);
+
+/* ---------------------------------------------------------------------------------------------
+ * Upload.  *_device_bytes gives the size of the device image of a format (all arrays the kernels
+ * read, plus decoding tables derived from the code lengths).  *_upload copies that image into the
+ * caller's device buffer `dev_buf` (256-byte aligned, at least *_device_bytes long) on `cuda_stream`
+ * and records the pointers in the handle.  The buffer stays owned by the caller and must outlive
+ * every dot call on the handle.  Uploading again (e.g. to another buffer) re-targets the handle.
+ * ------------------------------------------------------------------------------------------- */
+int hac_device_bytes (const hac_format*  f, size_t* out);
+int shac_device_bytes(const shac_format* f, size_t* out);
+int hac_upload (hac_format*  f, void* dev_buf, size_t dev_bytes, void* cuda_stream);
+int shac_upload(shac_format* f, void* dev_buf, size_t dev_bytes, void* cuda_stream);
+/* Point the handle at a device image that *_upload wrote earlier and that was then copied, byte
+ * for byte, to `dev_buf` (same device).  No copy is made. */
+int hac_attach (hac_format*  f, void* dev_buf, size_t dev_bytes);
+int shac_attach(shac_format* f, void* dev_buf, size_t dev_bytes);
+
+/* ---------------------------------------------------------------------------------------------
+ * hac_dot / shac_dot - Algorithms 1, 2 (one input) and 3 (a batch), on the device:
+ *       y[b*y_stride_b + j*y_stride_j] = sum_i W[i][j] * x[b*x_stride_b + i*x_stride_i]
+ * for b in [0, batch), j in [0, m).  x, y: device fp32; strides in elements, so X may be stored
+ * [batch][n] or [n][batch] and Y [batch][m] or [m][batch]; the batched kernels are fastest with
+ * x_stride_b == 1 and y_stride_b == 1.  x and y must not overlap.  Code words are decoded on the
+ * fly; the uncompressed weights are never written to global memory.  Products and sums are fp32.
+ *   workspace  device scratch of at least *_workspace_bytes(f, batch) bytes (may be NULL when that
+ *              is 0).  It holds partial sums of columns that span several segments; its contents
+ *              need not be initialised and are undefined afterwards.  Two dot calls that run
+ *              concurrently must not share it.
+ * Asynchronous on cuda_stream.  Errors: HAC_ERR_NOT_UPLOADED, HAC_ERR_INVALID_ARG (batch < 1, null
+ * pointers), HAC_ERR_BUFFER_TOO_SMALL, HAC_ERR_CUDA (launch failure).
+ * ------------------------------------------------------------------------------------------- */
+int hac_workspace_bytes (const hac_format*  f, int64_t batch, size_t* out);
+int shac_workspace_bytes(const shac_format* f, int64_t batch, size_t* out);
+int hac_dot (const hac_format* f, const float* x, int64_t batch, int64_t x_stride_i, int64_t x_stride_b,
+             float* y, int64_t y_stride_j, int64_t y_stride_b,
+             void* workspace, size_t workspace_bytes, void* cuda_stream);
+int shac_dot(const shac_format* f, const float* x, int64_t batch, int64_t x_stride_i, int64_t x_stride_b,
+             float* y, int64_t y_stride_j, int64_t y_stride_b,
+             void* workspace, size_t workspace_bytes, void* cuda_stream);
+
+/* The same product for HOST inputs and outputs (Algorithm 3's calling convention: X is batch x n,
+ * one input per row, Y is batch x m, both contiguous host fp32, ideally pinned).  The caller gives a
+ * device staging buffer `dev_scratch` of at least *_dot_host_scratch_bytes(f, batch) bytes; the call
+ * copies X to the device, runs the product, copies Y back and waits for cuda_stream. */
+int hac_dot_host_scratch_bytes (const hac_format*  f, int64_t batch, size_t* out);
+int shac_dot_host_scratch_bytes(const shac_format* f, int64_t batch, size_t* out);
+int hac_dot_host (const hac_format*  f, const float* X_host, int64_t batch, float* Y_host,
+                  void* dev_scratch, size_t dev_scratch_bytes, void* cuda_stream);
+int shac_dot_host(const shac_format* f, const float* X_host, int64_t batch, float* Y_host,
+                  void* dev_scratch, size_t dev_scratch_bytes, void* cuda_stream);
+
+/* ---------------------------------------------------------------------------------------------
+ * TEST ONLY: decode on the device into a caller's device buffer, to show that the kernels' decoder
+ * reproduces the quantized weights bit for bit (the formats are lossless, Sect. IV-B).  The product
+ * path never does this.  hac: W_colmajor[j*n + i] = Wq[i][j] (n*m floats).  shac: nz[p] for the nnz
+ * stored entries in CSC order.  Asynchronous on cuda_stream.
+ * ------------------------------------------------------------------------------------------- */
+int hac_debug_decode (const hac_format*  f, float* W_colmajor_dev, void* cuda_stream);
+int shac_debug_decode(const shac_format* f, float* nz_dev, void* cuda_stream);
+
+/* Number of kernels the last dot / debug call on this handle launched (for launch accounting). */
+int hac_last_launch_count (const hac_format*  f);
+int shac_last_launch_count(const shac_format* f);
+
+void hac_free (hac_format*  f);
+void shac_free(shac_format* f);
+
+const char* hac_status_string(int status);
+/* Text of the last CUDA error seen by this library on the calling thread ("" if none). */
+const char* hac_last_cuda_error(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif  /* HAC_H_ */

@@ -1,0 +1,619 @@
+// Host-side format builder: pruning (Sect. III-B), weight sharing (Sect. III-C.1, III-C.3),
+// Huffman code and the HAC / sHAC layouts (Sect. IV-B, IV-C), plus the offset index and the
+// decoding tables the kernels use.  One-off work per layer; everything here is integer or fp64
+// and must reproduce the format bit for bit on every run.
+#include <algorithm>
+#include <cmath>
+#include <cstring>
+#include <limits>
+#include <new>
+#include <numeric>
+
+#include "hac_internal.h"
+
+namespace hacb200 {
+
+namespace {
+
+// SplitMix64 (Steele, Lea, Flood, OOPSLA 2014) as a counter-based generator: draw i mixes
+// seed + (i + 1) * golden-ratio increment.
+inline uint64_t splitmix64_at(uint64_t seed, uint64_t i) {
+    uint64_t z = seed + (i + 1) * 0x9E3779B97F4A7C15ull;
+    z = (z ^ (z >> 30)) * 0xBF58476D1CE4E5B9ull;
+    z = (z ^ (z >> 27)) * 0x94D049BB133111EBull;
+    return z ^ (z >> 31);
+}
+
+struct Shared {                      // result of weight sharing over the q non-null weights
+    std::vector<float> level_value;  // value of each level (not yet merged / sorted)
+    std::vector<uint32_t> level_of;  // [q] level of each weight, column-major order
+};
+
+// Sect. III-C.1: Lloyd's k-means on scalars.  Centroids stay sorted, so the nearest centroid of w
+// is found by counting the midpoints below w; sums run in storage order in fp64.
+int share_kmeans(const std::vector<double>& data, uint32_t k, uint32_t iters, uint64_t seed,
+                 Shared& out) {
+    const size_t q = data.size();
+    std::vector<double> distinct(data);
+    std::sort(distinct.begin(), distinct.end());
+    distinct.erase(std::unique(distinct.begin(), distinct.end()), distinct.end());
+    out.level_of.resize(q);
+    if (distinct.size() <= k) {      // fewer distinct values than clusters: they are the codebook
+        out.level_value.resize(distinct.size());
+        for (size_t l = 0; l < distinct.size(); ++l) out.level_value[l] = (float)distinct[l];
+        for (size_t p = 0; p < q; ++p)
+            out.level_of[p] = (uint32_t)(std::lower_bound(distinct.begin(), distinct.end(), data[p]) -
+                                         distinct.begin());
+        return HAC_OK;
+    }
+    // seeded start: partial Fisher-Yates over the distinct values
+    std::vector<double> centroid(k);
+    {
+        const uint64_t U = distinct.size();
+        std::vector<uint32_t> perm(U);
+        std::iota(perm.begin(), perm.end(), 0u);
+        for (uint64_t i = 0; i < k; ++i) {
+            uint64_t j = i + splitmix64_at(seed, i) % (U - i);
+            std::swap(perm[i], perm[j]);
+            centroid[i] = distinct[perm[i]];
+        }
+        std::sort(centroid.begin(), centroid.end());
+    }
+    std::vector<double>().swap(distinct);
+    std::vector<double> mid(k > 1 ? k - 1 : 0), acc(k);
+    std::vector<int64_t> members(k);
+    for (uint32_t it = 0;; ++it) {
+        for (uint32_t l = 0; l + 1 < k; ++l) mid[l] = (centroid[l] + centroid[l + 1]) * 0.5;
+        std::fill(acc.begin(), acc.end(), 0.0);
+        std::fill(members.begin(), members.end(), (int64_t)0);
+        const double* mb = mid.data();
+        const double* me = mb + mid.size();
+        for (size_t p = 0; p < q; ++p) {
+            const double w = data[p];
+            const uint32_t l = (uint32_t)(std::lower_bound(mb, me, w) - mb);   // #midpoints < w
+            out.level_of[p] = l;
+            acc[l] += w;
+            members[l] += 1;
+        }
+        if (it == iters) break;
+        for (uint32_t l = 0; l < k; ++l)
+            if (members[l] > 0) centroid[l] = acc[l] / (double)members[l];
+        std::sort(centroid.begin(), centroid.end());
+    }
+    out.level_value.resize(k);
+    for (uint32_t l = 0; l < k; ++l) out.level_value[l] = (float)centroid[l];
+    return HAC_OK;
+}
+
+// Sect. III-C.3: uniform grid of k levels laid over [min, max] of the non-null weights.
+int share_uniform(const std::vector<double>& data, uint32_t k, Shared& out) {
+    const size_t q = data.size();
+    double lo = data[0], hi = data[0];
+    for (size_t p = 1; p < q; ++p) { lo = std::min(lo, data[p]); hi = std::max(hi, data[p]); }
+    out.level_of.assign(q, 0u);
+    if (hi == lo) { out.level_value.assign(1, (float)lo); return HAC_OK; }
+    const double delta = (hi - lo) / (double)(k - 1);
+    out.level_value.resize(k);
+    for (uint32_t l = 0; l < k; ++l) {
+        volatile double step = (double)l * delta;      // product rounded on its own (no fused add)
+        out.level_value[l] = (float)(lo + step);
+    }
+    const double top = (double)(k - 1);
+    for (size_t p = 0; p < q; ++p) {
+        double t = std::floor((data[p] - lo) / delta + 0.5);
+        if (t < 0.0) t = 0.0;
+        if (t > top) t = top;
+        out.level_of[p] = (uint32_t)t;
+    }
+    return HAC_OK;
+}
+
+int share_none(const std::vector<double>& data, Shared& out) {
+    std::vector<double> distinct(data);
+    std::sort(distinct.begin(), distinct.end());
+    distinct.erase(std::unique(distinct.begin(), distinct.end()), distinct.end());
+    if (distinct.size() > HAC_MAX_SYMBOLS) return HAC_ERR_K_TOO_LARGE;
+    out.level_value.resize(distinct.size());
+    for (size_t l = 0; l < distinct.size(); ++l) out.level_value[l] = (float)distinct[l];
+    out.level_of.resize(data.size());
+    for (size_t p = 0; p < data.size(); ++p)
+        out.level_of[p] = (uint32_t)(std::lower_bound(distinct.begin(), distinct.end(), data[p]) -
+                                     distinct.begin());
+    return HAC_OK;
+}
+
+// Huffman code lengths (Sect. IV-B) with the two-queue method: leaves in (count, id) order, merged
+// nodes in creation order, a leaf taken before a merged node of equal weight.
+int huffman_code_lengths(const std::vector<int64_t>& counts, std::vector<uint8_t>& len) {
+    const uint32_t k = (uint32_t)counts.size();
+    len.assign(k, 0);
+    if (k == 0) return HAC_OK;
+    if (k == 1) { len[0] = 1; return HAC_OK; }
+    std::vector<uint32_t> order(k);
+    std::iota(order.begin(), order.end(), 0u);
+    std::stable_sort(order.begin(), order.end(),
+                     [&](uint32_t a, uint32_t b) { return counts[a] < counts[b]; });
+    // nodes 0..k-1: leaves in sorted order; k..2k-2: merged nodes in creation order
+    std::vector<int64_t> weight(2 * k - 1);
+    std::vector<uint32_t> up(2 * k - 1, 0);
+    for (uint32_t i = 0; i < k; ++i) weight[i] = counts[order[i]];
+    uint32_t leaf = 0, inner = k, made = k;
+    auto pop = [&]() -> uint32_t {
+        if (leaf < k && (inner >= made || weight[leaf] <= weight[inner])) return leaf++;
+        return inner++;
+    };
+    while (made < 2 * k - 1) {
+        uint32_t a = pop();
+        uint32_t b = pop();
+        weight[made] = weight[a] + weight[b];
+        up[a] = made; up[b] = made;
+        ++made;
+    }
+    std::vector<uint32_t> depth(2 * k - 1, 0);
+    for (int64_t v = (int64_t)2 * k - 3; v >= 0; --v) depth[v] = depth[up[v]] + 1;
+    for (uint32_t i = 0; i < k; ++i) {
+        if (depth[i] > (uint32_t)kMaxCodeLen) return HAC_ERR_CODE_TOO_LONG;
+        len[order[i]] = (uint8_t)depth[i];
+    }
+    return HAC_OK;
+}
+
+// Canonical assignment: count the code words of each length, give each length its first code
+// (previous first + previous count, doubled), then hand codes out in symbol-id order per length.
+void canonical_assign(const std::vector<uint8_t>& len, std::vector<uint32_t>& codes) {
+    uint32_t per_len[kMaxCodeLen + 2] = {0};
+    for (uint8_t l : len) per_len[l]++;
+    uint64_t next[kMaxCodeLen + 2] = {0};
+    uint64_t code = 0;
+    for (int l = 1; l <= kMaxCodeLen; ++l) {
+        code = (code + per_len[l - 1]) << 1;
+        next[l] = code;
+    }
+    codes.resize(len.size());
+    for (size_t s = 0; s < len.size(); ++s) codes[s] = (uint32_t)next[len[s]]++;
+}
+
+struct BitWriter {
+    std::vector<uint32_t>& words;
+    uint64_t acc = 0;     // pending bits, right aligned
+    int pending = 0;
+    int64_t total = 0;
+    explicit BitWriter(std::vector<uint32_t>& w) : words(w) {}
+    inline void put(uint32_t code, int len) {
+        acc = (acc << len) | code;
+        pending += len;
+        total += len;
+        if (pending >= 32) {
+            pending -= 32;
+            words.push_back((uint32_t)(acc >> pending));
+        }
+    }
+    void finish() {
+        if (pending > 0) words.push_back((uint32_t)(acc << (32 - pending)));
+        pending = 0;
+    }
+};
+
+}  // namespace
+
+void make_decode_tables(Format& f) {
+    DecodeTables& t = f.tables;
+    const uint32_t k = (uint32_t)f.codebook.size();
+    t = DecodeTables();
+    if (k == 0) { t.lut_bits = 1; t.lut.assign(2, 0); return; }
+    std::vector<uint32_t> by_rank(k);
+    std::iota(by_rank.begin(), by_rank.end(), 0u);
+    std::stable_sort(by_rank.begin(), by_rank.end(),
+                     [&](uint32_t a, uint32_t b) { return f.code_len[a] < f.code_len[b]; });
+    t.rank_value.resize(k);
+    t.rank_symbol.resize(k);
+    for (uint32_t r = 0; r < k; ++r) {
+        t.rank_value[r] = f.codebook[by_rank[r]];
+        t.rank_symbol[r] = (uint16_t)by_rank[r];
+    }
+    t.lut_bits = std::min<int>((int)f.max_len, kLutBitsMax);
+    t.lut.assign((size_t)1 << t.lut_bits, 0);
+    uint32_t per_len[kMaxCodeLen + 2] = {0};
+    for (uint32_t s = 0; s < k; ++s) per_len[f.code_len[s]]++;
+    uint32_t rank = 0;
+    uint64_t first = 0;                      // first code of the current length
+    for (int l = 1; l <= kMaxCodeLen; ++l) {
+        first = (l == 1) ? 0 : (first + per_len[l - 1]) << 1;
+        t.first_left[l] = (uint32_t)(first << (32 - l));
+        t.rank_base[l] = rank;
+        t.limit[l] = (first + per_len[l]) << (32 - l);
+        rank += per_len[l];
+    }
+    t.limit[kMaxCodeLen + 1] = (uint64_t)1 << 32;
+    for (uint32_t r = 0; r < k; ++r) {
+        const uint32_t s = by_rank[r];
+        const int l = f.code_len[s];
+        if (l > t.lut_bits) continue;
+        const uint32_t lo = f.codes[s] << (t.lut_bits - l);
+        const uint32_t span = 1u << (t.lut_bits - l);
+        const uint16_t e = (uint16_t)((r << 5) | (uint32_t)l);
+        for (uint32_t i = 0; i < span; ++i) t.lut[lo + i] = e;
+    }
+}
+
+int build_impl(const float* W, int64_t n, int64_t m, int64_t ldw, const hac_build_params* p,
+                      bool sparse, Format& f) {
+    if (!W || !p || n < 1 || m < 1 || ldw < m) return HAC_ERR_INVALID_ARG;
+    if (!(p->sparsity >= 0.0 && p->sparsity < 1.0) || p->reserved != 0) return HAC_ERR_INVALID_ARG;
+    if (p->quantizer > HAC_QUANT_UNIFORM) return HAC_ERR_INVALID_ARG;
+    if (p->quantizer == HAC_QUANT_KMEANS && p->k < 1) return HAC_ERR_INVALID_ARG;
+    if (p->quantizer == HAC_QUANT_UNIFORM && p->k < 2) return HAC_ERR_INVALID_ARG;
+    if (p->seg_symbols > HAC_MAX_SEG_SYMBOLS) return HAC_ERR_INVALID_ARG;
+    if (p->ri_bits != 0 && p->ri_bits != 16 && p->ri_bits != 32) return HAC_ERR_INVALID_ARG;
+    if (n > (int64_t)1 << 31 || m > (int64_t)1 << 31 || n * m > ((int64_t)1 << 36))
+        return HAC_ERR_OFFSET_OVERFLOW;
+    f.sparse = sparse;
+    f.n = n; f.m = m;
+    f.S = p->seg_symbols ? p->seg_symbols : (sparse ? 32u : 64u);
+    f.ri_bits = sparse ? (p->ri_bits ? p->ri_bits : (n <= 65536 ? 16u : 32u)) : 0u;
+    if (sparse && f.ri_bits == 16 && n > 65536) return HAC_ERR_INVALID_ARG;
+    const int64_t total = n * m;
+
+    // column-major copy, input checks
+    std::vector<float> col(total);
+    for (int64_t i = 0; i < n; ++i) {
+        const float* row = W + i * ldw;
+        for (int64_t j = 0; j < m; ++j) {
+            float v = row[j];
+            if (!std::isfinite(v)) return HAC_ERR_NONFINITE_INPUT;
+            col[j * n + i] = (v == 0.0f) ? 0.0f : v;
+        }
+    }
+    // Sect. III-B: threshold = z-th smallest magnitude, entries at or below it go
+    const int64_t z = (int64_t)std::floor(p->sparsity * (double)total);
+    if (z > 0) {
+        std::vector<float> mag(total);
+        for (int64_t t = 0; t < total; ++t) mag[t] = std::fabs(col[t]);
+        std::nth_element(mag.begin(), mag.begin() + (z - 1), mag.end());
+        const float tau = mag[z - 1];
+        for (int64_t t = 0; t < total; ++t)
+            if (std::fabs(col[t]) <= tau) col[t] = 0.0f;
+    }
+    // non-null weights in column-major order
+    int64_t q = 0;
+    for (int64_t t = 0; t < total; ++t) q += (col[t] != 0.0f);
+    f.nnz = q;
+    if (q >= ((int64_t)1 << 32)) return HAC_ERR_OFFSET_OVERFLOW;
+    std::vector<double> data;
+    data.reserve(q);
+    for (int64_t t = 0; t < total; ++t)
+        if (col[t] != 0.0f) data.push_back((double)col[t]);
+
+    Shared sh;
+    if (q > 0) {
+        int rc = HAC_OK;
+        if (p->quantizer == HAC_QUANT_KMEANS) rc = share_kmeans(data, p->k, p->kmeans_iters, p->seed, sh);
+        else if (p->quantizer == HAC_QUANT_UNIFORM) rc = share_uniform(data, p->k, sh);
+        else rc = share_none(data, sh);
+        if (rc != HAC_OK) return rc;
+    }
+    std::vector<double>().swap(data);
+    for (float& v : sh.level_value) if (v == 0.0f) v = 0.0f;           // -0.0 -> +0.0
+
+    // alphabet: occupied levels (plus zero for HAC when a null entry exists), merged by value
+    const size_t nlev = sh.level_value.size();
+    std::vector<int64_t> level_count(nlev, 0);
+    for (int64_t t = 0; t < q; ++t) level_count[sh.level_of[t]]++;
+    std::vector<float> values;
+    for (size_t l = 0; l < nlev; ++l) if (level_count[l] > 0) values.push_back(sh.level_value[l]);
+    const int64_t nulls = total - q;
+    if (!sparse && nulls > 0) values.push_back(0.0f);
+    std::sort(values.begin(), values.end());
+    values.erase(std::unique(values.begin(), values.end()), values.end());
+    if (values.size() > HAC_MAX_SYMBOLS) return HAC_ERR_K_TOO_LARGE;
+    f.codebook = values;
+    const uint32_t k_eff = (uint32_t)values.size();
+    std::vector<uint32_t> level_symbol(nlev, 0);
+    for (size_t l = 0; l < nlev; ++l)
+        level_symbol[l] = (uint32_t)(std::lower_bound(values.begin(), values.end(), sh.level_value[l]) -
+                                     values.begin());
+    uint32_t zero_symbol = 0;
+    if (!sparse && nulls > 0)
+        zero_symbol = (uint32_t)(std::lower_bound(values.begin(), values.end(), 0.0f) - values.begin());
+    f.counts.assign(k_eff, 0);
+    for (size_t l = 0; l < nlev; ++l) if (level_count[l] > 0) f.counts[level_symbol[l]] += level_count[l];
+    if (!sparse && nulls > 0) f.counts[zero_symbol] += nulls;
+
+    int rc = huffman_code_lengths(f.counts, f.code_len);
+    if (rc != HAC_OK) return rc;
+    canonical_assign(f.code_len, f.codes);
+    f.max_len = 0; f.min_len = k_eff ? 255 : 0;
+    for (uint8_t l : f.code_len) { f.max_len = std::max<uint32_t>(f.max_len, l); f.min_len = std::min<uint32_t>(f.min_len, l); }
+    if ((uint64_t)f.S * f.max_len > 65535u) return HAC_ERR_OFFSET_OVERFLOW;   // sub_bits is 16 bit
+
+    // Sect. IV-B / IV-C: emit the code words column by column, recording the offset index on the way
+    const uint32_t S = f.S;
+    BitWriter bw(f.stream);
+    f.symbols = sparse ? q : total;
+    {
+        double expect = 0;
+        for (uint32_t s = 0; s < k_eff; ++s) expect += (double)f.counts[s] * f.code_len[s];
+        f.stream.reserve((size_t)(expect / 32) + 16);
+    }
+    if (sparse) {
+        f.cb.assign(m + 1, 0);
+        f.seg_first.assign(m + 1, 0);
+        if (f.ri_bits == 16) f.ri16.reserve(q); else f.ri32.reserve(q);
+    } else {
+        const uint32_t T = (uint32_t)((n + S - 1) / S);
+        f.G = (T + 31) / 32;
+        if ((uint64_t)f.G * (uint64_t)m >= ((uint64_t)1 << 31)) return HAC_ERR_OFFSET_OVERFLOW;
+    }
+    int64_t w = 0;   // running index into the non-null weights
+    for (int64_t j = 0; j < m; ++j) {
+        const float* c = col.data() + j * n;
+        uint32_t in_sub = 0, subs_in_col = 0;
+        int64_t sub_start_bit = bw.total;
+        auto open_segment_if_needed = [&]() {
+            if (in_sub == 0 && (subs_in_col % 32) == 0) {
+                f.seg_bit_off.push_back((uint64_t)bw.total);
+                f.sub_bits.resize(f.sub_bits.size() + 32, 0);
+                if (sparse) f.seg_col.push_back((uint32_t)j);
+            }
+            if (in_sub == 0) sub_start_bit = bw.total;
+        };
+        auto close_sub = [&]() {
+            f.sub_bits[f.sub_bits.size() - 32 + (subs_in_col % 32)] = (uint16_t)(bw.total - sub_start_bit);
+            ++subs_in_col;
+            in_sub = 0;
+        };
+        for (int64_t i = 0; i < n; ++i) {
+            const bool stored = (c[i] != 0.0f);
+            uint32_t s;
+            if (stored) s = level_symbol[sh.level_of[w++]];
+            else if (sparse) continue;
+            else s = zero_symbol;
+            open_segment_if_needed();
+            bw.put(f.codes[s], f.code_len[s]);
+            if (sparse) { if (f.ri_bits == 16) f.ri16.push_back((uint16_t)i); else f.ri32.push_back((uint32_t)i); }
+            if (++in_sub == S) close_sub();
+        }
+        if (in_sub > 0) close_sub();
+        if (sparse) {
+            f.cb[j + 1] = (uint32_t)w;
+            f.seg_first[j + 1] = (uint32_t)f.seg_bit_off.size();
+        }
+    }
+    bw.finish();
+    f.stream_bits = bw.total;
+    f.stream_words = (int64_t)f.stream.size();
+    const int64_t padded = ((f.stream_words + 3) / 4) * 4 + kStreamSlackWords;
+    f.pad_words = padded - f.stream_words;
+    f.stream.resize(padded, 0u);
+
+    // per-segment statistics used to size shared memory and to pick the reduction path
+    const size_t U = f.seg_bit_off.size();
+    f.max_unit_chunks = 1;
+    for (size_t u = 0; u < U; ++u) {
+        uint64_t bits = 0;
+        for (int l = 0; l < 32; ++l) bits += f.sub_bits[u * 32 + l];
+        const uint64_t first_chunk = f.seg_bit_off[u] >> 7;
+        const uint64_t last_word = ((f.seg_bit_off[u] + bits) >> 5) + 2;
+        f.max_unit_chunks = std::max<uint32_t>(f.max_unit_chunks, (uint32_t)((last_word >> 2) - first_chunk + 1));
+    }
+    if (sparse) {
+        f.max_units_per_col = 0;
+        f.has_empty_col = false;
+        for (int64_t j = 0; j < m; ++j) {
+            const uint32_t g = f.seg_first[j + 1] - f.seg_first[j];
+            f.max_units_per_col = std::max(f.max_units_per_col, g);
+            if (g == 0) f.has_empty_col = true;
+        }
+    } else {
+        f.max_units_per_col = f.G;
+    }
+    make_decode_tables(f);
+    return HAC_OK;
+}
+
+// Host decoder (canonical decoding by lengths, one symbol at a time); used by *_decode_host.
+int decode_on_host(const Format& f, float* Wq, int64_t ldq) {
+    if (!Wq || ldq < f.m) return HAC_ERR_INVALID_ARG;
+    for (int64_t i = 0; i < f.n; ++i) std::fill(Wq + i * ldq, Wq + i * ldq + f.m, 0.0f);
+    const DecodeTables& t = f.tables;
+    uint64_t bit = 0;
+    auto next_value = [&](float& v) -> bool {
+        uint64_t wi = bit >> 5;
+        uint32_t sh = (uint32_t)(bit & 31);
+        if ((int64_t)wi + 1 >= (int64_t)f.stream.size()) return false;
+        uint64_t two = ((uint64_t)f.stream[wi] << 32) | f.stream[wi + 1];
+        uint32_t top = (uint32_t)((two << sh) >> 32);
+        for (uint32_t l = f.min_len; l <= f.max_len; ++l) {
+            if ((uint64_t)top < t.limit[l]) {
+                uint32_t r = t.rank_base[l] + ((top - t.first_left[l]) >> (32 - l));
+                if (r >= t.rank_value.size()) return false;
+                v = t.rank_value[r];
+                bit += l;
+                return true;
+            }
+        }
+        return false;
+    };
+    if (!f.sparse) {
+        for (int64_t j = 0; j < f.m; ++j)
+            for (int64_t i = 0; i < f.n; ++i) {
+                float v;
+                if (!next_value(v)) return HAC_ERR_CORRUPT;
+                Wq[i * ldq + j] = v;
+            }
+    } else {
+        for (int64_t j = 0; j < f.m; ++j)
+            for (uint32_t p = f.cb[j]; p < f.cb[j + 1]; ++p) {
+                float v;
+                if (!next_value(v)) return HAC_ERR_CORRUPT;
+                const int64_t i = f.ri_bits == 16 ? (int64_t)f.ri16[p] : (int64_t)f.ri32[p];
+                Wq[i * ldq + j] = v;
+            }
+    }
+    return (int64_t)bit == f.stream_bits ? HAC_OK : HAC_ERR_CORRUPT;
+}
+
+void fill_size_report(const Format& f, hac_size_report* r) {
+    std::memset(r, 0, sizeof(*r));
+    r->n = f.n; r->m = f.m; r->nnz = f.nnz; r->symbols = f.symbols;
+    r->stream_bits = f.stream_bits;
+    r->stream_words = f.stream_words;
+    r->stream_bytes = 4 * f.stream_words;
+    r->pad_bytes = 4 * f.pad_words;
+    r->codebook_bytes = 4 * (int64_t)f.codebook.size();
+    r->code_len_bytes = (int64_t)f.code_len.size();
+    r->ri_bytes = f.sparse ? f.nnz * (int64_t)f.ri_bits / 8 : 0;
+    r->cb_bytes = f.sparse ? 4 * (f.m + 1) : 0;
+    r->offset_index_bytes = (int64_t)(f.seg_bit_off.size() * 8 + f.sub_bits.size() * 2 +
+                                      f.seg_first.size() * 4 + f.seg_col.size() * 4);
+    r->total_bytes = r->stream_bytes + r->pad_bytes + r->codebook_bytes + r->code_len_bytes +
+                     r->ri_bytes + r->cb_bytes + r->offset_index_bytes;
+    const int64_t k = (int64_t)f.codebook.size();
+    const double logk = k > 0 ? std::log2((double)k) : 0.0;
+    if (!f.sparse) {
+        r->paper_bits = 32 * f.stream_words + 6 * k * 32;
+        r->bound_bits = (double)f.n * (double)f.m * (1.0 + logk) + 6.0 * k * 32;
+    } else {
+        r->paper_bits = 32 * f.stream_words + 6 * k * 32 + 32 * (f.nnz + f.m + 1);
+        r->bound_bits = (double)f.nnz * (1.0 + logk) + 32.0 * (6.0 * k + (double)f.nnz + f.m + 1);
+    }
+    double H = 0.0;
+    for (int64_t c : f.counts)
+        if (c > 0) { double pr = (double)c / (double)f.symbols; H -= pr * std::log2(pr); }
+    r->entropy = H;
+    r->avg_code_len = f.symbols ? (double)f.stream_bits / (double)f.symbols : 0.0;
+    r->k_eff = (uint32_t)k;
+    r->max_code_len = f.max_len; r->min_code_len = f.min_len;
+    r->seg_symbols = f.S; r->ri_bits = f.ri_bits;
+    r->units = (uint32_t)f.seg_bit_off.size();
+}
+
+static size_t align256(size_t x) { return (x + 255) & ~(size_t)255; }
+
+ImageLayout image_layout(const Format& f) {
+    ImageLayout L{};
+    size_t o = 0;
+    auto take = [&](size_t bytes) { size_t at = o; o = align256(o + std::max<size_t>(bytes, 16)); return at; };
+    L.stream = take(f.stream.size() * 4);
+    L.lut = take(f.tables.lut.size() * 2);
+    L.rank_value = take(f.tables.rank_value.size() * 4);
+    L.limit = take(sizeof(f.tables.limit));
+    L.first_left = take(sizeof(f.tables.first_left));
+    L.rank_base = take(sizeof(f.tables.rank_base));
+    L.seg_bit_off = take(f.seg_bit_off.size() * 8);
+    L.sub_bits = take(f.sub_bits.size() * 2);
+    L.seg_col = take(f.seg_col.size() * 4);
+    L.seg_first = take(f.seg_first.size() * 4);
+    L.ri = take(f.ri_bits == 16 ? f.ri16.size() * 2 + 16 : f.ri32.size() * 4 + 16);
+    L.cb = take(f.cb.size() * 4);
+    L.total = o;
+    return L;
+}
+
+}  // namespace hacb200
+
+using hacb200::Format;
+
+extern "C" {
+
+int hac_build(const float* W, int64_t n, int64_t m, int64_t ldw, const hac_build_params* params,
+              hac_format** out) {
+    if (!out) return HAC_ERR_INVALID_ARG;
+    *out = nullptr;
+    hac_format* h = new (std::nothrow) hac_format();
+    if (!h) return HAC_ERR_ALLOC;
+    int rc;
+    try { rc = hacb200::build_impl(W, n, m, ldw, params, false, h->f); }
+    catch (const std::bad_alloc&) { rc = HAC_ERR_ALLOC; }
+    if (rc != HAC_OK) { delete h; return rc; }
+    *out = h;
+    return HAC_OK;
+}
+
+int shac_build(const float* W, int64_t n, int64_t m, int64_t ldw, const hac_build_params* params,
+               shac_format** out) {
+    if (!out) return HAC_ERR_INVALID_ARG;
+    *out = nullptr;
+    shac_format* h = new (std::nothrow) shac_format();
+    if (!h) return HAC_ERR_ALLOC;
+    int rc;
+    try { rc = hacb200::build_impl(W, n, m, ldw, params, true, h->f); }
+    catch (const std::bad_alloc&) { rc = HAC_ERR_ALLOC; }
+    if (rc != HAC_OK) { delete h; return rc; }
+    *out = h;
+    return HAC_OK;
+}
+
+int hac_sizes(const hac_format* f, hac_size_report* out) {
+    if (!f || !out) return HAC_ERR_INVALID_ARG;
+    hacb200::fill_size_report(f->f, out);
+    return HAC_OK;
+}
+int shac_sizes(const shac_format* f, hac_size_report* out) {
+    if (!f || !out) return HAC_ERR_INVALID_ARG;
+    hacb200::fill_size_report(f->f, out);
+    return HAC_OK;
+}
+
+static void fill_view(const Format& f, hac_host_view* v) {
+    v->n = f.n; v->m = f.m;
+    v->k_eff = (uint32_t)f.codebook.size();
+    v->seg_symbols = f.S;
+    v->codebook = f.codebook.data();
+    v->code_len = f.code_len.data();
+    v->codes = f.codes.data();
+    v->counts = f.counts.data();
+    v->stream = f.stream.data();
+    v->stream_bits = f.stream_bits;
+    v->stream_words = f.stream_words;
+    v->stream_pad_words = f.pad_words;
+    v->units = (uint32_t)f.seg_bit_off.size();
+    v->segs_per_col = f.sparse ? 0 : f.G;
+    v->seg_bit_off = f.seg_bit_off.data();
+    v->sub_bits = f.sub_bits.data();
+}
+
+int hac_export(const hac_format* f, hac_host_view* out) {
+    if (!f || !out) return HAC_ERR_INVALID_ARG;
+    fill_view(f->f, out);
+    return HAC_OK;
+}
+int shac_export(const shac_format* f, shac_host_view* out) {
+    if (!f || !out) return HAC_ERR_INVALID_ARG;
+    fill_view(f->f, &out->base);
+    out->nnz = f->f.nnz;
+    out->ri_bits = f->f.ri_bits;
+    out->ri = f->f.ri_bits == 16 ? (const void*)f->f.ri16.data() : (const void*)f->f.ri32.data();
+    out->cb = f->f.cb.data();
+    out->seg_first = f->f.seg_first.data();
+    out->seg_col = f->f.seg_col.data();
+    return HAC_OK;
+}
+
+int hac_decode_host(const hac_format* f, float* Wq, int64_t ldq) {
+    if (!f) return HAC_ERR_INVALID_ARG;
+    return hacb200::decode_on_host(f->f, Wq, ldq);
+}
+int shac_decode_host(const shac_format* f, float* Wq, int64_t ldq) {
+    if (!f) return HAC_ERR_INVALID_ARG;
+    return hacb200::decode_on_host(f->f, Wq, ldq);
+}
+
+const char* hac_status_string(int status) {
+    switch (status) {
+        case HAC_OK: return "ok";
+        case HAC_ERR_INVALID_ARG: return "invalid argument";
+        case HAC_ERR_ALLOC: return "host allocation failed";
+        case HAC_ERR_NONFINITE_INPUT: return "W holds NaN or Inf";
+        case HAC_ERR_K_TOO_LARGE: return "too many distinct values";
+        case HAC_ERR_CODE_TOO_LONG: return "Huffman code word longer than 32 bits";
+        case HAC_ERR_OFFSET_OVERFLOW: return "size or offset overflow";
+        case HAC_ERR_NOT_UPLOADED: return "format not uploaded to the device";
+        case HAC_ERR_BUFFER_TOO_SMALL: return "buffer too small";
+        case HAC_ERR_CUDA: return "CUDA error";
+        case HAC_ERR_CORRUPT: return "corrupt data";
+        default: return "unknown status";
+    }
+}
+
+}  // extern "C"

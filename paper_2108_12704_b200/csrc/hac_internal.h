@@ -1,0 +1,98 @@
+// Internal definitions shared by the host builder (hac_build.cpp) and the device side
+// (hac_kernels.cu) of the library.  Not part of the public boundary.
+#pragma once
+
+#include <cstddef>
+#include <cstdint>
+#include <vector>
+
+#include "hac.h"
+
+namespace hacb200 {
+
+constexpr int kMaxCodeLen = 32;
+constexpr int kLutBitsMax = 12;          // primary decode table: 2^L entries of 16 bits
+constexpr int kStreamSlackWords = 4;     // zero words after the stream (decoder reads ahead)
+
+// Decoding tables derived from the code lengths (canonical Huffman).  "rank" is the position of
+// a symbol in (length, id) order; values are stored in rank order so that short, frequent code
+// words use the first entries.
+struct DecodeTables {
+    int lut_bits = 0;                         // L = min(max_len, kLutBitsMax)
+    std::vector<uint16_t> lut;                // [2^L] (rank << 5) | len, 0 = code longer than L
+    std::vector<float> rank_value;            // [k_eff]
+    std::vector<uint16_t> rank_symbol;        // [k_eff] symbol id of each rank
+    uint64_t limit[kMaxCodeLen + 2] = {};     // left-aligned (32-bit) end of the codes of length l
+    uint32_t first_left[kMaxCodeLen + 2] = {};// left-aligned first code of length l
+    uint32_t rank_base[kMaxCodeLen + 2] = {}; // rank of the first code of length l
+};
+
+// Pointers into the device image, filled by upload/attach.
+struct DeviceImage {
+    void* base = nullptr;
+    size_t bytes = 0;
+    const uint32_t* stream = nullptr;
+    const uint16_t* lut = nullptr;
+    const float* rank_value = nullptr;
+    const uint64_t* limit = nullptr;          // [34]
+    const uint32_t* first_left = nullptr;     // [34]
+    const uint32_t* rank_base = nullptr;      // [34]
+    const uint64_t* seg_bit_off = nullptr;
+    const uint16_t* sub_bits = nullptr;
+    const uint32_t* seg_col = nullptr;
+    const uint32_t* seg_first = nullptr;
+    const void* ri = nullptr;
+    const uint32_t* cb = nullptr;
+};
+
+struct Format {
+    bool sparse = false;                      // sHAC
+    int64_t n = 0, m = 0;
+    int64_t nnz = 0;                          // entries surviving pruning
+    int64_t symbols = 0;                      // n*m (HAC) or nnz (sHAC)
+    uint32_t S = 0;                           // symbols per sub-segment
+    uint32_t G = 0;                           // HAC: segments per column
+    uint32_t ri_bits = 0;
+    // alphabet
+    std::vector<float> codebook;              // ascending
+    std::vector<uint8_t> code_len;
+    std::vector<uint32_t> codes;
+    std::vector<int64_t> counts;
+    uint32_t max_len = 0, min_len = 0;
+    // stream
+    std::vector<uint32_t> stream;             // stream_words data words + pad words
+    int64_t stream_bits = 0, stream_words = 0, pad_words = 0;
+    // sHAC
+    std::vector<uint16_t> ri16;
+    std::vector<uint32_t> ri32;
+    std::vector<uint32_t> cb;
+    // offset index
+    std::vector<uint64_t> seg_bit_off;
+    std::vector<uint16_t> sub_bits;
+    std::vector<uint32_t> seg_first, seg_col;
+    uint32_t max_unit_chunks = 0;             // largest 16-byte span a segment's stream covers
+    uint32_t max_units_per_col = 0;
+    bool has_empty_col = false;
+    // derived
+    DecodeTables tables;
+    DeviceImage dev;
+    mutable int last_launches = 0;
+};
+
+int build_impl(const float* W, int64_t n, int64_t m, int64_t ldw, const hac_build_params* p,
+               bool sparse, Format& f);
+void make_decode_tables(Format& f);
+int decode_on_host(const Format& f, float* Wq, int64_t ldq);
+void fill_size_report(const Format& f, hac_size_report* r);
+
+// device image layout: offsets of every section (256-byte aligned), total size
+struct ImageLayout {
+    size_t stream, lut, rank_value, limit, first_left, rank_base, seg_bit_off, sub_bits, seg_col,
+        seg_first, ri, cb, total;
+};
+ImageLayout image_layout(const Format& f);
+
+}  // namespace hacb200
+
+struct hac_format { hacb200::Format f; };
+struct shac_format { hacb200::Format f; };

@@ -1,0 +1,914 @@
+// Device side of the library: upload of a built format and the fused decode-multiply-accumulate
+// kernels for HAC (Algorithm 1) and sHAC (Algorithm 2), for one input and for a batch
+// (Algorithm 3), written for sm_100a.
+//
+// Work decomposition.  The offset index cuts every column into sub-segments of S symbols; 32
+// consecutive sub-segments form a segment, the work unit of one warp.  A warp reads the 32
+// sub-segment bit lengths, turns them into per-lane start bits with a shuffle scan, copies the
+// segment's span of the stream into shared memory with 128-bit coalesced loads, and then every
+// lane decodes its own sub-segment from shared memory with a table lookup per code word.  Partial
+// dot products are combined with warp shuffles; columns that span several segments are finished
+// by a small second kernel that adds the per-segment partials in a fixed order.
+#include <cuda_runtime.h>
+
+#include <algorithm>
+#include <cstdio>
+#include <cstdlib>
+#include <cstring>
+#include <string>
+
+#include "hac_internal.h"
+
+namespace hacb200 {
+
+static thread_local std::string g_last_cuda_error;
+
+static int cuda_fail(cudaError_t e, const char* what) {
+    g_last_cuda_error = std::string(what) + ": " + cudaGetErrorString(e);
+    return HAC_ERR_CUDA;
+}
+#define HAC_CUDA(call)                                              \
+    do {                                                            \
+        cudaError_t e_ = (call);                                    \
+        if (e_ != cudaSuccess) return cuda_fail(e_, #call);         \
+    } while (0)
+
+// ------------------------------------------------------------------------------------------------
+// Kernel-side view of a format (device pointers and scalars), passed by value.
+// ------------------------------------------------------------------------------------------------
+struct DevFormat {
+    const uint32_t* stream;
+    const uint16_t* lut;
+    const float* rank_value;
+    const uint64_t* limit;
+    const uint32_t* first_left;
+    const uint32_t* rank_base;
+    const uint64_t* seg_bit_off;
+    const uint16_t* sub_bits;
+    const uint32_t* seg_col;
+    const uint32_t* seg_first;
+    const void* ri;
+    const uint32_t* cb;
+    uint32_t n, m, units, G, S, k_eff, lut_bits, max_len, ri_bits, max_unit_chunks;
+};
+
+constexpr int kTableWords = 34;
+
+// Decoding tables in shared memory.
+struct SmemTables {
+    const uint16_t* lut;
+    const float* value;
+    const uint64_t* limit;
+    const uint32_t* first_left;
+    const uint32_t* rank_base;
+};
+
+__host__ __device__ inline size_t align16(size_t x) { return (x + 15) & ~(size_t)15; }
+
+__host__ __device__ inline size_t tables_smem_bytes(uint32_t lut_bits, uint32_t k_eff) {
+    return align16(((size_t)2 << lut_bits)) + align16((size_t)k_eff * 4) + align16(kTableWords * 8) +
+           2 * align16(kTableWords * 4);
+}
+
+// Copies the tables to shared memory (all threads of the block take part) and returns the carve-up.
+// `p` is advanced past the tables.
+__device__ inline SmemTables stage_tables(const DevFormat& f, unsigned char*& p) {
+    SmemTables t;
+    uint16_t* lut = reinterpret_cast<uint16_t*>(p);
+    p += align16((size_t)2 << f.lut_bits);
+    float* value = reinterpret_cast<float*>(p);
+    p += align16((size_t)f.k_eff * 4);
+    uint64_t* limit = reinterpret_cast<uint64_t*>(p);
+    p += align16(kTableWords * 8);
+    uint32_t* first_left = reinterpret_cast<uint32_t*>(p);
+    p += align16(kTableWords * 4);
+    uint32_t* rank_base = reinterpret_cast<uint32_t*>(p);
+    p += align16(kTableWords * 4);
+    const uint32_t lut_words = (1u << f.lut_bits) / 2;     // pairs of 16-bit entries
+    if (lut_words == 0) {
+        if (threadIdx.x < 2) lut[threadIdx.x] = f.lut[threadIdx.x];
+    } else {
+        const uint32_t* src = reinterpret_cast<const uint32_t*>(f.lut);
+        uint32_t* dst = reinterpret_cast<uint32_t*>(lut);
+        for (uint32_t i = threadIdx.x; i < lut_words; i += blockDim.x) dst[i] = src[i];
+    }
+    for (uint32_t i = threadIdx.x; i < f.k_eff; i += blockDim.x) value[i] = f.rank_value[i];
+    if (threadIdx.x < kTableWords) {
+        limit[threadIdx.x] = f.limit[threadIdx.x];
+        first_left[threadIdx.x] = f.first_left[threadIdx.x];
+        rank_base[threadIdx.x] = f.rank_base[threadIdx.x];
+    }
+    t.lut = lut; t.value = value; t.limit = limit; t.first_left = first_left; t.rank_base = rank_base;
+    return t;
+}
+
+// Per-lane bit reader over the staged span: `buf` holds the next bits left aligned, `avail` of
+// them valid; after refill() more than 32 are valid, enough for any code word.
+struct BitReader {
+    const uint32_t* words;
+    uint32_t next;
+    uint64_t buf;
+    int avail;
+    __device__ __forceinline__ void init(const uint32_t* w, uint32_t bitpos) {
+        words = w;
+        const uint32_t wi = bitpos >> 5, sh = bitpos & 31;
+        const uint64_t two = ((uint64_t)w[wi] << 32) | w[wi + 1];
+        buf = two << sh;
+        avail = 64 - (int)sh;
+        next = wi + 2;
+    }
+    __device__ __forceinline__ void refill() {
+        if (avail <= 32) {
+            buf |= (uint64_t)words[next++] << (32 - avail);
+            avail += 32;
+        }
+    }
+    __device__ __forceinline__ void skip(uint32_t len) { buf <<= len; avail -= (int)len; }
+};
+
+// One code word: table lookup on the top L bits; code words longer than L fall back to the
+// canonical length search.  Returns the rank of the symbol.
+__device__ __forceinline__ uint32_t decode_symbol(BitReader& br, const SmemTables& t, uint32_t lut_shift,
+                                                  uint32_t lut_bits, uint32_t max_len) {
+    br.refill();
+    const uint32_t top = (uint32_t)(br.buf >> 32);
+    const uint32_t e = t.lut[top >> lut_shift];
+    uint32_t len = e & 31u, rank = e >> 5;
+    if (len == 0) {
+        len = max_len; rank = 0;
+        for (uint32_t l = lut_bits + 1; l <= max_len; ++l) {
+            if ((uint64_t)top < t.limit[l]) {
+                len = l;
+                rank = t.rank_base[l] + ((top - t.first_left[l]) >> (32 - l));
+                break;
+            }
+        }
+    }
+    br.skip(len);
+    return rank;
+}
+
+// Start bit of each lane's sub-segment inside the segment (exclusive scan of the 32 lengths by
+// shuffles) and the segment's total bit length.
+__device__ __forceinline__ uint32_t lane_start_bits(uint32_t my_bits, uint32_t lane, uint32_t& total) {
+    uint32_t inc = my_bits;
+#pragma unroll
+    for (int d = 1; d < 32; d <<= 1) {
+        uint32_t v = __shfl_up_sync(0xffffffffu, inc, d);
+        if ((int)lane >= d) inc += v;
+    }
+    total = __shfl_sync(0xffffffffu, inc, 31);
+    return inc - my_bits;
+}
+
+// Copy the stream span of one segment to the warp's staging area with 128-bit coalesced loads.
+// Returns the bit position of the segment start relative to the staged span.
+__device__ __forceinline__ uint32_t stage_span(const DevFormat& f, uint64_t seg_bit, uint32_t total_bits,
+                                               uint4* stage, uint32_t lane) {
+    const uint64_t first_chunk = seg_bit >> 7;
+    const uint64_t last_word = ((seg_bit + total_bits) >> 5) + 2;
+    const uint32_t chunks = (uint32_t)((last_word >> 2) - first_chunk + 1);
+    const uint4* src = reinterpret_cast<const uint4*>(f.stream) + first_chunk;
+    for (uint32_t c = lane; c < chunks; c += 32) stage[c] = __ldg(src + c);
+    __syncwarp();
+    return (uint32_t)(seg_bit - (first_chunk << 7));
+}
+
+__device__ __forceinline__ float warp_sum(float v) {
+#pragma unroll
+    for (int d = 16; d > 0; d >>= 1) v += __shfl_xor_sync(0xffffffffu, v, d);
+    return v;
+}
+
+// ------------------------------------------------------------------------------------------------
+// HAC, one input vector (Algorithm 1 by segments).  x is staged in shared memory; a lane's rows
+// are consecutive, lanes are S rows apart, so one padding word per sub-segment (when S is even)
+// keeps the 32 lanes on distinct banks.
+//   kMode 0: product; 1: debug decode (values written to out[j*n + i]).
+// ------------------------------------------------------------------------------------------------
+template <int kMode, bool kXShared>
+__global__ void __launch_bounds__(1024) hac_vec_kernel(DevFormat f, const float* __restrict__ x, int64_t xs_i,
+                                                       float* __restrict__ y, int64_t ys_j,
+                                                       float* __restrict__ aux) {
+    extern __shared__ __align__(16) unsigned char smem[];
+    unsigned char* p = smem;
+    const SmemTables t = stage_tables(f, p);
+    const uint32_t pad = (f.S & 1u) ? 0u : 1u;
+    float* xs = reinterpret_cast<float*>(p);
+    if (kMode == 0 && kXShared) {
+        for (uint32_t i = threadIdx.x; i < f.n; i += blockDim.x) xs[i + pad * (i / f.S)] = x[(int64_t)i * xs_i];
+        p += align16(((size_t)f.n + (f.n / f.S + 1) * pad) * 4);
+    }
+    const uint32_t warp = threadIdx.x >> 5, lane = threadIdx.x & 31, warps = blockDim.x >> 5;
+    uint4* stage = reinterpret_cast<uint4*>(p) + (size_t)warp * f.max_unit_chunks;
+    __syncthreads();
+    const uint32_t lut_shift = 32 - f.lut_bits;
+
+    for (uint32_t u = blockIdx.x * warps + warp; u < f.units; u += gridDim.x * warps) {
+        const uint32_t j = u / f.G, g = u - j * f.G;
+        const uint32_t my_bits = f.sub_bits[(size_t)u * 32 + lane];
+        uint32_t total;
+        const uint32_t start = lane_start_bits(my_bits, lane, total);
+        const uint32_t base = stage_span(f, f.seg_bit_off[u], total, stage, lane);
+        const uint32_t sub = g * 32 + lane;                 // sub-segment number inside the column
+        const uint32_t row0 = sub * f.S;
+        const uint32_t count = row0 < f.n ? min(f.S, f.n - row0) : 0u;
+        BitReader br;
+        br.init(reinterpret_cast<const uint32_t*>(stage), base + start);
+        float acc = 0.0f;
+        if (kMode == 0) {
+            if (kXShared) {
+                const float* xl = xs + row0 + pad * sub;
+                for (uint32_t s = 0; s < count; ++s) {
+                    const uint32_t r = decode_symbol(br, t, lut_shift, f.lut_bits, f.max_len);
+                    acc = fmaf(xl[s], t.value[r], acc);
+                }
+            } else {
+                const float* xl = x + (int64_t)row0 * xs_i;
+                for (uint32_t s = 0; s < count; ++s) {
+                    const uint32_t r = decode_symbol(br, t, lut_shift, f.lut_bits, f.max_len);
+                    acc = fmaf(xl[(int64_t)s * xs_i], t.value[r], acc);
+                }
+            }
+            acc = warp_sum(acc);
+            if (lane == 0) {
+                if (f.G == 1) y[(int64_t)j * ys_j] = acc;
+                else aux[u] = acc;
+            }
+        } else {
+            float* out = aux + (size_t)j * f.n + row0;
+            for (uint32_t s = 0; s < count; ++s) {
+                const uint32_t r = decode_symbol(br, t, lut_shift, f.lut_bits, f.max_len);
+                out[s] = t.value[r];
+            }
+        }
+        __syncwarp();
+    }
+}
+
+// ------------------------------------------------------------------------------------------------
+// sHAC, one input vector (Algorithm 2 by segments): as above over the stored entries of a column,
+// with the row of each entry read from ri and x gathered from shared memory.
+// ------------------------------------------------------------------------------------------------
+template <int kMode, bool kXShared, typename RowT>
+__global__ void __launch_bounds__(1024) shac_vec_kernel(DevFormat f, const float* __restrict__ x, int64_t xs_i,
+                                                        float* __restrict__ y, int64_t ys_j,
+                                                        float* __restrict__ aux) {
+    extern __shared__ __align__(16) unsigned char smem[];
+    unsigned char* p = smem;
+    const SmemTables t = stage_tables(f, p);
+    float* xs = reinterpret_cast<float*>(p);
+    if (kMode == 0 && kXShared) {
+        for (uint32_t i = threadIdx.x; i < f.n; i += blockDim.x) xs[i] = x[(int64_t)i * xs_i];
+        p += align16((size_t)f.n * 4);
+    }
+    const uint32_t warp = threadIdx.x >> 5, lane = threadIdx.x & 31, warps = blockDim.x >> 5;
+    uint4* stage = reinterpret_cast<uint4*>(p) + (size_t)warp * f.max_unit_chunks;
+    __syncthreads();
+    const uint32_t lut_shift = 32 - f.lut_bits;
+    const RowT* __restrict__ ri = reinterpret_cast<const RowT*>(f.ri);
+
+    for (uint32_t u = blockIdx.x * warps + warp; u < f.units; u += gridDim.x * warps) {
+        const uint32_t j = f.seg_col[u];
+        const uint32_t first = f.seg_first[j];
+        const uint32_t g = u - first;
+        const uint32_t col_end = f.cb[j + 1];
+        const uint32_t my_bits = f.sub_bits[(size_t)u * 32 + lane];
+        uint32_t total;
+        const uint32_t start = lane_start_bits(my_bits, lane, total);
+        const uint32_t base = stage_span(f, f.seg_bit_off[u], total, stage, lane);
+        const uint32_t pos0 = f.cb[j] + (g * 32 + lane) * f.S;
+        const uint32_t count = pos0 < col_end ? min(f.S, col_end - pos0) : 0u;
+        BitReader br;
+        br.init(reinterpret_cast<const uint32_t*>(stage), base + start);
+        if (kMode == 0) {
+            float acc = 0.0f;
+            for (uint32_t s = 0; s < count; ++s) {
+                const uint32_t r = decode_symbol(br, t, lut_shift, f.lut_bits, f.max_len);
+                const uint32_t row = ri[pos0 + s];
+                const float xv = kXShared ? xs[row] : x[(int64_t)row * xs_i];
+                acc = fmaf(xv, t.value[r], acc);
+            }
+            acc = warp_sum(acc);
+            if (lane == 0) {
+                const bool single = (f.seg_first[j + 1] - first) == 1;
+                if (single) y[(int64_t)j * ys_j] = acc;
+                else aux[u] = acc;
+            }
+        } else {
+            for (uint32_t s = 0; s < count; ++s) {
+                const uint32_t r = decode_symbol(br, t, lut_shift, f.lut_bits, f.max_len);
+                aux[pos0 + s] = t.value[r];
+            }
+        }
+        __syncwarp();
+    }
+}
+
+// Columns made of several segments (or none): add the per-segment partials in segment order.
+//   partial[u*batch + b]; HAC: segments j*G .. j*G+G-1; sHAC: seg_first[j] .. seg_first[j+1]-1.
+// Columns with exactly one segment were written by the product kernel itself.
+__global__ void finalize_kernel(DevFormat f, bool sparse, const float* __restrict__ partial, uint32_t batch,
+                                float* __restrict__ y, int64_t ys_j, int64_t ys_b) {
+    const uint64_t idx = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (idx >= (uint64_t)f.m * batch) return;
+    const uint32_t j = (uint32_t)(idx / batch), b = (uint32_t)(idx % batch);
+    uint32_t u0, u1;
+    if (sparse) { u0 = f.seg_first[j]; u1 = f.seg_first[j + 1]; }
+    else { u0 = j * f.G; u1 = u0 + f.G; }
+    if (u1 - u0 == 1) return;
+    float s = 0.0f;
+    for (uint32_t u = u0; u < u1; ++u) s += partial[(size_t)u * batch + b];
+    y[(int64_t)j * ys_j + (int64_t)b * ys_b] = s;
+}
+
+// ------------------------------------------------------------------------------------------------
+// HAC, batch of inputs (Algorithm 3 without re-decoding W per input).  A block owns `kCols`
+// consecutive columns (one per warp) over the rows of one segment index g.  It alternates between
+// a decode phase (every lane decodes kSteps symbols of its sub-segment into a shared tile of
+// weights) and a product phase (the tile is applied to the matching rows of X, staged in shared
+// memory, for a tile of up to 32*kAcc inputs held in registers), so the stream is decoded once per
+// batch tile and never written to global memory.
+// ------------------------------------------------------------------------------------------------
+constexpr int kBatchSteps = 4;          // symbols decoded per lane per phase
+constexpr int kBatchRows = 32 * kBatchSteps;
+constexpr int kAccMax = 4;              // batch tile = 32 * kAcc inputs
+
+template <int kAcc>
+__global__ void __launch_bounds__(1024) hac_batch_kernel(DevFormat f, const float* __restrict__ x, int64_t xs_i,
+                                                         int64_t xs_b, uint32_t batch, float* __restrict__ y,
+                                                         int64_t ys_j, int64_t ys_b, float* __restrict__ partial,
+                                                         uint32_t col_blocks) {
+    extern __shared__ __align__(16) unsigned char smem[];
+    unsigned char* p = smem;
+    const SmemTables t = stage_tables(f, p);
+    const uint32_t warp = threadIdx.x >> 5, lane = threadIdx.x & 31, warps = blockDim.x >> 5;
+    constexpr uint32_t kTile = 32 * kAcc;
+    float* wt = reinterpret_cast<float*>(p);                       // [warps][kBatchRows]
+    p += align16((size_t)warps * kBatchRows * 4);
+    float* xt = reinterpret_cast<float*>(p);                       // [kBatchRows][kTile]
+    p += align16((size_t)kBatchRows * kTile * 4);
+    uint4* stage = reinterpret_cast<uint4*>(p) + (size_t)warp * f.max_unit_chunks;
+    __syncthreads();
+    const uint32_t lut_shift = 32 - f.lut_bits;
+    const uint32_t batch_tiles = (batch + kTile - 1) / kTile;
+    const uint32_t items = col_blocks * f.G * batch_tiles;
+
+    for (uint32_t item = blockIdx.x; item < items; item += gridDim.x) {
+        const uint32_t bt = item % batch_tiles;
+        const uint32_t rest = item / batch_tiles;
+        const uint32_t g = rest % f.G, cblk = rest / f.G;
+        const uint32_t j = cblk * warps + warp;
+        const bool live = j < f.m;
+        const uint32_t u = live ? j * f.G + g : 0u;
+        const uint32_t b0 = bt * kTile;
+        const uint32_t sub = g * 32 + lane;
+        const uint32_t row0 = sub * f.S;
+        uint32_t count = 0;
+        BitReader br;
+        br.words = reinterpret_cast<const uint32_t*>(stage); br.next = 0; br.buf = 0; br.avail = 64;
+        if (live) {
+            const uint32_t my_bits = f.sub_bits[(size_t)u * 32 + lane];
+            uint32_t total;
+            const uint32_t start = lane_start_bits(my_bits, lane, total);
+            const uint32_t base = stage_span(f, f.seg_bit_off[u], total, stage, lane);
+            count = row0 < f.n ? min(f.S, f.n - row0) : 0u;
+            br.init(reinterpret_cast<const uint32_t*>(stage), base + start);
+        }
+        float acc[kAcc];
+#pragma unroll
+        for (int a = 0; a < kAcc; ++a) acc[a] = 0.0f;
+        const uint32_t seg_rows = min(f.S, f.n - min(f.n, g * 32 * f.S));   // longest sub-segment here
+        for (uint32_t s0 = 0; s0 < seg_rows; s0 += kBatchSteps) {
+            // decode phase: kBatchSteps symbols per lane -> wt[warp][lane*kBatchSteps + s]
+#pragma unroll
+            for (int s = 0; s < kBatchSteps; ++s) {
+                float v = 0.0f;
+                if (s0 + s < count) v = t.value[decode_symbol(br, t, lut_shift, f.lut_bits, f.max_len)];
+                wt[warp * kBatchRows + lane * kBatchSteps + s] = v;
+            }
+            // matching rows of X: tile row r = l*kBatchSteps + s  <->  matrix row (g*32+l)*S + s0 + s
+            for (uint32_t idx = threadIdx.x; idx < kBatchRows * kTile; idx += blockDim.x) {
+                const uint32_t r = idx / kTile, bb = idx - r * kTile;
+                const uint32_t l = r / kBatchSteps, s = r - l * kBatchSteps;
+                const uint32_t row = (g * 32 + l) * f.S + s0 + s;
+                const uint32_t b = b0 + bb;
+                float v = 0.0f;
+                if (s0 + s < f.S && row < f.n && b < batch) v = x[(int64_t)row * xs_i + (int64_t)b * xs_b];
+                xt[idx] = v;
+            }
+            __syncthreads();
+            // product phase: this warp's column against the tile, lanes over inputs
+            const float* w = wt + warp * kBatchRows;
+#pragma unroll 4
+            for (uint32_t r = 0; r < kBatchRows; ++r) {
+                const float wv = w[r];
+#pragma unroll
+                for (int a = 0; a < kAcc; ++a) acc[a] = fmaf(wv, xt[r * kTile + a * 32 + lane], acc[a]);
+            }
+            __syncthreads();
+        }
+        if (live) {
+#pragma unroll
+            for (int a = 0; a < kAcc; ++a) {
+                const uint32_t b = b0 + a * 32 + lane;
+                if (b < batch) {
+                    if (f.G == 1) y[(int64_t)j * ys_j + (int64_t)b * ys_b] = acc[a];
+                    else partial[(size_t)u * batch + b] = acc[a];
+                }
+            }
+        }
+    }
+}
+
+// ------------------------------------------------------------------------------------------------
+// sHAC, batch of inputs.  One warp per segment: lanes decode kBatchSteps entries each into a small
+// shared tile of (value, row) pairs, then the warp walks the tile with lanes spread over the
+// inputs, gathering the rows of X (stored [n][batch] for coalesced access).
+// ------------------------------------------------------------------------------------------------
+template <int kAcc, typename RowT>
+__global__ void __launch_bounds__(1024) shac_batch_kernel(DevFormat f, const float* __restrict__ x, int64_t xs_i,
+                                                          int64_t xs_b, uint32_t batch, float* __restrict__ y,
+                                                          int64_t ys_j, int64_t ys_b,
+                                                          float* __restrict__ partial) {
+    extern __shared__ __align__(16) unsigned char smem[];
+    unsigned char* p = smem;
+    const SmemTables t = stage_tables(f, p);
+    const uint32_t warp = threadIdx.x >> 5, lane = threadIdx.x & 31, warps = blockDim.x >> 5;
+    constexpr uint32_t kTile = 32 * kAcc;
+    float* wv_all = reinterpret_cast<float*>(p);
+    p += align16((size_t)warps * kBatchRows * 4);
+    uint32_t* wr_all = reinterpret_cast<uint32_t*>(p);
+    p += align16((size_t)warps * kBatchRows * 4);
+    uint4* stage = reinterpret_cast<uint4*>(p) + (size_t)warp * f.max_unit_chunks;
+    float* wv = wv_all + warp * kBatchRows;
+    uint32_t* wr = wr_all + warp * kBatchRows;
+    __syncthreads();
+    const uint32_t lut_shift = 32 - f.lut_bits;
+    const RowT* __restrict__ ri = reinterpret_cast<const RowT*>(f.ri);
+    const uint32_t batch_tiles = (batch + kTile - 1) / kTile;
+    const uint64_t items = (uint64_t)f.units * batch_tiles;
+
+    for (uint64_t item = (uint64_t)blockIdx.x * warps + warp; item < items; item += (uint64_t)gridDim.x * warps) {
+        const uint32_t u = (uint32_t)(item / batch_tiles);
+        const uint32_t b0 = (uint32_t)(item % batch_tiles) * kTile;
+        const uint32_t j = f.seg_col[u];
+        const uint32_t first = f.seg_first[j];
+        const uint32_t g = u - first;
+        const uint32_t col_end = f.cb[j + 1];
+        const uint32_t my_bits = f.sub_bits[(size_t)u * 32 + lane];
+        uint32_t total;
+        const uint32_t start = lane_start_bits(my_bits, lane, total);
+        const uint32_t base = stage_span(f, f.seg_bit_off[u], total, stage, lane);
+        const uint32_t seg_pos0 = f.cb[j] + g * 32 * f.S;
+        const uint32_t pos0 = seg_pos0 + lane * f.S;
+        const uint32_t count = pos0 < col_end ? min(f.S, col_end - pos0) : 0u;
+        const uint32_t seg_rows = min(f.S, col_end - seg_pos0);
+        BitReader br;
+        br.init(reinterpret_cast<const uint32_t*>(stage), base + start);
+        float acc[kAcc];
+#pragma unroll
+        for (int a = 0; a < kAcc; ++a) acc[a] = 0.0f;
+        for (uint32_t s0 = 0; s0 < seg_rows; s0 += kBatchSteps) {
+#pragma unroll
+            for (int s = 0; s < kBatchSteps; ++s) {
+                float v = 0.0f;
+                uint32_t row = 0;
+                if (s0 + s < count) {
+                    v = t.value[decode_symbol(br, t, lut_shift, f.lut_bits, f.max_len)];
+                    row = ri[pos0 + s0 + s];
+                }
+                wv[lane * kBatchSteps + s] = v;
+                wr[lane * kBatchSteps + s] = row;
+            }
+            __syncwarp();
+#pragma unroll 4
+            for (uint32_t r = 0; r < kBatchRows; ++r) {
+                const float v = wv[r];
+                const float* xr = x + (int64_t)wr[r] * xs_i;
+#pragma unroll
+                for (int a = 0; a < kAcc; ++a) {
+                    const uint32_t b = b0 + a * 32 + lane;
+                    if (b < batch) acc[a] = fmaf(v, xr[(int64_t)b * xs_b], acc[a]);
+                }
+            }
+            __syncwarp();
+        }
+        const bool single = (f.seg_first[j + 1] - first) == 1;
+#pragma unroll
+        for (int a = 0; a < kAcc; ++a) {
+            const uint32_t b = b0 + a * 32 + lane;
+            if (b < batch) {
+                if (single) y[(int64_t)j * ys_j + (int64_t)b * ys_b] = acc[a];
+                else partial[(size_t)u * batch + b] = acc[a];
+            }
+        }
+    }
+}
+
+// X[batch][n] -> Xt[n][batch] (host-input path only).
+__global__ void transpose_kernel(const float* __restrict__ in, float* __restrict__ out, uint32_t rows,
+                                 uint32_t cols) {
+    __shared__ float tile[32][33];
+    const uint32_t c0 = blockIdx.x * 32, r0 = blockIdx.y * 32;
+    for (uint32_t r = threadIdx.y; r < 32; r += blockDim.y)
+        if (r0 + r < rows && c0 + threadIdx.x < cols) tile[r][threadIdx.x] = in[(size_t)(r0 + r) * cols + c0 + threadIdx.x];
+    __syncthreads();
+    for (uint32_t c = threadIdx.y; c < 32; c += blockDim.y)
+        if (c0 + c < cols && r0 + threadIdx.x < rows) out[(size_t)(c0 + c) * rows + r0 + threadIdx.x] = tile[threadIdx.x][c];
+}
+
+// ------------------------------------------------------------------------------------------------
+// Host side
+// ------------------------------------------------------------------------------------------------
+struct DeviceInfo {
+    int sms = 0;
+    int max_smem_optin = 0;
+    bool ok = false;
+};
+
+static int device_info(DeviceInfo& d) {
+    static thread_local DeviceInfo cache[64];
+    int dev = 0;
+    HAC_CUDA(cudaGetDevice(&dev));
+    if (dev >= 0 && dev < 64 && cache[dev].ok) { d = cache[dev]; return HAC_OK; }
+    HAC_CUDA(cudaDeviceGetAttribute(&d.sms, cudaDevAttrMultiProcessorCount, dev));
+    HAC_CUDA(cudaDeviceGetAttribute(&d.max_smem_optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev));
+    d.ok = true;
+    if (dev >= 0 && dev < 64) cache[dev] = d;
+    return HAC_OK;
+}
+
+static DevFormat dev_format(const Format& f) {
+    DevFormat d{};
+    d.stream = f.dev.stream; d.lut = f.dev.lut; d.rank_value = f.dev.rank_value;
+    d.limit = f.dev.limit; d.first_left = f.dev.first_left; d.rank_base = f.dev.rank_base;
+    d.seg_bit_off = f.dev.seg_bit_off; d.sub_bits = f.dev.sub_bits; d.seg_col = f.dev.seg_col;
+    d.seg_first = f.dev.seg_first; d.ri = f.dev.ri; d.cb = f.dev.cb;
+    d.n = (uint32_t)f.n; d.m = (uint32_t)f.m; d.units = (uint32_t)f.seg_bit_off.size();
+    d.G = f.G ? f.G : 1; d.S = f.S; d.k_eff = (uint32_t)f.codebook.size();
+    d.lut_bits = (uint32_t)f.tables.lut_bits; d.max_len = f.max_len; d.ri_bits = f.ri_bits;
+    d.max_unit_chunks = f.max_unit_chunks;
+    return d;
+}
+
+static void set_pointers(Format& f, void* dev_buf, size_t bytes) {
+    const ImageLayout L = image_layout(f);
+    unsigned char* b = static_cast<unsigned char*>(dev_buf);
+    f.dev.base = dev_buf; f.dev.bytes = bytes;
+    f.dev.stream = reinterpret_cast<const uint32_t*>(b + L.stream);
+    f.dev.lut = reinterpret_cast<const uint16_t*>(b + L.lut);
+    f.dev.rank_value = reinterpret_cast<const float*>(b + L.rank_value);
+    f.dev.limit = reinterpret_cast<const uint64_t*>(b + L.limit);
+    f.dev.first_left = reinterpret_cast<const uint32_t*>(b + L.first_left);
+    f.dev.rank_base = reinterpret_cast<const uint32_t*>(b + L.rank_base);
+    f.dev.seg_bit_off = reinterpret_cast<const uint64_t*>(b + L.seg_bit_off);
+    f.dev.sub_bits = reinterpret_cast<const uint16_t*>(b + L.sub_bits);
+    f.dev.seg_col = reinterpret_cast<const uint32_t*>(b + L.seg_col);
+    f.dev.seg_first = reinterpret_cast<const uint32_t*>(b + L.seg_first);
+    f.dev.ri = b + L.ri;
+    f.dev.cb = reinterpret_cast<const uint32_t*>(b + L.cb);
+}
+
+static int upload(Format& f, void* dev_buf, size_t dev_bytes, void* stream_) {
+    if (!dev_buf || (reinterpret_cast<uintptr_t>(dev_buf) & 255u)) return HAC_ERR_INVALID_ARG;
+    const ImageLayout L = image_layout(f);
+    if (dev_bytes < L.total) return HAC_ERR_BUFFER_TOO_SMALL;
+    cudaStream_t st = static_cast<cudaStream_t>(stream_);
+    unsigned char* b = static_cast<unsigned char*>(dev_buf);
+    auto put = [&](size_t off, const void* src, size_t bytes) -> cudaError_t {
+        if (bytes == 0) return cudaSuccess;
+        return cudaMemcpyAsync(b + off, src, bytes, cudaMemcpyHostToDevice, st);
+    };
+    HAC_CUDA(cudaMemsetAsync(dev_buf, 0, L.total, st));
+    HAC_CUDA(put(L.stream, f.stream.data(), f.stream.size() * 4));
+    HAC_CUDA(put(L.lut, f.tables.lut.data(), f.tables.lut.size() * 2));
+    HAC_CUDA(put(L.rank_value, f.tables.rank_value.data(), f.tables.rank_value.size() * 4));
+    HAC_CUDA(put(L.limit, f.tables.limit, sizeof(f.tables.limit)));
+    HAC_CUDA(put(L.first_left, f.tables.first_left, sizeof(f.tables.first_left)));
+    HAC_CUDA(put(L.rank_base, f.tables.rank_base, sizeof(f.tables.rank_base)));
+    HAC_CUDA(put(L.seg_bit_off, f.seg_bit_off.data(), f.seg_bit_off.size() * 8));
+    HAC_CUDA(put(L.sub_bits, f.sub_bits.data(), f.sub_bits.size() * 2));
+    HAC_CUDA(put(L.seg_col, f.seg_col.data(), f.seg_col.size() * 4));
+    HAC_CUDA(put(L.seg_first, f.seg_first.data(), f.seg_first.size() * 4));
+    if (f.ri_bits == 16) HAC_CUDA(put(L.ri, f.ri16.data(), f.ri16.size() * 2));
+    else HAC_CUDA(put(L.ri, f.ri32.data(), f.ri32.size() * 4));
+    HAC_CUDA(put(L.cb, f.cb.data(), f.cb.size() * 4));
+    // the source vectors are pageable host memory: wait so they may change or go away afterwards
+    HAC_CUDA(cudaStreamSynchronize(st));
+    set_pointers(f, dev_buf, dev_bytes);
+    return HAC_OK;
+}
+
+static int attach(Format& f, void* dev_buf, size_t dev_bytes) {
+    if (!dev_buf || (reinterpret_cast<uintptr_t>(dev_buf) & 255u)) return HAC_ERR_INVALID_ARG;
+    if (dev_bytes < image_layout(f).total) return HAC_ERR_BUFFER_TOO_SMALL;
+    set_pointers(f, dev_buf, dev_bytes);
+    return HAC_OK;
+}
+
+static bool needs_finalize(const Format& f) {
+    if (!f.sparse) return f.G > 1;
+    return f.max_units_per_col > 1 || f.has_empty_col;
+}
+
+static size_t workspace_bytes(const Format& f, int64_t batch) {
+    const bool partials = f.sparse ? f.max_units_per_col > 1 : f.G > 1;
+    return partials ? f.seg_bit_off.size() * (size_t)batch * 4 : 0;
+}
+
+static int env_int(const char* name, int fallback) {
+    const char* v = std::getenv(name);
+    return v && *v ? std::atoi(v) : fallback;
+}
+
+template <typename K>
+static int prepare_kernel(K kernel, size_t smem) {
+    if (smem > 48 * 1024) HAC_CUDA(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+    return HAC_OK;
+}
+
+// Largest number of warps per block (a multiple of `step`, at most `want`) whose shared memory
+// fits; 0 if not even `step` warps fit.
+static int fit_warps(size_t fixed, size_t per_warp, int want, int step, size_t budget) {
+    for (int w = want; w >= step; w -= step)
+        if (fixed + per_warp * (size_t)w <= budget) return w;
+    return 0;
+}
+
+static int launch_finalize(const Format& f, const DevFormat& d, const float* partial, int64_t batch, float* y,
+                           int64_t ys_j, int64_t ys_b, cudaStream_t st) {
+    const uint64_t total = (uint64_t)f.m * (uint64_t)batch;
+    const unsigned blocks = (unsigned)((total + 255) / 256);
+    finalize_kernel<<<blocks, 256, 0, st>>>(d, f.sparse, partial, (uint32_t)batch, y, ys_j, ys_b);
+    HAC_CUDA(cudaGetLastError());
+    f.last_launches++;
+    return HAC_OK;
+}
+
+// mode 0: product with one input; mode 1: debug decode into `aux`.
+static int launch_vec(const Format& f, int mode, const float* x, int64_t xs_i, float* y, int64_t ys_j,
+                      float* aux, cudaStream_t st) {
+    DeviceInfo di;
+    int rc = device_info(di);
+    if (rc) return rc;
+    const DevFormat d = dev_format(f);
+    if (d.units == 0) return HAC_OK;
+    const size_t budget = (size_t)di.max_smem_optin;
+    const size_t tab = tables_smem_bytes(d.lut_bits, d.k_eff);
+    const size_t per_warp = (size_t)d.max_unit_chunks * 16;
+    size_t xbytes = 0;
+    if (mode == 0) xbytes = f.sparse ? align16((size_t)f.n * 4) : align16(((size_t)f.n + (f.n / f.S + 1)) * 4);
+    const int want = std::min(32, std::max(1, env_int("HAC_B200_VEC_WARPS", 16)));
+    bool x_shared = mode == 0;
+    int warps = fit_warps(tab + xbytes, per_warp, want, 1, budget);
+    if (mode == 0 && warps < std::min(want, 4)) {        // x does not fit next to enough warps
+        x_shared = false;
+        xbytes = 0;
+        warps = fit_warps(tab, per_warp, want, 1, budget);
+    }
+    if (warps == 0) return HAC_ERR_BUFFER_TOO_SMALL;
+    const size_t smem = tab + xbytes + per_warp * warps;
+    const int threads = warps * 32;
+    int per_sm = 1;
+    void (*kernel)(DevFormat, const float*, int64_t, float*, int64_t, float*) = nullptr;
+    if (!f.sparse) {
+        kernel = mode == 1 ? hac_vec_kernel<1, false> : (x_shared ? hac_vec_kernel<0, true> : hac_vec_kernel<0, false>);
+    } else if (f.ri_bits == 16) {
+        kernel = mode == 1 ? shac_vec_kernel<1, false, uint16_t>
+                           : (x_shared ? shac_vec_kernel<0, true, uint16_t> : shac_vec_kernel<0, false, uint16_t>);
+    } else {
+        kernel = mode == 1 ? shac_vec_kernel<1, false, uint32_t>
+                           : (x_shared ? shac_vec_kernel<0, true, uint32_t> : shac_vec_kernel<0, false, uint32_t>);
+    }
+    rc = prepare_kernel(kernel, smem);
+    if (rc) return rc;
+    HAC_CUDA(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kernel, threads, smem));
+    per_sm = std::max(per_sm, 1);
+    const unsigned need = (d.units + warps - 1) / warps;
+    const unsigned grid = std::min<unsigned>(need, (unsigned)(di.sms * per_sm));
+    kernel<<<grid, threads, smem, st>>>(d, x, xs_i, y, ys_j, aux);
+    HAC_CUDA(cudaGetLastError());
+    f.last_launches++;
+    return HAC_OK;
+}
+
+template <int kAcc>
+static int launch_batch_t(const Format& f, const DeviceInfo& di, const DevFormat& d, const float* x, int64_t xs_i,
+                          int64_t xs_b, int64_t batch, float* y, int64_t ys_j, int64_t ys_b, float* partial,
+                          cudaStream_t st) {
+    const size_t budget = (size_t)di.max_smem_optin;
+    const size_t tab = tables_smem_bytes(d.lut_bits, d.k_eff);
+    constexpr uint32_t kTile = 32 * kAcc;
+    const uint32_t batch_tiles = (uint32_t)((batch + kTile - 1) / kTile);
+    int rc;
+    if (!f.sparse) {
+        const size_t fixed = tab + align16((size_t)kBatchRows * kTile * 4) + 16;
+        const size_t per_warp = (size_t)d.max_unit_chunks * 16 + kBatchRows * 4;
+        const int want = std::min(32, std::max(1, env_int("HAC_B200_BATCH_WARPS", 16)));
+        const int warps = fit_warps(fixed, per_warp, want, 1, budget);
+        if (warps == 0) return HAC_ERR_BUFFER_TOO_SMALL;
+        const size_t smem = fixed + per_warp * warps;
+        auto kernel = hac_batch_kernel<kAcc>;
+        rc = prepare_kernel(kernel, smem);
+        if (rc) return rc;
+        int per_sm = 1;
+        HAC_CUDA(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kernel, warps * 32, smem));
+        per_sm = std::max(per_sm, 1);
+        const uint32_t col_blocks = (uint32_t)((f.m + warps - 1) / warps);
+        const uint64_t items = (uint64_t)col_blocks * d.G * batch_tiles;
+        const unsigned grid = (unsigned)std::min<uint64_t>(items, (uint64_t)di.sms * per_sm);
+        kernel<<<grid, warps * 32, smem, st>>>(d, x, xs_i, xs_b, (uint32_t)batch, y, ys_j, ys_b, partial, col_blocks);
+    } else {
+        const size_t per_warp = (size_t)d.max_unit_chunks * 16 + 2 * kBatchRows * 4;
+        const int want = std::min(32, std::max(1, env_int("HAC_B200_BATCH_WARPS", 8)));
+        const int warps = fit_warps(tab + 32, per_warp, want, 1, budget);
+        if (warps == 0) return HAC_ERR_BUFFER_TOO_SMALL;
+        const size_t smem = tab + 32 + per_warp * warps;
+        void (*kernel)(DevFormat, const float*, int64_t, int64_t, uint32_t, float*, int64_t, int64_t, float*) =
+            f.ri_bits == 16 ? shac_batch_kernel<kAcc, uint16_t> : shac_batch_kernel<kAcc, uint32_t>;
+        rc = prepare_kernel(kernel, smem);
+        if (rc) return rc;
+        int per_sm = 1;
+        HAC_CUDA(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kernel, warps * 32, smem));
+        per_sm = std::max(per_sm, 1);
+        const uint64_t items = (uint64_t)d.units * batch_tiles;
+        const unsigned grid = (unsigned)std::min<uint64_t>((items + warps - 1) / warps, (uint64_t)di.sms * per_sm);
+        kernel<<<grid, warps * 32, smem, st>>>(d, x, xs_i, xs_b, (uint32_t)batch, y, ys_j, ys_b, partial);
+    }
+    HAC_CUDA(cudaGetLastError());
+    f.last_launches++;
+    return HAC_OK;
+}
+
+static int dot(const Format& f, const float* x, int64_t batch, int64_t xs_i, int64_t xs_b, float* y,
+               int64_t ys_j, int64_t ys_b, void* workspace, size_t workspace_bytes_given, void* stream_) {
+    if (!f.dev.base) return HAC_ERR_NOT_UPLOADED;
+    if (!x || !y || batch < 1 || batch > ((int64_t)1 << 24)) return HAC_ERR_INVALID_ARG;
+    const size_t need = workspace_bytes(f, batch);
+    if (need > 0 && (!workspace || workspace_bytes_given < need)) return HAC_ERR_BUFFER_TOO_SMALL;
+    cudaStream_t st = static_cast<cudaStream_t>(stream_);
+    f.last_launches = 0;
+    float* partial = static_cast<float*>(workspace);
+    const DevFormat d = dev_format(f);
+    int rc = HAC_OK;
+    if (d.units > 0) {
+        if (batch == 1) {
+            rc = launch_vec(f, 0, x, xs_i, y, ys_j, partial, st);
+        } else {
+            DeviceInfo di;
+            rc = device_info(di);
+            if (rc) return rc;
+            const int acc = (int)std::min<int64_t>(kAccMax, (batch + 31) / 32);
+            switch (acc) {
+                case 1: rc = launch_batch_t<1>(f, di, d, x, xs_i, xs_b, batch, y, ys_j, ys_b, partial, st); break;
+                case 2: rc = launch_batch_t<2>(f, di, d, x, xs_i, xs_b, batch, y, ys_j, ys_b, partial, st); break;
+                case 3: rc = launch_batch_t<3>(f, di, d, x, xs_i, xs_b, batch, y, ys_j, ys_b, partial, st); break;
+                default: rc = launch_batch_t<4>(f, di, d, x, xs_i, xs_b, batch, y, ys_j, ys_b, partial, st); break;
+            }
+        }
+        if (rc) return rc;
+    }
+    if (needs_finalize(f) || d.units == 0) rc = launch_finalize(f, d, partial, batch, y, ys_j, ys_b, st);
+    return rc;
+}
+
+static size_t host_scratch_bytes(const Format& f, int64_t batch) {
+    const size_t xb = align16((size_t)batch * f.n * 4 + 240) ;
+    const size_t yb = align16((size_t)batch * f.m * 4 + 240);
+    const size_t extra = batch > 1 ? xb : 0;               // transposed copy of X
+    return xb + extra + yb + align16(workspace_bytes(f, batch)) + 1024;
+}
+
+static int dot_host(const Format& f, const float* X, int64_t batch, float* Y, void* scratch, size_t scratch_bytes,
+                    void* stream_) {
+    if (!f.dev.base) return HAC_ERR_NOT_UPLOADED;
+    if (!X || !Y || !scratch || batch < 1) return HAC_ERR_INVALID_ARG;
+    if (scratch_bytes < host_scratch_bytes(f, batch)) return HAC_ERR_BUFFER_TOO_SMALL;
+    cudaStream_t st = static_cast<cudaStream_t>(stream_);
+    auto up = [](size_t v) { return (v + 255) & ~(size_t)255; };
+    unsigned char* b = static_cast<unsigned char*>(scratch);
+    b = reinterpret_cast<unsigned char*>(up(reinterpret_cast<uintptr_t>(b)));
+    float* xd = reinterpret_cast<float*>(b);
+    b += up((size_t)batch * f.n * 4);
+    float* xt = xd;
+    if (batch > 1) { xt = reinterpret_cast<float*>(b); b += up((size_t)batch * f.n * 4); }
+    float* yd = reinterpret_cast<float*>(b);
+    b += up((size_t)batch * f.m * 4);
+    void* ws = b;
+    HAC_CUDA(cudaMemcpyAsync(xd, X, (size_t)batch * f.n * 4, cudaMemcpyHostToDevice, st));
+    int extra = 0;
+    int rc;
+    if (batch > 1) {
+        dim3 grid((unsigned)((f.n + 31) / 32), (unsigned)((batch + 31) / 32));
+        transpose_kernel<<<grid, dim3(32, 8), 0, st>>>(xd, xt, (uint32_t)batch, (uint32_t)f.n);
+        HAC_CUDA(cudaGetLastError());
+        extra = 1;
+        rc = dot(f, xt, batch, batch, 1, yd, 1, f.m, ws, workspace_bytes(f, batch), stream_);
+    } else {
+        rc = dot(f, xd, 1, 1, f.n, yd, 1, f.m, ws, workspace_bytes(f, batch), stream_);
+    }
+    if (rc) return rc;
+    f.last_launches += extra;
+    HAC_CUDA(cudaMemcpyAsync(Y, yd, (size_t)batch * f.m * 4, cudaMemcpyDeviceToHost, st));
+    HAC_CUDA(cudaStreamSynchronize(st));
+    return HAC_OK;
+}
+
+static int debug_decode(const Format& f, float* out, void* stream_) {
+    if (!f.dev.base) return HAC_ERR_NOT_UPLOADED;
+    if (!out) return HAC_ERR_INVALID_ARG;
+    f.last_launches = 0;
+    return launch_vec(f, 1, nullptr, 0, nullptr, 0, out, static_cast<cudaStream_t>(stream_));
+}
+
+}  // namespace hacb200
+
+using namespace hacb200;
+
+extern "C" {
+
+int hac_device_bytes(const hac_format* f, size_t* out) {
+    if (!f || !out) return HAC_ERR_INVALID_ARG;
+    *out = image_layout(f->f).total;
+    return HAC_OK;
+}
+int shac_device_bytes(const shac_format* f, size_t* out) {
+    if (!f || !out) return HAC_ERR_INVALID_ARG;
+    *out = image_layout(f->f).total;
+    return HAC_OK;
+}
+int hac_upload(hac_format* f, void* dev_buf, size_t dev_bytes, void* cuda_stream) {
+    return f ? upload(f->f, dev_buf, dev_bytes, cuda_stream) : HAC_ERR_INVALID_ARG;
+}
+int shac_upload(shac_format* f, void* dev_buf, size_t dev_bytes, void* cuda_stream) {
+    return f ? upload(f->f, dev_buf, dev_bytes, cuda_stream) : HAC_ERR_INVALID_ARG;
+}
+int hac_attach(hac_format* f, void* dev_buf, size_t dev_bytes) {
+    return f ? attach(f->f, dev_buf, dev_bytes) : HAC_ERR_INVALID_ARG;
+}
+int shac_attach(shac_format* f, void* dev_buf, size_t dev_bytes) {
+    return f ? attach(f->f, dev_buf, dev_bytes) : HAC_ERR_INVALID_ARG;
+}
+
+int hac_workspace_bytes(const hac_format* f, int64_t batch, size_t* out) {
+    if (!f || !out || batch < 1) return HAC_ERR_INVALID_ARG;
+    *out = workspace_bytes(f->f, batch);
+    return HAC_OK;
+}
+int shac_workspace_bytes(const shac_format* f, int64_t batch, size_t* out) {
+    if (!f || !out || batch < 1) return HAC_ERR_INVALID_ARG;
+    *out = workspace_bytes(f->f, batch);
+    return HAC_OK;
+}
+
+int hac_dot(const hac_format* f, const float* x, int64_t batch, int64_t x_stride_i, int64_t x_stride_b, float* y,
+            int64_t y_stride_j, int64_t y_stride_b, void* workspace, size_t workspace_bytes_, void* cuda_stream) {
+    if (!f) return HAC_ERR_INVALID_ARG;
+    return dot(f->f, x, batch, x_stride_i, x_stride_b, y, y_stride_j, y_stride_b, workspace, workspace_bytes_,
+               cuda_stream);
+}
+int shac_dot(const shac_format* f, const float* x, int64_t batch, int64_t x_stride_i, int64_t x_stride_b, float* y,
+             int64_t y_stride_j, int64_t y_stride_b, void* workspace, size_t workspace_bytes_, void* cuda_stream) {
+    if (!f) return HAC_ERR_INVALID_ARG;
+    return dot(f->f, x, batch, x_stride_i, x_stride_b, y, y_stride_j, y_stride_b, workspace, workspace_bytes_,
+               cuda_stream);
+}
+
+int hac_dot_host_scratch_bytes(const hac_format* f, int64_t batch, size_t* out) {
+    if (!f || !out || batch < 1) return HAC_ERR_INVALID_ARG;
+    *out = host_scratch_bytes(f->f, batch);
+    return HAC_OK;
+}
+int shac_dot_host_scratch_bytes(const shac_format* f, int64_t batch, size_t* out) {
+    if (!f || !out || batch < 1) return HAC_ERR_INVALID_ARG;
+    *out = host_scratch_bytes(f->f, batch);
+    return HAC_OK;
+}
+int hac_dot_host(const hac_format* f, const float* X_host, int64_t batch, float* Y_host, void* dev_scratch,
+                 size_t dev_scratch_bytes, void* cuda_stream) {
+    if (!f) return HAC_ERR_INVALID_ARG;
+    return dot_host(f->f, X_host, batch, Y_host, dev_scratch, dev_scratch_bytes, cuda_stream);
+}
+int shac_dot_host(const shac_format* f, const float* X_host, int64_t batch, float* Y_host, void* dev_scratch,
+                  size_t dev_scratch_bytes, void* cuda_stream) {
+    if (!f) return HAC_ERR_INVALID_ARG;
+    return dot_host(f->f, X_host, batch, Y_host, dev_scratch, dev_scratch_bytes, cuda_stream);
+}
+
+int hac_debug_decode(const hac_format* f, float* W_colmajor_dev, void* cuda_stream) {
+    return f ? debug_decode(f->f, W_colmajor_dev, cuda_stream) : HAC_ERR_INVALID_ARG;
+}
+int shac_debug_decode(const shac_format* f, float* nz_dev, void* cuda_stream) {
+    return f ? debug_decode(f->f, nz_dev, cuda_stream) : HAC_ERR_INVALID_ARG;
+}
+
+int hac_last_launch_count(const hac_format* f) { return f ? f->f.last_launches : 0; }
+int shac_last_launch_count(const shac_format* f) { return f ? f->f.last_launches : 0; }
+
+void hac_free(hac_format* f) { delete f; }
+void shac_free(shac_format* f) { delete f; }
+
+const char* hac_last_cuda_error(void) { return g_last_cuda_error.c_str(); }
+
+}  // extern "C"

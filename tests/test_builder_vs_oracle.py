@@ -1,0 +1,147 @@
+"""The library's host builder against the oracle: every array of the formats bit for bit
+(codebook, code lengths, codes, stream words, ri, cb, offset index), on the same seeded
+inputs.  No GPU needed: only host entry points of the C ABI are called."""
+import dataclasses
+
+import numpy as np
+import pytest
+
+import synth_inputs as si
+from oracle import hac_oracle as orc
+import paper_2108_12704_b200 as hb
+
+
+def oracle_format(W, wl, kind):
+    Wq, mask = orc.quantize(W, wl.sparsity, wl.k, wl.quantizer, wl.kmeans_iters, wl.seed)
+    fmt = orc.hac_encode(Wq) if kind == "hac" else orc.shac_encode(Wq, mask)
+    return Wq, mask, fmt
+
+
+def library_format(W, wl, kind, S=0, ri_bits=0):
+    return hb.Format(kind, W, sparsity=wl.sparsity, k=wl.k, quantizer=wl.quantizer,
+                     kmeans_iters=wl.kmeans_iters, seed=wl.seed, seg_symbols=S, ri_bits=ri_bits)
+
+
+def assert_same_format(lib_fmt, ofmt, oidx, Wq):
+    e = lib_fmt.export()
+    assert np.array_equal(e["codebook"].view(np.uint32), ofmt["codebook"].view(np.uint32))
+    assert np.array_equal(e["code_len"], ofmt["code_len"])
+    assert np.array_equal(e["codes"], ofmt["codes"])
+    assert np.array_equal(e["counts"], ofmt["counts"])
+    assert e["stream_bits"] == ofmt["bits"]
+    N = len(ofmt["words"])
+    assert e["stream_words"] == N
+    assert np.array_equal(e["stream"][:N], ofmt["words"])
+    assert not e["stream"][N:].any() and e["stream_pad_words"] >= 4 and len(e["stream"]) % 4 == 0
+    assert np.array_equal(e["seg_bit_off"], oidx["seg_bit_off"])
+    assert np.array_equal(e["sub_bits"], oidx["sub_bits"])
+    if lib_fmt.kind == "shac":
+        assert np.array_equal(e["ri"].astype(np.int64), ofmt["ri"].astype(np.int64))
+        assert np.array_equal(e["cb"].astype(np.int64), ofmt["cb"])
+        assert np.array_equal(e["seg_first"], oidx["seg_first"])
+        assert np.array_equal(e["seg_col"], oidx["seg_col"])
+    else:
+        assert e["segs_per_col"] == oidx["G"]
+    assert np.array_equal(lib_fmt.decode_host().view(np.uint32), Wq.view(np.uint32))
+    return e
+
+
+CASES = [
+    (si.CFG1_TINY_SHAC, "shac", 0),
+    (si.CFG1_TINY_SHAC, "hac", 0),
+    (si.scaled(si.CFG2_DENSE_HAC, 300, 70), "hac", 0),
+    (si.scaled(si.CFG2_DENSE_HAC, 2100, 37), "hac", 64),      # two segments per column, ragged tail
+    (si.scaled(si.CFG3_FC_SHAC, 3000, 96), "shac", 0),
+    (si.scaled(si.CFG3_FC_SHAC, 3000, 96), "shac", 3),        # several segments per column
+    (si.scaled(si.CFG4_CONV, 460, 64), "shac", 0),
+    (si.scaled(si.CFG4_CONV, 460, 64), "hac", 16),
+]
+
+
+@pytest.mark.parametrize("wl,kind,S", CASES, ids=[f"{c[0].name}-{c[1]}-S{c[2]}" for c in CASES])
+def test_formats_bit_exact(wl, kind, S):
+    W = si.weights(wl)
+    Wq, mask, ofmt = oracle_format(W, wl, kind)
+    lf = library_format(W, wl, kind, S)
+    S_eff = S or (64 if kind == "hac" else 32)
+    oidx = orc.hac_offset_index(ofmt, S_eff) if kind == "hac" else orc.shac_offset_index(ofmt, S_eff)
+    assert_same_format(lf, ofmt, oidx, Wq)
+
+
+@pytest.mark.parametrize("k", [2, 8, 1024])
+@pytest.mark.parametrize("sp", [0.0, 0.9, 0.99])
+def test_sweep_cells_small(k, sp):
+    wl = dataclasses.replace(si.sweep_cells(192, 160)[0], sparsity=sp, k=k)
+    W = si.weights(wl)
+    for kind in ("hac", "shac"):
+        Wq, mask, ofmt = oracle_format(W, wl, kind)
+        lf = library_format(W, wl, kind)
+        S_eff = 64 if kind == "hac" else 32
+        oidx = orc.hac_offset_index(ofmt, S_eff) if kind == "hac" else orc.shac_offset_index(ofmt, S_eff)
+        assert_same_format(lf, ofmt, oidx, Wq)
+
+
+def test_sizes_report_matches_oracle_accounting():
+    wl = si.scaled(si.CFG4_CONV, 460, 64)
+    W = si.weights(wl)
+    for kind in ("hac", "shac"):
+        Wq, mask, ofmt = oracle_format(W, wl, kind)
+        r = library_format(W, wl, kind).sizes()
+        if kind == "hac":
+            assert r["paper_bits"] == orc.hac_paper_bits(ofmt)
+            assert r["bound_bits"] == pytest.approx(orc.cor1_bound_bits(wl.n, wl.m, len(ofmt["codebook"])), rel=1e-12)
+        else:
+            q = int(ofmt["cb"][-1])
+            assert r["nnz"] == q
+            assert r["paper_bits"] == orc.shac_paper_bits(ofmt)
+            assert r["bound_bits"] == pytest.approx(orc.cor2_bound_bits(wl.n, wl.m, q, len(ofmt["codebook"])), rel=1e-12)
+        assert r["paper_bits"] <= r["bound_bits"] + 31
+        assert r["entropy"] <= r["avg_code_len"] <= r["entropy"] + 1
+        assert r["total_bytes"] == (r["stream_bytes"] + r["pad_bytes"] + r["codebook_bytes"] + r["code_len_bytes"]
+                                    + r["ri_bytes"] + r["cb_bytes"] + r["offset_index_bytes"])
+        assert r["offset_index_bytes"] > 0
+
+
+def test_quantizer_none_and_special_inputs():
+    W = np.array([[1, 0, 4, 0, 0], [0, 10, 0, 0, 0], [2, 3, 0, 0, 5], [0, 0, 0, 0, 0], [0, 0, 0, 0, 6]],
+                 dtype=np.float32)                                   # Example 2 of the paper
+    lf = hb.Format("hac", W, quantizer=hb.QUANT_NONE, seg_symbols=5)
+    e = lf.export()
+    assert [f"{w:08X}" for w in e["stream"][:2]] == ["A5898680", "0E780000"]
+    assert e["seg_bit_off"].tolist() == [0, 11, 21, 29, 34]
+    ls = hb.Format("shac", W, quantizer=hb.QUANT_NONE)
+    es = ls.export()
+    assert f"{es['stream'][0]:08X}" == "4C977000"
+    assert (es["ri"] + 1).tolist() == [1, 3, 2, 3, 1, 3, 5] and (es["cb"] + 1).tolist() == [1, 3, 5, 6, 6, 8]
+    # all-zero matrix, single value, errors
+    Z = np.zeros((4, 3), dtype=np.float32)
+    assert hb.Format("shac", Z, quantizer=hb.QUANT_NONE).sizes()["nnz"] == 0
+    assert hb.Format("hac", Z, quantizer=hb.QUANT_NONE).sizes()["stream_bits"] == 12
+    with pytest.raises(hb.HacError) as ei:
+        hb.Format("hac", np.array([[np.inf, 1.0]], dtype=np.float32), quantizer=hb.QUANT_NONE)
+    assert ei.value.status == -3
+    with pytest.raises(hb.HacError) as ei:
+        hb.Format("hac", np.arange(5000, dtype=np.float32).reshape(50, 100) + 1, quantizer=hb.QUANT_NONE)
+    assert ei.value.status == -4
+    with pytest.raises(hb.HacError) as ei:
+        hb.Format("hac", W, sparsity=1.5)
+    assert ei.value.status == -1
+
+
+def test_library_exports_every_declared_symbol():
+    import re, os
+    header = open(os.path.join(os.path.dirname(__file__), "..", "include", "hac.h")).read()
+    declared = set(re.findall(r"\b(s?hac_[a-z_]+)\s*\(", header))
+    declared -= {"hac_build_params"}
+    lib = hb.load()
+    assert declared == set(hb.EXPORTS)
+    for name in declared:
+        assert hasattr(lib, name), name
+
+
+def test_device_calls_fail_loudly_without_upload():
+    W = si.weights(si.CFG1_TINY_SHAC)
+    lf = hb.Format("shac", W, sparsity=0.9, k=8, kmeans_iters=2)
+    lib = hb.load()
+    rc = lib.shac_dot(lf._h, 16, 1, 1, 0, 16, 1, 0, None, 0, None)
+    assert rc == -7          # HAC_ERR_NOT_UPLOADED: no silent fallback

@@ -1,0 +1,208 @@
+"""Parity of the CUDA path with the oracle, through the C ABI, on the same seeded inputs:
+decoded weights bit for bit, outputs within |y - y_ref| <= 1e-5 * sum_i |w_ij x_i| + 1e-7."""
+import dataclasses
+
+import numpy as np
+import pytest
+
+import synth_inputs as si
+from oracle import hac_oracle as orc
+import paper_2108_12704_b200 as hb
+
+pytestmark = pytest.mark.gpu
+
+torch = pytest.importorskip("torch")
+
+RTOL_A, ATOL = 1e-5, 1e-7
+
+
+def build_both(wl, kind, S=0, W=None, ri_bits=0):
+    W = si.weights(wl) if W is None else W
+    Wq, mask = orc.quantize(W, wl.sparsity, wl.k, wl.quantizer, wl.kmeans_iters, wl.seed)
+    lf = hb.Format(kind, W, sparsity=wl.sparsity, k=wl.k, quantizer=wl.quantizer, kmeans_iters=wl.kmeans_iters,
+                   seed=wl.seed, seg_symbols=S, ri_bits=ri_bits).upload()
+    return lf, Wq, mask
+
+
+def check_decode(lf, Wq, mask):
+    got = lf.debug_decode().cpu().numpy()
+    if lf.kind == "hac":
+        assert np.array_equal(got.view(np.uint32), np.ascontiguousarray(Wq.T).view(np.uint32))
+    else:
+        nz = Wq.T[mask.T]
+        assert np.array_equal(got.view(np.uint32), nz.view(np.uint32))
+
+
+def check_outputs(y, y_ref, a):
+    err = np.abs(y.astype(np.float64) - y_ref)
+    bound = RTOL_A * a + ATOL
+    worst = float((err / bound).max()) if err.size else 0.0
+    assert np.all(err <= bound), f"worst error / bound = {worst}"
+    return worst
+
+
+def run_dot(lf, X, layout="nb"):
+    """X: numpy [B, n].  Returns numpy [B, m]."""
+    B = X.shape[0]
+    if B == 1:
+        y = lf.dot(torch.from_numpy(X[0]).cuda())
+        torch.cuda.synchronize()
+        return y.cpu().numpy()[None, :]
+    if layout == "nb":
+        y = lf.dot(torch.from_numpy(np.ascontiguousarray(X.T)).cuda(), layout="nb")
+        torch.cuda.synchronize()
+        return y.cpu().numpy().T
+    y = lf.dot(torch.from_numpy(X).cuda(), layout="bn")
+    torch.cuda.synchronize()
+    return y.cpu().numpy()
+
+
+SMALL = [
+    # workload, kind, S, batches
+    (si.CFG1_TINY_SHAC, "shac", 0, (1, 5)),
+    (si.CFG1_TINY_SHAC, "hac", 0, (1, 33)),
+    (si.scaled(si.CFG2_DENSE_HAC, 2100, 70), "hac", 64, (1, 64)),        # 2 segments per column, ragged
+    (si.scaled(si.CFG2_DENSE_HAC, 1000, 130), "hac", 0, (1, 3)),
+    (si.scaled(si.CFG2_DENSE_HAC, 777, 45), "hac", 7, (1, 40)),          # odd S, 4 segments per column
+    (si.scaled(si.CFG3_FC_SHAC, 6000, 200), "shac", 0, (1, 16, 128)),
+    (si.scaled(si.CFG3_FC_SHAC, 6000, 90), "shac", 3, (1, 16)),          # several segments per column
+    (si.scaled(si.CFG4_CONV, 1152, 128), "shac", 0, (1, 200)),
+    (si.scaled(si.CFG4_CONV, 1152, 128), "hac", 0, (1, 200)),
+]
+
+
+@pytest.mark.parametrize("wl,kind,S,batches", SMALL, ids=[f"{c[0].name}-{c[1]}-S{c[2]}" for c in SMALL])
+def test_small_cases_element_by_element(wl, kind, S, batches):
+    lf, Wq, mask = build_both(wl, kind, S)
+    check_decode(lf, Wq, mask)
+    for B in batches:
+        X = si.inputs(wl, B)
+        y_ref, a = orc.dot_definition(Wq, X)
+        for layout in (("nb", "bn") if B > 1 else ("nb",)):
+            check_outputs(run_dot(lf, X, layout), y_ref, a)
+    # Algorithm 1 / 2 run literally give the same reference
+    x = si.inputs(wl, 1)[0]
+    ofmt = orc.hac_encode(Wq) if kind == "hac" else orc.shac_encode(Wq, mask)
+    y_alg = (orc.dot_hac if kind == "hac" else orc.dot_shac)(ofmt, x)
+    assert np.array_equal(y_alg, orc.dot_definition(Wq, x)[0][0])
+
+
+def test_host_entry_point():
+    wl = si.scaled(si.CFG3_FC_SHAC, 3000, 150)
+    for kind in ("shac", "hac"):
+        lf, Wq, mask = build_both(wl, kind)
+        for B in (1, 20):
+            X = si.inputs(wl, B)
+            y_ref, a = orc.dot_definition(Wq, X)
+            Xh = torch.from_numpy(X).pin_memory()
+            Yh = torch.empty((B, wl.m), dtype=torch.float32).pin_memory()
+            scratch = torch.empty(lf.dot_host_scratch_bytes(B), dtype=torch.uint8, device="cuda")
+            lf.dot_host(Xh, Yh, scratch)
+            check_outputs(Yh.numpy(), y_ref, a)
+
+
+def test_edge_cases():
+    rng = np.random.default_rng(77)
+    # empty columns (first, middle, last), an all-zero matrix, a single shared value
+    W = (rng.standard_normal((300, 40)) * 0.1).astype(np.float32)
+    W[:, 0] = 0; W[:, 17] = 0; W[:, 39] = 0
+    wl = dataclasses.replace(si.CFG1_TINY_SHAC, n=300, m=40, sparsity=0.5, k=8)
+    for kind in ("shac", "hac"):
+        lf, Wq, mask = build_both(wl, kind, W=W)
+        check_decode(lf, Wq, mask)
+        for B in (1, 9):
+            X = si.inputs(wl, B)
+            y_ref, a = orc.dot_definition(Wq, X)
+            y = run_dot(lf, X)
+            check_outputs(y, y_ref, a)
+            assert np.all(y[:, [0, 17, 39]] == 0)
+    Z = np.zeros((50, 6), dtype=np.float32)
+    wz = dataclasses.replace(wl, n=50, m=6, sparsity=0.0, quantizer=si.QUANT_NONE)
+    for kind in ("shac", "hac"):
+        lf, Wq, mask = build_both(wz, kind, W=Z)
+        for B in (1, 4):
+            assert np.all(run_dot(lf, si.inputs(wz, B)) == 0)
+    C1 = np.full((70, 9), 0.375, dtype=np.float32)
+    for kind in ("shac", "hac"):
+        lf, Wq, mask = build_both(wz, kind, W=C1)
+        check_decode(lf, Wq, mask)
+        X = si.inputs(dataclasses.replace(wz, n=70), 3)
+        y_ref, a = orc.dot_definition(Wq, X)
+        check_outputs(run_dot(lf, X), y_ref, a)
+
+
+def test_long_code_words_take_the_slow_path():
+    # geometric symbol frequencies: code lengths up to ~20 bits, beyond the primary table
+    rng = np.random.default_rng(5)
+    k = 22
+    p = 0.5 ** np.arange(1, k + 1)
+    p /= p.sum()
+    values = np.sort(rng.standard_normal(k).astype(np.float32))
+    W = values[rng.choice(k, size=(4096, 300), p=p)].astype(np.float32)
+    W[:k, 0] = values                                     # every value occurs
+    wl = dataclasses.replace(si.CFG1_TINY_SHAC, n=4096, m=300, sparsity=0.0, quantizer=si.QUANT_NONE)
+    for kind in ("hac", "shac"):
+        lf, Wq, mask = build_both(wl, kind, W=W)
+        assert lf.sizes()["max_code_len"] > 12
+        check_decode(lf, Wq, mask)
+        X = si.inputs(wl, 2)
+        y_ref, a = orc.dot_definition(Wq, X)
+        check_outputs(run_dot(lf, X), y_ref, a)
+        check_outputs(run_dot(lf, X[:1]), y_ref[:1], a[:1])
+
+
+def test_wide_row_index_and_large_n():
+    wl = si.scaled(si.CFG3_FC_SHAC, 70000, 24)            # n > 65536: 32-bit ri, x too large for shared memory
+    lf, Wq, mask = build_both(wl, "shac")
+    assert lf.sizes()["ri_bits"] == 32
+    check_decode(lf, Wq, mask)
+    for B in (1, 8):
+        X = si.inputs(wl, B)
+        y_ref, a = orc.dot_definition(Wq, X)
+        check_outputs(run_dot(lf, X), y_ref, a)
+    lf, Wq, mask = build_both(dataclasses.replace(wl, sparsity=0.5, k=16), "hac")
+    X = si.inputs(wl, 1)
+    y_ref, a = orc.dot_definition(Wq, X)
+    check_outputs(run_dot(lf, X), y_ref, a)
+
+
+def _full_size(wl, kind, batches, ncols=48, S=0):
+    lf, Wq, mask = build_both(wl, kind, S)
+    check_decode(lf, Wq, mask)
+    rng = np.random.default_rng(wl.seed)
+    cols = np.sort(rng.choice(wl.m, size=min(ncols, wl.m), replace=False))
+    worst = 0.0
+    for B in batches:
+        X = si.inputs(wl, B)
+        y = run_dot(lf, X)
+        rows = np.arange(B) if B <= 8 else np.sort(rng.choice(B, size=8, replace=False))
+        y_ref, a = orc.dot_definition(Wq, X[rows], cols=cols)
+        worst = max(worst, check_outputs(y[np.ix_(rows, cols)], y_ref, a))
+        if B == 1:                                          # all outputs, via Algorithm 1 / 2
+            ofmt = orc.hac_encode(Wq) if kind == "hac" else orc.shac_encode(Wq, mask)
+            y_alg = (orc.dot_hac if kind == "hac" else orc.dot_shac)(ofmt, X[0])
+            assert np.array_equal(y_alg[cols], y_ref[0])
+            a_all = np.abs(Wq.astype(np.float64)).T @ np.abs(X[0].astype(np.float64))
+            check_outputs(y[0], y_alg, a_all * (1 + 1e-9))
+    return worst
+
+
+def test_config2_dense_hac_full_size():
+    _full_size(si.CFG2_DENSE_HAC, "hac", (1, 64))
+
+
+def test_config3_fc_shac_full_size():
+    _full_size(si.CFG3_FC_SHAC, "shac", (1, 16, 128))
+
+
+def test_config4_conv_full_size():
+    wl = dataclasses.replace(si.CFG4_CONV, batches=(6272,))
+    _full_size(wl, "shac", (1, 6272))
+    _full_size(wl, "hac", (1, 6272))
+
+
+@pytest.mark.parametrize("sp,k", [(0.0, 2), (0.0, 1024), (0.5, 32), (0.9, 8), (0.99, 256), (0.95, 1024)])
+def test_config5_sweep_cells_full_size(sp, k):
+    wl = dataclasses.replace(si.sweep_cells()[0], sparsity=sp, k=k)
+    for kind in ("hac", "shac"):
+        _full_size(wl, kind, (1, 32), ncols=32)
