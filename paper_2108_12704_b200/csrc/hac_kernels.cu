@@ -54,98 +54,151 @@ struct DevFormat {
 
 constexpr int kTableWords = 34;
 
-// Decoding tables in shared memory.
-struct SmemTables {
-    const uint16_t* lut;
-    const float* value;
-    const uint64_t* limit;
-    const uint32_t* first_left;
-    const uint32_t* rank_base;
-};
+// ------------------------------------------------------------------------------------------------
+// Shared-memory access by 32-bit shared-space address (keeps address arithmetic in 32 bits).
+// The *_v forms are volatile: they read staging areas that are rewritten between segments.
+// ------------------------------------------------------------------------------------------------
+__device__ __forceinline__ uint32_t smem_addr(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+__device__ __forceinline__ uint32_t lds32(uint32_t a) {
+    uint32_t v; asm("ld.shared.u32 %0, [%1];" : "=r"(v) : "r"(a)); return v;
+}
+__device__ __forceinline__ uint32_t lds32_v(uint32_t a) {
+    uint32_t v; asm volatile("ld.shared.u32 %0, [%1];" : "=r"(v) : "r"(a) : "memory"); return v;
+}
+__device__ __forceinline__ uint32_t lds16(uint32_t a) {
+    uint16_t v; asm("ld.shared.u16 %0, [%1];" : "=h"(v) : "r"(a)); return v;
+}
+__device__ __forceinline__ uint32_t lds16_v(uint32_t a) {
+    uint16_t v; asm volatile("ld.shared.u16 %0, [%1];" : "=h"(v) : "r"(a) : "memory"); return v;
+}
+__device__ __forceinline__ float ldsf_v(uint32_t a) {
+    float v; asm volatile("ld.shared.f32 %0, [%1];" : "=f"(v) : "r"(a) : "memory"); return v;
+}
+__device__ __forceinline__ uint2 lds64(uint32_t a) {
+    uint2 v; asm("ld.shared.v2.u32 {%0, %1}, [%2];" : "=r"(v.x), "=r"(v.y) : "r"(a)); return v;
+}
 
 __host__ __device__ inline size_t align16(size_t x) { return (x + 15) & ~(size_t)15; }
 
-__host__ __device__ inline size_t tables_smem_bytes(uint32_t lut_bits, uint32_t k_eff) {
-    return align16(((size_t)2 << lut_bits)) + align16((size_t)k_eff * 4) + align16(kTableWords * 8) +
-           2 * align16(kTableWords * 4);
-}
-
-// Copies the tables to shared memory (all threads of the block take part) and returns the carve-up.
-// `p` is advanced past the tables.
-__device__ inline SmemTables stage_tables(const DevFormat& f, unsigned char*& p) {
-    SmemTables t;
-    uint16_t* lut = reinterpret_cast<uint16_t*>(p);
-    p += align16((size_t)2 << f.lut_bits);
-    float* value = reinterpret_cast<float*>(p);
-    p += align16((size_t)f.k_eff * 4);
-    uint64_t* limit = reinterpret_cast<uint64_t*>(p);
-    p += align16(kTableWords * 8);
-    uint32_t* first_left = reinterpret_cast<uint32_t*>(p);
-    p += align16(kTableWords * 4);
-    uint32_t* rank_base = reinterpret_cast<uint32_t*>(p);
-    p += align16(kTableWords * 4);
-    const uint32_t lut_words = (1u << f.lut_bits) / 2;     // pairs of 16-bit entries
-    if (lut_words == 0) {
-        if (threadIdx.x < 2) lut[threadIdx.x] = f.lut[threadIdx.x];
-    } else {
-        const uint32_t* src = reinterpret_cast<const uint32_t*>(f.lut);
-        uint32_t* dst = reinterpret_cast<uint32_t*>(lut);
-        for (uint32_t i = threadIdx.x; i < lut_words; i += blockDim.x) dst[i] = src[i];
-    }
-    for (uint32_t i = threadIdx.x; i < f.k_eff; i += blockDim.x) value[i] = f.rank_value[i];
-    if (threadIdx.x < kTableWords) {
-        limit[threadIdx.x] = f.limit[threadIdx.x];
-        first_left[threadIdx.x] = f.first_left[threadIdx.x];
-        rank_base[threadIdx.x] = f.rank_base[threadIdx.x];
-    }
-    t.lut = lut; t.value = value; t.limit = limit; t.first_left = first_left; t.rank_base = rank_base;
-    return t;
-}
-
-// Per-lane bit reader over the staged span: `buf` holds the next bits left aligned, `avail` of
-// them valid; after refill() more than 32 are valid, enough for any code word.
-struct BitReader {
-    const uint32_t* words;
-    uint32_t next;
-    uint64_t buf;
-    int avail;
-    __device__ __forceinline__ void init(const uint32_t* w, uint32_t bitpos) {
-        words = w;
-        const uint32_t wi = bitpos >> 5, sh = bitpos & 31;
-        const uint64_t two = ((uint64_t)w[wi] << 32) | w[wi + 1];
-        buf = two << sh;
-        avail = 64 - (int)sh;
-        next = wi + 2;
-    }
-    __device__ __forceinline__ void refill() {
-        if (avail <= 32) {
-            buf |= (uint64_t)words[next++] << (32 - avail);
-            avail += 32;
-        }
-    }
-    __device__ __forceinline__ void skip(uint32_t len) { buf <<= len; avail -= (int)len; }
+// How a kernel lays out its decoding tables in shared memory (chosen by the host per launch).
+//   level 1: 2^l1_bits entries {value bits, length}, 8 bytes each, stored `repl` times interleaved
+//            (entry i of replica r at index i*repl + r) so that lanes r, r+repl, .. read disjoint
+//            banks; length 0 marks a code word longer than l1_bits.
+//   level 2: the format's 16-bit table ((rank << 5) | length) over l2_bits bits, one copy, used only
+//            for code words longer than l1_bits; longer than l2_bits: search by length.
+struct TablePlan {
+    uint32_t l1_bits, repl_log2, l2_bits, has_l2;
 };
 
-// One code word: table lookup on the top L bits; code words longer than L fall back to the
-// canonical length search.  Returns the rank of the symbol.
-__device__ __forceinline__ uint32_t decode_symbol(BitReader& br, const SmemTables& t, uint32_t lut_shift,
-                                                  uint32_t lut_bits, uint32_t max_len) {
-    br.refill();
-    const uint32_t top = (uint32_t)(br.buf >> 32);
-    const uint32_t e = t.lut[top >> lut_shift];
-    uint32_t len = e & 31u, rank = e >> 5;
+__host__ __device__ inline size_t plan_smem_bytes(const TablePlan& tp, uint32_t k_eff) {
+    size_t b = ((size_t)8 << (tp.l1_bits + tp.repl_log2));
+    if (tp.has_l2) b += align16((size_t)2 << tp.l2_bits) + align16((size_t)k_eff * 4) + align16(kTableWords * 8) +
+                        2 * align16(kTableWords * 4);
+    return b;
+}
+
+// Per-thread handle on the staged tables (shared-space addresses).
+struct Decoder {
+    uint32_t l1_lane, l1_mul, l1_shift;
+    uint32_t l2, l2_shift, l2_bits, values, limit, first_left, rank_base, max_len;
+};
+
+// Builds the tables in shared memory (whole block takes part) and advances `p` past them.
+__device__ inline Decoder stage_decoder(const DevFormat& f, const TablePlan& tp, unsigned char*& p) {
+    Decoder d;
+    const uint32_t repl = 1u << tp.repl_log2;
+    uint2* l1 = reinterpret_cast<uint2*>(p);
+    p += (size_t)8 << (tp.l1_bits + tp.repl_log2);
+    const uint32_t entries = 1u << (tp.l1_bits + tp.repl_log2);
+    const uint32_t widen = f.lut_bits - tp.l1_bits;          // the format's table has >= l1_bits bits
+    for (uint32_t e = threadIdx.x; e < entries; e += blockDim.x) {
+        const uint32_t idx = e >> tp.repl_log2;
+        const uint32_t code = f.lut[(size_t)idx << widen];
+        const uint32_t len = code & 31u;
+        uint2 v = make_uint2(0u, 0u);
+        if (len != 0 && len <= tp.l1_bits) v = make_uint2(__float_as_uint(f.rank_value[code >> 5]), len);
+        l1[e] = v;
+    }
+    d.l1_lane = smem_addr(l1) + ((threadIdx.x & (repl - 1)) << 3);
+    d.l1_mul = 8u << tp.repl_log2;
+    d.l1_shift = 32 - tp.l1_bits;
+    d.l2 = d.values = d.limit = d.first_left = d.rank_base = 0;
+    d.l2_bits = tp.l2_bits; d.l2_shift = 32 - tp.l2_bits; d.max_len = f.max_len;
+    if (tp.has_l2) {
+        uint16_t* l2 = reinterpret_cast<uint16_t*>(p);
+        p += align16((size_t)2 << tp.l2_bits);
+        float* value = reinterpret_cast<float*>(p);
+        p += align16((size_t)f.k_eff * 4);
+        uint64_t* limit = reinterpret_cast<uint64_t*>(p);
+        p += align16(kTableWords * 8);
+        uint32_t* first_left = reinterpret_cast<uint32_t*>(p);
+        p += align16(kTableWords * 4);
+        uint32_t* rank_base = reinterpret_cast<uint32_t*>(p);
+        p += align16(kTableWords * 4);
+        for (uint32_t i = threadIdx.x; i < (1u << tp.l2_bits); i += blockDim.x) l2[i] = f.lut[i];
+        for (uint32_t i = threadIdx.x; i < f.k_eff; i += blockDim.x) value[i] = f.rank_value[i];
+        if (threadIdx.x < kTableWords) {
+            limit[threadIdx.x] = f.limit[threadIdx.x];
+            first_left[threadIdx.x] = f.first_left[threadIdx.x];
+            rank_base[threadIdx.x] = f.rank_base[threadIdx.x];
+        }
+        d.l2 = smem_addr(l2); d.values = smem_addr(value); d.limit = smem_addr(limit);
+        d.first_left = smem_addr(first_left); d.rank_base = smem_addr(rank_base);
+    }
+    return d;
+}
+
+// Per-lane bit reader over the staged span: a 64-bit window (hi, lo) that starts at a word
+// boundary, `off` bits of it (< 32) already consumed, `next` = shared address of the word after lo.
+struct BitReader {
+    uint32_t hi, lo, off, next;
+    __device__ __forceinline__ void init(uint32_t stage_addr, uint32_t bitpos) {
+        const uint32_t a = stage_addr + ((bitpos >> 5) << 2);
+        hi = lds32_v(a);
+        lo = lds32_v(a + 4);
+        off = bitpos & 31u;
+        next = a + 8;
+    }
+    __device__ __forceinline__ uint32_t peek() const { return __funnelshift_l(lo, hi, off); }
+    __device__ __forceinline__ void skip(uint32_t len) {
+        off += len;
+        if (off >= 32u) {
+            hi = lo;
+            lo = lds32_v(next);
+            next += 4;
+            off -= 32u;
+        }
+    }
+};
+
+// Code words longer than the level-1 table: level-2 lookup, then the search by length.
+__device__ __noinline__ uint2 decode_long(uint32_t top, const Decoder d) {
+    const uint32_t code = lds16(d.l2 + ((top >> d.l2_shift) << 1));
+    uint32_t len = code & 31u, rank = code >> 5;
     if (len == 0) {
-        len = max_len; rank = 0;
-        for (uint32_t l = lut_bits + 1; l <= max_len; ++l) {
-            if ((uint64_t)top < t.limit[l]) {
+        len = d.max_len; rank = 0;
+        for (uint32_t l = d.l2_bits + 1; l <= d.max_len; ++l) {
+            const uint32_t lim_lo = lds32(d.limit + l * 8), lim_hi = lds32(d.limit + l * 8 + 4);
+            if (lim_hi != 0 || top < lim_lo) {
                 len = l;
-                rank = t.rank_base[l] + ((top - t.first_left[l]) >> (32 - l));
+                rank = lds32(d.rank_base + l * 4) + ((top - lds32(d.first_left + l * 4)) >> (32 - l));
                 break;
             }
         }
     }
-    br.skip(len);
-    return rank;
+    return make_uint2(lds32(d.values + rank * 4), len);
+}
+
+// One code word -> the shared value it stands for.
+template <bool kLong>
+__device__ __forceinline__ float decode_value(BitReader& br, const Decoder& d) {
+    const uint32_t top = br.peek();
+    uint2 e = lds64(d.l1_lane + (top >> d.l1_shift) * d.l1_mul);
+    if (kLong) {
+        if (e.y == 0) e = decode_long(top, d);
+    }
+    br.skip(e.y);
+    return __uint_as_float(e.x);
 }
 
 // Start bit of each lane's sub-segment inside the segment (exclusive scan of the 32 lengths by
@@ -186,13 +239,13 @@ __device__ __forceinline__ float warp_sum(float v) {
 // keeps the 32 lanes on distinct banks.
 //   kMode 0: product; 1: debug decode (values written to out[j*n + i]).
 // ------------------------------------------------------------------------------------------------
-template <int kMode, bool kXShared>
-__global__ void __launch_bounds__(1024) hac_vec_kernel(DevFormat f, const float* __restrict__ x, int64_t xs_i,
-                                                       float* __restrict__ y, int64_t ys_j,
+template <int kMode, bool kXShared, bool kLong>
+__global__ void __launch_bounds__(1024) hac_vec_kernel(DevFormat f, TablePlan tp, const float* __restrict__ x,
+                                                       int64_t xs_i, float* __restrict__ y, int64_t ys_j,
                                                        float* __restrict__ aux) {
     extern __shared__ __align__(16) unsigned char smem[];
     unsigned char* p = smem;
-    const SmemTables t = stage_tables(f, p);
+    const Decoder dec = stage_decoder(f, tp, p);
     const uint32_t pad = (f.S & 1u) ? 0u : 1u;
     float* xs = reinterpret_cast<float*>(p);
     if (kMode == 0 && kXShared) {
@@ -201,8 +254,9 @@ __global__ void __launch_bounds__(1024) hac_vec_kernel(DevFormat f, const float*
     }
     const uint32_t warp = threadIdx.x >> 5, lane = threadIdx.x & 31, warps = blockDim.x >> 5;
     uint4* stage = reinterpret_cast<uint4*>(p) + (size_t)warp * f.max_unit_chunks;
+    const uint32_t stage_a = smem_addr(stage);
+    const uint32_t xs_a = smem_addr(xs);
     __syncthreads();
-    const uint32_t lut_shift = 32 - f.lut_bits;
 
     for (uint32_t u = blockIdx.x * warps + warp; u < f.units; u += gridDim.x * warps) {
         const uint32_t j = u / f.G, g = u - j * f.G;
@@ -214,20 +268,22 @@ __global__ void __launch_bounds__(1024) hac_vec_kernel(DevFormat f, const float*
         const uint32_t row0 = sub * f.S;
         const uint32_t count = row0 < f.n ? min(f.S, f.n - row0) : 0u;
         BitReader br;
-        br.init(reinterpret_cast<const uint32_t*>(stage), base + start);
-        float acc = 0.0f;
+        br.init(stage_a, base + start);
         if (kMode == 0) {
+            float acc = 0.0f;
             if (kXShared) {
-                const float* xl = xs + row0 + pad * sub;
+                uint32_t xa = xs_a + ((row0 + pad * sub) << 2);
+#pragma unroll 4
                 for (uint32_t s = 0; s < count; ++s) {
-                    const uint32_t r = decode_symbol(br, t, lut_shift, f.lut_bits, f.max_len);
-                    acc = fmaf(xl[s], t.value[r], acc);
+                    const float w = decode_value<kLong>(br, dec);
+                    acc = fmaf(ldsf_v(xa), w, acc);
+                    xa += 4;
                 }
             } else {
                 const float* xl = x + (int64_t)row0 * xs_i;
                 for (uint32_t s = 0; s < count; ++s) {
-                    const uint32_t r = decode_symbol(br, t, lut_shift, f.lut_bits, f.max_len);
-                    acc = fmaf(xl[(int64_t)s * xs_i], t.value[r], acc);
+                    const float w = decode_value<kLong>(br, dec);
+                    acc = fmaf(xl[(int64_t)s * xs_i], w, acc);
                 }
             }
             acc = warp_sum(acc);
@@ -237,10 +293,7 @@ __global__ void __launch_bounds__(1024) hac_vec_kernel(DevFormat f, const float*
             }
         } else {
             float* out = aux + (size_t)j * f.n + row0;
-            for (uint32_t s = 0; s < count; ++s) {
-                const uint32_t r = decode_symbol(br, t, lut_shift, f.lut_bits, f.max_len);
-                out[s] = t.value[r];
-            }
+            for (uint32_t s = 0; s < count; ++s) out[s] = decode_value<kLong>(br, dec);
         }
         __syncwarp();
     }
@@ -248,15 +301,16 @@ __global__ void __launch_bounds__(1024) hac_vec_kernel(DevFormat f, const float*
 
 // ------------------------------------------------------------------------------------------------
 // sHAC, one input vector (Algorithm 2 by segments): as above over the stored entries of a column,
-// with the row of each entry read from ri and x gathered from shared memory.
+// with the row of each entry taken from ri (the segment's slice of ri is staged in shared memory
+// by coalesced loads) and x gathered from shared memory.
 // ------------------------------------------------------------------------------------------------
-template <int kMode, bool kXShared, typename RowT>
-__global__ void __launch_bounds__(1024) shac_vec_kernel(DevFormat f, const float* __restrict__ x, int64_t xs_i,
-                                                        float* __restrict__ y, int64_t ys_j,
+template <int kMode, bool kXShared, bool kLong, typename RowT>
+__global__ void __launch_bounds__(1024) shac_vec_kernel(DevFormat f, TablePlan tp, const float* __restrict__ x,
+                                                        int64_t xs_i, float* __restrict__ y, int64_t ys_j,
                                                         float* __restrict__ aux) {
     extern __shared__ __align__(16) unsigned char smem[];
     unsigned char* p = smem;
-    const SmemTables t = stage_tables(f, p);
+    const Decoder dec = stage_decoder(f, tp, p);
     float* xs = reinterpret_cast<float*>(p);
     if (kMode == 0 && kXShared) {
         for (uint32_t i = threadIdx.x; i < f.n; i += blockDim.x) xs[i] = x[(int64_t)i * xs_i];
@@ -264,8 +318,12 @@ __global__ void __launch_bounds__(1024) shac_vec_kernel(DevFormat f, const float
     }
     const uint32_t warp = threadIdx.x >> 5, lane = threadIdx.x & 31, warps = blockDim.x >> 5;
     uint4* stage = reinterpret_cast<uint4*>(p) + (size_t)warp * f.max_unit_chunks;
+    p += align16((size_t)warps * f.max_unit_chunks * 16);
+    // row-index staging: 32*S entries plus up to 16 bytes of misalignment, per warp
+    const uint32_t ri_chunks = (32u * f.S * (uint32_t)sizeof(RowT) + 15u) / 16u + 1u;
+    uint4* ri_stage = reinterpret_cast<uint4*>(p) + (size_t)warp * ri_chunks;
+    const uint32_t stage_a = smem_addr(stage), ri_a = smem_addr(ri_stage), xs_a = smem_addr(xs);
     __syncthreads();
-    const uint32_t lut_shift = 32 - f.lut_bits;
     const RowT* __restrict__ ri = reinterpret_cast<const RowT*>(f.ri);
 
     for (uint32_t u = blockIdx.x * warps + warp; u < f.units; u += gridDim.x * warps) {
@@ -276,18 +334,32 @@ __global__ void __launch_bounds__(1024) shac_vec_kernel(DevFormat f, const float
         const uint32_t my_bits = f.sub_bits[(size_t)u * 32 + lane];
         uint32_t total;
         const uint32_t start = lane_start_bits(my_bits, lane, total);
-        const uint32_t base = stage_span(f, f.seg_bit_off[u], total, stage, lane);
-        const uint32_t pos0 = f.cb[j] + (g * 32 + lane) * f.S;
+        const uint32_t seg_pos0 = f.cb[j] + g * 32 * f.S;
+        const uint32_t seg_count = min(32u * f.S, col_end - seg_pos0);
+        uint32_t ri_lane = 0;
+        if (kMode == 0) {
+            // stage ri[seg_pos0 .. seg_pos0 + seg_count) from the enclosing 16-byte chunks
+            const uintptr_t byte0 = reinterpret_cast<uintptr_t>(ri + seg_pos0);
+            const uintptr_t chunk0 = byte0 & ~(uintptr_t)15;
+            const uint32_t chunks = (uint32_t)((byte0 + (uintptr_t)seg_count * sizeof(RowT) - chunk0 + 15) >> 4);
+            const uint4* src = reinterpret_cast<const uint4*>(chunk0);
+            for (uint32_t c = lane; c < chunks; c += 32) ri_stage[c] = __ldg(src + c);
+            ri_lane = ri_a + (uint32_t)(byte0 - chunk0) + lane * f.S * (uint32_t)sizeof(RowT);
+        }
+        const uint32_t base = stage_span(f, f.seg_bit_off[u], total, stage, lane);   // ends with __syncwarp
+        const uint32_t pos0 = seg_pos0 + lane * f.S;
         const uint32_t count = pos0 < col_end ? min(f.S, col_end - pos0) : 0u;
         BitReader br;
-        br.init(reinterpret_cast<const uint32_t*>(stage), base + start);
+        br.init(stage_a, base + start);
         if (kMode == 0) {
             float acc = 0.0f;
+#pragma unroll 4
             for (uint32_t s = 0; s < count; ++s) {
-                const uint32_t r = decode_symbol(br, t, lut_shift, f.lut_bits, f.max_len);
-                const uint32_t row = ri[pos0 + s];
-                const float xv = kXShared ? xs[row] : x[(int64_t)row * xs_i];
-                acc = fmaf(xv, t.value[r], acc);
+                const float w = decode_value<kLong>(br, dec);
+                const uint32_t row = sizeof(RowT) == 2 ? lds16_v(ri_lane) : lds32_v(ri_lane);
+                ri_lane += sizeof(RowT);
+                const float xv = kXShared ? ldsf_v(xs_a + (row << 2)) : x[(int64_t)row * xs_i];
+                acc = fmaf(xv, w, acc);
             }
             acc = warp_sum(acc);
             if (lane == 0) {
@@ -296,10 +368,7 @@ __global__ void __launch_bounds__(1024) shac_vec_kernel(DevFormat f, const float
                 else aux[u] = acc;
             }
         } else {
-            for (uint32_t s = 0; s < count; ++s) {
-                const uint32_t r = decode_symbol(br, t, lut_shift, f.lut_bits, f.max_len);
-                aux[pos0 + s] = t.value[r];
-            }
+            for (uint32_t s = 0; s < count; ++s) aux[pos0 + s] = decode_value<kLong>(br, dec);
         }
         __syncwarp();
     }
@@ -335,13 +404,13 @@ constexpr int kBatchRows = 32 * kBatchSteps;
 constexpr int kAccMax = 4;              // batch tile = 32 * kAcc inputs
 
 template <int kAcc>
-__global__ void __launch_bounds__(1024) hac_batch_kernel(DevFormat f, const float* __restrict__ x, int64_t xs_i,
-                                                         int64_t xs_b, uint32_t batch, float* __restrict__ y,
-                                                         int64_t ys_j, int64_t ys_b, float* __restrict__ partial,
-                                                         uint32_t col_blocks) {
+__global__ void __launch_bounds__(1024) hac_batch_kernel(DevFormat f, TablePlan tp, const float* __restrict__ x,
+                                                         int64_t xs_i, int64_t xs_b, uint32_t batch,
+                                                         float* __restrict__ y, int64_t ys_j, int64_t ys_b,
+                                                         float* __restrict__ partial, uint32_t col_blocks) {
     extern __shared__ __align__(16) unsigned char smem[];
     unsigned char* p = smem;
-    const SmemTables t = stage_tables(f, p);
+    const Decoder dec = stage_decoder(f, tp, p);
     const uint32_t warp = threadIdx.x >> 5, lane = threadIdx.x & 31, warps = blockDim.x >> 5;
     constexpr uint32_t kTile = 32 * kAcc;
     float* wt = reinterpret_cast<float*>(p);                       // [warps][kBatchRows]
@@ -349,8 +418,8 @@ __global__ void __launch_bounds__(1024) hac_batch_kernel(DevFormat f, const floa
     float* xt = reinterpret_cast<float*>(p);                       // [kBatchRows][kTile]
     p += align16((size_t)kBatchRows * kTile * 4);
     uint4* stage = reinterpret_cast<uint4*>(p) + (size_t)warp * f.max_unit_chunks;
+    const uint32_t stage_a = smem_addr(stage);
     __syncthreads();
-    const uint32_t lut_shift = 32 - f.lut_bits;
     const uint32_t batch_tiles = (batch + kTile - 1) / kTile;
     const uint32_t items = col_blocks * f.G * batch_tiles;
 
@@ -366,14 +435,14 @@ __global__ void __launch_bounds__(1024) hac_batch_kernel(DevFormat f, const floa
         const uint32_t row0 = sub * f.S;
         uint32_t count = 0;
         BitReader br;
-        br.words = reinterpret_cast<const uint32_t*>(stage); br.next = 0; br.buf = 0; br.avail = 64;
+        br.hi = br.lo = br.off = 0; br.next = stage_a;
         if (live) {
             const uint32_t my_bits = f.sub_bits[(size_t)u * 32 + lane];
             uint32_t total;
             const uint32_t start = lane_start_bits(my_bits, lane, total);
             const uint32_t base = stage_span(f, f.seg_bit_off[u], total, stage, lane);
             count = row0 < f.n ? min(f.S, f.n - row0) : 0u;
-            br.init(reinterpret_cast<const uint32_t*>(stage), base + start);
+            br.init(stage_a, base + start);
         }
         float acc[kAcc];
 #pragma unroll
@@ -384,7 +453,7 @@ __global__ void __launch_bounds__(1024) hac_batch_kernel(DevFormat f, const floa
 #pragma unroll
             for (int s = 0; s < kBatchSteps; ++s) {
                 float v = 0.0f;
-                if (s0 + s < count) v = t.value[decode_symbol(br, t, lut_shift, f.lut_bits, f.max_len)];
+                if (s0 + s < count) v = decode_value<true>(br, dec);
                 wt[warp * kBatchRows + lane * kBatchSteps + s] = v;
             }
             // matching rows of X: tile row r = l*kBatchSteps + s  <->  matrix row (g*32+l)*S + s0 + s
@@ -427,13 +496,13 @@ __global__ void __launch_bounds__(1024) hac_batch_kernel(DevFormat f, const floa
 // inputs, gathering the rows of X (stored [n][batch] for coalesced access).
 // ------------------------------------------------------------------------------------------------
 template <int kAcc, typename RowT>
-__global__ void __launch_bounds__(1024) shac_batch_kernel(DevFormat f, const float* __restrict__ x, int64_t xs_i,
-                                                          int64_t xs_b, uint32_t batch, float* __restrict__ y,
-                                                          int64_t ys_j, int64_t ys_b,
+__global__ void __launch_bounds__(1024) shac_batch_kernel(DevFormat f, TablePlan tp, const float* __restrict__ x,
+                                                          int64_t xs_i, int64_t xs_b, uint32_t batch,
+                                                          float* __restrict__ y, int64_t ys_j, int64_t ys_b,
                                                           float* __restrict__ partial) {
     extern __shared__ __align__(16) unsigned char smem[];
     unsigned char* p = smem;
-    const SmemTables t = stage_tables(f, p);
+    const Decoder dec = stage_decoder(f, tp, p);
     const uint32_t warp = threadIdx.x >> 5, lane = threadIdx.x & 31, warps = blockDim.x >> 5;
     constexpr uint32_t kTile = 32 * kAcc;
     float* wv_all = reinterpret_cast<float*>(p);
@@ -443,8 +512,8 @@ __global__ void __launch_bounds__(1024) shac_batch_kernel(DevFormat f, const flo
     uint4* stage = reinterpret_cast<uint4*>(p) + (size_t)warp * f.max_unit_chunks;
     float* wv = wv_all + warp * kBatchRows;
     uint32_t* wr = wr_all + warp * kBatchRows;
+    const uint32_t stage_a = smem_addr(stage);
     __syncthreads();
-    const uint32_t lut_shift = 32 - f.lut_bits;
     const RowT* __restrict__ ri = reinterpret_cast<const RowT*>(f.ri);
     const uint32_t batch_tiles = (batch + kTile - 1) / kTile;
     const uint64_t items = (uint64_t)f.units * batch_tiles;
@@ -465,7 +534,7 @@ __global__ void __launch_bounds__(1024) shac_batch_kernel(DevFormat f, const flo
         const uint32_t count = pos0 < col_end ? min(f.S, col_end - pos0) : 0u;
         const uint32_t seg_rows = min(f.S, col_end - seg_pos0);
         BitReader br;
-        br.init(reinterpret_cast<const uint32_t*>(stage), base + start);
+        br.init(stage_a, base + start);
         float acc[kAcc];
 #pragma unroll
         for (int a = 0; a < kAcc; ++a) acc[a] = 0.0f;
@@ -475,7 +544,7 @@ __global__ void __launch_bounds__(1024) shac_batch_kernel(DevFormat f, const flo
                 float v = 0.0f;
                 uint32_t row = 0;
                 if (s0 + s < count) {
-                    v = t.value[decode_symbol(br, t, lut_shift, f.lut_bits, f.max_len)];
+                    v = decode_value<true>(br, dec);
                     row = ri[pos0 + s0 + s];
                 }
                 wv[lane * kBatchSteps + s] = v;
@@ -646,6 +715,34 @@ static int launch_finalize(const Format& f, const DevFormat& d, const float* par
     return HAC_OK;
 }
 
+// Table plan: level-1 width and replication that fit `table_budget` bytes of shared memory.
+static TablePlan plan_tables(const DevFormat& d, size_t table_budget, int max_l1) {
+    TablePlan tp{};
+    tp.l2_bits = d.lut_bits;
+    tp.l1_bits = std::min<uint32_t>(d.lut_bits, (uint32_t)max_l1);
+    tp.repl_log2 = 4;
+    while (tp.repl_log2 > 0 && ((size_t)8 << (tp.l1_bits + tp.repl_log2)) > table_budget) tp.repl_log2--;
+    while (tp.l1_bits > 1 && ((size_t)8 << (tp.l1_bits + tp.repl_log2)) > table_budget) tp.l1_bits--;
+    tp.has_l2 = d.max_len > tp.l1_bits ? 1u : 0u;
+    return tp;
+}
+
+typedef void (*VecKernel)(DevFormat, TablePlan, const float*, int64_t, float*, int64_t, float*);
+
+template <bool kLong>
+static VecKernel pick_vec_kernel(const Format& f, int mode, bool x_shared) {
+    if (!f.sparse)
+        return mode == 1 ? hac_vec_kernel<1, false, kLong>
+                         : (x_shared ? hac_vec_kernel<0, true, kLong> : hac_vec_kernel<0, false, kLong>);
+    if (f.ri_bits == 16)
+        return mode == 1 ? shac_vec_kernel<1, false, kLong, uint16_t>
+                         : (x_shared ? shac_vec_kernel<0, true, kLong, uint16_t>
+                                     : shac_vec_kernel<0, false, kLong, uint16_t>);
+    return mode == 1 ? shac_vec_kernel<1, false, kLong, uint32_t>
+                     : (x_shared ? shac_vec_kernel<0, true, kLong, uint32_t>
+                                 : shac_vec_kernel<0, false, kLong, uint32_t>);
+}
+
 // mode 0: product with one input; mode 1: debug decode into `aux`.
 static int launch_vec(const Format& f, int mode, const float* x, int64_t xs_i, float* y, int64_t ys_j,
                       float* aux, cudaStream_t st) {
@@ -655,39 +752,37 @@ static int launch_vec(const Format& f, int mode, const float* x, int64_t xs_i, f
     const DevFormat d = dev_format(f);
     if (d.units == 0) return HAC_OK;
     const size_t budget = (size_t)di.max_smem_optin;
-    const size_t tab = tables_smem_bytes(d.lut_bits, d.k_eff);
-    const size_t per_warp = (size_t)d.max_unit_chunks * 16;
+    size_t per_warp = (size_t)d.max_unit_chunks * 16;
+    if (f.sparse && mode == 0) per_warp += ((size_t)(32u * f.S * (f.ri_bits / 8) + 15u) / 16u + 1u) * 16u;
     size_t xbytes = 0;
     if (mode == 0) xbytes = f.sparse ? align16((size_t)f.n * 4) : align16(((size_t)f.n + (f.n / f.S + 1)) * 4);
-    const int want = std::min(32, std::max(1, env_int("HAC_B200_VEC_WARPS", 16)));
+    const int want = std::min(32, std::max(1, env_int("HAC_B200_VEC_WARPS", 32)));
+    const int max_l1 = std::min(12, std::max(1, env_int("HAC_B200_L1_BITS", 10)));
+    // shared memory: tables + x + per-warp staging.  Prefer keeping x and all warps; shrink the
+    // level-1 table (fewer replicas, then fewer bits) before giving up warps.
     bool x_shared = mode == 0;
-    int warps = fit_warps(tab + xbytes, per_warp, want, 1, budget);
-    if (mode == 0 && warps < std::min(want, 4)) {        // x does not fit next to enough warps
-        x_shared = false;
-        xbytes = 0;
-        warps = fit_warps(tab, per_warp, want, 1, budget);
-    }
-    if (warps == 0) return HAC_ERR_BUFFER_TOO_SMALL;
-    const size_t smem = tab + xbytes + per_warp * warps;
+    const size_t min_tables = 4096;
+    if (x_shared && xbytes + min_tables + per_warp * std::min(want, 8) > budget) { x_shared = false; xbytes = 0; }
+    int warps = want;
+    while (warps > 1 && xbytes + min_tables + per_warp * (size_t)warps > budget) --warps;
+    if (xbytes + min_tables + per_warp * (size_t)warps > budget) return HAC_ERR_BUFFER_TOO_SMALL;
+    const size_t aux_tables = align16((size_t)2 << d.lut_bits) + align16((size_t)d.k_eff * 4) + 1024;
+    size_t table_budget = budget - xbytes - per_warp * (size_t)warps;
+    table_budget = table_budget > aux_tables + 1024 ? table_budget - aux_tables : 1024;
+    table_budget = std::min<size_t>(table_budget, (size_t)128 * 1024);
+    const TablePlan tp = plan_tables(d, table_budget, max_l1);
+    const size_t smem = plan_smem_bytes(tp, d.k_eff) + xbytes + per_warp * warps;
+    if (smem > budget) return HAC_ERR_BUFFER_TOO_SMALL;
     const int threads = warps * 32;
-    int per_sm = 1;
-    void (*kernel)(DevFormat, const float*, int64_t, float*, int64_t, float*) = nullptr;
-    if (!f.sparse) {
-        kernel = mode == 1 ? hac_vec_kernel<1, false> : (x_shared ? hac_vec_kernel<0, true> : hac_vec_kernel<0, false>);
-    } else if (f.ri_bits == 16) {
-        kernel = mode == 1 ? shac_vec_kernel<1, false, uint16_t>
-                           : (x_shared ? shac_vec_kernel<0, true, uint16_t> : shac_vec_kernel<0, false, uint16_t>);
-    } else {
-        kernel = mode == 1 ? shac_vec_kernel<1, false, uint32_t>
-                           : (x_shared ? shac_vec_kernel<0, true, uint32_t> : shac_vec_kernel<0, false, uint32_t>);
-    }
+    VecKernel kernel = tp.has_l2 ? pick_vec_kernel<true>(f, mode, x_shared) : pick_vec_kernel<false>(f, mode, x_shared);
     rc = prepare_kernel(kernel, smem);
     if (rc) return rc;
+    int per_sm = 1;
     HAC_CUDA(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kernel, threads, smem));
     per_sm = std::max(per_sm, 1);
     const unsigned need = (d.units + warps - 1) / warps;
     const unsigned grid = std::min<unsigned>(need, (unsigned)(di.sms * per_sm));
-    kernel<<<grid, threads, smem, st>>>(d, x, xs_i, y, ys_j, aux);
+    kernel<<<grid, threads, smem, st>>>(d, tp, x, xs_i, y, ys_j, aux);
     HAC_CUDA(cudaGetLastError());
     f.last_launches++;
     return HAC_OK;
@@ -698,7 +793,8 @@ static int launch_batch_t(const Format& f, const DeviceInfo& di, const DevFormat
                           int64_t xs_b, int64_t batch, float* y, int64_t ys_j, int64_t ys_b, float* partial,
                           cudaStream_t st) {
     const size_t budget = (size_t)di.max_smem_optin;
-    const size_t tab = tables_smem_bytes(d.lut_bits, d.k_eff);
+    const TablePlan tp = plan_tables(d, 32 * 1024, 10);
+    const size_t tab = plan_smem_bytes(tp, d.k_eff);
     constexpr uint32_t kTile = 32 * kAcc;
     const uint32_t batch_tiles = (uint32_t)((batch + kTile - 1) / kTile);
     int rc;
@@ -718,15 +814,16 @@ static int launch_batch_t(const Format& f, const DeviceInfo& di, const DevFormat
         const uint32_t col_blocks = (uint32_t)((f.m + warps - 1) / warps);
         const uint64_t items = (uint64_t)col_blocks * d.G * batch_tiles;
         const unsigned grid = (unsigned)std::min<uint64_t>(items, (uint64_t)di.sms * per_sm);
-        kernel<<<grid, warps * 32, smem, st>>>(d, x, xs_i, xs_b, (uint32_t)batch, y, ys_j, ys_b, partial, col_blocks);
+        kernel<<<grid, warps * 32, smem, st>>>(d, tp, x, xs_i, xs_b, (uint32_t)batch, y, ys_j, ys_b, partial,
+                                               col_blocks);
     } else {
         const size_t per_warp = (size_t)d.max_unit_chunks * 16 + 2 * kBatchRows * 4;
         const int want = std::min(32, std::max(1, env_int("HAC_B200_BATCH_WARPS", 8)));
         const int warps = fit_warps(tab + 32, per_warp, want, 1, budget);
         if (warps == 0) return HAC_ERR_BUFFER_TOO_SMALL;
         const size_t smem = tab + 32 + per_warp * warps;
-        void (*kernel)(DevFormat, const float*, int64_t, int64_t, uint32_t, float*, int64_t, int64_t, float*) =
-            f.ri_bits == 16 ? shac_batch_kernel<kAcc, uint16_t> : shac_batch_kernel<kAcc, uint32_t>;
+        void (*kernel)(DevFormat, TablePlan, const float*, int64_t, int64_t, uint32_t, float*, int64_t, int64_t,
+                       float*) = f.ri_bits == 16 ? shac_batch_kernel<kAcc, uint16_t> : shac_batch_kernel<kAcc, uint32_t>;
         rc = prepare_kernel(kernel, smem);
         if (rc) return rc;
         int per_sm = 1;
@@ -734,7 +831,7 @@ static int launch_batch_t(const Format& f, const DeviceInfo& di, const DevFormat
         per_sm = std::max(per_sm, 1);
         const uint64_t items = (uint64_t)d.units * batch_tiles;
         const unsigned grid = (unsigned)std::min<uint64_t>((items + warps - 1) / warps, (uint64_t)di.sms * per_sm);
-        kernel<<<grid, warps * 32, smem, st>>>(d, x, xs_i, xs_b, (uint32_t)batch, y, ys_j, ys_b, partial);
+        kernel<<<grid, warps * 32, smem, st>>>(d, tp, x, xs_i, xs_b, (uint32_t)batch, y, ys_j, ys_b, partial);
     }
     HAC_CUDA(cudaGetLastError());
     f.last_launches++;
