@@ -200,7 +200,7 @@ void make_decode_tables(Format& f) {
     DecodeTables& t = f.tables;
     const uint32_t k = (uint32_t)f.codebook.size();
     t = DecodeTables();
-    if (k == 0) { t.lut_bits = 1; t.lut.assign(2, 0); return; }
+    if (k == 0) { t.lut_bits = 1; t.lut.assign(2, 0); t.l1_bits = 1; t.l1.assign(4, 0u); return; }
     std::vector<uint32_t> by_rank(k);
     std::iota(by_rank.begin(), by_rank.end(), 0u);
     std::stable_sort(by_rank.begin(), by_rank.end(),
@@ -233,6 +233,49 @@ void make_decode_tables(Format& f) {
         const uint32_t span = 1u << (t.lut_bits - l);
         const uint16_t e = (uint16_t)((r << 5) | (uint32_t)l);
         for (uint32_t i = 0; i < span; ++i) t.lut[lo + i] = e;
+    }
+    // two-level table: direct entries for code words of at most l1_bits bits, sub-tables behind
+    // the prefixes that longer code words share
+    auto bits_of = [](float v) { uint32_t b; std::memcpy(&b, &v, 4); return b; };
+    t.l1_bits = std::min<int>((int)f.max_len, kL1BitsMax);
+    const uint32_t L1 = (uint32_t)t.l1_bits;
+    for (int sub_max = kSubBitsMax; sub_max >= 1; --sub_max) {
+        t.l1.assign((size_t)2 << L1, 0u);
+        t.sub.clear();
+        std::vector<uint32_t> longest((size_t)1 << L1, 0u);    // longest code word behind each prefix
+        for (uint32_t s = 0; s < k; ++s) {
+            const uint32_t l = f.code_len[s];
+            if (l <= L1) {
+                const uint32_t lo = f.codes[s] << (L1 - l), span = 1u << (L1 - l);
+                for (uint32_t i = 0; i < span; ++i) { t.l1[2 * (lo + i)] = bits_of(f.codebook[s]); t.l1[2 * (lo + i) + 1] = l; }
+            } else {
+                const uint32_t pre = f.codes[s] >> (l - L1);
+                longest[pre] = std::max(longest[pre], l);
+            }
+        }
+        std::vector<uint32_t> sub_base((size_t)1 << L1, 0u), sub_bits((size_t)1 << L1, 0u);
+        for (uint32_t pre = 0; pre < (1u << L1); ++pre) {
+            if (longest[pre] == 0) continue;
+            const uint32_t b = std::min<uint32_t>(longest[pre] - L1, (uint32_t)sub_max);
+            sub_base[pre] = (uint32_t)(t.sub.size() / 2);
+            sub_bits[pre] = b;
+            t.sub.resize(t.sub.size() + ((size_t)2 << b), 0u);
+            t.l1[2 * pre] = sub_base[pre] * 8u;
+            t.l1[2 * pre + 1] = 0x80000000u | b;
+        }
+        for (uint32_t s = 0; s < k; ++s) {
+            const uint32_t l = f.code_len[s];
+            if (l <= L1) continue;
+            const uint32_t pre = f.codes[s] >> (l - L1), b = sub_bits[pre];
+            if (l > L1 + b) continue;                          // left to the search over lengths
+            const uint32_t rem = f.codes[s] & ((1u << (l - L1)) - 1u);
+            const uint32_t lo = rem << (L1 + b - l), span = 1u << (L1 + b - l);
+            for (uint32_t i = 0; i < span; ++i) {
+                t.sub[2 * (sub_base[pre] + lo + i)] = bits_of(f.codebook[s]);
+                t.sub[2 * (sub_base[pre] + lo + i) + 1] = l;
+            }
+        }
+        if (t.sub.size() * 4 <= kSubTableBytesMax) break;
     }
 }
 
@@ -397,6 +440,19 @@ int build_impl(const float* W, int64_t n, int64_t m, int64_t ldw, const hac_buil
         f.max_unit_chunks = std::max<uint32_t>(f.max_unit_chunks, (uint32_t)((last_word >> 2) - first_chunk + 1));
     }
     if (sparse) {
+        f.unit_info.resize(U * 6);
+        for (size_t u = 0; u < U; ++u) {
+            const uint32_t j = f.seg_col[u];
+            const uint32_t g = (uint32_t)u - f.seg_first[j];
+            const uint32_t pos0 = f.cb[j] + g * 32u * S;
+            uint32_t* r = &f.unit_info[u * 6];
+            r[0] = (uint32_t)(f.seg_bit_off[u] & 0xffffffffu);
+            r[1] = (uint32_t)(f.seg_bit_off[u] >> 32);
+            r[2] = pos0;
+            r[3] = std::min<uint32_t>(32u * S, f.cb[j + 1] - pos0);
+            r[4] = j;
+            r[5] = (f.seg_first[j + 1] - f.seg_first[j]) == 1 ? 1u : 0u;
+        }
         f.max_units_per_col = 0;
         f.has_empty_col = false;
         for (int64_t j = 0; j < m; ++j) {
@@ -496,6 +552,8 @@ ImageLayout image_layout(const Format& f) {
     auto take = [&](size_t bytes) { size_t at = o; o = align256(o + std::max<size_t>(bytes, 16)); return at; };
     L.stream = take(f.stream.size() * 4);
     L.lut = take(f.tables.lut.size() * 2);
+    L.l1 = take(f.tables.l1.size() * 4);
+    L.sub = take(f.tables.sub.size() * 4);
     L.rank_value = take(f.tables.rank_value.size() * 4);
     L.limit = take(sizeof(f.tables.limit));
     L.first_left = take(sizeof(f.tables.first_left));
@@ -506,6 +564,7 @@ ImageLayout image_layout(const Format& f) {
     L.seg_first = take(f.seg_first.size() * 4);
     L.ri = take(f.ri_bits == 16 ? f.ri16.size() * 2 + 16 : f.ri32.size() * 4 + 16);
     L.cb = take(f.cb.size() * 4);
+    L.unit_info = take(f.unit_info.size() * 4);
     L.total = o;
     return L;
 }

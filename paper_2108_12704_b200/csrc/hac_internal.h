@@ -11,7 +11,10 @@
 namespace hacb200 {
 
 constexpr int kMaxCodeLen = 32;
-constexpr int kLutBitsMax = 12;          // primary decode table: 2^L entries of 16 bits
+constexpr int kLutBitsMax = 12;          // full-width decode table: 2^L entries of 16 bits
+constexpr int kL1BitsMax = 10;           // level-1 table of the kernels: 2^L1 entries of 8 bytes
+constexpr int kSubBitsMax = 8;           // widest level-2 sub-table
+constexpr size_t kSubTableBytesMax = 24 * 1024;
 constexpr int kStreamSlackWords = 4;     // zero words after the stream (decoder reads ahead)
 
 // Decoding tables derived from the code lengths (canonical Huffman).  "rank" is the position of
@@ -22,10 +25,19 @@ struct DecodeTables {
     std::vector<uint16_t> lut;                // [2^L] (rank << 5) | len, 0 = code longer than L
     std::vector<float> rank_value;            // [k_eff]
     std::vector<uint16_t> rank_symbol;        // [k_eff] symbol id of each rank
+    // Two-level table used by the kernels.  l1[i] for the L1-bit prefix i is {value bits, length}
+    // when the code word ends within the prefix, else {byte offset of a sub-table, 0x80000000 | b}:
+    // the sub-table is indexed by the next b bits and holds {value bits, length} or {0, 0} (code
+    // word longer than L1 + b: found by the search over lengths).
+    int l1_bits = 0;
+    std::vector<uint32_t> l1;                 // [2^l1_bits * 2]
+    std::vector<uint32_t> sub;                // [entries * 2]
     uint64_t limit[kMaxCodeLen + 2] = {};     // left-aligned (32-bit) end of the codes of length l
     uint32_t first_left[kMaxCodeLen + 2] = {};// left-aligned first code of length l
     uint32_t rank_base[kMaxCodeLen + 2] = {}; // rank of the first code of length l
 };
+
+struct uint2_host { uint32_t x, y; };
 
 // Pointers into the device image, filled by upload/attach.
 struct DeviceImage {
@@ -33,6 +45,8 @@ struct DeviceImage {
     size_t bytes = 0;
     const uint32_t* stream = nullptr;
     const uint16_t* lut = nullptr;
+    const uint2_host* l1 = nullptr;
+    const uint2_host* sub = nullptr;
     const float* rank_value = nullptr;
     const uint64_t* limit = nullptr;          // [34]
     const uint32_t* first_left = nullptr;     // [34]
@@ -43,6 +57,7 @@ struct DeviceImage {
     const uint32_t* seg_first = nullptr;
     const void* ri = nullptr;
     const uint32_t* cb = nullptr;
+    const void* unit_info = nullptr;
 };
 
 struct Format {
@@ -70,6 +85,7 @@ struct Format {
     std::vector<uint64_t> seg_bit_off;
     std::vector<uint16_t> sub_bits;
     std::vector<uint32_t> seg_first, seg_col;
+    std::vector<uint32_t> unit_info;          // sHAC, device only: 6 words per segment (see ShacUnit)
     uint32_t max_unit_chunks = 0;             // largest 16-byte span a segment's stream covers
     uint32_t max_units_per_col = 0;
     bool has_empty_col = false;
@@ -87,8 +103,8 @@ void fill_size_report(const Format& f, hac_size_report* r);
 
 // device image layout: offsets of every section (256-byte aligned), total size
 struct ImageLayout {
-    size_t stream, lut, rank_value, limit, first_left, rank_base, seg_bit_off, sub_bits, seg_col,
-        seg_first, ri, cb, total;
+    size_t stream, lut, l1, sub, rank_value, limit, first_left, rank_base, seg_bit_off, sub_bits, seg_col,
+        seg_first, ri, cb, unit_info, total;
 };
 ImageLayout image_layout(const Format& f);
 

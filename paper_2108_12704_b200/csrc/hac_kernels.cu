@@ -39,6 +39,8 @@ static int cuda_fail(cudaError_t e, const char* what) {
 struct DevFormat {
     const uint32_t* stream;
     const uint16_t* lut;
+    const uint2* l1;
+    const uint2* sub;
     const float* rank_value;
     const uint64_t* limit;
     const uint32_t* first_left;
@@ -49,10 +51,10 @@ struct DevFormat {
     const uint32_t* seg_first;
     const void* ri;
     const uint32_t* cb;
-    uint32_t n, m, units, G, S, k_eff, lut_bits, max_len, ri_bits, max_unit_chunks;
+    const void* unit_info;
+    uint32_t n, m, units, G, S, k_eff, lut_bits, max_len, ri_bits, max_unit_chunks, l1_bits, sub_bytes;
 };
 
-constexpr int kTableWords = 34;
 
 // ------------------------------------------------------------------------------------------------
 // Shared-memory access by 32-bit shared-space address (keeps address arithmetic in 32 bits).
@@ -80,71 +82,46 @@ __device__ __forceinline__ uint2 lds64(uint32_t a) {
 
 __host__ __device__ inline size_t align16(size_t x) { return (x + 15) & ~(size_t)15; }
 
-// How a kernel lays out its decoding tables in shared memory (chosen by the host per launch).
-//   level 1: 2^l1_bits entries {value bits, length}, 8 bytes each, stored `repl` times interleaved
-//            (entry i of replica r at index i*repl + r) so that lanes r, r+repl, .. read disjoint
-//            banks; length 0 marks a code word longer than l1_bits.
-//   level 2: the format's 16-bit table ((rank << 5) | length) over l2_bits bits, one copy, used only
-//            for code words longer than l1_bits; longer than l2_bits: search by length.
+// How a kernel lays out its decoding tables in shared memory (replication chosen by the host).
+//   level 1: the format's 2^l1_bits entries {value bits, length}, 8 bytes each, stored `repl` times
+//            interleaved (entry i of replica r at index i*repl + r) so that lanes r, r+repl, .. read
+//            disjoint banks.  An entry with the top bit of the second word set stands for a prefix
+//            shared by longer code words: {byte offset of a sub-table, 0x80000000 | b}.
+//   level 2: the sub-tables, one copy, indexed by the next b bits: {value bits, length}, or {0, 0}
+//            for code words longer still, which are found by a search over lengths in global memory.
 struct TablePlan {
-    uint32_t l1_bits, repl_log2, l2_bits, has_l2;
+    uint32_t repl_log2;
 };
 
-__host__ __device__ inline size_t plan_smem_bytes(const TablePlan& tp, uint32_t k_eff) {
-    size_t b = ((size_t)8 << (tp.l1_bits + tp.repl_log2));
-    if (tp.has_l2) b += align16((size_t)2 << tp.l2_bits) + align16((size_t)k_eff * 4) + align16(kTableWords * 8) +
-                        2 * align16(kTableWords * 4);
-    return b;
+__host__ __device__ inline size_t plan_smem_bytes(uint32_t l1_bits, uint32_t repl_log2, uint32_t sub_bytes) {
+    return ((size_t)8 << (l1_bits + repl_log2)) + align16(sub_bytes);
 }
 
-// Per-thread handle on the staged tables (shared-space addresses).
+// Per-thread handle on the staged tables (shared-space addresses) and the global fallbacks.
 struct Decoder {
-    uint32_t l1_lane, l1_mul, l1_shift;
-    uint32_t l2, l2_shift, l2_bits, values, limit, first_left, rank_base, max_len;
+    uint32_t l1_lane, l1_mul, l1_shift, l1_bits, sub;
 };
 
 // Builds the tables in shared memory (whole block takes part) and advances `p` past them.
-__device__ inline Decoder stage_decoder(const DevFormat& f, const TablePlan& tp, unsigned char*& p) {
+__device__ __forceinline__ Decoder stage_decoder(const DevFormat& f, const TablePlan& tp, unsigned char*& p) {
     Decoder d;
     const uint32_t repl = 1u << tp.repl_log2;
     uint2* l1 = reinterpret_cast<uint2*>(p);
-    p += (size_t)8 << (tp.l1_bits + tp.repl_log2);
-    const uint32_t entries = 1u << (tp.l1_bits + tp.repl_log2);
-    const uint32_t widen = f.lut_bits - tp.l1_bits;          // the format's table has >= l1_bits bits
-    for (uint32_t e = threadIdx.x; e < entries; e += blockDim.x) {
-        const uint32_t idx = e >> tp.repl_log2;
-        const uint32_t code = f.lut[(size_t)idx << widen];
-        const uint32_t len = code & 31u;
-        uint2 v = make_uint2(0u, 0u);
-        if (len != 0 && len <= tp.l1_bits) v = make_uint2(__float_as_uint(f.rank_value[code >> 5]), len);
-        l1[e] = v;
+    p += (size_t)8 << (f.l1_bits + tp.repl_log2);
+    uint2* sub = reinterpret_cast<uint2*>(p);
+    p += align16(f.sub_bytes);
+    // one level-1 entry per thread and pass: one global load, then `repl` stores
+    for (uint32_t idx = threadIdx.x; idx < (1u << f.l1_bits); idx += blockDim.x) {
+        const uint2 v = __ldg(f.l1 + idx);
+        uint2* dst = l1 + ((size_t)idx << tp.repl_log2);
+        for (uint32_t r = 0; r < repl; ++r) dst[r] = v;
     }
+    for (uint32_t i = threadIdx.x; i < f.sub_bytes / 8; i += blockDim.x) sub[i] = __ldg(f.sub + i);
     d.l1_lane = smem_addr(l1) + ((threadIdx.x & (repl - 1)) << 3);
     d.l1_mul = 8u << tp.repl_log2;
-    d.l1_shift = 32 - tp.l1_bits;
-    d.l2 = d.values = d.limit = d.first_left = d.rank_base = 0;
-    d.l2_bits = tp.l2_bits; d.l2_shift = 32 - tp.l2_bits; d.max_len = f.max_len;
-    if (tp.has_l2) {
-        uint16_t* l2 = reinterpret_cast<uint16_t*>(p);
-        p += align16((size_t)2 << tp.l2_bits);
-        float* value = reinterpret_cast<float*>(p);
-        p += align16((size_t)f.k_eff * 4);
-        uint64_t* limit = reinterpret_cast<uint64_t*>(p);
-        p += align16(kTableWords * 8);
-        uint32_t* first_left = reinterpret_cast<uint32_t*>(p);
-        p += align16(kTableWords * 4);
-        uint32_t* rank_base = reinterpret_cast<uint32_t*>(p);
-        p += align16(kTableWords * 4);
-        for (uint32_t i = threadIdx.x; i < (1u << tp.l2_bits); i += blockDim.x) l2[i] = f.lut[i];
-        for (uint32_t i = threadIdx.x; i < f.k_eff; i += blockDim.x) value[i] = f.rank_value[i];
-        if (threadIdx.x < kTableWords) {
-            limit[threadIdx.x] = f.limit[threadIdx.x];
-            first_left[threadIdx.x] = f.first_left[threadIdx.x];
-            rank_base[threadIdx.x] = f.rank_base[threadIdx.x];
-        }
-        d.l2 = smem_addr(l2); d.values = smem_addr(value); d.limit = smem_addr(limit);
-        d.first_left = smem_addr(first_left); d.rank_base = smem_addr(rank_base);
-    }
+    d.l1_shift = 32 - f.l1_bits;
+    d.l1_bits = f.l1_bits;
+    d.sub = smem_addr(sub);
     return d;
 }
 
@@ -171,31 +148,39 @@ struct BitReader {
     }
 };
 
-// Code words longer than the level-1 table: level-2 lookup, then the search by length.
-__device__ __noinline__ uint2 decode_long(uint32_t top, const Decoder d) {
-    const uint32_t code = lds16(d.l2 + ((top >> d.l2_shift) << 1));
+// Code words longer than both table levels (rare): the format's full-width 16-bit table, then the
+// search over lengths, all in global memory.
+__device__ __noinline__ uint2 decode_long(uint32_t top, const uint16_t* __restrict__ lut, uint32_t lut_bits,
+                                          const float* __restrict__ rank_value, const uint64_t* __restrict__ limit,
+                                          const uint32_t* __restrict__ first_left,
+                                          const uint32_t* __restrict__ rank_base, uint32_t max_len) {
+    const uint32_t code = lut[top >> (32 - lut_bits)];
     uint32_t len = code & 31u, rank = code >> 5;
     if (len == 0) {
-        len = d.max_len; rank = 0;
-        for (uint32_t l = d.l2_bits + 1; l <= d.max_len; ++l) {
-            const uint32_t lim_lo = lds32(d.limit + l * 8), lim_hi = lds32(d.limit + l * 8 + 4);
-            if (lim_hi != 0 || top < lim_lo) {
+        len = max_len; rank = 0;
+        for (uint32_t l = lut_bits + 1; l <= max_len; ++l) {
+            if ((uint64_t)top < limit[l]) {
                 len = l;
-                rank = lds32(d.rank_base + l * 4) + ((top - lds32(d.first_left + l * 4)) >> (32 - l));
+                rank = rank_base[l] + ((top - first_left[l]) >> (32 - l));
                 break;
             }
         }
     }
-    return make_uint2(lds32(d.values + rank * 4), len);
+    return make_uint2(__float_as_uint(rank_value[rank]), len);
 }
 
 // One code word -> the shared value it stands for.
 template <bool kLong>
-__device__ __forceinline__ float decode_value(BitReader& br, const Decoder& d) {
+__device__ __forceinline__ float decode_value(BitReader& br, const Decoder& d, const DevFormat& f) {
     const uint32_t top = br.peek();
     uint2 e = lds64(d.l1_lane + (top >> d.l1_shift) * d.l1_mul);
     if (kLong) {
-        if (e.y == 0) e = decode_long(top, d);
+        if ((int32_t)e.y < 0) {
+            const uint32_t q = (top << d.l1_bits) >> (32 - (e.y & 31u));
+            e = lds64(d.sub + e.x + (q << 3));
+            if (e.y == 0)
+                e = decode_long(top, f.lut, f.lut_bits, f.rank_value, f.limit, f.first_left, f.rank_base, f.max_len);
+        }
     }
     br.skip(e.y);
     return __uint_as_float(e.x);
@@ -244,6 +229,16 @@ __global__ void __launch_bounds__(1024) hac_vec_kernel(DevFormat f, TablePlan tp
                                                        int64_t xs_i, float* __restrict__ y, int64_t ys_j,
                                                        float* __restrict__ aux) {
     extern __shared__ __align__(16) unsigned char smem[];
+    const uint32_t warp = threadIdx.x >> 5, lane = threadIdx.x & 31, warps = blockDim.x >> 5;
+    // index entries of this warp's first segment: requested before the tables are staged so that
+    // the two trips to memory overlap
+    uint32_t u = blockIdx.x + gridDim.x * warp;
+    uint32_t my_bits = 0;
+    uint64_t seg_bit = 0;
+    if (u < f.units) {
+        my_bits = __ldg(f.sub_bits + (size_t)u * 32 + lane);
+        seg_bit = __ldg(f.seg_bit_off + u);
+    }
     unsigned char* p = smem;
     const Decoder dec = stage_decoder(f, tp, p);
     const uint32_t pad = (f.S & 1u) ? 0u : 1u;
@@ -252,37 +247,43 @@ __global__ void __launch_bounds__(1024) hac_vec_kernel(DevFormat f, TablePlan tp
         for (uint32_t i = threadIdx.x; i < f.n; i += blockDim.x) xs[i + pad * (i / f.S)] = x[(int64_t)i * xs_i];
         p += align16(((size_t)f.n + (f.n / f.S + 1) * pad) * 4);
     }
-    const uint32_t warp = threadIdx.x >> 5, lane = threadIdx.x & 31, warps = blockDim.x >> 5;
     uint4* stage = reinterpret_cast<uint4*>(p) + (size_t)warp * f.max_unit_chunks;
     const uint32_t stage_a = smem_addr(stage);
     const uint32_t xs_a = smem_addr(xs);
+    uint32_t total = 0, start = 0, base = 0;
+    if (u < f.units) {
+        start = lane_start_bits(my_bits, lane, total);
+        base = stage_span(f, seg_bit, total, stage, lane);
+    }
     __syncthreads();
 
-    for (uint32_t u = blockIdx.x * warps + warp; u < f.units; u += gridDim.x * warps) {
+    while (u < f.units) {
         const uint32_t j = u / f.G, g = u - j * f.G;
-        const uint32_t my_bits = f.sub_bits[(size_t)u * 32 + lane];
-        uint32_t total;
-        const uint32_t start = lane_start_bits(my_bits, lane, total);
-        const uint32_t base = stage_span(f, f.seg_bit_off[u], total, stage, lane);
         const uint32_t sub = g * 32 + lane;                 // sub-segment number inside the column
         const uint32_t row0 = sub * f.S;
         const uint32_t count = row0 < f.n ? min(f.S, f.n - row0) : 0u;
         BitReader br;
         br.init(stage_a, base + start);
+        // index entries of the next segment, in flight while this one is decoded
+        const uint32_t un = u + gridDim.x * warps;
+        if (un < f.units) {
+            my_bits = __ldg(f.sub_bits + (size_t)un * 32 + lane);
+            seg_bit = __ldg(f.seg_bit_off + un);
+        }
         if (kMode == 0) {
             float acc = 0.0f;
             if (kXShared) {
                 uint32_t xa = xs_a + ((row0 + pad * sub) << 2);
 #pragma unroll 4
                 for (uint32_t s = 0; s < count; ++s) {
-                    const float w = decode_value<kLong>(br, dec);
+                    const float w = decode_value<kLong>(br, dec, f);
                     acc = fmaf(ldsf_v(xa), w, acc);
                     xa += 4;
                 }
             } else {
                 const float* xl = x + (int64_t)row0 * xs_i;
                 for (uint32_t s = 0; s < count; ++s) {
-                    const float w = decode_value<kLong>(br, dec);
+                    const float w = decode_value<kLong>(br, dec, f);
                     acc = fmaf(xl[(int64_t)s * xs_i], w, acc);
                 }
             }
@@ -293,10 +294,30 @@ __global__ void __launch_bounds__(1024) hac_vec_kernel(DevFormat f, TablePlan tp
             }
         } else {
             float* out = aux + (size_t)j * f.n + row0;
-            for (uint32_t s = 0; s < count; ++s) out[s] = decode_value<kLong>(br, dec);
+            for (uint32_t s = 0; s < count; ++s) out[s] = decode_value<kLong>(br, dec, f);
         }
         __syncwarp();
+        u = un;
+        if (u < f.units) {
+            start = lane_start_bits(my_bits, lane, total);
+            base = stage_span(f, seg_bit, total, stage, lane);
+        }
     }
+}
+
+// Per-segment record of sHAC (derived at upload from cb, seg_first, seg_col): where the segment's
+// entries start in nz / ri, how many there are, its column, and whether it is the column's only one.
+struct ShacUnit {
+    uint64_t bit_off;
+    uint32_t pos0, count, col, single;
+};
+
+__device__ __forceinline__ ShacUnit load_unit(const ShacUnit* q) {     // records are 8-byte aligned
+    const uint2* w = reinterpret_cast<const uint2*>(q);
+    const uint2 a = __ldg(w), b = __ldg(w + 1), c = __ldg(w + 2);
+    ShacUnit r;
+    r.bit_off = ((uint64_t)a.y << 32) | a.x; r.pos0 = b.x; r.count = b.y; r.col = c.x; r.single = c.y;
+    return r;
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -309,6 +330,15 @@ __global__ void __launch_bounds__(1024) shac_vec_kernel(DevFormat f, TablePlan t
                                                         int64_t xs_i, float* __restrict__ y, int64_t ys_j,
                                                         float* __restrict__ aux) {
     extern __shared__ __align__(16) unsigned char smem[];
+    const uint32_t warp = threadIdx.x >> 5, lane = threadIdx.x & 31, warps = blockDim.x >> 5;
+    const ShacUnit* __restrict__ units = reinterpret_cast<const ShacUnit*>(f.unit_info);
+    uint32_t u = blockIdx.x + gridDim.x * warp;
+    uint32_t my_bits = 0;
+    ShacUnit info = {0, 0, 0, 0, 0};
+    if (u < f.units) {
+        my_bits = __ldg(f.sub_bits + (size_t)u * 32 + lane);
+        info = load_unit(units + u);
+    }
     unsigned char* p = smem;
     const Decoder dec = stage_decoder(f, tp, p);
     float* xs = reinterpret_cast<float*>(p);
@@ -316,61 +346,66 @@ __global__ void __launch_bounds__(1024) shac_vec_kernel(DevFormat f, TablePlan t
         for (uint32_t i = threadIdx.x; i < f.n; i += blockDim.x) xs[i] = x[(int64_t)i * xs_i];
         p += align16((size_t)f.n * 4);
     }
-    const uint32_t warp = threadIdx.x >> 5, lane = threadIdx.x & 31, warps = blockDim.x >> 5;
     uint4* stage = reinterpret_cast<uint4*>(p) + (size_t)warp * f.max_unit_chunks;
     p += align16((size_t)warps * f.max_unit_chunks * 16);
     // row-index staging: 32*S entries plus up to 16 bytes of misalignment, per warp
     const uint32_t ri_chunks = (32u * f.S * (uint32_t)sizeof(RowT) + 15u) / 16u + 1u;
     uint4* ri_stage = reinterpret_cast<uint4*>(p) + (size_t)warp * ri_chunks;
     const uint32_t stage_a = smem_addr(stage), ri_a = smem_addr(ri_stage), xs_a = smem_addr(xs);
-    __syncthreads();
     const RowT* __restrict__ ri = reinterpret_cast<const RowT*>(f.ri);
 
-    for (uint32_t u = blockIdx.x * warps + warp; u < f.units; u += gridDim.x * warps) {
-        const uint32_t j = f.seg_col[u];
-        const uint32_t first = f.seg_first[j];
-        const uint32_t g = u - first;
-        const uint32_t col_end = f.cb[j + 1];
-        const uint32_t my_bits = f.sub_bits[(size_t)u * 32 + lane];
+    // copies the segment's slice of ri and its span of the stream to shared memory
+    auto fetch = [&](const ShacUnit& un, uint32_t bits, uint32_t& start, uint32_t& base, uint32_t& ri_lane) {
         uint32_t total;
-        const uint32_t start = lane_start_bits(my_bits, lane, total);
-        const uint32_t seg_pos0 = f.cb[j] + g * 32 * f.S;
-        const uint32_t seg_count = min(32u * f.S, col_end - seg_pos0);
-        uint32_t ri_lane = 0;
+        start = lane_start_bits(bits, lane, total);
         if (kMode == 0) {
-            // stage ri[seg_pos0 .. seg_pos0 + seg_count) from the enclosing 16-byte chunks
-            const uintptr_t byte0 = reinterpret_cast<uintptr_t>(ri + seg_pos0);
+            const uintptr_t byte0 = reinterpret_cast<uintptr_t>(ri + un.pos0);
             const uintptr_t chunk0 = byte0 & ~(uintptr_t)15;
-            const uint32_t chunks = (uint32_t)((byte0 + (uintptr_t)seg_count * sizeof(RowT) - chunk0 + 15) >> 4);
+            const uint32_t chunks = (uint32_t)((byte0 + (uintptr_t)un.count * sizeof(RowT) - chunk0 + 15) >> 4);
             const uint4* src = reinterpret_cast<const uint4*>(chunk0);
             for (uint32_t c = lane; c < chunks; c += 32) ri_stage[c] = __ldg(src + c);
             ri_lane = ri_a + (uint32_t)(byte0 - chunk0) + lane * f.S * (uint32_t)sizeof(RowT);
         }
-        const uint32_t base = stage_span(f, f.seg_bit_off[u], total, stage, lane);   // ends with __syncwarp
-        const uint32_t pos0 = seg_pos0 + lane * f.S;
-        const uint32_t count = pos0 < col_end ? min(f.S, col_end - pos0) : 0u;
+        base = stage_span(f, un.bit_off, total, stage, lane);       // ends with __syncwarp
+    };
+    uint32_t start = 0, base = 0, ri_lane = 0;
+    if (u < f.units) fetch(info, my_bits, start, base, ri_lane);
+    __syncthreads();
+
+    while (u < f.units) {
+        const ShacUnit cur = info;
+        const uint32_t lane_pos = lane * f.S;
+        const uint32_t count = lane_pos < cur.count ? min(f.S, cur.count - lane_pos) : 0u;
         BitReader br;
         br.init(stage_a, base + start);
+        const uint32_t un = u + gridDim.x * warps;
+        if (un < f.units) {
+            my_bits = __ldg(f.sub_bits + (size_t)un * 32 + lane);
+            info = load_unit(units + un);
+        }
         if (kMode == 0) {
             float acc = 0.0f;
+            uint32_t ra = ri_lane;
 #pragma unroll 4
             for (uint32_t s = 0; s < count; ++s) {
-                const float w = decode_value<kLong>(br, dec);
-                const uint32_t row = sizeof(RowT) == 2 ? lds16_v(ri_lane) : lds32_v(ri_lane);
-                ri_lane += sizeof(RowT);
+                const float w = decode_value<kLong>(br, dec, f);
+                const uint32_t row = sizeof(RowT) == 2 ? lds16_v(ra) : lds32_v(ra);
+                ra += sizeof(RowT);
                 const float xv = kXShared ? ldsf_v(xs_a + (row << 2)) : x[(int64_t)row * xs_i];
                 acc = fmaf(xv, w, acc);
             }
             acc = warp_sum(acc);
             if (lane == 0) {
-                const bool single = (f.seg_first[j + 1] - first) == 1;
-                if (single) y[(int64_t)j * ys_j] = acc;
+                if (cur.single) y[(int64_t)cur.col * ys_j] = acc;
                 else aux[u] = acc;
             }
         } else {
-            for (uint32_t s = 0; s < count; ++s) aux[pos0 + s] = decode_value<kLong>(br, dec);
+            float* out = aux + cur.pos0 + lane_pos;
+            for (uint32_t s = 0; s < count; ++s) out[s] = decode_value<kLong>(br, dec, f);
         }
         __syncwarp();
+        u = un;
+        if (u < f.units) fetch(info, my_bits, start, base, ri_lane);
     }
 }
 
@@ -453,7 +488,7 @@ __global__ void __launch_bounds__(1024) hac_batch_kernel(DevFormat f, TablePlan 
 #pragma unroll
             for (int s = 0; s < kBatchSteps; ++s) {
                 float v = 0.0f;
-                if (s0 + s < count) v = decode_value<true>(br, dec);
+                if (s0 + s < count) v = decode_value<true>(br, dec, f);
                 wt[warp * kBatchRows + lane * kBatchSteps + s] = v;
             }
             // matching rows of X: tile row r = l*kBatchSteps + s  <->  matrix row (g*32+l)*S + s0 + s
@@ -544,7 +579,7 @@ __global__ void __launch_bounds__(1024) shac_batch_kernel(DevFormat f, TablePlan
                 float v = 0.0f;
                 uint32_t row = 0;
                 if (s0 + s < count) {
-                    v = decode_value<true>(br, dec);
+                    v = decode_value<true>(br, dec, f);
                     row = ri[pos0 + s0 + s];
                 }
                 wv[lane * kBatchSteps + s] = v;
@@ -611,9 +646,11 @@ static int device_info(DeviceInfo& d) {
 static DevFormat dev_format(const Format& f) {
     DevFormat d{};
     d.stream = f.dev.stream; d.lut = f.dev.lut; d.rank_value = f.dev.rank_value;
+    d.l1 = reinterpret_cast<const uint2*>(f.dev.l1); d.sub = reinterpret_cast<const uint2*>(f.dev.sub);
+    d.l1_bits = (uint32_t)f.tables.l1_bits; d.sub_bytes = (uint32_t)(f.tables.sub.size() * 4);
     d.limit = f.dev.limit; d.first_left = f.dev.first_left; d.rank_base = f.dev.rank_base;
     d.seg_bit_off = f.dev.seg_bit_off; d.sub_bits = f.dev.sub_bits; d.seg_col = f.dev.seg_col;
-    d.seg_first = f.dev.seg_first; d.ri = f.dev.ri; d.cb = f.dev.cb;
+    d.seg_first = f.dev.seg_first; d.ri = f.dev.ri; d.cb = f.dev.cb; d.unit_info = f.dev.unit_info;
     d.n = (uint32_t)f.n; d.m = (uint32_t)f.m; d.units = (uint32_t)f.seg_bit_off.size();
     d.G = f.G ? f.G : 1; d.S = f.S; d.k_eff = (uint32_t)f.codebook.size();
     d.lut_bits = (uint32_t)f.tables.lut_bits; d.max_len = f.max_len; d.ri_bits = f.ri_bits;
@@ -627,6 +664,8 @@ static void set_pointers(Format& f, void* dev_buf, size_t bytes) {
     f.dev.base = dev_buf; f.dev.bytes = bytes;
     f.dev.stream = reinterpret_cast<const uint32_t*>(b + L.stream);
     f.dev.lut = reinterpret_cast<const uint16_t*>(b + L.lut);
+    f.dev.l1 = reinterpret_cast<const uint2_host*>(b + L.l1);
+    f.dev.sub = reinterpret_cast<const uint2_host*>(b + L.sub);
     f.dev.rank_value = reinterpret_cast<const float*>(b + L.rank_value);
     f.dev.limit = reinterpret_cast<const uint64_t*>(b + L.limit);
     f.dev.first_left = reinterpret_cast<const uint32_t*>(b + L.first_left);
@@ -637,6 +676,7 @@ static void set_pointers(Format& f, void* dev_buf, size_t bytes) {
     f.dev.seg_first = reinterpret_cast<const uint32_t*>(b + L.seg_first);
     f.dev.ri = b + L.ri;
     f.dev.cb = reinterpret_cast<const uint32_t*>(b + L.cb);
+    f.dev.unit_info = b + L.unit_info;
 }
 
 static int upload(Format& f, void* dev_buf, size_t dev_bytes, void* stream_) {
@@ -652,6 +692,8 @@ static int upload(Format& f, void* dev_buf, size_t dev_bytes, void* stream_) {
     HAC_CUDA(cudaMemsetAsync(dev_buf, 0, L.total, st));
     HAC_CUDA(put(L.stream, f.stream.data(), f.stream.size() * 4));
     HAC_CUDA(put(L.lut, f.tables.lut.data(), f.tables.lut.size() * 2));
+    HAC_CUDA(put(L.l1, f.tables.l1.data(), f.tables.l1.size() * 4));
+    HAC_CUDA(put(L.sub, f.tables.sub.data(), f.tables.sub.size() * 4));
     HAC_CUDA(put(L.rank_value, f.tables.rank_value.data(), f.tables.rank_value.size() * 4));
     HAC_CUDA(put(L.limit, f.tables.limit, sizeof(f.tables.limit)));
     HAC_CUDA(put(L.first_left, f.tables.first_left, sizeof(f.tables.first_left)));
@@ -663,6 +705,7 @@ static int upload(Format& f, void* dev_buf, size_t dev_bytes, void* stream_) {
     if (f.ri_bits == 16) HAC_CUDA(put(L.ri, f.ri16.data(), f.ri16.size() * 2));
     else HAC_CUDA(put(L.ri, f.ri32.data(), f.ri32.size() * 4));
     HAC_CUDA(put(L.cb, f.cb.data(), f.cb.size() * 4));
+    HAC_CUDA(put(L.unit_info, f.unit_info.data(), f.unit_info.size() * 4));
     // the source vectors are pageable host memory: wait so they may change or go away afterwards
     HAC_CUDA(cudaStreamSynchronize(st));
     set_pointers(f, dev_buf, dev_bytes);
@@ -715,15 +758,11 @@ static int launch_finalize(const Format& f, const DevFormat& d, const float* par
     return HAC_OK;
 }
 
-// Table plan: level-1 width and replication that fit `table_budget` bytes of shared memory.
-static TablePlan plan_tables(const DevFormat& d, size_t table_budget, int max_l1) {
+// Table plan: the widest replication (at most 16 copies) of the level-1 table that fits.
+static TablePlan plan_tables(const DevFormat& d, size_t table_budget) {
     TablePlan tp{};
-    tp.l2_bits = d.lut_bits;
-    tp.l1_bits = std::min<uint32_t>(d.lut_bits, (uint32_t)max_l1);
     tp.repl_log2 = 4;
-    while (tp.repl_log2 > 0 && ((size_t)8 << (tp.l1_bits + tp.repl_log2)) > table_budget) tp.repl_log2--;
-    while (tp.l1_bits > 1 && ((size_t)8 << (tp.l1_bits + tp.repl_log2)) > table_budget) tp.l1_bits--;
-    tp.has_l2 = d.max_len > tp.l1_bits ? 1u : 0u;
+    while (tp.repl_log2 > 0 && plan_smem_bytes(d.l1_bits, tp.repl_log2, d.sub_bytes) > table_budget) tp.repl_log2--;
     return tp;
 }
 
@@ -757,31 +796,27 @@ static int launch_vec(const Format& f, int mode, const float* x, int64_t xs_i, f
     size_t xbytes = 0;
     if (mode == 0) xbytes = f.sparse ? align16((size_t)f.n * 4) : align16(((size_t)f.n + (f.n / f.S + 1)) * 4);
     const int want = std::min(32, std::max(1, env_int("HAC_B200_VEC_WARPS", 32)));
-    const int max_l1 = std::min(12, std::max(1, env_int("HAC_B200_L1_BITS", 10)));
-    // shared memory: tables + x + per-warp staging.  Prefer keeping x and all warps; shrink the
-    // level-1 table (fewer replicas, then fewer bits) before giving up warps.
+    // shared memory: tables + x + per-warp staging.  Prefer keeping x and all warps; give up
+    // replicas of the level-1 table before giving up warps.
     bool x_shared = mode == 0;
-    const size_t min_tables = 4096;
+    const size_t min_tables = plan_smem_bytes(d.l1_bits, 0, d.sub_bytes);
     if (x_shared && xbytes + min_tables + per_warp * std::min(want, 8) > budget) { x_shared = false; xbytes = 0; }
     int warps = want;
     while (warps > 1 && xbytes + min_tables + per_warp * (size_t)warps > budget) --warps;
     if (xbytes + min_tables + per_warp * (size_t)warps > budget) return HAC_ERR_BUFFER_TOO_SMALL;
-    const size_t aux_tables = align16((size_t)2 << d.lut_bits) + align16((size_t)d.k_eff * 4) + 1024;
-    size_t table_budget = budget - xbytes - per_warp * (size_t)warps;
-    table_budget = table_budget > aux_tables + 1024 ? table_budget - aux_tables : 1024;
-    table_budget = std::min<size_t>(table_budget, (size_t)128 * 1024);
-    const TablePlan tp = plan_tables(d, table_budget, max_l1);
-    const size_t smem = plan_smem_bytes(tp, d.k_eff) + xbytes + per_warp * warps;
+    const TablePlan tp = plan_tables(d, budget - xbytes - per_warp * (size_t)warps);
+    const size_t smem = plan_smem_bytes(d.l1_bits, tp.repl_log2, d.sub_bytes) + xbytes + per_warp * warps;
     if (smem > budget) return HAC_ERR_BUFFER_TOO_SMALL;
+    const bool has_long = d.max_len > d.l1_bits;
     const int threads = warps * 32;
-    VecKernel kernel = tp.has_l2 ? pick_vec_kernel<true>(f, mode, x_shared) : pick_vec_kernel<false>(f, mode, x_shared);
+    VecKernel kernel = has_long ? pick_vec_kernel<true>(f, mode, x_shared) : pick_vec_kernel<false>(f, mode, x_shared);
     rc = prepare_kernel(kernel, smem);
     if (rc) return rc;
     int per_sm = 1;
     HAC_CUDA(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kernel, threads, smem));
     per_sm = std::max(per_sm, 1);
-    const unsigned need = (d.units + warps - 1) / warps;
-    const unsigned grid = std::min<unsigned>(need, (unsigned)(di.sms * per_sm));
+    // spread the segments over all SMs (a block's warps take segments blockIdx + k * gridDim)
+    const unsigned grid = std::min<unsigned>(d.units, (unsigned)(di.sms * per_sm));
     kernel<<<grid, threads, smem, st>>>(d, tp, x, xs_i, y, ys_j, aux);
     HAC_CUDA(cudaGetLastError());
     f.last_launches++;
@@ -793,8 +828,8 @@ static int launch_batch_t(const Format& f, const DeviceInfo& di, const DevFormat
                           int64_t xs_b, int64_t batch, float* y, int64_t ys_j, int64_t ys_b, float* partial,
                           cudaStream_t st) {
     const size_t budget = (size_t)di.max_smem_optin;
-    const TablePlan tp = plan_tables(d, 32 * 1024, 10);
-    const size_t tab = plan_smem_bytes(tp, d.k_eff);
+    const TablePlan tp = plan_tables(d, std::max<size_t>(32 * 1024, plan_smem_bytes(d.l1_bits, 0, d.sub_bytes)));
+    const size_t tab = plan_smem_bytes(d.l1_bits, tp.repl_log2, d.sub_bytes);
     constexpr uint32_t kTile = 32 * kAcc;
     const uint32_t batch_tiles = (uint32_t)((batch + kTile - 1) / kTile);
     int rc;
