@@ -57,28 +57,19 @@ struct DevFormat {
 
 
 // ------------------------------------------------------------------------------------------------
-// Shared-memory access by 32-bit shared-space address (keeps address arithmetic in 32 bits).
-// The *_v forms are volatile: they read staging areas that are rewritten between segments.
+// All shared memory is one dynamic array; tables and staging areas are addressed by 32-bit byte
+// offsets into it, which keeps address arithmetic in 32 bits and lets the compiler schedule the
+// loads freely between the warp- and block-level barriers.
 // ------------------------------------------------------------------------------------------------
-__device__ __forceinline__ uint32_t smem_addr(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
-__device__ __forceinline__ uint32_t lds32(uint32_t a) {
-    uint32_t v; asm("ld.shared.u32 %0, [%1];" : "=r"(v) : "r"(a)); return v;
+extern __shared__ __align__(16) unsigned char smem[];
+
+__device__ __forceinline__ uint32_t smem_off(const void* p) {
+    return (uint32_t)(reinterpret_cast<const unsigned char*>(p) - smem);
 }
-__device__ __forceinline__ uint32_t lds32_v(uint32_t a) {
-    uint32_t v; asm volatile("ld.shared.u32 %0, [%1];" : "=r"(v) : "r"(a) : "memory"); return v;
-}
-__device__ __forceinline__ uint32_t lds16(uint32_t a) {
-    uint16_t v; asm("ld.shared.u16 %0, [%1];" : "=h"(v) : "r"(a)); return v;
-}
-__device__ __forceinline__ uint32_t lds16_v(uint32_t a) {
-    uint16_t v; asm volatile("ld.shared.u16 %0, [%1];" : "=h"(v) : "r"(a) : "memory"); return v;
-}
-__device__ __forceinline__ float ldsf_v(uint32_t a) {
-    float v; asm volatile("ld.shared.f32 %0, [%1];" : "=f"(v) : "r"(a) : "memory"); return v;
-}
-__device__ __forceinline__ uint2 lds64(uint32_t a) {
-    uint2 v; asm("ld.shared.v2.u32 {%0, %1}, [%2];" : "=r"(v.x), "=r"(v.y) : "r"(a)); return v;
-}
+__device__ __forceinline__ uint32_t lds32(uint32_t off) { return *reinterpret_cast<const uint32_t*>(smem + off); }
+__device__ __forceinline__ uint32_t lds16(uint32_t off) { return *reinterpret_cast<const uint16_t*>(smem + off); }
+__device__ __forceinline__ float ldsf(uint32_t off) { return *reinterpret_cast<const float*>(smem + off); }
+__device__ __forceinline__ uint2 lds64(uint32_t off) { return *reinterpret_cast<const uint2*>(smem + off); }
 
 __host__ __device__ inline size_t align16(size_t x) { return (x + 15) & ~(size_t)15; }
 
@@ -110,18 +101,30 @@ __device__ __forceinline__ Decoder stage_decoder(const DevFormat& f, const Table
     p += (size_t)8 << (f.l1_bits + tp.repl_log2);
     uint2* sub = reinterpret_cast<uint2*>(p);
     p += align16(f.sub_bytes);
-    // one level-1 entry per thread and pass: one global load, then `repl` stores
-    for (uint32_t idx = threadIdx.x; idx < (1u << f.l1_bits); idx += blockDim.x) {
-        const uint2 v = __ldg(f.l1 + idx);
-        uint2* dst = l1 + ((size_t)idx << tp.repl_log2);
-        for (uint32_t r = 0; r < repl; ++r) dst[r] = v;
+    // Each thread loads one entry; the warp then writes its 32 entries' replicas slot by slot, the
+    // value for a slot fetched from the lane that holds it, so that consecutive lanes write
+    // consecutive 8-byte slots (no bank conflicts) and every entry is read from memory once.
+    const uint32_t lane_ = threadIdx.x & 31u;
+    for (uint32_t idx0 = threadIdx.x - lane_; idx0 < (1u << f.l1_bits); idx0 += blockDim.x) {
+        const uint32_t idx = idx0 + lane_;
+        uint2 v = make_uint2(0u, 0u);
+        if (idx < (1u << f.l1_bits)) v = __ldg(f.l1 + idx);
+        uint2* dst = l1 + ((size_t)idx0 << tp.repl_log2);
+        const uint32_t warp_slots = min(32u, (1u << f.l1_bits) - idx0) << tp.repl_log2;
+        for (uint32_t s0 = 0; s0 < warp_slots; s0 += 32) {
+            const uint32_t src = (s0 + lane_) >> tp.repl_log2;
+            uint2 w;
+            w.x = __shfl_sync(0xffffffffu, v.x, src & 31u);
+            w.y = __shfl_sync(0xffffffffu, v.y, src & 31u);
+            if (s0 + lane_ < warp_slots) dst[s0 + lane_] = w;
+        }
     }
     for (uint32_t i = threadIdx.x; i < f.sub_bytes / 8; i += blockDim.x) sub[i] = __ldg(f.sub + i);
-    d.l1_lane = smem_addr(l1) + ((threadIdx.x & (repl - 1)) << 3);
+    d.l1_lane = smem_off(l1) + ((threadIdx.x & (repl - 1)) << 3);
     d.l1_mul = 8u << tp.repl_log2;
     d.l1_shift = 32 - f.l1_bits;
     d.l1_bits = f.l1_bits;
-    d.sub = smem_addr(sub);
+    d.sub = smem_off(sub);
     return d;
 }
 
@@ -131,8 +134,8 @@ struct BitReader {
     uint32_t hi, lo, off, next;
     __device__ __forceinline__ void init(uint32_t stage_addr, uint32_t bitpos) {
         const uint32_t a = stage_addr + ((bitpos >> 5) << 2);
-        hi = lds32_v(a);
-        lo = lds32_v(a + 4);
+        hi = lds32(a);
+        lo = lds32(a + 4);
         off = bitpos & 31u;
         next = a + 8;
     }
@@ -141,7 +144,7 @@ struct BitReader {
         off += len;
         if (off >= 32u) {
             hi = lo;
-            lo = lds32_v(next);
+            lo = lds32(next);
             next += 4;
             off -= 32u;
         }
@@ -186,6 +189,80 @@ __device__ __forceinline__ float decode_value(BitReader& br, const Decoder& d, c
     return __uint_as_float(e.x);
 }
 
+// ------------------------------------------------------------------------------------------------
+// Hand-scheduled decode step (PTX).  One step of one chain is split in two parts so that the parts
+// of several chains can be interleaved in program order:
+//   lookup : window -> level-1 entry                      (4 instructions)
+//   consume: advance the window by the code length, refill it from the staged span when 32 bits
+//            are used up, multiply-accumulate with x       (9 instructions)
+// Shared memory is addressed by absolute 32-bit shared-space addresses here.
+// ------------------------------------------------------------------------------------------------
+struct FastReader {
+    uint32_t hi, lo, off, next;          // next: shared address of the word after lo
+};
+
+__device__ __forceinline__ uint32_t shared_base() { return (uint32_t)__cvta_generic_to_shared(smem); }
+
+__device__ __forceinline__ void fast_lookup(const FastReader& r, uint32_t l1_shift, uint32_t l1_mul, uint32_t l1_lane,
+                                            uint32_t& top, uint32_t& val, uint32_t& len) {
+    asm volatile(
+        "{\n\t"
+        ".reg .b32 i;\n\t"
+        "shf.l.wrap.b32 %0, %3, %4, %5;\n\t"
+        "shr.u32 i, %0, %6;\n\t"
+        "mad.lo.u32 i, i, %7, %8;\n\t"
+        "ld.shared.v2.u32 {%1, %2}, [i];\n\t"
+        "}"
+        : "=r"(top), "=r"(val), "=r"(len)
+        : "r"(r.lo), "r"(r.hi), "r"(r.off), "r"(l1_shift), "r"(l1_mul), "r"(l1_lane)
+        : "memory");
+}
+
+template <int kXOffset>
+__device__ __forceinline__ void fast_consume(FastReader& r, uint32_t val, uint32_t len, uint32_t x_addr, float& acc) {
+    asm volatile(
+        "{\n\t"
+        ".reg .pred p;\n\t"
+        ".reg .f32 xv;\n\t"
+        "ld.shared.f32 xv, [%7+%8];\n\t"
+        "add.u32 %2, %2, %6;\n\t"
+        "setp.ge.u32 p, %2, 32;\n\t"
+        "@p mov.u32 %0, %1;\n\t"
+        "@p ld.shared.u32 %1, [%3];\n\t"
+        "@p add.u32 %3, %3, 4;\n\t"
+        "and.b32 %2, %2, 31;\n\t"
+        "fma.rn.f32 %4, xv, %5, %4;\n\t"
+        "}"
+        : "+r"(r.hi), "+r"(r.lo), "+r"(r.off), "+r"(r.next), "+f"(acc)
+        : "f"(__uint_as_float(val)), "r"(len), "r"(x_addr), "n"(kXOffset)
+        : "memory");
+}
+
+// Level-1 entry that stands for a prefix of longer code words: sub-table, then the search.
+__device__ __forceinline__ void resolve_long(uint32_t top, const Decoder& d, const DevFormat& f, uint32_t& val,
+                                             uint32_t& len) {
+    const uint32_t q = (top << d.l1_bits) >> (32 - (len & 31u));
+    uint2 e = lds64(d.sub + val + (q << 3));
+    if (e.y == 0) e = decode_long(top, f.lut, f.lut_bits, f.rank_value, f.limit, f.first_left, f.rank_base, f.max_len);
+    val = e.x; len = e.y;
+}
+
+// One step of kChains chains: lookups first, then the consumes, so that the table loads overlap.
+template <bool kLong, int kChains, int kXOffset>
+__device__ __forceinline__ void fast_step(FastReader (&r)[kChains], const Decoder& d, const DevFormat& f,
+                                          uint32_t l1_lane_abs, const uint32_t (&xa)[kChains], float (&acc)[kChains]) {
+    uint32_t top[kChains], val[kChains], len[kChains];
+#pragma unroll
+    for (int c = 0; c < kChains; ++c) fast_lookup(r[c], d.l1_shift, d.l1_mul, l1_lane_abs, top[c], val[c], len[c]);
+    if (kLong) {
+#pragma unroll
+        for (int c = 0; c < kChains; ++c)
+            if ((int32_t)len[c] < 0) resolve_long(top[c], d, f, val[c], len[c]);
+    }
+#pragma unroll
+    for (int c = 0; c < kChains; ++c) fast_consume<kXOffset>(r[c], val[c], len[c], xa[c], acc[c]);
+}
+
 // Start bit of each lane's sub-segment inside the segment (exclusive scan of the 32 lengths by
 // shuffles) and the segment's total bit length.
 __device__ __forceinline__ uint32_t lane_start_bits(uint32_t my_bits, uint32_t lane, uint32_t& total) {
@@ -224,84 +301,157 @@ __device__ __forceinline__ float warp_sum(float v) {
 // keeps the 32 lanes on distinct banks.
 //   kMode 0: product; 1: debug decode (values written to out[j*n + i]).
 // ------------------------------------------------------------------------------------------------
-template <int kMode, bool kXShared, bool kLong>
+template <int kMode, bool kXShared, bool kLong, int kChains>
 __global__ void __launch_bounds__(1024) hac_vec_kernel(DevFormat f, TablePlan tp, const float* __restrict__ x,
                                                        int64_t xs_i, float* __restrict__ y, int64_t ys_j,
                                                        float* __restrict__ aux) {
-    extern __shared__ __align__(16) unsigned char smem[];
+    // A warp works on kChains consecutive segments at a time (an "item"); every lane then runs
+    // kChains independent decode chains, which hides the latency of the dependent table lookups.
     const uint32_t warp = threadIdx.x >> 5, lane = threadIdx.x & 31, warps = blockDim.x >> 5;
-    // index entries of this warp's first segment: requested before the tables are staged so that
-    // the two trips to memory overlap
-    uint32_t u = blockIdx.x + gridDim.x * warp;
-    uint32_t my_bits = 0;
-    uint64_t seg_bit = 0;
-    if (u < f.units) {
-        my_bits = __ldg(f.sub_bits + (size_t)u * 32 + lane);
-        seg_bit = __ldg(f.seg_bit_off + u);
+    const uint32_t items = (f.units + kChains - 1) / kChains;
+    // index entries of this warp's first item: requested before the tables are staged so that the
+    // trips to memory overlap
+    uint32_t item = blockIdx.x + gridDim.x * warp;
+    uint32_t my_bits[kChains];
+    uint64_t seg_bit[kChains];
+#pragma unroll
+    for (int c = 0; c < kChains; ++c) {
+        const uint32_t u = item * kChains + c;
+        my_bits[c] = 0; seg_bit[c] = 0;
+        if (item < items && u < f.units) {
+            my_bits[c] = __ldg(f.sub_bits + (size_t)u * 32 + lane);
+            seg_bit[c] = __ldg(f.seg_bit_off + u);
+        }
     }
     unsigned char* p = smem;
     const Decoder dec = stage_decoder(f, tp, p);
     const uint32_t pad = (f.S & 1u) ? 0u : 1u;
     float* xs = reinterpret_cast<float*>(p);
     if (kMode == 0 && kXShared) {
-        for (uint32_t i = threadIdx.x; i < f.n; i += blockDim.x) xs[i + pad * (i / f.S)] = x[(int64_t)i * xs_i];
+#pragma unroll 4
+        for (uint32_t i = threadIdx.x; i < f.n; i += blockDim.x) xs[i + pad * (i / f.S)] = __ldg(x + (int64_t)i * xs_i);
         p += align16(((size_t)f.n + (f.n / f.S + 1) * pad) * 4);
     }
-    uint4* stage = reinterpret_cast<uint4*>(p) + (size_t)warp * f.max_unit_chunks;
-    const uint32_t stage_a = smem_addr(stage);
-    const uint32_t xs_a = smem_addr(xs);
-    uint32_t total = 0, start = 0, base = 0;
-    if (u < f.units) {
-        start = lane_start_bits(my_bits, lane, total);
-        base = stage_span(f, seg_bit, total, stage, lane);
-    }
+    uint4* stage = reinterpret_cast<uint4*>(p) + (size_t)warp * kChains * f.max_unit_chunks;
+    const uint32_t stage_a = smem_off(stage);
+    const uint32_t xs_a = smem_off(xs);
+    uint32_t start[kChains], base[kChains];
+    auto fetch = [&]() {
+#pragma unroll
+        for (int c = 0; c < kChains; ++c) {
+            uint32_t total;
+            start[c] = lane_start_bits(my_bits[c], lane, total);
+            base[c] = 0;
+            if (item * kChains + c < f.units)
+                base[c] = stage_span(f, seg_bit[c], total, stage + (size_t)c * f.max_unit_chunks, lane);
+        }
+    };
+    if (item < items) fetch();
     __syncthreads();
 
-    while (u < f.units) {
-        const uint32_t j = u / f.G, g = u - j * f.G;
-        const uint32_t sub = g * 32 + lane;                 // sub-segment number inside the column
-        const uint32_t row0 = sub * f.S;
-        const uint32_t count = row0 < f.n ? min(f.S, f.n - row0) : 0u;
-        BitReader br;
-        br.init(stage_a, base + start);
-        // index entries of the next segment, in flight while this one is decoded
-        const uint32_t un = u + gridDim.x * warps;
-        if (un < f.units) {
-            my_bits = __ldg(f.sub_bits + (size_t)un * 32 + lane);
-            seg_bit = __ldg(f.seg_bit_off + un);
+    while (item < items) {
+        BitReader br[kChains];
+        uint32_t count[kChains], xa[kChains];
+        float* out[kChains];
+        uint32_t common = f.S;
+#pragma unroll
+        for (int c = 0; c < kChains; ++c) {
+            const uint32_t u = item * kChains + c;
+            const uint32_t j = u / f.G, g = u - j * f.G;
+            const uint32_t sub = g * 32 + lane;              // sub-segment number inside the column
+            const uint32_t row0 = sub * f.S;
+            count[c] = (u < f.units && row0 < f.n) ? min(f.S, f.n - row0) : 0u;
+            common = min(common, count[c]);
+            xa[c] = xs_a + ((row0 + pad * sub) << 2);
+            out[c] = aux + (size_t)j * f.n + row0;
+            br[c].init(stage_a + c * f.max_unit_chunks * 16, base[c] + start[c]);
         }
-        if (kMode == 0) {
-            float acc = 0.0f;
-            if (kXShared) {
-                uint32_t xa = xs_a + ((row0 + pad * sub) << 2);
-#pragma unroll 4
-                for (uint32_t s = 0; s < count; ++s) {
-                    const float w = decode_value<kLong>(br, dec, f);
-                    acc = fmaf(ldsf_v(xa), w, acc);
-                    xa += 4;
-                }
+        // index entries of the next item, in flight while this one is decoded
+        const uint32_t next_item = item + gridDim.x * warps;
+#pragma unroll
+        for (int c = 0; c < kChains; ++c) {
+            const uint32_t u = next_item * kChains + c;
+            if (next_item < items && u < f.units) {
+                my_bits[c] = __ldg(f.sub_bits + (size_t)u * 32 + lane);
+                seg_bit[c] = __ldg(f.seg_bit_off + u);
             } else {
-                const float* xl = x + (int64_t)row0 * xs_i;
-                for (uint32_t s = 0; s < count; ++s) {
-                    const float w = decode_value<kLong>(br, dec, f);
-                    acc = fmaf(xl[(int64_t)s * xs_i], w, acc);
+                my_bits[c] = 0;
+            }
+        }
+        float acc[kChains];
+#pragma unroll
+        for (int c = 0; c < kChains; ++c) acc[c] = 0.0f;
+        if (kMode == 0 && kXShared) {
+            const uint32_t sb = shared_base();
+            FastReader fr[kChains];
+            uint32_t xabs[kChains];
+#pragma unroll
+            for (int c = 0; c < kChains; ++c) {
+                fr[c].hi = br[c].hi; fr[c].lo = br[c].lo; fr[c].off = br[c].off; fr[c].next = sb + br[c].next;
+                xabs[c] = sb + xa[c];
+            }
+            const uint32_t l1_abs = sb + dec.l1_lane;
+            uint32_t s = 0;
+            for (; s + 4 <= common; s += 4) {
+                fast_step<kLong, kChains, 0>(fr, dec, f, l1_abs, xabs, acc);
+                fast_step<kLong, kChains, 4>(fr, dec, f, l1_abs, xabs, acc);
+                fast_step<kLong, kChains, 8>(fr, dec, f, l1_abs, xabs, acc);
+                fast_step<kLong, kChains, 12>(fr, dec, f, l1_abs, xabs, acc);
+#pragma unroll
+                for (int c = 0; c < kChains; ++c) xabs[c] += 16;
+            }
+            for (; s < common; ++s) {
+                fast_step<kLong, kChains, 0>(fr, dec, f, l1_abs, xabs, acc);
+#pragma unroll
+                for (int c = 0; c < kChains; ++c) xabs[c] += 4;
+            }
+#pragma unroll
+            for (int c = 0; c < kChains; ++c) {
+                br[c].hi = fr[c].hi; br[c].lo = fr[c].lo; br[c].off = fr[c].off; br[c].next = fr[c].next - sb;
+                xa[c] = xabs[c] - sb;
+                for (uint32_t t = common; t < count[c]; ++t) {
+                    const float w = decode_value<kLong>(br[c], dec, f);
+                    acc[c] = fmaf(ldsf(xa[c]), w, acc[c]);
+                    xa[c] += 4;
                 }
             }
-            acc = warp_sum(acc);
-            if (lane == 0) {
-                if (f.G == 1) y[(int64_t)j * ys_j] = acc;
-                else aux[u] = acc;
+        } else if (kMode == 0) {
+#pragma unroll
+            for (int c = 0; c < kChains; ++c) {
+                const uint32_t u = item * kChains + c;
+                const uint32_t j = u / f.G, g = u - j * f.G;
+                const float* xl = x + (int64_t)((g * 32 + lane) * f.S) * xs_i;
+                for (uint32_t s = 0; s < count[c]; ++s) {
+                    const float w = decode_value<kLong>(br[c], dec, f);
+                    acc[c] = fmaf(xl[(int64_t)s * xs_i], w, acc[c]);
+                }
             }
         } else {
-            float* out = aux + (size_t)j * f.n + row0;
-            for (uint32_t s = 0; s < count; ++s) out[s] = decode_value<kLong>(br, dec, f);
+#pragma unroll
+            for (int c = 0; c < kChains; ++c)
+                for (uint32_t s = 0; s < count[c]; ++s) out[c][s] = decode_value<kLong>(br[c], dec, f);
+        }
+        if (kMode == 0) {
+#pragma unroll
+            for (int c = 0; c < kChains; ++c) acc[c] = warp_sum(acc[c]);
+            if (lane == 0) {
+                if (kChains == 2 && f.G == 2) {              // the item is one whole column
+                    y[(int64_t)item * ys_j] = acc[0] + acc[kChains - 1];
+                } else {
+#pragma unroll
+                    for (int c = 0; c < kChains; ++c) {
+                        const uint32_t u = item * kChains + c;
+                        if (u < f.units) {
+                            if (f.G == 1) y[(int64_t)u * ys_j] = acc[c];
+                            else aux[u] = acc[c];
+                        }
+                    }
+                }
+            }
         }
         __syncwarp();
-        u = un;
-        if (u < f.units) {
-            start = lane_start_bits(my_bits, lane, total);
-            base = stage_span(f, seg_bit, total, stage, lane);
-        }
+        item = next_item;
+        if (item < items) fetch();
     }
 }
 
@@ -329,7 +479,6 @@ template <int kMode, bool kXShared, bool kLong, typename RowT>
 __global__ void __launch_bounds__(1024) shac_vec_kernel(DevFormat f, TablePlan tp, const float* __restrict__ x,
                                                         int64_t xs_i, float* __restrict__ y, int64_t ys_j,
                                                         float* __restrict__ aux) {
-    extern __shared__ __align__(16) unsigned char smem[];
     const uint32_t warp = threadIdx.x >> 5, lane = threadIdx.x & 31, warps = blockDim.x >> 5;
     const ShacUnit* __restrict__ units = reinterpret_cast<const ShacUnit*>(f.unit_info);
     uint32_t u = blockIdx.x + gridDim.x * warp;
@@ -351,7 +500,7 @@ __global__ void __launch_bounds__(1024) shac_vec_kernel(DevFormat f, TablePlan t
     // row-index staging: 32*S entries plus up to 16 bytes of misalignment, per warp
     const uint32_t ri_chunks = (32u * f.S * (uint32_t)sizeof(RowT) + 15u) / 16u + 1u;
     uint4* ri_stage = reinterpret_cast<uint4*>(p) + (size_t)warp * ri_chunks;
-    const uint32_t stage_a = smem_addr(stage), ri_a = smem_addr(ri_stage), xs_a = smem_addr(xs);
+    const uint32_t stage_a = smem_off(stage), ri_a = smem_off(ri_stage), xs_a = smem_off(xs);
     const RowT* __restrict__ ri = reinterpret_cast<const RowT*>(f.ri);
 
     // copies the segment's slice of ri and its span of the stream to shared memory
@@ -389,9 +538,9 @@ __global__ void __launch_bounds__(1024) shac_vec_kernel(DevFormat f, TablePlan t
 #pragma unroll 4
             for (uint32_t s = 0; s < count; ++s) {
                 const float w = decode_value<kLong>(br, dec, f);
-                const uint32_t row = sizeof(RowT) == 2 ? lds16_v(ra) : lds32_v(ra);
+                const uint32_t row = sizeof(RowT) == 2 ? lds16(ra) : lds32(ra);
                 ra += sizeof(RowT);
-                const float xv = kXShared ? ldsf_v(xs_a + (row << 2)) : x[(int64_t)row * xs_i];
+                const float xv = kXShared ? ldsf(xs_a + (row << 2)) : x[(int64_t)row * xs_i];
                 acc = fmaf(xv, w, acc);
             }
             acc = warp_sum(acc);
@@ -443,7 +592,6 @@ __global__ void __launch_bounds__(1024) hac_batch_kernel(DevFormat f, TablePlan 
                                                          int64_t xs_i, int64_t xs_b, uint32_t batch,
                                                          float* __restrict__ y, int64_t ys_j, int64_t ys_b,
                                                          float* __restrict__ partial, uint32_t col_blocks) {
-    extern __shared__ __align__(16) unsigned char smem[];
     unsigned char* p = smem;
     const Decoder dec = stage_decoder(f, tp, p);
     const uint32_t warp = threadIdx.x >> 5, lane = threadIdx.x & 31, warps = blockDim.x >> 5;
@@ -453,7 +601,7 @@ __global__ void __launch_bounds__(1024) hac_batch_kernel(DevFormat f, TablePlan 
     float* xt = reinterpret_cast<float*>(p);                       // [kBatchRows][kTile]
     p += align16((size_t)kBatchRows * kTile * 4);
     uint4* stage = reinterpret_cast<uint4*>(p) + (size_t)warp * f.max_unit_chunks;
-    const uint32_t stage_a = smem_addr(stage);
+    const uint32_t stage_a = smem_off(stage);
     __syncthreads();
     const uint32_t batch_tiles = (batch + kTile - 1) / kTile;
     const uint32_t items = col_blocks * f.G * batch_tiles;
@@ -535,7 +683,6 @@ __global__ void __launch_bounds__(1024) shac_batch_kernel(DevFormat f, TablePlan
                                                           int64_t xs_i, int64_t xs_b, uint32_t batch,
                                                           float* __restrict__ y, int64_t ys_j, int64_t ys_b,
                                                           float* __restrict__ partial) {
-    extern __shared__ __align__(16) unsigned char smem[];
     unsigned char* p = smem;
     const Decoder dec = stage_decoder(f, tp, p);
     const uint32_t warp = threadIdx.x >> 5, lane = threadIdx.x & 31, warps = blockDim.x >> 5;
@@ -547,7 +694,7 @@ __global__ void __launch_bounds__(1024) shac_batch_kernel(DevFormat f, TablePlan
     uint4* stage = reinterpret_cast<uint4*>(p) + (size_t)warp * f.max_unit_chunks;
     float* wv = wv_all + warp * kBatchRows;
     uint32_t* wr = wr_all + warp * kBatchRows;
-    const uint32_t stage_a = smem_addr(stage);
+    const uint32_t stage_a = smem_off(stage);
     __syncthreads();
     const RowT* __restrict__ ri = reinterpret_cast<const RowT*>(f.ri);
     const uint32_t batch_tiles = (batch + kTile - 1) / kTile;
@@ -769,10 +916,14 @@ static TablePlan plan_tables(const DevFormat& d, size_t table_budget) {
 typedef void (*VecKernel)(DevFormat, TablePlan, const float*, int64_t, float*, int64_t, float*);
 
 template <bool kLong>
-static VecKernel pick_vec_kernel(const Format& f, int mode, bool x_shared) {
-    if (!f.sparse)
-        return mode == 1 ? hac_vec_kernel<1, false, kLong>
-                         : (x_shared ? hac_vec_kernel<0, true, kLong> : hac_vec_kernel<0, false, kLong>);
+static VecKernel pick_vec_kernel(const Format& f, int mode, bool x_shared, int chains) {
+    if (!f.sparse) {
+        if (chains == 2)
+            return mode == 1 ? hac_vec_kernel<1, false, kLong, 2>
+                             : (x_shared ? hac_vec_kernel<0, true, kLong, 2> : hac_vec_kernel<0, false, kLong, 2>);
+        return mode == 1 ? hac_vec_kernel<1, false, kLong, 1>
+                         : (x_shared ? hac_vec_kernel<0, true, kLong, 1> : hac_vec_kernel<0, false, kLong, 1>);
+    }
     if (f.ri_bits == 16)
         return mode == 1 ? shac_vec_kernel<1, false, kLong, uint16_t>
                          : (x_shared ? shac_vec_kernel<0, true, kLong, uint16_t>
@@ -784,14 +935,17 @@ static VecKernel pick_vec_kernel(const Format& f, int mode, bool x_shared) {
 
 // mode 0: product with one input; mode 1: debug decode into `aux`.
 static int launch_vec(const Format& f, int mode, const float* x, int64_t xs_i, float* y, int64_t ys_j,
-                      float* aux, cudaStream_t st) {
+                      float* aux, cudaStream_t st, bool* vec_direct = nullptr) {
     DeviceInfo di;
     int rc = device_info(di);
     if (rc) return rc;
     const DevFormat d = dev_format(f);
     if (d.units == 0) return HAC_OK;
     const size_t budget = (size_t)di.max_smem_optin;
-    size_t per_warp = (size_t)d.max_unit_chunks * 16;
+    // HAC: two decode chains per lane when two staging areas per warp fit next to a fully
+    // replicated table; sHAC: one
+    const int chains = (!f.sparse && d.units > 1) ? std::min(2, std::max(1, env_int("HAC_B200_CHAINS", 2))) : 1;
+    size_t per_warp = (size_t)d.max_unit_chunks * 16 * chains;
     if (f.sparse && mode == 0) per_warp += ((size_t)(32u * f.S * (f.ri_bits / 8) + 15u) / 16u + 1u) * 16u;
     size_t xbytes = 0;
     if (mode == 0) xbytes = f.sparse ? align16((size_t)f.n * 4) : align16(((size_t)f.n + (f.n / f.S + 1)) * 4);
@@ -809,15 +963,18 @@ static int launch_vec(const Format& f, int mode, const float* x, int64_t xs_i, f
     if (smem > budget) return HAC_ERR_BUFFER_TOO_SMALL;
     const bool has_long = d.max_len > d.l1_bits;
     const int threads = warps * 32;
-    VecKernel kernel = has_long ? pick_vec_kernel<true>(f, mode, x_shared) : pick_vec_kernel<false>(f, mode, x_shared);
+    VecKernel kernel = has_long ? pick_vec_kernel<true>(f, mode, x_shared, chains)
+                                : pick_vec_kernel<false>(f, mode, x_shared, chains);
     rc = prepare_kernel(kernel, smem);
     if (rc) return rc;
     int per_sm = 1;
     HAC_CUDA(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kernel, threads, smem));
     per_sm = std::max(per_sm, 1);
     // spread the segments over all SMs (a block's warps take segments blockIdx + k * gridDim)
-    const unsigned grid = std::min<unsigned>(d.units, (unsigned)(di.sms * per_sm));
+    const unsigned items = (d.units + chains - 1) / chains;
+    const unsigned grid = std::min<unsigned>(items, (unsigned)(di.sms * per_sm));
     kernel<<<grid, threads, smem, st>>>(d, tp, x, xs_i, y, ys_j, aux);
+    if (vec_direct) *vec_direct = (!f.sparse && (f.G == 1 || (chains == 2 && f.G == 2)));
     HAC_CUDA(cudaGetLastError());
     f.last_launches++;
     return HAC_OK;
@@ -884,9 +1041,10 @@ static int dot(const Format& f, const float* x, int64_t batch, int64_t xs_i, int
     float* partial = static_cast<float*>(workspace);
     const DevFormat d = dev_format(f);
     int rc = HAC_OK;
+    bool direct = false;                     // the product kernel wrote every output itself
     if (d.units > 0) {
         if (batch == 1) {
-            rc = launch_vec(f, 0, x, xs_i, y, ys_j, partial, st);
+            rc = launch_vec(f, 0, x, xs_i, y, ys_j, partial, st, &direct);
         } else {
             DeviceInfo di;
             rc = device_info(di);
@@ -901,7 +1059,7 @@ static int dot(const Format& f, const float* x, int64_t batch, int64_t xs_i, int
         }
         if (rc) return rc;
     }
-    if (needs_finalize(f) || d.units == 0) rc = launch_finalize(f, d, partial, batch, y, ys_j, ys_b, st);
+    if ((needs_finalize(f) && !direct) || d.units == 0) rc = launch_finalize(f, d, partial, batch, y, ys_j, ys_b, st);
     return rc;
 }
 
