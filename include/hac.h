@@ -211,6 +211,36 @@ int shac_dot_host(const shac_format* f, const float* X_host, int64_t batch, floa
                   void* dev_scratch, size_t dev_scratch_bytes, void* cuda_stream);
 
 /* ---------------------------------------------------------------------------------------------
+ * hac_dot_noalloc - the HAC product of hac_dot for callers that cannot hand over a workspace.
+ * (The paper has no counterpart: this is a packaging variant of hac_dot, not a different method.)
+ *
+ * hac_dot needs a device workspace whenever a column of W spans several segments, and the caller has
+ * to get that memory from somewhere.  Some hosts cannot: an inference server that carves up all
+ * device memory at start-up and forbids later cudaMalloc calls (they serialise the device and can
+ * fail under fragmentation), or a plugin that runs inside another program's memory plan and owns no
+ * allocator at all.  For them this call keeps the partial sums in a buffer that is part of the
+ * library image itself: a file-scope device array of HAC_NOALLOC_SCRATCH_BYTES bytes, present on
+ * every GPU that loads the library until the process exits.  The call makes no cudaMalloc / cudaFree
+ * and uses no allocating library routine; x and y are still the caller's.
+ *
+ * Arguments and result as hac_dot, without the workspace pair.
+ *   - A product whose partial sums need more than HAC_NOALLOC_SCRATCH_BYTES (see hac_workspace_bytes)
+ *     is refused with HAC_ERR_BUFFER_TOO_SMALL and nothing is launched; hac_last_cuda_error() then
+ *     names the two sizes.  Use hac_dot with your own workspace for those.
+ *   - The first call on each device looks up the device address of the buffer (one
+ *     cudaGetSymbolAddress with that device current).  Make that first call outside any stream
+ *     capture.
+ *   - All calls on a device share the one buffer, and it keeps whatever the previous call left there.
+ *     Nothing in it has to start at zero: every slot the finishing kernel reads is written by the
+ *     product kernel of the same call first.  Two calls that may overlap on the GPU (different
+ *     streams, or different handles on different threads) race on it and give wrong sums; run them on
+ *     one stream, or order them with events.
+ * ------------------------------------------------------------------------------------------- */
+#define HAC_NOALLOC_SCRATCH_BYTES (4u << 20)
+int hac_dot_noalloc(const hac_format* f, const float* x, int64_t batch, int64_t x_stride_i, int64_t x_stride_b,
+                    float* y, int64_t y_stride_j, int64_t y_stride_b, void* cuda_stream);
+
+/* ---------------------------------------------------------------------------------------------
  * TEST ONLY: decode on the device into a caller's device buffer, to show that the kernels' decoder
  * reproduces the quantized weights bit for bit (the formats are lossless, Sect. IV-B).  The product
  * path never does this.  hac: W_colmajor[j*n + i] = Wq[i][j] (n*m floats).  shac: nz[p] for the nnz

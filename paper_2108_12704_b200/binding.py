@@ -61,7 +61,7 @@ EXPORTS = (
     "hac_build", "shac_build", "hac_sizes", "shac_sizes", "hac_export", "shac_export",
     "hac_decode_host", "shac_decode_host", "hac_device_bytes", "shac_device_bytes", "hac_upload",
     "shac_upload", "hac_attach", "shac_attach", "hac_workspace_bytes", "shac_workspace_bytes", "hac_dot",
-    "shac_dot", "hac_dot_host_scratch_bytes", "shac_dot_host_scratch_bytes", "hac_dot_host",
+    "shac_dot", "hac_dot_noalloc", "hac_dot_host_scratch_bytes", "shac_dot_host_scratch_bytes", "hac_dot_host",
     "shac_dot_host", "hac_debug_decode", "shac_debug_decode", "hac_last_launch_count",
     "shac_last_launch_count", "hac_free", "shac_free", "hac_status_string", "hac_last_cuda_error",
 )
@@ -98,6 +98,7 @@ def load():
         getattr(lib, f"{kind}_last_launch_count").argtypes = [vp]
         getattr(lib, f"{kind}_free").argtypes = [vp]
         getattr(lib, f"{kind}_free").restype = None
+    lib.hac_dot_noalloc.argtypes = [vp, fp, i64, i64, i64, fp, i64, i64, vp]
     lib.hac_status_string.argtypes = [C.c_int]
     lib.hac_status_string.restype = C.c_char_p
     lib.hac_last_cuda_error.restype = C.c_char_p
@@ -251,6 +252,32 @@ class Format:
         wb = workspace.numel() * workspace.element_size() if workspace is not None else 0
         st = torch.cuda.current_stream().cuda_stream
         _check(self._fn("dot")(self._h, x.data_ptr(), B, xs_i, xs_b, y.data_ptr(), ys_j, ys_b, wp, wb, st), "dot")
+        return y
+
+    def dot_noalloc(self, x, y=None, layout="nb"):
+        """hac_dot_noalloc of the C ABI: like dot(), but the partial sums go to the buffer built into
+        the library instead of a workspace tensor (HAC only; refused with status -8 if they do not
+        fit).  For hosts that are not allowed to allocate device memory; y is still the caller's, and
+        is only created here as a convenience when it is not passed."""
+        import torch
+        assert self.kind == "hac" and x.is_cuda and x.dtype == torch.float32
+        if x.dim() == 1:
+            B, xs_i, xs_b, yshape = 1, x.stride(0), 0, (self.m,)
+        elif layout == "nb":
+            B, xs_i, xs_b, yshape = x.shape[1], x.stride(0), x.stride(1), (self.m, x.shape[1])
+        else:
+            B, xs_i, xs_b, yshape = x.shape[0], x.stride(1), x.stride(0), (x.shape[0], self.m)
+        if y is None:
+            y = torch.empty(yshape, dtype=torch.float32, device=x.device)
+        if y.dim() == 1:
+            ys_j, ys_b = y.stride(0), 0
+        elif layout == "nb":
+            ys_j, ys_b = y.stride(0), y.stride(1)
+        else:
+            ys_j, ys_b = y.stride(1), y.stride(0)
+        st = torch.cuda.current_stream().cuda_stream
+        _check(self._lib.hac_dot_noalloc(self._h, x.data_ptr(), B, xs_i, xs_b, y.data_ptr(), ys_j, ys_b, st),
+               "hac_dot_noalloc")
         return y
 
     def dot_host_scratch_bytes(self, batch: int) -> int:

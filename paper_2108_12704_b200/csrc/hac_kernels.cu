@@ -15,6 +15,7 @@
 #include <cstdio>
 #include <cstdlib>
 #include <cstring>
+#include <mutex>
 #include <string>
 
 #include "hac_internal.h"
@@ -1105,6 +1106,45 @@ static int dot_host(const Format& f, const float* X, int64_t batch, float* Y, vo
     return HAC_OK;
 }
 
+// Scratch of hac_dot_noalloc: part of the library image, one copy per device that loads it.
+static __device__ __align__(256) unsigned char g_noalloc_scratch[HAC_NOALLOC_SCRATCH_BYTES];
+
+// Device address of g_noalloc_scratch on the current device, looked up once per device.  In host
+// code the array's name only stands for the symbol; the kernels need the address this returns.
+static int noalloc_scratch_address(void** out) {
+    static std::mutex guard;
+    static void* address[64] = {};
+    int dev = 0;
+    HAC_CUDA(cudaGetDevice(&dev));
+    if (dev < 0 || dev >= 64) return HAC_ERR_INVALID_ARG;
+    std::lock_guard<std::mutex> lock(guard);
+    if (!address[dev]) {
+        void* ptr = nullptr;
+        HAC_CUDA(cudaGetSymbolAddress(&ptr, g_noalloc_scratch));
+        if (!ptr) return HAC_ERR_CUDA;
+        address[dev] = ptr;
+    }
+    *out = address[dev];
+    return HAC_OK;
+}
+
+static int dot_noalloc(const Format& f, const float* x, int64_t batch, int64_t xs_i, int64_t xs_b, float* y,
+                       int64_t ys_j, int64_t ys_b, void* stream_) {
+    if (!f.dev.base) return HAC_ERR_NOT_UPLOADED;
+    if (!x || !y || batch < 1 || batch > ((int64_t)1 << 24)) return HAC_ERR_INVALID_ARG;
+    const size_t need = workspace_bytes(f, batch);
+    if (need > (size_t)HAC_NOALLOC_SCRATCH_BYTES) {
+        g_last_cuda_error = "hac_dot_noalloc: this product needs " + std::to_string(need) +
+                            " bytes of partial sums, the built-in buffer holds " +
+                            std::to_string((size_t)HAC_NOALLOC_SCRATCH_BYTES);
+        return HAC_ERR_BUFFER_TOO_SMALL;
+    }
+    void* scratch = nullptr;
+    const int rc = noalloc_scratch_address(&scratch);
+    if (rc != HAC_OK) return rc;
+    return dot(f, x, batch, xs_i, xs_b, y, ys_j, ys_b, scratch, (size_t)HAC_NOALLOC_SCRATCH_BYTES, stream_);
+}
+
 static int debug_decode(const Format& f, float* out, void* stream_) {
     if (!f.dev.base) return HAC_ERR_NOT_UPLOADED;
     if (!out) return HAC_ERR_INVALID_ARG;
@@ -1163,6 +1203,12 @@ int shac_dot(const shac_format* f, const float* x, int64_t batch, int64_t x_stri
     if (!f) return HAC_ERR_INVALID_ARG;
     return dot(f->f, x, batch, x_stride_i, x_stride_b, y, y_stride_j, y_stride_b, workspace, workspace_bytes_,
                cuda_stream);
+}
+
+int hac_dot_noalloc(const hac_format* f, const float* x, int64_t batch, int64_t x_stride_i, int64_t x_stride_b,
+                    float* y, int64_t y_stride_j, int64_t y_stride_b, void* cuda_stream) {
+    if (!f) return HAC_ERR_INVALID_ARG;
+    return dot_noalloc(f->f, x, batch, x_stride_i, x_stride_b, y, y_stride_j, y_stride_b, cuda_stream);
 }
 
 int hac_dot_host_scratch_bytes(const hac_format* f, int64_t batch, size_t* out) {
