@@ -61,7 +61,8 @@ typedef struct hac_build_params {
     uint32_t quantizer;     /* HAC_QUANT_*                                                              */
     uint32_t kmeans_iters;  /* Lloyd iterations, run in full (no early stop)                            */
     uint32_t seg_symbols;   /* S: symbols per sub-segment of the offset index, 1..HAC_MAX_SEG_SYMBOLS;
-                               0 = default (64 for HAC, 32 for sHAC)                                    */
+                               0 = default: 64 for HAC; for sHAC about (entries of the fullest column)/64,
+                               rounded up so that S * ri_bits / 32 is odd (reported by *_sizes)         */
     uint64_t seed;          /* seed of the k-means initialisation                                       */
     uint32_t ri_bits;       /* sHAC: width of a stored row index, 16 or 32; 0 = 16 if n <= 65536 else 32
                                (the footnote of Sect. IV-A: ri needs only ceil(log n) bits)             */

@@ -292,8 +292,8 @@ int build_impl(const float* W, int64_t n, int64_t m, int64_t ldw, const hac_buil
         return HAC_ERR_OFFSET_OVERFLOW;
     f.sparse = sparse;
     f.n = n; f.m = m;
-    f.S = p->seg_symbols ? p->seg_symbols : (sparse ? 32u : 64u);
     f.ri_bits = sparse ? (p->ri_bits ? p->ri_bits : (n <= 65536 ? 16u : 32u)) : 0u;
+    f.S = p->seg_symbols ? p->seg_symbols : (sparse ? 0u : 64u);   // sHAC default: chosen from the data below
     if (sparse && f.ri_bits == 16 && n > 65536) return HAC_ERR_INVALID_ARG;
     const int64_t total = n * m;
 
@@ -322,6 +322,20 @@ int build_impl(const float* W, int64_t n, int64_t m, int64_t ldw, const hac_buil
     for (int64_t t = 0; t < total; ++t) q += (col[t] != 0.0f);
     f.nnz = q;
     if (q >= ((int64_t)1 << 32)) return HAC_ERR_OFFSET_OVERFLOW;
+    if (f.S == 0) {
+        // sHAC default: two segments cover the fullest column, and the sub-segments' slices of ri
+        // start an odd number of 32-bit words apart (keeps the 32 lanes on distinct shared-memory banks)
+        int64_t fullest = 0;
+        for (int64_t j = 0; j < m; ++j) {
+            int64_t c = 0;
+            const float* cj = col.data() + j * n;
+            for (int64_t i = 0; i < n; ++i) c += (cj[i] != 0.0f);
+            fullest = std::max(fullest, c);
+        }
+        uint32_t S = (uint32_t)std::min<int64_t>(256, std::max<int64_t>(4, (fullest + 63) / 64));
+        if (f.ri_bits == 16) { while (S % 4 != 2) ++S; } else { S |= 1u; }
+        f.S = S;
+    }
     std::vector<double> data;
     data.reserve(q);
     for (int64_t t = 0; t < total; ++t)
@@ -440,18 +454,25 @@ int build_impl(const float* W, int64_t n, int64_t m, int64_t ldw, const hac_buil
         f.max_unit_chunks = std::max<uint32_t>(f.max_unit_chunks, (uint32_t)((last_word >> 2) - first_chunk + 1));
     }
     if (sparse) {
-        f.unit_info.resize(U * 6);
-        for (size_t u = 0; u < U; ++u) {
-            const uint32_t j = f.seg_col[u];
-            const uint32_t g = (uint32_t)u - f.seg_first[j];
-            const uint32_t pos0 = f.cb[j] + g * 32u * S;
-            uint32_t* r = &f.unit_info[u * 6];
-            r[0] = (uint32_t)(f.seg_bit_off[u] & 0xffffffffu);
-            r[1] = (uint32_t)(f.seg_bit_off[u] >> 32);
-            r[2] = pos0;
-            r[3] = std::min<uint32_t>(32u * S, f.cb[j + 1] - pos0);
-            r[4] = j;
-            r[5] = (f.seg_first[j + 1] - f.seg_first[j]) == 1 ? 1u : 0u;
+        // device-only work list: an item is one or two consecutive segments of one column
+        f.item_info.clear();
+        for (int64_t j = 0; j < m; ++j) {
+            const uint32_t u_begin = f.seg_first[j], u_end = f.seg_first[j + 1];
+            for (uint32_t u = u_begin; u < u_end; u += 2) {
+                const uint32_t in_item = std::min(2u, u_end - u);
+                uint32_t rec[12] = {0};
+                for (uint32_t c = 0; c < in_item; ++c) {
+                    const uint32_t pos0 = f.cb[j] + (u + c - u_begin) * 32u * S;
+                    rec[4 * c + 0] = (uint32_t)(f.seg_bit_off[u + c] & 0xffffffffu);
+                    rec[4 * c + 1] = (uint32_t)(f.seg_bit_off[u + c] >> 32);
+                    rec[4 * c + 2] = pos0;
+                    rec[4 * c + 3] = std::min<uint32_t>(32u * S, f.cb[j + 1] - pos0);
+                }
+                rec[8] = (uint32_t)j;
+                rec[9] = in_item | ((u_end - u_begin) <= 2 ? 0x100u : 0u);   // bit 8: the item is the whole column
+                rec[10] = u;
+                f.item_info.insert(f.item_info.end(), rec, rec + 12);
+            }
         }
         f.max_units_per_col = 0;
         f.has_empty_col = false;
@@ -564,7 +585,7 @@ ImageLayout image_layout(const Format& f) {
     L.seg_first = take(f.seg_first.size() * 4);
     L.ri = take(f.ri_bits == 16 ? f.ri16.size() * 2 + 16 : f.ri32.size() * 4 + 16);
     L.cb = take(f.cb.size() * 4);
-    L.unit_info = take(f.unit_info.size() * 4);
+    L.unit_info = take(f.item_info.size() * 4);
     L.total = o;
     return L;
 }

@@ -85,7 +85,7 @@ struct Format {
     std::vector<uint64_t> seg_bit_off;
     std::vector<uint16_t> sub_bits;
     std::vector<uint32_t> seg_first, seg_col;
-    std::vector<uint32_t> unit_info;          // sHAC, device only: 6 words per segment (see ShacUnit)
+    std::vector<uint32_t> item_info;          // sHAC, device only: 12 words per work item (see ShacItem)
     uint32_t max_unit_chunks = 0;             // largest 16-byte span a segment's stream covers
     uint32_t max_units_per_col = 0;
     bool has_empty_col = false;

@@ -17,6 +17,7 @@
 #include <cstring>
 #include <mutex>
 #include <string>
+#include <type_traits>
 
 #include "hac_internal.h"
 
@@ -53,7 +54,7 @@ struct DevFormat {
     const void* ri;
     const uint32_t* cb;
     const void* unit_info;
-    uint32_t n, m, units, G, S, k_eff, lut_bits, max_len, ri_bits, max_unit_chunks, l1_bits, sub_bytes;
+    uint32_t n, m, units, G, S, k_eff, lut_bits, max_len, ri_bits, max_unit_chunks, l1_bits, sub_bytes, items;
 };
 
 
@@ -83,6 +84,7 @@ __host__ __device__ inline size_t align16(size_t x) { return (x + 15) & ~(size_t
 //            for code words longer still, which are found by a search over lengths in global memory.
 struct TablePlan {
     uint32_t repl_log2;
+    uint32_t x_bulk;      // sHAC: x is contiguous and 16-byte aligned, so it is brought in by one bulk async copy
 };
 
 __host__ __device__ inline size_t plan_smem_bytes(uint32_t l1_bits, uint32_t repl_log2, uint32_t sub_bytes) {
@@ -237,6 +239,92 @@ __device__ __forceinline__ void fast_consume(FastReader& r, uint32_t val, uint32
         : "+r"(r.hi), "+r"(r.lo), "+r"(r.off), "+r"(r.next), "+f"(acc)
         : "f"(__uint_as_float(val)), "r"(len), "r"(x_addr), "n"(kXOffset)
         : "memory");
+}
+
+// Same step for sHAC: the row of the entry comes from the staged slice of ri, x is gathered by row.
+template <int kRowBytes, int kRiOffset>
+__device__ __forceinline__ void fast_consume_sparse(FastReader& r, uint32_t val, uint32_t len, uint32_t ri_addr,
+                                                    uint32_t xs_abs, float& acc) {
+    if (kRowBytes == 2) {
+        asm volatile(
+            "{\n\t"
+            ".reg .pred p;\n\t"
+            ".reg .f32 xv;\n\t"
+            ".reg .b32 row;\n\t"
+            ".reg .b16 r16;\n\t"
+            "ld.shared.u16 r16, [%7+%9];\n\t"
+            "cvt.u32.u16 row, r16;\n\t"
+            "mad.lo.u32 row, row, 4, %8;\n\t"
+            "ld.shared.f32 xv, [row];\n\t"
+            "add.u32 %2, %2, %6;\n\t"
+            "setp.ge.u32 p, %2, 32;\n\t"
+            "@p mov.u32 %0, %1;\n\t"
+            "@p ld.shared.u32 %1, [%3];\n\t"
+            "@p add.u32 %3, %3, 4;\n\t"
+            "and.b32 %2, %2, 31;\n\t"
+            "fma.rn.f32 %4, xv, %5, %4;\n\t"
+            "}"
+            : "+r"(r.hi), "+r"(r.lo), "+r"(r.off), "+r"(r.next), "+f"(acc)
+            : "f"(__uint_as_float(val)), "r"(len), "r"(ri_addr), "r"(xs_abs), "n"(kRiOffset)
+            : "memory");
+    } else {
+        asm volatile(
+            "{\n\t"
+            ".reg .pred p;\n\t"
+            ".reg .f32 xv;\n\t"
+            ".reg .b32 row;\n\t"
+            "ld.shared.u32 row, [%7+%9];\n\t"
+            "mad.lo.u32 row, row, 4, %8;\n\t"
+            "ld.shared.f32 xv, [row];\n\t"
+            "add.u32 %2, %2, %6;\n\t"
+            "setp.ge.u32 p, %2, 32;\n\t"
+            "@p mov.u32 %0, %1;\n\t"
+            "@p ld.shared.u32 %1, [%3];\n\t"
+            "@p add.u32 %3, %3, 4;\n\t"
+            "and.b32 %2, %2, 31;\n\t"
+            "fma.rn.f32 %4, xv, %5, %4;\n\t"
+            "}"
+            : "+r"(r.hi), "+r"(r.lo), "+r"(r.off), "+r"(r.next), "+f"(acc)
+            : "f"(__uint_as_float(val)), "r"(len), "r"(ri_addr), "r"(xs_abs), "n"(kRiOffset)
+            : "memory");
+    }
+}
+
+// ------------------------------------------------------------------------------------------------
+// Bulk asynchronous copy global -> shared (TMA, untiled form) with completion on an mbarrier.
+// Source, destination and size must be multiples of 16 bytes.  The wait is bounded: it returns
+// false if the copy has not landed after kBulkWaitTries polls, and the caller then copies with
+// ordinary loads instead.
+// ------------------------------------------------------------------------------------------------
+constexpr uint32_t kBulkWaitTries = 200000;
+
+__device__ __forceinline__ void mbar_init(uint32_t mbar, uint32_t arrivals) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(mbar), "r"(arrivals) : "memory");
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t mbar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(mbar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void bulk_copy_g2s(uint32_t dst, const void* src, uint32_t bytes, uint32_t mbar) {
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(dst),
+                 "l"(src), "r"(bytes), "r"(mbar)
+                 : "memory");
+}
+__device__ __forceinline__ bool mbar_wait_bounded(uint32_t mbar, uint32_t parity) {
+    for (uint32_t t = 0; t < kBulkWaitTries; ++t) {
+        uint32_t done;
+        asm volatile(
+            "{\n\t"
+            ".reg .pred p;\n\t"
+            "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+            "selp.u32 %0, 1, 0, p;\n\t"
+            "}"
+            : "=r"(done)
+            : "r"(mbar), "r"(parity)
+            : "memory");
+        if (done) return true;
+    }
+    return false;
 }
 
 // Level-1 entry that stands for a prefix of longer code words: sub-table, then the search.
@@ -456,106 +544,209 @@ __global__ void __launch_bounds__(1024) hac_vec_kernel(DevFormat f, TablePlan tp
     }
 }
 
-// Per-segment record of sHAC (derived at upload from cb, seg_first, seg_col): where the segment's
-// entries start in nz / ri, how many there are, its column, and whether it is the column's only one.
-struct ShacUnit {
-    uint64_t bit_off;
-    uint32_t pos0, count, col, single;
+// Work item of the sHAC single-input kernel (derived on the host from cb and the offset index): one
+// or two consecutive segments of one column.  For each segment: where its code words start in the
+// stream, where its entries start in nz / ri, and how many there are.
+struct ShacItem {
+    uint64_t bit_off[2];
+    uint32_t pos0[2], count[2];
+    uint32_t col, segments, whole_column, first_unit;
 };
 
-__device__ __forceinline__ ShacUnit load_unit(const ShacUnit* q) {     // records are 8-byte aligned
-    const uint2* w = reinterpret_cast<const uint2*>(q);
-    const uint2 a = __ldg(w), b = __ldg(w + 1), c = __ldg(w + 2);
-    ShacUnit r;
-    r.bit_off = ((uint64_t)a.y << 32) | a.x; r.pos0 = b.x; r.count = b.y; r.col = c.x; r.single = c.y;
+__device__ __forceinline__ ShacItem load_item(const void* base, uint32_t index) {     // 48-byte records
+    const uint4* w = reinterpret_cast<const uint4*>(base) + (size_t)index * 3;
+    const uint4 a = __ldg(w), b = __ldg(w + 1), c = __ldg(w + 2);
+    ShacItem r;
+    r.bit_off[0] = ((uint64_t)a.y << 32) | a.x; r.pos0[0] = a.z; r.count[0] = a.w;
+    r.bit_off[1] = ((uint64_t)b.y << 32) | b.x; r.pos0[1] = b.z; r.count[1] = b.w;
+    r.col = c.x; r.segments = c.y & 0xffu; r.whole_column = (c.y >> 8) & 1u; r.first_unit = c.z;
     return r;
 }
 
 // ------------------------------------------------------------------------------------------------
-// sHAC, one input vector (Algorithm 2 by segments): as above over the stored entries of a column,
-// with the row of each entry taken from ri (the segment's slice of ri is staged in shared memory
-// by coalesced loads) and x gathered from shared memory.
+// sHAC, one input vector (Algorithm 2 by segments): as the HAC kernel over the stored entries of a
+// column, with the row of each entry taken from ri (the segment's slice of ri is staged in shared
+// memory by coalesced loads) and x gathered from shared memory.  A warp takes one item (up to two
+// segments of a column) at a time, so every lane runs two independent decode chains.
 // ------------------------------------------------------------------------------------------------
 template <int kMode, bool kXShared, bool kLong, typename RowT>
 __global__ void __launch_bounds__(1024) shac_vec_kernel(DevFormat f, TablePlan tp, const float* __restrict__ x,
                                                         int64_t xs_i, float* __restrict__ y, int64_t ys_j,
                                                         float* __restrict__ aux) {
+    constexpr int kChains = 2;
+    constexpr int kRow = (int)sizeof(RowT);
     const uint32_t warp = threadIdx.x >> 5, lane = threadIdx.x & 31, warps = blockDim.x >> 5;
-    const ShacUnit* __restrict__ units = reinterpret_cast<const ShacUnit*>(f.unit_info);
-    uint32_t u = blockIdx.x + gridDim.x * warp;
-    uint32_t my_bits = 0;
-    ShacUnit info = {0, 0, 0, 0, 0};
-    if (u < f.units) {
-        my_bits = __ldg(f.sub_bits + (size_t)u * 32 + lane);
-        info = load_unit(units + u);
-    }
+    uint32_t item = blockIdx.x + gridDim.x * warp;
+    uint32_t my_bits[kChains] = {0, 0};
+    ShacItem info;
+    info.segments = 0;
+    auto load_index = [&](uint32_t it) {
+        info = load_item(f.unit_info, it);
+#pragma unroll
+        for (int c = 0; c < kChains; ++c)
+            my_bits[c] = (uint32_t)c < info.segments ? __ldg(f.sub_bits + (size_t)(info.first_unit + c) * 32 + lane) : 0u;
+    };
+    if (item < f.items) load_index(item);
     unsigned char* p = smem;
-    const Decoder dec = stage_decoder(f, tp, p);
+    // x: one bulk asynchronous copy when it is contiguous and aligned (it overlaps the table fill
+    // and the first segment fetch), ordinary loads otherwise
+    const uint32_t mbar = shared_base();
+    p += 16;
     float* xs = reinterpret_cast<float*>(p);
-    if (kMode == 0 && kXShared) {
-        for (uint32_t i = threadIdx.x; i < f.n; i += blockDim.x) xs[i] = x[(int64_t)i * xs_i];
-        p += align16((size_t)f.n * 4);
+    const bool bulk = kMode == 0 && kXShared && tp.x_bulk;
+    const uint32_t bulk_bytes = (f.n & ~3u) * 4u;
+    if (kMode == 0 && kXShared) p += align16((size_t)f.n * 4);
+    if (bulk) {
+        if (threadIdx.x == 0) mbar_init(mbar, 1);
+        __syncthreads();
+        if (threadIdx.x == 0 && bulk_bytes > 0) {
+            mbar_expect_tx(mbar, bulk_bytes);
+            bulk_copy_g2s(shared_base() + smem_off(xs), x, bulk_bytes, mbar);
+        }
+        for (uint32_t i = (f.n & ~3u) + threadIdx.x; i < f.n; i += blockDim.x) xs[i] = x[i];
     }
-    uint4* stage = reinterpret_cast<uint4*>(p) + (size_t)warp * f.max_unit_chunks;
-    p += align16((size_t)warps * f.max_unit_chunks * 16);
-    // row-index staging: 32*S entries plus up to 16 bytes of misalignment, per warp
-    const uint32_t ri_chunks = (32u * f.S * (uint32_t)sizeof(RowT) + 15u) / 16u + 1u;
-    uint4* ri_stage = reinterpret_cast<uint4*>(p) + (size_t)warp * ri_chunks;
+    const Decoder dec = stage_decoder(f, tp, p);
+    if (kMode == 0 && kXShared && !bulk) {
+#pragma unroll 8
+        for (uint32_t i = threadIdx.x; i < f.n; i += blockDim.x) xs[i] = __ldg(x + (int64_t)i * xs_i);
+    }
+    uint4* stage = reinterpret_cast<uint4*>(p) + (size_t)warp * kChains * f.max_unit_chunks;
+    p += align16((size_t)warps * kChains * f.max_unit_chunks * 16);
+    // row-index staging: 32*S entries plus up to 16 bytes of misalignment, per segment
+    const uint32_t ri_chunks = (32u * f.S * (uint32_t)kRow + 15u) / 16u + 1u;
+    uint4* ri_stage = reinterpret_cast<uint4*>(p) + (size_t)warp * kChains * ri_chunks;
     const uint32_t stage_a = smem_off(stage), ri_a = smem_off(ri_stage), xs_a = smem_off(xs);
     const RowT* __restrict__ ri = reinterpret_cast<const RowT*>(f.ri);
 
-    // copies the segment's slice of ri and its span of the stream to shared memory
-    auto fetch = [&](const ShacUnit& un, uint32_t bits, uint32_t& start, uint32_t& base, uint32_t& ri_lane) {
-        uint32_t total;
-        start = lane_start_bits(bits, lane, total);
-        if (kMode == 0) {
-            const uintptr_t byte0 = reinterpret_cast<uintptr_t>(ri + un.pos0);
-            const uintptr_t chunk0 = byte0 & ~(uintptr_t)15;
-            const uint32_t chunks = (uint32_t)((byte0 + (uintptr_t)un.count * sizeof(RowT) - chunk0 + 15) >> 4);
-            const uint4* src = reinterpret_cast<const uint4*>(chunk0);
-            for (uint32_t c = lane; c < chunks; c += 32) ri_stage[c] = __ldg(src + c);
-            ri_lane = ri_a + (uint32_t)(byte0 - chunk0) + lane * f.S * (uint32_t)sizeof(RowT);
-        }
-        base = stage_span(f, un.bit_off, total, stage, lane);       // ends with __syncwarp
-    };
-    uint32_t start = 0, base = 0, ri_lane = 0;
-    if (u < f.units) fetch(info, my_bits, start, base, ri_lane);
-    __syncthreads();
-
-    while (u < f.units) {
-        const ShacUnit cur = info;
-        const uint32_t lane_pos = lane * f.S;
-        const uint32_t count = lane_pos < cur.count ? min(f.S, cur.count - lane_pos) : 0u;
-        BitReader br;
-        br.init(stage_a, base + start);
-        const uint32_t un = u + gridDim.x * warps;
-        if (un < f.units) {
-            my_bits = __ldg(f.sub_bits + (size_t)un * 32 + lane);
-            info = load_unit(units + un);
-        }
-        if (kMode == 0) {
-            float acc = 0.0f;
-            uint32_t ra = ri_lane;
-#pragma unroll 4
-            for (uint32_t s = 0; s < count; ++s) {
-                const float w = decode_value<kLong>(br, dec, f);
-                const uint32_t row = sizeof(RowT) == 2 ? lds16(ra) : lds32(ra);
-                ra += sizeof(RowT);
-                const float xv = kXShared ? ldsf(xs_a + (row << 2)) : x[(int64_t)row * xs_i];
-                acc = fmaf(xv, w, acc);
+    // copies each segment's slice of ri and its span of the stream to shared memory
+    uint32_t start[kChains], base[kChains], ri_lane[kChains];
+    auto fetch = [&]() {
+#pragma unroll
+        for (int c = 0; c < kChains; ++c) {
+            uint32_t total;
+            start[c] = lane_start_bits(my_bits[c], lane, total);
+            base[c] = 0; ri_lane[c] = ri_a;
+            if ((uint32_t)c < info.segments) {
+                if (kMode == 0) {
+                    const uintptr_t byte0 = reinterpret_cast<uintptr_t>(ri + info.pos0[c]);
+                    const uintptr_t chunk0 = byte0 & ~(uintptr_t)15;
+                    const uint32_t chunks = (uint32_t)((byte0 + (uintptr_t)info.count[c] * kRow - chunk0 + 15) >> 4);
+                    const uint4* src = reinterpret_cast<const uint4*>(chunk0);
+                    uint4* dst = ri_stage + (size_t)c * ri_chunks;
+                    for (uint32_t k = lane; k < chunks; k += 32) dst[k] = __ldg(src + k);
+                    ri_lane[c] = ri_a + c * ri_chunks * 16 + (uint32_t)(byte0 - chunk0) + lane * f.S * (uint32_t)kRow;
+                }
+                base[c] = stage_span(f, info.bit_off[c], total, stage + (size_t)c * f.max_unit_chunks, lane);
             }
-            acc = warp_sum(acc);
-            if (lane == 0) {
-                if (cur.single) y[(int64_t)cur.col * ys_j] = acc;
-                else aux[u] = acc;
-            }
-        } else {
-            float* out = aux + cur.pos0 + lane_pos;
-            for (uint32_t s = 0; s < count; ++s) out[s] = decode_value<kLong>(br, dec, f);
         }
         __syncwarp();
-        u = un;
-        if (u < f.units) fetch(info, my_bits, start, base, ri_lane);
+    };
+    if (item < f.items) fetch();
+    if (bulk) {
+        const bool landed = bulk_bytes == 0 || mbar_wait_bounded(mbar, 0);
+        if (__syncthreads_or(landed ? 0 : 1)) {             // late or lost: copy x the ordinary way
+            for (uint32_t i = threadIdx.x; i < f.n; i += blockDim.x) xs[i] = x[i];
+        }
+    }
+    __syncthreads();
+
+    while (item < f.items) {
+        const ShacItem cur = info;
+        BitReader br[kChains];
+        uint32_t count[kChains];
+        uint32_t common = f.S;
+        const uint32_t lane_pos = lane * f.S;
+#pragma unroll
+        for (int c = 0; c < kChains; ++c) {
+            count[c] = ((uint32_t)c < cur.segments && lane_pos < cur.count[c]) ? min(f.S, cur.count[c] - lane_pos) : 0u;
+            common = min(common, count[c]);
+            br[c].init(stage_a + c * f.max_unit_chunks * 16, base[c] + start[c]);
+        }
+        const uint32_t next_item = item + gridDim.x * warps;
+        if (next_item < f.items) load_index(next_item);
+        float acc[kChains] = {0.0f, 0.0f};
+        if (kMode == 0 && kXShared) {
+            const uint32_t sb = shared_base();
+            FastReader fr[kChains];
+            uint32_t ra[kChains];
+#pragma unroll
+            for (int c = 0; c < kChains; ++c) {
+                fr[c].hi = br[c].hi; fr[c].lo = br[c].lo; fr[c].off = br[c].off; fr[c].next = sb + br[c].next;
+                ra[c] = sb + ri_lane[c];
+            }
+            const uint32_t l1_abs = sb + dec.l1_lane, xs_abs = sb + xs_a;
+            auto step = [&](auto offset) {          // one entry of every chain: lookups first, then the rest
+                uint32_t top[kChains], val[kChains], len[kChains];
+#pragma unroll
+                for (int c = 0; c < kChains; ++c) fast_lookup(fr[c], dec.l1_shift, dec.l1_mul, l1_abs, top[c], val[c], len[c]);
+                if (kLong) {
+#pragma unroll
+                    for (int c = 0; c < kChains; ++c)
+                        if ((int32_t)len[c] < 0) resolve_long(top[c], dec, f, val[c], len[c]);
+                }
+#pragma unroll
+                for (int c = 0; c < kChains; ++c)
+                    fast_consume_sparse<kRow, decltype(offset)::value * kRow>(fr[c], val[c], len[c], ra[c], xs_abs, acc[c]);
+            };
+            uint32_t s = 0;
+            for (; s + 4 <= common; s += 4) {
+                step(std::integral_constant<int, 0>());
+                step(std::integral_constant<int, 1>());
+                step(std::integral_constant<int, 2>());
+                step(std::integral_constant<int, 3>());
+#pragma unroll
+                for (int c = 0; c < kChains; ++c) ra[c] += 4 * kRow;
+            }
+            for (; s < common; ++s) {
+                step(std::integral_constant<int, 0>());
+#pragma unroll
+                for (int c = 0; c < kChains; ++c) ra[c] += kRow;
+            }
+#pragma unroll
+            for (int c = 0; c < kChains; ++c) {              // the longer chain's remainder
+                br[c].hi = fr[c].hi; br[c].lo = fr[c].lo; br[c].off = fr[c].off; br[c].next = fr[c].next - sb;
+                uint32_t r = ra[c] - sb;
+                for (uint32_t t = common; t < count[c]; ++t) {
+                    const float w = decode_value<kLong>(br[c], dec, f);
+                    const uint32_t row = kRow == 2 ? lds16(r) : lds32(r);
+                    r += kRow;
+                    acc[c] = fmaf(ldsf(xs_a + (row << 2)), w, acc[c]);
+                }
+            }
+        } else if (kMode == 0) {
+#pragma unroll
+            for (int c = 0; c < kChains; ++c) {
+                uint32_t r = ri_lane[c];
+                for (uint32_t t = 0; t < count[c]; ++t) {
+                    const float w = decode_value<kLong>(br[c], dec, f);
+                    const uint32_t row = kRow == 2 ? lds16(r) : lds32(r);
+                    r += kRow;
+                    acc[c] = fmaf(x[(int64_t)row * xs_i], w, acc[c]);
+                }
+            }
+        } else {
+#pragma unroll
+            for (int c = 0; c < kChains; ++c) {
+                float* out = aux + cur.pos0[c] + lane_pos;
+                for (uint32_t t = 0; t < count[c]; ++t) out[t] = decode_value<kLong>(br[c], dec, f);
+            }
+        }
+        if (kMode == 0) {
+#pragma unroll
+            for (int c = 0; c < kChains; ++c) acc[c] = warp_sum(acc[c]);
+            if (lane == 0) {
+                if (cur.whole_column) {
+                    y[(int64_t)cur.col * ys_j] = acc[0] + acc[1];
+                } else {
+#pragma unroll
+                    for (int c = 0; c < kChains; ++c)
+                        if ((uint32_t)c < cur.segments) aux[cur.first_unit + c] = acc[c];
+                }
+            }
+        }
+        __syncwarp();
+        item = next_item;
+        if (item < f.items) fetch();
     }
 }
 
@@ -563,14 +754,14 @@ __global__ void __launch_bounds__(1024) shac_vec_kernel(DevFormat f, TablePlan t
 //   partial[u*batch + b]; HAC: segments j*G .. j*G+G-1; sHAC: seg_first[j] .. seg_first[j+1]-1.
 // Columns with exactly one segment were written by the product kernel itself.
 __global__ void finalize_kernel(DevFormat f, bool sparse, const float* __restrict__ partial, uint32_t batch,
-                                float* __restrict__ y, int64_t ys_j, int64_t ys_b) {
+                                float* __restrict__ y, int64_t ys_j, int64_t ys_b, uint32_t direct_up_to) {
     const uint64_t idx = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x;
     if (idx >= (uint64_t)f.m * batch) return;
     const uint32_t j = (uint32_t)(idx / batch), b = (uint32_t)(idx % batch);
     uint32_t u0, u1;
     if (sparse) { u0 = f.seg_first[j]; u1 = f.seg_first[j + 1]; }
     else { u0 = j * f.G; u1 = u0 + f.G; }
-    if (u1 - u0 == 1) return;
+    if (u1 - u0 >= 1 && u1 - u0 <= direct_up_to) return;       // written by the product kernel itself
     float s = 0.0f;
     for (uint32_t u = u0; u < u1; ++u) s += partial[(size_t)u * batch + b];
     y[(int64_t)j * ys_j + (int64_t)b * ys_b] = s;
@@ -796,6 +987,7 @@ static DevFormat dev_format(const Format& f) {
     d.stream = f.dev.stream; d.lut = f.dev.lut; d.rank_value = f.dev.rank_value;
     d.l1 = reinterpret_cast<const uint2*>(f.dev.l1); d.sub = reinterpret_cast<const uint2*>(f.dev.sub);
     d.l1_bits = (uint32_t)f.tables.l1_bits; d.sub_bytes = (uint32_t)(f.tables.sub.size() * 4);
+    d.items = (uint32_t)(f.item_info.size() / 12);
     d.limit = f.dev.limit; d.first_left = f.dev.first_left; d.rank_base = f.dev.rank_base;
     d.seg_bit_off = f.dev.seg_bit_off; d.sub_bits = f.dev.sub_bits; d.seg_col = f.dev.seg_col;
     d.seg_first = f.dev.seg_first; d.ri = f.dev.ri; d.cb = f.dev.cb; d.unit_info = f.dev.unit_info;
@@ -853,7 +1045,7 @@ static int upload(Format& f, void* dev_buf, size_t dev_bytes, void* stream_) {
     if (f.ri_bits == 16) HAC_CUDA(put(L.ri, f.ri16.data(), f.ri16.size() * 2));
     else HAC_CUDA(put(L.ri, f.ri32.data(), f.ri32.size() * 4));
     HAC_CUDA(put(L.cb, f.cb.data(), f.cb.size() * 4));
-    HAC_CUDA(put(L.unit_info, f.unit_info.data(), f.unit_info.size() * 4));
+    HAC_CUDA(put(L.unit_info, f.item_info.data(), f.item_info.size() * 4));
     // the source vectors are pageable host memory: wait so they may change or go away afterwards
     HAC_CUDA(cudaStreamSynchronize(st));
     set_pointers(f, dev_buf, dev_bytes);
@@ -867,13 +1059,10 @@ static int attach(Format& f, void* dev_buf, size_t dev_bytes) {
     return HAC_OK;
 }
 
-static bool needs_finalize(const Format& f) {
-    if (!f.sparse) return f.G > 1;
-    return f.max_units_per_col > 1 || f.has_empty_col;
-}
-
 static size_t workspace_bytes(const Format& f, int64_t batch) {
-    const bool partials = f.sparse ? f.max_units_per_col > 1 : f.G > 1;
+    // sHAC with one input handles up to two segments of a column in one warp; the batched kernels
+    // and HAC keep one partial per segment
+    const bool partials = f.sparse ? f.max_units_per_col > (batch == 1 ? 2u : 1u) : f.G > 1;
     return partials ? f.seg_bit_off.size() * (size_t)batch * 4 : 0;
 }
 
@@ -897,10 +1086,10 @@ static int fit_warps(size_t fixed, size_t per_warp, int want, int step, size_t b
 }
 
 static int launch_finalize(const Format& f, const DevFormat& d, const float* partial, int64_t batch, float* y,
-                           int64_t ys_j, int64_t ys_b, cudaStream_t st) {
+                           int64_t ys_j, int64_t ys_b, cudaStream_t st, uint32_t direct_up_to) {
     const uint64_t total = (uint64_t)f.m * (uint64_t)batch;
     const unsigned blocks = (unsigned)((total + 255) / 256);
-    finalize_kernel<<<blocks, 256, 0, st>>>(d, f.sparse, partial, (uint32_t)batch, y, ys_j, ys_b);
+    finalize_kernel<<<blocks, 256, 0, st>>>(d, f.sparse, partial, (uint32_t)batch, y, ys_j, ys_b, direct_up_to);
     HAC_CUDA(cudaGetLastError());
     f.last_launches++;
     return HAC_OK;
@@ -945,22 +1134,26 @@ static int launch_vec(const Format& f, int mode, const float* x, int64_t xs_i, f
     const size_t budget = (size_t)di.max_smem_optin;
     // HAC: two decode chains per lane when two staging areas per warp fit next to a fully
     // replicated table; sHAC: one
-    const int chains = (!f.sparse && d.units > 1) ? std::min(2, std::max(1, env_int("HAC_B200_CHAINS", 2))) : 1;
+    const int chains = f.sparse ? 2 : (d.units > 1 ? std::min(2, std::max(1, env_int("HAC_B200_CHAINS", 2))) : 1);
     size_t per_warp = (size_t)d.max_unit_chunks * 16 * chains;
-    if (f.sparse && mode == 0) per_warp += ((size_t)(32u * f.S * (f.ri_bits / 8) + 15u) / 16u + 1u) * 16u;
+    if (f.sparse && mode == 0) per_warp += ((size_t)(32u * f.S * (f.ri_bits / 8) + 15u) / 16u + 1u) * 16u * chains;
     size_t xbytes = 0;
     if (mode == 0) xbytes = f.sparse ? align16((size_t)f.n * 4) : align16(((size_t)f.n + (f.n / f.S + 1)) * 4);
     const int want = std::min(32, std::max(1, env_int("HAC_B200_VEC_WARPS", 32)));
     // shared memory: tables + x + per-warp staging.  Prefer keeping x and all warps; give up
     // replicas of the level-1 table before giving up warps.
     bool x_shared = mode == 0;
-    const size_t min_tables = plan_smem_bytes(d.l1_bits, 0, d.sub_bytes);
+    const size_t min_tables = plan_smem_bytes(d.l1_bits, 0, d.sub_bytes) + 16;
     if (x_shared && xbytes + min_tables + per_warp * std::min(want, 8) > budget) { x_shared = false; xbytes = 0; }
     int warps = want;
     while (warps > 1 && xbytes + min_tables + per_warp * (size_t)warps > budget) --warps;
     if (xbytes + min_tables + per_warp * (size_t)warps > budget) return HAC_ERR_BUFFER_TOO_SMALL;
-    const TablePlan tp = plan_tables(d, budget - xbytes - per_warp * (size_t)warps);
-    const size_t smem = plan_smem_bytes(d.l1_bits, tp.repl_log2, d.sub_bytes) + xbytes + per_warp * warps;
+    const size_t fixed = f.sparse ? 16 : 0;                 // mbarrier of the bulk copy of x
+    TablePlan tp = plan_tables(d, budget - fixed - xbytes - per_warp * (size_t)warps);
+    tp.x_bulk = (f.sparse && mode == 0 && x_shared && xs_i == 1 && (reinterpret_cast<uintptr_t>(x) & 15u) == 0 &&
+                 env_int("HAC_B200_X_BULK", 1) != 0)
+                    ? 1u : 0u;
+    const size_t smem = fixed + plan_smem_bytes(d.l1_bits, tp.repl_log2, d.sub_bytes) + xbytes + per_warp * warps;
     if (smem > budget) return HAC_ERR_BUFFER_TOO_SMALL;
     const bool has_long = d.max_len > d.l1_bits;
     const int threads = warps * 32;
@@ -972,7 +1165,7 @@ static int launch_vec(const Format& f, int mode, const float* x, int64_t xs_i, f
     HAC_CUDA(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kernel, threads, smem));
     per_sm = std::max(per_sm, 1);
     // spread the segments over all SMs (a block's warps take segments blockIdx + k * gridDim)
-    const unsigned items = (d.units + chains - 1) / chains;
+    const unsigned items = f.sparse ? d.items : (d.units + chains - 1) / chains;
     const unsigned grid = std::min<unsigned>(items, (unsigned)(di.sms * per_sm));
     kernel<<<grid, threads, smem, st>>>(d, tp, x, xs_i, y, ys_j, aux);
     if (vec_direct) *vec_direct = (!f.sparse && (f.G == 1 || (chains == 2 && f.G == 2)));
@@ -1060,7 +1253,18 @@ static int dot(const Format& f, const float* x, int64_t batch, int64_t xs_i, int
         }
         if (rc) return rc;
     }
-    if ((needs_finalize(f) && !direct) || d.units == 0) rc = launch_finalize(f, d, partial, batch, y, ys_j, ys_b, st);
+    // columns the product kernel did not finish itself (several segments, or none at all)
+    uint32_t direct_up_to = 1;
+    bool finish;
+    if (!f.sparse) {
+        finish = f.G > 1 && !direct;
+    } else if (batch == 1) {
+        direct_up_to = 2;
+        finish = f.max_units_per_col > 2 || f.has_empty_col;
+    } else {
+        finish = f.max_units_per_col > 1 || f.has_empty_col;
+    }
+    if (finish || d.units == 0) rc = launch_finalize(f, d, partial, batch, y, ys_j, ys_b, st, direct_up_to);
     return rc;
 }
 

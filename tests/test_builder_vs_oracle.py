@@ -63,7 +63,8 @@ def test_formats_bit_exact(wl, kind, S):
     W = si.weights(wl)
     Wq, mask, ofmt = oracle_format(W, wl, kind)
     lf = library_format(W, wl, kind, S)
-    S_eff = S or (64 if kind == "hac" else 32)
+    S_eff = lf.sizes()["seg_symbols"]
+    assert S_eff == S or (S == 0 and (S_eff == 64 if kind == "hac" else S_eff % 4 == 2))
     oidx = orc.hac_offset_index(ofmt, S_eff) if kind == "hac" else orc.shac_offset_index(ofmt, S_eff)
     assert_same_format(lf, ofmt, oidx, Wq)
 
@@ -76,7 +77,7 @@ def test_sweep_cells_small(k, sp):
     for kind in ("hac", "shac"):
         Wq, mask, ofmt = oracle_format(W, wl, kind)
         lf = library_format(W, wl, kind)
-        S_eff = 64 if kind == "hac" else 32
+        S_eff = lf.sizes()["seg_symbols"]
         oidx = orc.hac_offset_index(ofmt, S_eff) if kind == "hac" else orc.shac_offset_index(ofmt, S_eff)
         assert_same_format(lf, ofmt, oidx, Wq)
 
