@@ -241,6 +241,23 @@ __device__ __forceinline__ void fast_consume(FastReader& r, uint32_t val, uint32
         : "memory");
 }
 
+// The consume part alone (no multiply-accumulate): used where the decoded value goes to a tile.
+__device__ __forceinline__ void fast_consume_value(FastReader& r, uint32_t len) {
+    asm volatile(
+        "{\n\t"
+        ".reg .pred p;\n\t"
+        "add.u32 %2, %2, %4;\n\t"
+        "setp.ge.u32 p, %2, 32;\n\t"
+        "@p mov.u32 %0, %1;\n\t"
+        "@p ld.shared.u32 %1, [%3];\n\t"
+        "@p add.u32 %3, %3, 4;\n\t"
+        "and.b32 %2, %2, 31;\n\t"
+        "}"
+        : "+r"(r.hi), "+r"(r.lo), "+r"(r.off), "+r"(r.next)
+        : "r"(len)
+        : "memory");
+}
+
 // Same step for sHAC: the row of the entry comes from the staged slice of ri, x is gathered by row.
 template <int kRowBytes, int kRiOffset>
 __device__ __forceinline__ void fast_consume_sparse(FastReader& r, uint32_t val, uint32_t len, uint32_t ri_addr,
@@ -768,99 +785,221 @@ __global__ void finalize_kernel(DevFormat f, bool sparse, const float* __restric
 }
 
 // ------------------------------------------------------------------------------------------------
-// HAC, batch of inputs (Algorithm 3 without re-decoding W per input).  A block owns `kCols`
-// consecutive columns (one per warp) over the rows of one segment index g.  It alternates between
-// a decode phase (every lane decodes kSteps symbols of its sub-segment into a shared tile of
-// weights) and a product phase (the tile is applied to the matching rows of X, staged in shared
-// memory, for a tile of up to 32*kAcc inputs held in registers), so the stream is decoded once per
-// batch tile and never written to global memory.
+// HAC, batch of inputs (Algorithm 3 without re-decoding W per input), on the tensor cores.
+//
+// A block owns kGemmCols consecutive columns of W (one per warp),
+// a range of segment indices g (all of them unless the grid would be too small) and a tile of
+// kGemmBatch inputs.  It alternates between
+//   decode : every lane decodes 4 symbols of its sub-segment; the values are split
+//            into two TF32 parts (w = hi + lo) and stored as a [column][row] tile in shared memory;
+//   stage  : the 128 matching rows of X are copied to shared memory;
+//   product: the 32 x 64 output tile is updated with m16n8k8 TF32 tensor-core instructions, three
+//            per tile (lo*hi + hi*lo + hi*hi, fp32 accumulation), which keeps the result within
+//            about 1e-6 of sum |w x|.  The 16 row-steps of a chunk are split over 8 warp groups, whose
+//            partial tiles are added once at the end.
+// The stream is decoded once per batch tile and never written to global memory.
+// Fragment layout of mma.sync.m16n8k8 (gid = lane / 4, tig = lane % 4):
+//   A (16 x 8): a0 (gid, tig)  a1 (gid+8, tig)  a2 (gid, tig+4)  a3 (gid+8, tig+4)
+//   B ( 8 x 8): b0 (tig, gid)  b1 (tig+4, gid)
+//   C (16 x 8): c0 (gid, 2tig) c1 (gid, 2tig+1) c2 (gid+8, 2tig) c3 (gid+8, 2tig+1)
 // ------------------------------------------------------------------------------------------------
 constexpr int kBatchSteps = 4;          // symbols decoded per lane per phase
 constexpr int kBatchRows = 32 * kBatchSteps;
-constexpr int kAccMax = 4;              // batch tile = 32 * kAcc inputs
+constexpr int kAccMax = 4;              // sHAC batch tile = 32 * kAcc inputs
+constexpr int kGemmCols = 32;
+constexpr int kGemmBatch = 64;
+constexpr int kGemmWarps = 32;
+constexpr int kWtStride = kBatchRows + 4;     // floats per column of the weight tile (bank-conflict free)
+constexpr int kXtStride = kGemmBatch + 8;     // floats per row of the input tile
 
-template <int kAcc>
-__global__ void __launch_bounds__(1024) hac_batch_kernel(DevFormat f, TablePlan tp, const float* __restrict__ x,
-                                                         int64_t xs_i, int64_t xs_b, uint32_t batch,
-                                                         float* __restrict__ y, int64_t ys_j, int64_t ys_b,
-                                                         float* __restrict__ partial, uint32_t col_blocks) {
+__device__ __forceinline__ uint32_t to_tf32(float v) {
+    uint32_t r;
+    asm("cvt.rna.tf32.f32 %0, %1;" : "=r"(r) : "f"(v));
+    return r;
+}
+__device__ __forceinline__ void mma_tf32(float (&c)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
+    asm volatile(
+        "mma.sync.aligned.m16n8k8.row.col.f32.tf32.tf32.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+        : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+        : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
+}
+
+__host__ __device__ inline size_t gemm_tile_bytes() {
+    return align16((size_t)2 * kGemmCols * kWtStride * 4) + align16((size_t)kBatchRows * kXtStride * 4);
+}
+
+__global__ void __launch_bounds__(kGemmWarps * 32) hac_gemm_kernel(DevFormat f, TablePlan tp,
+                                                                  const float* __restrict__ x, int64_t xs_i,
+                                                                  int64_t xs_b, uint32_t batch, float* __restrict__ y,
+                                                                  int64_t ys_j, int64_t ys_b,
+                                                                  float* __restrict__ partial, uint32_t col_blocks,
+                                                                  uint32_t row_splits, uint32_t vec_x) {
+    const uint32_t warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const uint32_t gid = lane >> 2, tig = lane & 3;
+    // block -> (column block, row split, batch tile)
+    const uint32_t cblk = blockIdx.x % col_blocks;
+    const uint32_t rest = blockIdx.x / col_blocks;
+    const uint32_t rs = rest % row_splits, bt = rest / row_splits;
+    const uint32_t g_begin = (uint32_t)(((uint64_t)f.G * rs) / row_splits);
+    const uint32_t g_end = (uint32_t)(((uint64_t)f.G * (rs + 1)) / row_splits);
+    const uint32_t b0 = bt * kGemmBatch;
+
     unsigned char* p = smem;
     const Decoder dec = stage_decoder(f, tp, p);
-    const uint32_t warp = threadIdx.x >> 5, lane = threadIdx.x & 31, warps = blockDim.x >> 5;
-    constexpr uint32_t kTile = 32 * kAcc;
-    float* wt = reinterpret_cast<float*>(p);                       // [warps][kBatchRows]
-    p += align16((size_t)warps * kBatchRows * 4);
-    float* xt = reinterpret_cast<float*>(p);                       // [kBatchRows][kTile]
-    p += align16((size_t)kBatchRows * kTile * 4);
+    float* wt_hi = reinterpret_cast<float*>(p);                       // [kGemmCols][kWtStride]
+    float* wt_lo = wt_hi + kGemmCols * kWtStride;
+    p += align16((size_t)2 * kGemmCols * kWtStride * 4);
+    float* xt = reinterpret_cast<float*>(p);                          // [kBatchRows][kXtStride]
+    p += align16((size_t)kBatchRows * kXtStride * 4);
     uint4* stage = reinterpret_cast<uint4*>(p) + (size_t)warp * f.max_unit_chunks;
     const uint32_t stage_a = smem_off(stage);
     __syncthreads();
-    const uint32_t batch_tiles = (batch + kTile - 1) / kTile;
-    const uint32_t items = col_blocks * f.G * batch_tiles;
 
-    for (uint32_t item = blockIdx.x; item < items; item += gridDim.x) {
-        const uint32_t bt = item % batch_tiles;
-        const uint32_t rest = item / batch_tiles;
-        const uint32_t g = rest % f.G, cblk = rest / f.G;
-        const uint32_t j = cblk * warps + warp;
-        const bool live = j < f.m;
-        const uint32_t u = live ? j * f.G + g : 0u;
-        const uint32_t b0 = bt * kTile;
-        const uint32_t sub = g * 32 + lane;
-        const uint32_t row0 = sub * f.S;
-        uint32_t count = 0;
-        BitReader br;
-        br.hi = br.lo = br.off = 0; br.next = stage_a;
-        if (live) {
-            const uint32_t my_bits = f.sub_bits[(size_t)u * 32 + lane];
-            uint32_t total;
-            const uint32_t start = lane_start_bits(my_bits, lane, total);
-            const uint32_t base = stage_span(f, f.seg_bit_off[u], total, stage, lane);
-            count = row0 < f.n ? min(f.S, f.n - row0) : 0u;
-            br.init(stage_a, base + start);
-        }
-        float acc[kAcc];
+    // product-phase role of this warp: a quarter of the inputs (2 tiles of 8), two of the 16 row-steps
+    const uint32_t n_quarter = warp & 3u, ksplit = warp >> 2;
+    float acc[2][2][4];
 #pragma unroll
-        for (int a = 0; a < kAcc; ++a) acc[a] = 0.0f;
-        const uint32_t seg_rows = min(f.S, f.n - min(f.n, g * 32 * f.S));   // longest sub-segment here
-        for (uint32_t s0 = 0; s0 < seg_rows; s0 += kBatchSteps) {
-            // decode phase: kBatchSteps symbols per lane -> wt[warp][lane*kBatchSteps + s]
+    for (int mt = 0; mt < 2; ++mt)
 #pragma unroll
-            for (int s = 0; s < kBatchSteps; ++s) {
-                float v = 0.0f;
-                if (s0 + s < count) v = decode_value<true>(br, dec, f);
-                wt[warp * kBatchRows + lane * kBatchSteps + s] = v;
-            }
-            // matching rows of X: tile row r = l*kBatchSteps + s  <->  matrix row (g*32+l)*S + s0 + s
-            for (uint32_t idx = threadIdx.x; idx < kBatchRows * kTile; idx += blockDim.x) {
-                const uint32_t r = idx / kTile, bb = idx - r * kTile;
-                const uint32_t l = r / kBatchSteps, s = r - l * kBatchSteps;
-                const uint32_t row = (g * 32 + l) * f.S + s0 + s;
-                const uint32_t b = b0 + bb;
-                float v = 0.0f;
-                if (s0 + s < f.S && row < f.n && b < batch) v = x[(int64_t)row * xs_i + (int64_t)b * xs_b];
-                xt[idx] = v;
-            }
-            __syncthreads();
-            // product phase: this warp's column against the tile, lanes over inputs
-            const float* w = wt + warp * kBatchRows;
-#pragma unroll 4
-            for (uint32_t r = 0; r < kBatchRows; ++r) {
-                const float wv = w[r];
+        for (int nt = 0; nt < 2; ++nt)
 #pragma unroll
-                for (int a = 0; a < kAcc; ++a) acc[a] = fmaf(wv, xt[r * kTile + a * 32 + lane], acc[a]);
-            }
-            __syncthreads();
-        }
-        if (live) {
+            for (int i = 0; i < 4; ++i) acc[mt][nt][i] = 0.0f;
+
+    // rows of X for one chunk, two float4 per thread, fetched one chunk ahead of their use
+    constexpr int kXPerThread = kBatchRows * (kGemmBatch / 4) / (kGemmWarps * 32);
+    float4 xr[kXPerThread];
+    auto load_x = [&](uint32_t g, uint32_t s0) {
 #pragma unroll
-            for (int a = 0; a < kAcc; ++a) {
-                const uint32_t b = b0 + a * 32 + lane;
-                if (b < batch) {
-                    if (f.G == 1) y[(int64_t)j * ys_j + (int64_t)b * ys_b] = acc[a];
-                    else partial[(size_t)u * batch + b] = acc[a];
+        for (int i = 0; i < kXPerThread; ++i) {
+            const uint32_t idx = threadIdx.x + i * (kGemmWarps * 32);
+            const uint32_t r = idx / (kGemmBatch / 4), q = idx % (kGemmBatch / 4);
+            const uint32_t l = r / kBatchSteps, s = r % kBatchSteps;
+            const uint32_t row = (g * 32 + l) * f.S + s0 + s;      // tile row r <-> matrix row
+            const uint32_t b = b0 + q * 4;
+            float4 v = make_float4(0.0f, 0.0f, 0.0f, 0.0f);
+            if (s0 + s < f.S && row < f.n) {
+                const float* src = x + (int64_t)row * xs_i + (int64_t)b * xs_b;
+                if (vec_x && b + 3 < batch) {
+                    v = __ldg(reinterpret_cast<const float4*>(src));
+                } else {
+                    if (b < batch) v.x = __ldg(src);
+                    if (b + 1 < batch) v.y = __ldg(src + xs_b);
+                    if (b + 2 < batch) v.z = __ldg(src + 2 * xs_b);
+                    if (b + 3 < batch) v.w = __ldg(src + 3 * xs_b);
                 }
             }
+            xr[i] = v;
+        }
+    };
+    auto store_x = [&]() {
+#pragma unroll
+        for (int i = 0; i < kXPerThread; ++i) {
+            const uint32_t idx = threadIdx.x + i * (kGemmWarps * 32);
+            const uint32_t r = idx / (kGemmBatch / 4), q = idx % (kGemmBatch / 4);
+            *reinterpret_cast<float4*>(xt + r * kXtStride + q * 4) = xr[i];
+        }
+    };
+    if (g_begin < g_end) load_x(g_begin, 0);
+
+    const uint32_t sb = shared_base();
+    const uint32_t l1_abs = sb + dec.l1_lane;
+    const uint32_t j_mine = cblk * kGemmCols + warp;                  // decode-phase role: one column per warp
+    for (uint32_t g = g_begin; g < g_end; ++g) {
+        FastReader fr;
+        uint32_t count = 0;
+        fr.hi = fr.lo = fr.off = 0; fr.next = sb + stage_a;
+        if (j_mine < f.m) {
+            const uint32_t u = j_mine * f.G + g;
+            const uint32_t my_bits = __ldg(f.sub_bits + (size_t)u * 32 + lane);
+            uint32_t total;
+            const uint32_t start = lane_start_bits(my_bits, lane, total);
+            const uint32_t base = stage_span(f, __ldg(f.seg_bit_off + u), total, stage, lane);
+            const uint32_t row0 = (g * 32 + lane) * f.S;
+            count = row0 < f.n ? min(f.S, f.n - row0) : 0u;
+            BitReader br;
+            br.init(stage_a, base + start);
+            fr.hi = br.hi; fr.lo = br.lo; fr.off = br.off; fr.next = sb + br.next;
+        }
+        const uint32_t seg_rows = min(f.S, f.n - min(f.n, g * 32 * f.S));     // longest sub-segment here
+        for (uint32_t s0 = 0; s0 < seg_rows; s0 += kBatchSteps) {
+            // decode: 4 symbols -> tile rows lane*4 .. lane*4+3 of this warp's column, as TF32 hi + lo
+            float hi[kBatchSteps], lo[kBatchSteps];
+#pragma unroll
+            for (int s = 0; s < kBatchSteps; ++s) {
+                uint32_t top = 0, val = 0, len = 0;
+                if (s0 + s < count) {
+                    fast_lookup(fr, dec.l1_shift, dec.l1_mul, l1_abs, top, val, len);
+                    if ((int32_t)len < 0) resolve_long(top, dec, f, val, len);
+                    fast_consume_value(fr, len);
+                }
+                const float w = __uint_as_float(val);
+                hi[s] = __uint_as_float(to_tf32(w));
+                lo[s] = __uint_as_float(to_tf32(w - hi[s]));
+            }
+            const uint32_t at = warp * kWtStride + lane * kBatchSteps;
+            *reinterpret_cast<float4*>(wt_hi + at) = make_float4(hi[0], hi[1], hi[2], hi[3]);
+            *reinterpret_cast<float4*>(wt_lo + at) = make_float4(lo[0], lo[1], lo[2], lo[3]);
+            store_x();
+            __syncthreads();
+            // the next chunk's rows of X are requested now and land during the product phase
+            if (s0 + kBatchSteps < seg_rows) load_x(g, s0 + kBatchSteps);
+            else if (g + 1 < g_end) load_x(g + 1, 0);
+            // product: row-steps 2*ksplit and 2*ksplit+1 (8 tile rows each)
+#pragma unroll
+            for (int kq = 0; kq < 2; ++kq) {
+                const uint32_t k0 = (2 * ksplit + kq) * 8;
+                uint32_t b_hi[2][2], b_lo[2][2];
+#pragma unroll
+                for (int nt = 0; nt < 2; ++nt) {
+                    const uint32_t col = n_quarter * 16 + nt * 8 + gid;
+                    const float x0 = xt[(k0 + tig) * kXtStride + col];
+                    const float x1 = xt[(k0 + tig + 4) * kXtStride + col];
+                    b_hi[nt][0] = to_tf32(x0); b_hi[nt][1] = to_tf32(x1);
+                    b_lo[nt][0] = to_tf32(x0 - __uint_as_float(b_hi[nt][0]));
+                    b_lo[nt][1] = to_tf32(x1 - __uint_as_float(b_hi[nt][1]));
+                }
+#pragma unroll
+                for (int mt = 0; mt < 2; ++mt) {
+                    const uint32_t c0 = (16 * mt + gid) * kWtStride + k0 + tig;
+                    const uint32_t c8 = c0 + 8 * kWtStride;
+                    uint32_t a_hi[4], a_lo[4];
+                    a_hi[0] = __float_as_uint(wt_hi[c0]);     a_lo[0] = __float_as_uint(wt_lo[c0]);
+                    a_hi[1] = __float_as_uint(wt_hi[c8]);     a_lo[1] = __float_as_uint(wt_lo[c8]);
+                    a_hi[2] = __float_as_uint(wt_hi[c0 + 4]); a_lo[2] = __float_as_uint(wt_lo[c0 + 4]);
+                    a_hi[3] = __float_as_uint(wt_hi[c8 + 4]); a_lo[3] = __float_as_uint(wt_lo[c8 + 4]);
+#pragma unroll
+                    for (int nt = 0; nt < 2; ++nt) {
+                        mma_tf32(acc[mt][nt], a_lo, b_hi[nt][0], b_hi[nt][1]);
+                        mma_tf32(acc[mt][nt], a_hi, b_lo[nt][0], b_lo[nt][1]);
+                        mma_tf32(acc[mt][nt], a_hi, b_hi[nt][0], b_hi[nt][1]);
+                    }
+                }
+            }
+            __syncthreads();
+        }
+    }
+    // add the 8 row-split partial tiles: red[warp][register][lane] reuses the tile area
+    float* red = wt_hi;
+#pragma unroll
+    for (int mt = 0; mt < 2; ++mt)
+#pragma unroll
+        for (int nt = 0; nt < 2; ++nt)
+#pragma unroll
+            for (int i = 0; i < 4; ++i) red[(warp * 16 + (mt * 8 + nt * 4 + i)) * 32 + lane] = acc[mt][nt][i];
+    __syncthreads();
+    for (uint32_t o = threadIdx.x; o < kGemmCols * kGemmBatch; o += blockDim.x) {
+        const uint32_t col = o / kGemmBatch, bb = o % kGemmBatch;
+        const uint32_t quarter = bb / 16, nt = (bb % 16) / 8, cpos = bb % 8;
+        const uint32_t mt = col / 16, r16 = col % 16;
+        const uint32_t reg = mt * 8 + nt * 4 + (r16 / 8) * 2 + (cpos & 1u);
+        const uint32_t ln = (r16 % 8) * 4 + cpos / 2;
+        float sum = 0.0f;
+#pragma unroll
+        for (uint32_t ks = 0; ks < kGemmWarps / 4; ++ks) sum += red[((ks * 4 + quarter) * 16 + reg) * 32 + ln];
+        const uint32_t j = cblk * kGemmCols + col, b = b0 + bb;
+        if (j < f.m && b < batch) {
+            if (row_splits == 1) y[(int64_t)j * ys_j + (int64_t)b * ys_b] = sum;
+            else partial[((size_t)j * row_splits + rs) * batch + b] = sum;
         }
     }
 }
@@ -1174,6 +1313,38 @@ static int launch_vec(const Format& f, int mode, const float* x, int64_t xs_i, f
     return HAC_OK;
 }
 
+// Row splits of the tensor-core HAC kernel: 1 (a block owns whole columns and writes y itself)
+// unless that leaves most of the SMs idle.
+static uint32_t gemm_row_splits(const Format& f, int64_t batch, int sms) {
+    const uint64_t blocks = (uint64_t)((f.m + kGemmCols - 1) / kGemmCols) * (uint64_t)((batch + kGemmBatch - 1) / kGemmBatch);
+    if (blocks * 5 >= (uint64_t)sms * 3 || f.G <= 1) return 1;
+    return (uint32_t)std::min<uint64_t>(f.G, std::max<uint64_t>(1, (uint64_t)sms / blocks));
+}
+
+static int launch_gemm(const Format& f, const DeviceInfo& di, const DevFormat& d, const float* x, int64_t xs_i,
+                       int64_t xs_b, int64_t batch, float* y, int64_t ys_j, int64_t ys_b, float* partial,
+                       cudaStream_t st, uint32_t* row_splits_out) {
+    const size_t budget = (size_t)di.max_smem_optin;
+    const size_t fixed = gemm_tile_bytes() + (size_t)kGemmWarps * d.max_unit_chunks * 16;
+    if (fixed + plan_smem_bytes(d.l1_bits, 0, d.sub_bytes) > budget) return HAC_ERR_BUFFER_TOO_SMALL;
+    const TablePlan tp = plan_tables(d, budget - fixed);
+    const size_t smem = fixed + plan_smem_bytes(d.l1_bits, tp.repl_log2, d.sub_bytes);
+    int rc = prepare_kernel(hac_gemm_kernel, smem);
+    if (rc) return rc;
+    const uint32_t col_blocks = (uint32_t)((f.m + kGemmCols - 1) / kGemmCols);
+    const uint32_t batch_tiles = (uint32_t)((batch + kGemmBatch - 1) / kGemmBatch);
+    const uint32_t rs = gemm_row_splits(f, batch, di.sms);
+    const uint32_t vec_x = (xs_b == 1 && (xs_i % 4) == 0 && (reinterpret_cast<uintptr_t>(x) & 15u) == 0) ? 1u : 0u;
+    const uint64_t grid = (uint64_t)col_blocks * rs * batch_tiles;
+    if (grid > 0x7fffffffull) return HAC_ERR_OFFSET_OVERFLOW;
+    hac_gemm_kernel<<<(unsigned)grid, kGemmWarps * 32, smem, st>>>(d, tp, x, xs_i, xs_b, (uint32_t)batch, y, ys_j, ys_b,
+                                                                  partial, col_blocks, rs, vec_x);
+    HAC_CUDA(cudaGetLastError());
+    f.last_launches++;
+    *row_splits_out = rs;
+    return HAC_OK;
+}
+
 template <int kAcc>
 static int launch_batch_t(const Format& f, const DeviceInfo& di, const DevFormat& d, const float* x, int64_t xs_i,
                           int64_t xs_b, int64_t batch, float* y, int64_t ys_j, int64_t ys_b, float* partial,
@@ -1183,42 +1354,21 @@ static int launch_batch_t(const Format& f, const DeviceInfo& di, const DevFormat
     const size_t tab = plan_smem_bytes(d.l1_bits, tp.repl_log2, d.sub_bytes);
     constexpr uint32_t kTile = 32 * kAcc;
     const uint32_t batch_tiles = (uint32_t)((batch + kTile - 1) / kTile);
-    int rc;
-    if (!f.sparse) {
-        const size_t fixed = tab + align16((size_t)kBatchRows * kTile * 4) + 16;
-        const size_t per_warp = (size_t)d.max_unit_chunks * 16 + kBatchRows * 4;
-        const int want = std::min(32, std::max(1, env_int("HAC_B200_BATCH_WARPS", 16)));
-        const int warps = fit_warps(fixed, per_warp, want, 1, budget);
-        if (warps == 0) return HAC_ERR_BUFFER_TOO_SMALL;
-        const size_t smem = fixed + per_warp * warps;
-        auto kernel = hac_batch_kernel<kAcc>;
-        rc = prepare_kernel(kernel, smem);
-        if (rc) return rc;
-        int per_sm = 1;
-        HAC_CUDA(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kernel, warps * 32, smem));
-        per_sm = std::max(per_sm, 1);
-        const uint32_t col_blocks = (uint32_t)((f.m + warps - 1) / warps);
-        const uint64_t items = (uint64_t)col_blocks * d.G * batch_tiles;
-        const unsigned grid = (unsigned)std::min<uint64_t>(items, (uint64_t)di.sms * per_sm);
-        kernel<<<grid, warps * 32, smem, st>>>(d, tp, x, xs_i, xs_b, (uint32_t)batch, y, ys_j, ys_b, partial,
-                                               col_blocks);
-    } else {
-        const size_t per_warp = (size_t)d.max_unit_chunks * 16 + 2 * kBatchRows * 4;
-        const int want = std::min(32, std::max(1, env_int("HAC_B200_BATCH_WARPS", 8)));
-        const int warps = fit_warps(tab + 32, per_warp, want, 1, budget);
-        if (warps == 0) return HAC_ERR_BUFFER_TOO_SMALL;
-        const size_t smem = tab + 32 + per_warp * warps;
-        void (*kernel)(DevFormat, TablePlan, const float*, int64_t, int64_t, uint32_t, float*, int64_t, int64_t,
-                       float*) = f.ri_bits == 16 ? shac_batch_kernel<kAcc, uint16_t> : shac_batch_kernel<kAcc, uint32_t>;
-        rc = prepare_kernel(kernel, smem);
-        if (rc) return rc;
-        int per_sm = 1;
-        HAC_CUDA(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kernel, warps * 32, smem));
-        per_sm = std::max(per_sm, 1);
-        const uint64_t items = (uint64_t)d.units * batch_tiles;
-        const unsigned grid = (unsigned)std::min<uint64_t>((items + warps - 1) / warps, (uint64_t)di.sms * per_sm);
-        kernel<<<grid, warps * 32, smem, st>>>(d, tp, x, xs_i, xs_b, (uint32_t)batch, y, ys_j, ys_b, partial);
-    }
+    const size_t per_warp = (size_t)d.max_unit_chunks * 16 + 2 * kBatchRows * 4;
+    const int want = std::min(32, std::max(1, env_int("HAC_B200_BATCH_WARPS", 8)));
+    const int warps = fit_warps(tab + 32, per_warp, want, 1, budget);
+    if (warps == 0) return HAC_ERR_BUFFER_TOO_SMALL;
+    const size_t smem = tab + 32 + per_warp * warps;
+    void (*kernel)(DevFormat, TablePlan, const float*, int64_t, int64_t, uint32_t, float*, int64_t, int64_t,
+                   float*) = f.ri_bits == 16 ? shac_batch_kernel<kAcc, uint16_t> : shac_batch_kernel<kAcc, uint32_t>;
+    int rc = prepare_kernel(kernel, smem);
+    if (rc) return rc;
+    int per_sm = 1;
+    HAC_CUDA(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kernel, warps * 32, smem));
+    per_sm = std::max(per_sm, 1);
+    const uint64_t items = (uint64_t)d.units * batch_tiles;
+    const unsigned grid = (unsigned)std::min<uint64_t>((items + warps - 1) / warps, (uint64_t)di.sms * per_sm);
+    kernel<<<grid, warps * 32, smem, st>>>(d, tp, x, xs_i, xs_b, (uint32_t)batch, y, ys_j, ys_b, partial);
     HAC_CUDA(cudaGetLastError());
     f.last_launches++;
     return HAC_OK;
@@ -1236,6 +1386,7 @@ static int dot(const Format& f, const float* x, int64_t batch, int64_t xs_i, int
     const DevFormat d = dev_format(f);
     int rc = HAC_OK;
     bool direct = false;                     // the product kernel wrote every output itself
+    uint32_t gemm_splits = 0;                // batched HAC: row splits used (1 = outputs written directly)
     if (d.units > 0) {
         if (batch == 1) {
             rc = launch_vec(f, 0, x, xs_i, y, ys_j, partial, st, &direct);
@@ -1243,12 +1394,16 @@ static int dot(const Format& f, const float* x, int64_t batch, int64_t xs_i, int
             DeviceInfo di;
             rc = device_info(di);
             if (rc) return rc;
-            const int acc = (int)std::min<int64_t>(kAccMax, (batch + 31) / 32);
-            switch (acc) {
-                case 1: rc = launch_batch_t<1>(f, di, d, x, xs_i, xs_b, batch, y, ys_j, ys_b, partial, st); break;
-                case 2: rc = launch_batch_t<2>(f, di, d, x, xs_i, xs_b, batch, y, ys_j, ys_b, partial, st); break;
-                case 3: rc = launch_batch_t<3>(f, di, d, x, xs_i, xs_b, batch, y, ys_j, ys_b, partial, st); break;
-                default: rc = launch_batch_t<4>(f, di, d, x, xs_i, xs_b, batch, y, ys_j, ys_b, partial, st); break;
+            if (!f.sparse) {
+                rc = launch_gemm(f, di, d, x, xs_i, xs_b, batch, y, ys_j, ys_b, partial, st, &gemm_splits);
+            } else {
+                const int acc = (int)std::min<int64_t>(kAccMax, (batch + 31) / 32);
+                switch (acc) {
+                    case 1: rc = launch_batch_t<1>(f, di, d, x, xs_i, xs_b, batch, y, ys_j, ys_b, partial, st); break;
+                    case 2: rc = launch_batch_t<2>(f, di, d, x, xs_i, xs_b, batch, y, ys_j, ys_b, partial, st); break;
+                    case 3: rc = launch_batch_t<3>(f, di, d, x, xs_i, xs_b, batch, y, ys_j, ys_b, partial, st); break;
+                    default: rc = launch_batch_t<4>(f, di, d, x, xs_i, xs_b, batch, y, ys_j, ys_b, partial, st); break;
+                }
             }
         }
         if (rc) return rc;
@@ -1256,7 +1411,11 @@ static int dot(const Format& f, const float* x, int64_t batch, int64_t xs_i, int
     // columns the product kernel did not finish itself (several segments, or none at all)
     uint32_t direct_up_to = 1;
     bool finish;
-    if (!f.sparse) {
+    DevFormat dfin = d;
+    if (!f.sparse && batch > 1) {
+        finish = gemm_splits > 1;            // partial[(j * splits + split) * batch + b]
+        dfin.G = gemm_splits;
+    } else if (!f.sparse) {
         finish = f.G > 1 && !direct;
     } else if (batch == 1) {
         direct_up_to = 2;
@@ -1264,7 +1423,7 @@ static int dot(const Format& f, const float* x, int64_t batch, int64_t xs_i, int
     } else {
         finish = f.max_units_per_col > 1 || f.has_empty_col;
     }
-    if (finish || d.units == 0) rc = launch_finalize(f, d, partial, batch, y, ys_j, ys_b, st, direct_up_to);
+    if (finish || d.units == 0) rc = launch_finalize(f, dfin, partial, batch, y, ys_j, ys_b, st, direct_up_to);
     return rc;
 }
 
