@@ -1005,6 +1005,217 @@ __global__ void __launch_bounds__(kGemmWarps * 32) hac_gemm_kernel(DevFormat f, 
 }
 
 // ------------------------------------------------------------------------------------------------
+// The same batched HAC product on the 5th-generation tensor cores (tcgen05), accumulators in
+// tensor memory.  One MMA is D[64 inputs][32 columns] += X[64][8] * W[32][8]^T in TF32; both operands
+// are read by the tensor core straight from shared memory ("K-major", no swizzle): a group of four
+// consecutive K elements of one row is a 16-byte unit, 8 rows form a 128-byte core matrix, core
+// matrices of successive 8-row groups are kTcSbo bytes apart, the two K halves of an MMA are LBO
+// bytes apart.  Strides are padded so that the stores of the decode phase hit distinct banks.
+// Split precision as above: x_lo*w_hi + x_hi*w_lo + x_hi*w_hi, every part rounded to TF32 first.
+// For 64 inputs the accumulator rows sit in tensor-memory lanes 0-15, 32-47, 64-79 and 96-111.
+// ------------------------------------------------------------------------------------------------
+constexpr int kTcSteps = 2;                         // symbols decoded per lane per chunk
+constexpr int kTcRows = 32 * kTcSteps;              // K per chunk (64)
+constexpr int kTcKSteps = kTcRows / 8;              // MMAs (of K = 8) per chunk and product
+constexpr int kTcSbo = 128;
+constexpr int kTcXLbo = 1024, kTcXKst = 2048;       // X tile: 64 rows -> 8 core matrices per K half
+constexpr int kTcWLbo = 528, kTcWKst = 1056;        // W tile: 32 rows -> 4 core matrices, padded
+constexpr int kTcCols = 32, kTcBatch = 64, kTcWarps = 32;
+constexpr uint32_t kTcWaitTries = 4000000;
+
+__host__ __device__ inline size_t tc_tile_bytes() {
+    return (size_t)2 * kTcKSteps * kTcXKst + (size_t)2 * kTcKSteps * kTcWKst;
+}
+__device__ __forceinline__ uint64_t tc_desc(uint32_t shared_addr, uint32_t lbo_bytes) {
+    return (uint64_t)((shared_addr >> 4) & 0x3fffu) | ((uint64_t)((lbo_bytes >> 4) & 0x3fffu) << 16) |
+           ((uint64_t)((kTcSbo >> 4) & 0x3fffu) << 32) | ((uint64_t)1 << 46);
+}
+__device__ __forceinline__ void tc_mma(uint32_t tmem, uint64_t a, uint64_t b, uint32_t idesc, uint32_t accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::tf32 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(tmem), "l"(a), "l"(b), "r"(idesc), "r"(accumulate) : "memory");
+}
+__device__ __forceinline__ void tc_commit(uint32_t mbar) {
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(mbar) : "memory");
+}
+__device__ __forceinline__ bool tc_wait(uint32_t mbar, uint32_t parity) {
+    for (uint32_t t = 0; t < kTcWaitTries; ++t) {
+        uint32_t done;
+        asm volatile("{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}"
+                     : "=r"(done) : "r"(mbar), "r"(parity) : "memory");
+        if (done) return true;
+    }
+    return false;
+}
+
+__global__ void __launch_bounds__(kTcWarps * 32) hac_gemm_tc_kernel(DevFormat f, TablePlan tp,
+                                                                   const float* __restrict__ x, int64_t xs_i,
+                                                                   int64_t xs_b, uint32_t batch, float* __restrict__ y,
+                                                                   int64_t ys_j, int64_t ys_b,
+                                                                   float* __restrict__ partial, uint32_t col_blocks,
+                                                                   uint32_t row_splits) {
+    const uint32_t warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const uint32_t cblk = blockIdx.x % col_blocks;
+    const uint32_t rest = blockIdx.x / col_blocks;
+    const uint32_t rs = rest % row_splits, bt = rest / row_splits;
+    const uint32_t g_begin = (uint32_t)(((uint64_t)f.G * rs) / row_splits);
+    const uint32_t g_end = (uint32_t)(((uint64_t)f.G * (rs + 1)) / row_splits);
+    const uint32_t b0 = bt * kTcBatch;
+    const uint32_t sb = shared_base();
+
+    // shared memory: [mbarrier, tensor-memory address] [tables] [X hi, X lo, W hi, W lo tiles] [staged spans]
+    unsigned char* p = smem;
+    const uint32_t mbar = sb;
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem + 8);
+    p += 16;
+    if (threadIdx.x == 0) mbar_init(mbar, 1);
+    __syncwarp();
+    if (warp == 0) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(sb + 8), "r"(32u) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    const Decoder dec = stage_decoder(f, tp, p);
+    p = smem + ((smem_off(p) + 127u) & ~127u);
+    unsigned char* x_hi = p;
+    unsigned char* x_lo = x_hi + kTcKSteps * kTcXKst;
+    unsigned char* w_hi = x_lo + kTcKSteps * kTcXKst;
+    unsigned char* w_lo = w_hi + kTcKSteps * kTcWKst;
+    p = w_lo + kTcKSteps * kTcWKst;
+    uint4* stage = reinterpret_cast<uint4*>(p) + (size_t)warp * f.max_unit_chunks;
+    const uint32_t stage_a = smem_off(stage);
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    __syncthreads();
+    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+    const uint32_t tmem = *tmem_slot;
+
+    // staging role: K group q (tile rows 4q..4q+3 = sub-segments 2q and 2q+1, two symbols each), input b
+    const uint32_t xq = threadIdx.x / kTcBatch, xb = threadIdx.x % kTcBatch;
+    const uint32_t x_at = (xq >> 1) * kTcXKst + (xq & 1u) * kTcXLbo + (xb >> 3) * kTcSbo + (xb & 7u) * 16;
+    float xr[4];
+    auto load_x = [&](uint32_t g, uint32_t s0) {
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            const uint32_t l = 2 * xq + (i >> 1), s = i & 1;
+            const uint32_t row = (g * 32 + l) * f.S + s0 + s;
+            float v = 0.0f;
+            if (s0 + s < f.S && row < f.n && b0 + xb < batch) v = __ldg(x + (int64_t)row * xs_i + (int64_t)(b0 + xb) * xs_b);
+            xr[i] = v;
+        }
+    };
+    if (g_begin < g_end) load_x(g_begin, 0);
+    // decode role: column cblk*32 + warp; tile row of symbol s of lane l is 2l + s
+    const uint32_t j_mine = cblk * kTcCols + warp;
+    const uint32_t wq = lane >> 1;
+    const uint32_t w_at = (wq >> 1) * kTcWKst + (wq & 1u) * kTcWLbo + (warp >> 3) * kTcSbo + (warp & 7u) * 16 + (lane & 1u) * 8;
+    const uint32_t l1_abs = sb + dec.l1_lane;
+    const uint32_t idesc = (1u << 4) | (2u << 7) | (2u << 10) | ((uint32_t)(kTcCols >> 3) << 17) | ((uint32_t)(kTcBatch >> 4) << 24);
+    uint32_t chunk = 0;
+    bool lost = false;                       // a wait ran out: results are not to be trusted
+
+    for (uint32_t g = g_begin; g < g_end; ++g) {
+        FastReader fr;
+        uint32_t count = 0;
+        fr.hi = fr.lo = fr.off = 0; fr.next = sb + stage_a;
+        if (j_mine < f.m) {
+            const uint32_t u = j_mine * f.G + g;
+            const uint32_t my_bits = __ldg(f.sub_bits + (size_t)u * 32 + lane);
+            uint32_t total;
+            const uint32_t start = lane_start_bits(my_bits, lane, total);
+            const uint32_t base = stage_span(f, __ldg(f.seg_bit_off + u), total, stage, lane);
+            const uint32_t row0 = (g * 32 + lane) * f.S;
+            count = row0 < f.n ? min(f.S, f.n - row0) : 0u;
+            BitReader br;
+            br.init(stage_a, base + start);
+            fr.hi = br.hi; fr.lo = br.lo; fr.off = br.off; fr.next = sb + br.next;
+        }
+        const uint32_t seg_rows = min(f.S, f.n - min(f.n, g * 32 * f.S));
+        for (uint32_t s0 = 0; s0 < seg_rows; s0 += kTcSteps, ++chunk) {
+            float hi[kTcSteps], lo[kTcSteps];
+#pragma unroll
+            for (int s = 0; s < kTcSteps; ++s) {
+                uint32_t top = 0, val = 0, len = 0;
+                if (s0 + s < count) {
+                    fast_lookup(fr, dec.l1_shift, dec.l1_mul, l1_abs, top, val, len);
+                    if ((int32_t)len < 0) resolve_long(top, dec, f, val, len);
+                    fast_consume_value(fr, len);
+                }
+                const float w = __uint_as_float(val);
+                hi[s] = __uint_as_float(to_tf32(w));
+                lo[s] = __uint_as_float(to_tf32(w - hi[s]));
+            }
+            float xh[4], xl[4];
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                xh[i] = __uint_as_float(to_tf32(xr[i]));
+                xl[i] = __uint_as_float(to_tf32(xr[i] - xh[i]));
+            }
+            // the tensor core must be done reading the previous chunk's tiles before they change
+            if (chunk > 0 && !tc_wait(mbar, (chunk - 1) & 1u)) lost = true;
+            *reinterpret_cast<float2*>(w_hi + w_at) = make_float2(hi[0], hi[1]);
+            *reinterpret_cast<float2*>(w_lo + w_at) = make_float2(lo[0], lo[1]);
+            *reinterpret_cast<float4*>(x_hi + x_at) = make_float4(xh[0], xh[1], xh[2], xh[3]);
+            *reinterpret_cast<float4*>(x_lo + x_at) = make_float4(xl[0], xl[1], xl[2], xl[3]);
+            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+            asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+            __syncthreads();
+            if (threadIdx.x == 0) {
+                asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+#pragma unroll
+                for (int ks = 0; ks < kTcKSteps; ++ks) {
+                    const uint64_t a_hi = tc_desc(sb + smem_off(x_hi) + ks * kTcXKst, kTcXLbo);
+                    const uint64_t a_lo = tc_desc(sb + smem_off(x_lo) + ks * kTcXKst, kTcXLbo);
+                    const uint64_t b_hi = tc_desc(sb + smem_off(w_hi) + ks * kTcWKst, kTcWLbo);
+                    const uint64_t b_lo = tc_desc(sb + smem_off(w_lo) + ks * kTcWKst, kTcWLbo);
+                    tc_mma(tmem, a_lo, b_hi, idesc, (chunk | (uint32_t)ks) ? 1u : 0u);
+                    tc_mma(tmem, a_hi, b_lo, idesc, 1u);
+                    tc_mma(tmem, a_hi, b_hi, idesc, 1u);
+                }
+                tc_commit(mbar);
+            }
+            // the next chunk's rows of X are requested now and land while it is being decoded
+            if (s0 + kTcSteps < seg_rows) load_x(g, s0 + kTcSteps);
+            else if (g + 1 < g_end) load_x(g + 1, 0);
+        }
+    }
+    if (chunk > 0 && !tc_wait(mbar, (chunk - 1) & 1u)) lost = true;
+    const bool any_lost = __syncthreads_or(lost ? 1 : 0) != 0;
+    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+    if (warp < 4) {                          // warp w reads tensor-memory lanes 32w..32w+31: inputs 16w..16w+15
+        uint32_t r[32];
+        if (chunk > 0 && !any_lost) {
+            const uint32_t src = tmem + ((warp * 32u) << 16);
+            asm volatile(
+                "tcgen05.ld.sync.aligned.32x32b.x32.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,%17,%18,%19,"
+                "%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31}, [%32];"
+                : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+                  "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
+                  "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
+                  "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+                : "r"(src) : "memory");
+            asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+        } else {
+#pragma unroll
+            for (int c = 0; c < 32; ++c) r[c] = any_lost ? 0x7fc00000u : 0u;       // NaN marks a lost wait
+        }
+        const uint32_t b = b0 + warp * 16 + lane;
+        if (lane < 16 && b < batch) {
+#pragma unroll
+            for (int c = 0; c < 32; ++c) {
+                const uint32_t j = cblk * kTcCols + c;
+                if (j < f.m) {
+                    if (row_splits == 1) y[(int64_t)j * ys_j + (int64_t)b * ys_b] = __uint_as_float(r[c]);
+                    else partial[((size_t)j * row_splits + rs) * batch + b] = __uint_as_float(r[c]);
+                }
+            }
+        }
+    }
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    __syncthreads();
+    if (warp == 0) asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(32u) : "memory");
+}
+
+// ------------------------------------------------------------------------------------------------
 // sHAC, batch of inputs.  One warp per segment: lanes decode kBatchSteps entries each into a small
 // shared tile of (value, row) pairs, then the warp walks the tile with lanes spread over the
 // inputs, gathering the rows of X (stored [n][batch] for coalesced access).
@@ -1345,6 +1556,30 @@ static int launch_gemm(const Format& f, const DeviceInfo& di, const DevFormat& d
     return HAC_OK;
 }
 
+// The tcgen05 variant of launch_gemm (same block decomposition and partial layout).
+static int launch_gemm_tc(const Format& f, const DeviceInfo& di, const DevFormat& d, const float* x, int64_t xs_i,
+                          int64_t xs_b, int64_t batch, float* y, int64_t ys_j, int64_t ys_b, float* partial,
+                          cudaStream_t st, uint32_t* row_splits_out) {
+    const size_t budget = (size_t)di.max_smem_optin;
+    const size_t fixed = 16 + 128 + tc_tile_bytes() + (size_t)kTcWarps * d.max_unit_chunks * 16;
+    if (fixed + plan_smem_bytes(d.l1_bits, 0, d.sub_bytes) > budget) return HAC_ERR_BUFFER_TOO_SMALL;
+    const TablePlan tp = plan_tables(d, budget - fixed);
+    const size_t smem = fixed + plan_smem_bytes(d.l1_bits, tp.repl_log2, d.sub_bytes);
+    int rc = prepare_kernel(hac_gemm_tc_kernel, smem);
+    if (rc) return rc;
+    const uint32_t col_blocks = (uint32_t)((f.m + kTcCols - 1) / kTcCols);
+    const uint32_t batch_tiles = (uint32_t)((batch + kTcBatch - 1) / kTcBatch);
+    const uint32_t rs = gemm_row_splits(f, batch, di.sms);
+    const uint64_t grid = (uint64_t)col_blocks * rs * batch_tiles;
+    if (grid > 0x7fffffffull) return HAC_ERR_OFFSET_OVERFLOW;
+    hac_gemm_tc_kernel<<<(unsigned)grid, kTcWarps * 32, smem, st>>>(d, tp, x, xs_i, xs_b, (uint32_t)batch, y, ys_j,
+                                                                   ys_b, partial, col_blocks, rs);
+    HAC_CUDA(cudaGetLastError());
+    f.last_launches++;
+    *row_splits_out = rs;
+    return HAC_OK;
+}
+
 template <int kAcc>
 static int launch_batch_t(const Format& f, const DeviceInfo& di, const DevFormat& d, const float* x, int64_t xs_i,
                           int64_t xs_b, int64_t batch, float* y, int64_t ys_j, int64_t ys_b, float* partial,
@@ -1395,7 +1630,10 @@ static int dot(const Format& f, const float* x, int64_t batch, int64_t xs_i, int
             rc = device_info(di);
             if (rc) return rc;
             if (!f.sparse) {
-                rc = launch_gemm(f, di, d, x, xs_i, xs_b, batch, y, ys_j, ys_b, partial, st, &gemm_splits);
+                if (env_int("HAC_B200_GEMM_TC", 0) != 0)
+                    rc = launch_gemm_tc(f, di, d, x, xs_i, xs_b, batch, y, ys_j, ys_b, partial, st, &gemm_splits);
+                else
+                    rc = launch_gemm(f, di, d, x, xs_i, xs_b, batch, y, ys_j, ys_b, partial, st, &gemm_splits);
             } else {
                 const int acc = (int)std::min<int64_t>(kAccMax, (batch + 31) / 32);
                 switch (acc) {
