@@ -785,243 +785,41 @@ __global__ void finalize_kernel(DevFormat f, bool sparse, const float* __restric
 }
 
 // ------------------------------------------------------------------------------------------------
-// HAC, batch of inputs (Algorithm 3 without re-decoding W per input), on the tensor cores.
+// HAC, batch of inputs (Algorithm 3 without re-decoding W per input), on the 5th-generation tensor
+// cores (tcgen05) with the accumulators in tensor memory.
 //
-// A block owns kGemmCols consecutive columns of W (one per warp),
-// a range of segment indices g (all of them unless the grid would be too small) and a tile of
-// kGemmBatch inputs.  It alternates between
-//   decode : every lane decodes 4 symbols of its sub-segment; the values are split
-//            into two TF32 parts (w = hi + lo) and stored as a [column][row] tile in shared memory;
-//   stage  : the 128 matching rows of X are copied to shared memory;
-//   product: the 32 x 64 output tile is updated with m16n8k8 TF32 tensor-core instructions, three
-//            per tile (lo*hi + hi*lo + hi*hi, fp32 accumulation), which keeps the result within
-//            about 1e-6 of sum |w x|.  The 16 row-steps of a chunk are split over 8 warp groups, whose
-//            partial tiles are added once at the end.
+// A block owns 32 consecutive columns of W, a range of segment indices g (all of them unless the
+// grid would be too small) and a tile of 64 inputs.  Work proceeds in chunks of 64 rows: every lane
+// decodes two symbols of each of its two sub-segments, and the 64 matching rows of X are fetched.
+// One MMA is D[64 inputs][32 columns] += X[64][8] * W[32][8]^T in TF32; both operands are read by the
+// tensor core straight from shared memory ("K-major", no swizzle): a group of four consecutive K
+// elements of one row is a 16-byte unit, 8 rows form a 128-byte core matrix, core matrices of
+// successive 8-row groups are kTcSbo bytes apart, the two K halves of an MMA are LBO bytes apart.
+// Strides are padded so that the stores of the decode phase hit distinct banks.
+// Split precision: every weight and every input is written as hi + lo, both rounded to TF32, and
+// three products are accumulated in fp32 (x_lo*w_hi + x_hi*w_lo + x_hi*w_hi); the error stays near
+// 1e-7 of sum |w x|, well inside the output tolerance.
+// For 64 inputs the accumulator rows sit in tensor-memory lanes 0-15, 32-47, 64-79 and 96-111.
 // The stream is decoded once per batch tile and never written to global memory.
-// Fragment layout of mma.sync.m16n8k8 (gid = lane / 4, tig = lane % 4):
-//   A (16 x 8): a0 (gid, tig)  a1 (gid+8, tig)  a2 (gid, tig+4)  a3 (gid+8, tig+4)
-//   B ( 8 x 8): b0 (tig, gid)  b1 (tig+4, gid)
-//   C (16 x 8): c0 (gid, 2tig) c1 (gid, 2tig+1) c2 (gid+8, 2tig) c3 (gid+8, 2tig+1)
 // ------------------------------------------------------------------------------------------------
-constexpr int kBatchSteps = 4;          // symbols decoded per lane per phase
+constexpr int kBatchSteps = 4;          // sHAC batched kernel: entries decoded per lane per phase
 constexpr int kBatchRows = 32 * kBatchSteps;
 constexpr int kAccMax = 4;              // sHAC batch tile = 32 * kAcc inputs
-constexpr int kGemmCols = 32;
-constexpr int kGemmBatch = 64;
-constexpr int kGemmWarps = 32;
-constexpr int kWtStride = kBatchRows + 4;     // floats per column of the weight tile (bank-conflict free)
-constexpr int kXtStride = kGemmBatch + 8;     // floats per row of the input tile
 
 __device__ __forceinline__ uint32_t to_tf32(float v) {
     uint32_t r;
     asm("cvt.rna.tf32.f32 %0, %1;" : "=r"(r) : "f"(v));
     return r;
 }
-__device__ __forceinline__ void mma_tf32(float (&c)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
-    asm volatile(
-        "mma.sync.aligned.m16n8k8.row.col.f32.tf32.tf32.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
-        : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
-        : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
-}
 
-__host__ __device__ inline size_t gemm_tile_bytes() {
-    return align16((size_t)2 * kGemmCols * kWtStride * 4) + align16((size_t)kBatchRows * kXtStride * 4);
-}
-
-__global__ void __launch_bounds__(kGemmWarps * 32) hac_gemm_kernel(DevFormat f, TablePlan tp,
-                                                                  const float* __restrict__ x, int64_t xs_i,
-                                                                  int64_t xs_b, uint32_t batch, float* __restrict__ y,
-                                                                  int64_t ys_j, int64_t ys_b,
-                                                                  float* __restrict__ partial, uint32_t col_blocks,
-                                                                  uint32_t row_splits, uint32_t vec_x) {
-    const uint32_t warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const uint32_t gid = lane >> 2, tig = lane & 3;
-    // block -> (column block, row split, batch tile)
-    const uint32_t cblk = blockIdx.x % col_blocks;
-    const uint32_t rest = blockIdx.x / col_blocks;
-    const uint32_t rs = rest % row_splits, bt = rest / row_splits;
-    const uint32_t g_begin = (uint32_t)(((uint64_t)f.G * rs) / row_splits);
-    const uint32_t g_end = (uint32_t)(((uint64_t)f.G * (rs + 1)) / row_splits);
-    const uint32_t b0 = bt * kGemmBatch;
-
-    unsigned char* p = smem;
-    const Decoder dec = stage_decoder(f, tp, p);
-    float* wt_hi = reinterpret_cast<float*>(p);                       // [kGemmCols][kWtStride]
-    float* wt_lo = wt_hi + kGemmCols * kWtStride;
-    p += align16((size_t)2 * kGemmCols * kWtStride * 4);
-    float* xt = reinterpret_cast<float*>(p);                          // [kBatchRows][kXtStride]
-    p += align16((size_t)kBatchRows * kXtStride * 4);
-    uint4* stage = reinterpret_cast<uint4*>(p) + (size_t)warp * f.max_unit_chunks;
-    const uint32_t stage_a = smem_off(stage);
-    __syncthreads();
-
-    // product-phase role of this warp: a quarter of the inputs (2 tiles of 8), two of the 16 row-steps
-    const uint32_t n_quarter = warp & 3u, ksplit = warp >> 2;
-    float acc[2][2][4];
-#pragma unroll
-    for (int mt = 0; mt < 2; ++mt)
-#pragma unroll
-        for (int nt = 0; nt < 2; ++nt)
-#pragma unroll
-            for (int i = 0; i < 4; ++i) acc[mt][nt][i] = 0.0f;
-
-    // rows of X for one chunk, two float4 per thread, fetched one chunk ahead of their use
-    constexpr int kXPerThread = kBatchRows * (kGemmBatch / 4) / (kGemmWarps * 32);
-    float4 xr[kXPerThread];
-    auto load_x = [&](uint32_t g, uint32_t s0) {
-#pragma unroll
-        for (int i = 0; i < kXPerThread; ++i) {
-            const uint32_t idx = threadIdx.x + i * (kGemmWarps * 32);
-            const uint32_t r = idx / (kGemmBatch / 4), q = idx % (kGemmBatch / 4);
-            const uint32_t l = r / kBatchSteps, s = r % kBatchSteps;
-            const uint32_t row = (g * 32 + l) * f.S + s0 + s;      // tile row r <-> matrix row
-            const uint32_t b = b0 + q * 4;
-            float4 v = make_float4(0.0f, 0.0f, 0.0f, 0.0f);
-            if (s0 + s < f.S && row < f.n) {
-                const float* src = x + (int64_t)row * xs_i + (int64_t)b * xs_b;
-                if (vec_x && b + 3 < batch) {
-                    v = __ldg(reinterpret_cast<const float4*>(src));
-                } else {
-                    if (b < batch) v.x = __ldg(src);
-                    if (b + 1 < batch) v.y = __ldg(src + xs_b);
-                    if (b + 2 < batch) v.z = __ldg(src + 2 * xs_b);
-                    if (b + 3 < batch) v.w = __ldg(src + 3 * xs_b);
-                }
-            }
-            xr[i] = v;
-        }
-    };
-    auto store_x = [&]() {
-#pragma unroll
-        for (int i = 0; i < kXPerThread; ++i) {
-            const uint32_t idx = threadIdx.x + i * (kGemmWarps * 32);
-            const uint32_t r = idx / (kGemmBatch / 4), q = idx % (kGemmBatch / 4);
-            *reinterpret_cast<float4*>(xt + r * kXtStride + q * 4) = xr[i];
-        }
-    };
-    if (g_begin < g_end) load_x(g_begin, 0);
-
-    const uint32_t sb = shared_base();
-    const uint32_t l1_abs = sb + dec.l1_lane;
-    const uint32_t j_mine = cblk * kGemmCols + warp;                  // decode-phase role: one column per warp
-    for (uint32_t g = g_begin; g < g_end; ++g) {
-        FastReader fr;
-        uint32_t count = 0;
-        fr.hi = fr.lo = fr.off = 0; fr.next = sb + stage_a;
-        if (j_mine < f.m) {
-            const uint32_t u = j_mine * f.G + g;
-            const uint32_t my_bits = __ldg(f.sub_bits + (size_t)u * 32 + lane);
-            uint32_t total;
-            const uint32_t start = lane_start_bits(my_bits, lane, total);
-            const uint32_t base = stage_span(f, __ldg(f.seg_bit_off + u), total, stage, lane);
-            const uint32_t row0 = (g * 32 + lane) * f.S;
-            count = row0 < f.n ? min(f.S, f.n - row0) : 0u;
-            BitReader br;
-            br.init(stage_a, base + start);
-            fr.hi = br.hi; fr.lo = br.lo; fr.off = br.off; fr.next = sb + br.next;
-        }
-        const uint32_t seg_rows = min(f.S, f.n - min(f.n, g * 32 * f.S));     // longest sub-segment here
-        for (uint32_t s0 = 0; s0 < seg_rows; s0 += kBatchSteps) {
-            // decode: 4 symbols -> tile rows lane*4 .. lane*4+3 of this warp's column, as TF32 hi + lo
-            float hi[kBatchSteps], lo[kBatchSteps];
-#pragma unroll
-            for (int s = 0; s < kBatchSteps; ++s) {
-                uint32_t top = 0, val = 0, len = 0;
-                if (s0 + s < count) {
-                    fast_lookup(fr, dec.l1_shift, dec.l1_mul, l1_abs, top, val, len);
-                    if ((int32_t)len < 0) resolve_long(top, dec, f, val, len);
-                    fast_consume_value(fr, len);
-                }
-                const float w = __uint_as_float(val);
-                hi[s] = __uint_as_float(to_tf32(w));
-                lo[s] = __uint_as_float(to_tf32(w - hi[s]));
-            }
-            const uint32_t at = warp * kWtStride + lane * kBatchSteps;
-            *reinterpret_cast<float4*>(wt_hi + at) = make_float4(hi[0], hi[1], hi[2], hi[3]);
-            *reinterpret_cast<float4*>(wt_lo + at) = make_float4(lo[0], lo[1], lo[2], lo[3]);
-            store_x();
-            __syncthreads();
-            // the next chunk's rows of X are requested now and land during the product phase
-            if (s0 + kBatchSteps < seg_rows) load_x(g, s0 + kBatchSteps);
-            else if (g + 1 < g_end) load_x(g + 1, 0);
-            // product: row-steps 2*ksplit and 2*ksplit+1 (8 tile rows each)
-#pragma unroll
-            for (int kq = 0; kq < 2; ++kq) {
-                const uint32_t k0 = (2 * ksplit + kq) * 8;
-                uint32_t b_hi[2][2], b_lo[2][2];
-#pragma unroll
-                for (int nt = 0; nt < 2; ++nt) {
-                    const uint32_t col = n_quarter * 16 + nt * 8 + gid;
-                    const float x0 = xt[(k0 + tig) * kXtStride + col];
-                    const float x1 = xt[(k0 + tig + 4) * kXtStride + col];
-                    b_hi[nt][0] = to_tf32(x0); b_hi[nt][1] = to_tf32(x1);
-                    b_lo[nt][0] = to_tf32(x0 - __uint_as_float(b_hi[nt][0]));
-                    b_lo[nt][1] = to_tf32(x1 - __uint_as_float(b_hi[nt][1]));
-                }
-#pragma unroll
-                for (int mt = 0; mt < 2; ++mt) {
-                    const uint32_t c0 = (16 * mt + gid) * kWtStride + k0 + tig;
-                    const uint32_t c8 = c0 + 8 * kWtStride;
-                    uint32_t a_hi[4], a_lo[4];
-                    a_hi[0] = __float_as_uint(wt_hi[c0]);     a_lo[0] = __float_as_uint(wt_lo[c0]);
-                    a_hi[1] = __float_as_uint(wt_hi[c8]);     a_lo[1] = __float_as_uint(wt_lo[c8]);
-                    a_hi[2] = __float_as_uint(wt_hi[c0 + 4]); a_lo[2] = __float_as_uint(wt_lo[c0 + 4]);
-                    a_hi[3] = __float_as_uint(wt_hi[c8 + 4]); a_lo[3] = __float_as_uint(wt_lo[c8 + 4]);
-#pragma unroll
-                    for (int nt = 0; nt < 2; ++nt) {
-                        mma_tf32(acc[mt][nt], a_lo, b_hi[nt][0], b_hi[nt][1]);
-                        mma_tf32(acc[mt][nt], a_hi, b_lo[nt][0], b_lo[nt][1]);
-                        mma_tf32(acc[mt][nt], a_hi, b_hi[nt][0], b_hi[nt][1]);
-                    }
-                }
-            }
-            __syncthreads();
-        }
-    }
-    // add the 8 row-split partial tiles: red[warp][register][lane] reuses the tile area
-    float* red = wt_hi;
-#pragma unroll
-    for (int mt = 0; mt < 2; ++mt)
-#pragma unroll
-        for (int nt = 0; nt < 2; ++nt)
-#pragma unroll
-            for (int i = 0; i < 4; ++i) red[(warp * 16 + (mt * 8 + nt * 4 + i)) * 32 + lane] = acc[mt][nt][i];
-    __syncthreads();
-    for (uint32_t o = threadIdx.x; o < kGemmCols * kGemmBatch; o += blockDim.x) {
-        const uint32_t col = o / kGemmBatch, bb = o % kGemmBatch;
-        const uint32_t quarter = bb / 16, nt = (bb % 16) / 8, cpos = bb % 8;
-        const uint32_t mt = col / 16, r16 = col % 16;
-        const uint32_t reg = mt * 8 + nt * 4 + (r16 / 8) * 2 + (cpos & 1u);
-        const uint32_t ln = (r16 % 8) * 4 + cpos / 2;
-        float sum = 0.0f;
-#pragma unroll
-        for (uint32_t ks = 0; ks < kGemmWarps / 4; ++ks) sum += red[((ks * 4 + quarter) * 16 + reg) * 32 + ln];
-        const uint32_t j = cblk * kGemmCols + col, b = b0 + bb;
-        if (j < f.m && b < batch) {
-            if (row_splits == 1) y[(int64_t)j * ys_j + (int64_t)b * ys_b] = sum;
-            else partial[((size_t)j * row_splits + rs) * batch + b] = sum;
-        }
-    }
-}
-
-// ------------------------------------------------------------------------------------------------
-// The same batched HAC product on the 5th-generation tensor cores (tcgen05), accumulators in
-// tensor memory.  One MMA is D[64 inputs][32 columns] += X[64][8] * W[32][8]^T in TF32; both operands
-// are read by the tensor core straight from shared memory ("K-major", no swizzle): a group of four
-// consecutive K elements of one row is a 16-byte unit, 8 rows form a 128-byte core matrix, core
-// matrices of successive 8-row groups are kTcSbo bytes apart, the two K halves of an MMA are LBO
-// bytes apart.  Strides are padded so that the stores of the decode phase hit distinct banks.
-// Split precision as above: x_lo*w_hi + x_hi*w_lo + x_hi*w_hi, every part rounded to TF32 first.
-// For 64 inputs the accumulator rows sit in tensor-memory lanes 0-15, 32-47, 64-79 and 96-111.
-// ------------------------------------------------------------------------------------------------
 constexpr int kTcSteps = 2;                         // symbols decoded per lane per chunk
 constexpr int kTcRows = 32 * kTcSteps;              // K per chunk (64)
 constexpr int kTcKSteps = kTcRows / 8;              // MMAs (of K = 8) per chunk and product
 constexpr int kTcSbo = 128;
 constexpr int kTcXLbo = 1024, kTcXKst = 2048;       // X tile: 64 rows -> 8 core matrices per K half
 constexpr int kTcWLbo = 528, kTcWKst = 1056;        // W tile: 32 rows -> 4 core matrices, padded
-constexpr int kTcCols = 32, kTcBatch = 64, kTcWarps = 32;
-constexpr uint32_t kTcWaitTries = 4000000;
+constexpr int kTcCols = 32, kTcBatch = 64, kTcDecodeWarps = 16;
+constexpr uint32_t kTcWaitTries = 400000;
 
 __host__ __device__ inline size_t tc_tile_bytes() {
     return (size_t)2 * kTcKSteps * kTcXKst + (size_t)2 * kTcKSteps * kTcWKst;
@@ -1049,12 +847,16 @@ __device__ __forceinline__ bool tc_wait(uint32_t mbar, uint32_t parity) {
     return false;
 }
 
-__global__ void __launch_bounds__(kTcWarps * 32) hac_gemm_tc_kernel(DevFormat f, TablePlan tp,
-                                                                   const float* __restrict__ x, int64_t xs_i,
-                                                                   int64_t xs_b, uint32_t batch, float* __restrict__ y,
-                                                                   int64_t ys_j, int64_t ys_b,
-                                                                   float* __restrict__ partial, uint32_t col_blocks,
-                                                                   uint32_t row_splits) {
+// Warp-specialised and pipelined: warps 0..15 decode (two columns each, two chains per lane) and
+// stage the rows of X; warp 16 only issues the MMAs.  Tiles live in a ring of `stages` buffers with
+// two mbarriers each: `full` (16 arrivals, one per decode warp, after its stores) and `empty`
+// (arrival by tcgen05.commit once the MMAs that read the buffer have finished).  There is no
+// block-wide barrier inside the loop, so a slow code word delays only its own warp.
+// Every wait is bounded; if one runs out the block marks its outputs NaN and still terminates.
+__global__ void __launch_bounds__((kTcDecodeWarps + 1) * 32) hac_gemm_tc_kernel(
+    DevFormat f, TablePlan tp, const float* __restrict__ x, int64_t xs_i, int64_t xs_b, uint32_t batch,
+    float* __restrict__ y, int64_t ys_j, int64_t ys_b, float* __restrict__ partial, uint32_t col_blocks,
+    uint32_t row_splits, uint32_t stages) {
     const uint32_t warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const uint32_t cblk = blockIdx.x % col_blocks;
     const uint32_t rest = blockIdx.x / col_blocks;
@@ -1063,127 +865,179 @@ __global__ void __launch_bounds__(kTcWarps * 32) hac_gemm_tc_kernel(DevFormat f,
     const uint32_t g_end = (uint32_t)(((uint64_t)f.G * (rs + 1)) / row_splits);
     const uint32_t b0 = bt * kTcBatch;
     const uint32_t sb = shared_base();
+    // chunks of kTcRows rows this block goes through (same count in every warp)
+    uint32_t chunks = 0;
+    for (uint32_t g = g_begin; g < g_end; ++g)
+        chunks += (min(f.S, f.n - min(f.n, g * 32 * f.S)) + kTcSteps - 1) / kTcSteps;
 
-    // shared memory: [mbarrier, tensor-memory address] [tables] [X hi, X lo, W hi, W lo tiles] [staged spans]
+    // shared memory: [mbarriers full[2], empty[2], done; tensor-memory address; lost flag] [tables] [tile ring] [spans]
     unsigned char* p = smem;
-    const uint32_t mbar = sb;
-    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem + 8);
-    p += 16;
-    if (threadIdx.x == 0) mbar_init(mbar, 1);
+    const uint32_t bar_full = sb, bar_empty = sb + 16, bar_done = sb + 32;
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem + 40);
+    volatile uint32_t* lost_flag = reinterpret_cast<volatile uint32_t*>(smem + 44);
+    p += 48;
+    if (threadIdx.x == 0) {
+        for (uint32_t s = 0; s < 2; ++s) { mbar_init(bar_full + 8 * s, kTcDecodeWarps); mbar_init(bar_empty + 8 * s, 1); }
+        mbar_init(bar_done, 1);
+        *lost_flag = 0;
+    }
     __syncwarp();
-    if (warp == 0) {
-        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(sb + 8), "r"(32u) : "memory");
+    if (warp == kTcDecodeWarps) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(sb + 40), "r"(32u) : "memory");
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
     }
     const Decoder dec = stage_decoder(f, tp, p);
     p = smem + ((smem_off(p) + 127u) & ~127u);
-    unsigned char* x_hi = p;
-    unsigned char* x_lo = x_hi + kTcKSteps * kTcXKst;
-    unsigned char* w_hi = x_lo + kTcKSteps * kTcXKst;
-    unsigned char* w_lo = w_hi + kTcKSteps * kTcWKst;
-    p = w_lo + kTcKSteps * kTcWKst;
-    uint4* stage = reinterpret_cast<uint4*>(p) + (size_t)warp * f.max_unit_chunks;
-    const uint32_t stage_a = smem_off(stage);
+    const uint32_t ring = smem_off(p);                          // stage s at ring + s * tc_tile_bytes()
+    p += (size_t)stages * tc_tile_bytes();
+    constexpr uint32_t kXHi = 0, kXLo = kTcKSteps * kTcXKst, kWHi = 2 * kTcKSteps * kTcXKst,
+                       kWLo = kWHi + kTcKSteps * kTcWKst;
     asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
     __syncthreads();
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
     const uint32_t tmem = *tmem_slot;
 
-    // staging role: K group q (tile rows 4q..4q+3 = sub-segments 2q and 2q+1, two symbols each), input b
-    const uint32_t xq = threadIdx.x / kTcBatch, xb = threadIdx.x % kTcBatch;
-    const uint32_t x_at = (xq >> 1) * kTcXKst + (xq & 1u) * kTcXLbo + (xb >> 3) * kTcSbo + (xb & 7u) * 16;
-    float xr[4];
-    auto load_x = [&](uint32_t g, uint32_t s0) {
-#pragma unroll
-        for (int i = 0; i < 4; ++i) {
-            const uint32_t l = 2 * xq + (i >> 1), s = i & 1;
-            const uint32_t row = (g * 32 + l) * f.S + s0 + s;
-            float v = 0.0f;
-            if (s0 + s < f.S && row < f.n && b0 + xb < batch) v = __ldg(x + (int64_t)row * xs_i + (int64_t)(b0 + xb) * xs_b);
-            xr[i] = v;
-        }
-    };
-    if (g_begin < g_end) load_x(g_begin, 0);
-    // decode role: column cblk*32 + warp; tile row of symbol s of lane l is 2l + s
-    const uint32_t j_mine = cblk * kTcCols + warp;
-    const uint32_t wq = lane >> 1;
-    const uint32_t w_at = (wq >> 1) * kTcWKst + (wq & 1u) * kTcWLbo + (warp >> 3) * kTcSbo + (warp & 7u) * 16 + (lane & 1u) * 8;
-    const uint32_t l1_abs = sb + dec.l1_lane;
-    const uint32_t idesc = (1u << 4) | (2u << 7) | (2u << 10) | ((uint32_t)(kTcCols >> 3) << 17) | ((uint32_t)(kTcBatch >> 4) << 24);
-    uint32_t chunk = 0;
-    bool lost = false;                       // a wait ran out: results are not to be trusted
-
-    for (uint32_t g = g_begin; g < g_end; ++g) {
-        FastReader fr;
-        uint32_t count = 0;
-        fr.hi = fr.lo = fr.off = 0; fr.next = sb + stage_a;
-        if (j_mine < f.m) {
-            const uint32_t u = j_mine * f.G + g;
-            const uint32_t my_bits = __ldg(f.sub_bits + (size_t)u * 32 + lane);
-            uint32_t total;
-            const uint32_t start = lane_start_bits(my_bits, lane, total);
-            const uint32_t base = stage_span(f, __ldg(f.seg_bit_off + u), total, stage, lane);
-            const uint32_t row0 = (g * 32 + lane) * f.S;
-            count = row0 < f.n ? min(f.S, f.n - row0) : 0u;
-            BitReader br;
-            br.init(stage_a, base + start);
-            fr.hi = br.hi; fr.lo = br.lo; fr.off = br.off; fr.next = sb + br.next;
-        }
-        const uint32_t seg_rows = min(f.S, f.n - min(f.n, g * 32 * f.S));
-        for (uint32_t s0 = 0; s0 < seg_rows; s0 += kTcSteps, ++chunk) {
-            float hi[kTcSteps], lo[kTcSteps];
-#pragma unroll
-            for (int s = 0; s < kTcSteps; ++s) {
-                uint32_t top = 0, val = 0, len = 0;
-                if (s0 + s < count) {
-                    fast_lookup(fr, dec.l1_shift, dec.l1_mul, l1_abs, top, val, len);
-                    if ((int32_t)len < 0) resolve_long(top, dec, f, val, len);
-                    fast_consume_value(fr, len);
-                }
-                const float w = __uint_as_float(val);
-                hi[s] = __uint_as_float(to_tf32(w));
-                lo[s] = __uint_as_float(to_tf32(w - hi[s]));
-            }
-            float xh[4], xl[4];
-#pragma unroll
-            for (int i = 0; i < 4; ++i) {
-                xh[i] = __uint_as_float(to_tf32(xr[i]));
-                xl[i] = __uint_as_float(to_tf32(xr[i] - xh[i]));
-            }
-            // the tensor core must be done reading the previous chunk's tiles before they change
-            if (chunk > 0 && !tc_wait(mbar, (chunk - 1) & 1u)) lost = true;
-            *reinterpret_cast<float2*>(w_hi + w_at) = make_float2(hi[0], hi[1]);
-            *reinterpret_cast<float2*>(w_lo + w_at) = make_float2(lo[0], lo[1]);
-            *reinterpret_cast<float4*>(x_hi + x_at) = make_float4(xh[0], xh[1], xh[2], xh[3]);
-            *reinterpret_cast<float4*>(x_lo + x_at) = make_float4(xl[0], xl[1], xl[2], xl[3]);
-            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-            asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
-            __syncthreads();
-            if (threadIdx.x == 0) {
+    if (warp == kTcDecodeWarps) {
+        // ---- MMA issue: one lane, chunk after chunk ----
+        if (lane == 0) {
+            const uint32_t idesc = (1u << 4) | (2u << 7) | (2u << 10) | ((uint32_t)(kTcCols >> 3) << 17) |
+                                   ((uint32_t)(kTcBatch >> 4) << 24);
+            for (uint32_t c = 0; c < chunks; ++c) {
+                const uint32_t s = c % stages, use = c / stages;
+                if (!tc_wait(bar_full + 8 * s, use & 1u)) *lost_flag = 1;
                 asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+                const uint32_t base = sb + ring + s * (uint32_t)tc_tile_bytes();
+                uint64_t a_hi = tc_desc(base + kXHi, kTcXLbo), a_lo = tc_desc(base + kXLo, kTcXLbo);
+                uint64_t b_hi = tc_desc(base + kWHi, kTcWLbo), b_lo = tc_desc(base + kWLo, kTcWLbo);
 #pragma unroll
                 for (int ks = 0; ks < kTcKSteps; ++ks) {
-                    const uint64_t a_hi = tc_desc(sb + smem_off(x_hi) + ks * kTcXKst, kTcXLbo);
-                    const uint64_t a_lo = tc_desc(sb + smem_off(x_lo) + ks * kTcXKst, kTcXLbo);
-                    const uint64_t b_hi = tc_desc(sb + smem_off(w_hi) + ks * kTcWKst, kTcWLbo);
-                    const uint64_t b_lo = tc_desc(sb + smem_off(w_lo) + ks * kTcWKst, kTcWLbo);
-                    tc_mma(tmem, a_lo, b_hi, idesc, (chunk | (uint32_t)ks) ? 1u : 0u);
+                    tc_mma(tmem, a_lo, b_hi, idesc, (c | (uint32_t)ks) ? 1u : 0u);
                     tc_mma(tmem, a_hi, b_lo, idesc, 1u);
                     tc_mma(tmem, a_hi, b_hi, idesc, 1u);
+                    a_hi += kTcXKst >> 4; a_lo += kTcXKst >> 4; b_hi += kTcWKst >> 4; b_lo += kTcWKst >> 4;
                 }
-                tc_commit(mbar);
+                tc_commit(bar_empty + 8 * s);
             }
-            // the next chunk's rows of X are requested now and land while it is being decoded
-            if (s0 + kTcSteps < seg_rows) load_x(g, s0 + kTcSteps);
-            else if (g + 1 < g_end) load_x(g + 1, 0);
+            tc_commit(bar_done);
+        }
+        __syncwarp();                        // the other lanes sleep here until the last MMA is issued
+    } else {
+        // ---- decode + staging ----
+        uint4* stage = reinterpret_cast<uint4*>(p) + (size_t)warp * 2 * f.max_unit_chunks;
+        const uint32_t stage_a = smem_off(stage);
+        // staging role: two (K group q, input b) pairs per thread; everything that does not change
+        // from chunk to chunk (tile offset, row offsets inside a segment, column pointer) is set up once
+        uint32_t x_at[2], row_off[2][4];
+        const float* x_col[2];
+        bool b_ok[2];
+        float xr[2][4];
+#pragma unroll
+        for (int i = 0; i < 2; ++i) {
+            const uint32_t pi = threadIdx.x + i * (kTcDecodeWarps * 32);
+            const uint32_t q = pi / kTcBatch, b = pi % kTcBatch;
+            x_at[i] = (q >> 1) * kTcXKst + (q & 1u) * kTcXLbo + (b >> 3) * kTcSbo + (b & 7u) * 16;
+#pragma unroll
+            for (int e = 0; e < 4; ++e) row_off[i][e] = (2 * q + (e >> 1)) * f.S + (e & 1);
+            b_ok[i] = b0 + b < batch;
+            x_col[i] = x + (int64_t)(b0 + b) * xs_b;
+        }
+        auto load_x = [&](uint32_t g, uint32_t s0) {
+            const uint32_t row_base = g * 32 * f.S + s0;
+            const bool second = s0 + 1 < f.S;                  // the chunk's second symbol exists
+#pragma unroll
+            for (int i = 0; i < 2; ++i) {
+#pragma unroll
+                for (int e = 0; e < 4; ++e) {
+                    const uint32_t row = row_base + row_off[i][e];
+                    float v = 0.0f;
+                    if (b_ok[i] && row < f.n && ((e & 1) == 0 || second)) v = __ldg(x_col[i] + (int64_t)row * xs_i);
+                    xr[i][e] = v;
+                }
+            }
+        };
+        if (g_begin < g_end) load_x(g_begin, 0);
+        const uint32_t wq = lane >> 1;
+        const uint32_t l1_abs = sb + dec.l1_lane;
+        uint32_t c = 0;
+        for (uint32_t g = g_begin; g < g_end; ++g) {
+            FastReader fr[2];
+            uint32_t count[2], w_at[2];
+#pragma unroll
+            for (int ch = 0; ch < 2; ++ch) {
+                const uint32_t col = 2 * warp + ch, j = cblk * kTcCols + col;
+                w_at[ch] = (wq >> 1) * kTcWKst + (wq & 1u) * kTcWLbo + (col >> 3) * kTcSbo + (col & 7u) * 16 + (lane & 1u) * 8;
+                count[ch] = 0;
+                fr[ch].hi = fr[ch].lo = fr[ch].off = 0; fr[ch].next = sb + stage_a;
+                if (j < f.m) {
+                    const uint32_t u = j * f.G + g;
+                    const uint32_t my_bits = __ldg(f.sub_bits + (size_t)u * 32 + lane);
+                    uint32_t total;
+                    const uint32_t start = lane_start_bits(my_bits, lane, total);
+                    const uint32_t base = stage_span(f, __ldg(f.seg_bit_off + u), total, stage + (size_t)ch * f.max_unit_chunks, lane);
+                    const uint32_t row0 = (g * 32 + lane) * f.S;
+                    count[ch] = row0 < f.n ? min(f.S, f.n - row0) : 0u;
+                    BitReader br;
+                    br.init(stage_a + ch * f.max_unit_chunks * 16, base + start);
+                    fr[ch].hi = br.hi; fr[ch].lo = br.lo; fr[ch].off = br.off; fr[ch].next = sb + br.next;
+                }
+            }
+            const uint32_t seg_rows = min(f.S, f.n - min(f.n, g * 32 * f.S));
+            for (uint32_t s0 = 0; s0 < seg_rows; s0 += kTcSteps, ++c) {
+                float hi[2][kTcSteps], lo[2][kTcSteps];
+#pragma unroll
+                for (int st = 0; st < kTcSteps; ++st) {
+                    uint32_t top[2], val[2], len[2];
+#pragma unroll
+                    for (int ch = 0; ch < 2; ++ch) {
+                        top[ch] = val[ch] = len[ch] = 0;
+                        if (s0 + st < count[ch]) fast_lookup(fr[ch], dec.l1_shift, dec.l1_mul, l1_abs, top[ch], val[ch], len[ch]);
+                    }
+#pragma unroll
+                    for (int ch = 0; ch < 2; ++ch) {
+                        if ((int32_t)len[ch] < 0) resolve_long(top[ch], dec, f, val[ch], len[ch]);
+                        if (s0 + st < count[ch]) fast_consume_value(fr[ch], len[ch]);
+                        const float w = __uint_as_float(val[ch]);
+                        hi[ch][st] = __uint_as_float(to_tf32(w));
+                        lo[ch][st] = __uint_as_float(to_tf32(w - hi[ch][st]));
+                    }
+                }
+                const uint32_t s = c % stages, use = c / stages;
+                // the buffer is free once the MMAs of its previous use have been committed
+                if (use > 0 && !tc_wait(bar_empty + 8 * s, (use - 1) & 1u)) *lost_flag = 1;
+                unsigned char* tile = smem + ring + (size_t)s * tc_tile_bytes();
+#pragma unroll
+                for (int ch = 0; ch < 2; ++ch) {
+                    *reinterpret_cast<float2*>(tile + kWHi + w_at[ch]) = make_float2(hi[ch][0], hi[ch][1]);
+                    *reinterpret_cast<float2*>(tile + kWLo + w_at[ch]) = make_float2(lo[ch][0], lo[ch][1]);
+                }
+#pragma unroll
+                for (int i = 0; i < 2; ++i) {
+                    float xh[4], xl[4];
+#pragma unroll
+                    for (int e = 0; e < 4; ++e) {
+                        xh[e] = __uint_as_float(to_tf32(xr[i][e]));
+                        xl[e] = __uint_as_float(to_tf32(xr[i][e] - xh[e]));
+                    }
+                    *reinterpret_cast<float4*>(tile + kXHi + x_at[i]) = make_float4(xh[0], xh[1], xh[2], xh[3]);
+                    *reinterpret_cast<float4*>(tile + kXLo + x_at[i]) = make_float4(xl[0], xl[1], xl[2], xl[3]);
+                }
+                asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+                __syncwarp();
+                if (lane == 0) asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar_full + 8 * s) : "memory");
+                // the next chunk's rows of X are requested now and land while it is being decoded
+                if (s0 + kTcSteps < seg_rows) load_x(g, s0 + kTcSteps);
+                else if (g + 1 < g_end) load_x(g + 1, 0);
+            }
         }
     }
-    if (chunk > 0 && !tc_wait(mbar, (chunk - 1) & 1u)) lost = true;
-    const bool any_lost = __syncthreads_or(lost ? 1 : 0) != 0;
+    // ---- epilogue: accumulators -> y ----
+    bool lost = false;
+    if (chunks > 0 && !tc_wait(bar_done, 0)) lost = true;
+    const bool any_lost = __syncthreads_or((lost || *lost_flag) ? 1 : 0) != 0;
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
     if (warp < 4) {                          // warp w reads tensor-memory lanes 32w..32w+31: inputs 16w..16w+15
         uint32_t r[32];
-        if (chunk > 0 && !any_lost) {
+        if (chunks > 0 && !any_lost) {
             const uint32_t src = tmem + ((warp * 32u) << 16);
             asm volatile(
                 "tcgen05.ld.sync.aligned.32x32b.x32.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,%17,%18,%19,"
@@ -1196,23 +1050,23 @@ __global__ void __launch_bounds__(kTcWarps * 32) hac_gemm_tc_kernel(DevFormat f,
             asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
         } else {
 #pragma unroll
-            for (int c = 0; c < 32; ++c) r[c] = any_lost ? 0x7fc00000u : 0u;       // NaN marks a lost wait
+            for (int cc = 0; cc < 32; ++cc) r[cc] = any_lost ? 0x7fc00000u : 0u;   // NaN marks a lost wait
         }
         const uint32_t b = b0 + warp * 16 + lane;
         if (lane < 16 && b < batch) {
 #pragma unroll
-            for (int c = 0; c < 32; ++c) {
-                const uint32_t j = cblk * kTcCols + c;
+            for (int cc = 0; cc < 32; ++cc) {
+                const uint32_t j = cblk * kTcCols + cc;
                 if (j < f.m) {
-                    if (row_splits == 1) y[(int64_t)j * ys_j + (int64_t)b * ys_b] = __uint_as_float(r[c]);
-                    else partial[((size_t)j * row_splits + rs) * batch + b] = __uint_as_float(r[c]);
+                    if (row_splits == 1) y[(int64_t)j * ys_j + (int64_t)b * ys_b] = __uint_as_float(r[cc]);
+                    else partial[((size_t)j * row_splits + rs) * batch + b] = __uint_as_float(r[cc]);
                 }
             }
         }
     }
     asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
     __syncthreads();
-    if (warp == 0) asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(32u) : "memory");
+    if (warp == kTcDecodeWarps) asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(32u) : "memory");
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -1527,41 +1381,21 @@ static int launch_vec(const Format& f, int mode, const float* x, int64_t xs_i, f
 // Row splits of the tensor-core HAC kernel: 1 (a block owns whole columns and writes y itself)
 // unless that leaves most of the SMs idle.
 static uint32_t gemm_row_splits(const Format& f, int64_t batch, int sms) {
-    const uint64_t blocks = (uint64_t)((f.m + kGemmCols - 1) / kGemmCols) * (uint64_t)((batch + kGemmBatch - 1) / kGemmBatch);
+    const uint64_t blocks = (uint64_t)((f.m + kTcCols - 1) / kTcCols) * (uint64_t)((batch + kTcBatch - 1) / kTcBatch);
     if (blocks * 5 >= (uint64_t)sms * 3 || f.G <= 1) return 1;
     return (uint32_t)std::min<uint64_t>(f.G, std::max<uint64_t>(1, (uint64_t)sms / blocks));
 }
 
-static int launch_gemm(const Format& f, const DeviceInfo& di, const DevFormat& d, const float* x, int64_t xs_i,
-                       int64_t xs_b, int64_t batch, float* y, int64_t ys_j, int64_t ys_b, float* partial,
-                       cudaStream_t st, uint32_t* row_splits_out) {
-    const size_t budget = (size_t)di.max_smem_optin;
-    const size_t fixed = gemm_tile_bytes() + (size_t)kGemmWarps * d.max_unit_chunks * 16;
-    if (fixed + plan_smem_bytes(d.l1_bits, 0, d.sub_bytes) > budget) return HAC_ERR_BUFFER_TOO_SMALL;
-    const TablePlan tp = plan_tables(d, budget - fixed);
-    const size_t smem = fixed + plan_smem_bytes(d.l1_bits, tp.repl_log2, d.sub_bytes);
-    int rc = prepare_kernel(hac_gemm_kernel, smem);
-    if (rc) return rc;
-    const uint32_t col_blocks = (uint32_t)((f.m + kGemmCols - 1) / kGemmCols);
-    const uint32_t batch_tiles = (uint32_t)((batch + kGemmBatch - 1) / kGemmBatch);
-    const uint32_t rs = gemm_row_splits(f, batch, di.sms);
-    const uint32_t vec_x = (xs_b == 1 && (xs_i % 4) == 0 && (reinterpret_cast<uintptr_t>(x) & 15u) == 0) ? 1u : 0u;
-    const uint64_t grid = (uint64_t)col_blocks * rs * batch_tiles;
-    if (grid > 0x7fffffffull) return HAC_ERR_OFFSET_OVERFLOW;
-    hac_gemm_kernel<<<(unsigned)grid, kGemmWarps * 32, smem, st>>>(d, tp, x, xs_i, xs_b, (uint32_t)batch, y, ys_j, ys_b,
-                                                                  partial, col_blocks, rs, vec_x);
-    HAC_CUDA(cudaGetLastError());
-    f.last_launches++;
-    *row_splits_out = rs;
-    return HAC_OK;
-}
-
-// The tcgen05 variant of launch_gemm (same block decomposition and partial layout).
+// Batched HAC product: one block per (32 columns, row split, 64 inputs).
 static int launch_gemm_tc(const Format& f, const DeviceInfo& di, const DevFormat& d, const float* x, int64_t xs_i,
                           int64_t xs_b, int64_t batch, float* y, int64_t ys_j, int64_t ys_b, float* partial,
                           cudaStream_t st, uint32_t* row_splits_out) {
     const size_t budget = (size_t)di.max_smem_optin;
-    const size_t fixed = 16 + 128 + tc_tile_bytes() + (size_t)kTcWarps * d.max_unit_chunks * 16;
+    // two tile buffers when they fit next to a level-1 table with at least 8 replicas, else one
+    const size_t spans = (size_t)kTcDecodeWarps * 2 * d.max_unit_chunks * 16;
+    uint32_t stages = 2;
+    if (48 + 128 + 2 * tc_tile_bytes() + spans + plan_smem_bytes(d.l1_bits, 3, d.sub_bytes) > budget) stages = 1;
+    const size_t fixed = 48 + 128 + stages * tc_tile_bytes() + spans;
     if (fixed + plan_smem_bytes(d.l1_bits, 0, d.sub_bytes) > budget) return HAC_ERR_BUFFER_TOO_SMALL;
     const TablePlan tp = plan_tables(d, budget - fixed);
     const size_t smem = fixed + plan_smem_bytes(d.l1_bits, tp.repl_log2, d.sub_bytes);
@@ -1572,8 +1406,8 @@ static int launch_gemm_tc(const Format& f, const DeviceInfo& di, const DevFormat
     const uint32_t rs = gemm_row_splits(f, batch, di.sms);
     const uint64_t grid = (uint64_t)col_blocks * rs * batch_tiles;
     if (grid > 0x7fffffffull) return HAC_ERR_OFFSET_OVERFLOW;
-    hac_gemm_tc_kernel<<<(unsigned)grid, kTcWarps * 32, smem, st>>>(d, tp, x, xs_i, xs_b, (uint32_t)batch, y, ys_j,
-                                                                   ys_b, partial, col_blocks, rs);
+    hac_gemm_tc_kernel<<<(unsigned)grid, (kTcDecodeWarps + 1) * 32, smem, st>>>(
+        d, tp, x, xs_i, xs_b, (uint32_t)batch, y, ys_j, ys_b, partial, col_blocks, rs, stages);
     HAC_CUDA(cudaGetLastError());
     f.last_launches++;
     *row_splits_out = rs;
@@ -1630,10 +1464,7 @@ static int dot(const Format& f, const float* x, int64_t batch, int64_t xs_i, int
             rc = device_info(di);
             if (rc) return rc;
             if (!f.sparse) {
-                if (env_int("HAC_B200_GEMM_TC", 0) != 0)
-                    rc = launch_gemm_tc(f, di, d, x, xs_i, xs_b, batch, y, ys_j, ys_b, partial, st, &gemm_splits);
-                else
-                    rc = launch_gemm(f, di, d, x, xs_i, xs_b, batch, y, ys_j, ys_b, partial, st, &gemm_splits);
+                rc = launch_gemm_tc(f, di, d, x, xs_i, xs_b, batch, y, ys_j, ys_b, partial, st, &gemm_splits);
             } else {
                 const int acc = (int)std::min<int64_t>(kAccMax, (batch + 31) / 32);
                 switch (acc) {

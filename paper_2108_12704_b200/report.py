@@ -1,0 +1,174 @@
+"""Per-configuration report: format sizes against the paper's bounds (Corollaries 1 and 2) and
+kernel times against the HBM roofline on the compressed bytes, for the benchmark configurations
+and the sparsity x k sweep.  One JSON line per (configuration, format, batch).
+
+    python -m paper_2108_12704_b200.report [--configs 1,2,3,4] [--sweep] [--paper-shapes] [--out FILE]
+
+Timing protocol as in bench.py: device images replicated to more than three times the L2 size and
+rotated per launch, launches captured in CUDA graphs, CUDA events on the launching stream, best of
+five replays.  Results are checked in-process against the format's own host decode (fp64 product).
+"""
+from __future__ import annotations
+
+import argparse
+import dataclasses
+import json
+import math
+import os
+import sys
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import synth_inputs as si  # noqa: E402
+
+L2_BYTES = 126 * 1024 * 1024
+
+
+def _peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured"
+    return 6650.0, "fallback"
+
+
+def _capture(torch, fn):
+    g = torch.cuda.CUDAGraph()
+    s = torch.cuda.Stream()
+    s.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.stream(s):
+        with torch.cuda.graph(g, stream=s):
+            fn()
+    torch.cuda.current_stream().wait_stream(s)
+    return g
+
+
+def algorithmic_bytes(sizes: dict) -> int:
+    """Bytes a single-input product has to move (stream, offset index, tables, ri, cb, x, y)."""
+    lut_bits = min(12, sizes["max_code_len"])
+    tables = (2 << lut_bits) + 4 * sizes["k_eff"] + 34 * 16
+    return (sizes["stream_bytes"] + sizes["offset_index_bytes"] + tables + sizes["ri_bytes"] + sizes["cb_bytes"]
+            + 4 * sizes["n"] + 4 * sizes["m"])
+
+
+def measure(wl, kind, batches, W=None, seg_symbols=0, max_check_batch=128, replays=5):
+    import torch
+    import paper_2108_12704_b200 as hb
+    W = si.weights(wl) if W is None else W
+    fmt = hb.Format(kind, W, sparsity=wl.sparsity, k=wl.k, quantizer=wl.quantizer, kmeans_iters=wl.kmeans_iters,
+                    seed=wl.seed, seg_symbols=seg_symbols).upload()
+    sizes = fmt.sizes()
+    peak, peak_kind = _peaks()
+    nbytes = fmt.device_bytes()
+    R = min(64, max(2, math.ceil(3 * L2_BYTES / nbytes)))
+    reps = []
+    for _ in range(R):
+        buf = torch.empty(nbytes + 256, dtype=torch.uint8, device="cuda")
+        off = (-buf.data_ptr()) % 256
+        view = buf[off:off + nbytes]
+        view.copy_(fmt.image())
+        reps.append(view)
+    Wq = fmt.decode_host().astype(np.float64)
+    dense_bytes = 4 * wl.n * wl.m
+    common = dict(config=wl.config, workload=wl.name, format=kind, n=wl.n, m=wl.m, sparsity=wl.sparsity, k=wl.k,
+                  k_eff=sizes["k_eff"], nnz=sizes["nnz"], seg_symbols=sizes["seg_symbols"],
+                  avg_code_len=round(sizes["avg_code_len"], 4), entropy=round(sizes["entropy"], 4),
+                  max_code_len=sizes["max_code_len"], stream_bytes=sizes["stream_bytes"],
+                  offset_index_bytes=sizes["offset_index_bytes"], ri_bytes=sizes["ri_bytes"],
+                  total_bytes=sizes["total_bytes"], psi=round(sizes["total_bytes"] / dense_bytes, 5),
+                  paper_bits=sizes["paper_bits"], bound_bits=sizes["bound_bits"],
+                  bound_over_size=round(sizes["bound_bits"] / max(1, sizes["paper_bits"]), 3))
+    rows = []
+    for B in batches:
+        Xh = si.inputs(wl, B)
+        nx = R if B == 1 else min(R, max(1, (1 << 28) // max(1, 4 * wl.n * B)))
+        if B == 1:
+            xs = [torch.from_numpy(Xh[0]).cuda() for _ in range(nx)]
+            ys = [torch.empty(wl.m, device="cuda") for _ in range(nx)]
+        else:
+            xt = torch.from_numpy(np.ascontiguousarray(Xh.T)).cuda()
+            xs = [xt.clone() for _ in range(nx)]
+            ys = [torch.empty((wl.m, B), device="cuda") for _ in range(nx)]
+        ws = torch.empty(max(16, fmt.workspace_bytes(B)), dtype=torch.uint8, device="cuda")
+
+        def step(r):
+            fmt.attach(reps[r])
+            fmt.dot(xs[r % nx], ys[r % nx], ws)
+
+        step(0)
+        torch.cuda.synchronize()
+        ok = None
+        if B <= max_check_batch:
+            got = ys[0].cpu().numpy().astype(np.float64)
+            got = got[None] if B == 1 else got.T
+            ref = Xh.astype(np.float64) @ Wq
+            tol = 1e-5 * (np.abs(Xh.astype(np.float64)) @ np.abs(Wq)) + 1e-7
+            ok = bool(np.all(np.abs(got - ref) <= tol))
+        for i in range(3):
+            step(i % R)
+        g = _capture(torch, lambda: [step(r) for r in range(R)])
+        g.replay()
+        torch.cuda.synchronize()
+        best = float("inf")
+        for _ in range(replays):
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            g.replay()
+            e1.record()
+            torch.cuda.synchronize()
+            best = min(best, e0.elapsed_time(e1) / R * 1e3)
+        row = dict(common, batch=B, us=round(best, 2), within_tolerance=ok, launches=fmt.last_launch_count(),
+                   gweights_per_s=round(wl.n * wl.m * B / best / 1e3, 1),
+                   symbols_per_s=round(sizes["symbols"] / best * 1e6, 0))
+        if B == 1:
+            ab = algorithmic_bytes(sizes)
+            row.update(algorithmic_bytes=ab, gb_per_s=round(ab / best / 1e3, 1),
+                       frac_of_hbm=round(ab / best / 1e3 / peak, 4), hbm_peak=f"{peak} GB/s ({peak_kind})",
+                       frac_of_8tb=round(ab / best / 1e3 / 8000.0, 4))
+        rows.append(row)
+        del xs, ys
+    return rows
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--configs", default="1,2,3,4")
+    ap.add_argument("--sweep", action="store_true", help="configuration 5: sparsity x k grid, HAC and sHAC")
+    ap.add_argument("--paper-shapes", action="store_true", help="the fully connected shapes of the paper's Sect. V-C")
+    ap.add_argument("--out", default="")
+    args = ap.parse_args()
+    out = open(args.out, "w") if args.out else None
+
+    def emit(rows):
+        for r in rows:
+            line = json.dumps(r)
+            print(line, flush=True)
+            if out:
+                out.write(line + "\n")
+                out.flush()
+
+    wanted = {int(c) for c in args.configs.split(",") if c}
+    table = {1: si.CFG1_TINY_SHAC, 2: si.CFG2_DENSE_HAC, 3: si.CFG3_FC_SHAC, 4: si.CFG4_CONV}
+    for c in sorted(wanted):
+        wl = table[c]
+        W = si.weights(wl)
+        for kind in wl.formats:
+            emit(measure(wl, kind, wl.batches if c != 4 else (1,) + tuple(wl.batches), W=W))
+    if args.sweep:
+        cells = si.sweep_cells()
+        W = si.weights(cells[0])
+        for wl in cells:
+            for kind in wl.formats:
+                emit(measure(wl, kind, wl.batches, W=W))
+    if args.paper_shapes:
+        for wl in si.paper_shaped_cells():
+            for kind in wl.formats:
+                emit(measure(wl, kind, (1, 8)))
+
+
+if __name__ == "__main__":
+    main()
