@@ -38,6 +38,22 @@ GEMM_BATCH = 64
 FALLBACK_HBM_GBS = 6650.0
 
 
+# dram__bytes_read.sum + dram__bytes_write.sum per launch of the GEMV kernel from one ncu capture
+# (profiles/hac_vec_kernel_config2_gemv.md), valid only for the kernel source it was taken on.
+NCU_GEMV_TRAFFIC = {"bytes": 14609408, "kernel_source_sha256": "7fa49c5e66de4356a666e1accfd3519ac453363b011bd9a49be284dffa769a3d"}
+
+
+def gemv_traffic():
+    import hashlib
+    src = os.path.join(ROOT, "paper_2108_12704_b200", "csrc", "hac_kernels.cu")
+    try:
+        with open(src, "rb") as f:
+            same = hashlib.sha256(f.read()).hexdigest() == NCU_GEMV_TRAFFIC["kernel_source_sha256"]
+    except OSError:
+        same = False
+    return NCU_GEMV_TRAFFIC["bytes"] if same else None
+
+
 def measured_peaks():
     path = os.path.join(ROOT, "MEASURED_PEAKS.json")
     if os.path.exists(path):
@@ -382,7 +398,7 @@ def run_ours(args):
     roofline = {"kernel": "hac_vec_kernel (GEMV, batch 1)", "bound": "hbm", "achieved": achieved,
                 "peak": peaks["hbm_gbs"], "peak_source": f"of {peak_kind}", "unit": "GB/s",
                 "frac": achieved / peaks["hbm_gbs"], "frac_of_nominal_8TBs": achieved / 8000.0,
-                "traffic": None, "algorithmic_bytes_per_launch": alg_bytes, "avg_launch_us": gemv_s * 1e6,
+                "traffic": gemv_traffic(), "algorithmic_bytes_per_launch": alg_bytes, "avg_launch_us": gemv_s * 1e6,
                 "symbols_per_s": sizes["symbols"] / gemv_s}
     gemm_flops = 2.0 * n * m * GEMM_BATCH
     tf32_peak = peaks.get("bf16_tflops", 1590.0) * 0.5        # measured bf16 x nominal tf32/bf16 ratio
