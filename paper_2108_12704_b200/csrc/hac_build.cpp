@@ -277,6 +277,42 @@ void make_decode_tables(Format& f) {
         }
         if (t.sub.size() * 4 <= kSubTableBytesMax) break;
     }
+    // zero-run table: for streams that are mostly 1-bit zero code words
+    t.l1_runs.clear();
+    t.zero_len = 0;
+    double zero_share = 0.0;
+    if (!f.sparse) {
+        for (uint32_t s = 0; s < k; ++s)
+            if (f.codebook[s] == 0.0f) {
+                t.zero_len = f.code_len[s];
+                zero_share = f.symbols ? (double)f.counts[s] / (double)f.symbols : 0.0;
+            }
+    }
+    // (measured: a gain from about 90 % zeros on; below that the plain table is as fast or faster)
+    if (t.zero_len == 1 && zero_share >= 0.9 && t.zero_len < L1) {
+        const uint32_t zero_bits = bits_of(0.0f);
+        t.l1_runs.assign((size_t)2 << L1, 0u);
+        const uint32_t mask = (1u << L1) - 1u;
+        for (uint32_t idx = 0; idx < (1u << L1); ++idx) {
+            uint32_t pos = 0, covered = 0, value = zero_bits;
+            while (covered < 200) {
+                const uint32_t at = (idx << pos) & mask;            // the remaining bits, left aligned
+                const uint32_t v = t.l1[2 * at], meta = t.l1[2 * at + 1];
+                if ((meta & 0x80000000u) || meta == 0 || meta > L1 - pos) break;   // does not end inside the prefix
+                pos += meta;
+                ++covered;
+                if (v != zero_bits) { value = v; break; }
+                if (pos >= L1) break;
+            }
+            if (covered == 0) {                                     // a single long code word: keep the entry
+                t.l1_runs[2 * idx] = t.l1[2 * idx];
+                t.l1_runs[2 * idx + 1] = t.l1[2 * idx + 1];
+            } else {
+                t.l1_runs[2 * idx] = value;
+                t.l1_runs[2 * idx + 1] = pos | (covered << 8);
+            }
+        }
+    }
 }
 
 int build_impl(const float* W, int64_t n, int64_t m, int64_t ldw, const hac_build_params* p,
@@ -575,6 +611,7 @@ ImageLayout image_layout(const Format& f) {
     L.lut = take(f.tables.lut.size() * 2);
     L.l1 = take(f.tables.l1.size() * 4);
     L.sub = take(f.tables.sub.size() * 4);
+    L.l1_runs = take(f.tables.l1_runs.size() * 4);
     L.rank_value = take(f.tables.rank_value.size() * 4);
     L.limit = take(sizeof(f.tables.limit));
     L.first_left = take(sizeof(f.tables.first_left));

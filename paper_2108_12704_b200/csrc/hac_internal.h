@@ -32,6 +32,12 @@ struct DecodeTables {
     int l1_bits = 0;
     std::vector<uint32_t> l1;                 // [2^l1_bits * 2]
     std::vector<uint32_t> sub;                // [entries * 2]
+    // Zero-run variant of l1 (HAC with a short code word for 0): an entry covers as many zero symbols
+    // as fit in the prefix plus, if it fits too, the non-zero symbol after them:
+    // {value bits of that symbol (0 if none), length | (symbols covered << 8)}; prefixes of longer code
+    // words keep their sub-table entry.  Empty when the format has no use for it.
+    std::vector<uint32_t> l1_runs;            // [2^l1_bits * 2]
+    uint32_t zero_len = 0;                    // code length of the zero symbol (0 = none)
     uint64_t limit[kMaxCodeLen + 2] = {};     // left-aligned (32-bit) end of the codes of length l
     uint32_t first_left[kMaxCodeLen + 2] = {};// left-aligned first code of length l
     uint32_t rank_base[kMaxCodeLen + 2] = {}; // rank of the first code of length l
@@ -47,6 +53,7 @@ struct DeviceImage {
     const uint16_t* lut = nullptr;
     const uint2_host* l1 = nullptr;
     const uint2_host* sub = nullptr;
+    const uint2_host* l1_runs = nullptr;
     const float* rank_value = nullptr;
     const uint64_t* limit = nullptr;          // [34]
     const uint32_t* first_left = nullptr;     // [34]
@@ -103,7 +110,7 @@ void fill_size_report(const Format& f, hac_size_report* r);
 
 // device image layout: offsets of every section (256-byte aligned), total size
 struct ImageLayout {
-    size_t stream, lut, l1, sub, rank_value, limit, first_left, rank_base, seg_bit_off, sub_bits, seg_col,
+    size_t stream, lut, l1, sub, l1_runs, rank_value, limit, first_left, rank_base, seg_bit_off, sub_bits, seg_col,
         seg_first, ri, cb, unit_info, total;
 };
 ImageLayout image_layout(const Format& f);

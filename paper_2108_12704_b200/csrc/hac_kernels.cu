@@ -84,6 +84,7 @@ __host__ __device__ inline size_t align16(size_t x) { return (x + 15) & ~(size_t
 //            for code words longer still, which are found by a search over lengths in global memory.
 struct TablePlan {
     uint32_t repl_log2;
+    uint32_t zero_len;    // HAC zero-run table in use: code length of the zero symbol
     uint32_t x_bulk;      // sHAC: x is contiguous and 16-byte aligned, so it is brought in by one bulk async copy
 };
 
@@ -108,6 +109,16 @@ __device__ __forceinline__ Decoder stage_decoder(const DevFormat& f, const Table
     // value for a slot fetched from the lane that holds it, so that consecutive lanes write
     // consecutive 8-byte slots (no bank conflicts) and every entry is read from memory once.
     const uint32_t lane_ = threadIdx.x & 31u;
+    // all loads of the first pass are issued before any of them is used, so that the block pays
+    // one trip to memory for its tables, not one per table
+    constexpr int kSubAhead = 4;
+    uint2 sub_v[kSubAhead];
+    const uint32_t sub_entries = f.sub_bytes / 8;
+#pragma unroll
+    for (int k = 0; k < kSubAhead; ++k) {
+        const uint32_t i = threadIdx.x + k * blockDim.x;
+        sub_v[k] = i < sub_entries ? __ldg(f.sub + i) : make_uint2(0u, 0u);
+    }
     for (uint32_t idx0 = threadIdx.x - lane_; idx0 < (1u << f.l1_bits); idx0 += blockDim.x) {
         const uint32_t idx = idx0 + lane_;
         uint2 v = make_uint2(0u, 0u);
@@ -122,7 +133,12 @@ __device__ __forceinline__ Decoder stage_decoder(const DevFormat& f, const Table
             if (s0 + lane_ < warp_slots) dst[s0 + lane_] = w;
         }
     }
-    for (uint32_t i = threadIdx.x; i < f.sub_bytes / 8; i += blockDim.x) sub[i] = __ldg(f.sub + i);
+#pragma unroll
+    for (int k = 0; k < kSubAhead; ++k) {
+        const uint32_t i = threadIdx.x + k * blockDim.x;
+        if (i < sub_entries) sub[i] = sub_v[k];
+    }
+    for (uint32_t i = threadIdx.x + kSubAhead * blockDim.x; i < sub_entries; i += blockDim.x) sub[i] = __ldg(f.sub + i);
     d.l1_lane = smem_off(l1) + ((threadIdx.x & (repl - 1)) << 3);
     d.l1_mul = 8u << tp.repl_log2;
     d.l1_shift = 32 - f.l1_bits;
@@ -407,7 +423,7 @@ __device__ __forceinline__ float warp_sum(float v) {
 // keeps the 32 lanes on distinct banks.
 //   kMode 0: product; 1: debug decode (values written to out[j*n + i]).
 // ------------------------------------------------------------------------------------------------
-template <int kMode, bool kXShared, bool kLong, int kChains>
+template <int kMode, bool kXShared, bool kLong, int kChains, bool kRuns>
 __global__ void __launch_bounds__(1024) hac_vec_kernel(DevFormat f, TablePlan tp, const float* __restrict__ x,
                                                        int64_t xs_i, float* __restrict__ y, int64_t ys_j,
                                                        float* __restrict__ aux) {
@@ -429,13 +445,29 @@ __global__ void __launch_bounds__(1024) hac_vec_kernel(DevFormat f, TablePlan tp
             seg_bit[c] = __ldg(f.seg_bit_off + u);
         }
     }
+    // the first elements of x are requested together with the tables (one trip to memory for both)
+    constexpr int kXAhead = 4;
+    float x_v[kXAhead];
+    if (kMode == 0 && kXShared) {
+#pragma unroll
+        for (int k = 0; k < kXAhead; ++k) {
+            const uint32_t i = threadIdx.x + k * blockDim.x;
+            x_v[k] = i < f.n ? __ldg(x + (int64_t)i * xs_i) : 0.0f;
+        }
+    }
     unsigned char* p = smem;
     const Decoder dec = stage_decoder(f, tp, p);
     const uint32_t pad = (f.S & 1u) ? 0u : 1u;
     float* xs = reinterpret_cast<float*>(p);
     if (kMode == 0 && kXShared) {
+#pragma unroll
+        for (int k = 0; k < kXAhead; ++k) {
+            const uint32_t i = threadIdx.x + k * blockDim.x;
+            if (i < f.n) xs[i + pad * (i / f.S)] = x_v[k];
+        }
 #pragma unroll 4
-        for (uint32_t i = threadIdx.x; i < f.n; i += blockDim.x) xs[i + pad * (i / f.S)] = __ldg(x + (int64_t)i * xs_i);
+        for (uint32_t i = threadIdx.x + kXAhead * blockDim.x; i < f.n; i += blockDim.x)
+            xs[i + pad * (i / f.S)] = __ldg(x + (int64_t)i * xs_i);
         p += align16(((size_t)f.n + (f.n / f.S + 1) * pad) * 4);
     }
     uint4* stage = reinterpret_cast<uint4*>(p) + (size_t)warp * kChains * f.max_unit_chunks;
@@ -487,7 +519,33 @@ __global__ void __launch_bounds__(1024) hac_vec_kernel(DevFormat f, TablePlan tp
         float acc[kChains];
 #pragma unroll
         for (int c = 0; c < kChains; ++c) acc[c] = 0.0f;
-        if (kMode == 0 && kXShared) {
+        if (kMode == 0 && kXShared && kRuns) {
+            // zero-run table: one lookup covers a run of zero entries and the non-zero entry after it
+            const uint32_t sb = shared_base();
+            const uint32_t l1_abs = sb + dec.l1_lane;
+#pragma unroll
+            for (int c = 0; c < kChains; ++c) {
+                FastReader fr;
+                fr.hi = br[c].hi; fr.lo = br[c].lo; fr.off = br[c].off; fr.next = sb + br[c].next;
+                uint32_t left = count[c], xat = xa[c];
+                while (left > 0) {
+                    uint32_t top, val, meta;
+                    fast_lookup(fr, dec.l1_shift, dec.l1_mul, l1_abs, top, val, meta);
+                    uint32_t covered = 1;
+                    if ((int32_t)meta < 0) {
+                        resolve_long(top, dec, f, val, meta);
+                    } else {
+                        covered = meta >> 8;
+                        meta &= 0xffu;
+                        if (covered > left) { covered = 1; meta = tp.zero_len; val = 0u; }   // the run crosses the end: take one zero
+                    }
+                    fast_consume_value(fr, meta);
+                    xat += covered << 2;
+                    acc[c] = fmaf(ldsf(xat - 4), __uint_as_float(val), acc[c]);
+                    left -= covered;
+                }
+            }
+        } else if (kMode == 0 && kXShared) {
             const uint32_t sb = shared_base();
             FastReader fr[kChains];
             uint32_t xabs[kChains];
@@ -1210,6 +1268,7 @@ static void set_pointers(Format& f, void* dev_buf, size_t bytes) {
     f.dev.lut = reinterpret_cast<const uint16_t*>(b + L.lut);
     f.dev.l1 = reinterpret_cast<const uint2_host*>(b + L.l1);
     f.dev.sub = reinterpret_cast<const uint2_host*>(b + L.sub);
+    f.dev.l1_runs = reinterpret_cast<const uint2_host*>(b + L.l1_runs);
     f.dev.rank_value = reinterpret_cast<const float*>(b + L.rank_value);
     f.dev.limit = reinterpret_cast<const uint64_t*>(b + L.limit);
     f.dev.first_left = reinterpret_cast<const uint32_t*>(b + L.first_left);
@@ -1238,6 +1297,7 @@ static int upload(Format& f, void* dev_buf, size_t dev_bytes, void* stream_) {
     HAC_CUDA(put(L.lut, f.tables.lut.data(), f.tables.lut.size() * 2));
     HAC_CUDA(put(L.l1, f.tables.l1.data(), f.tables.l1.size() * 4));
     HAC_CUDA(put(L.sub, f.tables.sub.data(), f.tables.sub.size() * 4));
+    HAC_CUDA(put(L.l1_runs, f.tables.l1_runs.data(), f.tables.l1_runs.size() * 4));
     HAC_CUDA(put(L.rank_value, f.tables.rank_value.data(), f.tables.rank_value.size() * 4));
     HAC_CUDA(put(L.limit, f.tables.limit, sizeof(f.tables.limit)));
     HAC_CUDA(put(L.first_left, f.tables.first_left, sizeof(f.tables.first_left)));
@@ -1310,13 +1370,15 @@ static TablePlan plan_tables(const DevFormat& d, size_t table_budget) {
 typedef void (*VecKernel)(DevFormat, TablePlan, const float*, int64_t, float*, int64_t, float*);
 
 template <bool kLong>
-static VecKernel pick_vec_kernel(const Format& f, int mode, bool x_shared, int chains) {
+static VecKernel pick_vec_kernel(const Format& f, int mode, bool x_shared, int chains, bool runs) {
     if (!f.sparse) {
+        if (runs) return chains == 2 ? hac_vec_kernel<0, true, kLong, 2, true> : hac_vec_kernel<0, true, kLong, 1, true>;
         if (chains == 2)
-            return mode == 1 ? hac_vec_kernel<1, false, kLong, 2>
-                             : (x_shared ? hac_vec_kernel<0, true, kLong, 2> : hac_vec_kernel<0, false, kLong, 2>);
-        return mode == 1 ? hac_vec_kernel<1, false, kLong, 1>
-                         : (x_shared ? hac_vec_kernel<0, true, kLong, 1> : hac_vec_kernel<0, false, kLong, 1>);
+            return mode == 1 ? hac_vec_kernel<1, false, kLong, 2, false>
+                             : (x_shared ? hac_vec_kernel<0, true, kLong, 2, false>
+                                         : hac_vec_kernel<0, false, kLong, 2, false>);
+        return mode == 1 ? hac_vec_kernel<1, false, kLong, 1, false>
+                         : (x_shared ? hac_vec_kernel<0, true, kLong, 1, false> : hac_vec_kernel<0, false, kLong, 1, false>);
     }
     if (f.ri_bits == 16)
         return mode == 1 ? shac_vec_kernel<1, false, kLong, uint16_t>
@@ -1361,8 +1423,13 @@ static int launch_vec(const Format& f, int mode, const float* x, int64_t xs_i, f
     if (smem > budget) return HAC_ERR_BUFFER_TOO_SMALL;
     const bool has_long = d.max_len > d.l1_bits;
     const int threads = warps * 32;
-    VecKernel kernel = has_long ? pick_vec_kernel<true>(f, mode, x_shared, chains)
-                                : pick_vec_kernel<false>(f, mode, x_shared, chains);
+    // HAC with a short code word for zero: the zero-run table replaces the level-1 table
+    const bool runs = !f.sparse && mode == 0 && x_shared && !f.tables.l1_runs.empty() &&
+                      env_int("HAC_B200_ZERO_RUNS", 1) != 0;
+    DevFormat dk = d;
+    if (runs) { dk.l1 = reinterpret_cast<const uint2*>(f.dev.l1_runs); tp.zero_len = f.tables.zero_len; }
+    VecKernel kernel = has_long ? pick_vec_kernel<true>(f, mode, x_shared, chains, runs)
+                                : pick_vec_kernel<false>(f, mode, x_shared, chains, runs);
     rc = prepare_kernel(kernel, smem);
     if (rc) return rc;
     int per_sm = 1;
@@ -1371,7 +1438,7 @@ static int launch_vec(const Format& f, int mode, const float* x, int64_t xs_i, f
     // spread the segments over all SMs (a block's warps take segments blockIdx + k * gridDim)
     const unsigned items = f.sparse ? d.items : (d.units + chains - 1) / chains;
     const unsigned grid = std::min<unsigned>(items, (unsigned)(di.sms * per_sm));
-    kernel<<<grid, threads, smem, st>>>(d, tp, x, xs_i, y, ys_j, aux);
+    kernel<<<grid, threads, smem, st>>>(dk, tp, x, xs_i, y, ys_j, aux);
     if (vec_direct) *vec_direct = (!f.sparse && (f.G == 1 || (chains == 2 && f.G == 2)));
     HAC_CUDA(cudaGetLastError());
     f.last_launches++;
