@@ -849,15 +849,16 @@ __global__ void finalize_kernel(DevFormat f, bool sparse, const float* __restric
 // A block owns 32 consecutive columns of W, a range of segment indices g (all of them unless the
 // grid would be too small) and a tile of 64 inputs.  Work proceeds in chunks of 64 rows: every lane
 // decodes two symbols of each of its two sub-segments, and the 64 matching rows of X are fetched.
-// One MMA is D[64 inputs][32 columns] += X[64][8] * W[32][8]^T in TF32; both operands are read by the
-// tensor core straight from shared memory ("K-major", no swizzle): a group of four consecutive K
-// elements of one row is a 16-byte unit, 8 rows form a 128-byte core matrix, core matrices of
-// successive 8-row groups are kTcSbo bytes apart, the two K halves of an MMA are LBO bytes apart.
-// Strides are padded so that the stores of the decode phase hit distinct banks.
-// Split precision: every weight and every input is written as hi + lo, both rounded to TF32, and
-// three products are accumulated in fp32 (x_lo*w_hi + x_hi*w_lo + x_hi*w_hi); the error stays near
-// 1e-7 of sum |w x|, well inside the output tolerance.
-// For 64 inputs the accumulator rows sit in tensor-memory lanes 0-15, 32-47, 64-79 and 96-111.
+// Both operands are read by the tensor core straight from shared memory in TF32 ("K-major", no
+// swizzle): a group of four consecutive K elements of one row is a 16-byte unit, 8 rows form a
+// 128-byte core matrix, core matrices of successive 8-row groups are kTcSbo bytes apart, the two K
+// halves of an MMA are LBO bytes apart.  Strides are padded so that the stores of the decode phase
+// hit distinct banks.
+// Split precision: every weight and every input is written as hi + lo, both rounded to TF32.  The
+// hi and lo parts are stacked along M (inputs) and N (columns), so one MMA
+// D[128][64] += [x_hi; x_lo][128][8] * [w_hi; w_lo][64][8]^T forms all four partial products; the
+// epilogue adds the four quadrants in fp32.  The error stays near 1e-7 of sum |w x|, well inside the
+// output tolerance.  Accumulator row r sits in tensor-memory lane r.
 // The stream is decoded once per batch tile and never written to global memory.
 // ------------------------------------------------------------------------------------------------
 constexpr int kBatchSteps = 4;          // sHAC batched kernel: entries decoded per lane per phase
@@ -869,18 +870,29 @@ __device__ __forceinline__ uint32_t to_tf32(float v) {
     asm("cvt.rna.tf32.f32 %0, %1;" : "=r"(r) : "f"(v));
     return r;
 }
+__device__ __forceinline__ void sts64(uint32_t addr, float a, float b) {
+    asm volatile("st.shared.v2.f32 [%0], {%1, %2};" ::"r"(addr), "f"(a), "f"(b) : "memory");
+}
+__device__ __forceinline__ void sts128(uint32_t addr, float a, float b, float c, float d) {
+    asm volatile("st.shared.v4.f32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "f"(a), "f"(b), "f"(c), "f"(d) : "memory");
+}
 
 constexpr int kTcSteps = 2;                         // symbols decoded per lane per chunk
 constexpr int kTcRows = 32 * kTcSteps;              // K per chunk (64)
 constexpr int kTcKSteps = kTcRows / 8;              // MMAs (of K = 8) per chunk and product
 constexpr int kTcSbo = 128;
-constexpr int kTcXLbo = 1024, kTcXKst = 2048;       // X tile: 64 rows -> 8 core matrices per K half
-constexpr int kTcWLbo = 528, kTcWKst = 1056;        // W tile: 32 rows -> 4 core matrices, padded
+// One MMA per 8 rows covers all split products: A stacks x_hi (rows 0-63) on x_lo (rows 64-127),
+// B stacks w_hi (rows 0-31) on w_lo (rows 32-63); D[128][64] then holds x_hi*w_hi, x_hi*w_lo,
+// x_lo*w_hi and x_lo*w_lo in its four quadrants, which the epilogue adds.
+constexpr int kTcXLbo = 2048, kTcXKst = 4096;       // A tile: 128 rows -> 16 core matrices per K half
+constexpr int kTcXLoRows = 8 * kTcSbo;              // byte offset of the x_lo rows inside a K half
+constexpr int kTcWLbo = 1040, kTcWKst = 2080;       // B tile: 64 rows -> 8 core matrices, padded
+constexpr int kTcWLoRows = 4 * kTcSbo;              // byte offset of the w_lo rows
 constexpr int kTcCols = 32, kTcBatch = 64, kTcDecodeWarps = 16;
 constexpr uint32_t kTcWaitTries = 400000;
 
 __host__ __device__ inline size_t tc_tile_bytes() {
-    return (size_t)2 * kTcKSteps * kTcXKst + (size_t)2 * kTcKSteps * kTcWKst;
+    return (size_t)kTcKSteps * kTcXKst + (size_t)kTcKSteps * kTcWKst;
 }
 __device__ __forceinline__ uint64_t tc_desc(uint32_t shared_addr, uint32_t lbo_bytes) {
     return (uint64_t)((shared_addr >> 4) & 0x3fffu) | ((uint64_t)((lbo_bytes >> 4) & 0x3fffu) << 16) |
@@ -891,6 +903,12 @@ __device__ __forceinline__ void tc_mma(uint32_t tmem, uint64_t a, uint64_t b, ui
         "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
         "tcgen05.mma.cta_group::1.kind::tf32 [%0], %1, %2, %3, p;\n\t}"
         ::"r"(tmem), "l"(a), "l"(b), "r"(idesc), "r"(accumulate) : "memory");
+}
+__device__ __forceinline__ void tc_mma_acc(uint32_t tmem, uint64_t a, uint64_t b, uint32_t idesc) {   // D += A * B
+    asm volatile(
+        "{\n\t.reg .pred p;\n\tsetp.eq.b32 p, 0, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::tf32 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(tmem), "l"(a), "l"(b), "r"(idesc) : "memory");
 }
 __device__ __forceinline__ void tc_commit(uint32_t mbar) {
     asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(mbar) : "memory");
@@ -905,6 +923,18 @@ __device__ __forceinline__ bool tc_wait(uint32_t mbar, uint32_t parity) {
     return false;
 }
 
+// 32 consecutive 32-bit columns of this warp's 32 tensor-memory lanes, one lane per thread.
+__device__ __forceinline__ void tmem_ld32(uint32_t (&r)[32], uint32_t taddr) {
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x32.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,%17,%18,%19,"
+        "%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31}, [%32];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+          "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
+          "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
+          "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+        : "r"(taddr) : "memory");
+}
+
 // Warp-specialised and pipelined: warps 0..15 decode (two columns each, two chains per lane) and
 // stage the rows of X; warp 16 only issues the MMAs.  Tiles live in a ring of `stages` buffers with
 // two mbarriers each: `full` (16 arrivals, one per decode warp, after its stores) and `empty`
@@ -914,7 +944,7 @@ __device__ __forceinline__ bool tc_wait(uint32_t mbar, uint32_t parity) {
 __global__ void __launch_bounds__((kTcDecodeWarps + 1) * 32) hac_gemm_tc_kernel(
     DevFormat f, TablePlan tp, const float* __restrict__ x, int64_t xs_i, int64_t xs_b, uint32_t batch,
     float* __restrict__ y, int64_t ys_j, int64_t ys_b, float* __restrict__ partial, uint32_t col_blocks,
-    uint32_t row_splits, uint32_t stages) {
+    uint32_t row_splits, uint32_t stages, uint32_t x_small) {
     const uint32_t warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const uint32_t cblk = blockIdx.x % col_blocks;
     const uint32_t rest = blockIdx.x / col_blocks;
@@ -941,15 +971,14 @@ __global__ void __launch_bounds__((kTcDecodeWarps + 1) * 32) hac_gemm_tc_kernel(
     }
     __syncwarp();
     if (warp == kTcDecodeWarps) {
-        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(sb + 40), "r"(32u) : "memory");
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(sb + 40), "r"(64u) : "memory");
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
     }
     const Decoder dec = stage_decoder(f, tp, p);
     p = smem + ((smem_off(p) + 127u) & ~127u);
     const uint32_t ring = smem_off(p);                          // stage s at ring + s * tc_tile_bytes()
     p += (size_t)stages * tc_tile_bytes();
-    constexpr uint32_t kXHi = 0, kXLo = kTcKSteps * kTcXKst, kWHi = 2 * kTcKSteps * kTcXKst,
-                       kWLo = kWHi + kTcKSteps * kTcWKst;
+    constexpr uint32_t kXHi = 0, kXLo = kTcXLoRows, kWHi = kTcKSteps * kTcXKst, kWLo = kWHi + kTcWLoRows;
     asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
     __syncthreads();
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
@@ -958,21 +987,21 @@ __global__ void __launch_bounds__((kTcDecodeWarps + 1) * 32) hac_gemm_tc_kernel(
     if (warp == kTcDecodeWarps) {
         // ---- MMA issue: one lane, chunk after chunk ----
         if (lane == 0) {
-            const uint32_t idesc = (1u << 4) | (2u << 7) | (2u << 10) | ((uint32_t)(kTcCols >> 3) << 17) |
-                                   ((uint32_t)(kTcBatch >> 4) << 24);
+            // D f32, A and B tf32, both K-major, N = 64 (w_hi | w_lo), M = 128 (x_hi | x_lo)
+            const uint32_t idesc = (1u << 4) | (2u << 7) | (2u << 10) | ((uint32_t)((2 * kTcCols) >> 3) << 17) |
+                                   ((uint32_t)((2 * kTcBatch) >> 4) << 24);
             for (uint32_t c = 0; c < chunks; ++c) {
                 const uint32_t s = c % stages, use = c / stages;
                 if (!tc_wait(bar_full + 8 * s, use & 1u)) *lost_flag = 1;
                 asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+                // descriptors differ from MMA to MMA only in the 14-bit start-address field (low word)
                 const uint32_t base = sb + ring + s * (uint32_t)tc_tile_bytes();
-                uint64_t a_hi = tc_desc(base + kXHi, kTcXLbo), a_lo = tc_desc(base + kXLo, kTcXLbo);
-                uint64_t b_hi = tc_desc(base + kWHi, kTcWLbo), b_lo = tc_desc(base + kWLo, kTcWLbo);
+                const uint64_t a0 = tc_desc(base + kXHi, kTcXLbo), b0d = tc_desc(base + kWHi, kTcWLbo);
 #pragma unroll
                 for (int ks = 0; ks < kTcKSteps; ++ks) {
-                    tc_mma(tmem, a_lo, b_hi, idesc, (c | (uint32_t)ks) ? 1u : 0u);
-                    tc_mma(tmem, a_hi, b_lo, idesc, 1u);
-                    tc_mma(tmem, a_hi, b_hi, idesc, 1u);
-                    a_hi += kTcXKst >> 4; a_lo += kTcXKst >> 4; b_hi += kTcWKst >> 4; b_lo += kTcWKst >> 4;
+                    const uint64_t a = a0 + (uint64_t)(ks * (kTcXKst >> 4)), b = b0d + (uint64_t)(ks * (kTcWKst >> 4));
+                    if (ks == 0) tc_mma(tmem, a, b, idesc, c == 0 ? 0u : 1u);
+                    else tc_mma_acc(tmem, a, b, idesc);
                 }
                 tc_commit(bar_empty + 8 * s);
             }
@@ -999,17 +1028,32 @@ __global__ void __launch_bounds__((kTcDecodeWarps + 1) * 32) hac_gemm_tc_kernel(
             b_ok[i] = b0 + b < batch;
             x_col[i] = x + (int64_t)(b0 + b) * xs_b;
         }
+        const int32_t xs_i32 = (int32_t)xs_i;                   // used only when x_small (offsets fit 31 bits)
         auto load_x = [&](uint32_t g, uint32_t s0) {
             const uint32_t row_base = g * 32 * f.S + s0;
-            const bool second = s0 + 1 < f.S;                  // the chunk's second symbol exists
+            // interior chunk: every row of the tile exists (rows run up to row_base + 31*S + 1)
+            const bool interior = s0 + 1 < f.S && row_base + 31u * f.S + 1u < f.n;
+            if (interior && x_small) {
+                const int32_t base_off = (int32_t)row_base * xs_i32;
 #pragma unroll
-            for (int i = 0; i < 2; ++i) {
+                for (int i = 0; i < 2; ++i) {
 #pragma unroll
-                for (int e = 0; e < 4; ++e) {
-                    const uint32_t row = row_base + row_off[i][e];
-                    float v = 0.0f;
-                    if (b_ok[i] && row < f.n && ((e & 1) == 0 || second)) v = __ldg(x_col[i] + (int64_t)row * xs_i);
-                    xr[i][e] = v;
+                    for (int e = 0; e < 4; ++e) {
+                        const int32_t off = base_off + (int32_t)row_off[i][e] * xs_i32;
+                        xr[i][e] = b_ok[i] ? __ldg(x_col[i] + off) : 0.0f;
+                    }
+                }
+            } else {
+                const bool second = s0 + 1 < f.S;              // the chunk's second symbol exists
+#pragma unroll
+                for (int i = 0; i < 2; ++i) {
+#pragma unroll
+                    for (int e = 0; e < 4; ++e) {
+                        const uint32_t row = row_base + row_off[i][e];
+                        float v = 0.0f;
+                        if (b_ok[i] && row < f.n && ((e & 1) == 0 || second)) v = __ldg(x_col[i] + (int64_t)row * xs_i);
+                        xr[i][e] = v;
+                    }
                 }
             }
         };
@@ -1040,33 +1084,56 @@ __global__ void __launch_bounds__((kTcDecodeWarps + 1) * 32) hac_gemm_tc_kernel(
                 }
             }
             const uint32_t seg_rows = min(f.S, f.n - min(f.n, g * 32 * f.S));
+            // symbols every lane of the warp still has in both chains (lets whole chunks skip the per-lane checks)
+            const uint32_t common = __reduce_min_sync(0xffffffffu, min(count[0], count[1]));
             for (uint32_t s0 = 0; s0 < seg_rows; s0 += kTcSteps, ++c) {
                 float hi[2][kTcSteps], lo[2][kTcSteps];
+                if (s0 + kTcSteps <= common) {
 #pragma unroll
-                for (int st = 0; st < kTcSteps; ++st) {
-                    uint32_t top[2], val[2], len[2];
+                    for (int st = 0; st < kTcSteps; ++st) {
+                        uint32_t top[2], val[2], len[2];
 #pragma unroll
-                    for (int ch = 0; ch < 2; ++ch) {
-                        top[ch] = val[ch] = len[ch] = 0;
-                        if (s0 + st < count[ch]) fast_lookup(fr[ch], dec.l1_shift, dec.l1_mul, l1_abs, top[ch], val[ch], len[ch]);
+                        for (int ch = 0; ch < 2; ++ch) fast_lookup(fr[ch], dec.l1_shift, dec.l1_mul, l1_abs, top[ch], val[ch], len[ch]);
+                        if ((int32_t)(len[0] | len[1]) < 0) {
+#pragma unroll
+                            for (int ch = 0; ch < 2; ++ch)
+                                if ((int32_t)len[ch] < 0) resolve_long(top[ch], dec, f, val[ch], len[ch]);
+                        }
+#pragma unroll
+                        for (int ch = 0; ch < 2; ++ch) {
+                            fast_consume_value(fr[ch], len[ch]);
+                            const float w = __uint_as_float(val[ch]);
+                            hi[ch][st] = __uint_as_float(to_tf32(w));
+                            lo[ch][st] = __uint_as_float(to_tf32(w - hi[ch][st]));
+                        }
                     }
+                } else {
 #pragma unroll
-                    for (int ch = 0; ch < 2; ++ch) {
-                        if ((int32_t)len[ch] < 0) resolve_long(top[ch], dec, f, val[ch], len[ch]);
-                        if (s0 + st < count[ch]) fast_consume_value(fr[ch], len[ch]);
-                        const float w = __uint_as_float(val[ch]);
-                        hi[ch][st] = __uint_as_float(to_tf32(w));
-                        lo[ch][st] = __uint_as_float(to_tf32(w - hi[ch][st]));
+                    for (int st = 0; st < kTcSteps; ++st) {
+                        uint32_t top[2], val[2], len[2];
+#pragma unroll
+                        for (int ch = 0; ch < 2; ++ch) {
+                            top[ch] = val[ch] = len[ch] = 0;
+                            if (s0 + st < count[ch]) fast_lookup(fr[ch], dec.l1_shift, dec.l1_mul, l1_abs, top[ch], val[ch], len[ch]);
+                        }
+#pragma unroll
+                        for (int ch = 0; ch < 2; ++ch) {
+                            if ((int32_t)len[ch] < 0) resolve_long(top[ch], dec, f, val[ch], len[ch]);
+                            if (s0 + st < count[ch]) fast_consume_value(fr[ch], len[ch]);
+                            const float w = __uint_as_float(val[ch]);
+                            hi[ch][st] = __uint_as_float(to_tf32(w));
+                            lo[ch][st] = __uint_as_float(to_tf32(w - hi[ch][st]));
+                        }
                     }
                 }
                 const uint32_t s = c % stages, use = c / stages;
                 // the buffer is free once the MMAs of its previous use have been committed
                 if (use > 0 && !tc_wait(bar_empty + 8 * s, (use - 1) & 1u)) *lost_flag = 1;
-                unsigned char* tile = smem + ring + (size_t)s * tc_tile_bytes();
+                const uint32_t tile = sb + ring + s * (uint32_t)tc_tile_bytes();
 #pragma unroll
                 for (int ch = 0; ch < 2; ++ch) {
-                    *reinterpret_cast<float2*>(tile + kWHi + w_at[ch]) = make_float2(hi[ch][0], hi[ch][1]);
-                    *reinterpret_cast<float2*>(tile + kWLo + w_at[ch]) = make_float2(lo[ch][0], lo[ch][1]);
+                    sts64(tile + kWHi + w_at[ch], hi[ch][0], hi[ch][1]);
+                    sts64(tile + kWLo + w_at[ch], lo[ch][0], lo[ch][1]);
                 }
 #pragma unroll
                 for (int i = 0; i < 2; ++i) {
@@ -1076,8 +1143,8 @@ __global__ void __launch_bounds__((kTcDecodeWarps + 1) * 32) hac_gemm_tc_kernel(
                         xh[e] = __uint_as_float(to_tf32(xr[i][e]));
                         xl[e] = __uint_as_float(to_tf32(xr[i][e] - xh[e]));
                     }
-                    *reinterpret_cast<float4*>(tile + kXHi + x_at[i]) = make_float4(xh[0], xh[1], xh[2], xh[3]);
-                    *reinterpret_cast<float4*>(tile + kXLo + x_at[i]) = make_float4(xl[0], xl[1], xl[2], xl[3]);
+                    sts128(tile + kXHi + x_at[i], xh[0], xh[1], xh[2], xh[3]);
+                    sts128(tile + kXLo + x_at[i], xl[0], xl[1], xl[2], xl[3]);
                 }
                 asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
                 __syncwarp();
@@ -1093,38 +1160,45 @@ __global__ void __launch_bounds__((kTcDecodeWarps + 1) * 32) hac_gemm_tc_kernel(
     if (chunks > 0 && !tc_wait(bar_done, 0)) lost = true;
     const bool any_lost = __syncthreads_or((lost || *lost_flag) ? 1 : 0) != 0;
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-    if (warp < 4) {                          // warp w reads tensor-memory lanes 32w..32w+31: inputs 16w..16w+15
-        uint32_t r[32];
+    // Accumulator row r sits in tensor-memory lane r: warps 0,1 hold the x_hi rows of inputs 0..63,
+    // warps 2,3 the x_lo rows; columns 0..31 are the w_hi products, 32..63 the w_lo products.
+    float acc[kTcCols];
+    float* fold = reinterpret_cast<float*>(smem + ring);     // [column][input], the tiles are no longer in use
+    if (warp < 4) {
         if (chunks > 0 && !any_lost) {
+            uint32_t r0[32], r1[32];
             const uint32_t src = tmem + ((warp * 32u) << 16);
-            asm volatile(
-                "tcgen05.ld.sync.aligned.32x32b.x32.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,%17,%18,%19,"
-                "%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31}, [%32];"
-                : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
-                  "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
-                  "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
-                  "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
-                : "r"(src) : "memory");
+            tmem_ld32(r0, src);
+            tmem_ld32(r1, src + kTcCols);
             asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+#pragma unroll
+            for (int cc = 0; cc < kTcCols; ++cc) acc[cc] = __uint_as_float(r1[cc]) + __uint_as_float(r0[cc]);
         } else {
 #pragma unroll
-            for (int cc = 0; cc < 32; ++cc) r[cc] = any_lost ? 0x7fc00000u : 0u;   // NaN marks a lost wait
+            for (int cc = 0; cc < kTcCols; ++cc) acc[cc] = any_lost ? __uint_as_float(0x7fc00000u) : 0.f;   // NaN marks a lost wait
         }
-        const uint32_t b = b0 + warp * 16 + lane;
-        if (lane < 16 && b < batch) {
+        if (warp >= 2) {
 #pragma unroll
-            for (int cc = 0; cc < 32; ++cc) {
-                const uint32_t j = cblk * kTcCols + cc;
-                if (j < f.m) {
-                    if (row_splits == 1) y[(int64_t)j * ys_j + (int64_t)b * ys_b] = __uint_as_float(r[cc]);
-                    else partial[((size_t)j * row_splits + rs) * batch + b] = __uint_as_float(r[cc]);
-                }
-            }
+            for (int cc = 0; cc < kTcCols; ++cc) fold[cc * kTcBatch + (warp - 2) * 32 + lane] = acc[cc];
         }
     }
     asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
     __syncthreads();
-    if (warp == kTcDecodeWarps) asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(32u) : "memory");
+    if (warp < 2) {
+        const uint32_t b = b0 + warp * 32 + lane;
+        if (b < batch) {
+#pragma unroll
+            for (int cc = 0; cc < kTcCols; ++cc) {
+                const uint32_t j = cblk * kTcCols + cc;
+                if (j < f.m) {
+                    const float v = fold[cc * kTcBatch + warp * 32 + lane] + acc[cc];
+                    if (row_splits == 1) y[(int64_t)j * ys_j + (int64_t)b * ys_b] = v;
+                    else partial[((size_t)j * row_splits + rs) * batch + b] = v;
+                }
+            }
+        }
+    }
+    if (warp == kTcDecodeWarps) asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(64u) : "memory");
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -1473,8 +1547,10 @@ static int launch_gemm_tc(const Format& f, const DeviceInfo& di, const DevFormat
     const uint32_t rs = gemm_row_splits(f, batch, di.sms);
     const uint64_t grid = (uint64_t)col_blocks * rs * batch_tiles;
     if (grid > 0x7fffffffull) return HAC_ERR_OFFSET_OVERFLOW;
+    // row offsets into x fit 31 bits: the kernel may use 32-bit offsets from the column pointer
+    const uint32_t x_small = (xs_i >= 0 && (uint64_t)xs_i * (uint64_t)(f.n + 1) < ((uint64_t)1 << 31)) ? 1u : 0u;
     hac_gemm_tc_kernel<<<(unsigned)grid, (kTcDecodeWarps + 1) * 32, smem, st>>>(
-        d, tp, x, xs_i, xs_b, (uint32_t)batch, y, ys_j, ys_b, partial, col_blocks, rs, stages);
+        d, tp, x, xs_i, xs_b, (uint32_t)batch, y, ys_j, ys_b, partial, col_blocks, rs, stages, x_small);
     HAC_CUDA(cudaGetLastError());
     f.last_launches++;
     *row_splits_out = rs;
