@@ -184,12 +184,13 @@ int shac_attach(shac_format* f, void* dev_buf, size_t dev_bytes);
  * [batch][n] or [n][batch] and Y [batch][m] or [m][batch]; the batched kernels are fastest with
  * x_stride_b == 1 and y_stride_b == 1.  x and y must not overlap.  Code words are decoded on the
  * fly; the uncompressed weights are never written to global memory.  Products and sums are fp32.
- *   workspace  device scratch of at least *_workspace_bytes(f, batch) bytes (may be NULL when that
- *              is 0).  It holds partial sums of columns that span several segments; its contents
- *              need not be initialised and are undefined afterwards.  Two dot calls that run
- *              concurrently must not share it.
+ *   workspace  device scratch of at least *_workspace_bytes(f, batch) bytes, 16-byte aligned (may be
+ *              NULL when that is 0).  It holds partial sums of columns that span several segments
+ *              and, for a batched HAC product, the inputs split into two TF32 parts and arranged
+ *              in the tiles the tensor-core kernel reads; its contents need not be initialised and
+ *              are undefined afterwards.  Two dot calls that run concurrently must not share it.
  * Asynchronous on cuda_stream.  Errors: HAC_ERR_NOT_UPLOADED, HAC_ERR_INVALID_ARG (batch < 1, null
- * pointers), HAC_ERR_BUFFER_TOO_SMALL, HAC_ERR_CUDA (launch failure).
+ * pointers, misaligned workspace), HAC_ERR_BUFFER_TOO_SMALL, HAC_ERR_CUDA (launch failure).
  * ------------------------------------------------------------------------------------------- */
 int hac_workspace_bytes (const hac_format*  f, int64_t batch, size_t* out);
 int shac_workspace_bytes(const shac_format* f, int64_t batch, size_t* out);
@@ -225,7 +226,7 @@ int shac_dot_host(const shac_format* f, const float* X_host, int64_t batch, floa
  * and uses no allocating library routine; x and y are still the caller's.
  *
  * Arguments and result as hac_dot, without the workspace pair.
- *   - A product whose partial sums need more than HAC_NOALLOC_SCRATCH_BYTES (see hac_workspace_bytes)
+ *   - A product whose workspace would exceed HAC_NOALLOC_SCRATCH_BYTES (see hac_workspace_bytes)
  *     is refused with HAC_ERR_BUFFER_TOO_SMALL and nothing is launched; hac_last_cuda_error() then
  *     names the two sizes.  Use hac_dot with your own workspace for those.
  *   - The first call on each device looks up the device address of the buffer (one

@@ -888,6 +888,8 @@ constexpr int kTcXLbo = 2048, kTcXKst = 4096;       // A tile: 128 rows -> 16 co
 constexpr int kTcXLoRows = 8 * kTcSbo;              // byte offset of the x_lo rows inside a K half
 constexpr int kTcWLbo = 1040, kTcWKst = 2080;       // B tile: 64 rows -> 8 core matrices, padded
 constexpr int kTcWLoRows = 4 * kTcSbo;              // byte offset of the w_lo rows
+constexpr uint32_t kTcXTileBytes = kTcKSteps * kTcXKst;   // one A tile (x_hi and x_lo of 64 rows x 64 inputs)
+static_assert(kTcSteps == 2, "the A tile layout pairs two lanes x two symbols per 16-byte unit");
 constexpr int kTcCols = 32, kTcBatch = 64, kTcDecodeWarps = 16;
 constexpr uint32_t kTcWaitTries = 400000;
 
@@ -935,16 +937,52 @@ __device__ __forceinline__ void tmem_ld32(uint32_t (&r)[32], uint32_t taddr) {
         : "r"(taddr) : "memory");
 }
 
+// A tiles of hac_gemm_tc_kernel, made once per product: for every (batch tile, segment g, chunk)
+// the 64 rows the chunk multiplies (row of K index 2*lane + step = g*32*S + lane*S + s0 + step) of
+// 64 inputs, split into TF32 hi and lo parts and stored exactly as the tile sits in shared memory,
+// so that the product kernel brings a tile in with a single bulk copy.  Rows past the matrix and
+// inputs past the batch are zero.  Tile ((bt*G + g)*cps + chunk) starts at that index times
+// kTcXTileBytes.  Four blocks of 256 threads per tile, one 16-byte unit of each part per thread.
+__global__ void __launch_bounds__(256) hac_pack_x_kernel(DevFormat f, const float* __restrict__ x, int64_t xs_i,
+                                                         int64_t xs_b, uint32_t batch, unsigned char* __restrict__ xpack,
+                                                         uint32_t cps) {
+    const uint32_t tile = blockIdx.x >> 2;
+    const uint32_t ci = tile % cps, g = (tile / cps) % f.G, bt = tile / (cps * f.G);
+    const uint32_t s0 = ci * kTcSteps;
+    const uint32_t seg_rows = min(f.S, f.n - min(f.n, g * 32 * f.S));
+    if (s0 >= seg_rows) return;                       // no chunk here (last segment of a ragged matrix)
+    const uint32_t pi = (blockIdx.x & 3u) * 256 + threadIdx.x;
+    const uint32_t q = pi / kTcBatch, b = pi % kTcBatch;
+    const bool b_ok = bt * kTcBatch + b < batch;
+    const float* xc = x + (int64_t)(bt * kTcBatch + b) * xs_b;
+    float hi[4], lo[4];
+#pragma unroll
+    for (int e = 0; e < 4; ++e) {
+        const uint32_t step = e & 1, sub = 2 * q + (e >> 1);
+        const uint64_t row = (uint64_t)g * 32 * f.S + (uint64_t)sub * f.S + s0 + step;
+        float v = 0.0f;
+        if (b_ok && s0 + step < f.S && row < f.n) v = __ldg(xc + (int64_t)row * xs_i);
+        hi[e] = __uint_as_float(to_tf32(v));
+        lo[e] = __uint_as_float(to_tf32(v - hi[e]));
+    }
+    unsigned char* at = xpack + (size_t)tile * kTcXTileBytes + (q >> 1) * kTcXKst + (q & 1u) * kTcXLbo +
+                        (b >> 3) * kTcSbo + (b & 7u) * 16;
+    *reinterpret_cast<float4*>(at) = make_float4(hi[0], hi[1], hi[2], hi[3]);
+    *reinterpret_cast<float4*>(at + kTcXLoRows) = make_float4(lo[0], lo[1], lo[2], lo[3]);
+}
+
 // Warp-specialised and pipelined: warps 0..15 decode (two columns each, two chains per lane) and
-// stage the rows of X; warp 16 only issues the MMAs.  Tiles live in a ring of `stages` buffers with
-// two mbarriers each: `full` (16 arrivals, one per decode warp, after its stores) and `empty`
-// (arrival by tcgen05.commit once the MMAs that read the buffer have finished).  There is no
-// block-wide barrier inside the loop, so a slow code word delays only its own warp.
+// write the W tiles; one lane of warp 16 fetches the X tiles, which hac_pack_x_kernel has already
+// split and laid out as the tensor core reads them, with one bulk copy each, and issues the MMAs.
+// Tiles live in a ring of `stages` buffers with three mbarriers each: `full` (16 arrivals, one per
+// decode warp, after its stores), `xin` (the bytes of the bulk copy) and `empty` (arrival by
+// tcgen05.commit once the MMAs that read the buffer have finished).  There is no block-wide barrier
+// inside the loop, so a slow code word delays only its own warp.
 // Every wait is bounded; if one runs out the block marks its outputs NaN and still terminates.
-__global__ void __launch_bounds__((kTcDecodeWarps + 1) * 32) hac_gemm_tc_kernel(
-    DevFormat f, TablePlan tp, const float* __restrict__ x, int64_t xs_i, int64_t xs_b, uint32_t batch,
+__global__ void __launch_bounds__((kTcDecodeWarps + 1) * 32, 1) hac_gemm_tc_kernel(
+    DevFormat f, TablePlan tp, const unsigned char* __restrict__ xpack, uint32_t batch,
     float* __restrict__ y, int64_t ys_j, int64_t ys_b, float* __restrict__ partial, uint32_t col_blocks,
-    uint32_t row_splits, uint32_t stages, uint32_t x_small) {
+    uint32_t row_splits, uint32_t stages) {
     const uint32_t warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const uint32_t cblk = blockIdx.x % col_blocks;
     const uint32_t rest = blockIdx.x / col_blocks;
@@ -958,27 +996,31 @@ __global__ void __launch_bounds__((kTcDecodeWarps + 1) * 32) hac_gemm_tc_kernel(
     for (uint32_t g = g_begin; g < g_end; ++g)
         chunks += (min(f.S, f.n - min(f.n, g * 32 * f.S)) + kTcSteps - 1) / kTcSteps;
 
-    // shared memory: [mbarriers full[2], empty[2], done; tensor-memory address; lost flag] [tables] [tile ring] [spans]
+    // shared memory: [mbarriers full[2], empty[2], xin[2], done; tensor-memory address; lost flag] [tables] [tile ring] [spans]
     unsigned char* p = smem;
-    const uint32_t bar_full = sb, bar_empty = sb + 16, bar_done = sb + 32;
-    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem + 40);
-    volatile uint32_t* lost_flag = reinterpret_cast<volatile uint32_t*>(smem + 44);
-    p += 48;
+    const uint32_t bar_full = sb, bar_empty = sb + 16, bar_xin = sb + 32, bar_done = sb + 48;
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem + 56);
+    volatile uint32_t* lost_flag = reinterpret_cast<volatile uint32_t*>(smem + 60);
+    p += 64;
     if (threadIdx.x == 0) {
-        for (uint32_t s = 0; s < 2; ++s) { mbar_init(bar_full + 8 * s, kTcDecodeWarps); mbar_init(bar_empty + 8 * s, 1); }
+        for (uint32_t s = 0; s < 2; ++s) {
+            mbar_init(bar_full + 8 * s, kTcDecodeWarps);
+            mbar_init(bar_empty + 8 * s, 1);
+            mbar_init(bar_xin + 8 * s, 1);
+        }
         mbar_init(bar_done, 1);
         *lost_flag = 0;
     }
     __syncwarp();
     if (warp == kTcDecodeWarps) {
-        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(sb + 40), "r"(64u) : "memory");
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(sb + 56), "r"(64u) : "memory");
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
     }
     const Decoder dec = stage_decoder(f, tp, p);
     p = smem + ((smem_off(p) + 127u) & ~127u);
     const uint32_t ring = smem_off(p);                          // stage s at ring + s * tc_tile_bytes()
     p += (size_t)stages * tc_tile_bytes();
-    constexpr uint32_t kXHi = 0, kXLo = kTcXLoRows, kWHi = kTcKSteps * kTcXKst, kWLo = kWHi + kTcWLoRows;
+    constexpr uint32_t kXHi = 0, kWHi = kTcKSteps * kTcXKst, kWLo = kWHi + kTcWLoRows;
     asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
     __syncthreads();
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
@@ -990,9 +1032,28 @@ __global__ void __launch_bounds__((kTcDecodeWarps + 1) * 32) hac_gemm_tc_kernel(
             // D f32, A and B tf32, both K-major, N = 64 (w_hi | w_lo), M = 128 (x_hi | x_lo)
             const uint32_t idesc = (1u << 4) | (2u << 7) | (2u << 10) | ((uint32_t)((2 * kTcCols) >> 3) << 17) |
                                    ((uint32_t)((2 * kTcBatch) >> 4) << 24);
+            // X tiles of this block: consecutive in xpack (every segment but the matrix's last has cps chunks)
+            const uint32_t cps = (f.S + kTcSteps - 1) / kTcSteps;
+            const unsigned char* xt = xpack + ((size_t)bt * f.G + g_begin) * cps * (size_t)kTcXTileBytes;
+            auto fetch_x = [&](uint32_t cc) {
+                const uint32_t s = cc % stages;
+                mbar_expect_tx(bar_xin + 8 * s, kTcXTileBytes);
+                bulk_copy_g2s(sb + ring + s * (uint32_t)tc_tile_bytes() + kXHi, xt + (size_t)cc * kTcXTileBytes,
+                              kTcXTileBytes, bar_xin + 8 * s);
+            };
+            for (uint32_t cc = 0; cc < min(stages, chunks); ++cc) fetch_x(cc);
+            uint32_t late = 0;               // buffers whose X tile had not landed when its wait ran out
             for (uint32_t c = 0; c < chunks; ++c) {
                 const uint32_t s = c % stages, use = c / stages;
+                // refill the buffer of the previous chunk as soon as its MMAs are through
+                if (c >= 1 && c - 1 + stages < chunks) {
+                    const uint32_t sp = (c - 1) % stages;
+                    if (!tc_wait(bar_empty + 8 * sp, ((c - 1) / stages) & 1u)) *lost_flag = 1;
+                    fetch_x(c - 1 + stages);
+                }
                 if (!tc_wait(bar_full + 8 * s, use & 1u)) *lost_flag = 1;
+                if (!tc_wait(bar_xin + 8 * s, use & 1u)) { *lost_flag = 1; late |= 1u << s; }
+                else late &= ~(1u << s);
                 asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
                 // descriptors differ from MMA to MMA only in the 14-bit start-address field (low word)
                 const uint32_t base = sb + ring + s * (uint32_t)tc_tile_bytes();
@@ -1006,58 +1067,15 @@ __global__ void __launch_bounds__((kTcDecodeWarps + 1) * 32) hac_gemm_tc_kernel(
                 tc_commit(bar_empty + 8 * s);
             }
             tc_commit(bar_done);
+            // a copy that was late must not outlive the block: give it one more bounded wait
+            for (uint32_t s = 0; s < stages; ++s)
+                if (late & (1u << s)) (void)tc_wait(bar_xin + 8 * s, ((chunks - 1 - ((chunks - 1 - s) % stages)) / stages) & 1u);
         }
         __syncwarp();                        // the other lanes sleep here until the last MMA is issued
     } else {
         // ---- decode + staging ----
         uint4* stage = reinterpret_cast<uint4*>(p) + (size_t)warp * 2 * f.max_unit_chunks;
         const uint32_t stage_a = smem_off(stage);
-        // staging role: two (K group q, input b) pairs per thread; everything that does not change
-        // from chunk to chunk (tile offset, row offsets inside a segment, column pointer) is set up once
-        uint32_t x_at[2], row_off[2][4];
-        const float* x_col[2];
-        bool b_ok[2];
-        float xr[2][4];
-#pragma unroll
-        for (int i = 0; i < 2; ++i) {
-            const uint32_t pi = threadIdx.x + i * (kTcDecodeWarps * 32);
-            const uint32_t q = pi / kTcBatch, b = pi % kTcBatch;
-            x_at[i] = (q >> 1) * kTcXKst + (q & 1u) * kTcXLbo + (b >> 3) * kTcSbo + (b & 7u) * 16;
-#pragma unroll
-            for (int e = 0; e < 4; ++e) row_off[i][e] = (2 * q + (e >> 1)) * f.S + (e & 1);
-            b_ok[i] = b0 + b < batch;
-            x_col[i] = x + (int64_t)(b0 + b) * xs_b;
-        }
-        const int32_t xs_i32 = (int32_t)xs_i;                   // used only when x_small (offsets fit 31 bits)
-        auto load_x = [&](uint32_t g, uint32_t s0) {
-            const uint32_t row_base = g * 32 * f.S + s0;
-            // interior chunk: every row of the tile exists (rows run up to row_base + 31*S + 1)
-            const bool interior = s0 + 1 < f.S && row_base + 31u * f.S + 1u < f.n;
-            if (interior && x_small) {
-                const int32_t base_off = (int32_t)row_base * xs_i32;
-#pragma unroll
-                for (int i = 0; i < 2; ++i) {
-#pragma unroll
-                    for (int e = 0; e < 4; ++e) {
-                        const int32_t off = base_off + (int32_t)row_off[i][e] * xs_i32;
-                        xr[i][e] = b_ok[i] ? __ldg(x_col[i] + off) : 0.0f;
-                    }
-                }
-            } else {
-                const bool second = s0 + 1 < f.S;              // the chunk's second symbol exists
-#pragma unroll
-                for (int i = 0; i < 2; ++i) {
-#pragma unroll
-                    for (int e = 0; e < 4; ++e) {
-                        const uint32_t row = row_base + row_off[i][e];
-                        float v = 0.0f;
-                        if (b_ok[i] && row < f.n && ((e & 1) == 0 || second)) v = __ldg(x_col[i] + (int64_t)row * xs_i);
-                        xr[i][e] = v;
-                    }
-                }
-            }
-        };
-        if (g_begin < g_end) load_x(g_begin, 0);
         const uint32_t wq = lane >> 1;
         const uint32_t l1_abs = sb + dec.l1_lane;
         uint32_t c = 0;
@@ -1135,23 +1153,9 @@ __global__ void __launch_bounds__((kTcDecodeWarps + 1) * 32) hac_gemm_tc_kernel(
                     sts64(tile + kWHi + w_at[ch], hi[ch][0], hi[ch][1]);
                     sts64(tile + kWLo + w_at[ch], lo[ch][0], lo[ch][1]);
                 }
-#pragma unroll
-                for (int i = 0; i < 2; ++i) {
-                    float xh[4], xl[4];
-#pragma unroll
-                    for (int e = 0; e < 4; ++e) {
-                        xh[e] = __uint_as_float(to_tf32(xr[i][e]));
-                        xl[e] = __uint_as_float(to_tf32(xr[i][e] - xh[e]));
-                    }
-                    sts128(tile + kXHi + x_at[i], xh[0], xh[1], xh[2], xh[3]);
-                    sts128(tile + kXLo + x_at[i], xl[0], xl[1], xl[2], xl[3]);
-                }
                 asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
                 __syncwarp();
                 if (lane == 0) asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar_full + 8 * s) : "memory");
-                // the next chunk's rows of X are requested now and land while it is being decoded
-                if (s0 + kTcSteps < seg_rows) load_x(g, s0 + kTcSteps);
-                else if (g + 1 < g_end) load_x(g + 1, 0);
             }
         }
     }
@@ -1397,11 +1401,24 @@ static int attach(Format& f, void* dev_buf, size_t dev_bytes) {
     return HAC_OK;
 }
 
-static size_t workspace_bytes(const Format& f, int64_t batch) {
+static size_t partial_bytes(const Format& f, int64_t batch) {
     // sHAC with one input handles up to two segments of a column in one warp; the batched kernels
     // and HAC keep one partial per segment
     const bool partials = f.sparse ? f.max_units_per_col > (batch == 1 ? 2u : 1u) : f.G > 1;
     return partials ? f.seg_bit_off.size() * (size_t)batch * 4 : 0;
+}
+
+// Batched HAC: the A tiles of the tensor-core kernel (see hac_pack_x_kernel).
+static size_t xpack_bytes(const Format& f, int64_t batch) {
+    if (f.sparse || batch <= 1 || f.symbols == 0) return 0;
+    const size_t cps = (f.S + kTcSteps - 1) / kTcSteps, tiles = (size_t)((batch + kTcBatch - 1) / kTcBatch) * f.G * cps;
+    return tiles * kTcXTileBytes;
+}
+
+// Workspace of one product: [partial sums, rounded up to 256 bytes][A tiles].
+static size_t workspace_bytes(const Format& f, int64_t batch) {
+    const size_t xp = xpack_bytes(f, batch);
+    return xp ? ((partial_bytes(f, batch) + 255) & ~(size_t)255) + xp : partial_bytes(f, batch);
 }
 
 static int env_int(const char* name, int fallback) {
@@ -1530,13 +1547,13 @@ static uint32_t gemm_row_splits(const Format& f, int64_t batch, int sms) {
 // Batched HAC product: one block per (32 columns, row split, 64 inputs).
 static int launch_gemm_tc(const Format& f, const DeviceInfo& di, const DevFormat& d, const float* x, int64_t xs_i,
                           int64_t xs_b, int64_t batch, float* y, int64_t ys_j, int64_t ys_b, float* partial,
-                          cudaStream_t st, uint32_t* row_splits_out) {
+                          unsigned char* xpack, cudaStream_t st, uint32_t* row_splits_out) {
     const size_t budget = (size_t)di.max_smem_optin;
     // two tile buffers when they fit next to a level-1 table with at least 8 replicas, else one
     const size_t spans = (size_t)kTcDecodeWarps * 2 * d.max_unit_chunks * 16;
     uint32_t stages = 2;
-    if (48 + 128 + 2 * tc_tile_bytes() + spans + plan_smem_bytes(d.l1_bits, 3, d.sub_bytes) > budget) stages = 1;
-    const size_t fixed = 48 + 128 + stages * tc_tile_bytes() + spans;
+    if (64 + 128 + 2 * tc_tile_bytes() + spans + plan_smem_bytes(d.l1_bits, 3, d.sub_bytes) > budget) stages = 1;
+    const size_t fixed = 64 + 128 + stages * tc_tile_bytes() + spans;
     if (fixed + plan_smem_bytes(d.l1_bits, 0, d.sub_bytes) > budget) return HAC_ERR_BUFFER_TOO_SMALL;
     const TablePlan tp = plan_tables(d, budget - fixed);
     const size_t smem = fixed + plan_smem_bytes(d.l1_bits, tp.repl_log2, d.sub_bytes);
@@ -1547,10 +1564,14 @@ static int launch_gemm_tc(const Format& f, const DeviceInfo& di, const DevFormat
     const uint32_t rs = gemm_row_splits(f, batch, di.sms);
     const uint64_t grid = (uint64_t)col_blocks * rs * batch_tiles;
     if (grid > 0x7fffffffull) return HAC_ERR_OFFSET_OVERFLOW;
-    // row offsets into x fit 31 bits: the kernel may use 32-bit offsets from the column pointer
-    const uint32_t x_small = (xs_i >= 0 && (uint64_t)xs_i * (uint64_t)(f.n + 1) < ((uint64_t)1 << 31)) ? 1u : 0u;
+    const uint32_t cps = (d.S + kTcSteps - 1) / kTcSteps;
+    const uint64_t pack_blocks = (uint64_t)batch_tiles * d.G * cps * 4;
+    if (pack_blocks > 0x7fffffffull) return HAC_ERR_OFFSET_OVERFLOW;
+    hac_pack_x_kernel<<<(unsigned)pack_blocks, 256, 0, st>>>(d, x, xs_i, xs_b, (uint32_t)batch, xpack, cps);
+    HAC_CUDA(cudaGetLastError());
+    f.last_launches++;
     hac_gemm_tc_kernel<<<(unsigned)grid, (kTcDecodeWarps + 1) * 32, smem, st>>>(
-        d, tp, x, xs_i, xs_b, (uint32_t)batch, y, ys_j, ys_b, partial, col_blocks, rs, stages, x_small);
+        d, tp, xpack, (uint32_t)batch, y, ys_j, ys_b, partial, col_blocks, rs, stages);
     HAC_CUDA(cudaGetLastError());
     f.last_launches++;
     *row_splits_out = rs;
@@ -1592,6 +1613,7 @@ static int dot(const Format& f, const float* x, int64_t batch, int64_t xs_i, int
     if (!x || !y || batch < 1 || batch > ((int64_t)1 << 24)) return HAC_ERR_INVALID_ARG;
     const size_t need = workspace_bytes(f, batch);
     if (need > 0 && (!workspace || workspace_bytes_given < need)) return HAC_ERR_BUFFER_TOO_SMALL;
+    if (need > 0 && (reinterpret_cast<uintptr_t>(workspace) & 15u)) return HAC_ERR_INVALID_ARG;
     cudaStream_t st = static_cast<cudaStream_t>(stream_);
     f.last_launches = 0;
     float* partial = static_cast<float*>(workspace);
@@ -1607,7 +1629,8 @@ static int dot(const Format& f, const float* x, int64_t batch, int64_t xs_i, int
             rc = device_info(di);
             if (rc) return rc;
             if (!f.sparse) {
-                rc = launch_gemm_tc(f, di, d, x, xs_i, xs_b, batch, y, ys_j, ys_b, partial, st, &gemm_splits);
+                unsigned char* xpack = static_cast<unsigned char*>(workspace) + ((partial_bytes(f, batch) + 255) & ~(size_t)255);
+                rc = launch_gemm_tc(f, di, d, x, xs_i, xs_b, batch, y, ys_j, ys_b, partial, xpack, st, &gemm_splits);
             } else {
                 const int acc = (int)std::min<int64_t>(kAccMax, (batch + 31) / 32);
                 switch (acc) {
@@ -1710,7 +1733,7 @@ static int dot_noalloc(const Format& f, const float* x, int64_t batch, int64_t x
     const size_t need = workspace_bytes(f, batch);
     if (need > (size_t)HAC_NOALLOC_SCRATCH_BYTES) {
         g_last_cuda_error = "hac_dot_noalloc: this product needs " + std::to_string(need) +
-                            " bytes of partial sums, the built-in buffer holds " +
+                            " bytes of workspace, the built-in buffer holds " +
                             std::to_string((size_t)HAC_NOALLOC_SCRATCH_BYTES);
         return HAC_ERR_BUFFER_TOO_SMALL;
     }
