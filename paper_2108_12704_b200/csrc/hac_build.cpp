@@ -482,12 +482,19 @@ int build_impl(const float* W, int64_t n, int64_t m, int64_t ldw, const hac_buil
     // per-segment statistics used to size shared memory and to pick the reduction path
     const size_t U = f.seg_bit_off.size();
     f.max_unit_chunks = 1;
+    f.max_sub_chunks = 1;
     for (size_t u = 0; u < U; ++u) {
         uint64_t bits = 0;
         for (int l = 0; l < 32; ++l) bits += f.sub_bits[u * 32 + l];
         const uint64_t first_chunk = f.seg_bit_off[u] >> 7;
         const uint64_t last_word = ((f.seg_bit_off[u] + bits) >> 5) + 2;
         f.max_unit_chunks = std::max<uint32_t>(f.max_unit_chunks, (uint32_t)((last_word >> 2) - first_chunk + 1));
+        uint64_t at = f.seg_bit_off[u];
+        for (int l = 0; l < 32; ++l) {
+            const uint64_t sub_last_word = ((at + f.sub_bits[u * 32 + l]) >> 5) + 2;
+            f.max_sub_chunks = std::max<uint32_t>(f.max_sub_chunks, (uint32_t)((sub_last_word >> 2) - (at >> 7) + 1));
+            at += f.sub_bits[u * 32 + l];
+        }
     }
     if (sparse) {
         // device-only work list: an item is one or two consecutive segments of one column

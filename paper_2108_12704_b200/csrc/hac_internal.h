@@ -94,6 +94,7 @@ struct Format {
     std::vector<uint32_t> seg_first, seg_col;
     std::vector<uint32_t> item_info;          // sHAC, device only: 12 words per work item (see ShacItem)
     uint32_t max_unit_chunks = 0;             // largest 16-byte span a segment's stream covers
+    uint32_t max_sub_chunks = 0;              // same for a single sub-segment
     uint32_t max_units_per_col = 0;
     bool has_empty_col = false;
     // derived

@@ -54,7 +54,7 @@ struct DevFormat {
     const void* ri;
     const uint32_t* cb;
     const void* unit_info;
-    uint32_t n, m, units, G, S, k_eff, lut_bits, max_len, ri_bits, max_unit_chunks, l1_bits, sub_bytes, items;
+    uint32_t n, m, units, G, S, k_eff, lut_bits, max_len, ri_bits, max_unit_chunks, max_sub_chunks, l1_bits, sub_bytes, items;
 };
 
 
@@ -844,21 +844,24 @@ __global__ void finalize_kernel(DevFormat f, bool sparse, const float* __restric
 
 // ------------------------------------------------------------------------------------------------
 // HAC, batch of inputs (Algorithm 3 without re-decoding W per input), on the 5th-generation tensor
-// cores (tcgen05) with the accumulators in tensor memory.
+// cores (tcgen05): Y^T[columns][inputs] = W^T X^T, with W^T as the A operand in tensor memory, X as
+// the B operand in shared memory and the accumulators in tensor memory.
 //
-// A block owns 32 consecutive columns of W, a range of segment indices g (all of them unless the
-// grid would be too small) and a tile of 64 inputs.  Work proceeds in chunks of 64 rows: every lane
-// decodes two symbols of each of its two sub-segments, and the 64 matching rows of X are fetched.
-// Both operands are read by the tensor core straight from shared memory in TF32 ("K-major", no
-// swizzle): a group of four consecutive K elements of one row is a 16-byte unit, 8 rows form a
-// 128-byte core matrix, core matrices of successive 8-row groups are kTcSbo bytes apart, the two K
-// halves of an MMA are LBO bytes apart.  Strides are padded so that the stores of the decode phase
-// hit distinct banks.
-// Split precision: every weight and every input is written as hi + lo, both rounded to TF32.  The
-// hi and lo parts are stacked along M (inputs) and N (columns), so one MMA
-// D[128][64] += [x_hi; x_lo][128][8] * [w_hi; w_lo][64][8]^T forms all four partial products; the
-// epilogue adds the four quadrants in fp32.  The error stays near 1e-7 of sum |w x|, well inside the
-// output tolerance.  Accumulator row r sits in tensor-memory lane r.
+// A block owns 128 consecutive columns of W (one per tensor-memory lane), a range of sub-segments
+// ("tasks": S consecutive rows of every column) and a tile of 64 inputs.  A decode warp serves one
+// quarter of the lanes: lane l of the warp decodes column 32q + l, all lanes walking the same rows,
+// so the symbols a lane decodes one after the other are consecutive K elements of its own
+// accumulator row: they go from registers to tensor memory (tcgen05.st) without a transpose and
+// without passing through shared memory.  Four warps ("slots") per quarter work on four different
+// tasks at a time; each slot has a ring of stages of 16 rows in tensor memory.
+// Split precision: every weight and every input is written as hi + lo, both rounded to TF32, and
+//   D[128][0:64]   += w_hi * x_hi^T + w_lo * x_hi^T        D[128][64:128] += w_hi * x_lo^T
+// with one MMA of N = 128 (B = x_hi stacked on x_lo) and one of N = 64 per 8 rows; the epilogue adds
+// the two halves in fp32.  The error stays near 1e-7 of sum |w x|, well inside the output tolerance.
+// X is split and tiled once per product by hac_pack_x_kernel, exactly as the tensor core reads it
+// ("K-major", no swizzle: four consecutive K elements of one row form a 16-byte unit, 8 rows a
+// 128-byte core matrix, successive 8-row groups are kGSbo bytes apart, the two K halves of an MMA
+// kGXLbo bytes apart), and comes in with one bulk copy per 16 rows.
 // The stream is decoded once per batch tile and never written to global memory.
 // ------------------------------------------------------------------------------------------------
 constexpr int kBatchSteps = 4;          // sHAC batched kernel: entries decoded per lane per phase
@@ -870,47 +873,35 @@ __device__ __forceinline__ uint32_t to_tf32(float v) {
     asm("cvt.rna.tf32.f32 %0, %1;" : "=r"(r) : "f"(v));
     return r;
 }
-__device__ __forceinline__ void sts64(uint32_t addr, float a, float b) {
-    asm volatile("st.shared.v2.f32 [%0], {%1, %2};" ::"r"(addr), "f"(a), "f"(b) : "memory");
-}
-__device__ __forceinline__ void sts128(uint32_t addr, float a, float b, float c, float d) {
-    asm volatile("st.shared.v4.f32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "f"(a), "f"(b), "f"(c), "f"(d) : "memory");
-}
 
-constexpr int kTcSteps = 2;                         // symbols decoded per lane per chunk
-constexpr int kTcRows = 32 * kTcSteps;              // K per chunk (64)
-constexpr int kTcKSteps = kTcRows / 8;              // MMAs (of K = 8) per chunk and product
-constexpr int kTcSbo = 128;
-// One MMA per 8 rows covers all split products: A stacks x_hi (rows 0-63) on x_lo (rows 64-127),
-// B stacks w_hi (rows 0-31) on w_lo (rows 32-63); D[128][64] then holds x_hi*w_hi, x_hi*w_lo,
-// x_lo*w_hi and x_lo*w_lo in its four quadrants, which the epilogue adds.
-constexpr int kTcXLbo = 2048, kTcXKst = 4096;       // A tile: 128 rows -> 16 core matrices per K half
-constexpr int kTcXLoRows = 8 * kTcSbo;              // byte offset of the x_lo rows inside a K half
-constexpr int kTcWLbo = 1040, kTcWKst = 2080;       // B tile: 64 rows -> 8 core matrices, padded
-constexpr int kTcWLoRows = 4 * kTcSbo;              // byte offset of the w_lo rows
-constexpr uint32_t kTcXTileBytes = kTcKSteps * kTcXKst;   // one A tile (x_hi and x_lo of 64 rows x 64 inputs)
-static_assert(kTcSteps == 2, "the A tile layout pairs two lanes x two symbols per 16-byte unit");
-constexpr int kTcCols = 32, kTcBatch = 64, kTcDecodeWarps = 16;
+constexpr int kGCols = 128;                         // columns of W per block = accumulator rows
+constexpr int kGBatch = 64;                         // inputs per batch tile
+constexpr int kGRows = 16;                          // rows of W per tensor-memory stage (two k-steps of 8)
+constexpr int kGSlots = 4;                          // decode warps per quarter of the lanes
+constexpr int kGStages = 3;                         // stages per slot
+constexpr int kGDecodeWarps = 4 * kGSlots;
+constexpr uint32_t kGDCols = 2 * kGBatch;           // accumulator columns: x_hi products | x_lo products
+constexpr uint32_t kGACols = 2 * kGRows;            // columns of a stage: w_hi | w_lo
+constexpr uint32_t kGTmemCols = 512;
+static_assert(kGDCols + kGSlots * kGStages * kGACols <= kGTmemCols, "tensor memory holds D and every stage");
+constexpr int kGSbo = 128, kGXLbo = 2048, kGXKst = 4096;   // B tile: 128 rows (x_hi of 64 inputs, then x_lo)
+constexpr uint32_t kGXLoRows = 8 * kGSbo;           // byte offset of the x_lo rows inside a K half
+constexpr uint32_t kGXTileBytes = (kGRows / 8) * kGXKst;
+constexpr int kGXStagesMax = 8;
+constexpr uint32_t kGMaxSplits = 8;                 // row splits of a product (sizes the partial sums)
 constexpr uint32_t kTcWaitTries = 400000;
 
-__host__ __device__ inline size_t tc_tile_bytes() {
-    return (size_t)kTcKSteps * kTcXKst + (size_t)kTcKSteps * kTcWKst;
-}
+// shared-memory operand descriptor: K-major, no swizzle
 __device__ __forceinline__ uint64_t tc_desc(uint32_t shared_addr, uint32_t lbo_bytes) {
     return (uint64_t)((shared_addr >> 4) & 0x3fffu) | ((uint64_t)((lbo_bytes >> 4) & 0x3fffu) << 16) |
-           ((uint64_t)((kTcSbo >> 4) & 0x3fffu) << 32) | ((uint64_t)1 << 46);
+           ((uint64_t)((kGSbo >> 4) & 0x3fffu) << 32) | ((uint64_t)1 << 46);
 }
-__device__ __forceinline__ void tc_mma(uint32_t tmem, uint64_t a, uint64_t b, uint32_t idesc, uint32_t accumulate) {
+// D (tensor memory) (+)= A (tensor memory: lane = row, one column per K element) * B (shared memory)^T
+__device__ __forceinline__ void tc_mma_ts(uint32_t d_tmem, uint32_t a_tmem, uint64_t b, uint32_t idesc, uint32_t accumulate) {
     asm volatile(
         "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
-        "tcgen05.mma.cta_group::1.kind::tf32 [%0], %1, %2, %3, p;\n\t}"
-        ::"r"(tmem), "l"(a), "l"(b), "r"(idesc), "r"(accumulate) : "memory");
-}
-__device__ __forceinline__ void tc_mma_acc(uint32_t tmem, uint64_t a, uint64_t b, uint32_t idesc) {   // D += A * B
-    asm volatile(
-        "{\n\t.reg .pred p;\n\tsetp.eq.b32 p, 0, 0;\n\t"
-        "tcgen05.mma.cta_group::1.kind::tf32 [%0], %1, %2, %3, p;\n\t}"
-        ::"r"(tmem), "l"(a), "l"(b), "r"(idesc) : "memory");
+        "tcgen05.mma.cta_group::1.kind::tf32 [%0], [%1], %2, %3, p;\n\t}"
+        ::"r"(d_tmem), "r"(a_tmem), "l"(b), "r"(idesc), "r"(accumulate) : "memory");
 }
 __device__ __forceinline__ void tc_commit(uint32_t mbar) {
     asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(mbar) : "memory");
@@ -936,273 +927,286 @@ __device__ __forceinline__ void tmem_ld32(uint32_t (&r)[32], uint32_t taddr) {
           "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
         : "r"(taddr) : "memory");
 }
+// 16 consecutive columns of this thread's tensor-memory lane.
+__device__ __forceinline__ void tmem_st16(uint32_t taddr, const uint32_t (&v)[16]) {
+    asm volatile(
+        "tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16};"
+        ::"r"(taddr), "r"(v[0]), "r"(v[1]), "r"(v[2]), "r"(v[3]), "r"(v[4]), "r"(v[5]), "r"(v[6]), "r"(v[7]),
+          "r"(v[8]), "r"(v[9]), "r"(v[10]), "r"(v[11]), "r"(v[12]), "r"(v[13]), "r"(v[14]), "r"(v[15]) : "memory");
+}
+__device__ __forceinline__ void cp_async16(uint32_t dst, const void* src) {
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst), "l"(src) : "memory");
+}
 
-// A tiles of hac_gemm_tc_kernel, made once per product: for every (batch tile, segment g, chunk)
-// the 64 rows the chunk multiplies (row of K index 2*lane + step = g*32*S + lane*S + s0 + step) of
-// 64 inputs, split into TF32 hi and lo parts and stored exactly as the tile sits in shared memory,
-// so that the product kernel brings a tile in with a single bulk copy.  Rows past the matrix and
-// inputs past the batch are zero.  Tile ((bt*G + g)*cps + chunk) starts at that index times
-// kTcXTileBytes.  Four blocks of 256 threads per tile, one 16-byte unit of each part per thread.
+// B tiles of hac_gemm_tc_kernel, made once per product: tile ((bt*T + task)*cpt + chunk), T tasks
+// per column and cpt chunks of 16 rows per task, holds rows task*S + 16*chunk .. +15 of the 64
+// inputs of batch tile bt, split into TF32 hi and lo parts and stored exactly as the tile sits in
+// shared memory.  Rows past the task or the matrix and inputs past the batch are zero.
+// One block of 256 threads per tile, one 16-byte unit of each part per thread.
 __global__ void __launch_bounds__(256) hac_pack_x_kernel(DevFormat f, const float* __restrict__ x, int64_t xs_i,
                                                          int64_t xs_b, uint32_t batch, unsigned char* __restrict__ xpack,
-                                                         uint32_t cps) {
-    const uint32_t tile = blockIdx.x >> 2;
-    const uint32_t ci = tile % cps, g = (tile / cps) % f.G, bt = tile / (cps * f.G);
-    const uint32_t s0 = ci * kTcSteps;
-    const uint32_t seg_rows = min(f.S, f.n - min(f.n, g * 32 * f.S));
-    if (s0 >= seg_rows) return;                       // no chunk here (last segment of a ragged matrix)
-    const uint32_t pi = (blockIdx.x & 3u) * 256 + threadIdx.x;
-    const uint32_t q = pi / kTcBatch, b = pi % kTcBatch;
-    const bool b_ok = bt * kTcBatch + b < batch;
-    const float* xc = x + (int64_t)(bt * kTcBatch + b) * xs_b;
+                                                         uint32_t tasks, uint32_t cpt) {
+    const uint32_t tile = blockIdx.x;
+    const uint32_t ci = tile % cpt, task = (tile / cpt) % tasks, bt = tile / (cpt * tasks);
+    const uint64_t r0 = (uint64_t)task * f.S;
+    const uint32_t cnt = (uint32_t)min((uint64_t)f.S, (uint64_t)f.n - r0);
+    if (ci * kGRows >= cnt) return;                   // no such chunk (last task of a ragged matrix)
+    const uint32_t b = threadIdx.x % kGBatch, kg = threadIdx.x / kGBatch;      // K group of 4 rows
+    const bool b_ok = bt * kGBatch + b < batch;
+    const float* xc = x + (int64_t)(bt * kGBatch + b) * xs_b;
     float hi[4], lo[4];
 #pragma unroll
     for (int e = 0; e < 4; ++e) {
-        const uint32_t step = e & 1, sub = 2 * q + (e >> 1);
-        const uint64_t row = (uint64_t)g * 32 * f.S + (uint64_t)sub * f.S + s0 + step;
+        const uint32_t in_task = ci * kGRows + kg * 4 + e;
         float v = 0.0f;
-        if (b_ok && s0 + step < f.S && row < f.n) v = __ldg(xc + (int64_t)row * xs_i);
+        if (b_ok && in_task < cnt) v = __ldg(xc + (int64_t)(r0 + in_task) * xs_i);
         hi[e] = __uint_as_float(to_tf32(v));
         lo[e] = __uint_as_float(to_tf32(v - hi[e]));
     }
-    unsigned char* at = xpack + (size_t)tile * kTcXTileBytes + (q >> 1) * kTcXKst + (q & 1u) * kTcXLbo +
-                        (b >> 3) * kTcSbo + (b & 7u) * 16;
+    unsigned char* at = xpack + (size_t)tile * kGXTileBytes + (kg >> 1) * kGXKst + (kg & 1u) * kGXLbo +
+                        (b >> 3) * kGSbo + (b & 7u) * 16;
     *reinterpret_cast<float4*>(at) = make_float4(hi[0], hi[1], hi[2], hi[3]);
-    *reinterpret_cast<float4*>(at + kTcXLoRows) = make_float4(lo[0], lo[1], lo[2], lo[3]);
+    *reinterpret_cast<float4*>(at + kGXLoRows) = make_float4(lo[0], lo[1], lo[2], lo[3]);
 }
 
-// Warp-specialised and pipelined: warps 0..15 decode (two columns each, two chains per lane) and
-// write the W tiles; one lane of warp 16 fetches the X tiles, which hac_pack_x_kernel has already
-// split and laid out as the tensor core reads them, with one bulk copy each, and issues the MMAs.
-// Tiles live in a ring of `stages` buffers with three mbarriers each: `full` (16 arrivals, one per
-// decode warp, after its stores), `xin` (the bytes of the bulk copy) and `empty` (arrival by
-// tcgen05.commit once the MMAs that read the buffer have finished).  There is no block-wide barrier
-// inside the loop, so a slow code word delays only its own warp.
+// Warps 0..15 decode: warp w serves lane quarter q = w % 4 (columns 32q..32q+31 of the block) as
+// slot w / 4, taking every fourth task of the block.  A lane copies the stream bytes of its own
+// sub-segment to a private shared-memory buffer (cp.async, the next task's while the current one is
+// being decoded), decodes 16 symbols, splits them and stores them to its tensor-memory lane.
+// One lane of warp 16 fetches the X tiles (ring of `xstages` buffers, one bulk copy each) and issues
+// the MMAs in task order.  mbarriers: per slot and stage `full` (4 arrivals: one per quarter's warp,
+// after its tensor-memory stores) and `empty` (tcgen05.commit once the MMAs that read the stage have
+// finished); per X buffer `xin` (bytes of the bulk copy) and `xempty` (commit).
 // Every wait is bounded; if one runs out the block marks its outputs NaN and still terminates.
-__global__ void __launch_bounds__((kTcDecodeWarps + 1) * 32, 1) hac_gemm_tc_kernel(
-    DevFormat f, TablePlan tp, const unsigned char* __restrict__ xpack, uint32_t batch,
-    float* __restrict__ y, int64_t ys_j, int64_t ys_b, float* __restrict__ partial, uint32_t col_blocks,
-    uint32_t row_splits, uint32_t stages) {
+__global__ void __launch_bounds__((kGDecodeWarps + 1) * 32, 1) hac_gemm_tc_kernel(
+    DevFormat f, TablePlan tp, const unsigned char* __restrict__ xpack, uint32_t batch, float* __restrict__ y,
+    int64_t ys_j, int64_t ys_b, float* __restrict__ partial, uint32_t col_blocks, uint32_t row_splits,
+    uint32_t xstages, uint32_t slot_bytes, uint32_t nbuf) {
     const uint32_t warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const uint32_t cblk = blockIdx.x % col_blocks;
     const uint32_t rest = blockIdx.x / col_blocks;
     const uint32_t rs = rest % row_splits, bt = rest / row_splits;
-    const uint32_t g_begin = (uint32_t)(((uint64_t)f.G * rs) / row_splits);
-    const uint32_t g_end = (uint32_t)(((uint64_t)f.G * (rs + 1)) / row_splits);
-    const uint32_t b0 = bt * kTcBatch;
+    const uint32_t tasks = (uint32_t)(((uint64_t)f.n + f.S - 1) / f.S);          // sub-segments of a column
+    const uint32_t t_begin = (uint32_t)(((uint64_t)tasks * rs) / row_splits);
+    const uint32_t t_end = (uint32_t)(((uint64_t)tasks * (rs + 1)) / row_splits);
+    const uint32_t ntl = t_end - t_begin;
+    const uint32_t cpt = (f.S + kGRows - 1) / kGRows;                           // chunks of 16 rows per task
+    // every task but the matrix's last has S rows, so chunk c of the block is chunk c % cpt of task c / cpt
+    uint32_t chunks = ntl * cpt;
+    if (ntl > 0 && t_end == tasks) chunks -= cpt - ((f.n - (tasks - 1) * f.S) + kGRows - 1) / kGRows;
     const uint32_t sb = shared_base();
-    // chunks of kTcRows rows this block goes through (same count in every warp)
-    uint32_t chunks = 0;
-    for (uint32_t g = g_begin; g < g_end; ++g)
-        chunks += (min(f.S, f.n - min(f.n, g * 32 * f.S)) + kTcSteps - 1) / kTcSteps;
 
-    // shared memory: [mbarriers full[2], empty[2], xin[2], done; tensor-memory address; lost flag] [tables] [tile ring] [spans]
-    unsigned char* p = smem;
-    const uint32_t bar_full = sb, bar_empty = sb + 16, bar_xin = sb + 32, bar_done = sb + 48;
-    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem + 56);
-    volatile uint32_t* lost_flag = reinterpret_cast<volatile uint32_t*>(smem + 60);
-    p += 64;
+    // shared memory: [mbarriers; tensor-memory address; lost flag] [tables] [X ring] [per-lane stream buffers]
+    const uint32_t bar_full = sb, bar_empty = sb + 96, bar_xin = sb + 192, bar_xempty = sb + 256, bar_done = sb + 320;
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem + 328);
+    volatile uint32_t* lost_flag = reinterpret_cast<volatile uint32_t*>(smem + 332);
+    unsigned char* p = smem + 384;
     if (threadIdx.x == 0) {
-        for (uint32_t s = 0; s < 2; ++s) {
-            mbar_init(bar_full + 8 * s, kTcDecodeWarps);
-            mbar_init(bar_empty + 8 * s, 1);
-            mbar_init(bar_xin + 8 * s, 1);
-        }
+        for (uint32_t i = 0; i < kGSlots * kGStages; ++i) { mbar_init(bar_full + 8 * i, 4); mbar_init(bar_empty + 8 * i, 1); }
+        for (uint32_t i = 0; i < kGXStagesMax; ++i) { mbar_init(bar_xin + 8 * i, 1); mbar_init(bar_xempty + 8 * i, 1); }
         mbar_init(bar_done, 1);
         *lost_flag = 0;
     }
     __syncwarp();
-    if (warp == kTcDecodeWarps) {
-        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(sb + 56), "r"(64u) : "memory");
+    if (warp == kGDecodeWarps) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(sb + 328), "r"(kGTmemCols) : "memory");
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
     }
     const Decoder dec = stage_decoder(f, tp, p);
     p = smem + ((smem_off(p) + 127u) & ~127u);
-    const uint32_t ring = smem_off(p);                          // stage s at ring + s * tc_tile_bytes()
-    p += (size_t)stages * tc_tile_bytes();
-    constexpr uint32_t kXHi = 0, kWHi = kTcKSteps * kTcXKst, kWLo = kWHi + kTcWLoRows;
+    const uint32_t xring = smem_off(p);
+    p += (size_t)xstages * kGXTileBytes;
+    const uint32_t spans = smem_off(p);
     asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
     __syncthreads();
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
     const uint32_t tmem = *tmem_slot;
 
-    if (warp == kTcDecodeWarps) {
-        // ---- MMA issue: one lane, chunk after chunk ----
-        if (lane == 0) {
-            // D f32, A and B tf32, both K-major, N = 64 (w_hi | w_lo), M = 128 (x_hi | x_lo)
-            const uint32_t idesc = (1u << 4) | (2u << 7) | (2u << 10) | ((uint32_t)((2 * kTcCols) >> 3) << 17) |
-                                   ((uint32_t)((2 * kTcBatch) >> 4) << 24);
-            // X tiles of this block: consecutive in xpack (every segment but the matrix's last has cps chunks)
-            const uint32_t cps = (f.S + kTcSteps - 1) / kTcSteps;
-            const unsigned char* xt = xpack + ((size_t)bt * f.G + g_begin) * cps * (size_t)kTcXTileBytes;
-            auto fetch_x = [&](uint32_t cc) {
-                const uint32_t s = cc % stages;
-                mbar_expect_tx(bar_xin + 8 * s, kTcXTileBytes);
-                bulk_copy_g2s(sb + ring + s * (uint32_t)tc_tile_bytes() + kXHi, xt + (size_t)cc * kTcXTileBytes,
-                              kTcXTileBytes, bar_xin + 8 * s);
+    if (warp == kGDecodeWarps) {
+        // ---- X tiles in, MMAs out: one lane, chunk after chunk ----
+        if (lane == 0 && chunks > 0) {
+            // D f32, A and B tf32, both K-major, M = 128; N = 128 (x_hi | x_lo) for w_hi, N = 64 (x_hi) for w_lo
+            const uint32_t idesc_base = (1u << 4) | (2u << 7) | (2u << 10) | ((uint32_t)(kGCols >> 4) << 24);
+            const uint32_t idesc_wide = idesc_base | ((uint32_t)((2 * kGBatch) >> 3) << 17);
+            const uint32_t idesc_half = idesc_base | ((uint32_t)(kGBatch >> 3) << 17);
+            const unsigned char* xt = xpack + ((size_t)bt * tasks + t_begin) * cpt * (size_t)kGXTileBytes;
+            auto fetch_x = [&](uint32_t c) {
+                const uint32_t s = c % xstages;
+                mbar_expect_tx(bar_xin + 8 * s, kGXTileBytes);
+                bulk_copy_g2s(sb + xring + s * kGXTileBytes, xt + (size_t)c * kGXTileBytes, kGXTileBytes, bar_xin + 8 * s);
             };
-            for (uint32_t cc = 0; cc < min(stages, chunks); ++cc) fetch_x(cc);
-            uint32_t late = 0;               // buffers whose X tile had not landed when its wait ran out
+            uint32_t pc = 0;                 // next chunk whose X tile is to be fetched
+            for (; pc < min(xstages, chunks); ++pc) fetch_x(pc);
             for (uint32_t c = 0; c < chunks; ++c) {
-                const uint32_t s = c % stages, use = c / stages;
-                // refill the buffer of the previous chunk as soon as its MMAs are through
-                if (c >= 1 && c - 1 + stages < chunks) {
-                    const uint32_t sp = (c - 1) % stages;
-                    if (!tc_wait(bar_empty + 8 * sp, ((c - 1) / stages) & 1u)) *lost_flag = 1;
-                    fetch_x(c - 1 + stages);
-                }
-                if (!tc_wait(bar_full + 8 * s, use & 1u)) *lost_flag = 1;
-                if (!tc_wait(bar_xin + 8 * s, use & 1u)) { *lost_flag = 1; late |= 1u << s; }
-                else late &= ~(1u << s);
+                const uint32_t tl = c / cpt, ci = c - tl * cpt;
+                const uint32_t slot = tl % kGSlots, k = (tl / kGSlots) * cpt + ci;    // k-th chunk of that slot
+                const uint32_t stage = slot * kGStages + k % kGStages, xs = c % xstages;
+                if (!tc_wait(bar_full + 8 * stage, (k / kGStages) & 1u)) *lost_flag = 1;
+                if (!tc_wait(bar_xin + 8 * xs, (c / xstages) & 1u)) *lost_flag = 1;
                 asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-                // descriptors differ from MMA to MMA only in the 14-bit start-address field (low word)
-                const uint32_t base = sb + ring + s * (uint32_t)tc_tile_bytes();
-                const uint64_t a0 = tc_desc(base + kXHi, kTcXLbo), b0d = tc_desc(base + kWHi, kTcWLbo);
+                const uint32_t a_col = tmem + kGDCols + stage * kGACols;
+                const uint64_t b_desc = tc_desc(sb + xring + xs * kGXTileBytes, kGXLbo);
 #pragma unroll
-                for (int ks = 0; ks < kTcKSteps; ++ks) {
-                    const uint64_t a = a0 + (uint64_t)(ks * (kTcXKst >> 4)), b = b0d + (uint64_t)(ks * (kTcWKst >> 4));
-                    if (ks == 0) tc_mma(tmem, a, b, idesc, c == 0 ? 0u : 1u);
-                    else tc_mma_acc(tmem, a, b, idesc);
+                for (int ks = 0; ks < kGRows / 8; ++ks) {
+                    const uint64_t b = b_desc + (uint64_t)(ks * (kGXKst >> 4));
+                    tc_mma_ts(tmem, a_col + ks * 8, b, idesc_wide, (c | (uint32_t)ks) ? 1u : 0u);
+                    tc_mma_ts(tmem, a_col + kGRows + ks * 8, b, idesc_half, 1u);
                 }
-                tc_commit(bar_empty + 8 * s);
+                tc_commit(bar_empty + 8 * stage);
+                tc_commit(bar_xempty + 8 * xs);
+                // the X buffer of the previous chunk is free about now: refill it behind the MMAs just issued
+                if (pc < chunks && pc - xstages + 1 <= c) {
+                    if (!tc_wait(bar_xempty + 8 * (pc % xstages), ((pc / xstages) - 1) & 1u)) *lost_flag = 1;
+                    fetch_x(pc);
+                    ++pc;
+                }
             }
             tc_commit(bar_done);
-            // a copy that was late must not outlive the block: give it one more bounded wait
-            for (uint32_t s = 0; s < stages; ++s)
-                if (late & (1u << s)) (void)tc_wait(bar_xin + 8 * s, ((chunks - 1 - ((chunks - 1 - s) % stages)) / stages) & 1u);
         }
         __syncwarp();                        // the other lanes sleep here until the last MMA is issued
     } else {
-        // ---- decode + staging ----
-        uint4* stage = reinterpret_cast<uint4*>(p) + (size_t)warp * 2 * f.max_unit_chunks;
-        const uint32_t stage_a = smem_off(stage);
-        const uint32_t wq = lane >> 1;
+        // ---- decode -> tensor memory ----
+        const uint32_t q = warp & 3u, slot = warp >> 2;
+        const uint32_t j = cblk * kGCols + q * 32 + lane;
+        const bool valid = j < f.m;
+        const bool all_valid = __all_sync(0xffffffffu, valid);
+        const uint32_t buf_stride = 32 * slot_bytes;
+        const uint32_t my_buf = spans + warp * nbuf * buf_stride + lane * slot_bytes;       // buffer 0 of this lane
         const uint32_t l1_abs = sb + dec.l1_lane;
-        uint32_t c = 0;
-        for (uint32_t g = g_begin; g < g_end; ++g) {
-            FastReader fr[2];
-            uint32_t count[2], w_at[2];
+        const uint32_t a_base = tmem + ((q * 32u) << 16) + kGDCols + slot * kGStages * kGACols;
+        // Starts the copy of this lane's sub-segment of `task` into buffer `buf`; returns the bit
+        // position of the sub-segment's first code word inside the buffer.
+        auto start_copy = [&](uint32_t task, uint32_t buf) -> uint32_t {
+            uint32_t bitpos = 0;
+            if (valid) {
+                const uint32_t g = task >> 5, t = task & 31u;
+                const size_t u = (size_t)j * f.G + g;
+                const uint4* lens = reinterpret_cast<const uint4*>(f.sub_bits + u * 32);
+                uint32_t before = 0, mine = 0;
 #pragma unroll
-            for (int ch = 0; ch < 2; ++ch) {
-                const uint32_t col = 2 * warp + ch, j = cblk * kTcCols + col;
-                w_at[ch] = (wq >> 1) * kTcWKst + (wq & 1u) * kTcWLbo + (col >> 3) * kTcSbo + (col & 7u) * 16 + (lane & 1u) * 8;
-                count[ch] = 0;
-                fr[ch].hi = fr[ch].lo = fr[ch].off = 0; fr[ch].next = sb + stage_a;
-                if (j < f.m) {
-                    const uint32_t u = j * f.G + g;
-                    const uint32_t my_bits = __ldg(f.sub_bits + (size_t)u * 32 + lane);
-                    uint32_t total;
-                    const uint32_t start = lane_start_bits(my_bits, lane, total);
-                    const uint32_t base = stage_span(f, __ldg(f.seg_bit_off + u), total, stage + (size_t)ch * f.max_unit_chunks, lane);
-                    const uint32_t row0 = (g * 32 + lane) * f.S;
-                    count[ch] = row0 < f.n ? min(f.S, f.n - row0) : 0u;
-                    BitReader br;
-                    br.init(stage_a + ch * f.max_unit_chunks * 16, base + start);
-                    fr[ch].hi = br.hi; fr[ch].lo = br.lo; fr[ch].off = br.off; fr[ch].next = sb + br.next;
+                for (int v4 = 0; v4 < 4; ++v4) {
+                    const uint4 v = __ldg(lens + v4);
+                    const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+                    for (int e = 0; e < 4; ++e) {
+                        const uint32_t t0 = (uint32_t)(8 * v4 + 2 * e), lo16 = w[e] & 0xffffu, hi16 = w[e] >> 16;
+                        before += (t0 < t ? lo16 : 0u) + (t0 + 1 < t ? hi16 : 0u);
+                        mine = t0 == t ? lo16 : (t0 + 1 == t ? hi16 : mine);
+                    }
                 }
+                const uint64_t start = __ldg(f.seg_bit_off + u) + before;
+                const uint64_t first_chunk = start >> 7;
+                const uint64_t last_word = ((start + mine) >> 5) + 2;
+                const uint32_t nch = (uint32_t)((last_word >> 2) - first_chunk + 1);
+                const uint4* src = reinterpret_cast<const uint4*>(f.stream) + first_chunk;
+                const uint32_t dst = sb + my_buf + buf * buf_stride;
+                for (uint32_t c = 0; c < nch; ++c) cp_async16(dst + 16 * c, src + c);
+                bitpos = (uint32_t)(start - (first_chunk << 7));
             }
-            const uint32_t seg_rows = min(f.S, f.n - min(f.n, g * 32 * f.S));
-            // symbols every lane of the warp still has in both chains (lets whole chunks skip the per-lane checks)
-            const uint32_t common = __reduce_min_sync(0xffffffffu, min(count[0], count[1]));
-            for (uint32_t s0 = 0; s0 < seg_rows; s0 += kTcSteps, ++c) {
-                float hi[2][kTcSteps], lo[2][kTcSteps];
-                if (s0 + kTcSteps <= common) {
+            asm volatile("cp.async.commit_group;" ::: "memory");
+            return bitpos;
+        };
+        uint32_t buf = 0, bitpos = 0, k = 0;
+        if (slot < ntl) bitpos = start_copy(t_begin + slot, 0);
+        for (uint32_t tl = slot; tl < ntl; tl += kGSlots) {
+            const uint32_t task = t_begin + tl;
+            const bool more = tl + kGSlots < ntl;
+            uint32_t next_bitpos = 0;
+            if (nbuf == 2 && more) {
+                next_bitpos = start_copy(task + kGSlots, buf ^ 1u);
+                asm volatile("cp.async.wait_group 1;" ::: "memory");
+            } else {
+                asm volatile("cp.async.wait_group 0;" ::: "memory");
+            }
+            FastReader fr;
+            fr.hi = fr.lo = fr.off = 0; fr.next = sb + my_buf;
+            if (valid) {
+                BitReader br;
+                br.init(my_buf + buf * buf_stride, bitpos);
+                fr.hi = br.hi; fr.lo = br.lo; fr.off = br.off; fr.next = sb + br.next;
+            }
+            const uint32_t cnt = (uint32_t)min((uint64_t)f.S, (uint64_t)f.n - (uint64_t)task * f.S);
+            for (uint32_t r = 0; r < cnt; r += kGRows, ++k) {
+                uint32_t hi[kGRows], lo[kGRows];
+                if (all_valid && r + kGRows <= cnt) {
 #pragma unroll
-                    for (int st = 0; st < kTcSteps; ++st) {
-                        uint32_t top[2], val[2], len[2];
-#pragma unroll
-                        for (int ch = 0; ch < 2; ++ch) fast_lookup(fr[ch], dec.l1_shift, dec.l1_mul, l1_abs, top[ch], val[ch], len[ch]);
-                        if ((int32_t)(len[0] | len[1]) < 0) {
-#pragma unroll
-                            for (int ch = 0; ch < 2; ++ch)
-                                if ((int32_t)len[ch] < 0) resolve_long(top[ch], dec, f, val[ch], len[ch]);
-                        }
-#pragma unroll
-                        for (int ch = 0; ch < 2; ++ch) {
-                            fast_consume_value(fr[ch], len[ch]);
-                            const float w = __uint_as_float(val[ch]);
-                            hi[ch][st] = __uint_as_float(to_tf32(w));
-                            lo[ch][st] = __uint_as_float(to_tf32(w - hi[ch][st]));
-                        }
+                    for (int s = 0; s < kGRows; ++s) {
+                        uint32_t top, val, len;
+                        fast_lookup(fr, dec.l1_shift, dec.l1_mul, l1_abs, top, val, len);
+                        if ((int32_t)len < 0) resolve_long(top, dec, f, val, len);
+                        fast_consume_value(fr, len);
+                        hi[s] = to_tf32(__uint_as_float(val));
+                        lo[s] = to_tf32(__uint_as_float(val) - __uint_as_float(hi[s]));
                     }
                 } else {
 #pragma unroll
-                    for (int st = 0; st < kTcSteps; ++st) {
-                        uint32_t top[2], val[2], len[2];
-#pragma unroll
-                        for (int ch = 0; ch < 2; ++ch) {
-                            top[ch] = val[ch] = len[ch] = 0;
-                            if (s0 + st < count[ch]) fast_lookup(fr[ch], dec.l1_shift, dec.l1_mul, l1_abs, top[ch], val[ch], len[ch]);
+                    for (int s = 0; s < kGRows; ++s) {
+                        uint32_t top = 0, val = 0, len = 0;
+                        if (valid && r + s < cnt) {
+                            fast_lookup(fr, dec.l1_shift, dec.l1_mul, l1_abs, top, val, len);
+                            if ((int32_t)len < 0) resolve_long(top, dec, f, val, len);
+                            fast_consume_value(fr, len);
                         }
-#pragma unroll
-                        for (int ch = 0; ch < 2; ++ch) {
-                            if ((int32_t)len[ch] < 0) resolve_long(top[ch], dec, f, val[ch], len[ch]);
-                            if (s0 + st < count[ch]) fast_consume_value(fr[ch], len[ch]);
-                            const float w = __uint_as_float(val[ch]);
-                            hi[ch][st] = __uint_as_float(to_tf32(w));
-                            lo[ch][st] = __uint_as_float(to_tf32(w - hi[ch][st]));
-                        }
+                        hi[s] = to_tf32(__uint_as_float(val));
+                        lo[s] = to_tf32(__uint_as_float(val) - __uint_as_float(hi[s]));
                     }
                 }
-                const uint32_t s = c % stages, use = c / stages;
-                // the buffer is free once the MMAs of its previous use have been committed
-                if (use > 0 && !tc_wait(bar_empty + 8 * s, (use - 1) & 1u)) *lost_flag = 1;
-                const uint32_t tile = sb + ring + s * (uint32_t)tc_tile_bytes();
-#pragma unroll
-                for (int ch = 0; ch < 2; ++ch) {
-                    sts64(tile + kWHi + w_at[ch], hi[ch][0], hi[ch][1]);
-                    sts64(tile + kWLo + w_at[ch], lo[ch][0], lo[ch][1]);
+                const uint32_t st = k % kGStages, stage = slot * kGStages + st;
+                // the stage is free once the MMAs of its previous use have been committed (one lane polls)
+                if (k >= kGStages) {
+                    if (lane == 0 && !tc_wait(bar_empty + 8 * stage, ((k / kGStages) - 1) & 1u)) *lost_flag = 1;
+                    __syncwarp();
                 }
-                asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+                asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+                tmem_st16(a_base + st * kGACols, hi);
+                tmem_st16(a_base + st * kGACols + kGRows, lo);
+                asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
+                asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
                 __syncwarp();
-                if (lane == 0) asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar_full + 8 * s) : "memory");
+                if (lane == 0) asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar_full + 8 * stage) : "memory");
             }
+            if (nbuf == 2) { buf ^= 1u; bitpos = next_bitpos; }
+            else if (more) bitpos = start_copy(task + kGSlots, 0);
         }
     }
     // ---- epilogue: accumulators -> y ----
     bool lost = false;
-    if (chunks > 0 && !tc_wait(bar_done, 0)) lost = true;
+    // the MMA-issuing lane alone waits for the last commit; everyone else sleeps in the block barrier below
+    if (chunks > 0 && warp == kGDecodeWarps && lane == 0 && !tc_wait(bar_done, 0)) lost = true;
     const bool any_lost = __syncthreads_or((lost || *lost_flag) ? 1 : 0) != 0;
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-    // Accumulator row r sits in tensor-memory lane r: warps 0,1 hold the x_hi rows of inputs 0..63,
-    // warps 2,3 the x_lo rows; columns 0..31 are the w_hi products, 32..63 the w_lo products.
-    float acc[kTcCols];
-    float* fold = reinterpret_cast<float*>(smem + ring);     // [column][input], the tiles are no longer in use
     if (warp < 4) {
-        if (chunks > 0 && !any_lost) {
+        // lane l of warp q holds column 32q + l: inputs 0..63 in accumulator columns 0..63 (x_hi products)
+        // and 64..127 (x_lo products)
+        const uint32_t j = cblk * kGCols + warp * 32 + lane;
+#pragma unroll 1
+        for (uint32_t half = 0; half < 2; ++half) {
             uint32_t r0[32], r1[32];
-            const uint32_t src = tmem + ((warp * 32u) << 16);
-            tmem_ld32(r0, src);
-            tmem_ld32(r1, src + kTcCols);
-            asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+            if (chunks > 0 && !any_lost) {
+                const uint32_t src = tmem + ((warp * 32u) << 16) + half * 32;
+                tmem_ld32(r0, src);
+                tmem_ld32(r1, src + kGBatch);
+                asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+            } else {
 #pragma unroll
-            for (int cc = 0; cc < kTcCols; ++cc) acc[cc] = __uint_as_float(r1[cc]) + __uint_as_float(r0[cc]);
-        } else {
+                for (int cc = 0; cc < 32; ++cc) { r0[cc] = any_lost ? 0x7fc00000u : 0u; r1[cc] = 0u; }   // NaN marks a lost wait
+            }
+            if (j < f.m) {
 #pragma unroll
-            for (int cc = 0; cc < kTcCols; ++cc) acc[cc] = any_lost ? __uint_as_float(0x7fc00000u) : 0.f;   // NaN marks a lost wait
-        }
-        if (warp >= 2) {
-#pragma unroll
-            for (int cc = 0; cc < kTcCols; ++cc) fold[cc * kTcBatch + (warp - 2) * 32 + lane] = acc[cc];
-        }
-    }
-    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
-    __syncthreads();
-    if (warp < 2) {
-        const uint32_t b = b0 + warp * 32 + lane;
-        if (b < batch) {
-#pragma unroll
-            for (int cc = 0; cc < kTcCols; ++cc) {
-                const uint32_t j = cblk * kTcCols + cc;
-                if (j < f.m) {
-                    const float v = fold[cc * kTcBatch + warp * 32 + lane] + acc[cc];
-                    if (row_splits == 1) y[(int64_t)j * ys_j + (int64_t)b * ys_b] = v;
-                    else partial[((size_t)j * row_splits + rs) * batch + b] = v;
+                for (int cc = 0; cc < 32; ++cc) {
+                    const uint32_t b = bt * kGBatch + half * 32 + cc;
+                    if (b < batch) {
+                        const float v = __uint_as_float(r1[cc]) + __uint_as_float(r0[cc]);
+                        if (row_splits == 1) y[(int64_t)j * ys_j + (int64_t)b * ys_b] = v;
+                        else partial[((size_t)j * row_splits + rs) * batch + b] = v;
+                    }
                 }
             }
         }
     }
-    if (warp == kTcDecodeWarps) asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(64u) : "memory");
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    __syncthreads();
+    if (warp == kGDecodeWarps) asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(kGTmemCols) : "memory");
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -1335,6 +1339,7 @@ static DevFormat dev_format(const Format& f) {
     d.G = f.G ? f.G : 1; d.S = f.S; d.k_eff = (uint32_t)f.codebook.size();
     d.lut_bits = (uint32_t)f.tables.lut_bits; d.max_len = f.max_len; d.ri_bits = f.ri_bits;
     d.max_unit_chunks = f.max_unit_chunks;
+    d.max_sub_chunks = f.max_sub_chunks;
     return d;
 }
 
@@ -1401,21 +1406,29 @@ static int attach(Format& f, void* dev_buf, size_t dev_bytes) {
     return HAC_OK;
 }
 
+// Tasks of the batched HAC kernel: sub-segments (S rows) of a column.
+static uint32_t gemm_tasks(const Format& f) { return f.S ? (uint32_t)((f.n + f.S - 1) / f.S) : 0u; }
+
 static size_t partial_bytes(const Format& f, int64_t batch) {
-    // sHAC with one input handles up to two segments of a column in one warp; the batched kernels
-    // and HAC keep one partial per segment
+    // batched HAC: one partial per row split of the product kernel
+    if (!f.sparse && batch > 1) {
+        const uint32_t t = gemm_tasks(f);
+        return t > 1 ? (size_t)std::min<uint32_t>(t, kGMaxSplits) * (size_t)f.m * (size_t)batch * 4 : 0;
+    }
+    // sHAC with one input handles up to two segments of a column in one warp; the batched sHAC kernel
+    // and HAC with one input keep one partial per segment
     const bool partials = f.sparse ? f.max_units_per_col > (batch == 1 ? 2u : 1u) : f.G > 1;
     return partials ? f.seg_bit_off.size() * (size_t)batch * 4 : 0;
 }
 
-// Batched HAC: the A tiles of the tensor-core kernel (see hac_pack_x_kernel).
+// Batched HAC: the B tiles of the tensor-core kernel (see hac_pack_x_kernel).
 static size_t xpack_bytes(const Format& f, int64_t batch) {
     if (f.sparse || batch <= 1 || f.symbols == 0) return 0;
-    const size_t cps = (f.S + kTcSteps - 1) / kTcSteps, tiles = (size_t)((batch + kTcBatch - 1) / kTcBatch) * f.G * cps;
-    return tiles * kTcXTileBytes;
+    const size_t cpt = (f.S + kGRows - 1) / kGRows;
+    return (size_t)((batch + kGBatch - 1) / kGBatch) * gemm_tasks(f) * cpt * kGXTileBytes;
 }
 
-// Workspace of one product: [partial sums, rounded up to 256 bytes][A tiles].
+// Workspace of one product: [partial sums, rounded up to 256 bytes][B tiles].
 static size_t workspace_bytes(const Format& f, int64_t batch) {
     const size_t xp = xpack_bytes(f, batch);
     return xp ? ((partial_bytes(f, batch) + 255) & ~(size_t)255) + xp : partial_bytes(f, batch);
@@ -1537,41 +1550,53 @@ static int launch_vec(const Format& f, int mode, const float* x, int64_t xs_i, f
 }
 
 // Row splits of the tensor-core HAC kernel: 1 (a block owns whole columns and writes y itself)
-// unless that leaves most of the SMs idle.
+// unless that leaves most of the SMs idle; a split keeps at least one task per decode slot.
 static uint32_t gemm_row_splits(const Format& f, int64_t batch, int sms) {
-    const uint64_t blocks = (uint64_t)((f.m + kTcCols - 1) / kTcCols) * (uint64_t)((batch + kTcBatch - 1) / kTcBatch);
-    if (blocks * 5 >= (uint64_t)sms * 3 || f.G <= 1) return 1;
-    return (uint32_t)std::min<uint64_t>(f.G, std::max<uint64_t>(1, (uint64_t)sms / blocks));
+    const uint64_t blocks = (uint64_t)((f.m + kGCols - 1) / kGCols) * (uint64_t)((batch + kGBatch - 1) / kGBatch);
+    const uint32_t tasks = gemm_tasks(f);
+    if (blocks * 5 >= (uint64_t)sms * 3 || tasks <= 1) return 1;
+    const uint64_t by_sms = std::max<uint64_t>(1, (uint64_t)sms / blocks);
+    const uint64_t by_tasks = std::max<uint32_t>(1, tasks / kGSlots);
+    return (uint32_t)std::min<uint64_t>(std::min<uint64_t>(by_sms, by_tasks), kGMaxSplits);
 }
 
-// Batched HAC product: one block per (32 columns, row split, 64 inputs).
+// Batched HAC product: one block per (128 columns, row split, 64 inputs).
 static int launch_gemm_tc(const Format& f, const DeviceInfo& di, const DevFormat& d, const float* x, int64_t xs_i,
                           int64_t xs_b, int64_t batch, float* y, int64_t ys_j, int64_t ys_b, float* partial,
                           unsigned char* xpack, cudaStream_t st, uint32_t* row_splits_out) {
     const size_t budget = (size_t)di.max_smem_optin;
-    // two tile buffers when they fit next to a level-1 table with at least 8 replicas, else one
-    const size_t spans = (size_t)kTcDecodeWarps * 2 * d.max_unit_chunks * 16;
-    uint32_t stages = 2;
-    if (64 + 128 + 2 * tc_tile_bytes() + spans + plan_smem_bytes(d.l1_bits, 3, d.sub_bytes) > budget) stages = 1;
-    const size_t fixed = 64 + 128 + stages * tc_tile_bytes() + spans;
-    if (fixed + plan_smem_bytes(d.l1_bits, 0, d.sub_bytes) > budget) return HAC_ERR_BUFFER_TOO_SMALL;
+    const uint32_t slot_bytes = d.max_sub_chunks * 16;
+    // shared memory: the deepest X ring and double stream buffers that still leave room for a level-1
+    // table with 8 replicas; failing that, the first combination that fits at all
+    static const uint32_t kChoices[][2] = {{2, 6}, {2, 4}, {1, 6}, {1, 4}, {1, 2}};      // {stream buffers, X buffers}
+    uint32_t nbuf = 0, xstages = 0;
+    size_t fixed = 0;
+    for (uint32_t want_repl : {3u, 0u}) {
+        for (const auto& c : kChoices) {
+            const size_t fx = 384 + 128 + (size_t)c[1] * kGXTileBytes + (size_t)kGDecodeWarps * c[0] * 32 * slot_bytes;
+            if (fx + plan_smem_bytes(d.l1_bits, want_repl, d.sub_bytes) <= budget) { nbuf = c[0]; xstages = c[1]; fixed = fx; break; }
+        }
+        if (nbuf) break;
+    }
+    if (!nbuf) return HAC_ERR_BUFFER_TOO_SMALL;
     const TablePlan tp = plan_tables(d, budget - fixed);
-    const size_t smem = fixed + plan_smem_bytes(d.l1_bits, tp.repl_log2, d.sub_bytes);
+    // the block allocates all of tensor memory: ask for enough shared memory that no second block shares the SM
+    const size_t smem = std::max(fixed + plan_smem_bytes(d.l1_bits, tp.repl_log2, d.sub_bytes), budget / 2 + 1024);
     int rc = prepare_kernel(hac_gemm_tc_kernel, smem);
     if (rc) return rc;
-    const uint32_t col_blocks = (uint32_t)((f.m + kTcCols - 1) / kTcCols);
-    const uint32_t batch_tiles = (uint32_t)((batch + kTcBatch - 1) / kTcBatch);
+    const uint32_t col_blocks = (uint32_t)((f.m + kGCols - 1) / kGCols);
+    const uint32_t batch_tiles = (uint32_t)((batch + kGBatch - 1) / kGBatch);
     const uint32_t rs = gemm_row_splits(f, batch, di.sms);
     const uint64_t grid = (uint64_t)col_blocks * rs * batch_tiles;
     if (grid > 0x7fffffffull) return HAC_ERR_OFFSET_OVERFLOW;
-    const uint32_t cps = (d.S + kTcSteps - 1) / kTcSteps;
-    const uint64_t pack_blocks = (uint64_t)batch_tiles * d.G * cps * 4;
+    const uint32_t tasks = gemm_tasks(f), cpt = (d.S + kGRows - 1) / kGRows;
+    const uint64_t pack_blocks = (uint64_t)batch_tiles * tasks * cpt;
     if (pack_blocks > 0x7fffffffull) return HAC_ERR_OFFSET_OVERFLOW;
-    hac_pack_x_kernel<<<(unsigned)pack_blocks, 256, 0, st>>>(d, x, xs_i, xs_b, (uint32_t)batch, xpack, cps);
+    hac_pack_x_kernel<<<(unsigned)pack_blocks, 256, 0, st>>>(d, x, xs_i, xs_b, (uint32_t)batch, xpack, tasks, cpt);
     HAC_CUDA(cudaGetLastError());
     f.last_launches++;
-    hac_gemm_tc_kernel<<<(unsigned)grid, (kTcDecodeWarps + 1) * 32, smem, st>>>(
-        d, tp, xpack, (uint32_t)batch, y, ys_j, ys_b, partial, col_blocks, rs, stages);
+    hac_gemm_tc_kernel<<<(unsigned)grid, (kGDecodeWarps + 1) * 32, smem, st>>>(
+        d, tp, xpack, (uint32_t)batch, y, ys_j, ys_b, partial, col_blocks, rs, xstages, slot_bytes, nbuf);
     HAC_CUDA(cudaGetLastError());
     f.last_launches++;
     *row_splits_out = rs;
