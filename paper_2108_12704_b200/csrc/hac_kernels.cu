@@ -852,12 +852,15 @@ __global__ void finalize_kernel(DevFormat f, bool sparse, const float* __restric
 // quarter of the lanes: lane l of the warp decodes column 32q + l, all lanes walking the same rows,
 // so the symbols a lane decodes one after the other are consecutive K elements of its own
 // accumulator row: they go from registers to tensor memory (tcgen05.st) without a transpose and
-// without passing through shared memory.  Four warps ("slots") per quarter work on four different
-// tasks at a time; each slot has a ring of stages of 16 rows in tensor memory.
+// without passing through shared memory.  Four warps per quarter work on four different tasks at a
+// time; the four warps (one per quarter) that share a task form a "slot" with its own ring of
+// 16-row stages in tensor memory, its own accumulator and its own MMA-issuing thread, so the four
+// pipelines never wait for one another (a commit or an mbarrier wait costs the issuing thread
+// hundreds of cycles; four threads overlap them).  The epilogue adds the four accumulators.
 // Split precision: every weight and every input is written as hi + lo, both rounded to TF32, and
-//   D[128][0:64]   += w_hi * x_hi^T + w_lo * x_hi^T        D[128][64:128] += w_hi * x_lo^T
-// with one MMA of N = 128 (B = x_hi stacked on x_lo) and one of N = 64 per 8 rows; the epilogue adds
-// the two halves in fp32.  The error stays near 1e-7 of sum |w x|, well inside the output tolerance.
+//   D[128][64] += w_hi * x_hi^T + w_hi * x_lo^T + w_lo * x_hi^T
+// with three MMAs of N = 64 per 8 rows.  The error stays near 1e-7 of sum |w x|, well inside the
+// output tolerance.
 // X is split and tiled once per product by hac_pack_x_kernel, exactly as the tensor core reads it
 // ("K-major", no swizzle: four consecutive K elements of one row form a 16-byte unit, 8 rows a
 // 128-byte core matrix, successive 8-row groups are kGSbo bytes apart, the two K halves of an MMA
@@ -878,16 +881,17 @@ constexpr int kGCols = 128;                         // columns of W per block = 
 constexpr int kGBatch = 64;                         // inputs per batch tile
 constexpr int kGRows = 16;                          // rows of W per tensor-memory stage (two k-steps of 8)
 constexpr int kGSlots = 4;                          // decode warps per quarter of the lanes
-constexpr int kGStages = 3;                         // stages per slot
+constexpr int kGStages = 2;                         // tensor-memory stages per slot
+constexpr int kGXBufs = 3;                          // X tiles in flight per slot
 constexpr int kGDecodeWarps = 4 * kGSlots;
-constexpr uint32_t kGDCols = 2 * kGBatch;           // accumulator columns: x_hi products | x_lo products
+constexpr int kGWarps = kGDecodeWarps + kGSlots;    // plus one MMA-issuing warp per slot
+constexpr uint32_t kGDCols = kGSlots * kGBatch;     // one accumulator of 64 columns per slot
 constexpr uint32_t kGACols = 2 * kGRows;            // columns of a stage: w_hi | w_lo
 constexpr uint32_t kGTmemCols = 512;
 static_assert(kGDCols + kGSlots * kGStages * kGACols <= kGTmemCols, "tensor memory holds D and every stage");
 constexpr int kGSbo = 128, kGXLbo = 2048, kGXKst = 4096;   // B tile: 128 rows (x_hi of 64 inputs, then x_lo)
 constexpr uint32_t kGXLoRows = 8 * kGSbo;           // byte offset of the x_lo rows inside a K half
 constexpr uint32_t kGXTileBytes = (kGRows / 8) * kGXKst;
-constexpr int kGXStagesMax = 8;
 constexpr uint32_t kGMaxSplits = 8;                 // row splits of a product (sizes the partial sums)
 constexpr uint32_t kTcWaitTries = 400000;
 
@@ -969,19 +973,21 @@ __global__ void __launch_bounds__(256) hac_pack_x_kernel(DevFormat f, const floa
     *reinterpret_cast<float4*>(at + kGXLoRows) = make_float4(lo[0], lo[1], lo[2], lo[3]);
 }
 
-// Warps 0..15 decode: warp w serves lane quarter q = w % 4 (columns 32q..32q+31 of the block) as
-// slot w / 4, taking every fourth task of the block.  A lane copies the stream bytes of its own
-// sub-segment to a private shared-memory buffer (cp.async, the next task's while the current one is
-// being decoded), decodes 16 symbols, splits them and stores them to its tensor-memory lane.
-// One lane of warp 16 fetches the X tiles (ring of `xstages` buffers, one bulk copy each) and issues
-// the MMAs in task order.  mbarriers: per slot and stage `full` (4 arrivals: one per quarter's warp,
-// after its tensor-memory stores) and `empty` (tcgen05.commit once the MMAs that read the stage have
-// finished); per X buffer `xin` (bytes of the bulk copy) and `xempty` (commit).
+// Warps 0..15 decode: warp w serves lane quarter q = w % 4 (columns 32q..32q+31 of the block) in
+// slot w / 4, which takes every fourth task of the block.  A lane copies the stream bytes of its own
+// sub-segment to a private shared-memory buffer (cp.async), decodes 16 symbols, splits them and
+// stores them to its tensor-memory lane.  Warp 16 + i holds the MMA-issuing thread of slot i, which
+// also fetches the slot's X tiles (three buffers, one bulk copy per 16 rows).
+// mbarriers, per slot and stage: `full` (5 arrivals: one per quarter's warp after its tensor-memory
+// stores, one from the thread that requests the X tile, plus the bytes of that bulk copy) and `empty`
+// (tcgen05.commit once the MMAs that read the stage have finished).  The X tile of chunk k + 1 is
+// requested when chunk k turns full: by then the decode warps have seen chunk k - 2 committed, which
+// is the chunk that last used that X buffer.
 // Every wait is bounded; if one runs out the block marks its outputs NaN and still terminates.
-__global__ void __launch_bounds__((kGDecodeWarps + 1) * 32, 1) hac_gemm_tc_kernel(
+__global__ void __launch_bounds__(kGWarps * 32, 1) hac_gemm_tc_kernel(
     DevFormat f, TablePlan tp, const unsigned char* __restrict__ xpack, uint32_t batch, float* __restrict__ y,
     int64_t ys_j, int64_t ys_b, float* __restrict__ partial, uint32_t col_blocks, uint32_t row_splits,
-    uint32_t xstages, uint32_t slot_bytes, uint32_t nbuf) {
+    uint32_t slot_bytes, uint32_t nbuf) {
     const uint32_t warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const uint32_t cblk = blockIdx.x % col_blocks;
     const uint32_t rest = blockIdx.x / col_blocks;
@@ -991,75 +997,77 @@ __global__ void __launch_bounds__((kGDecodeWarps + 1) * 32, 1) hac_gemm_tc_kerne
     const uint32_t t_end = (uint32_t)(((uint64_t)tasks * (rs + 1)) / row_splits);
     const uint32_t ntl = t_end - t_begin;
     const uint32_t cpt = (f.S + kGRows - 1) / kGRows;                           // chunks of 16 rows per task
-    // every task but the matrix's last has S rows, so chunk c of the block is chunk c % cpt of task c / cpt
-    uint32_t chunks = ntl * cpt;
-    if (ntl > 0 && t_end == tasks) chunks -= cpt - ((f.n - (tasks - 1) * f.S) + kGRows - 1) / kGRows;
+    const uint32_t last_chunks = ((f.n - (tasks - 1) * f.S) + kGRows - 1) / kGRows;   // of the matrix's last task
     const uint32_t sb = shared_base();
 
-    // shared memory: [mbarriers; tensor-memory address; lost flag] [tables] [X ring] [per-lane stream buffers]
-    const uint32_t bar_full = sb, bar_empty = sb + 96, bar_xin = sb + 192, bar_xempty = sb + 256, bar_done = sb + 320;
-    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem + 328);
-    volatile uint32_t* lost_flag = reinterpret_cast<volatile uint32_t*>(smem + 332);
-    unsigned char* p = smem + 384;
+    // shared memory: [mbarriers; tensor-memory address; lost flag] [tables] [X buffers] [per-lane stream buffers]
+    const uint32_t bar_full = sb, bar_empty = sb + 64, bar_done = sb + 128;       // [slot][stage], 8 bytes each
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem + 136);
+    volatile uint32_t* lost_flag = reinterpret_cast<volatile uint32_t*>(smem + 140);
+    unsigned char* p = smem + 256;
     if (threadIdx.x == 0) {
-        for (uint32_t i = 0; i < kGSlots * kGStages; ++i) { mbar_init(bar_full + 8 * i, 4); mbar_init(bar_empty + 8 * i, 1); }
-        for (uint32_t i = 0; i < kGXStagesMax; ++i) { mbar_init(bar_xin + 8 * i, 1); mbar_init(bar_xempty + 8 * i, 1); }
-        mbar_init(bar_done, 1);
+        for (uint32_t i = 0; i < kGSlots * kGStages; ++i) { mbar_init(bar_full + 8 * i, 5); mbar_init(bar_empty + 8 * i, 1); }
+        mbar_init(bar_done, kGSlots);
         *lost_flag = 0;
     }
     __syncwarp();
     if (warp == kGDecodeWarps) {
-        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(sb + 328), "r"(kGTmemCols) : "memory");
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(sb + 136), "r"(kGTmemCols) : "memory");
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
     }
     const Decoder dec = stage_decoder(f, tp, p);
     p = smem + ((smem_off(p) + 127u) & ~127u);
-    const uint32_t xring = smem_off(p);
-    p += (size_t)xstages * kGXTileBytes;
+    const uint32_t xring = smem_off(p);                                        // [slot][buffer]
+    p += (size_t)kGSlots * kGXBufs * kGXTileBytes;
     const uint32_t spans = smem_off(p);
     asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
     __syncthreads();
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
     const uint32_t tmem = *tmem_slot;
+    // chunks of slot s: its tasks are s, s + 4, .. (index within the block); all but the matrix's last have cpt
+    auto slot_chunks = [&](uint32_t s) -> uint32_t {
+        if (s >= ntl) return 0u;
+        const uint32_t nt = (ntl - s + kGSlots - 1) / kGSlots;
+        uint32_t c = nt * cpt;
+        if (t_end == tasks && (ntl - 1) % kGSlots == s) c -= cpt - last_chunks;
+        return c;
+    };
 
-    if (warp == kGDecodeWarps) {
-        // ---- X tiles in, MMAs out: one lane, chunk after chunk ----
-        if (lane == 0 && chunks > 0) {
-            // D f32, A and B tf32, both K-major, M = 128; N = 128 (x_hi | x_lo) for w_hi, N = 64 (x_hi) for w_lo
-            const uint32_t idesc_base = (1u << 4) | (2u << 7) | (2u << 10) | ((uint32_t)(kGCols >> 4) << 24);
-            const uint32_t idesc_wide = idesc_base | ((uint32_t)((2 * kGBatch) >> 3) << 17);
-            const uint32_t idesc_half = idesc_base | ((uint32_t)(kGBatch >> 3) << 17);
-            const unsigned char* xt = xpack + ((size_t)bt * tasks + t_begin) * cpt * (size_t)kGXTileBytes;
-            auto fetch_x = [&](uint32_t c) {
-                const uint32_t s = c % xstages;
-                mbar_expect_tx(bar_xin + 8 * s, kGXTileBytes);
-                bulk_copy_g2s(sb + xring + s * kGXTileBytes, xt + (size_t)c * kGXTileBytes, kGXTileBytes, bar_xin + 8 * s);
+    if (warp >= kGDecodeWarps) {
+        // ---- slot's X tiles in, MMAs out: one lane, chunk after chunk ----
+        const uint32_t slot = warp - kGDecodeWarps;
+        if (lane == 0) {
+            const uint32_t nchunks = slot_chunks(slot);
+            // D f32, A and B tf32, both K-major, M = 128, N = 64
+            const uint32_t idesc = (1u << 4) | (2u << 7) | (2u << 10) | ((uint32_t)(kGBatch >> 3) << 17) |
+                                   ((uint32_t)(kGCols >> 4) << 24);
+            const unsigned char* xt = xpack + (size_t)bt * tasks * cpt * (size_t)kGXTileBytes;
+            const uint32_t xbuf0 = sb + xring + slot * kGXBufs * kGXTileBytes;
+            const uint32_t full0 = bar_full + 8 * slot * kGStages, empty0 = bar_empty + 8 * slot * kGStages;
+            const uint32_t d_col = tmem + slot * kGBatch;
+            // chunk k of the slot is chunk k % cpt of task t_begin + slot + 4 * (k / cpt)
+            auto fetch_x = [&](uint32_t k) {
+                const uint32_t task = t_begin + slot + kGSlots * (k / cpt), ci = k % cpt;
+                const uint32_t bar = full0 + 8 * (k % kGStages);
+                mbar_expect_tx(bar, kGXTileBytes);
+                bulk_copy_g2s(xbuf0 + (k % kGXBufs) * kGXTileBytes, xt + ((size_t)task * cpt + ci) * kGXTileBytes, kGXTileBytes, bar);
             };
-            uint32_t pc = 0;                 // next chunk whose X tile is to be fetched
-            for (; pc < min(xstages, chunks); ++pc) fetch_x(pc);
-            for (uint32_t c = 0; c < chunks; ++c) {
-                const uint32_t tl = c / cpt, ci = c - tl * cpt;
-                const uint32_t slot = tl % kGSlots, k = (tl / kGSlots) * cpt + ci;    // k-th chunk of that slot
-                const uint32_t stage = slot * kGStages + k % kGStages, xs = c % xstages;
-                if (!tc_wait(bar_full + 8 * stage, (k / kGStages) & 1u)) *lost_flag = 1;
-                if (!tc_wait(bar_xin + 8 * xs, (c / xstages) & 1u)) *lost_flag = 1;
+            if (nchunks > 0) fetch_x(0);
+            for (uint32_t k = 0; k < nchunks; ++k) {
+                const uint32_t st = k % kGStages;
+                if (!tc_wait(full0 + 8 * st, (k / kGStages) & 1u)) *lost_flag = 1;
+                if (k + 1 < nchunks) fetch_x(k + 1);
                 asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-                const uint32_t a_col = tmem + kGDCols + stage * kGACols;
-                const uint64_t b_desc = tc_desc(sb + xring + xs * kGXTileBytes, kGXLbo);
+                const uint32_t a_col = tmem + kGDCols + (slot * kGStages + st) * kGACols;
+                const uint64_t b_hi = tc_desc(xbuf0 + (k % kGXBufs) * kGXTileBytes, kGXLbo);
 #pragma unroll
                 for (int ks = 0; ks < kGRows / 8; ++ks) {
-                    const uint64_t b = b_desc + (uint64_t)(ks * (kGXKst >> 4));
-                    tc_mma_ts(tmem, a_col + ks * 8, b, idesc_wide, (c | (uint32_t)ks) ? 1u : 0u);
-                    tc_mma_ts(tmem, a_col + kGRows + ks * 8, b, idesc_half, 1u);
+                    const uint64_t bh = b_hi + (uint64_t)(ks * (kGXKst >> 4)), bl = bh + (uint64_t)(kGXLoRows >> 4);
+                    tc_mma_ts(d_col, a_col + ks * 8, bh, idesc, (k | (uint32_t)ks) ? 1u : 0u);          // w_hi * x_hi
+                    tc_mma_ts(d_col, a_col + ks * 8, bl, idesc, 1u);                                    // w_hi * x_lo
+                    tc_mma_ts(d_col, a_col + kGRows + ks * 8, bh, idesc, 1u);                           // w_lo * x_hi
                 }
-                tc_commit(bar_empty + 8 * stage);
-                tc_commit(bar_xempty + 8 * xs);
-                // the X buffer of the previous chunk is free about now: refill it behind the MMAs just issued
-                if (pc < chunks && pc - xstages + 1 <= c) {
-                    if (!tc_wait(bar_xempty + 8 * (pc % xstages), ((pc / xstages) - 1) & 1u)) *lost_flag = 1;
-                    fetch_x(pc);
-                    ++pc;
-                }
+                tc_commit(empty0 + 8 * st);
             }
             tc_commit(bar_done);
         }
@@ -1074,6 +1082,7 @@ __global__ void __launch_bounds__((kGDecodeWarps + 1) * 32, 1) hac_gemm_tc_kerne
         const uint32_t my_buf = spans + warp * nbuf * buf_stride + lane * slot_bytes;       // buffer 0 of this lane
         const uint32_t l1_abs = sb + dec.l1_lane;
         const uint32_t a_base = tmem + ((q * 32u) << 16) + kGDCols + slot * kGStages * kGACols;
+        const uint32_t full0 = bar_full + 8 * slot * kGStages, empty0 = bar_empty + 8 * slot * kGStages;
         // Starts the copy of this lane's sub-segment of `task` into buffer `buf`; returns the bit
         // position of the sub-segment's first code word inside the buffer.
         auto start_copy = [&](uint32_t task, uint32_t buf) -> uint32_t {
@@ -1151,10 +1160,10 @@ __global__ void __launch_bounds__((kGDecodeWarps + 1) * 32, 1) hac_gemm_tc_kerne
                         lo[s] = to_tf32(__uint_as_float(val) - __uint_as_float(hi[s]));
                     }
                 }
-                const uint32_t st = k % kGStages, stage = slot * kGStages + st;
+                const uint32_t st = k % kGStages;
                 // the stage is free once the MMAs of its previous use have been committed (one lane polls)
                 if (k >= kGStages) {
-                    if (lane == 0 && !tc_wait(bar_empty + 8 * stage, ((k / kGStages) - 1) & 1u)) *lost_flag = 1;
+                    if (lane == 0 && !tc_wait(empty0 + 8 * st, ((k / kGStages) - 1) & 1u)) *lost_flag = 1;
                     __syncwarp();
                 }
                 asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
@@ -1163,7 +1172,7 @@ __global__ void __launch_bounds__((kGDecodeWarps + 1) * 32, 1) hac_gemm_tc_kerne
                 asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
                 asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
                 __syncwarp();
-                if (lane == 0) asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar_full + 8 * stage) : "memory");
+                if (lane == 0) asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(full0 + 8 * st) : "memory");
             }
             if (nbuf == 2) { buf ^= 1u; bitpos = next_bitpos; }
             else if (more) bitpos = start_copy(task + kGSlots, 0);
@@ -1171,34 +1180,36 @@ __global__ void __launch_bounds__((kGDecodeWarps + 1) * 32, 1) hac_gemm_tc_kerne
     }
     // ---- epilogue: accumulators -> y ----
     bool lost = false;
-    // the MMA-issuing lane alone waits for the last commit; everyone else sleeps in the block barrier below
-    if (chunks > 0 && warp == kGDecodeWarps && lane == 0 && !tc_wait(bar_done, 0)) lost = true;
+    // one lane waits for the last commits; everyone else sleeps in the block barrier below
+    if (warp == kGDecodeWarps && lane == 0 && !tc_wait(bar_done, 0)) lost = true;
     const bool any_lost = __syncthreads_or((lost || *lost_flag) ? 1 : 0) != 0;
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
     if (warp < 4) {
-        // lane l of warp q holds column 32q + l: inputs 0..63 in accumulator columns 0..63 (x_hi products)
-        // and 64..127 (x_lo products)
+        // lane l of warp q holds column 32q + l; slot s accumulated its tasks in columns 64s..64s+63
         const uint32_t j = cblk * kGCols + warp * 32 + lane;
 #pragma unroll 1
         for (uint32_t half = 0; half < 2; ++half) {
-            uint32_t r0[32], r1[32];
-            if (chunks > 0 && !any_lost) {
-                const uint32_t src = tmem + ((warp * 32u) << 16) + half * 32;
-                tmem_ld32(r0, src);
-                tmem_ld32(r1, src + kGBatch);
-                asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
-            } else {
+            float acc[32];
 #pragma unroll
-                for (int cc = 0; cc < 32; ++cc) { r0[cc] = any_lost ? 0x7fc00000u : 0u; r1[cc] = 0u; }   // NaN marks a lost wait
+            for (int cc = 0; cc < 32; ++cc) acc[cc] = any_lost ? __uint_as_float(0x7fc00000u) : 0.0f;   // NaN marks a lost wait
+            if (!any_lost) {
+#pragma unroll 1
+                for (uint32_t s = 0; s < kGSlots; ++s) {
+                    if (slot_chunks(s) == 0) continue;                   // that accumulator was never written
+                    uint32_t r[32];
+                    tmem_ld32(r, tmem + ((warp * 32u) << 16) + s * kGBatch + half * 32);
+                    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+#pragma unroll
+                    for (int cc = 0; cc < 32; ++cc) acc[cc] += __uint_as_float(r[cc]);
+                }
             }
             if (j < f.m) {
 #pragma unroll
                 for (int cc = 0; cc < 32; ++cc) {
                     const uint32_t b = bt * kGBatch + half * 32 + cc;
                     if (b < batch) {
-                        const float v = __uint_as_float(r1[cc]) + __uint_as_float(r0[cc]);
-                        if (row_splits == 1) y[(int64_t)j * ys_j + (int64_t)b * ys_b] = v;
-                        else partial[((size_t)j * row_splits + rs) * batch + b] = v;
+                        if (row_splits == 1) y[(int64_t)j * ys_j + (int64_t)b * ys_b] = acc[cc];
+                        else partial[((size_t)j * row_splits + rs) * batch + b] = acc[cc];
                     }
                 }
             }
@@ -1566,15 +1577,14 @@ static int launch_gemm_tc(const Format& f, const DeviceInfo& di, const DevFormat
                           unsigned char* xpack, cudaStream_t st, uint32_t* row_splits_out) {
     const size_t budget = (size_t)di.max_smem_optin;
     const uint32_t slot_bytes = d.max_sub_chunks * 16;
-    // shared memory: the deepest X ring and double stream buffers that still leave room for a level-1
-    // table with 8 replicas; failing that, the first combination that fits at all
-    static const uint32_t kChoices[][2] = {{2, 6}, {2, 4}, {1, 6}, {1, 4}, {1, 2}};      // {stream buffers, X buffers}
-    uint32_t nbuf = 0, xstages = 0;
+    // shared memory: double stream buffers if they still leave room for a level-1 table with 8 replicas,
+    // else single ones with the widest table that fits
+    uint32_t nbuf = 0;
     size_t fixed = 0;
-    for (uint32_t want_repl : {3u, 0u}) {
-        for (const auto& c : kChoices) {
-            const size_t fx = 384 + 128 + (size_t)c[1] * kGXTileBytes + (size_t)kGDecodeWarps * c[0] * 32 * slot_bytes;
-            if (fx + plan_smem_bytes(d.l1_bits, want_repl, d.sub_bytes) <= budget) { nbuf = c[0]; xstages = c[1]; fixed = fx; break; }
+    for (uint32_t want_repl : {3u, 2u, 1u, 0u}) {
+        for (uint32_t nb : {2u, 1u}) {
+            const size_t fx = 256 + 128 + (size_t)kGSlots * kGXBufs * kGXTileBytes + (size_t)kGDecodeWarps * nb * 32 * slot_bytes;
+            if (fx + plan_smem_bytes(d.l1_bits, want_repl, d.sub_bytes) <= budget) { nbuf = nb; fixed = fx; break; }
         }
         if (nbuf) break;
     }
@@ -1595,8 +1605,8 @@ static int launch_gemm_tc(const Format& f, const DeviceInfo& di, const DevFormat
     hac_pack_x_kernel<<<(unsigned)pack_blocks, 256, 0, st>>>(d, x, xs_i, xs_b, (uint32_t)batch, xpack, tasks, cpt);
     HAC_CUDA(cudaGetLastError());
     f.last_launches++;
-    hac_gemm_tc_kernel<<<(unsigned)grid, (kGDecodeWarps + 1) * 32, smem, st>>>(
-        d, tp, xpack, (uint32_t)batch, y, ys_j, ys_b, partial, col_blocks, rs, xstages, slot_bytes, nbuf);
+    hac_gemm_tc_kernel<<<(unsigned)grid, kGWarps * 32, smem, st>>>(
+        d, tp, xpack, (uint32_t)batch, y, ys_j, ys_b, partial, col_blocks, rs, slot_bytes, nbuf);
     HAC_CUDA(cudaGetLastError());
     f.last_launches++;
     *row_splits_out = rs;
