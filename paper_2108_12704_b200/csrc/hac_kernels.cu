@@ -97,7 +97,29 @@ struct Decoder {
     uint32_t l1_lane, l1_mul, l1_shift, l1_bits, sub;
 };
 
-// Builds the tables in shared memory (whole block takes part) and advances `p` past them.
+// TF32 split of a shared value for the tensor-core kernel, packed with the code length:
+//   .y = hi | length   (hi = the value rounded to TF32: its low 13 bits are zero, the length, at most 32, sits in the low 6)
+//   .x = lo            (the remainder value - hi, rounded to TF32)
+// An entry that stands for a prefix of longer code words becomes {byte offset of the sub-table,
+// kSplitLong | b}; a sub-table slot of a code word longer still stays {0, 0}.
+constexpr uint32_t kSplitLong = 0x1000u;
+__device__ __forceinline__ uint32_t round_tf32(float v) {
+    uint32_t r;
+    asm("cvt.rna.tf32.f32 %0, %1;" : "=r"(r) : "f"(v));
+    return r;
+}
+__device__ __forceinline__ uint2 split_entry(uint2 e) {
+    if ((int32_t)e.y < 0) return make_uint2(e.x, kSplitLong | (e.y & 31u));
+    if (e.y == 0) return make_uint2(0u, 0u);
+    const float v = __uint_as_float(e.x);
+    const uint32_t hi = round_tf32(v) & 0xffffe000u;
+    const uint32_t lo = round_tf32(v - __uint_as_float(hi)) & 0xffffe000u;
+    return make_uint2(lo, hi | e.y);
+}
+
+// Builds the tables in shared memory (whole block takes part) and advances `p` past them.  With
+// kSplit the entries are stored in the split form above.
+template <bool kSplit = false>
 __device__ __forceinline__ Decoder stage_decoder(const DevFormat& f, const TablePlan& tp, unsigned char*& p) {
     Decoder d;
     const uint32_t repl = 1u << tp.repl_log2;
@@ -118,11 +140,13 @@ __device__ __forceinline__ Decoder stage_decoder(const DevFormat& f, const Table
     for (int k = 0; k < kSubAhead; ++k) {
         const uint32_t i = threadIdx.x + k * blockDim.x;
         sub_v[k] = i < sub_entries ? __ldg(f.sub + i) : make_uint2(0u, 0u);
+        if (kSplit) sub_v[k] = split_entry(sub_v[k]);
     }
     for (uint32_t idx0 = threadIdx.x - lane_; idx0 < (1u << f.l1_bits); idx0 += blockDim.x) {
         const uint32_t idx = idx0 + lane_;
         uint2 v = make_uint2(0u, 0u);
         if (idx < (1u << f.l1_bits)) v = __ldg(f.l1 + idx);
+        if (kSplit) v = split_entry(v);
         uint2* dst = l1 + ((size_t)idx0 << tp.repl_log2);
         const uint32_t warp_slots = min(32u, (1u << f.l1_bits) - idx0) << tp.repl_log2;
         for (uint32_t s0 = 0; s0 < warp_slots; s0 += 32) {
@@ -138,7 +162,8 @@ __device__ __forceinline__ Decoder stage_decoder(const DevFormat& f, const Table
         const uint32_t i = threadIdx.x + k * blockDim.x;
         if (i < sub_entries) sub[i] = sub_v[k];
     }
-    for (uint32_t i = threadIdx.x + kSubAhead * blockDim.x; i < sub_entries; i += blockDim.x) sub[i] = __ldg(f.sub + i);
+    for (uint32_t i = threadIdx.x + kSubAhead * blockDim.x; i < sub_entries; i += blockDim.x)
+        sub[i] = kSplit ? split_entry(__ldg(f.sub + i)) : __ldg(f.sub + i);
     d.l1_lane = smem_off(l1) + ((threadIdx.x & (repl - 1)) << 3);
     d.l1_mul = 8u << tp.repl_log2;
     d.l1_shift = 32 - f.l1_bits;
@@ -367,6 +392,16 @@ __device__ __forceinline__ void resolve_long(uint32_t top, const Decoder& d, con
     uint2 e = lds64(d.sub + val + (q << 3));
     if (e.y == 0) e = decode_long(top, f.lut, f.lut_bits, f.rank_value, f.limit, f.first_left, f.rank_base, f.max_len);
     val = e.x; len = e.y;
+}
+
+// The same for tables in the split form (see split_entry): lo and hi | length come back.
+__device__ __forceinline__ void resolve_long_split(uint32_t top, const Decoder& d, const DevFormat& f, uint32_t& lo,
+                                                   uint32_t& hi_len) {
+    const uint32_t q = (top << d.l1_bits) >> (32 - (hi_len & 31u));
+    uint2 e = lds64(d.sub + lo + (q << 3));
+    if (e.y == 0)
+        e = split_entry(decode_long(top, f.lut, f.lut_bits, f.rank_value, f.limit, f.first_left, f.rank_base, f.max_len));
+    lo = e.x; hi_len = e.y;
 }
 
 // One step of kChains chains: lookups first, then the consumes, so that the table loads overlap.
@@ -842,6 +877,35 @@ __global__ void finalize_kernel(DevFormat f, bool sparse, const float* __restric
     y[(int64_t)j * ys_j + (int64_t)b * ys_b] = s;
 }
 
+// Row splits of the batched HAC kernel: y[j][b] = sum over splits of partial[split][b][j], added in
+// split order.  A block handles 32 columns x 32 inputs: it reads along the columns (contiguous in
+// the partial sums) and writes along whichever of the two indices is contiguous in y.
+__global__ void __launch_bounds__(256) gemm_finalize_kernel(const float* __restrict__ partial, uint32_t splits,
+                                                            uint32_t m, uint32_t batch, float* __restrict__ y,
+                                                            int64_t ys_j, int64_t ys_b) {
+    __shared__ float tile[32][33];
+    const uint32_t j0 = blockIdx.x * 32, b0 = blockIdx.y * 32;
+    for (uint32_t bb = threadIdx.y; bb < 32; bb += blockDim.y) {
+        const uint32_t j = j0 + threadIdx.x, b = b0 + bb;
+        float sum = 0.0f;
+        if (j < m && b < batch)
+            for (uint32_t r = 0; r < splits; ++r) sum += partial[((size_t)r * batch + b) * m + j];
+        tile[bb][threadIdx.x] = sum;
+    }
+    __syncthreads();
+    if (ys_b == 1 && ys_j != 1) {
+        for (uint32_t jj = threadIdx.y; jj < 32; jj += blockDim.y) {
+            const uint32_t j = j0 + jj, b = b0 + threadIdx.x;
+            if (j < m && b < batch) y[(int64_t)j * ys_j + b] = tile[threadIdx.x][jj];
+        }
+    } else {
+        for (uint32_t bb = threadIdx.y; bb < 32; bb += blockDim.y) {
+            const uint32_t j = j0 + threadIdx.x, b = b0 + bb;
+            if (j < m && b < batch) y[(int64_t)j * ys_j + (int64_t)b * ys_b] = tile[bb][threadIdx.x];
+        }
+    }
+}
+
 // ------------------------------------------------------------------------------------------------
 // HAC, batch of inputs (Algorithm 3 without re-decoding W per input), on the 5th-generation tensor
 // cores (tcgen05): Y^T[columns][inputs] = W^T X^T, with W^T as the A operand in tensor memory, X as
@@ -852,19 +916,21 @@ __global__ void finalize_kernel(DevFormat f, bool sparse, const float* __restric
 // quarter of the lanes: lane l of the warp decodes column 32q + l, all lanes walking the same rows,
 // so the symbols a lane decodes one after the other are consecutive K elements of its own
 // accumulator row: they go from registers to tensor memory (tcgen05.st) without a transpose and
-// without passing through shared memory.  Four warps per quarter work on four different tasks at a
-// time; the four warps (one per quarter) that share a task form a "slot" with its own ring of
-// 16-row stages in tensor memory, its own accumulator and its own MMA-issuing thread, so the four
+// without passing through shared memory.  A lane decodes kGChains tasks at a time, so a stage of 16
+// K elements is made of kGChainRows rows of each of them (K need not be contiguous rows of W as long
+// as the X tile lists the same rows in the same order).  Four warps per quarter work on different
+// tasks at a time; the four warps (one per quarter) that share their tasks form a "slot" with its own
+// ring of stages in tensor memory, its own accumulator and its own MMA-issuing thread, so the four
 // pipelines never wait for one another (a commit or an mbarrier wait costs the issuing thread
 // hundreds of cycles; four threads overlap them).  The epilogue adds the four accumulators.
 // Split precision: every weight and every input is written as hi + lo, both rounded to TF32, and
 //   D[128][64] += w_hi * x_hi^T + w_hi * x_lo^T + w_lo * x_hi^T
-// with three MMAs of N = 64 per 8 rows.  The error stays near 1e-7 of sum |w x|, well inside the
+// with three MMAs of N = 64 per 8 K elements.  The error stays near 1e-7 of sum |w x|, well inside the
 // output tolerance.
 // X is split and tiled once per product by hac_pack_x_kernel, exactly as the tensor core reads it
 // ("K-major", no swizzle: four consecutive K elements of one row form a 16-byte unit, 8 rows a
 // 128-byte core matrix, successive 8-row groups are kGSbo bytes apart, the two K halves of an MMA
-// kGXLbo bytes apart), and comes in with one bulk copy per 16 rows.
+// kGXLbo bytes apart), and comes in with one bulk copy per stage.
 // The stream is decoded once per batch tile and never written to global memory.
 // ------------------------------------------------------------------------------------------------
 constexpr int kBatchSteps = 4;          // sHAC batched kernel: entries decoded per lane per phase
@@ -881,8 +947,10 @@ constexpr int kGCols = 128;                         // columns of W per block = 
 constexpr int kGBatch = 64;                         // inputs per batch tile
 constexpr int kGRows = 16;                          // rows of W per tensor-memory stage (two k-steps of 8)
 constexpr int kGSlots = 4;                          // decode warps per quarter of the lanes
-constexpr int kGStages = 2;                         // tensor-memory stages per slot
-constexpr int kGXBufs = 3;                          // X tiles in flight per slot
+constexpr int kGStages = 2;                         // tensor-memory stages per slot (each with its own X tile)
+constexpr int kGChains = 2;                         // tasks a decode lane works on at a time
+constexpr int kGChainRows = kGRows / kGChains;      // rows of each of them in a stage
+static_assert(kGChainRows % 4 == 0, "a task fills whole 16-byte units of the X tile");
 constexpr int kGDecodeWarps = 4 * kGSlots;
 constexpr int kGWarps = kGDecodeWarps + kGSlots;    // plus one MMA-issuing warp per slot
 constexpr uint32_t kGDCols = kGSlots * kGBatch;     // one accumulator of 64 columns per slot
@@ -920,6 +988,19 @@ __device__ __forceinline__ bool tc_wait(uint32_t mbar, uint32_t parity) {
     return false;
 }
 
+// The same wait for a thread that expects to wait long (the MMA-issuing thread, which is ahead of the
+// decode warps most of the time): it sleeps between polls so that it does not take issue slots from them.
+__device__ __forceinline__ bool tc_wait_idle(uint32_t mbar, uint32_t parity) {
+    for (uint32_t t = 0; t < kTcWaitTries; ++t) {
+        uint32_t done;
+        asm volatile("{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}"
+                     : "=r"(done) : "r"(mbar), "r"(parity) : "memory");
+        if (done) return true;
+        __nanosleep(64);
+    }
+    return false;
+}
+
 // 32 consecutive 32-bit columns of this warp's 32 tensor-memory lanes, one lane per thread.
 __device__ __forceinline__ void tmem_ld32(uint32_t (&r)[32], uint32_t taddr) {
     asm volatile(
@@ -942,62 +1023,105 @@ __device__ __forceinline__ void cp_async16(uint32_t dst, const void* src) {
     asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst), "l"(src) : "memory");
 }
 
-// B tiles of hac_gemm_tc_kernel, made once per product: tile ((bt*T + task)*cpt + chunk), T tasks
-// per column and cpt chunks of 16 rows per task, holds rows task*S + 16*chunk .. +15 of the 64
-// inputs of batch tile bt, split into TF32 hi and lo parts and stored exactly as the tile sits in
+// Work split of the batched HAC kernel.  The tasks (sub-segments) of a column are cut into `row_splits`
+// contiguous ranges, one per block; inside a block, slot s and chain c of its `pr`-th round take the
+// block's task (pr * kGChains + c) * kGSlots + s.
+__host__ __device__ inline uint32_t gemm_split_begin(uint32_t tasks, uint32_t rs, uint32_t row_splits) {
+    return (uint32_t)(((uint64_t)tasks * rs) / row_splits);
+}
+__host__ __device__ inline uint32_t gemm_slot_rounds(uint32_t ntl, uint32_t slot) {
+    return slot < ntl ? (ntl - slot + kGChains * kGSlots - 1) / (kGChains * kGSlots) : 0u;
+}
+
+// B tiles of hac_gemm_tc_kernel, made once per product.  Tile ((((bt * row_splits + rs) * kGSlots + slot)
+// * max_rounds + pr) * cpr + ci) holds what slot `slot` of block (rs, bt) multiplies in chunk ci of its
+// round pr: for each of its kGChains tasks, rows ci * kGChainRows .. + kGChainRows - 1 of that task, for the
+// 64 inputs of batch tile bt, split into TF32 hi and lo parts and stored exactly as the tile sits in
 // shared memory.  Rows past the task or the matrix and inputs past the batch are zero.
 // One block of 256 threads per tile, one 16-byte unit of each part per thread.
 __global__ void __launch_bounds__(256) hac_pack_x_kernel(DevFormat f, const float* __restrict__ x, int64_t xs_i,
                                                          int64_t xs_b, uint32_t batch, unsigned char* __restrict__ xpack,
-                                                         uint32_t tasks, uint32_t cpt) {
-    const uint32_t tile = blockIdx.x;
-    const uint32_t ci = tile % cpt, task = (tile / cpt) % tasks, bt = tile / (cpt * tasks);
-    const uint64_t r0 = (uint64_t)task * f.S;
-    const uint32_t cnt = (uint32_t)min((uint64_t)f.S, (uint64_t)f.n - r0);
-    if (ci * kGRows >= cnt) return;                   // no such chunk (last task of a ragged matrix)
+                                                         uint32_t tasks, uint32_t row_splits, uint32_t max_rounds,
+                                                         uint32_t cpr, uint32_t pack_blocks,
+                                                         uint64_t* __restrict__ task_off) {
+    if (blockIdx.x >= pack_blocks) {
+        // The remaining blocks turn the offset index into start bits per task, stored [task][column]
+        // so that the lanes of a decode warp (consecutive columns, same task) read them coalesced:
+        // task_off[t * m + j] = first bit of rows t*S.. of column j; entry `tasks` is the column's end.
+        const uint32_t idx = (blockIdx.x - pack_blocks) * blockDim.x + threadIdx.x;     // g * m + j
+        if (idx >= f.G * f.m) return;
+        const uint32_t g = idx / f.m, j = idx - g * f.m;
+        const size_t u = (size_t)j * f.G + g;
+        uint64_t at = __ldg(f.seg_bit_off + u);
+        const uint4* lens = reinterpret_cast<const uint4*>(f.sub_bits + u * 32);
+#pragma unroll
+        for (int v4 = 0; v4 < 4; ++v4) {
+            const uint4 v = __ldg(lens + v4);
+            const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+            for (int e = 0; e < 8; ++e) {
+                const uint32_t t = g * 32 + (uint32_t)(8 * v4 + e);
+                if (t <= tasks) task_off[(size_t)t * f.m + j] = at;
+                if (t < tasks) at += (e & 1) ? (w[e >> 1] >> 16) : (w[e >> 1] & 0xffffu);
+            }
+        }
+        if (tasks == (g + 1) * 32) task_off[(size_t)tasks * f.m + j] = at;      // the last group is full
+        return;
+    }
+    uint32_t t = blockIdx.x;
+    const uint32_t ci = t % cpr; t /= cpr;
+    const uint32_t pr = t % max_rounds; t /= max_rounds;
+    const uint32_t slot = t % kGSlots; t /= kGSlots;
+    const uint32_t rs = t % row_splits, bt = t / row_splits;
+    const uint32_t t_begin = gemm_split_begin(tasks, rs, row_splits);
+    const uint32_t ntl = gemm_split_begin(tasks, rs + 1, row_splits) - t_begin;
+    if (pr >= gemm_slot_rounds(ntl, slot)) return;   // the slot has no such round: the tile is never read
     const uint32_t b = threadIdx.x % kGBatch, kg = threadIdx.x / kGBatch;      // K group of 4 rows
+    const uint32_t chain = (kg * 4) / kGChainRows, row0 = (kg * 4) % kGChainRows;
+    const uint32_t tl = (pr * kGChains + chain) * kGSlots + slot;
+    const uint64_t r0 = (uint64_t)(t_begin + tl) * f.S;
+    const uint32_t cnt = tl < ntl ? (uint32_t)min((uint64_t)f.S, (uint64_t)f.n - r0) : 0u;
     const bool b_ok = bt * kGBatch + b < batch;
     const float* xc = x + (int64_t)(bt * kGBatch + b) * xs_b;
     float hi[4], lo[4];
 #pragma unroll
     for (int e = 0; e < 4; ++e) {
-        const uint32_t in_task = ci * kGRows + kg * 4 + e;
+        const uint32_t in_task = ci * kGChainRows + row0 + e;
         float v = 0.0f;
         if (b_ok && in_task < cnt) v = __ldg(xc + (int64_t)(r0 + in_task) * xs_i);
         hi[e] = __uint_as_float(to_tf32(v));
         lo[e] = __uint_as_float(to_tf32(v - hi[e]));
     }
-    unsigned char* at = xpack + (size_t)tile * kGXTileBytes + (kg >> 1) * kGXKst + (kg & 1u) * kGXLbo +
+    unsigned char* at = xpack + (size_t)blockIdx.x * kGXTileBytes + (kg >> 1) * kGXKst + (kg & 1u) * kGXLbo +
                         (b >> 3) * kGSbo + (b & 7u) * 16;
     *reinterpret_cast<float4*>(at) = make_float4(hi[0], hi[1], hi[2], hi[3]);
     *reinterpret_cast<float4*>(at + kGXLoRows) = make_float4(lo[0], lo[1], lo[2], lo[3]);
 }
 
 // Warps 0..15 decode: warp w serves lane quarter q = w % 4 (columns 32q..32q+31 of the block) in
-// slot w / 4, which takes every fourth task of the block.  A lane copies the stream bytes of its own
-// sub-segment to a private shared-memory buffer (cp.async), decodes 16 symbols, splits them and
-// stores them to its tensor-memory lane.  Warp 16 + i holds the MMA-issuing thread of slot i, which
-// also fetches the slot's X tiles (three buffers, one bulk copy per 16 rows).
+// slot w / 4.  In every round a lane works on kGChains tasks of its column at once (independent decode
+// chains, interleaved instruction by instruction, which hides the latency of the dependent table
+// lookups): it copies the stream bytes of those sub-segments to private shared-memory buffers
+// (cp.async), and per stage decodes kGChainRows symbols of each, splits them and stores them to its
+// tensor-memory lane.  Warp 16 + i holds the MMA-issuing thread of slot i, which also fetches the
+// slot's X tiles (one bulk copy per stage).
 // mbarriers, per slot and stage: `full` (5 arrivals: one per quarter's warp after its tensor-memory
 // stores, one from the thread that requests the X tile, plus the bytes of that bulk copy) and `empty`
-// (tcgen05.commit once the MMAs that read the stage have finished).  The X tile of chunk k + 1 is
-// requested when chunk k turns full: by then the decode warps have seen chunk k - 2 committed, which
-// is the chunk that last used that X buffer.
+// (tcgen05.commit once the MMAs that read the stage have finished).  The X tile of chunk k + 1 shares
+// its buffer with chunk k - 1 and is requested once that chunk's MMAs have been committed.
 // Every wait is bounded; if one runs out the block marks its outputs NaN and still terminates.
 __global__ void __launch_bounds__(kGWarps * 32, 1) hac_gemm_tc_kernel(
     DevFormat f, TablePlan tp, const unsigned char* __restrict__ xpack, uint32_t batch, float* __restrict__ y,
-    int64_t ys_j, int64_t ys_b, float* __restrict__ partial, uint32_t col_blocks, uint32_t row_splits,
-    uint32_t slot_bytes, uint32_t nbuf) {
+    int64_t ys_j, int64_t ys_b, float* __restrict__ partial, const uint64_t* __restrict__ task_off,
+    uint32_t col_blocks, uint32_t row_splits, uint32_t max_rounds, uint32_t slot_bytes, uint32_t nbuf) {
     const uint32_t warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const uint32_t cblk = blockIdx.x % col_blocks;
     const uint32_t rest = blockIdx.x / col_blocks;
     const uint32_t rs = rest % row_splits, bt = rest / row_splits;
     const uint32_t tasks = (uint32_t)(((uint64_t)f.n + f.S - 1) / f.S);          // sub-segments of a column
-    const uint32_t t_begin = (uint32_t)(((uint64_t)tasks * rs) / row_splits);
-    const uint32_t t_end = (uint32_t)(((uint64_t)tasks * (rs + 1)) / row_splits);
-    const uint32_t ntl = t_end - t_begin;
-    const uint32_t cpt = (f.S + kGRows - 1) / kGRows;                           // chunks of 16 rows per task
-    const uint32_t last_chunks = ((f.n - (tasks - 1) * f.S) + kGRows - 1) / kGRows;   // of the matrix's last task
+    const uint32_t t_begin = gemm_split_begin(tasks, rs, row_splits);
+    const uint32_t ntl = gemm_split_begin(tasks, rs + 1, row_splits) - t_begin;
+    const uint32_t cpr = (f.S + kGChainRows - 1) / kGChainRows;                  // chunks (stages) per round
     const uint32_t sb = shared_base();
 
     // shared memory: [mbarriers; tensor-memory address; lost flag] [tables] [X buffers] [per-lane stream buffers]
@@ -1015,51 +1139,75 @@ __global__ void __launch_bounds__(kGWarps * 32, 1) hac_gemm_tc_kernel(
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(sb + 136), "r"(kGTmemCols) : "memory");
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
     }
-    const Decoder dec = stage_decoder(f, tp, p);
+    // Decode warps: where the sub-segments of the first two rounds start (start bits per task and column,
+    // written by hac_pack_x_kernel), requested before the tables are staged so that the trips to memory
+    // overlap.
+    const uint32_t dq = warp & 3u, dslot = warp >> 2;
+    const uint32_t dj = cblk * kGCols + dq * 32 + lane;                       // this lane's column
+    const bool dvalid = warp < kGDecodeWarps && dj < f.m;
+    const uint32_t rounds = warp < kGDecodeWarps ? gemm_slot_rounds(ntl, dslot) : 0u;
+    // first 16-byte chunk of the stream that holds a sub-segment, and (chunks it spans << 7) | bit
+    // position of its first code word inside the first chunk
+    struct Loc { uint32_t chunk, span; };
+    auto locate = [&](uint32_t pr, Loc (&loc)[kGChains]) {
+#pragma unroll
+        for (int c = 0; c < kGChains; ++c) {
+            loc[c].chunk = 0; loc[c].span = 0;
+            const uint32_t tl = (pr * kGChains + c) * kGSlots + dslot;
+            if (!dvalid || pr >= rounds || tl >= ntl) continue;
+            const uint64_t* at = task_off + (size_t)(t_begin + tl) * f.m + dj;
+            const uint64_t start = __ldg(at);
+            const uint32_t mine = (uint32_t)(__ldg(at + f.m) - start);
+            const uint64_t first_chunk = start >> 7;
+            const uint64_t last_word = ((start + mine) >> 5) + 2;
+            loc[c].chunk = (uint32_t)first_chunk;
+            loc[c].span = ((uint32_t)((last_word >> 2) - first_chunk + 1) << 7) | (uint32_t)(start - (first_chunk << 7));
+        }
+    };
+    Loc loc_cur[kGChains], loc_next[kGChains];
+    locate(0, loc_cur);
+    locate(1, loc_next);
+    const Decoder dec = stage_decoder<true>(f, tp, p);
     p = smem + ((smem_off(p) + 127u) & ~127u);
-    const uint32_t xring = smem_off(p);                                        // [slot][buffer]
-    p += (size_t)kGSlots * kGXBufs * kGXTileBytes;
+    const uint32_t xring = smem_off(p);                                        // [slot][stage]
+    p += (size_t)kGSlots * kGStages * kGXTileBytes;
     const uint32_t spans = smem_off(p);
     asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
     __syncthreads();
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
     const uint32_t tmem = *tmem_slot;
-    // chunks of slot s: its tasks are s, s + 4, .. (index within the block); all but the matrix's last have cpt
-    auto slot_chunks = [&](uint32_t s) -> uint32_t {
-        if (s >= ntl) return 0u;
-        const uint32_t nt = (ntl - s + kGSlots - 1) / kGSlots;
-        uint32_t c = nt * cpt;
-        if (t_end == tasks && (ntl - 1) % kGSlots == s) c -= cpt - last_chunks;
-        return c;
-    };
 
     if (warp >= kGDecodeWarps) {
         // ---- slot's X tiles in, MMAs out: one lane, chunk after chunk ----
         const uint32_t slot = warp - kGDecodeWarps;
         if (lane == 0) {
-            const uint32_t nchunks = slot_chunks(slot);
+            const uint32_t nchunks = gemm_slot_rounds(ntl, slot) * cpr;
             // D f32, A and B tf32, both K-major, M = 128, N = 64
             const uint32_t idesc = (1u << 4) | (2u << 7) | (2u << 10) | ((uint32_t)(kGBatch >> 3) << 17) |
                                    ((uint32_t)(kGCols >> 4) << 24);
-            const unsigned char* xt = xpack + (size_t)bt * tasks * cpt * (size_t)kGXTileBytes;
-            const uint32_t xbuf0 = sb + xring + slot * kGXBufs * kGXTileBytes;
+            // the slot's tiles are consecutive: chunk k of the slot is chunk k % cpr of its round k / cpr
+            const unsigned char* xt = xpack + ((((size_t)bt * row_splits + rs) * kGSlots + slot) * max_rounds) * cpr *
+                                                  (size_t)kGXTileBytes;
+            const uint32_t xbuf0 = sb + xring + slot * kGStages * kGXTileBytes;
             const uint32_t full0 = bar_full + 8 * slot * kGStages, empty0 = bar_empty + 8 * slot * kGStages;
             const uint32_t d_col = tmem + slot * kGBatch;
-            // chunk k of the slot is chunk k % cpt of task t_begin + slot + 4 * (k / cpt)
             auto fetch_x = [&](uint32_t k) {
-                const uint32_t task = t_begin + slot + kGSlots * (k / cpt), ci = k % cpt;
                 const uint32_t bar = full0 + 8 * (k % kGStages);
                 mbar_expect_tx(bar, kGXTileBytes);
-                bulk_copy_g2s(xbuf0 + (k % kGXBufs) * kGXTileBytes, xt + ((size_t)task * cpt + ci) * kGXTileBytes, kGXTileBytes, bar);
+                bulk_copy_g2s(xbuf0 + (k % kGStages) * kGXTileBytes, xt + (size_t)k * kGXTileBytes, kGXTileBytes, bar);
             };
-            if (nchunks > 0) fetch_x(0);
+            for (uint32_t k = 0; k < kGStages && k < nchunks; ++k) fetch_x(k);
             for (uint32_t k = 0; k < nchunks; ++k) {
                 const uint32_t st = k % kGStages;
-                if (!tc_wait(full0 + 8 * st, (k / kGStages) & 1u)) *lost_flag = 1;
-                if (k + 1 < nchunks) fetch_x(k + 1);
+                // the X tile of chunk k + 1 goes where that of chunk k - 1 was: wait for that chunk's MMAs
+                if (k >= 1 && k + 1 < nchunks && k + 1 >= kGStages) {
+                    if (!tc_wait(empty0 + 8 * ((k - 1) % kGStages), ((k - 1) / kGStages) & 1u)) *lost_flag = 1;
+                    fetch_x(k + 1);
+                }
+                if (!tc_wait_idle(full0 + 8 * st, (k / kGStages) & 1u)) *lost_flag = 1;
                 asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
                 const uint32_t a_col = tmem + kGDCols + (slot * kGStages + st) * kGACols;
-                const uint64_t b_hi = tc_desc(xbuf0 + (k % kGXBufs) * kGXTileBytes, kGXLbo);
+                const uint64_t b_hi = tc_desc(xbuf0 + st * kGXTileBytes, kGXLbo);
 #pragma unroll
                 for (int ks = 0; ks < kGRows / 8; ++ks) {
                     const uint64_t bh = b_hi + (uint64_t)(ks * (kGXKst >> 4)), bl = bh + (uint64_t)(kGXLoRows >> 4);
@@ -1074,90 +1222,90 @@ __global__ void __launch_bounds__(kGWarps * 32, 1) hac_gemm_tc_kernel(
         __syncwarp();                        // the other lanes sleep here until the last MMA is issued
     } else {
         // ---- decode -> tensor memory ----
-        const uint32_t q = warp & 3u, slot = warp >> 2;
-        const uint32_t j = cblk * kGCols + q * 32 + lane;
-        const bool valid = j < f.m;
+        const uint32_t q = dq, slot = dslot;
+        const bool valid = dvalid;
         const bool all_valid = __all_sync(0xffffffffu, valid);
         const uint32_t buf_stride = 32 * slot_bytes;
-        const uint32_t my_buf = spans + warp * nbuf * buf_stride + lane * slot_bytes;       // buffer 0 of this lane
+        // this lane's buffers: [parity][chain], buf_stride apart
+        const uint32_t my_buf = spans + warp * nbuf * kGChains * buf_stride + lane * slot_bytes;
         const uint32_t l1_abs = sb + dec.l1_lane;
         const uint32_t a_base = tmem + ((q * 32u) << 16) + kGDCols + slot * kGStages * kGACols;
         const uint32_t full0 = bar_full + 8 * slot * kGStages, empty0 = bar_empty + 8 * slot * kGStages;
-        // Starts the copy of this lane's sub-segment of `task` into buffer `buf`; returns the bit
-        // position of the sub-segment's first code word inside the buffer.
-        auto start_copy = [&](uint32_t task, uint32_t buf) -> uint32_t {
-            uint32_t bitpos = 0;
-            if (valid) {
-                const uint32_t g = task >> 5, t = task & 31u;
-                const size_t u = (size_t)j * f.G + g;
-                const uint4* lens = reinterpret_cast<const uint4*>(f.sub_bits + u * 32);
-                uint32_t before = 0, mine = 0;
+        // the copies of one round (the located sub-segment of every chain), as one cp.async group
+        auto copy_round = [&](const Loc (&loc)[kGChains], uint32_t par) {
+            const uint4* stream4 = reinterpret_cast<const uint4*>(f.stream);
 #pragma unroll
-                for (int v4 = 0; v4 < 4; ++v4) {
-                    const uint4 v = __ldg(lens + v4);
-                    const uint32_t w[4] = {v.x, v.y, v.z, v.w};
-#pragma unroll
-                    for (int e = 0; e < 4; ++e) {
-                        const uint32_t t0 = (uint32_t)(8 * v4 + 2 * e), lo16 = w[e] & 0xffffu, hi16 = w[e] >> 16;
-                        before += (t0 < t ? lo16 : 0u) + (t0 + 1 < t ? hi16 : 0u);
-                        mine = t0 == t ? lo16 : (t0 + 1 == t ? hi16 : mine);
-                    }
-                }
-                const uint64_t start = __ldg(f.seg_bit_off + u) + before;
-                const uint64_t first_chunk = start >> 7;
-                const uint64_t last_word = ((start + mine) >> 5) + 2;
-                const uint32_t nch = (uint32_t)((last_word >> 2) - first_chunk + 1);
-                const uint4* src = reinterpret_cast<const uint4*>(f.stream) + first_chunk;
-                const uint32_t dst = sb + my_buf + buf * buf_stride;
-                for (uint32_t c = 0; c < nch; ++c) cp_async16(dst + 16 * c, src + c);
-                bitpos = (uint32_t)(start - (first_chunk << 7));
+            for (int c = 0; c < kGChains; ++c) {
+                const uint4* src = stream4 + loc[c].chunk;
+                const uint32_t dst = sb + my_buf + (par * kGChains + c) * buf_stride, nch = loc[c].span >> 7;
+                for (uint32_t i = 0; i < nch; ++i) cp_async16(dst + 16 * i, src + i);
             }
             asm volatile("cp.async.commit_group;" ::: "memory");
-            return bitpos;
         };
-        uint32_t buf = 0, bitpos = 0, k = 0;
-        if (slot < ntl) bitpos = start_copy(t_begin + slot, 0);
-        for (uint32_t tl = slot; tl < ntl; tl += kGSlots) {
-            const uint32_t task = t_begin + tl;
-            const bool more = tl + kGSlots < ntl;
-            uint32_t next_bitpos = 0;
+        uint32_t par = 0, k = 0;
+        if (rounds > 0) copy_round(loc_cur, 0);
+        for (uint32_t pr = 0; pr < rounds; ++pr) {
+            const bool more = pr + 1 < rounds;
             if (nbuf == 2 && more) {
-                next_bitpos = start_copy(task + kGSlots, buf ^ 1u);
+                copy_round(loc_next, par ^ 1u);
                 asm volatile("cp.async.wait_group 1;" ::: "memory");
             } else {
                 asm volatile("cp.async.wait_group 0;" ::: "memory");
             }
-            FastReader fr;
-            fr.hi = fr.lo = fr.off = 0; fr.next = sb + my_buf;
-            if (valid) {
-                BitReader br;
-                br.init(my_buf + buf * buf_stride, bitpos);
-                fr.hi = br.hi; fr.lo = br.lo; fr.off = br.off; fr.next = sb + br.next;
-            }
-            const uint32_t cnt = (uint32_t)min((uint64_t)f.S, (uint64_t)f.n - (uint64_t)task * f.S);
-            for (uint32_t r = 0; r < cnt; r += kGRows, ++k) {
-                uint32_t hi[kGRows], lo[kGRows];
-                if (all_valid && r + kGRows <= cnt) {
+            // the index entries of the round after next are in flight while this round is decoded
+            Loc loc_after[kGChains];
+            locate(pr + 2, loc_after);
+            uint32_t bitpos[kGChains];
 #pragma unroll
-                    for (int s = 0; s < kGRows; ++s) {
-                        uint32_t top, val, len;
-                        fast_lookup(fr, dec.l1_shift, dec.l1_mul, l1_abs, top, val, len);
-                        if ((int32_t)len < 0) resolve_long(top, dec, f, val, len);
-                        fast_consume_value(fr, len);
-                        hi[s] = to_tf32(__uint_as_float(val));
-                        lo[s] = to_tf32(__uint_as_float(val) - __uint_as_float(hi[s]));
+            for (int c = 0; c < kGChains; ++c) bitpos[c] = loc_cur[c].span & 127u;
+            FastReader fr[kGChains];
+            uint32_t cnt[kGChains];
+            uint32_t full_rows = f.S;                 // rows every chain of the round has
+#pragma unroll
+            for (int c = 0; c < kGChains; ++c) {
+                const uint32_t tl = (pr * kGChains + c) * kGSlots + slot;
+                cnt[c] = tl < ntl ? (uint32_t)min((uint64_t)f.S, (uint64_t)f.n - (uint64_t)(t_begin + tl) * f.S) : 0u;
+                full_rows = min(full_rows, cnt[c]);
+                fr[c].hi = fr[c].lo = fr[c].off = 0; fr[c].next = sb + my_buf;
+                if (valid && cnt[c] > 0) {
+                    BitReader br;
+                    br.init(my_buf + (par * kGChains + c) * buf_stride, bitpos[c]);
+                    fr[c].hi = br.hi; fr[c].lo = br.lo; fr[c].off = br.off; fr[c].next = sb + br.next;
+                }
+            }
+            for (uint32_t r = 0; r < cpr * kGChainRows; r += kGChainRows, ++k) {
+                uint32_t hi[kGRows], lo[kGRows];
+                // the table entries are {lo, hi | length}: the symbol is ready for the tensor core as it is
+                if (all_valid && r + kGChainRows <= full_rows) {
+#pragma unroll
+                    for (int s = 0; s < kGChainRows; ++s) {
+                        uint32_t top[kGChains], wl[kGChains], wh[kGChains];
+#pragma unroll
+                        for (int c = 0; c < kGChains; ++c) fast_lookup(fr[c], dec.l1_shift, dec.l1_mul, l1_abs, top[c], wl[c], wh[c]);
+#pragma unroll
+                        for (int c = 0; c < kGChains; ++c)
+                            if (wh[c] & kSplitLong) resolve_long_split(top[c], dec, f, wl[c], wh[c]);
+#pragma unroll
+                        for (int c = 0; c < kGChains; ++c) {
+                            fast_consume_value(fr[c], wh[c] & 63u);
+                            hi[c * kGChainRows + s] = wh[c] & 0xffffe000u;
+                            lo[c * kGChainRows + s] = wl[c];
+                        }
                     }
                 } else {
 #pragma unroll
-                    for (int s = 0; s < kGRows; ++s) {
-                        uint32_t top = 0, val = 0, len = 0;
-                        if (valid && r + s < cnt) {
-                            fast_lookup(fr, dec.l1_shift, dec.l1_mul, l1_abs, top, val, len);
-                            if ((int32_t)len < 0) resolve_long(top, dec, f, val, len);
-                            fast_consume_value(fr, len);
+                    for (int s = 0; s < kGChainRows; ++s) {
+#pragma unroll
+                        for (int c = 0; c < kGChains; ++c) {
+                            uint32_t top = 0, wl = 0, wh = 0;
+                            if (valid && r + s < cnt[c]) {
+                                fast_lookup(fr[c], dec.l1_shift, dec.l1_mul, l1_abs, top, wl, wh);
+                                if (wh & kSplitLong) resolve_long_split(top, dec, f, wl, wh);
+                                fast_consume_value(fr[c], wh & 63u);
+                            }
+                            hi[c * kGChainRows + s] = wh & 0xffffe000u;
+                            lo[c * kGChainRows + s] = wl;
                         }
-                        hi[s] = to_tf32(__uint_as_float(val));
-                        lo[s] = to_tf32(__uint_as_float(val) - __uint_as_float(hi[s]));
                     }
                 }
                 const uint32_t st = k % kGStages;
@@ -1174,14 +1322,16 @@ __global__ void __launch_bounds__(kGWarps * 32, 1) hac_gemm_tc_kernel(
                 __syncwarp();
                 if (lane == 0) asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(full0 + 8 * st) : "memory");
             }
-            if (nbuf == 2) { buf ^= 1u; bitpos = next_bitpos; }
-            else if (more) bitpos = start_copy(task + kGSlots, 0);
+            if (nbuf == 2) par ^= 1u;
+            else if (more) copy_round(loc_next, 0);
+#pragma unroll
+            for (int c = 0; c < kGChains; ++c) { loc_cur[c] = loc_next[c]; loc_next[c] = loc_after[c]; }
         }
     }
     // ---- epilogue: accumulators -> y ----
     bool lost = false;
     // one lane waits for the last commits; everyone else sleeps in the block barrier below
-    if (warp == kGDecodeWarps && lane == 0 && !tc_wait(bar_done, 0)) lost = true;
+    if (warp == kGDecodeWarps && lane == 0 && !tc_wait_idle(bar_done, 0)) lost = true;
     const bool any_lost = __syncthreads_or((lost || *lost_flag) ? 1 : 0) != 0;
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
     if (warp < 4) {
@@ -1195,7 +1345,7 @@ __global__ void __launch_bounds__(kGWarps * 32, 1) hac_gemm_tc_kernel(
             if (!any_lost) {
 #pragma unroll 1
                 for (uint32_t s = 0; s < kGSlots; ++s) {
-                    if (slot_chunks(s) == 0) continue;                   // that accumulator was never written
+                    if (gemm_slot_rounds(ntl, s) == 0) continue;         // that accumulator was never written
                     uint32_t r[32];
                     tmem_ld32(r, tmem + ((warp * 32u) << 16) + s * kGBatch + half * 32);
                     asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
@@ -1203,14 +1353,34 @@ __global__ void __launch_bounds__(kGWarps * 32, 1) hac_gemm_tc_kernel(
                     for (int cc = 0; cc < 32; ++cc) acc[cc] += __uint_as_float(r[cc]);
                 }
             }
-            if (j < f.m) {
+            // Stores are made along whichever index is contiguous in memory.  The partial sums are laid
+            // out [split][input][column], so lanes (columns) are contiguous there, and so they are in y
+            // when y_stride_j is 1; otherwise the 32 x 32 block goes through shared memory (the stream
+            // buffers are free by now) and is stored with the lanes along the inputs.
+            const uint32_t b0 = bt * kGBatch + half * 32;
+            if (row_splits > 1) {
+                if (j < f.m) {
 #pragma unroll
-                for (int cc = 0; cc < 32; ++cc) {
-                    const uint32_t b = bt * kGBatch + half * 32 + cc;
-                    if (b < batch) {
-                        if (row_splits == 1) y[(int64_t)j * ys_j + (int64_t)b * ys_b] = acc[cc];
-                        else partial[((size_t)j * row_splits + rs) * batch + b] = acc[cc];
-                    }
+                    for (int cc = 0; cc < 32; ++cc)
+                        if (b0 + cc < batch) partial[((size_t)rs * batch + b0 + cc) * f.m + j] = acc[cc];
+                }
+            } else if (ys_j == 1) {
+                if (j < f.m) {
+#pragma unroll
+                    for (int cc = 0; cc < 32; ++cc)
+                        if (b0 + cc < batch) y[(int64_t)j + (int64_t)(b0 + cc) * ys_b] = acc[cc];
+                }
+            } else {
+                float* tile = reinterpret_cast<float*>(smem + spans) + warp * (32 * 33);
+                __syncwarp();
+#pragma unroll
+                for (int cc = 0; cc < 32; ++cc) tile[cc * 33 + lane] = acc[cc];
+                __syncwarp();
+                const uint32_t jw = cblk * kGCols + warp * 32;
+                if (b0 + lane < batch) {
+                    float* yb = y + (int64_t)(b0 + lane) * ys_b;
+                    const uint32_t jn = min(32u, f.m > jw ? f.m - jw : 0u);
+                    for (uint32_t jj = 0; jj < jn; ++jj) yb[(int64_t)(jw + jj) * ys_j] = tile[lane * 33 + jj];
                 }
             }
         }
@@ -1432,17 +1602,50 @@ static size_t partial_bytes(const Format& f, int64_t batch) {
     return partials ? f.seg_bit_off.size() * (size_t)batch * 4 : 0;
 }
 
-// Batched HAC: the B tiles of the tensor-core kernel (see hac_pack_x_kernel).
-static size_t xpack_bytes(const Format& f, int64_t batch) {
-    if (f.sparse || batch <= 1 || f.symbols == 0) return 0;
-    const size_t cpt = (f.S + kGRows - 1) / kGRows;
-    return (size_t)((batch + kGBatch - 1) / kGBatch) * gemm_tasks(f) * cpt * kGXTileBytes;
+// Row splits of the tensor-core HAC kernel: 1 (a block owns whole columns and writes y itself)
+// unless that leaves most of the SMs idle; a split keeps at least one task per decode chain.
+static uint32_t gemm_row_splits(const Format& f, int64_t batch, int sms) {
+    const uint64_t blocks = (uint64_t)((f.m + kGCols - 1) / kGCols) * (uint64_t)((batch + kGBatch - 1) / kGBatch);
+    const uint32_t tasks = gemm_tasks(f);
+    if (blocks * 5 >= (uint64_t)sms * 3 || tasks <= 1) return 1;
+    const uint64_t by_sms = std::max<uint64_t>(1, (uint64_t)sms / blocks);
+    const uint64_t by_tasks = std::max<uint32_t>(1, tasks / (kGSlots * kGChains));
+    return (uint32_t)std::min<uint64_t>(std::min<uint64_t>(by_sms, by_tasks), kGMaxSplits);
 }
 
-// Workspace of one product: [partial sums, rounded up to 256 bytes][B tiles].
+// Batched HAC: the B tiles of the tensor-core kernel (see hac_pack_x_kernel).  Their number depends on
+// the row split, which depends on the device; without a current device (a size query before any CUDA
+// call) the split that needs most is assumed.
+static uint32_t gemm_max_rounds(const Format& f, uint32_t row_splits) {
+    const uint32_t tasks = gemm_tasks(f);
+    const uint32_t max_ntl = (tasks + row_splits - 1) / row_splits;
+    return (max_ntl + kGChains * kGSlots - 1) / (kGChains * kGSlots);
+}
+static size_t xpack_bytes(const Format& f, int64_t batch) {
+    if (f.sparse || batch <= 1 || f.symbols == 0) return 0;
+    const size_t cpr = (f.S + kGChainRows - 1) / kGChainRows;
+    size_t tiles = 0;
+    DeviceInfo di;
+    if (device_info(di) == HAC_OK) {
+        const uint32_t rs = gemm_row_splits(f, batch, di.sms);
+        tiles = (size_t)rs * kGSlots * gemm_max_rounds(f, rs) * cpr;
+    } else {
+        for (uint32_t rs = 1; rs <= kGMaxSplits; ++rs)
+            tiles = std::max(tiles, (size_t)rs * kGSlots * gemm_max_rounds(f, rs) * cpr);
+    }
+    return (size_t)((batch + kGBatch - 1) / kGBatch) * tiles * kGXTileBytes;
+}
+
+// Batched HAC: start bit of every task of every column, [tasks + 1][m] (see hac_pack_x_kernel).
+static size_t task_off_bytes(const Format& f, int64_t batch) {
+    if (f.sparse || batch <= 1 || f.symbols == 0) return 0;
+    return ((size_t)gemm_tasks(f) + 1) * (size_t)f.m * 8;
+}
+
+// Workspace of one product: [partial sums, rounded up to 256 bytes][B tiles][task start bits].
 static size_t workspace_bytes(const Format& f, int64_t batch) {
     const size_t xp = xpack_bytes(f, batch);
-    return xp ? ((partial_bytes(f, batch) + 255) & ~(size_t)255) + xp : partial_bytes(f, batch);
+    return xp ? ((partial_bytes(f, batch) + 255) & ~(size_t)255) + xp + task_off_bytes(f, batch) : partial_bytes(f, batch);
 }
 
 static int env_int(const char* name, int fallback) {
@@ -1560,17 +1763,6 @@ static int launch_vec(const Format& f, int mode, const float* x, int64_t xs_i, f
     return HAC_OK;
 }
 
-// Row splits of the tensor-core HAC kernel: 1 (a block owns whole columns and writes y itself)
-// unless that leaves most of the SMs idle; a split keeps at least one task per decode slot.
-static uint32_t gemm_row_splits(const Format& f, int64_t batch, int sms) {
-    const uint64_t blocks = (uint64_t)((f.m + kGCols - 1) / kGCols) * (uint64_t)((batch + kGBatch - 1) / kGBatch);
-    const uint32_t tasks = gemm_tasks(f);
-    if (blocks * 5 >= (uint64_t)sms * 3 || tasks <= 1) return 1;
-    const uint64_t by_sms = std::max<uint64_t>(1, (uint64_t)sms / blocks);
-    const uint64_t by_tasks = std::max<uint32_t>(1, tasks / kGSlots);
-    return (uint32_t)std::min<uint64_t>(std::min<uint64_t>(by_sms, by_tasks), kGMaxSplits);
-}
-
 // Batched HAC product: one block per (128 columns, row split, 64 inputs).
 static int launch_gemm_tc(const Format& f, const DeviceInfo& di, const DevFormat& d, const float* x, int64_t xs_i,
                           int64_t xs_b, int64_t batch, float* y, int64_t ys_j, int64_t ys_b, float* partial,
@@ -1583,7 +1775,9 @@ static int launch_gemm_tc(const Format& f, const DeviceInfo& di, const DevFormat
     size_t fixed = 0;
     for (uint32_t want_repl : {3u, 2u, 1u, 0u}) {
         for (uint32_t nb : {2u, 1u}) {
-            const size_t fx = 256 + 128 + (size_t)kGSlots * kGXBufs * kGXTileBytes + (size_t)kGDecodeWarps * nb * 32 * slot_bytes;
+            // the stream buffers double as the epilogue's four 32 x 33 transpose tiles
+            const size_t fx = 256 + 128 + (size_t)kGSlots * kGStages * kGXTileBytes +
+                              std::max<size_t>((size_t)kGDecodeWarps * nb * kGChains * 32 * slot_bytes, 4 * 32 * 33 * 4);
             if (fx + plan_smem_bytes(d.l1_bits, want_repl, d.sub_bytes) <= budget) { nbuf = nb; fixed = fx; break; }
         }
         if (nbuf) break;
@@ -1599,14 +1793,20 @@ static int launch_gemm_tc(const Format& f, const DeviceInfo& di, const DevFormat
     const uint32_t rs = gemm_row_splits(f, batch, di.sms);
     const uint64_t grid = (uint64_t)col_blocks * rs * batch_tiles;
     if (grid > 0x7fffffffull) return HAC_ERR_OFFSET_OVERFLOW;
-    const uint32_t tasks = gemm_tasks(f), cpt = (d.S + kGRows - 1) / kGRows;
-    const uint64_t pack_blocks = (uint64_t)batch_tiles * tasks * cpt;
+    const uint32_t tasks = gemm_tasks(f), cpr = (d.S + kGChainRows - 1) / kGChainRows;
+    const uint32_t max_rounds = gemm_max_rounds(f, rs);
+    const uint64_t pack_blocks = (uint64_t)batch_tiles * rs * kGSlots * max_rounds * cpr;
     if (pack_blocks > 0x7fffffffull) return HAC_ERR_OFFSET_OVERFLOW;
-    hac_pack_x_kernel<<<(unsigned)pack_blocks, 256, 0, st>>>(d, x, xs_i, xs_b, (uint32_t)batch, xpack, tasks, cpt);
+    // the B tiles are a multiple of 8 bytes, so the start bits that follow them are aligned
+    uint64_t* task_off = reinterpret_cast<uint64_t*>(xpack + xpack_bytes(f, batch));
+    const uint64_t off_blocks = ((uint64_t)d.G * d.m + 255) / 256;
+    if (pack_blocks + off_blocks > 0x7fffffffull) return HAC_ERR_OFFSET_OVERFLOW;
+    hac_pack_x_kernel<<<(unsigned)(pack_blocks + off_blocks), 256, 0, st>>>(d, x, xs_i, xs_b, (uint32_t)batch, xpack, tasks, rs,
+                                                                           max_rounds, cpr, (uint32_t)pack_blocks, task_off);
     HAC_CUDA(cudaGetLastError());
     f.last_launches++;
     hac_gemm_tc_kernel<<<(unsigned)grid, kGWarps * 32, smem, st>>>(
-        d, tp, xpack, (uint32_t)batch, y, ys_j, ys_b, partial, col_blocks, rs, slot_bytes, nbuf);
+        d, tp, xpack, (uint32_t)batch, y, ys_j, ys_b, partial, task_off, col_blocks, rs, max_rounds, slot_bytes, nbuf);
     HAC_CUDA(cudaGetLastError());
     f.last_launches++;
     *row_splits_out = rs;
@@ -1683,8 +1883,14 @@ static int dot(const Format& f, const float* x, int64_t batch, int64_t xs_i, int
     bool finish;
     DevFormat dfin = d;
     if (!f.sparse && batch > 1) {
-        finish = gemm_splits > 1;            // partial[(j * splits + split) * batch + b]
-        dfin.G = gemm_splits;
+        if (gemm_splits > 1) {               // partial[split][b][j]
+            dim3 grid((unsigned)((f.m + 31) / 32), (unsigned)((batch + 31) / 32));
+            gemm_finalize_kernel<<<grid, dim3(32, 8), 0, st>>>(partial, gemm_splits, (uint32_t)f.m, (uint32_t)batch, y,
+                                                               ys_j, ys_b);
+            HAC_CUDA(cudaGetLastError());
+            f.last_launches++;
+        }
+        finish = false;
     } else if (!f.sparse) {
         finish = f.G > 1 && !direct;
     } else if (batch == 1) {
