@@ -433,16 +433,28 @@ __device__ __forceinline__ uint32_t lane_start_bits(uint32_t my_bits, uint32_t l
     return inc - my_bits;
 }
 
-// Copy the stream span of one segment to the warp's staging area with 128-bit coalesced loads.
-// Returns the bit position of the segment start relative to the staged span.
+// Asynchronous 16-byte copy global -> shared (both 16-byte aligned); copies_landed() waits for all
+// of this thread's copies.
+__device__ __forceinline__ void cp_async16(uint32_t dst, const void* src) {
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst), "l"(src) : "memory");
+}
+__device__ __forceinline__ void copies_landed() {
+    asm volatile("cp.async.commit_group;" ::: "memory");
+    asm volatile("cp.async.wait_group 0;" ::: "memory");
+}
+
+// Copy the stream span of one segment to the warp's staging area, 16 bytes per lane and request,
+// coalesced and asynchronous: the caller waits with copies_landed() and a warp (or block) barrier
+// before the lanes read the span.  Returns the bit position of the segment start relative to the
+// staged span.
 __device__ __forceinline__ uint32_t stage_span(const DevFormat& f, uint64_t seg_bit, uint32_t total_bits,
                                                uint4* stage, uint32_t lane) {
     const uint64_t first_chunk = seg_bit >> 7;
     const uint64_t last_word = ((seg_bit + total_bits) >> 5) + 2;
     const uint32_t chunks = (uint32_t)((last_word >> 2) - first_chunk + 1);
     const uint4* src = reinterpret_cast<const uint4*>(f.stream) + first_chunk;
-    for (uint32_t c = lane; c < chunks; c += 32) stage[c] = __ldg(src + c);
-    __syncwarp();
+    const uint32_t dst = (uint32_t)__cvta_generic_to_shared(stage);
+    for (uint32_t c = lane; c < chunks; c += 32) cp_async16(dst + 16 * c, src + c);
     return (uint32_t)(seg_bit - (first_chunk << 7));
 }
 
@@ -490,24 +502,14 @@ __global__ void __launch_bounds__(1024) hac_vec_kernel(DevFormat f, TablePlan tp
             x_v[k] = i < f.n ? __ldg(x + (int64_t)i * xs_i) : 0.0f;
         }
     }
-    unsigned char* p = smem;
-    const Decoder dec = stage_decoder(f, tp, p);
+    // The layout of shared memory is known up front: [tables][x][staging areas].  The first item's spans
+    // are requested (asynchronous copies) before the tables and x are staged, so that the block pays one
+    // trip to memory for all three.
     const uint32_t pad = (f.S & 1u) ? 0u : 1u;
-    float* xs = reinterpret_cast<float*>(p);
-    if (kMode == 0 && kXShared) {
-#pragma unroll
-        for (int k = 0; k < kXAhead; ++k) {
-            const uint32_t i = threadIdx.x + k * blockDim.x;
-            if (i < f.n) xs[i + pad * (i / f.S)] = x_v[k];
-        }
-#pragma unroll 4
-        for (uint32_t i = threadIdx.x + kXAhead * blockDim.x; i < f.n; i += blockDim.x)
-            xs[i + pad * (i / f.S)] = __ldg(x + (int64_t)i * xs_i);
-        p += align16(((size_t)f.n + (f.n / f.S + 1) * pad) * 4);
-    }
-    uint4* stage = reinterpret_cast<uint4*>(p) + (size_t)warp * kChains * f.max_unit_chunks;
+    const size_t table_bytes = plan_smem_bytes(f.l1_bits, tp.repl_log2, f.sub_bytes);
+    const size_t x_bytes = (kMode == 0 && kXShared) ? align16(((size_t)f.n + (f.n / f.S + 1) * pad) * 4) : 0;
+    uint4* stage = reinterpret_cast<uint4*>(smem + table_bytes + x_bytes) + (size_t)warp * kChains * f.max_unit_chunks;
     const uint32_t stage_a = smem_off(stage);
-    const uint32_t xs_a = smem_off(xs);
     uint32_t start[kChains], base[kChains];
     auto fetch = [&]() {
 #pragma unroll
@@ -520,6 +522,21 @@ __global__ void __launch_bounds__(1024) hac_vec_kernel(DevFormat f, TablePlan tp
         }
     };
     if (item < items) fetch();
+    unsigned char* p = smem;
+    const Decoder dec = stage_decoder(f, tp, p);
+    float* xs = reinterpret_cast<float*>(p);
+    if (kMode == 0 && kXShared) {
+#pragma unroll
+        for (int k = 0; k < kXAhead; ++k) {
+            const uint32_t i = threadIdx.x + k * blockDim.x;
+            if (i < f.n) xs[i + pad * (i / f.S)] = x_v[k];
+        }
+#pragma unroll 4
+        for (uint32_t i = threadIdx.x + kXAhead * blockDim.x; i < f.n; i += blockDim.x)
+            xs[i + pad * (i / f.S)] = __ldg(x + (int64_t)i * xs_i);
+    }
+    const uint32_t xs_a = smem_off(xs);
+    copies_landed();
     __syncthreads();
 
     while (item < items) {
@@ -650,7 +667,11 @@ __global__ void __launch_bounds__(1024) hac_vec_kernel(DevFormat f, TablePlan tp
         }
         __syncwarp();
         item = next_item;
-        if (item < items) fetch();
+        if (item < items) {
+            fetch();
+            copies_landed();
+            __syncwarp();
+        }
     }
 }
 
@@ -715,20 +736,20 @@ __global__ void __launch_bounds__(1024) shac_vec_kernel(DevFormat f, TablePlan t
         }
         for (uint32_t i = (f.n & ~3u) + threadIdx.x; i < f.n; i += blockDim.x) xs[i] = x[i];
     }
-    const Decoder dec = stage_decoder(f, tp, p);
-    if (kMode == 0 && kXShared && !bulk) {
-#pragma unroll 8
-        for (uint32_t i = threadIdx.x; i < f.n; i += blockDim.x) xs[i] = __ldg(x + (int64_t)i * xs_i);
-    }
-    uint4* stage = reinterpret_cast<uint4*>(p) + (size_t)warp * kChains * f.max_unit_chunks;
-    p += align16((size_t)warps * kChains * f.max_unit_chunks * 16);
+    // [tables] follow at p; the staging areas come after them.  The first item's slices of ri and spans of
+    // the stream are requested (asynchronous copies) before the tables are staged, so that the trips to
+    // memory overlap.
+    unsigned char* after_tables = p + plan_smem_bytes(f.l1_bits, tp.repl_log2, f.sub_bytes);
+    uint4* stage = reinterpret_cast<uint4*>(after_tables) + (size_t)warp * kChains * f.max_unit_chunks;
+    after_tables += align16((size_t)warps * kChains * f.max_unit_chunks * 16);
     // row-index staging: 32*S entries plus up to 16 bytes of misalignment, per segment
     const uint32_t ri_chunks = (32u * f.S * (uint32_t)kRow + 15u) / 16u + 1u;
-    uint4* ri_stage = reinterpret_cast<uint4*>(p) + (size_t)warp * kChains * ri_chunks;
+    uint4* ri_stage = reinterpret_cast<uint4*>(after_tables) + (size_t)warp * kChains * ri_chunks;
     const uint32_t stage_a = smem_off(stage), ri_a = smem_off(ri_stage), xs_a = smem_off(xs);
     const RowT* __restrict__ ri = reinterpret_cast<const RowT*>(f.ri);
 
-    // copies each segment's slice of ri and its span of the stream to shared memory
+    // requests each segment's slice of ri and its span of the stream (copies_landed() and a barrier
+    // come before they are read)
     uint32_t start[kChains], base[kChains], ri_lane[kChains];
     auto fetch = [&]() {
 #pragma unroll
@@ -742,16 +763,21 @@ __global__ void __launch_bounds__(1024) shac_vec_kernel(DevFormat f, TablePlan t
                     const uintptr_t chunk0 = byte0 & ~(uintptr_t)15;
                     const uint32_t chunks = (uint32_t)((byte0 + (uintptr_t)info.count[c] * kRow - chunk0 + 15) >> 4);
                     const uint4* src = reinterpret_cast<const uint4*>(chunk0);
-                    uint4* dst = ri_stage + (size_t)c * ri_chunks;
-                    for (uint32_t k = lane; k < chunks; k += 32) dst[k] = __ldg(src + k);
+                    const uint32_t dst = shared_base() + ri_a + c * ri_chunks * 16;
+                    for (uint32_t k = lane; k < chunks; k += 32) cp_async16(dst + 16 * k, src + k);
                     ri_lane[c] = ri_a + c * ri_chunks * 16 + (uint32_t)(byte0 - chunk0) + lane * f.S * (uint32_t)kRow;
                 }
                 base[c] = stage_span(f, info.bit_off[c], total, stage + (size_t)c * f.max_unit_chunks, lane);
             }
         }
-        __syncwarp();
     };
     if (item < f.items) fetch();
+    const Decoder dec = stage_decoder(f, tp, p);
+    if (kMode == 0 && kXShared && !bulk) {
+#pragma unroll 8
+        for (uint32_t i = threadIdx.x; i < f.n; i += blockDim.x) xs[i] = __ldg(x + (int64_t)i * xs_i);
+    }
+    copies_landed();
     if (bulk) {
         const bool landed = bulk_bytes == 0 || mbar_wait_bounded(mbar, 0);
         if (__syncthreads_or(landed ? 0 : 1)) {             // late or lost: copy x the ordinary way
@@ -856,7 +882,11 @@ __global__ void __launch_bounds__(1024) shac_vec_kernel(DevFormat f, TablePlan t
         }
         __syncwarp();
         item = next_item;
-        if (item < f.items) fetch();
+        if (item < f.items) {
+            fetch();
+            copies_landed();
+            __syncwarp();
+        }
     }
 }
 
@@ -1018,9 +1048,6 @@ __device__ __forceinline__ void tmem_st16(uint32_t taddr, const uint32_t (&v)[16
         "tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16};"
         ::"r"(taddr), "r"(v[0]), "r"(v[1]), "r"(v[2]), "r"(v[3]), "r"(v[4]), "r"(v[5]), "r"(v[6]), "r"(v[7]),
           "r"(v[8]), "r"(v[9]), "r"(v[10]), "r"(v[11]), "r"(v[12]), "r"(v[13]), "r"(v[14]), "r"(v[15]) : "memory");
-}
-__device__ __forceinline__ void cp_async16(uint32_t dst, const void* src) {
-    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst), "l"(src) : "memory");
 }
 
 // Work split of the batched HAC kernel.  The tasks (sub-segments) of a column are cut into `row_splits`
@@ -1428,6 +1455,8 @@ __global__ void __launch_bounds__(1024) shac_batch_kernel(DevFormat f, TablePlan
         uint32_t total;
         const uint32_t start = lane_start_bits(my_bits, lane, total);
         const uint32_t base = stage_span(f, f.seg_bit_off[u], total, stage, lane);
+        copies_landed();
+        __syncwarp();
         const uint32_t seg_pos0 = f.cb[j] + g * 32 * f.S;
         const uint32_t pos0 = seg_pos0 + lane * f.S;
         const uint32_t count = pos0 < col_end ? min(f.S, col_end - pos0) : 0u;
