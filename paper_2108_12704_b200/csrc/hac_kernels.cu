@@ -536,8 +536,9 @@ __global__ void __launch_bounds__(1024) hac_vec_kernel(DevFormat f, TablePlan tp
             xs[i + pad * (i / f.S)] = __ldg(x + (int64_t)i * xs_i);
     }
     const uint32_t xs_a = smem_off(xs);
-    copies_landed();
-    __syncthreads();
+    __syncthreads();                       // tables and x are in place
+    copies_landed();                       // a warp starts as soon as its own spans have landed
+    __syncwarp();
 
     while (item < items) {
         BitReader br[kChains];
@@ -777,14 +778,15 @@ __global__ void __launch_bounds__(1024) shac_vec_kernel(DevFormat f, TablePlan t
 #pragma unroll 8
         for (uint32_t i = threadIdx.x; i < f.n; i += blockDim.x) xs[i] = __ldg(x + (int64_t)i * xs_i);
     }
-    copies_landed();
     if (bulk) {
         const bool landed = bulk_bytes == 0 || mbar_wait_bounded(mbar, 0);
         if (__syncthreads_or(landed ? 0 : 1)) {             // late or lost: copy x the ordinary way
             for (uint32_t i = threadIdx.x; i < f.n; i += blockDim.x) xs[i] = x[i];
         }
     }
-    __syncthreads();
+    __syncthreads();                       // tables and x are in place
+    copies_landed();                       // a warp starts as soon as its own slices and spans have landed
+    __syncwarp();
 
     while (item < f.items) {
         const ShacItem cur = info;
