@@ -433,6 +433,15 @@ __device__ __forceinline__ uint32_t lane_start_bits(uint32_t my_bits, uint32_t l
     return inc - my_bits;
 }
 
+// Programmatic dependent launch.  The product kernels are launched so that they may start while the
+// kernel before them in the stream is still draining: everything they read before depends_wait() is
+// part of the uploaded format (stream, index, tables), which no kernel writes, so fetching it early is
+// safe; x, the workspace and y are touched only after depends_wait(), which returns once the earlier
+// kernel has completed and its writes are visible.  allow_dependents() lets the kernel after this one
+// do the same.
+__device__ __forceinline__ void allow_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+__device__ __forceinline__ void depends_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+
 // Asynchronous 16-byte copy global -> shared (both 16-byte aligned); copies_landed() waits for all
 // of this thread's copies.
 __device__ __forceinline__ void cp_async16(uint32_t dst, const void* src) {
@@ -476,6 +485,7 @@ __global__ void __launch_bounds__(1024) hac_vec_kernel(DevFormat f, TablePlan tp
                                                        float* __restrict__ aux) {
     // A warp works on kChains consecutive segments at a time (an "item"); every lane then runs
     // kChains independent decode chains, which hides the latency of the dependent table lookups.
+    allow_dependents();
     const uint32_t warp = threadIdx.x >> 5, lane = threadIdx.x & 31, warps = blockDim.x >> 5;
     const uint32_t items = (f.units + kChains - 1) / kChains;
     // index entries of this warp's first item: requested before the tables are staged so that the
@@ -490,16 +500,6 @@ __global__ void __launch_bounds__(1024) hac_vec_kernel(DevFormat f, TablePlan tp
         if (item < items && u < f.units) {
             my_bits[c] = __ldg(f.sub_bits + (size_t)u * 32 + lane);
             seg_bit[c] = __ldg(f.seg_bit_off + u);
-        }
-    }
-    // the first elements of x are requested together with the tables (one trip to memory for both)
-    constexpr int kXAhead = 4;
-    float x_v[kXAhead];
-    if (kMode == 0 && kXShared) {
-#pragma unroll
-        for (int k = 0; k < kXAhead; ++k) {
-            const uint32_t i = threadIdx.x + k * blockDim.x;
-            x_v[k] = i < f.n ? __ldg(x + (int64_t)i * xs_i) : 0.0f;
         }
     }
     // The layout of shared memory is known up front: [tables][x][staging areas].  The first item's spans
@@ -522,6 +522,18 @@ __global__ void __launch_bounds__(1024) hac_vec_kernel(DevFormat f, TablePlan tp
         }
     };
     if (item < items) fetch();
+    // everything above reads the format only; x and the outputs belong to the kernels before this one
+    depends_wait();
+    // the first elements of x are requested together with the tables (one trip to memory for both)
+    constexpr int kXAhead = 4;
+    float x_v[kXAhead];
+    if (kMode == 0 && kXShared) {
+#pragma unroll
+        for (int k = 0; k < kXAhead; ++k) {
+            const uint32_t i = threadIdx.x + k * blockDim.x;
+            x_v[k] = i < f.n ? __ldg(x + (int64_t)i * xs_i) : 0.0f;
+        }
+    }
     unsigned char* p = smem;
     const Decoder dec = stage_decoder(f, tp, p);
     float* xs = reinterpret_cast<float*>(p);
@@ -707,6 +719,7 @@ __global__ void __launch_bounds__(1024) shac_vec_kernel(DevFormat f, TablePlan t
                                                         float* __restrict__ aux) {
     constexpr int kChains = 2;
     constexpr int kRow = (int)sizeof(RowT);
+    allow_dependents();
     const uint32_t warp = threadIdx.x >> 5, lane = threadIdx.x & 31, warps = blockDim.x >> 5;
     uint32_t item = blockIdx.x + gridDim.x * warp;
     uint32_t my_bits[kChains] = {0, 0};
@@ -728,15 +741,7 @@ __global__ void __launch_bounds__(1024) shac_vec_kernel(DevFormat f, TablePlan t
     const bool bulk = kMode == 0 && kXShared && tp.x_bulk;
     const uint32_t bulk_bytes = (f.n & ~3u) * 4u;
     if (kMode == 0 && kXShared) p += align16((size_t)f.n * 4);
-    if (bulk) {
-        if (threadIdx.x == 0) mbar_init(mbar, 1);
-        __syncthreads();
-        if (threadIdx.x == 0 && bulk_bytes > 0) {
-            mbar_expect_tx(mbar, bulk_bytes);
-            bulk_copy_g2s(shared_base() + smem_off(xs), x, bulk_bytes, mbar);
-        }
-        for (uint32_t i = (f.n & ~3u) + threadIdx.x; i < f.n; i += blockDim.x) xs[i] = x[i];
-    }
+    if (bulk && threadIdx.x == 0) mbar_init(mbar, 1);
     // [tables] follow at p; the staging areas come after them.  The first item's slices of ri and spans of
     // the stream are requested (asynchronous copies) before the tables are staged, so that the trips to
     // memory overlap.
@@ -773,6 +778,16 @@ __global__ void __launch_bounds__(1024) shac_vec_kernel(DevFormat f, TablePlan t
         }
     };
     if (item < f.items) fetch();
+    // everything above reads the format only; x and the outputs belong to the kernels before this one
+    depends_wait();
+    if (bulk) {
+        __syncthreads();                   // the mbarrier is initialised
+        if (threadIdx.x == 0 && bulk_bytes > 0) {
+            mbar_expect_tx(mbar, bulk_bytes);
+            bulk_copy_g2s(shared_base() + smem_off(xs), x, bulk_bytes, mbar);
+        }
+        for (uint32_t i = (f.n & ~3u) + threadIdx.x; i < f.n; i += blockDim.x) xs[i] = x[i];
+    }
     const Decoder dec = stage_decoder(f, tp, p);
     if (kMode == 0 && kXShared && !bulk) {
 #pragma unroll 8
@@ -897,6 +912,8 @@ __global__ void __launch_bounds__(1024) shac_vec_kernel(DevFormat f, TablePlan t
 // Columns with exactly one segment were written by the product kernel itself.
 __global__ void finalize_kernel(DevFormat f, bool sparse, const float* __restrict__ partial, uint32_t batch,
                                 float* __restrict__ y, int64_t ys_j, int64_t ys_b, uint32_t direct_up_to) {
+    allow_dependents();
+    depends_wait();
     const uint64_t idx = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x;
     if (idx >= (uint64_t)f.m * batch) return;
     const uint32_t j = (uint32_t)(idx / batch), b = (uint32_t)(idx % batch);
@@ -916,6 +933,8 @@ __global__ void __launch_bounds__(256) gemm_finalize_kernel(const float* __restr
                                                             uint32_t m, uint32_t batch, float* __restrict__ y,
                                                             int64_t ys_j, int64_t ys_b) {
     __shared__ float tile[32][33];
+    allow_dependents();
+    depends_wait();
     const uint32_t j0 = blockIdx.x * 32, b0 = blockIdx.y * 32;
     for (uint32_t bb = threadIdx.y; bb < 32; bb += blockDim.y) {
         const uint32_t j = j0 + threadIdx.x, b = b0 + bb;
@@ -1073,6 +1092,8 @@ __global__ void __launch_bounds__(256) hac_pack_x_kernel(DevFormat f, const floa
                                                          uint32_t tasks, uint32_t row_splits, uint32_t max_rounds,
                                                          uint32_t cpr, uint32_t pack_blocks,
                                                          uint64_t* __restrict__ task_off) {
+    allow_dependents();
+    depends_wait();                        // x may come from the kernel before; the workspace may still be read by it
     if (blockIdx.x >= pack_blocks) {
         // The remaining blocks turn the offset index into start bits per task, stored [task][column]
         // so that the lanes of a decode warp (consecutive columns, same task) read them coalesced:
@@ -1143,6 +1164,7 @@ __global__ void __launch_bounds__(kGWarps * 32, 1) hac_gemm_tc_kernel(
     DevFormat f, TablePlan tp, const unsigned char* __restrict__ xpack, uint32_t batch, float* __restrict__ y,
     int64_t ys_j, int64_t ys_b, float* __restrict__ partial, const uint64_t* __restrict__ task_off,
     uint32_t col_blocks, uint32_t row_splits, uint32_t max_rounds, uint32_t slot_bytes, uint32_t nbuf) {
+    allow_dependents();
     const uint32_t warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const uint32_t cblk = blockIdx.x % col_blocks;
     const uint32_t rest = blockIdx.x / col_blocks;
@@ -1169,8 +1191,7 @@ __global__ void __launch_bounds__(kGWarps * 32, 1) hac_gemm_tc_kernel(
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
     }
     // Decode warps: where the sub-segments of the first two rounds start (start bits per task and column,
-    // written by hac_pack_x_kernel), requested before the tables are staged so that the trips to memory
-    // overlap.
+    // written by hac_pack_x_kernel).
     const uint32_t dq = warp & 3u, dslot = warp >> 2;
     const uint32_t dj = cblk * kGCols + dq * 32 + lane;                       // this lane's column
     const bool dvalid = warp < kGDecodeWarps && dj < f.m;
@@ -1193,6 +1214,10 @@ __global__ void __launch_bounds__(kGWarps * 32, 1) hac_gemm_tc_kernel(
             loc[c].span = ((uint32_t)((last_word >> 2) - first_chunk + 1) << 7) | (uint32_t)(start - (first_chunk << 7));
         }
     };
+    // Tensor memory and barriers need nothing from the kernel before this one (hac_pack_x_kernel), so they
+    // are set up while it still runs; its output is read from here on.  The start bits are requested
+    // before the tables are staged so that the trips to memory overlap.
+    depends_wait();
     Loc loc_cur[kGChains], loc_next[kGChains];
     locate(0, loc_cur);
     locate(1, loc_next);
@@ -1690,6 +1715,20 @@ static int prepare_kernel(K kernel, size_t smem) {
     return HAC_OK;
 }
 
+// Launch with programmatic stream serialization: the kernel may start while the one before it in the
+// stream drains; it calls depends_wait() before touching anything an earlier kernel may have written.
+template <typename... KArgs, typename... Args>
+static int launch_dependent(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st, Args... args) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid; cfg.blockDim = block; cfg.dynamicSmemBytes = smem; cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = env_int("HAC_B200_PDL", 1) != 0 ? 1 : 0;
+    cfg.attrs = attr; cfg.numAttrs = 1;
+    HAC_CUDA(cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...));
+    return HAC_OK;
+}
+
 // Largest number of warps per block (a multiple of `step`, at most `want`) whose shared memory
 // fits; 0 if not even `step` warps fit.
 static int fit_warps(size_t fixed, size_t per_warp, int want, int step, size_t budget) {
@@ -1702,8 +1741,9 @@ static int launch_finalize(const Format& f, const DevFormat& d, const float* par
                            int64_t ys_j, int64_t ys_b, cudaStream_t st, uint32_t direct_up_to) {
     const uint64_t total = (uint64_t)f.m * (uint64_t)batch;
     const unsigned blocks = (unsigned)((total + 255) / 256);
-    finalize_kernel<<<blocks, 256, 0, st>>>(d, f.sparse, partial, (uint32_t)batch, y, ys_j, ys_b, direct_up_to);
-    HAC_CUDA(cudaGetLastError());
+    const int rc = launch_dependent(finalize_kernel, dim3(blocks), dim3(256), 0, st, d, f.sparse, partial, (uint32_t)batch, y,
+                                    ys_j, ys_b, direct_up_to);
+    if (rc) return rc;
     f.last_launches++;
     return HAC_OK;
 }
@@ -1787,7 +1827,8 @@ static int launch_vec(const Format& f, int mode, const float* x, int64_t xs_i, f
     // spread the segments over all SMs (a block's warps take segments blockIdx + k * gridDim)
     const unsigned items = f.sparse ? d.items : (d.units + chains - 1) / chains;
     const unsigned grid = std::min<unsigned>(items, (unsigned)(di.sms * per_sm));
-    kernel<<<grid, threads, smem, st>>>(dk, tp, x, xs_i, y, ys_j, aux);
+    rc = launch_dependent(kernel, dim3(grid), dim3((unsigned)threads), smem, st, dk, tp, x, xs_i, y, ys_j, aux);
+    if (rc) return rc;
     if (vec_direct) *vec_direct = (!f.sparse && (f.G == 1 || (chains == 2 && f.G == 2)));
     HAC_CUDA(cudaGetLastError());
     f.last_launches++;
@@ -1832,13 +1873,14 @@ static int launch_gemm_tc(const Format& f, const DeviceInfo& di, const DevFormat
     uint64_t* task_off = reinterpret_cast<uint64_t*>(xpack + xpack_bytes(f, batch));
     const uint64_t off_blocks = ((uint64_t)d.G * d.m + 255) / 256;
     if (pack_blocks + off_blocks > 0x7fffffffull) return HAC_ERR_OFFSET_OVERFLOW;
-    hac_pack_x_kernel<<<(unsigned)(pack_blocks + off_blocks), 256, 0, st>>>(d, x, xs_i, xs_b, (uint32_t)batch, xpack, tasks, rs,
-                                                                           max_rounds, cpr, (uint32_t)pack_blocks, task_off);
-    HAC_CUDA(cudaGetLastError());
+    rc = launch_dependent(hac_pack_x_kernel, dim3((unsigned)(pack_blocks + off_blocks)), dim3(256), 0, st, d, x, xs_i, xs_b,
+                          (uint32_t)batch, xpack, tasks, rs, max_rounds, cpr, (uint32_t)pack_blocks, task_off);
+    if (rc) return rc;
     f.last_launches++;
-    hac_gemm_tc_kernel<<<(unsigned)grid, kGWarps * 32, smem, st>>>(
-        d, tp, xpack, (uint32_t)batch, y, ys_j, ys_b, partial, task_off, col_blocks, rs, max_rounds, slot_bytes, nbuf);
-    HAC_CUDA(cudaGetLastError());
+    rc = launch_dependent(hac_gemm_tc_kernel, dim3((unsigned)grid), dim3(kGWarps * 32), smem, st, d, tp,
+                          (const unsigned char*)xpack, (uint32_t)batch, y, ys_j, ys_b, partial, (const uint64_t*)task_off,
+                          col_blocks, rs, max_rounds, slot_bytes, nbuf);
+    if (rc) return rc;
     f.last_launches++;
     *row_splits_out = rs;
     return HAC_OK;
@@ -1916,6 +1958,8 @@ static int dot(const Format& f, const float* x, int64_t batch, int64_t xs_i, int
     if (!f.sparse && batch > 1) {
         if (gemm_splits > 1) {               // partial[split][b][j]
             dim3 grid((unsigned)((f.m + 31) / 32), (unsigned)((batch + 31) / 32));
+            // launched the ordinary way: started early, its blocks only took the idle SMs from the product
+            // kernel's successor (measured: slower)
             gemm_finalize_kernel<<<grid, dim3(32, 8), 0, st>>>(partial, gemm_splits, (uint32_t)f.m, (uint32_t)batch, y,
                                                                ys_j, ys_b);
             HAC_CUDA(cudaGetLastError());
