@@ -187,9 +187,14 @@ int shac_attach(shac_format* f, void* dev_buf, size_t dev_bytes);
  *   workspace  device scratch of at least *_workspace_bytes(f, batch) bytes, 16-byte aligned (may be
  *              NULL when that is 0).  It holds partial sums of columns that span several segments
  *              and, for a batched HAC product, the inputs split into two TF32 parts and arranged
- *              in the tiles the tensor-core kernel reads; its contents need not be initialised and
- *              are undefined afterwards.  Two dot calls that run concurrently must not share it.
- * Asynchronous on cuda_stream.  Errors: HAC_ERR_NOT_UPLOADED, HAC_ERR_INVALID_ARG (batch < 1, null
+ *              in the tiles the tensor-core kernel reads, plus the start bit of every sub-segment
+ *              of every column (rebuilt from the offset index on each call); its contents need not
+ *              be initialised and are undefined afterwards.  Two dot calls that run concurrently
+ *              must not share it.
+ * Asynchronous on cuda_stream.  The kernels are launched with programmatic stream serialization:
+ * they may begin fetching the uploaded format while the kernel before them in the stream is still
+ * finishing, but read x and the workspace and write y only once that kernel has completed, so the
+ * usual stream ordering holds for everything the caller can observe.  Errors: HAC_ERR_NOT_UPLOADED, HAC_ERR_INVALID_ARG (batch < 1, null
  * pointers, misaligned workspace), HAC_ERR_BUFFER_TOO_SMALL, HAC_ERR_CUDA (launch failure).
  * ------------------------------------------------------------------------------------------- */
 int hac_workspace_bytes (const hac_format*  f, int64_t batch, size_t* out);
