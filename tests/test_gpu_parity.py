@@ -206,3 +206,35 @@ def test_config5_sweep_cells_full_size(sp, k):
     wl = dataclasses.replace(si.sweep_cells()[0], sparsity=sp, k=k)
     for kind in ("hac", "shac"):
         _full_size(wl, kind, (1, 32), ncols=32)
+
+
+def test_chained_products_keep_stream_order():
+    """Two layers back to back on one stream, the second reading what the first wrote, then the same
+    buffers reused at once for another input: the kernels may start early (they are launched with
+    programmatic stream serialization) but must not read x or write y before the kernel ahead of them
+    is done."""
+    wl = si.scaled(si.CFG2_DENSE_HAC, 1536, 1536)
+    lf, Wq, mask = build_both(wl, "hac", 64)
+    Wd = Wq.astype(np.float64)
+    for B in (1, 64):
+        X = si.inputs(wl, B)
+        ws = torch.empty(max(16, lf.workspace_bytes(B)), dtype=torch.uint8, device="cuda")
+        x0 = torch.from_numpy(X[0] if B == 1 else np.ascontiguousarray(X.T)).cuda()
+        shape = (wl.m,) if B == 1 else (wl.m, B)
+        y1 = torch.empty(shape, device="cuda")
+        y2 = torch.empty(shape, device="cuda")
+        outs = []
+        for rep in range(3):                       # no synchronisation between the launches
+            lf.dot(x0, y1, ws)
+            lf.dot(y1, y2, ws)
+            outs.append(y2.clone())
+            x0 = x0 * 0.5                          # a new input in a new buffer; y1, y2 and ws are reused
+        torch.cuda.synchronize()
+        Xd = X.astype(np.float64)
+        for rep, got in enumerate(outs):
+            h1 = (Xd * 0.5 ** rep) @ Wd
+            ref = h1 @ Wd
+            a = np.abs(h1) @ np.abs(Wd) + (np.abs(Xd * 0.5 ** rep) @ np.abs(Wd)) @ np.abs(Wd)
+            g = got.cpu().numpy()
+            g = g[None] if B == 1 else g.T
+            check_outputs(g, ref, a)
