@@ -1447,13 +1447,15 @@ __global__ void __launch_bounds__(kGWarps * 32, 1) hac_gemm_tc_kernel(
 // ------------------------------------------------------------------------------------------------
 // sHAC, batch of inputs.  One warp per segment: lanes decode kBatchSteps entries each into a small
 // shared tile of (value, row) pairs, then the warp walks the tile with lanes spread over the
-// inputs, gathering the rows of X (stored [n][batch] for coalesced access).
+// inputs, gathering the rows of X (stored [n][batch] for coalesced access).  With 16 inputs or fewer
+// the lanes are split into groups of `narrow` (a power of two that holds the batch): every group
+// takes its own entry of the tile, and the groups' sums are added with shuffles at the end.
 // ------------------------------------------------------------------------------------------------
 template <int kAcc, typename RowT>
 __global__ void __launch_bounds__(1024) shac_batch_kernel(DevFormat f, TablePlan tp, const float* __restrict__ x,
                                                           int64_t xs_i, int64_t xs_b, uint32_t batch,
                                                           float* __restrict__ y, int64_t ys_j, int64_t ys_b,
-                                                          float* __restrict__ partial) {
+                                                          float* __restrict__ partial, uint32_t narrow) {
     unsigned char* p = smem;
     const Decoder dec = stage_decoder(f, tp, p);
     const uint32_t warp = threadIdx.x >> 5, lane = threadIdx.x & 31, warps = blockDim.x >> 5;
@@ -1506,23 +1508,37 @@ __global__ void __launch_bounds__(1024) shac_batch_kernel(DevFormat f, TablePlan
                 wr[lane * kBatchSteps + s] = row;
             }
             __syncwarp();
+            if (kAcc == 1 && narrow) {
+                // few inputs: `narrow` lanes per entry, 32 / narrow entries at a time
+                const uint32_t e = lane / narrow, b = lane % narrow;
+                if (b < batch) {
 #pragma unroll 4
-            for (uint32_t r = 0; r < kBatchRows; ++r) {
-                const float v = wv[r];
-                const float* xr = x + (int64_t)wr[r] * xs_i;
+                    for (uint32_t r = e; r < kBatchRows; r += 32 / narrow)
+                        acc[0] = fmaf(wv[r], x[(int64_t)wr[r] * xs_i + (int64_t)b * xs_b], acc[0]);
+                }
+            } else {
+#pragma unroll 4
+                for (uint32_t r = 0; r < kBatchRows; ++r) {
+                    const float v = wv[r];
+                    const float* xr = x + (int64_t)wr[r] * xs_i;
 #pragma unroll
-                for (int a = 0; a < kAcc; ++a) {
-                    const uint32_t b = b0 + a * 32 + lane;
-                    if (b < batch) acc[a] = fmaf(v, xr[(int64_t)b * xs_b], acc[a]);
+                    for (int a = 0; a < kAcc; ++a) {
+                        const uint32_t b = b0 + a * 32 + lane;
+                        if (b < batch) acc[a] = fmaf(v, xr[(int64_t)b * xs_b], acc[a]);
+                    }
                 }
             }
             __syncwarp();
         }
+        if (kAcc == 1 && narrow) {               // add the entry groups; lanes 0 .. narrow-1 hold the sums
+            for (uint32_t d = narrow; d < 32; d <<= 1) acc[0] += __shfl_xor_sync(0xffffffffu, acc[0], d);
+        }
+        const bool writer = !(kAcc == 1 && narrow) || lane < narrow;
         const bool single = (f.seg_first[j + 1] - first) == 1;
 #pragma unroll
         for (int a = 0; a < kAcc; ++a) {
             const uint32_t b = b0 + a * 32 + lane;
-            if (b < batch) {
+            if (writer && b < batch) {
                 if (single) y[(int64_t)j * ys_j + (int64_t)b * ys_b] = acc[a];
                 else partial[(size_t)u * batch + b] = acc[a];
             }
@@ -1901,7 +1917,7 @@ static int launch_batch_t(const Format& f, const DeviceInfo& di, const DevFormat
     if (warps == 0) return HAC_ERR_BUFFER_TOO_SMALL;
     const size_t smem = tab + 32 + per_warp * warps;
     void (*kernel)(DevFormat, TablePlan, const float*, int64_t, int64_t, uint32_t, float*, int64_t, int64_t,
-                   float*) = f.ri_bits == 16 ? shac_batch_kernel<kAcc, uint16_t> : shac_batch_kernel<kAcc, uint32_t>;
+                   float*, uint32_t) = f.ri_bits == 16 ? shac_batch_kernel<kAcc, uint16_t> : shac_batch_kernel<kAcc, uint32_t>;
     int rc = prepare_kernel(kernel, smem);
     if (rc) return rc;
     int per_sm = 1;
@@ -1909,7 +1925,10 @@ static int launch_batch_t(const Format& f, const DeviceInfo& di, const DevFormat
     per_sm = std::max(per_sm, 1);
     const uint64_t items = (uint64_t)d.units * batch_tiles;
     const unsigned grid = (unsigned)std::min<uint64_t>((items + warps - 1) / warps, (uint64_t)di.sms * per_sm);
-    kernel<<<grid, warps * 32, smem, st>>>(d, tp, x, xs_i, xs_b, (uint32_t)batch, y, ys_j, ys_b, partial);
+    // up to 16 inputs: the smallest power of two that holds them, as lanes per entry
+    uint32_t narrow = 0;
+    if (batch <= 16) { narrow = 2; while ((int64_t)narrow < batch) narrow <<= 1; }
+    kernel<<<grid, warps * 32, smem, st>>>(d, tp, x, xs_i, xs_b, (uint32_t)batch, y, ys_j, ys_b, partial, narrow);
     HAC_CUDA(cudaGetLastError());
     f.last_launches++;
     return HAC_OK;
