@@ -40,7 +40,7 @@ FALLBACK_HBM_GBS = 6650.0
 
 # dram__bytes_read.sum + dram__bytes_write.sum per launch of the GEMV kernel from one ncu capture
 # (profiles/hac_vec_kernel_config2_gemv.md), valid only for the kernel source it was taken on.
-NCU_GEMV_TRAFFIC = {"bytes": 14615296, "kernel_source_sha256": "8a1c382a2e26cf358a0e8319b8b3c159d9b62c313a47d6132a54e8e144b6ab18"}
+NCU_GEMV_TRAFFIC = {"bytes": 14614272, "kernel_source_sha256": "14e5175af6d210027e5ccc6ba5ef054b7bf11874a842147d62ad04e0ed508fa6"}
 
 
 def gemv_traffic():
