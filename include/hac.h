@@ -50,6 +50,8 @@ extern "C" {
 #define HAC_QUANT_NONE     0u   /* W already holds few distinct values                            */
 #define HAC_QUANT_KMEANS   1u   /* CWS, Sect. III-C.1                                             */
 #define HAC_QUANT_UNIFORM  2u   /* UQ,  Sect. III-C.3, grid over [min, max] of the non-null weights */
+#define HAC_QUANT_GRID     3u   /* UQ as printed in Sect. III-C.3 with d = 0: w = delta * round(w / delta),
+                                   delta tuned by bisection to leave at most k distinct values          */
 
 typedef struct hac_format  hac_format;    /* HAC : stream, codebook, code lengths, offset index          */
 typedef struct shac_format shac_format;   /* sHAC: stream of nz, ri, cb, codebook, lengths, offset index */
@@ -135,8 +137,10 @@ typedef struct shac_host_view {
  *   params see hac_build_params.
  *   out    receives the new handle.
  * Steps: entries with |w| <= the floor(sparsity*n*m)-th smallest magnitude become 0; the others are
- * replaced by one of k shared values (k-means over them in column-major order, or a uniform grid
- * over their range); distinct values sorted ascending form the codebook; a Huffman code over the
+ * replaced by one of k shared values (k-means over them in column-major order, a uniform grid over
+ * their range, or the zero-anchored grid delta * round(w / delta) whose delta is found by 70 halvings
+ * of [0, 4 max|w|]: a trial delta that leaves at most k distinct values becomes the upper end, the
+ * upper end is used; weights with at most k distinct values are kept as they are); distinct values sorted ascending form the codebook; a Huffman code over the
  * symbol counts (HAC: every entry, zeros included; sHAC: stored entries only) is made canonical;
  * code words are concatenated column by column, most significant bit first, into 32-bit words.
  * Offset index (the column-offset vector suggested in the paper's conclusions, refined): each column

@@ -190,6 +190,48 @@ def uniform_share(Wp: np.ndarray, k: int):
     return _scatter_colmajor(mask, values), mask
 
 
+def grid_levels(data: np.ndarray, delta: float) -> np.ndarray:
+    """round(w / delta) of the formula of Sect. III-C.3 with d = 0, rounding half up."""
+    return np.floor(data / np.float64(delta) + 0.5)
+
+
+def grid_delta(data: np.ndarray, k: int, steps: int = 70) -> float:
+    """The interval size delta of the zero-anchored grid, chosen so that the wanted number k of
+    values results (the setting of uUQ in Sect. V; the paper gives no procedure): bisection on [0, 4 max|w|], `steps` halvings (enough to
+    end on neighbouring doubles for k up to 2048); a trial
+    delta that leaves at most k distinct values becomes the upper end, one that leaves more
+    the lower end; the upper end is returned (it always satisfies the bound: at 4 max|w| every
+    weight rounds to 0)."""
+    a = np.float64(0.0)
+    b = np.float64(4.0) * np.abs(data).max()
+    for _ in range(steps):
+        mid = np.float64(0.5) * (a + b)
+        if len(np.unique(grid_levels(data, mid))) <= k:
+            b = mid
+        else:
+            a = mid
+    return float(b)
+
+
+def grid_share(Wp: np.ndarray, k: int):
+    """UQ exactly as printed in Sect. III-C.3, with the bias d = 0 of the paper's experiments:
+    w = delta * round(w0 / delta) over the non-null weights, delta from grid_delta.  A weight that
+    rounds to level 0 becomes the value 0.0 but stays a stored entry (it survived pruning).
+    When the non-null weights already have at most k distinct values they are kept as they are.
+    Returns (Wq, mask)."""
+    data, mask = _nonnull_colmajor(Wp)
+    if k < 2:
+        raise ValueError("grid quantization needs k >= 2")
+    if data.size == 0:
+        return np.zeros_like(Wp), mask
+    if len(np.unique(data)) <= k:
+        return _scatter_colmajor(mask, data.astype(np.float32)), mask
+    delta = np.float64(grid_delta(data, k))
+    values = (grid_levels(data, delta) * delta).astype(np.float32)
+    values[values == 0] = np.float32(0.0)                  # -0.0 -> +0.0
+    return _scatter_colmajor(mask, values), mask
+
+
 def share_none(Wp: np.ndarray):
     """No weight sharing: the matrix already holds few distinct values."""
     Wq = Wp.copy()
@@ -199,7 +241,8 @@ def share_none(Wp: np.ndarray):
 
 def quantize(W: np.ndarray, sparsity: float, k: int, quantizer: int, iters: int = 20, seed: int = 0):
     """Pruning then weight sharing, as chained in Sect. III-C.1.  quantizer:
-    0 none, 1 k-means (CWS), 2 uniform (UQ).  Returns (Wq, mask)."""
+    0 none, 1 k-means (CWS), 2 uniform (UQ over [min, max]), 3 uniform (UQ on the zero-anchored
+    grid of the printed formula).  Returns (Wq, mask)."""
     Wp = prune(W, sparsity)
     if quantizer == 0:
         return share_none(Wp)
@@ -207,6 +250,8 @@ def quantize(W: np.ndarray, sparsity: float, k: int, quantizer: int, iters: int 
         return kmeans_share(Wp, k, iters, seed)
     if quantizer == 2:
         return uniform_share(Wp, k)
+    if quantizer == 3:
+        return grid_share(Wp, k)
     raise ValueError("unknown quantizer")
 
 

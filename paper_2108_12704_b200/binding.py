@@ -10,7 +10,7 @@ import numpy as np
 
 from . import build as _build
 
-QUANT_NONE, QUANT_KMEANS, QUANT_UNIFORM = 0, 1, 2
+QUANT_NONE, QUANT_KMEANS, QUANT_UNIFORM, QUANT_GRID = 0, 1, 2, 3
 
 
 class HacError(RuntimeError):

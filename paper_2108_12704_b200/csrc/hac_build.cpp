@@ -108,6 +108,69 @@ int share_uniform(const std::vector<double>& data, uint32_t k, Shared& out) {
     return HAC_OK;
 }
 
+int share_none(const std::vector<double>& data, Shared& out);
+
+// Sect. III-C.3 as printed, with d = 0: w = delta * round(w / delta) (rounding half up).  delta is tuned
+// to the number of values wanted (the paper's setting for uUQ): 70 halvings of [0, 4 max|w|]; a trial
+// delta that leaves at most k distinct levels becomes the upper end, and the upper end is used.
+int share_grid(const std::vector<double>& data, uint32_t k, Shared& out) {
+    const size_t q = data.size();
+    {
+        std::vector<double> distinct(data);
+        std::sort(distinct.begin(), distinct.end());
+        distinct.erase(std::unique(distinct.begin(), distinct.end()), distinct.end());
+        if (distinct.size() <= k) return share_none(data, out);
+    }
+    double amax = 0.0;
+    for (size_t p = 0; p < q; ++p) amax = std::max(amax, std::fabs(data[p]));
+    std::vector<int64_t> lev(q);
+    std::vector<unsigned char> seen;
+    // number of distinct levels at `delta`; stops counting once it exceeds `limit`
+    auto distinct_levels = [&](double delta, uint64_t limit) -> uint64_t {
+        int64_t lo = INT64_MAX, hi = INT64_MIN;
+        for (size_t p = 0; p < q; ++p) {
+            const double t = std::floor(data[p] / delta + 0.5);
+            if (!(std::fabs(t) < 9.0e18)) return limit + 1;          // delta far too small
+            lev[p] = (int64_t)t;
+            lo = std::min(lo, lev[p]); hi = std::max(hi, lev[p]);
+        }
+        const uint64_t span = (uint64_t)(hi - lo) + 1;
+        if (span <= ((uint64_t)1 << 26)) {
+            seen.assign(span, 0);
+            uint64_t count = 0;
+            for (size_t p = 0; p < q; ++p) {
+                unsigned char& s = seen[(size_t)(lev[p] - lo)];
+                if (!s) { s = 1; if (++count > limit) return count; }
+            }
+            return count;
+        }
+        std::vector<int64_t> sorted(lev);
+        std::sort(sorted.begin(), sorted.end());
+        return (uint64_t)(std::unique(sorted.begin(), sorted.end()) - sorted.begin());
+    };
+    double a = 0.0, b = 4.0 * amax;
+    for (int it = 0; it < 70; ++it) {
+        const double mid = 0.5 * (a + b);
+        if (distinct_levels(mid, k) <= k) b = mid; else a = mid;
+    }
+    const double delta = b;
+    int64_t lo = INT64_MAX, hi = INT64_MIN;
+    for (size_t p = 0; p < q; ++p) {
+        lev[p] = (int64_t)std::floor(data[p] / delta + 0.5);
+        lo = std::min(lo, lev[p]); hi = std::max(hi, lev[p]);
+    }
+    const uint64_t span = (uint64_t)(hi - lo) + 1;
+    if (span > ((uint64_t)1 << 26)) return HAC_ERR_K_TOO_LARGE;
+    out.level_value.resize(span);
+    for (uint64_t l = 0; l < span; ++l) {
+        volatile double v = (double)(lo + (int64_t)l) * delta;
+        out.level_value[l] = (float)v;
+    }
+    out.level_of.resize(q);
+    for (size_t p = 0; p < q; ++p) out.level_of[p] = (uint32_t)(lev[p] - lo);
+    return HAC_OK;
+}
+
 int share_none(const std::vector<double>& data, Shared& out) {
     std::vector<double> distinct(data);
     std::sort(distinct.begin(), distinct.end());
@@ -319,9 +382,9 @@ int build_impl(const float* W, int64_t n, int64_t m, int64_t ldw, const hac_buil
                       bool sparse, Format& f) {
     if (!W || !p || n < 1 || m < 1 || ldw < m) return HAC_ERR_INVALID_ARG;
     if (!(p->sparsity >= 0.0 && p->sparsity < 1.0) || p->reserved != 0) return HAC_ERR_INVALID_ARG;
-    if (p->quantizer > HAC_QUANT_UNIFORM) return HAC_ERR_INVALID_ARG;
+    if (p->quantizer > HAC_QUANT_GRID) return HAC_ERR_INVALID_ARG;
     if (p->quantizer == HAC_QUANT_KMEANS && p->k < 1) return HAC_ERR_INVALID_ARG;
-    if (p->quantizer == HAC_QUANT_UNIFORM && p->k < 2) return HAC_ERR_INVALID_ARG;
+    if ((p->quantizer == HAC_QUANT_UNIFORM || p->quantizer == HAC_QUANT_GRID) && p->k < 2) return HAC_ERR_INVALID_ARG;
     if (p->seg_symbols > HAC_MAX_SEG_SYMBOLS) return HAC_ERR_INVALID_ARG;
     if (p->ri_bits != 0 && p->ri_bits != 16 && p->ri_bits != 32) return HAC_ERR_INVALID_ARG;
     if (n > (int64_t)1 << 31 || m > (int64_t)1 << 31 || n * m > ((int64_t)1 << 36))
@@ -382,6 +445,7 @@ int build_impl(const float* W, int64_t n, int64_t m, int64_t ldw, const hac_buil
         int rc = HAC_OK;
         if (p->quantizer == HAC_QUANT_KMEANS) rc = share_kmeans(data, p->k, p->kmeans_iters, p->seed, sh);
         else if (p->quantizer == HAC_QUANT_UNIFORM) rc = share_uniform(data, p->k, sh);
+        else if (p->quantizer == HAC_QUANT_GRID) rc = share_grid(data, p->k, sh);
         else rc = share_none(data, sh);
         if (rc != HAC_OK) return rc;
     }

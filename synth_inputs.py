@@ -20,6 +20,7 @@ import numpy as np
 QUANT_NONE = 0
 QUANT_KMEANS = 1
 QUANT_UNIFORM = 2
+QUANT_GRID = 3
 
 
 @dataclasses.dataclass(frozen=True)

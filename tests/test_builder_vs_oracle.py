@@ -55,6 +55,9 @@ CASES = [
     (si.scaled(si.CFG3_FC_SHAC, 3000, 96), "shac", 3),        # several segments per column
     (si.scaled(si.CFG4_CONV, 460, 64), "shac", 0),
     (si.scaled(si.CFG4_CONV, 460, 64), "hac", 16),
+    (dataclasses.replace(si.scaled(si.CFG2_DENSE_HAC, 300, 70), quantizer=si.QUANT_GRID, k=64), "hac", 0),
+    (dataclasses.replace(si.scaled(si.CFG3_FC_SHAC, 3000, 96), quantizer=si.QUANT_GRID, k=9), "shac", 0),
+    (dataclasses.replace(si.scaled(si.CFG4_CONV, 460, 64), quantizer=si.QUANT_GRID, k=2), "hac", 16),
 ]
 
 

@@ -188,3 +188,48 @@ def test_uniform_on_pruned_matrix_keeps_zeros():
     assert np.array_equal(mask, Wp != 0)
     assert np.all(Wq[~mask] == 0)
     assert Wq[mask].min() == Wp[mask].min() and Wq[mask].max() == Wp[mask].max()
+
+
+# ---------------------------------------------------------------- zero-anchored grid (Sect. III-C.3 as printed, d = 0)
+def test_grid_levels_round_half_up_on_a_hand_example():
+    data = np.array([0.26, -0.26, 0.74, 0.75, -0.75, 1.0, 0.24, -0.25])
+    # w / 0.5 = 0.52 -0.52 1.48 1.5 -1.5 2.0 0.48 -0.5 ; nearest integer, halves upwards
+    assert orc.grid_levels(data, 0.5).tolist() == [1, -1, 1, 2, -1, 2, 0, 0]
+
+
+@pytest.mark.parametrize("k", [2, 3, 16, 256])
+def test_grid_share_invariants(k):
+    rng = np.random.default_rng(100 + k)
+    W = rng.standard_normal((96, 40)).astype(np.float32)
+    Wq, mask = orc.grid_share(W, k)
+    data = W.T[mask.T].astype(np.float64)
+    delta = orc.grid_delta(data, k)
+    assert mask.all() and len(np.unique(Wq)) <= k
+    levels = Wq.astype(np.float64) / delta
+    assert np.abs(levels - np.round(levels)).max() < 1e-4                 # multiples of delta: the grid passes through 0
+    err = np.abs(Wq.astype(np.float64) - W.astype(np.float64))
+    assert err.max() <= delta / 2 + np.spacing(np.float32(np.abs(W).max()))
+    # delta is tuned: the next smaller double already leaves more than k values
+    assert len(np.unique(orc.grid_levels(data, delta))) <= k
+    assert len(np.unique(orc.grid_levels(data, np.nextafter(delta, 0.0)))) > k
+    # and it sits where some weight crosses a rounding boundary: delta = |w| / (t - 1/2), t = 1, 2, ..
+    t = np.round(np.abs(data) / delta + 0.5)
+    t = t[t >= 1]
+    cand = np.abs(data)[np.round(np.abs(data) / delta + 0.5) >= 1] / (t - 0.5)
+    assert np.min(np.abs(cand - delta)) <= 4 * np.spacing(delta)
+
+
+def test_grid_share_small_weights_become_stored_zeros_and_symmetry_holds():
+    rng = np.random.default_rng(7)
+    half = rng.standard_normal(300).astype(np.float32)
+    W = np.concatenate([half, -half]).reshape(20, 30)
+    Wp = orc.prune(W, 0.25)
+    Wq, mask = orc.grid_share(Wp, 5)
+    assert np.array_equal(mask, Wp != 0)
+    assert np.all(Wq[~mask] == 0)
+    assert np.any((Wq == 0) & mask)                     # survivors below delta/2 round to 0 but stay stored entries
+    assert np.array_equal(np.unique(Wq), -np.unique(Wq)[::-1])
+    # few distinct values: kept as they are
+    V = np.array([[0.5, -1.25, 0.0], [3.0, 0.5, 3.0]], dtype=np.float32)
+    Vq, vm = orc.grid_share(V, 4)
+    assert np.array_equal(Vq, V) and np.array_equal(vm, V != 0)
