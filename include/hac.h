@@ -52,6 +52,9 @@ extern "C" {
 #define HAC_QUANT_UNIFORM  2u   /* UQ,  Sect. III-C.3, grid over [min, max] of the non-null weights */
 #define HAC_QUANT_GRID     3u   /* UQ as printed in Sect. III-C.3 with d = 0: w = delta * round(w / delta),
                                    delta tuned by bisection to leave at most k distinct values          */
+#define HAC_QUANT_PWS      4u   /* PWS, Sect. III-C.2: k representatives at the i/(k-1) quantiles of the non-null
+                                   weights; a weight between two of them goes to the upper one with probability
+                                   (w - lo)/(hi - lo), drawn with SplitMix64 from `seed` and the weight's position */
 
 typedef struct hac_format  hac_format;    /* HAC : stream, codebook, code lengths, offset index          */
 typedef struct shac_format shac_format;   /* sHAC: stream of nz, ri, cb, codebook, lengths, offset index */
@@ -65,7 +68,7 @@ typedef struct hac_build_params {
     uint32_t seg_symbols;   /* S: symbols per sub-segment of the offset index, 1..HAC_MAX_SEG_SYMBOLS;
                                0 = default: 64 for HAC; for sHAC about (entries of the fullest column)/64,
                                rounded up so that S * ri_bits / 32 is odd (reported by *_sizes)         */
-    uint64_t seed;          /* seed of the k-means initialisation                                       */
+    uint64_t seed;          /* seed of the k-means initialisation and of the draws of PWS               */
     uint32_t ri_bits;       /* sHAC: width of a stored row index, 16 or 32; 0 = 16 if n <= 65536 else 32
                                (the footnote of Sect. IV-A: ri needs only ceil(log n) bits)             */
     uint32_t reserved;      /* must be 0                                                                */
@@ -140,7 +143,10 @@ typedef struct shac_host_view {
  * replaced by one of k shared values (k-means over them in column-major order, a uniform grid over
  * their range, or the zero-anchored grid delta * round(w / delta) whose delta is found by 70 halvings
  * of [0, 4 max|w|]: a trial delta that leaves at most k distinct values becomes the upper end, the
- * upper end is used; weights with at most k distinct values are kept as they are); distinct values sorted ascending form the codebook; a Huffman code over the
+ * upper end is used; or probabilistic sharing between the two neighbouring i/(k-1) quantiles, the
+ * i-th quantile being the order statistic floor(i (q-1)/(k-1)) of the q non-null weights and weight
+ * p using the uniform number (SplitMix64(seed + (p+1) * 0x9E3779B97F4A7C15) >> 11) * 2^-53; weights
+ * with at most k distinct values are kept as they are); distinct values sorted ascending form the codebook; a Huffman code over the
  * symbol counts (HAC: every entry, zeros included; sHAC: stored entries only) is made canonical;
  * code words are concatenated column by column, most significant bit first, into 32-bit words.
  * Offset index (the column-offset vector suggested in the paper's conclusions, refined): each column

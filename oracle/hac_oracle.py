@@ -88,7 +88,7 @@ def prune(W: np.ndarray, sparsity: float) -> np.ndarray:
 # ----------------------------------------------------------------------------
 # SplitMix64 (Steele, Lea, Flood, "Fast splittable pseudorandom number
 # generators", OOPSLA 2014), used as a counter-based generator: the i-th draw
-# mixes seed + (i + 1) * gamma.  Only the k-means initialisation draws numbers.
+# mixes seed + (i + 1) * gamma.  The k-means initialisation and PWS draw numbers.
 # ----------------------------------------------------------------------------
 _M64 = (1 << 64) - 1
 
@@ -232,6 +232,47 @@ def grid_share(Wp: np.ndarray, k: int):
     return _scatter_colmajor(mask, values), mask
 
 
+def splitmix64_many(seed: int, count: int) -> np.ndarray:
+    """splitmix64(seed, i) for i = 0 .. count-1 (uint64 arithmetic wraps, as the generator wants)."""
+    with np.errstate(over="ignore"):
+        z = np.uint64(seed & _M64) + (np.arange(count, dtype=np.uint64) + np.uint64(1)) * np.uint64(0x9E3779B97F4A7C15)
+        z = (z ^ (z >> np.uint64(30))) * np.uint64(0xBF58476D1CE4E5B9)
+        z = (z ^ (z >> np.uint64(27))) * np.uint64(0x94D049BB133111EB)
+        return z ^ (z >> np.uint64(31))
+
+
+def pws_extremes(data: np.ndarray, k: int) -> np.ndarray:
+    """The k representatives of PWS (Sect. III-C.2): the extremes of k - 1 intervals that hold equal
+    shares of the weights, i.e. the i/(k-1) quantiles, i = 0 .. k-1, taken as order statistics
+    s[floor(i (q-1) / (k-1))] of the sorted weights; equal ones are listed once."""
+    srt = np.sort(data)
+    q = len(srt)
+    pos = [(i * (q - 1)) // (k - 1) for i in range(k)]
+    return np.unique(srt[pos])
+
+
+def pws_share(Wp: np.ndarray, k: int, seed: int):
+    """PWS (Sect. III-C.2): a weight w inside the interval [lo, hi) of two neighbouring representatives
+    becomes hi with probability (w - lo) / (hi - lo) and lo otherwise, which makes the result an
+    unbiased estimate of w.  Weight p (column-major position among the non-null weights) uses the
+    uniform number (splitmix64(seed, p) >> 11) * 2^-53.  Weights with at most k distinct values
+    are kept as they are.  Returns (Wq, mask)."""
+    data, mask = _nonnull_colmajor(Wp)
+    if k < 2:
+        raise ValueError("PWS needs k >= 2")
+    if data.size == 0:
+        return np.zeros_like(Wp), mask
+    if len(np.unique(data)) <= k:
+        return _scatter_colmajor(mask, data.astype(np.float32)), mask
+    ext = pws_extremes(data, k)
+    j = np.clip(np.searchsorted(ext, data, side="right") - 1, 0, len(ext) - 2)
+    lo, hi = ext[j], ext[j + 1]
+    p_hi = (data - lo) / (hi - lo)
+    u = (splitmix64_many(seed, len(data)) >> np.uint64(11)).astype(np.float64) * np.float64(2.0 ** -53)
+    values = np.where(u < p_hi, hi, lo).astype(np.float32)
+    return _scatter_colmajor(mask, values), mask
+
+
 def share_none(Wp: np.ndarray):
     """No weight sharing: the matrix already holds few distinct values."""
     Wq = Wp.copy()
@@ -242,7 +283,7 @@ def share_none(Wp: np.ndarray):
 def quantize(W: np.ndarray, sparsity: float, k: int, quantizer: int, iters: int = 20, seed: int = 0):
     """Pruning then weight sharing, as chained in Sect. III-C.1.  quantizer:
     0 none, 1 k-means (CWS), 2 uniform (UQ over [min, max]), 3 uniform (UQ on the zero-anchored
-    grid of the printed formula).  Returns (Wq, mask)."""
+    grid of the printed formula), 4 probabilistic (PWS).  Returns (Wq, mask)."""
     Wp = prune(W, sparsity)
     if quantizer == 0:
         return share_none(Wp)
@@ -252,6 +293,8 @@ def quantize(W: np.ndarray, sparsity: float, k: int, quantizer: int, iters: int 
         return uniform_share(Wp, k)
     if quantizer == 3:
         return grid_share(Wp, k)
+    if quantizer == 4:
+        return pws_share(Wp, k, seed)
     raise ValueError("unknown quantizer")
 
 

@@ -1,7 +1,7 @@
 """HAC / sHAC compressed-domain products on NVIDIA B200: Python binding of libhac_b200.so.
 
 The functions carry the names of the C ABI (include/hac.h) and only marshal arguments."""
-from .binding import (Format, HacError, QUANT_GRID, QUANT_KMEANS, QUANT_NONE, QUANT_UNIFORM, EXPORTS, load,
+from .binding import (Format, HacError, QUANT_GRID, QUANT_KMEANS, QUANT_NONE, QUANT_PWS, QUANT_UNIFORM, EXPORTS, load,
                       library_path)
 
 
@@ -27,5 +27,5 @@ def shac_dot(fmt: Format, x, y=None, workspace=None, layout="nb"):
     return fmt.dot(x, y, workspace, layout)
 
 
-__all__ = ["Format", "HacError", "QUANT_NONE", "QUANT_KMEANS", "QUANT_UNIFORM", "QUANT_GRID", "EXPORTS", "load",
+__all__ = ["Format", "HacError", "QUANT_NONE", "QUANT_KMEANS", "QUANT_UNIFORM", "QUANT_GRID", "QUANT_PWS", "EXPORTS", "load",
            "library_path", "hac_build", "shac_build", "hac_dot", "shac_dot"]

@@ -10,7 +10,7 @@ import numpy as np
 
 from . import build as _build
 
-QUANT_NONE, QUANT_KMEANS, QUANT_UNIFORM, QUANT_GRID = 0, 1, 2, 3
+QUANT_NONE, QUANT_KMEANS, QUANT_UNIFORM, QUANT_GRID, QUANT_PWS = 0, 1, 2, 3, 4
 
 
 class HacError(RuntimeError):

@@ -171,6 +171,38 @@ int share_grid(const std::vector<double>& data, uint32_t k, Shared& out) {
     return HAC_OK;
 }
 
+// Sect. III-C.2 (PWS): k representatives at the i/(k-1) quantiles (order statistics of the sorted
+// weights); a weight between two neighbouring ones becomes the upper one with probability
+// (w - lo)/(hi - lo), else the lower one.  One uniform number per weight, from its position.
+int share_pws(const std::vector<double>& data, uint32_t k, uint64_t seed, Shared& out) {
+    const size_t q = data.size();
+    std::vector<double> srt(data);
+    std::sort(srt.begin(), srt.end());
+    {
+        std::vector<double> distinct(srt);
+        distinct.erase(std::unique(distinct.begin(), distinct.end()), distinct.end());
+        if (distinct.size() <= k) return share_none(data, out);
+    }
+    std::vector<double> ext(k);
+    for (uint32_t i = 0; i < k; ++i) ext[i] = srt[(size_t)(((uint64_t)i * (uint64_t)(q - 1)) / (uint64_t)(k - 1))];
+    ext.erase(std::unique(ext.begin(), ext.end()), ext.end());
+    std::vector<double>().swap(srt);
+    const size_t r = ext.size();
+    out.level_value.resize(r);
+    for (size_t l = 0; l < r; ++l) out.level_value[l] = (float)ext[l];
+    out.level_of.resize(q);
+    for (size_t p = 0; p < q; ++p) {
+        const double w = data[p];
+        size_t j = (size_t)(std::upper_bound(ext.begin(), ext.end(), w) - ext.begin());    // extremes <= w
+        j = j == 0 ? 0 : j - 1;
+        if (j > r - 2) j = r - 2;
+        const double p_hi = (w - ext[j]) / (ext[j + 1] - ext[j]);
+        const double u = (double)(splitmix64_at(seed, (uint64_t)p) >> 11) * 0x1.0p-53;
+        out.level_of[p] = (uint32_t)(u < p_hi ? j + 1 : j);
+    }
+    return HAC_OK;
+}
+
 int share_none(const std::vector<double>& data, Shared& out) {
     std::vector<double> distinct(data);
     std::sort(distinct.begin(), distinct.end());
@@ -382,9 +414,9 @@ int build_impl(const float* W, int64_t n, int64_t m, int64_t ldw, const hac_buil
                       bool sparse, Format& f) {
     if (!W || !p || n < 1 || m < 1 || ldw < m) return HAC_ERR_INVALID_ARG;
     if (!(p->sparsity >= 0.0 && p->sparsity < 1.0) || p->reserved != 0) return HAC_ERR_INVALID_ARG;
-    if (p->quantizer > HAC_QUANT_GRID) return HAC_ERR_INVALID_ARG;
+    if (p->quantizer > HAC_QUANT_PWS) return HAC_ERR_INVALID_ARG;
     if (p->quantizer == HAC_QUANT_KMEANS && p->k < 1) return HAC_ERR_INVALID_ARG;
-    if ((p->quantizer == HAC_QUANT_UNIFORM || p->quantizer == HAC_QUANT_GRID) && p->k < 2) return HAC_ERR_INVALID_ARG;
+    if (p->quantizer >= HAC_QUANT_UNIFORM && p->k < 2) return HAC_ERR_INVALID_ARG;
     if (p->seg_symbols > HAC_MAX_SEG_SYMBOLS) return HAC_ERR_INVALID_ARG;
     if (p->ri_bits != 0 && p->ri_bits != 16 && p->ri_bits != 32) return HAC_ERR_INVALID_ARG;
     if (n > (int64_t)1 << 31 || m > (int64_t)1 << 31 || n * m > ((int64_t)1 << 36))
@@ -446,6 +478,7 @@ int build_impl(const float* W, int64_t n, int64_t m, int64_t ldw, const hac_buil
         if (p->quantizer == HAC_QUANT_KMEANS) rc = share_kmeans(data, p->k, p->kmeans_iters, p->seed, sh);
         else if (p->quantizer == HAC_QUANT_UNIFORM) rc = share_uniform(data, p->k, sh);
         else if (p->quantizer == HAC_QUANT_GRID) rc = share_grid(data, p->k, sh);
+        else if (p->quantizer == HAC_QUANT_PWS) rc = share_pws(data, p->k, p->seed, sh);
         else rc = share_none(data, sh);
         if (rc != HAC_OK) return rc;
     }

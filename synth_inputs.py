@@ -21,6 +21,7 @@ QUANT_NONE = 0
 QUANT_KMEANS = 1
 QUANT_UNIFORM = 2
 QUANT_GRID = 3
+QUANT_PWS = 4
 
 
 @dataclasses.dataclass(frozen=True)

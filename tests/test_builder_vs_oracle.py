@@ -58,6 +58,9 @@ CASES = [
     (dataclasses.replace(si.scaled(si.CFG2_DENSE_HAC, 300, 70), quantizer=si.QUANT_GRID, k=64), "hac", 0),
     (dataclasses.replace(si.scaled(si.CFG3_FC_SHAC, 3000, 96), quantizer=si.QUANT_GRID, k=9), "shac", 0),
     (dataclasses.replace(si.scaled(si.CFG4_CONV, 460, 64), quantizer=si.QUANT_GRID, k=2), "hac", 16),
+    (dataclasses.replace(si.scaled(si.CFG2_DENSE_HAC, 300, 70), quantizer=si.QUANT_PWS, k=64), "hac", 0),
+    (dataclasses.replace(si.scaled(si.CFG3_FC_SHAC, 3000, 96), quantizer=si.QUANT_PWS, k=2), "shac", 0),
+    (dataclasses.replace(si.scaled(si.CFG4_CONV, 460, 64), quantizer=si.QUANT_PWS, k=17), "shac", 5),
 ]
 
 

@@ -69,7 +69,7 @@ SMALL = [
     (si.scaled(si.CFG4_CONV, 1152, 128), "shac", 0, (1, 200)),
     (si.scaled(si.CFG4_CONV, 1152, 128), "hac", 0, (1, 200)),
     (dataclasses.replace(si.scaled(si.CFG4_CONV, 1152, 128), quantizer=si.QUANT_GRID, k=33), "shac", 0, (1, 12)),
-    (dataclasses.replace(si.scaled(si.CFG2_DENSE_HAC, 900, 140), quantizer=si.QUANT_GRID, k=200), "hac", 0, (1, 70)),
+    (dataclasses.replace(si.scaled(si.CFG2_DENSE_HAC, 900, 140), quantizer=si.QUANT_GRID, k=200), "hac", 0, (1, 70)),    (dataclasses.replace(si.scaled(si.CFG3_FC_SHAC, 5000, 150), quantizer=si.QUANT_PWS, k=32), "shac", 0, (1, 7)),
 ]
 
 

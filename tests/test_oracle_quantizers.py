@@ -233,3 +233,65 @@ def test_grid_share_small_weights_become_stored_zeros_and_symmetry_holds():
     V = np.array([[0.5, -1.25, 0.0], [3.0, 0.5, 3.0]], dtype=np.float32)
     Vq, vm = orc.grid_share(V, 4)
     assert np.array_equal(Vq, V) and np.array_equal(vm, V != 0)
+
+
+# ---------------------------------------------------------------- PWS (Sect. III-C.2)
+def test_splitmix64_many_equals_the_scalar_generator():
+    for seed in (0, 1234567, (1 << 64) - 5):
+        assert orc.splitmix64_many(seed, 50).tolist() == [orc.splitmix64(seed, i) for i in range(50)]
+
+
+def test_pws_two_values_is_the_two_point_law_of_the_paper():
+    # k = 2: every weight becomes min or max, the maximum with probability (w - min) / (max - min)
+    rng = np.random.default_rng(11)
+    W = rng.uniform(-1.0, 3.0, size=(30, 20)).astype(np.float32)
+    lo, hi = np.float64(W.min()), np.float64(W.max())
+    ups = np.zeros(W.shape)
+    trials = 400
+    for seed in range(trials):
+        Wq, mask = orc.pws_share(W, 2, seed)
+        assert set(np.unique(Wq).tolist()) <= {float(W.min()), float(W.max())}
+        ups += Wq == W.max()
+    p = (W.astype(np.float64) - lo) / (hi - lo)
+    # frequencies within 5 standard deviations of the law, and the estimate is unbiased on average
+    assert np.all(np.abs(ups / trials - p) <= 5 * np.sqrt(p * (1 - p) / trials) + 1e-12)
+    est = lo + (hi - lo) * ups / trials
+    assert abs(float((est - W).mean())) < 5 * (hi - lo) * 0.5 / np.sqrt(trials * W.size)
+
+
+@pytest.mark.parametrize("k", [3, 8, 64])
+def test_pws_values_bracket_the_weight_and_representatives_are_quantiles(k):
+    rng = np.random.default_rng(k)
+    W = rng.standard_normal((120, 50)).astype(np.float32)
+    Wq, mask = orc.pws_share(W, k, seed=5)
+    data = np.sort(W.ravel().astype(np.float64))
+    q = data.size
+    ext = np.unique([data[(i * (q - 1)) // (k - 1)] for i in range(k)])
+    assert ext[0] == data[0] and ext[-1] == data[-1] and len(ext) <= k
+    assert np.array_equal(orc.pws_extremes(W.T.ravel().astype(np.float64), k), ext)
+    assert set(np.unique(Wq).tolist()) <= set(ext.astype(np.float32).tolist())
+    # the two neighbours of w among the representatives, by brute force
+    w64, q64 = W.astype(np.float64).ravel(), Wq.astype(np.float64).ravel()
+    for w, v in zip(w64[::37], q64[::37]):
+        below = ext[ext <= w].max()
+        above = ext[ext > w].min() if (ext > w).any() else ext[-1]
+        assert np.float32(v) in (np.float32(below), np.float32(above))
+    # a representative is reproduced exactly
+    hit = np.isin(w64, ext)
+    assert np.array_equal(q64[hit].astype(np.float32), w64[hit].astype(np.float32))
+    # the intervals between neighbouring representatives hold equal shares of the weights
+    shares = np.array([((data >= a) & (data < b)).sum() for a, b in zip(ext[:-1], ext[1:])])
+    assert np.all(np.abs(shares - (q - 1) / (k - 1)) <= 1.0)
+    # same seed, same result; another seed, another draw
+    assert np.array_equal(orc.pws_share(W, k, seed=5)[0], Wq)
+    assert not np.array_equal(orc.pws_share(W, k, seed=6)[0], Wq)
+
+
+def test_pws_with_256_values_codes_at_8_bits_like_the_papers_table():
+    # equiprobable representatives: Huffman lengths close to log2 k, the occupancy 0.2500 = 8/32 the paper
+    # reports for PWS at k = 256 on dense layers
+    rng = np.random.default_rng(3)
+    W = rng.standard_normal((512, 256)).astype(np.float32)
+    Wq, mask = orc.pws_share(W, 256, seed=1)
+    fmt = orc.hac_encode(Wq)
+    assert 7.9 <= fmt["bits"] / W.size <= 8.05
