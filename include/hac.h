@@ -192,7 +192,8 @@ int shac_attach(shac_format* f, void* dev_buf, size_t dev_bytes);
  *       y[b*y_stride_b + j*y_stride_j] = sum_i W[i][j] * x[b*x_stride_b + i*x_stride_i]
  * for b in [0, batch), j in [0, m).  x, y: device fp32; strides in elements, so X may be stored
  * [batch][n] or [n][batch] and Y [batch][m] or [m][batch]; the batched kernels are fastest with
- * x_stride_b == 1 and y_stride_b == 1.  x and y must not overlap.  Code words are decoded on the
+ * x_stride_b == 1 and y_stride_b == 1 (a HAC format built with sub-segments of several hundred symbols does
+ * not fit the batched kernel's buffers and is then multiplied input by input).  x and y must not overlap.  Code words are decoded on the
  * fly; the uncompressed weights are never written to global memory.  Products and sums are fp32.
  *   workspace  device scratch of at least *_workspace_bytes(f, batch) bytes, 16-byte aligned (may be
  *              NULL when that is 0).  It holds partial sums of columns that span several segments

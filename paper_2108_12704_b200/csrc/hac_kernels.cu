@@ -1717,7 +1717,10 @@ static size_t task_off_bytes(const Format& f, int64_t batch) {
 // Workspace of one product: [partial sums, rounded up to 256 bytes][B tiles][task start bits].
 static size_t workspace_bytes(const Format& f, int64_t batch) {
     const size_t xp = xpack_bytes(f, batch);
-    return xp ? ((partial_bytes(f, batch) + 255) & ~(size_t)255) + xp + task_off_bytes(f, batch) : partial_bytes(f, batch);
+    if (!xp) return partial_bytes(f, batch);
+    // never less than a single-input product needs: a batch falls back to those when the tensor-core kernel
+    // cannot hold the format's sub-segments
+    return std::max(((partial_bytes(f, batch) + 255) & ~(size_t)255) + xp + task_off_bytes(f, batch), partial_bytes(f, 1));
 }
 
 static int env_int(const char* name, int fallback) {
@@ -1958,6 +1961,17 @@ static int dot(const Format& f, const float* x, int64_t batch, int64_t xs_i, int
             if (!f.sparse) {
                 unsigned char* xpack = static_cast<unsigned char*>(workspace) + ((partial_bytes(f, batch) + 255) & ~(size_t)255);
                 rc = launch_gemm_tc(f, di, d, x, xs_i, xs_b, batch, y, ys_j, ys_b, partial, xpack, st, &gemm_splits);
+                if (rc == HAC_ERR_BUFFER_TOO_SMALL) {
+                    // Sub-segments too long for the per-lane stream buffers of the tensor-core kernel (a very
+                    // large S): one single-input product per input instead.  Slow, but every format works.
+                    rc = HAC_OK;
+                    for (int64_t b = 0; b < batch && rc == HAC_OK; ++b) {
+                        bool wrote_y = false;
+                        rc = launch_vec(f, 0, x + b * xs_b, xs_i, y + b * ys_b, ys_j, partial, st, &wrote_y);
+                        if (rc == HAC_OK && f.G > 1 && !wrote_y)
+                            rc = launch_finalize(f, d, partial, 1, y + b * ys_b, ys_j, 0, st, 1);
+                    }
+                }
             } else {
                 const int acc = (int)std::min<int64_t>(kAccMax, (batch + 31) / 32);
                 switch (acc) {

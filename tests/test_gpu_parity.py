@@ -70,6 +70,8 @@ SMALL = [
     (si.scaled(si.CFG4_CONV, 1152, 128), "hac", 0, (1, 200)),
     (dataclasses.replace(si.scaled(si.CFG4_CONV, 1152, 128), quantizer=si.QUANT_GRID, k=33), "shac", 0, (1, 12)),
     (dataclasses.replace(si.scaled(si.CFG2_DENSE_HAC, 900, 140), quantizer=si.QUANT_GRID, k=200), "hac", 0, (1, 70)),    (dataclasses.replace(si.scaled(si.CFG3_FC_SHAC, 5000, 150), quantizer=si.QUANT_PWS, k=32), "shac", 0, (1, 7)),
+    (si.scaled(si.CFG2_DENSE_HAC, 3000, 40), "hac", 1024, (1, 3)),       # largest S: the batch runs input by input
+    (si.scaled(si.CFG2_DENSE_HAC, 40000, 12), "hac", 512, (1, 2)),       # and with several segments per column
 ]
 
 
