@@ -1662,6 +1662,14 @@ static int attach(Format& f, void* dev_buf, size_t dev_bytes) {
 // Tasks of the batched HAC kernel: sub-segments (S rows) of a column.
 static uint32_t gemm_tasks(const Format& f) { return f.S ? (uint32_t)((f.n + f.S - 1) / f.S) : 0u; }
 
+// Whether the single-input sHAC kernel can hold the format: it stages two segments' spans and slices of
+// ri per warp, which a very large S with 32-bit row indices can push past the shared memory of an SM
+// (227 KB on sm_100); such formats take the batched kernel for a single input too.
+static bool shac_vec_fits(const Format& f) {
+    const size_t per_warp = ((size_t)f.max_unit_chunks * 16 + ((size_t)(32u * f.S * (f.ri_bits / 8) + 15u) / 16u + 1u) * 16u) * 2;
+    return 16 + plan_smem_bytes((uint32_t)f.tables.l1_bits, 0, (uint32_t)(f.tables.sub.size() * 4)) + per_warp <= (size_t)232448;
+}
+
 static size_t partial_bytes(const Format& f, int64_t batch) {
     // batched HAC: one partial per row split of the product kernel
     if (!f.sparse && batch > 1) {
@@ -1670,7 +1678,7 @@ static size_t partial_bytes(const Format& f, int64_t batch) {
     }
     // sHAC with one input handles up to two segments of a column in one warp; the batched sHAC kernel
     // and HAC with one input keep one partial per segment
-    const bool partials = f.sparse ? f.max_units_per_col > (batch == 1 ? 2u : 1u) : f.G > 1;
+    const bool partials = f.sparse ? f.max_units_per_col > ((batch == 1 && shac_vec_fits(f)) ? 2u : 1u) : f.G > 1;
     return partials ? f.seg_bit_off.size() * (size_t)batch * 4 : 0;
 }
 
@@ -1951,9 +1959,16 @@ static int dot(const Format& f, const float* x, int64_t batch, int64_t xs_i, int
     int rc = HAC_OK;
     bool direct = false;                     // the product kernel wrote every output itself
     uint32_t gemm_splits = 0;                // batched HAC: row splits used (1 = outputs written directly)
+    bool wide_single = false;                // sHAC, one input, through the batched kernel (see shac_vec_fits)
     if (d.units > 0) {
-        if (batch == 1) {
+        if (batch == 1 && (!f.sparse || shac_vec_fits(f))) {
             rc = launch_vec(f, 0, x, xs_i, y, ys_j, partial, st, &direct);
+        } else if (batch == 1) {
+            DeviceInfo di;
+            rc = device_info(di);
+            if (rc) return rc;
+            rc = launch_batch_t<1>(f, di, d, x, xs_i, xs_b, batch, y, ys_j, ys_b, partial, st);
+            wide_single = true;
         } else {
             DeviceInfo di;
             rc = device_info(di);
@@ -2001,7 +2016,7 @@ static int dot(const Format& f, const float* x, int64_t batch, int64_t xs_i, int
         finish = false;
     } else if (!f.sparse) {
         finish = f.G > 1 && !direct;
-    } else if (batch == 1) {
+    } else if (batch == 1 && !wide_single) {
         direct_up_to = 2;
         finish = f.max_units_per_col > 2 || f.has_empty_col;
     } else {

@@ -242,3 +242,16 @@ def test_chained_products_keep_stream_order():
             g = got.cpu().numpy()
             g = g[None] if B == 1 else g.T
             check_outputs(g, ref, a)
+
+
+def test_largest_sub_segments_with_wide_row_indices():
+    """S = 1024 with 32-bit row indices: two staged segments do not fit the shared memory of an SM, so a
+    single input goes through the batched kernel; the result must not change."""
+    wl = dataclasses.replace(si.scaled(si.CFG3_FC_SHAC, 70000, 6), sparsity=0.2, k=64)
+    lf, Wq, mask = build_both(wl, "shac", 1024)
+    assert lf.sizes()["ri_bits"] == 32
+    check_decode(lf, Wq, mask)
+    for B in (1, 3):
+        X = si.inputs(wl, B)
+        y_ref, a = orc.dot_definition(Wq, X)
+        check_outputs(run_dot(lf, X), y_ref, a)
