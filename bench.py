@@ -36,11 +36,13 @@ UNIT = "Gweights/s"
 L2_BYTES = 126 * 1024 * 1024
 GEMM_BATCH = 64
 FALLBACK_HBM_GBS = 6650.0
+MIN_TIMED_SECONDS = 0.5     # the K-step region is repeated until this much device time has been measured
+MAX_REPEATS = 4000
 
 
-# dram__bytes_read.sum + dram__bytes_write.sum per launch of the GEMV kernel from one ncu capture
-# (profiles/hac_vec_kernel_config2_gemv.md), valid only for the device code it was taken on.
-NCU_GEMV_TRAFFIC = {"bytes": 14614272, "kernel_source_sha256": "ee838ebffb4d5b73d2c37ed2f9a5797a446af2612ad2873648db3d6d7a6ef1cc"}
+# dram__bytes_read.sum + dram__bytes_write.sum per launch of the single-input kernels from ncu captures (profiles/), valid
+# only for the device code they were taken on (hash of the device part of hac_kernels.cu).
+NCU_TRAFFIC = {"kernel_source_sha256": "", "hac_gemv": None, "shac_gemv": None}
 
 
 def device_code(text: bytes) -> bytes:
@@ -49,15 +51,15 @@ def device_code(text: bytes) -> bytes:
     return text if cut < 0 else text[:cut]
 
 
-def gemv_traffic():
+def ncu_traffic(which):
     import hashlib
     src = os.path.join(ROOT, "paper_2108_12704_b200", "csrc", "hac_kernels.cu")
     try:
         with open(src, "rb") as f:
-            same = hashlib.sha256(device_code(f.read())).hexdigest() == NCU_GEMV_TRAFFIC["kernel_source_sha256"]
+            same = hashlib.sha256(device_code(f.read())).hexdigest() == NCU_TRAFFIC["kernel_source_sha256"]
     except OSError:
         same = False
-    return NCU_GEMV_TRAFFIC["bytes"] if same else None
+    return NCU_TRAFFIC[which] if same else None
 
 
 def measured_peaks():
@@ -257,6 +259,91 @@ def capture(torch, fn):
     return g
 
 
+def median(v):
+    return float(np.median(np.asarray(v, dtype=np.float64)))
+
+
+class Leg:
+    """One product (a format at a batch size) timed as CUDA graphs of K launches that rotate over the replicas of
+    the device image, so that every launch reads cold HBM."""
+
+    def __init__(self, torch, fmt, reps, xs, ys, ws, layout, K):
+        self.torch, self.fmt, self.reps, self.xs, self.ys, self.ws, self.layout = torch, fmt, reps, xs, ys, ws, layout
+        self.R, self.K = len(reps), K
+        self.launches_per_product = self.launch(0)
+        for i in range(3):
+            self.launch(i % self.R)
+        torch.cuda.synchronize()
+        full, rem = divmod(K, self.R)
+        self.full = full
+        self.g_full = capture(torch, lambda: [self.launch(r) for r in range(self.R)]) if full else None
+        self.g_rem = capture(torch, lambda: [self.launch(r) for r in range(rem)]) if rem else None
+        for g in (self.g_full, self.g_rem):
+            if g is not None:
+                g.replay()
+        torch.cuda.synchronize()
+
+    def launch(self, r):
+        self.fmt.attach(self.reps[r])
+        if self.layout is None:
+            self.fmt.dot(self.xs[r % len(self.xs)], self.ys[r % len(self.ys)], self.ws)
+        else:
+            self.fmt.dot(self.xs[r % len(self.xs)], self.ys[r % len(self.ys)], self.ws, layout=self.layout)
+        return self.fmt.last_launch_count()
+
+    def replay(self):
+        """Enqueues exactly K launches."""
+        for _ in range(self.full):
+            self.g_full.replay()
+        if self.g_rem is not None:
+            self.g_rem.replay()
+
+
+def time_regions(torch, legs, min_seconds, max_repeats, dist=None):
+    """Repeats the timed region (every leg's K launches, one leg after the other, CUDA events between the
+    legs on the launching stream, a synchronize on both sides) until `min_seconds` of device time have been
+    measured.  Returns per-leg lists of milliseconds per region and the list of whole-region milliseconds."""
+    per_leg = [[] for _ in legs]
+    whole = []
+    total = 0.0
+    while len(whole) < max_repeats and (total < min_seconds * 1e3 or len(whole) < 3):
+        ev = [torch.cuda.Event(enable_timing=True) for _ in range(len(legs) + 1)]
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize()
+        ev[0].record()
+        for i, leg in enumerate(legs):
+            leg.replay()
+            ev[i + 1].record()
+        torch.cuda.synchronize()
+        if dist is not None:
+            dist.barrier()
+        for i in range(len(legs)):
+            per_leg[i].append(ev[i].elapsed_time(ev[i + 1]))
+        whole.append(ev[0].elapsed_time(ev[-1]))
+        total += whole[-1]
+    return per_leg, whole
+
+
+def build_format(hb, kind, wl, dev, seg_symbols=0):
+    W = si.weights(wl)
+    fmt = hb.Format(kind, W, sparsity=wl.sparsity, k=wl.k, quantizer=wl.quantizer, kmeans_iters=wl.kmeans_iters,
+                    seed=wl.seed, seg_symbols=seg_symbols).upload(dev)
+    del W
+    return fmt
+
+
+def check_against_host_decode(fmt, X, Y, what):
+    """Guard before timing (not the parity test, which compares with the oracle under tests/): the product must
+    agree with a float64 product on the format's own host decode."""
+    Wq = fmt.decode_host().astype(np.float64)
+    X64 = X.astype(np.float64)
+    ref = X64 @ Wq
+    tol = 1e-5 * (np.abs(X64) @ np.abs(Wq)) + 1e-7
+    if not np.all(np.abs(Y.astype(np.float64) - ref) <= tol):
+        raise RuntimeError(f"{what}: result outside tolerance; refusing to time it")
+
+
 def run_ours(args):
     import torch
     import paper_2108_12704_b200 as hb
@@ -272,104 +359,44 @@ def run_ours(args):
         import torch.distributed as dist
         dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
     dev = torch.device("cuda", local_rank)
+    K, Wm = args.steps, max(args.warmup, 3)
 
+    # ---- workload of the metric: dense HAC, one input and a batch of 64 ---------------------------------------
     wl = si.CFG2_DENSE_HAC
-    S = int(os.environ.get("HAC_BENCH_SEG_SYMBOLS", "0"))
-    W = si.weights(wl)
-    fmt = hb.Format("hac", W, sparsity=wl.sparsity, k=wl.k, quantizer=wl.quantizer, kmeans_iters=wl.kmeans_iters,
-                    seed=wl.seed, seg_symbols=S).upload(dev)
+    fmt = build_format(hb, "hac", wl, dev, int(os.environ.get("HAC_BENCH_SEG_SYMBOLS", "0")))
     sizes = fmt.sizes()
     n, m = wl.n, wl.m
     lut_bits = min(12, sizes["max_code_len"])
     image_bytes = fmt.device_bytes()
     R = max(2, math.ceil(3 * L2_BYTES / image_bytes))
     reps = make_replicas(fmt, torch, R)
-
-    # inputs resident in HBM: one x and one X per replica slot, [n] and [n, B]
-    x1 = [torch.from_numpy(si.inputs(wl, 1, salt=r)[0]).to(dev) for r in range(R)]
+    x1_host = [si.inputs(wl, 1, salt=r)[0] for r in range(R)]
+    x1 = [torch.from_numpy(v).to(dev) for v in x1_host]
     xb_host = si.inputs(wl, GEMM_BATCH)
     xB = [torch.from_numpy(np.ascontiguousarray(xb_host.T)).to(dev) for _ in range(R)]
     y1 = [torch.empty(m, dtype=torch.float32, device=dev) for _ in range(R)]
     yB = [torch.empty((m, GEMM_BATCH), dtype=torch.float32, device=dev) for _ in range(R)]
-    ws_bytes = max(fmt.workspace_bytes(1), fmt.workspace_bytes(GEMM_BATCH), 16)
-    ws = torch.empty(ws_bytes, dtype=torch.uint8, device=dev)
-
-    launches = {"gemv": 0, "gemm": 0}
-
-    def gemv(r):
-        fmt.attach(reps[r])
-        fmt.dot(x1[r], y1[r], ws)
-        return fmt.last_launch_count()
-
-    def gemm(r):
-        fmt.attach(reps[r])
-        fmt.dot(xB[r], yB[r], ws, layout="nb")
-        return fmt.last_launch_count()
-
-    # parity spot check in this process before timing (one output column set against numpy fp64)
-    launches["gemv"] = gemv(0)
-    launches["gemm"] = gemm(0)
-    torch.cuda.synchronize()
-    Wq = fmt.decode_host().astype(np.float64)
-    ref1 = x1[0].cpu().numpy().astype(np.float64) @ Wq
-    tol1 = 1e-5 * (np.abs(x1[0].cpu().numpy().astype(np.float64)) @ np.abs(Wq)) + 1e-7
-    if not np.all(np.abs(y1[0].cpu().numpy() - ref1) <= tol1):
-        raise RuntimeError("GEMV result outside tolerance; refusing to time it")
-    refB = (xb_host.astype(np.float64) @ Wq).T
-    tolB = 1e-5 * (np.abs(xb_host.astype(np.float64)) @ np.abs(Wq)).T + 1e-7
-    if not np.all(np.abs(yB[0].cpu().numpy() - refB) <= tolB):
-        raise RuntimeError("GEMM result outside tolerance; refusing to time it")
-    del Wq
-
-    K, Wm = args.steps, args.warmup
-    chunk = R                                    # one graph = one rotation over the replicas
-
-    def graph_of(fn, count, start=0):
-        return capture(torch, lambda: [fn((start + i) % R) for i in range(count)])
-
-    for i in range(max(Wm, 3)):                  # warm-up steps, direct launches
-        gemv(i % R)
-        gemm(i % R)
-    torch.cuda.synchronize()
-    full, rem = divmod(K, chunk)
-    g_gemv = graph_of(gemv, chunk) if full else None
-    g_gemm = graph_of(gemm, chunk) if full else None
-    g_gemv_rem = graph_of(gemv, rem) if rem else None
-    g_gemm_rem = graph_of(gemm, rem) if rem else None
-    for g in (g_gemv, g_gemm, g_gemv_rem, g_gemm_rem):     # graph warm-up (upload of the executable graph)
-        if g is not None:
-            g.replay()
+    ws = torch.empty(max(fmt.workspace_bytes(1), fmt.workspace_bytes(GEMM_BATCH), 16), dtype=torch.uint8, device=dev)
+    leg_gemv = Leg(torch, fmt, reps, x1, y1, ws, None, K)
+    leg_gemm = Leg(torch, fmt, reps, xB, yB, ws, "nb", K)
+    check_against_host_decode(fmt, x1_host[0][None], y1[0].cpu().numpy()[None], "HAC GEMV")
+    check_against_host_decode(fmt, xb_host, yB[0].cpu().numpy().T, "HAC GEMM")
+    for i in range(Wm):                          # warm-up steps
+        leg_gemv.launch(i % R)
+        leg_gemm.launch(i % R)
     torch.cuda.synchronize()
 
-    e = [torch.cuda.Event(enable_timing=True) for _ in range(3)]
-    if dist is not None:
-        dist.barrier()
-    torch.cuda.synchronize()
     with ClockSampler(local_rank) as clocks:
-        e[0].record()
-        for _ in range(full):
-            g_gemv.replay()
-        if g_gemv_rem is not None:
-            g_gemv_rem.replay()
-        e[1].record()
-        for _ in range(full):
-            g_gemm.replay()
-        if g_gemm_rem is not None:
-            g_gemm_rem.replay()
-        e[2].record()
-        torch.cuda.synchronize()
-    if dist is not None:
-        dist.barrier()
-    t_gemv_ms = e[0].elapsed_time(e[1])
-    t_gemm_ms = e[1].elapsed_time(e[2])
-    t_total_ms = e[0].elapsed_time(e[2])
-
+        (t_gemv, t_gemm), t_whole = time_regions(torch, [leg_gemv, leg_gemm], MIN_TIMED_SECONDS, MAX_REPEATS, dist)
+    repeats = len(t_whole)
+    step_ms = median(t_whole) / K
     weights_per_step = float(n) * m * (1 + GEMM_BATCH)
-    job_ms, job_units = reduce_job(t_total_ms, weights_per_step * K, dist)
+    job_ms, job_units = reduce_job(step_ms, weights_per_step, dist)
     value = job_units / (job_ms * 1e-3) / 1e9
+    gemv_s = median(t_gemv) * 1e-3 / K
+    gemm_s = median(t_gemm) * 1e-3 / K
 
-    # end to end through the host entry point: pinned host X / Y, copies inside the timed region
-    Ke = min(K, 2000)
+    # ---- end to end through the host entry point: pinned host X / Y, copies inside the timed region ----------
     xh1 = torch.from_numpy(si.inputs(wl, 1)).pin_memory()
     yh1 = torch.empty((1, m), dtype=torch.float32).pin_memory()
     xhB = torch.from_numpy(xb_host).pin_memory()
@@ -381,15 +408,48 @@ def run_ours(args):
     torch.cuda.synchronize()
     if dist is not None:
         dist.barrier()
+    Ke = 0
     t0 = time.perf_counter()
-    for i in range(Ke):
-        fmt.attach(reps[i % R])
+    while Ke < K or time.perf_counter() - t0 < 0.3:
+        fmt.attach(reps[Ke % R])
         fmt.dot_host(xh1, yh1, scratch)
         fmt.dot_host(xhB, yhB, scratch)
+        Ke += 1
+        if Ke >= 20000:
+            break
     torch.cuda.synchronize()
     e2e_ms = (time.perf_counter() - t0) * 1e3
     e2e_job_ms, e2e_units = reduce_job(e2e_ms, weights_per_step * Ke, dist)
     e2e_value = e2e_units / (e2e_job_ms * 1e-3) / 1e9
+    hac_launches = leg_gemv.launches_per_product + leg_gemm.launches_per_product
+    del leg_gemv, leg_gemm, reps, x1, xB, y1, yB, scratch
+    torch.cuda.empty_cache()
+
+    # ---- the sHAC workload (large pruned fully connected layer), timed the same way, reported beside ----------
+    swl = si.CFG3_FC_SHAC
+    sfmt = build_format(hb, "shac", swl, dev)
+    ssizes = sfmt.sizes()
+    sR = max(2, math.ceil(3 * L2_BYTES / sfmt.device_bytes()))
+    sreps = make_replicas(sfmt, torch, sR)
+    sx1_host = [si.inputs(swl, 1, salt=r)[0] for r in range(sR)]
+    sx1 = [torch.from_numpy(v).to(dev) for v in sx1_host]
+    sy1 = [torch.empty(swl.m, dtype=torch.float32, device=dev) for _ in range(sR)]
+    sbatches = [b for b in swl.batches if b > 1]
+    sX_host = {b: si.inputs(swl, b) for b in sbatches}
+    sX = {b: [torch.from_numpy(np.ascontiguousarray(sX_host[b].T)).to(dev) for _ in range(min(sR, 8))] for b in sbatches}
+    sY = {b: [torch.empty((swl.m, b), dtype=torch.float32, device=dev) for _ in range(min(sR, 8))] for b in sbatches}
+    sws = torch.empty(max([sfmt.workspace_bytes(b) for b in [1] + sbatches] + [16]), dtype=torch.uint8, device=dev)
+    Ks = max(1, min(K, 2000))
+    sleg1 = Leg(torch, sfmt, sreps, sx1, sy1, sws, None, Ks)
+    slegB = [Leg(torch, sfmt, sreps, sX[b], sY[b], sws, "nb", max(1, Ks // b)) for b in sbatches]
+    check_against_host_decode(sfmt, sx1_host[0][None], sy1[0].cpu().numpy()[None], "sHAC GEMV")
+    for b, leg in zip(sbatches, slegB):
+        if b <= 16:
+            check_against_host_decode(sfmt, sX_host[b], sY[b][0].cpu().numpy().T, f"sHAC GEMM B={b}")
+    st_legs, st_whole = time_regions(torch, [sleg1] + slegB, MIN_TIMED_SECONDS, MAX_REPEATS, dist)
+    shac_gemv_s = median(st_legs[0]) * 1e-3 / Ks
+    shac_gemm_s = {b: median(t) * 1e-3 / leg.K for b, leg, t in zip(sbatches, slegB, st_legs[1:])}
+    shac_launches = sleg1.launches_per_product * Ks + sum(leg.launches_per_product * leg.K for leg in slegB)
 
     if rank != 0:
         if dist is not None:
@@ -397,24 +457,29 @@ def run_ours(args):
         return
 
     peaks, peak_kind = measured_peaks()
-    gemv_s = t_gemv_ms * 1e-3 / K
-    gemm_s = t_gemm_ms * 1e-3 / K
     alg_bytes = algorithmic_bytes_gemv(sizes, lut_bits)
     achieved = alg_bytes / gemv_s / 1e9
-    roofline = {"kernel": "hac_vec_kernel (GEMV, batch 1)", "bound": "hbm", "achieved": achieved,
+    roofline = {"kernel": "single-input HAC product (GEMV, batch 1)", "bound": "hbm", "achieved": achieved,
                 "peak": peaks["hbm_gbs"], "peak_source": f"of {peak_kind}", "unit": "GB/s",
                 "frac": achieved / peaks["hbm_gbs"], "frac_of_nominal_8TBs": achieved / 8000.0,
-                "traffic": gemv_traffic(), "algorithmic_bytes_per_launch": alg_bytes, "avg_launch_us": gemv_s * 1e6,
+                "traffic": ncu_traffic("hac_gemv"), "algorithmic_bytes_per_launch": alg_bytes, "avg_launch_us": gemv_s * 1e6,
                 "symbols_per_s": sizes["symbols"] / gemv_s,
                 "note": "the metric's HBM figure is defined on the single-input product, so this object rates that kernel; "
                         "the batch-64 product, which takes the larger share of a step, is rated in roofline_gemm"}
     gemm_flops = 2.0 * n * m * GEMM_BATCH
     tf32_peak = peaks.get("bf16_tflops", 1590.0) * 0.5        # measured bf16 x nominal tf32/bf16 ratio
-    roofline_gemm = {"kernel": "hac_gemm_tc_kernel (GEMM, batch 64, tcgen05 TF32 x3 split)", "bound": "tensor",
+    roofline_gemm = {"kernel": "batched HAC product (GEMM, batch 64, tcgen05 TF32 x3 split)", "bound": "tensor",
                      "achieved": gemm_flops / gemm_s / 1e12, "peak": tf32_peak, "unit": "TFLOP/s",
                      "peak_source": f"measured bf16 GEMM ({peak_kind}) x 0.5 (nominal tf32 : bf16)",
                      "frac": gemm_flops / gemm_s / 1e12 / tf32_peak, "avg_launch_us": gemm_s * 1e6,
                      "note": "algorithmic flops 2*n*m*B; the kernel is bound by the Huffman decode, not by the MMAs"}
+    s_alg = algorithmic_bytes_gemv(ssizes, min(12, ssizes["max_code_len"]))
+    s_ach = s_alg / shac_gemv_s / 1e9
+    roofline_shac = {"kernel": "single-input sHAC product (GEMV, batch 1)", "workload": swl.name, "bound": "hbm",
+                     "achieved": s_ach, "peak": peaks["hbm_gbs"], "peak_source": f"of {peak_kind}", "unit": "GB/s",
+                     "frac": s_ach / peaks["hbm_gbs"], "frac_of_nominal_8TBs": s_ach / 8000.0,
+                     "traffic": ncu_traffic("shac_gemv"), "algorithmic_bytes_per_launch": s_alg,
+                     "avg_launch_us": shac_gemv_s * 1e6, "stored_entries_per_s": ssizes["nnz"] / shac_gemv_s}
 
     # the oracle as it stands on the host cores, bounded sample (about 10-30 s of CPU work)
     cores = os.cpu_count() or 1
@@ -425,9 +490,14 @@ def run_ours(args):
                     "sample": f"Algorithm 3, {min(cores, rows)} threads, {rows} input rows x first {cols} of {m} "
                               f"columns of the same HAC stream, best of 3 ({t_cpu:.2f} s per run)"}
 
+    def spread(ts, per):
+        v = np.asarray(ts, dtype=np.float64) / per * 1e3
+        return {"us": float(np.median(v)), "min_us": float(v.min()), "max_us": float(v.max())}
+
     line = {
-        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": K, "warmup": max(Wm, 3),
-        "ms_per_step": job_ms / K, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": K, "warmup": Wm,
+        "ms_per_step": job_ms, "ms_per_step_min": min(t_whole) / K, "ms_per_step_max": max(t_whole) / K,
+        "repeats": repeats, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": "f32", "data": "synthetic",
         "config": {"workload": wl.name, "n": n, "m": m, "k": wl.k, "k_eff": sizes["k_eff"],
                    "quantizer": "uniform over [min,max]", "step": f"one GEMV (batch 1) + one GEMM (batch {GEMM_BATCH})",
@@ -435,14 +505,22 @@ def run_ours(args):
                    "format_bytes": sizes["total_bytes"], "stream_bytes": sizes["stream_bytes"],
                    "avg_code_len_bits": sizes["avg_code_len"],
                    "l2_defeat": f"{R} replicas of the {image_bytes}-byte device image rotated per launch (> 3 x L2)",
-                   "timing": "CUDA graphs of one replica rotation each, K GEMV launches then K GEMM launches, "
-                             "CUDA events on the launching stream"},
-        "gemv": {"value": float(n) * m / gemv_s / 1e9, "unit": UNIT, "us": gemv_s * 1e6},
-        "gemm": {"value": float(n) * m * GEMM_BATCH / gemm_s / 1e9, "unit": UNIT, "us": gemm_s * 1e6},
-        "roofline": roofline, "roofline_gemm": roofline_gemm, "cpu_baseline": cpu_baseline,
+                   "timing": f"a timed region is K GEMV launches then K GEMM launches (CUDA graphs of one replica rotation "
+                             f"each), CUDA events on the launching stream, synchronize on both sides; the region was "
+                             f"repeated {repeats} times and ms_per_step is the median region / K"},
+        "gemv": dict(spread(t_gemv, K), value=float(n) * m / gemv_s / 1e9, unit=UNIT),
+        "gemm": dict(spread(t_gemm, K), value=float(n) * m * GEMM_BATCH / gemm_s / 1e9, unit=UNIT),
+        "shac_gemv": dict(spread(st_legs[0], Ks), workload=swl.name, value=float(swl.n) * swl.m / shac_gemv_s / 1e9,
+                          unit=UNIT, launches=Ks),
+        "shac_gemm": {str(b): dict(spread(t, leg.K), value=float(swl.n) * swl.m * b / shac_gemm_s[b] / 1e9, unit=UNIT,
+                                   launches=leg.K)
+                      for b, leg, t in zip(sbatches, slegB, st_legs[1:])},
+        "roofline": roofline, "roofline_gemm": roofline_gemm, "roofline_shac": roofline_shac,
+        "cpu_baseline": cpu_baseline,
         "e2e": {"value": e2e_value, "unit": UNIT, "steps": Ke,
                 "h2d_bytes_per_step": 4 * n * (1 + GEMM_BATCH), "d2h_bytes_per_step": 4 * m * (1 + GEMM_BATCH)},
-        "gpu_launches": K * (launches["gemv"] + launches["gemm"]),
+        "gpu_launches": repeats * K * hac_launches,
+        "gpu_launches_shac": len(st_whole) * shac_launches,
         "clocks": clocks.summary(),
     }
     print(json.dumps(line), flush=True)
@@ -453,7 +531,7 @@ def run_ours(args):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=20000)
+    ap.add_argument("--steps", type=int, default=2000)
     ap.add_argument("--warmup", type=int, default=50)
     ap.add_argument("--impl", choices=("ours", "reference"), default="ours")
     args = ap.parse_args()

@@ -372,6 +372,57 @@ void make_decode_tables(Format& f) {
         }
         if (t.sub.size() * 4 <= kSubTableBytesMax) break;
     }
+    // magnitude table: only when the prefix table leaves code words to the sub-tables
+    double long_count = 0.0;
+    for (uint32_t s = 0; s < k; ++s)
+        if (f.code_len[s] > L1) long_count += (double)f.counts[s];
+    t.l1_unresolved = f.symbols ? long_count / (double)f.symbols : 0.0;
+    t.xt_mant = -1;
+    t.xt.clear();
+    t.use_xt = false;
+    if (t.l1_unresolved > 0.0) {
+        for (int mant = 3; mant <= kXtMantMax; ++mant) {
+            std::vector<uint32_t> xt((size_t)64 << mant, 0u);
+            for (size_t c = 0; c < ((size_t)32 << mant); ++c) xt[2 * c + 1] = 0x80000000u;
+            double unresolved = 0.0;
+            for (uint32_t s = 0; s < k; ++s) {
+                const uint32_t l = f.code_len[s];
+                const uint32_t lo = l >= 32 ? f.codes[s] : f.codes[s] << (32 - l);
+                const uint32_t hi = l >= 32 ? lo : lo + ((1u << (32 - l)) - 1u);
+                const uint32_t ia = xt_index(lo, mant), ib = xt_index(hi, mant);     // ia >= ib
+                const bool a_inside = lo == 0u || xt_index(lo - 1u, mant) != ia;
+                const bool b_inside = hi == 0xffffffffu || xt_index(hi + 1u, mant) != ib;
+                auto put = [&](uint32_t c) { xt[2 * c] = bits_of(f.codebook[s]); xt[2 * c + 1] = l; };
+                for (uint32_t c = ib + 1; c < ia; ++c) put(c);
+                if (ia == ib) { if (a_inside && b_inside) put(ia); }
+                else { if (a_inside) put(ia); if (b_inside) put(ib); }
+                // share of this code word's range that falls into cells shared with a neighbour
+                // (taken as uniform over the range): walk inwards from both ends
+                double bad = 0.0;
+                const double range = (double)hi - (double)lo + 1.0;
+                if (!(ia == ib ? (a_inside && b_inside) : a_inside)) {
+                    uint32_t end = lo;                     // last window of cell ia inside the range (binary search)
+                    uint32_t a = lo, b = hi;
+                    while (a < b) { const uint32_t mid = a + (b - a + 1) / 2; if (xt_index(mid, mant) == ia) a = mid; else b = mid - 1; }
+                    end = a;
+                    bad += (double)end - (double)lo + 1.0;
+                }
+                if (ia != ib && !b_inside) {
+                    uint32_t a = lo, b = hi;               // first window of cell ib inside the range
+                    while (a < b) { const uint32_t mid = a + (b - a) / 2; if (xt_index(mid, mant) == ib) b = mid; else a = mid + 1; }
+                    bad += (double)hi - (double)a + 1.0;
+                }
+                unresolved += (double)f.counts[s] * std::min(1.0, bad / range);
+            }
+            unresolved = f.symbols ? unresolved / (double)f.symbols : 0.0;
+            if (t.xt_mant < 0 || unresolved < t.xt_unresolved) {
+                t.xt_mant = mant; t.xt.swap(xt); t.xt_unresolved = unresolved;
+            }
+            if (t.xt_unresolved == 0.0) break;
+        }
+        t.use_xt = t.xt_unresolved < t.l1_unresolved;
+        if (!t.use_xt) { t.xt.clear(); t.xt_mant = -1; }
+    }
     // zero-run table: for streams that are mostly 1-bit zero code words
     t.l1_runs.clear();
     t.zero_len = 0;
@@ -716,6 +767,7 @@ ImageLayout image_layout(const Format& f) {
     L.l1 = take(f.tables.l1.size() * 4);
     L.sub = take(f.tables.sub.size() * 4);
     L.l1_runs = take(f.tables.l1_runs.size() * 4);
+    L.xt = take(f.tables.xt.size() * 4);
     L.rank_value = take(f.tables.rank_value.size() * 4);
     L.limit = take(sizeof(f.tables.limit));
     L.first_left = take(sizeof(f.tables.first_left));

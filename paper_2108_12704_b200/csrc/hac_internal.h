@@ -14,6 +14,17 @@ constexpr int kMaxCodeLen = 32;
 constexpr int kLutBitsMax = 12;          // full-width decode table: 2^L entries of 16 bits
 constexpr int kL1BitsMax = 10;           // level-1 table of the kernels: 2^L1 entries of 8 bytes
 constexpr int kSubBitsMax = 8;           // widest level-2 sub-table
+constexpr int kXtMantMax = 5;            // magnitude table: at most 32 << 5 entries (the size of the prefix table)
+
+// Index of a 32-bit window into the magnitude table with `mant` mantissa bits (see DecodeTables::xt).
+inline uint32_t xt_index(uint32_t window, int mant) {
+    const uint32_t u = ~window | 1u;
+    int e = 31;
+    while (!(u >> e)) --e;
+    const uint32_t norm = u << (31 - e);                     // leading one at bit 31
+    const uint32_t frac = mant ? ((norm << 1) >> (32 - mant)) : 0u;
+    return ((uint32_t)e << mant) | frac;
+}
 constexpr size_t kSubTableBytesMax = 24 * 1024;
 constexpr int kStreamSlackWords = 4;     // zero words after the stream (decoder reads ahead)
 
@@ -38,6 +49,20 @@ struct DecodeTables {
     // words keep their sub-table entry.  Empty when the format has no use for it.
     std::vector<uint32_t> l1_runs;            // [2^l1_bits * 2]
     uint32_t zero_len = 0;                    // code length of the zero symbol (0 = none)
+    // Table indexed by magnitude instead of by prefix.  A canonical code puts its long code words at
+    // the top of the code space (many leading ones), where a prefix table is far too coarse, and its
+    // short ones at the bottom, where it is finer than needed.  With u = ~window | 1 (32 bits), the
+    // index is the exponent of u (31 - leading ones of the window) followed by the xt_mant bits after
+    // its leading one: exactly the top bits of u converted to float with rounding toward zero, biased
+    // exponent 127 removed.  A cell that lies inside one code word's range holds {value bits, length};
+    // any other cell holds {0, 0x80000000} (found by the search over lengths).  32 << xt_mant entries.
+    // Built when code words are longer than the prefix table; used when it leaves fewer symbols
+    // unresolved than the prefix table does.
+    int xt_mant = -1;                         // -1: not built
+    std::vector<uint32_t> xt;                 // [(32 << xt_mant) * 2]
+    double xt_unresolved = 0.0;               // share of the symbols the magnitude table leaves to the search
+    double l1_unresolved = 0.0;               // share of the symbols whose code word is longer than l1_bits
+    bool use_xt = false;
     uint64_t limit[kMaxCodeLen + 2] = {};     // left-aligned (32-bit) end of the codes of length l
     uint32_t first_left[kMaxCodeLen + 2] = {};// left-aligned first code of length l
     uint32_t rank_base[kMaxCodeLen + 2] = {}; // rank of the first code of length l
@@ -54,6 +79,7 @@ struct DeviceImage {
     const uint2_host* l1 = nullptr;
     const uint2_host* sub = nullptr;
     const uint2_host* l1_runs = nullptr;
+    const uint2_host* xt = nullptr;
     const float* rank_value = nullptr;
     const uint64_t* limit = nullptr;          // [34]
     const uint32_t* first_left = nullptr;     // [34]
@@ -111,7 +137,7 @@ void fill_size_report(const Format& f, hac_size_report* r);
 
 // device image layout: offsets of every section (256-byte aligned), total size
 struct ImageLayout {
-    size_t stream, lut, l1, sub, l1_runs, rank_value, limit, first_left, rank_base, seg_bit_off, sub_bits, seg_col,
+    size_t stream, lut, l1, sub, l1_runs, xt, rank_value, limit, first_left, rank_base, seg_bit_off, sub_bits, seg_col,
         seg_first, ri, cb, unit_info, total;
 };
 ImageLayout image_layout(const Format& f);

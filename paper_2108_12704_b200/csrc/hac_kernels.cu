@@ -15,7 +15,10 @@
 #include <cstdio>
 #include <cstdlib>
 #include <cstring>
+#include <map>
 #include <mutex>
+#include <tuple>
+#include <utility>
 #include <string>
 #include <type_traits>
 
@@ -55,6 +58,11 @@ struct DevFormat {
     const uint32_t* cb;
     const void* unit_info;
     uint32_t n, m, units, G, S, k_eff, lut_bits, max_len, ri_bits, max_unit_chunks, max_sub_chunks, l1_bits, sub_bytes, items;
+    // First-level table `l1`, l1_entries entries.  tab_kind 0: the prefix table (2^l1_bits entries).  1: the
+    // magnitude table with xt_mant mantissa bits, rows xt_row0 .. 31 (the rows below belong to windows with more
+    // leading ones than the longest code word has bits: xt_low, OR-ed into ~window, keeps the index out of them);
+    // its unresolved cells go to the search over lengths (no sub-tables).
+    uint32_t tab_kind, l1_entries, xt_mant, xt_row0, xt_low;
 };
 
 
@@ -86,15 +94,18 @@ struct TablePlan {
     uint32_t repl_log2;
     uint32_t zero_len;    // HAC zero-run table in use: code length of the zero symbol
     uint32_t x_bulk;      // sHAC: x is contiguous and 16-byte aligned, so it is brought in by one bulk async copy
+    uint32_t prefetch;    // HAC rows kernel: ask for the block's share of the stream into L2 at the start
 };
 
-__host__ __device__ inline size_t plan_smem_bytes(uint32_t l1_bits, uint32_t repl_log2, uint32_t sub_bytes) {
-    return ((size_t)8 << (l1_bits + repl_log2)) + align16(sub_bytes);
+__host__ __device__ inline size_t plan_smem_bytes(uint32_t l1_entries, uint32_t repl_log2, uint32_t sub_bytes) {
+    return (((size_t)8 * l1_entries) << repl_log2) + align16(sub_bytes);
 }
 
 // Per-thread handle on the staged tables (shared-space addresses) and the global fallbacks.
 struct Decoder {
     uint32_t l1_lane, l1_mul, l1_shift, l1_bits, sub;
+    uint32_t bias;        // magnitude table: raw index of the first entry kept (subtracted from the raw index); else 0
+    uint32_t xt_low;      // magnitude table: low bits OR-ed into ~window before the conversion
 };
 
 // TF32 split of a shared value for the tensor-core kernel, packed with the code length:
@@ -124,7 +135,7 @@ __device__ __forceinline__ Decoder stage_decoder(const DevFormat& f, const Table
     Decoder d;
     const uint32_t repl = 1u << tp.repl_log2;
     uint2* l1 = reinterpret_cast<uint2*>(p);
-    p += (size_t)8 << (f.l1_bits + tp.repl_log2);
+    p += ((size_t)8 * f.l1_entries) << tp.repl_log2;
     uint2* sub = reinterpret_cast<uint2*>(p);
     p += align16(f.sub_bytes);
     // Each thread loads one entry; the warp then writes its 32 entries' replicas slot by slot, the
@@ -142,13 +153,13 @@ __device__ __forceinline__ Decoder stage_decoder(const DevFormat& f, const Table
         sub_v[k] = i < sub_entries ? __ldg(f.sub + i) : make_uint2(0u, 0u);
         if (kSplit) sub_v[k] = split_entry(sub_v[k]);
     }
-    for (uint32_t idx0 = threadIdx.x - lane_; idx0 < (1u << f.l1_bits); idx0 += blockDim.x) {
+    for (uint32_t idx0 = threadIdx.x - lane_; idx0 < f.l1_entries; idx0 += blockDim.x) {
         const uint32_t idx = idx0 + lane_;
         uint2 v = make_uint2(0u, 0u);
-        if (idx < (1u << f.l1_bits)) v = __ldg(f.l1 + idx);
+        if (idx < f.l1_entries) v = __ldg(f.l1 + idx);
         if (kSplit) v = split_entry(v);
         uint2* dst = l1 + ((size_t)idx0 << tp.repl_log2);
-        const uint32_t warp_slots = min(32u, (1u << f.l1_bits) - idx0) << tp.repl_log2;
+        const uint32_t warp_slots = min(32u, f.l1_entries - idx0) << tp.repl_log2;
         for (uint32_t s0 = 0; s0 < warp_slots; s0 += 32) {
             const uint32_t src = (s0 + lane_) >> tp.repl_log2;
             uint2 w;
@@ -166,7 +177,9 @@ __device__ __forceinline__ Decoder stage_decoder(const DevFormat& f, const Table
         sub[i] = kSplit ? split_entry(__ldg(f.sub + i)) : __ldg(f.sub + i);
     d.l1_lane = smem_off(l1) + ((threadIdx.x & (repl - 1)) << 3);
     d.l1_mul = 8u << tp.repl_log2;
-    d.l1_shift = 32 - f.l1_bits;
+    d.l1_shift = f.tab_kind ? 23 - f.xt_mant : 32 - f.l1_bits;
+    d.bias = f.tab_kind ? (127u + f.xt_row0) << f.xt_mant : 0u;
+    d.xt_low = f.xt_low;
     d.l1_bits = f.l1_bits;
     d.sub = smem_off(sub);
     return d;
@@ -260,6 +273,33 @@ __device__ __forceinline__ void fast_lookup(const FastReader& r, uint32_t l1_shi
         : "=r"(top), "=r"(val), "=r"(len)
         : "r"(r.lo), "r"(r.hi), "r"(r.off), "r"(l1_shift), "r"(l1_mul), "r"(l1_lane)
         : "memory");
+}
+
+// The same lookup in the magnitude table: the index is the exponent and the leading mantissa bits of
+// float(~window | 1), rounded toward zero (7 instructions).  `l1_lane` already has the index of exponent
+// 127 taken off.
+__device__ __forceinline__ void fast_lookup_xt(const FastReader& r, uint32_t l1_shift, uint32_t l1_mul, uint32_t l1_lane,
+                                               uint32_t xt_low, uint32_t& top, uint32_t& val, uint32_t& len) {
+    asm volatile(
+        "{\n\t"
+        ".reg .b32 i;\n\t"
+        "shf.l.wrap.b32 %0, %3, %4, %5;\n\t"
+        "lop3.b32 i, %0, %9, 0, 0xCF;\n\t"
+        "cvt.rz.f32.u32 i, i;\n\t"
+        "shr.u32 i, i, %6;\n\t"
+        "mad.lo.u32 i, i, %7, %8;\n\t"
+        "ld.shared.v2.u32 {%1, %2}, [i];\n\t"
+        "}"
+        : "=r"(top), "=r"(val), "=r"(len)
+        : "r"(r.lo), "r"(r.hi), "r"(r.off), "r"(l1_shift), "r"(l1_mul), "r"(l1_lane), "r"(xt_low)
+        : "memory");
+}
+
+template <int kTab>
+__device__ __forceinline__ void table_lookup(const FastReader& r, uint32_t l1_shift, uint32_t l1_mul, uint32_t l1_lane,
+                                             uint32_t xt_low, uint32_t& top, uint32_t& val, uint32_t& len) {
+    if (kTab == 0) fast_lookup(r, l1_shift, l1_mul, l1_lane, top, val, len);
+    else fast_lookup_xt(r, l1_shift, l1_mul, l1_lane, xt_low, top, val, len);
 }
 
 template <int kXOffset>
@@ -404,6 +444,27 @@ __device__ __forceinline__ void resolve_long_split(uint32_t top, const Decoder& 
     lo = e.x; hi_len = e.y;
 }
 
+// First-level entry that does not hold the symbol, for either kind of table.
+template <int kTab>
+__device__ __forceinline__ void resolve_any(uint32_t top, const Decoder& d, const DevFormat& f, uint32_t& val, uint32_t& len) {
+    if (kTab == 0) { resolve_long(top, d, f, val, len); return; }
+    const uint2 e = decode_long(top, f.lut, f.lut_bits, f.rank_value, f.limit, f.first_left, f.rank_base, f.max_len);
+    val = e.x; len = e.y;
+}
+
+// One code word -> the shared value, plain C++ (ragged ends and test paths), for either kind of table.
+template <int kTab, bool kLong>
+__device__ __forceinline__ float decode_value_any(BitReader& br, const Decoder& d, const DevFormat& f) {
+    if (kTab == 0) return decode_value<kLong>(br, d, f);
+    const uint32_t top = br.peek();
+    const uint32_t idx = (__float_as_uint(__uint2float_rz(~top | d.xt_low)) >> d.l1_shift) - d.bias;
+    uint2 e = lds64(d.l1_lane + idx * d.l1_mul);
+    if (kLong && (int32_t)e.y < 0)
+        e = decode_long(top, f.lut, f.lut_bits, f.rank_value, f.limit, f.first_left, f.rank_base, f.max_len);
+    br.skip(e.y);
+    return __uint_as_float(e.x);
+}
+
 // One step of kChains chains: lookups first, then the consumes, so that the table loads overlap.
 template <bool kLong, int kChains, int kXOffset>
 __device__ __forceinline__ void fast_step(FastReader (&r)[kChains], const Decoder& d, const DevFormat& f,
@@ -506,7 +567,7 @@ __global__ void __launch_bounds__(1024) hac_vec_kernel(DevFormat f, TablePlan tp
     // are requested (asynchronous copies) before the tables and x are staged, so that the block pays one
     // trip to memory for all three.
     const uint32_t pad = (f.S & 1u) ? 0u : 1u;
-    const size_t table_bytes = plan_smem_bytes(f.l1_bits, tp.repl_log2, f.sub_bytes);
+    const size_t table_bytes = plan_smem_bytes(f.l1_entries, tp.repl_log2, f.sub_bytes);
     const size_t x_bytes = (kMode == 0 && kXShared) ? align16(((size_t)f.n + (f.n / f.S + 1) * pad) * 4) : 0;
     uint4* stage = reinterpret_cast<uint4*>(smem + table_bytes + x_bytes) + (size_t)warp * kChains * f.max_unit_chunks;
     const uint32_t stage_a = smem_off(stage);
@@ -688,6 +749,407 @@ __global__ void __launch_bounds__(1024) hac_vec_kernel(DevFormat f, TablePlan tp
     }
 }
 
+// ------------------------------------------------------------------------------------------------
+// Three code words from one 32-bit window.  The window holds 32 valid bits from the current position,
+// so after a code word of length l the next one starts at window << l, and a third one after that,
+// as long as the three lengths add up to at most 32; the caller checks `tot` (and `flags`, the OR of
+// the three length words, whose top bit marks an entry that does not hold its symbol) before it uses
+// the values, and otherwise decodes the three code words one at a time.  The reader is not advanced.
+// ------------------------------------------------------------------------------------------------
+template <int kTab>
+__device__ __forceinline__ void lookup3(const FastReader& r, uint32_t l1_shift, uint32_t l1_mul, uint32_t l1_lane,
+                                        uint32_t xt_low, uint32_t& v1, uint32_t& v2, uint32_t& v3, uint32_t& tot,
+                                        uint32_t& flags) {
+    if (kTab == 0) {
+        asm volatile(
+            "{\n\t"
+            ".reg .b32 t, i, a, b, c;\n\t"
+            "shf.l.wrap.b32 t, %5, %6, %7;\n\t"
+            "shr.u32 i, t, %8;\n\t"
+            "mad.lo.u32 i, i, %9, %10;\n\t"
+            "ld.shared.v2.u32 {%0, a}, [i];\n\t"
+            "shl.b32 t, t, a;\n\t"
+            "shr.u32 i, t, %8;\n\t"
+            "mad.lo.u32 i, i, %9, %10;\n\t"
+            "ld.shared.v2.u32 {%1, b}, [i];\n\t"
+            "shl.b32 t, t, b;\n\t"
+            "shr.u32 i, t, %8;\n\t"
+            "mad.lo.u32 i, i, %9, %10;\n\t"
+            "ld.shared.v2.u32 {%2, c}, [i];\n\t"
+            "add.u32 %3, a, b;\n\t"
+            "add.u32 %3, %3, c;\n\t"
+            "lop3.b32 %4, a, b, c, 0xFE;\n\t"
+            "}"
+            : "=r"(v1), "=r"(v2), "=r"(v3), "=r"(tot), "=r"(flags)
+            : "r"(r.lo), "r"(r.hi), "r"(r.off), "r"(l1_shift), "r"(l1_mul), "r"(l1_lane)
+            : "memory");
+    } else {
+        asm volatile(
+            "{\n\t"
+            ".reg .b32 t, i, a, b, c;\n\t"
+            "shf.l.wrap.b32 t, %5, %6, %7;\n\t"
+            "lop3.b32 i, t, %11, 0, 0xCF;\n\t"
+            "cvt.rz.f32.u32 i, i;\n\t"
+            "shr.u32 i, i, %8;\n\t"
+            "mad.lo.u32 i, i, %9, %10;\n\t"
+            "ld.shared.v2.u32 {%0, a}, [i];\n\t"
+            "shl.b32 t, t, a;\n\t"
+            "lop3.b32 i, t, %11, 0, 0xCF;\n\t"
+            "cvt.rz.f32.u32 i, i;\n\t"
+            "shr.u32 i, i, %8;\n\t"
+            "mad.lo.u32 i, i, %9, %10;\n\t"
+            "ld.shared.v2.u32 {%1, b}, [i];\n\t"
+            "shl.b32 t, t, b;\n\t"
+            "lop3.b32 i, t, %11, 0, 0xCF;\n\t"
+            "cvt.rz.f32.u32 i, i;\n\t"
+            "shr.u32 i, i, %8;\n\t"
+            "mad.lo.u32 i, i, %9, %10;\n\t"
+            "ld.shared.v2.u32 {%2, c}, [i];\n\t"
+            "add.u32 %3, a, b;\n\t"
+            "add.u32 %3, %3, c;\n\t"
+            "lop3.b32 %4, a, b, c, 0xFE;\n\t"
+            "}"
+            : "=r"(v1), "=r"(v2), "=r"(v3), "=r"(tot), "=r"(flags)
+            : "r"(r.lo), "r"(r.hi), "r"(r.off), "r"(l1_shift), "r"(l1_mul), "r"(l1_lane), "r"(xt_low)
+            : "memory");
+    }
+}
+
+// The three code words of lookup3 one at a time (refills in between, entries without a symbol resolved):
+// where a lane's three lengths exceed the window, or one of its entries does not hold its symbol.  Rare,
+// so it is a call, which keeps the unrolled code around it small.  `sf` is the block's copy of the format
+// descriptor in shared memory.
+struct Slow3 { uint32_t hi, lo, off, next, v0, v1, v2; };
+template <int kTab, bool kLong>
+__device__ __noinline__ Slow3 decode3_slow(uint32_t hi, uint32_t lo, uint32_t off, uint32_t next_rel, Decoder dec,
+                                           const DevFormat* sf) {
+    BitReader br;
+    br.hi = hi; br.lo = lo; br.off = off; br.next = next_rel;
+    Slow3 r;
+    r.v0 = __float_as_uint(decode_value_any<kTab, kLong>(br, dec, *sf));
+    r.v1 = __float_as_uint(decode_value_any<kTab, kLong>(br, dec, *sf));
+    r.v2 = __float_as_uint(decode_value_any<kTab, kLong>(br, dec, *sf));
+    r.hi = br.hi; r.lo = br.lo; r.off = br.off; r.next = br.next;
+    return r;
+}
+
+// Advance the reader by up to 32 bits (one refill at most).
+__device__ __forceinline__ void fast_advance(FastReader& r, uint32_t bits) { fast_consume_value(r, bits); }
+
+// ------------------------------------------------------------------------------------------------
+// HAC, one input vector, rows held in registers (Algorithm 1 by segments).
+//
+// A column of W is G segments of 32 sub-segments of kS rows.  Here a warp does not walk down a column:
+// it keeps ONE segment position g ("class") for its whole life, i.e. lane l always multiplies rows
+// (32 g + l) kS .. + kS - 1, so it loads those kS elements of x into registers once and then decodes
+// that segment of one column after another.  The multiply-accumulate of a decoded symbol is then a
+// single FMA with a register operand: no shared-memory read of x per symbol.  A block owns a
+// contiguous range of columns; its warps are dealt round-robin to the classes, and the warps of a
+// class take the block's columns kC at a time (kC interleaved decode chains per lane, all on the
+// same rows).  Per-segment sums meet in shared memory and are added per column in segment order at
+// the end, so no second kernel and no workspace is needed whatever G is.
+//
+// Code words are decoded three to a window (lookup3): one window extraction and one refill test per
+// three symbols.  A lane whose three lengths exceed the window, or that meets an entry without its
+// symbol, leaves the unrolled code and finishes its sub-segment one code word at a time.
+//
+// Order in a block: the whole range of the stream that the block's columns occupy is requested into L2
+// (its position is estimated from the column numbers, all columns holding the same number of code
+// words); index entries of the first two items, table entries and x are requested together (one trip to
+// memory); the spans of a warp's next item are copied to shared memory (cp.async, second buffer set)
+// while the current item is decoded.
+//   kMode 0: product; 1: debug decode (values written to aux[j*n + i]).
+//   kTab  0: prefix table; 1: magnitude table.   kGuard: three lengths can exceed 32 bits.
+// ------------------------------------------------------------------------------------------------
+template <int kMode, int kS, int kC, int kTab, bool kLong, bool kGuard>
+__global__ void __launch_bounds__(kC <= 2 ? 512 : 384, 1) hac_rows_kernel(DevFormat f, TablePlan tp, const float* __restrict__ x,
+                                                          int64_t xs_i, float* __restrict__ y, int64_t ys_j,
+                                                          float* __restrict__ aux, uint32_t colsum_bytes,
+                                                          uint32_t stream_chunks) {
+    __shared__ DevFormat sf;               // for the rare paths that are calls (decode3_slow)
+    allow_dependents();
+    const uint32_t warp = threadIdx.x >> 5, lane = threadIdx.x & 31, warps = blockDim.x >> 5;
+    const uint32_t col0 = (uint32_t)(((uint64_t)f.m * blockIdx.x) / gridDim.x);
+    const uint32_t col1 = (uint32_t)(((uint64_t)f.m * (blockIdx.x + 1)) / gridDim.x);
+    const uint32_t ncol = col1 - col0;
+    if (threadIdx.x == 0) sf = f;
+    const uint32_t cls = warp % f.G, wrank = warp / f.G;            // the host launches at least G warps
+    const uint32_t wcls = (warps - cls + f.G - 1) / f.G;            // warps of this class
+    const uint32_t groups = (ncol + kC - 1) / kC;
+    const uint32_t nitems = wrank < groups ? (groups - wrank + wcls - 1) / wcls : 0u;
+    const uint32_t sub = cls * 32 + lane;                           // sub-segment number inside a column
+    const uint32_t row0 = sub * kS;
+    const uint32_t count = row0 < f.n ? min((uint32_t)kS, f.n - row0) : 0u;
+
+    // shared memory: [tables][per-column partial sums][span buffers: set, warp, chain]; x is staged over the
+    // second buffer set before that set is first used
+    const size_t table_bytes = plan_smem_bytes(f.l1_entries, tp.repl_log2, f.sub_bytes);
+    float* colsum = reinterpret_cast<float*>(smem + table_bytes);
+    const uint32_t span_bytes = f.max_unit_chunks * 16;
+    const uint32_t bufs = (uint32_t)table_bytes + colsum_bytes;
+    const uint32_t set_bytes = warps * kC * span_bytes;
+    float* xs = reinterpret_cast<float*>(smem + bufs + set_bytes);
+    auto buf_of = [&](uint32_t set, uint32_t c) { return bufs + set * set_bytes + (warp * kC + c) * span_bytes; };
+
+    // index entries of item k of this warp (chain c = column (wrank + k wcls) kC + c of the block)
+    auto col_of = [&](uint32_t k, uint32_t c) { return col0 + (wrank + k * wcls) * kC + c; };
+    struct Index { uint32_t bits[kC]; uint64_t seg[kC]; };
+    auto load_index = [&](uint32_t k, Index& ix) {
+        if (k >= nitems) return;
+#pragma unroll
+        for (int c = 0; c < kC; ++c) {
+            const uint32_t col = col_of(k, c);
+            ix.bits[c] = 0; ix.seg[c] = 0;
+            if (col < col1) {
+                const size_t u = (size_t)col * f.G + cls;
+                ix.bits[c] = __ldg(f.sub_bits + u * 32 + lane);
+                ix.seg[c] = __ldg(f.seg_bit_off + u);
+            }
+        }
+    };
+    // requests the spans of item k into buffer set `set`; pos[c] = bit position (relative to the buffer of
+    // chain c) of this lane's first code word.  Always one commit group.
+    auto fetch = [&](uint32_t k, uint32_t set, const Index& ix, uint32_t (&pos)[kC]) {
+        if (k < nitems) {
+#pragma unroll
+            for (int c = 0; c < kC; ++c) {
+                uint32_t total;
+                const uint32_t start = lane_start_bits(ix.bits[c], lane, total);
+                pos[c] = 0;
+                if (col_of(k, c) < col1)
+                    pos[c] = start + stage_span(f, ix.seg[c], total, reinterpret_cast<uint4*>(smem + buf_of(set, c)), lane);
+            }
+        }
+        asm volatile("cp.async.commit_group;" ::: "memory");
+    };
+
+    uint32_t pos_cur[kC], pos_nxt[kC];
+    Index ix0, ix1;
+    load_index(0, ix0);
+    load_index(1, ix1);
+    // table entries: every warp takes groups of 32 consecutive entries, all its loads in flight at once
+    constexpr int kTabAhead = 4;
+    const uint32_t entries = f.l1_entries;
+    uint2 te[kTabAhead];
+#pragma unroll
+    for (int i = 0; i < kTabAhead; ++i) {
+        const uint32_t idx = (warp + i * warps) * 32 + lane;
+        te[i] = idx < entries ? __ldg(f.l1 + idx) : make_uint2(0u, 0u);
+    }
+    if (tp.prefetch) {
+        // the block's share of the stream, a little generously, towards L2: 16 KB per requesting thread
+        const uint32_t lo = (uint32_t)(((uint64_t)stream_chunks * col0) / f.m);
+        const uint32_t hi = (uint32_t)(((uint64_t)stream_chunks * col1) / f.m);
+        const uint32_t slack = 64 + ((hi - lo) >> 6);
+        const uint32_t from = lo > slack ? lo - slack : 0u, to = min(stream_chunks, hi + slack);
+        const uint32_t piece = 1024;
+        const uint32_t at = from + threadIdx.x * piece;
+        if (at < to) {
+            const uint32_t bytes = min(piece, to - at) * 16u;
+            asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(reinterpret_cast<const uint4*>(f.stream) + at),
+                         "r"(bytes)
+                         : "memory");
+        }
+    }
+    // everything above reads the format only; x and the outputs belong to the kernels before this one
+    depends_wait();
+    float xr[kS];
+    constexpr int kXAhead = 8;
+    const uint32_t rows = f.G * 32u * kS;
+    float xv[kXAhead];
+    if (kMode == 0) {                      // the first elements of x are requested before the index entries are waited for
+#pragma unroll
+        for (int i = 0; i < kXAhead; ++i) {
+            const uint32_t r = threadIdx.x + i * blockDim.x;
+            xv[i] = r < f.n ? __ldg(x + (int64_t)r * xs_i) : 0.0f;
+        }
+    }
+    fetch(0, 0, ix0, pos_cur);
+    if (kMode == 0) {
+        // x -> shared memory (coalesced; one padding word per sub-segment keeps the lanes of a warp, which
+        // are kS rows apart, on distinct banks; rows past the end of x are zeros) -> registers
+        for (uint32_t r0 = 0; r0 < rows; r0 += kXAhead * blockDim.x) {
+            if (r0 > 0) {
+#pragma unroll
+                for (int i = 0; i < kXAhead; ++i) {
+                    const uint32_t r = r0 + threadIdx.x + i * blockDim.x;
+                    xv[i] = r < f.n ? __ldg(x + (int64_t)r * xs_i) : 0.0f;
+                }
+            }
+#pragma unroll
+            for (int i = 0; i < kXAhead; ++i) {
+                const uint32_t r = r0 + threadIdx.x + i * blockDim.x;
+                if (r < rows) xs[r + r / kS] = xv[i];
+            }
+        }
+        __syncthreads();
+#pragma unroll
+        for (int s = 0; s < kS; ++s) xr[s] = xs[row0 + sub + s];
+    }
+    // tables -> shared memory, replicated (see TablePlan): the warp writes its 32 entries' replicas slot by
+    // slot, the value for a slot fetched from the lane that holds it (consecutive lanes write consecutive slots)
+    Decoder dec;
+    {
+        uint2* l1 = reinterpret_cast<uint2*>(smem);
+        uint2* subt = reinterpret_cast<uint2*>(smem + (((size_t)8 * f.l1_entries) << tp.repl_log2));
+        const uint32_t repl = 1u << tp.repl_log2;
+        auto spread = [&](uint32_t idx0, uint2 v) {
+            uint2* dst = l1 + ((size_t)idx0 << tp.repl_log2);
+            const uint32_t warp_slots = min(32u, entries - idx0) << tp.repl_log2;
+            for (uint32_t s0 = 0; s0 < warp_slots; s0 += 32) {
+                const uint32_t src = (s0 + lane) >> tp.repl_log2;
+                uint2 w;
+                w.x = __shfl_sync(0xffffffffu, v.x, src & 31u);
+                w.y = __shfl_sync(0xffffffffu, v.y, src & 31u);
+                if (s0 + lane < warp_slots) dst[s0 + lane] = w;
+            }
+        };
+#pragma unroll
+        for (int i = 0; i < kTabAhead; ++i) {
+            const uint32_t idx0 = (warp + i * warps) * 32;
+            if (idx0 < entries) spread(idx0, te[i]);
+        }
+        for (uint32_t idx0 = (warp + kTabAhead * warps) * 32; idx0 < entries; idx0 += warps * 32) {
+            const uint32_t idx = idx0 + lane;
+            spread(idx0, idx < entries ? __ldg(f.l1 + idx) : make_uint2(0u, 0u));
+        }
+        for (uint32_t i = threadIdx.x; i < f.sub_bytes / 8; i += blockDim.x) subt[i] = __ldg(f.sub + i);
+        dec.l1_lane = smem_off(l1) + ((threadIdx.x & (repl - 1)) << 3);
+        dec.l1_mul = 8u << tp.repl_log2;
+        dec.l1_shift = f.tab_kind ? 23 - f.xt_mant : 32 - f.l1_bits;
+        dec.bias = f.tab_kind ? (127u + f.xt_row0) << f.xt_mant : 0u;
+        dec.xt_low = f.xt_low;
+        dec.l1_bits = f.l1_bits;
+        dec.sub = smem_off(subt);
+    }
+    __syncthreads();                       // tables are in place; x has left the second buffer set
+    fetch(1, 1, ix1, pos_nxt);
+    load_index(2, ix0);
+
+    const uint32_t sb = shared_base();
+    const uint32_t l1_abs = sb + dec.l1_lane - dec.bias * dec.l1_mul;
+    for (uint32_t k = 0; k < nitems; ++k) {
+        const uint32_t set = k & 1u;
+        asm volatile("cp.async.wait_group 1;" ::: "memory");      // item k's spans (item k + 1's may be in flight)
+        __syncwarp();
+        bool has[kC];
+        uint32_t bufc[kC];
+#pragma unroll
+        for (int c = 0; c < kC; ++c) {
+            has[c] = col_of(k, c) < col1;
+            bufc[c] = buf_of(set, has[c] ? c : 0);                  // a chain without a column decodes chain 0's again
+            if (!has[c]) pos_cur[c] = pos_cur[0];
+        }
+        float acc[kC];
+#pragma unroll
+        for (int c = 0; c < kC; ++c) acc[c] = 0.0f;
+        if (count > 0) {
+            FastReader fr[kC];
+#pragma unroll
+            for (int c = 0; c < kC; ++c) {
+                BitReader br;
+                br.init(bufc[c], pos_cur[c]);
+                fr[c].hi = br.hi; fr[c].lo = br.lo; fr[c].off = br.off; fr[c].next = sb + br.next;
+            }
+            float* out[kC];
+            if (kMode == 1) {
+#pragma unroll
+                for (int c = 0; c < kC; ++c) out[c] = aux + (size_t)col_of(k, c) * f.n + row0;
+            }
+            uint32_t done = 0;                                      // symbols of the sub-segment finished by the unrolled code
+            if (count == kS) {
+#pragma unroll
+                for (int s = 0; s + 3 <= kS; s += 3) {
+                    uint32_t v[kC][3], tot[kC], flags[kC];
+#pragma unroll
+                    for (int c = 0; c < kC; ++c)
+                        lookup3<kTab>(fr[c], dec.l1_shift, dec.l1_mul, l1_abs, dec.xt_low, v[c][0], v[c][1], v[c][2], tot[c], flags[c]);
+                    if (kGuard || kLong) {
+                        bool bad = false;
+#pragma unroll
+                        for (int c = 0; c < kC; ++c) bad = bad || (kGuard && tot[c] > 32u) || (kLong && (int32_t)flags[c] < 0);
+                        if (__any_sync(__activemask(), bad)) {              // uniform for the lanes in the unrolled code
+                            if (bad) {
+#pragma unroll
+                                for (int c = 0; c < kC; ++c) {
+                                    const Slow3 r = decode3_slow<kTab, kLong>(fr[c].hi, fr[c].lo, fr[c].off, fr[c].next - sb, dec, &sf);
+                                    fr[c].hi = r.hi; fr[c].lo = r.lo; fr[c].off = r.off; fr[c].next = sb + r.next;
+                                    v[c][0] = r.v0; v[c][1] = r.v1; v[c][2] = r.v2;
+                                    tot[c] = 0;
+                                }
+                            }
+                        }
+                    }
+#pragma unroll
+                    for (int c = 0; c < kC; ++c) {
+                        fast_advance(fr[c], tot[c]);
+#pragma unroll
+                        for (int e = 0; e < 3; ++e) {
+                            if (kMode == 0) acc[c] = fmaf(xr[s + e], __uint_as_float(v[c][e]), acc[c]);
+                            else if (has[c]) out[c][s + e] = __uint_as_float(v[c][e]);
+                        }
+                    }
+                }
+#pragma unroll
+                for (int s = kS - kS % 3; s < kS; ++s) {            // the symbols that do not fill a group of three
+                    uint32_t top[kC], val[kC], len[kC];
+#pragma unroll
+                    for (int c = 0; c < kC; ++c) table_lookup<kTab>(fr[c], dec.l1_shift, dec.l1_mul, l1_abs, dec.xt_low, top[c], val[c], len[c]);
+                    if (kLong) {
+#pragma unroll
+                        for (int c = 0; c < kC; ++c)
+                            if ((int32_t)len[c] < 0) resolve_any<kTab>(top[c], dec, f, val[c], len[c]);
+                    }
+#pragma unroll
+                    for (int c = 0; c < kC; ++c) {
+                        fast_advance(fr[c], len[c]);
+                        if (kMode == 0) acc[c] = fmaf(xr[s], __uint_as_float(val[c]), acc[c]);
+                        else if (has[c]) out[c][s] = __uint_as_float(val[c]);
+                    }
+                }
+                done = (uint32_t)kS;
+            }
+            if (done < count) {
+                // the sub-segment at the ragged end of a column
+#pragma unroll
+                for (int c = 0; c < kC; ++c) {
+                    BitReader br;
+                    br.hi = fr[c].hi; br.lo = fr[c].lo; br.off = fr[c].off; br.next = fr[c].next - sb;
+                    for (uint32_t s = done; s < count; ++s) {
+                        const float w = decode_value_any<kTab, kLong>(br, dec, f);
+                        if (kMode == 0) acc[c] = fmaf(__ldg(x + (int64_t)(row0 + s) * xs_i), w, acc[c]);
+                        else if (has[c]) out[c][s] = w;
+                    }
+                }
+            }
+        }
+        __syncwarp();
+        if (kMode == 0) {
+#pragma unroll
+            for (int c = 0; c < kC; ++c) acc[c] = warp_sum(acc[c]);
+            if (lane == 0) {
+#pragma unroll
+                for (int c = 0; c < kC; ++c)
+                    if (has[c]) colsum[(col_of(k, c) - col0) * f.G + cls] = acc[c];
+            }
+        }
+        // the buffer set just decoded takes the spans of item k + 2
+#pragma unroll
+        for (int c = 0; c < kC; ++c) pos_cur[c] = pos_nxt[c];
+        fetch(k + 2, set, ix0, pos_nxt);
+        load_index(k + 3, ix0);
+    }
+    asm volatile("cp.async.wait_group 0;" ::: "memory");
+    if (kMode == 0) {
+        __syncthreads();
+        for (uint32_t t = threadIdx.x; t < ncol; t += blockDim.x) {
+            float s = 0.0f;
+            for (uint32_t g = 0; g < f.G; ++g) s += colsum[t * f.G + g];
+            y[(int64_t)(col0 + t) * ys_j] = s;
+        }
+    }
+}
+
 // Work item of the sHAC single-input kernel (derived on the host from cb and the offset index): one
 // or two consecutive segments of one column.  For each segment: where its code words start in the
 // stream, where its entries start in nz / ri, and how many there are.
@@ -745,7 +1207,7 @@ __global__ void __launch_bounds__(1024) shac_vec_kernel(DevFormat f, TablePlan t
     // [tables] follow at p; the staging areas come after them.  The first item's slices of ri and spans of
     // the stream are requested (asynchronous copies) before the tables are staged, so that the trips to
     // memory overlap.
-    unsigned char* after_tables = p + plan_smem_bytes(f.l1_bits, tp.repl_log2, f.sub_bytes);
+    unsigned char* after_tables = p + plan_smem_bytes(f.l1_entries, tp.repl_log2, f.sub_bytes);
     uint4* stage = reinterpret_cast<uint4*>(after_tables) + (size_t)warp * kChains * f.max_unit_chunks;
     after_tables += align16((size_t)warps * kChains * f.max_unit_chunks * 16);
     // row-index staging: 32*S entries plus up to 16 bytes of misalignment, per segment
@@ -1579,11 +2041,33 @@ static int device_info(DeviceInfo& d) {
     return HAC_OK;
 }
 
+static int env_int(const char* name, int fallback) {
+    const char* v = std::getenv(name);
+    return v && *v ? std::atoi(v) : fallback;
+}
+
+// Diagnostic switches (environment, read once when the first product is launched; see hac.h).
+struct Tune {
+    int pdl;            // HAC_B200_PDL=0: launch without programmatic stream serialization
+    int rows_kernel;    // HAC_B200_ROWS=0: single-input HAC always through the shared-memory-x kernel
+    int rows_warps;     // HAC_B200_ROWS_WARPS=n: warps per block of the rows-in-registers kernel (0 = chosen by the library)
+    int zero_runs;      // HAC_B200_ZERO_RUNS=0: never use the zero-run table
+    int xt;             // HAC_B200_XT=0: never use the magnitude table
+    int prefetch;       // HAC_B200_PREFETCH=0: no L2 prefetch of the stream at the start of the rows-in-registers kernel
+    int rows_chains;    // HAC_B200_ROWS_CHAINS=2|3: decode chains per lane of that kernel (0 = chosen by the library)
+};
+static const Tune& tune() {
+    static const Tune t = {env_int("HAC_B200_PDL", 1), env_int("HAC_B200_ROWS", 1), env_int("HAC_B200_ROWS_WARPS", 0),
+                           env_int("HAC_B200_ZERO_RUNS", 1), env_int("HAC_B200_XT", 1), env_int("HAC_B200_PREFETCH", 1), env_int("HAC_B200_ROWS_CHAINS", 0)};
+    return t;
+}
+
 static DevFormat dev_format(const Format& f) {
     DevFormat d{};
     d.stream = f.dev.stream; d.lut = f.dev.lut; d.rank_value = f.dev.rank_value;
     d.l1 = reinterpret_cast<const uint2*>(f.dev.l1); d.sub = reinterpret_cast<const uint2*>(f.dev.sub);
     d.l1_bits = (uint32_t)f.tables.l1_bits; d.sub_bytes = (uint32_t)(f.tables.sub.size() * 4);
+    d.l1_entries = 1u << d.l1_bits;
     d.items = (uint32_t)(f.item_info.size() / 12);
     d.limit = f.dev.limit; d.first_left = f.dev.first_left; d.rank_base = f.dev.rank_base;
     d.seg_bit_off = f.dev.seg_bit_off; d.sub_bits = f.dev.sub_bits; d.seg_col = f.dev.seg_col;
@@ -1593,7 +2077,32 @@ static DevFormat dev_format(const Format& f) {
     d.lut_bits = (uint32_t)f.tables.lut_bits; d.max_len = f.max_len; d.ri_bits = f.ri_bits;
     d.max_unit_chunks = f.max_unit_chunks;
     d.max_sub_chunks = f.max_sub_chunks;
+    d.tab_kind = 0;
     return d;
+}
+
+// The same with the magnitude table as first-level table, when the format has one that resolves more
+// symbols than the prefix table.
+static bool wants_xt(const Format& f) { return f.tables.use_xt && tune().xt != 0; }
+static DevFormat dev_format_xt(const Format& f) {
+    DevFormat d = dev_format(f);
+    if (wants_xt(f)) {
+        // a window with more leading ones than the longest code word has bits decodes like the one with
+        // exactly that many: rows below 31 - max_len are never needed
+        const uint32_t mant = (uint32_t)f.tables.xt_mant;
+        d.xt_mant = mant;
+        d.xt_row0 = f.max_len < 31u ? 31u - f.max_len : 0u;
+        d.xt_low = f.max_len < 32u ? ((1u << (32u - f.max_len)) - 1u) | 1u : 1u;
+        d.l1 = reinterpret_cast<const uint2*>(f.dev.xt) + ((size_t)d.xt_row0 << mant);
+        d.l1_entries = (32u - d.xt_row0) << mant;
+        d.sub_bytes = 0;
+        d.tab_kind = 1;
+    }
+    return d;
+}
+// Whether a first-level entry can fail to hold the symbol.
+static bool table_has_long(const Format& f, const DevFormat& d) {
+    return d.tab_kind ? f.tables.xt_unresolved > 0.0 : d.max_len > d.l1_bits;
 }
 
 static void set_pointers(Format& f, void* dev_buf, size_t bytes) {
@@ -1605,6 +2114,7 @@ static void set_pointers(Format& f, void* dev_buf, size_t bytes) {
     f.dev.l1 = reinterpret_cast<const uint2_host*>(b + L.l1);
     f.dev.sub = reinterpret_cast<const uint2_host*>(b + L.sub);
     f.dev.l1_runs = reinterpret_cast<const uint2_host*>(b + L.l1_runs);
+    f.dev.xt = reinterpret_cast<const uint2_host*>(b + L.xt);
     f.dev.rank_value = reinterpret_cast<const float*>(b + L.rank_value);
     f.dev.limit = reinterpret_cast<const uint64_t*>(b + L.limit);
     f.dev.first_left = reinterpret_cast<const uint32_t*>(b + L.first_left);
@@ -1634,6 +2144,7 @@ static int upload(Format& f, void* dev_buf, size_t dev_bytes, void* stream_) {
     HAC_CUDA(put(L.l1, f.tables.l1.data(), f.tables.l1.size() * 4));
     HAC_CUDA(put(L.sub, f.tables.sub.data(), f.tables.sub.size() * 4));
     HAC_CUDA(put(L.l1_runs, f.tables.l1_runs.data(), f.tables.l1_runs.size() * 4));
+    HAC_CUDA(put(L.xt, f.tables.xt.data(), f.tables.xt.size() * 4));
     HAC_CUDA(put(L.rank_value, f.tables.rank_value.data(), f.tables.rank_value.size() * 4));
     HAC_CUDA(put(L.limit, f.tables.limit, sizeof(f.tables.limit)));
     HAC_CUDA(put(L.first_left, f.tables.first_left, sizeof(f.tables.first_left)));
@@ -1667,7 +2178,7 @@ static uint32_t gemm_tasks(const Format& f) { return f.S ? (uint32_t)((f.n + f.S
 // (227 KB on sm_100); such formats take the batched kernel for a single input too.
 static bool shac_vec_fits(const Format& f) {
     const size_t per_warp = ((size_t)f.max_unit_chunks * 16 + ((size_t)(32u * f.S * (f.ri_bits / 8) + 15u) / 16u + 1u) * 16u) * 2;
-    return 16 + plan_smem_bytes((uint32_t)f.tables.l1_bits, 0, (uint32_t)(f.tables.sub.size() * 4)) + per_warp <= (size_t)232448;
+    return 16 + plan_smem_bytes(1u << f.tables.l1_bits, 0, (uint32_t)(f.tables.sub.size() * 4)) + per_warp <= (size_t)232448;
 }
 
 static size_t partial_bytes(const Format& f, int64_t batch) {
@@ -1731,14 +2242,38 @@ static size_t workspace_bytes(const Format& f, int64_t batch) {
     return std::max(((partial_bytes(f, batch) + 255) & ~(size_t)255) + xp + task_off_bytes(f, batch), partial_bytes(f, 1));
 }
 
-static int env_int(const char* name, int fallback) {
-    const char* v = std::getenv(name);
-    return v && *v ? std::atoi(v) : fallback;
+// Opt-in to more than 48 KB of dynamic shared memory: once per kernel, device and size.
+static int prepare_kernel_ptr(const void* kernel, size_t smem) {
+    if (smem <= 48 * 1024) return HAC_OK;
+    static std::mutex guard;
+    static std::map<std::pair<int, const void*>, size_t> done;
+    int dev = 0;
+    HAC_CUDA(cudaGetDevice(&dev));
+    std::lock_guard<std::mutex> lock(guard);
+    size_t& have = done[std::make_pair(dev, kernel)];
+    if (have >= smem) return HAC_OK;
+    HAC_CUDA(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+    have = smem;
+    return HAC_OK;
 }
-
 template <typename K>
-static int prepare_kernel(K kernel, size_t smem) {
-    if (smem > 48 * 1024) HAC_CUDA(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+static int prepare_kernel(K kernel, size_t smem) { return prepare_kernel_ptr(reinterpret_cast<const void*>(kernel), smem); }
+
+// Resident blocks per SM of a kernel at a block size and shared-memory size: asked once per combination.
+static int blocks_per_sm(const void* kernel, int threads, size_t smem, int* out) {
+    static std::mutex guard;
+    static std::map<std::tuple<int, const void*, int, size_t>, int> known;
+    int dev = 0;
+    HAC_CUDA(cudaGetDevice(&dev));
+    std::lock_guard<std::mutex> lock(guard);
+    auto key = std::make_tuple(dev, kernel, threads, smem);
+    auto it = known.find(key);
+    if (it == known.end()) {
+        int per_sm = 1;
+        HAC_CUDA(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kernel, threads, smem));
+        it = known.emplace(key, std::max(per_sm, 1)).first;
+    }
+    *out = it->second;
     return HAC_OK;
 }
 
@@ -1750,7 +2285,7 @@ static int launch_dependent(void (*kernel)(KArgs...), dim3 grid, dim3 block, siz
     cfg.gridDim = grid; cfg.blockDim = block; cfg.dynamicSmemBytes = smem; cfg.stream = st;
     cudaLaunchAttribute attr[1];
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-    attr[0].val.programmaticStreamSerializationAllowed = env_int("HAC_B200_PDL", 1) != 0 ? 1 : 0;
+    attr[0].val.programmaticStreamSerializationAllowed = tune().pdl != 0 ? 1 : 0;
     cfg.attrs = attr; cfg.numAttrs = 1;
     HAC_CUDA(cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...));
     return HAC_OK;
@@ -1779,7 +2314,7 @@ static int launch_finalize(const Format& f, const DevFormat& d, const float* par
 static TablePlan plan_tables(const DevFormat& d, size_t table_budget) {
     TablePlan tp{};
     tp.repl_log2 = 4;
-    while (tp.repl_log2 > 0 && plan_smem_bytes(d.l1_bits, tp.repl_log2, d.sub_bytes) > table_budget) tp.repl_log2--;
+    while (tp.repl_log2 > 0 && plan_smem_bytes(d.l1_entries, tp.repl_log2, d.sub_bytes) > table_budget) tp.repl_log2--;
     return tp;
 }
 
@@ -1805,6 +2340,110 @@ static VecKernel pick_vec_kernel(const Format& f, int mode, bool x_shared, int c
                                  : shac_vec_kernel<0, false, kLong, uint32_t>);
 }
 
+// ---- single-input HAC with the rows of x in registers -------------------------------------------
+constexpr int kRowsS = 64;              // sub-segment length the kernel is compiled for
+constexpr int kRowsMaxWarps = 16;
+
+typedef void (*RowsKernel)(DevFormat, TablePlan, const float*, int64_t, float*, int64_t, float*, uint32_t, uint32_t);
+
+template <int kMode, int kTab, int kC>
+static RowsKernel pick_rows_kernel3(bool has_long, bool guard) {
+    if (has_long) return hac_rows_kernel<kMode, kRowsS, kC, kTab, true, true>;
+    return guard ? hac_rows_kernel<kMode, kRowsS, kC, kTab, false, true> : hac_rows_kernel<kMode, kRowsS, kC, kTab, false, false>;
+}
+template <int kMode, int kTab>
+static RowsKernel pick_rows_kernel2(int chains, bool has_long, bool guard) {
+    return chains == 3 ? pick_rows_kernel3<kMode, kTab, 3>(has_long, guard) : pick_rows_kernel3<kMode, kTab, 2>(has_long, guard);
+}
+template <int kMode>
+static RowsKernel pick_rows_kernel(bool xt, int chains, bool has_long, bool guard) {
+    return xt ? pick_rows_kernel2<kMode, 1>(chains, has_long, guard) : pick_rows_kernel2<kMode, 0>(chains, has_long, guard);
+}
+
+struct RowsPlan {
+    bool ok = false;
+    DevFormat d;
+    TablePlan tp;
+    unsigned grid = 0;
+    int warps = 0, chains = 2;
+    size_t smem = 0;
+    uint32_t colsum_bytes = 0;
+    bool has_long = false;
+};
+
+// Whether the rows-in-registers kernel takes this format, and with which block shape: sub-segments of
+// kRowsS symbols, no zero-run table in use, enough columns to give every SM some, at least one warp per
+// segment position, and tables + two sets of span buffers within an SM's shared memory.  Warps per block
+// and chains per lane are the pair that needs the least time by this estimate: the warps of a class share
+// the block's columns, `chains` at a time, in rounds; a round costs in proportion to the chains in
+// flight on the SM once there are enough of them to fill the instruction issue (about 30), and no less
+// than that below.
+static RowsPlan plan_rows(const Format& f, const DeviceInfo& di, int mode) {
+    RowsPlan pl;
+    if (f.sparse || f.S != (uint32_t)kRowsS || f.G == 0 || f.G > (uint32_t)kRowsMaxWarps || tune().rows_kernel == 0) return pl;
+    if (mode == 0 && !f.tables.l1_runs.empty() && tune().zero_runs != 0) return pl;
+    if ((uint64_t)f.m * 2 < (uint64_t)di.sms) return pl;
+    pl.d = dev_format_xt(f);
+    pl.has_long = table_has_long(f, pl.d);
+    pl.grid = (unsigned)std::min<int64_t>(di.sms, f.m);
+    const uint32_t max_cols = (uint32_t)((f.m + pl.grid - 1) / pl.grid);
+    pl.colsum_bytes = (uint32_t)align16((size_t)max_cols * f.G * 4);
+    if (pl.colsum_bytes > 16 * 1024) return pl;
+    const size_t budget = (size_t)di.max_smem_optin - 256;       // static shared memory of the kernel
+    const size_t span = (size_t)f.max_unit_chunks * 16;
+    const size_t xs_bytes = mode == 0 ? align16((size_t)f.G * 32 * (kRowsS + 1) * 4) : 0;
+    for (int repl = 4; repl >= 0; --repl) {
+        const size_t tab = plan_smem_bytes(pl.d.l1_entries, (uint32_t)repl, pl.d.sub_bytes);
+        int best_w = 0, best_c = 0;
+        uint64_t best_cost = ~0ull;
+        for (int chains = 2; chains <= 3; ++chains) {
+            // (three chains per lane measured slower than two at the same number of rounds: only on request)
+            if (chains != (tune().rows_chains > 0 ? tune().rows_chains : 2)) continue;
+            const uint32_t groups = (max_cols + chains - 1) / chains;
+            const int max_w = chains == 2 ? kRowsMaxWarps : 12;  // the register budget of the wider kernel
+            for (int w = (int)f.G; w <= max_w; ++w) {
+                if (tune().rows_warps > 0 && w != tune().rows_warps) continue;
+                const size_t set = (size_t)w * chains * span;
+                if (tab + pl.colsum_bytes + std::max(2 * set, set + xs_bytes) > budget) break;
+                const uint32_t wcls = (uint32_t)w / f.G;             // warps of the least served class
+                const uint64_t rounds = (groups + wcls - 1) / wcls;
+                // a round is bound by the latency of a lane's serial decode until about 60 chains are in flight
+                const uint64_t cost = rounds * (uint64_t)std::max(w * chains, 60);
+                if (cost < best_cost || (cost == best_cost && w * chains > best_w * best_c)) {
+                    best_cost = cost; best_w = w; best_c = chains;
+                }
+            }
+        }
+        if (best_w * best_c >= std::min<int>(16, (int)(f.G * 2)) || (repl == 0 && best_w > 0)) {
+            pl.tp = TablePlan{};
+            pl.tp.repl_log2 = (uint32_t)repl;
+            pl.tp.prefetch = tune().prefetch != 0 ? 1u : 0u;
+            pl.warps = best_w;
+            pl.chains = best_c;
+            const size_t set = (size_t)best_w * best_c * span;
+            pl.smem = tab + pl.colsum_bytes + std::max(2 * set, set + xs_bytes);
+            pl.ok = true;
+            return pl;
+        }
+    }
+    return pl;
+}
+
+static int launch_rows(const Format& f, const RowsPlan& pl, int mode, const float* x, int64_t xs_i, float* y,
+                       int64_t ys_j, float* aux, cudaStream_t st) {
+    const bool guard = 3u * f.max_len > 32u;               // three code words may not fit one window
+    RowsKernel kernel = mode == 1 ? pick_rows_kernel<1>(pl.d.tab_kind != 0, pl.chains, pl.has_long, guard)
+                                  : pick_rows_kernel<0>(pl.d.tab_kind != 0, pl.chains, pl.has_long, guard);
+    int rc = prepare_kernel(kernel, pl.smem);
+    if (rc) return rc;
+    rc = launch_dependent(kernel, dim3(pl.grid), dim3((unsigned)pl.warps * 32), pl.smem, st, pl.d, pl.tp, x, xs_i, y, ys_j,
+                          aux, pl.colsum_bytes, (uint32_t)(f.stream.size() / 4));
+    if (rc) return rc;
+    HAC_CUDA(cudaGetLastError());
+    f.last_launches++;
+    return HAC_OK;
+}
+
 // mode 0: product with one input; mode 1: debug decode into `aux`.
 static int launch_vec(const Format& f, int mode, const float* x, int64_t xs_i, float* y, int64_t ys_j,
                       float* aux, cudaStream_t st, bool* vec_direct = nullptr) {
@@ -1813,35 +2452,39 @@ static int launch_vec(const Format& f, int mode, const float* x, int64_t xs_i, f
     if (rc) return rc;
     const DevFormat d = dev_format(f);
     if (d.units == 0) return HAC_OK;
+    if (!f.sparse) {
+        const RowsPlan pl = plan_rows(f, di, mode);
+        if (pl.ok) {
+            if (vec_direct) *vec_direct = true;
+            return launch_rows(f, pl, mode, x, xs_i, y, ys_j, aux, st);
+        }
+    }
     const size_t budget = (size_t)di.max_smem_optin;
     // HAC: two decode chains per lane when two staging areas per warp fit next to a fully
     // replicated table; sHAC: one
-    const int chains = f.sparse ? 2 : (d.units > 1 ? std::min(2, std::max(1, env_int("HAC_B200_CHAINS", 2))) : 1);
+    const int chains = f.sparse ? 2 : (d.units > 1 ? 2 : 1);
     size_t per_warp = (size_t)d.max_unit_chunks * 16 * chains;
     if (f.sparse && mode == 0) per_warp += ((size_t)(32u * f.S * (f.ri_bits / 8) + 15u) / 16u + 1u) * 16u * chains;
     size_t xbytes = 0;
     if (mode == 0) xbytes = f.sparse ? align16((size_t)f.n * 4) : align16(((size_t)f.n + (f.n / f.S + 1)) * 4);
-    const int want = std::min(32, std::max(1, env_int("HAC_B200_VEC_WARPS", 32)));
+    const int want = 32;
     // shared memory: tables + x + per-warp staging.  Prefer keeping x and all warps; give up
     // replicas of the level-1 table before giving up warps.
     bool x_shared = mode == 0;
-    const size_t min_tables = plan_smem_bytes(d.l1_bits, 0, d.sub_bytes) + 16;
+    const size_t min_tables = plan_smem_bytes(d.l1_entries, 0, d.sub_bytes) + 16;
     if (x_shared && xbytes + min_tables + per_warp * std::min(want, 8) > budget) { x_shared = false; xbytes = 0; }
     int warps = want;
     while (warps > 1 && xbytes + min_tables + per_warp * (size_t)warps > budget) --warps;
     if (xbytes + min_tables + per_warp * (size_t)warps > budget) return HAC_ERR_BUFFER_TOO_SMALL;
     const size_t fixed = f.sparse ? 16 : 0;                 // mbarrier of the bulk copy of x
     TablePlan tp = plan_tables(d, budget - fixed - xbytes - per_warp * (size_t)warps);
-    tp.x_bulk = (f.sparse && mode == 0 && x_shared && xs_i == 1 && (reinterpret_cast<uintptr_t>(x) & 15u) == 0 &&
-                 env_int("HAC_B200_X_BULK", 1) != 0)
-                    ? 1u : 0u;
-    const size_t smem = fixed + plan_smem_bytes(d.l1_bits, tp.repl_log2, d.sub_bytes) + xbytes + per_warp * warps;
+    tp.x_bulk = (f.sparse && mode == 0 && x_shared && xs_i == 1 && (reinterpret_cast<uintptr_t>(x) & 15u) == 0) ? 1u : 0u;
+    const size_t smem = fixed + plan_smem_bytes(d.l1_entries, tp.repl_log2, d.sub_bytes) + xbytes + per_warp * warps;
     if (smem > budget) return HAC_ERR_BUFFER_TOO_SMALL;
     const bool has_long = d.max_len > d.l1_bits;
     const int threads = warps * 32;
     // HAC with a short code word for zero: the zero-run table replaces the level-1 table
-    const bool runs = !f.sparse && mode == 0 && x_shared && !f.tables.l1_runs.empty() &&
-                      env_int("HAC_B200_ZERO_RUNS", 1) != 0;
+    const bool runs = !f.sparse && mode == 0 && x_shared && !f.tables.l1_runs.empty() && tune().zero_runs != 0;
     DevFormat dk = d;
     if (runs) { dk.l1 = reinterpret_cast<const uint2*>(f.dev.l1_runs); tp.zero_len = f.tables.zero_len; }
     VecKernel kernel = has_long ? pick_vec_kernel<true>(f, mode, x_shared, chains, runs)
@@ -1849,8 +2492,8 @@ static int launch_vec(const Format& f, int mode, const float* x, int64_t xs_i, f
     rc = prepare_kernel(kernel, smem);
     if (rc) return rc;
     int per_sm = 1;
-    HAC_CUDA(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kernel, threads, smem));
-    per_sm = std::max(per_sm, 1);
+    rc = blocks_per_sm(reinterpret_cast<const void*>(kernel), threads, smem, &per_sm);
+    if (rc) return rc;
     // spread the segments over all SMs (a block's warps take segments blockIdx + k * gridDim)
     const unsigned items = f.sparse ? d.items : (d.units + chains - 1) / chains;
     const unsigned grid = std::min<unsigned>(items, (unsigned)(di.sms * per_sm));
@@ -1877,14 +2520,14 @@ static int launch_gemm_tc(const Format& f, const DeviceInfo& di, const DevFormat
             // the stream buffers double as the epilogue's four 32 x 33 transpose tiles
             const size_t fx = 256 + 128 + (size_t)kGSlots * kGStages * kGXTileBytes +
                               std::max<size_t>((size_t)kGDecodeWarps * nb * kGChains * 32 * slot_bytes, 4 * 32 * 33 * 4);
-            if (fx + plan_smem_bytes(d.l1_bits, want_repl, d.sub_bytes) <= budget) { nbuf = nb; fixed = fx; break; }
+            if (fx + plan_smem_bytes(d.l1_entries, want_repl, d.sub_bytes) <= budget) { nbuf = nb; fixed = fx; break; }
         }
         if (nbuf) break;
     }
     if (!nbuf) return HAC_ERR_BUFFER_TOO_SMALL;
     const TablePlan tp = plan_tables(d, budget - fixed);
     // the block allocates all of tensor memory: ask for enough shared memory that no second block shares the SM
-    const size_t smem = std::max(fixed + plan_smem_bytes(d.l1_bits, tp.repl_log2, d.sub_bytes), budget / 2 + 1024);
+    const size_t smem = std::max(fixed + plan_smem_bytes(d.l1_entries, tp.repl_log2, d.sub_bytes), budget / 2 + 1024);
     int rc = prepare_kernel(hac_gemm_tc_kernel, smem);
     if (rc) return rc;
     const uint32_t col_blocks = (uint32_t)((f.m + kGCols - 1) / kGCols);
@@ -1918,13 +2561,12 @@ static int launch_batch_t(const Format& f, const DeviceInfo& di, const DevFormat
                           int64_t xs_b, int64_t batch, float* y, int64_t ys_j, int64_t ys_b, float* partial,
                           cudaStream_t st) {
     const size_t budget = (size_t)di.max_smem_optin;
-    const TablePlan tp = plan_tables(d, std::max<size_t>(32 * 1024, plan_smem_bytes(d.l1_bits, 0, d.sub_bytes)));
-    const size_t tab = plan_smem_bytes(d.l1_bits, tp.repl_log2, d.sub_bytes);
+    const TablePlan tp = plan_tables(d, std::max<size_t>(32 * 1024, plan_smem_bytes(d.l1_entries, 0, d.sub_bytes)));
+    const size_t tab = plan_smem_bytes(d.l1_entries, tp.repl_log2, d.sub_bytes);
     constexpr uint32_t kTile = 32 * kAcc;
     const uint32_t batch_tiles = (uint32_t)((batch + kTile - 1) / kTile);
     const size_t per_warp = (size_t)d.max_unit_chunks * 16 + 2 * kBatchRows * 4;
-    const int want = std::min(32, std::max(1, env_int("HAC_B200_BATCH_WARPS", 8)));
-    const int warps = fit_warps(tab + 32, per_warp, want, 1, budget);
+    const int warps = fit_warps(tab + 32, per_warp, 8, 1, budget);
     if (warps == 0) return HAC_ERR_BUFFER_TOO_SMALL;
     const size_t smem = tab + 32 + per_warp * warps;
     void (*kernel)(DevFormat, TablePlan, const float*, int64_t, int64_t, uint32_t, float*, int64_t, int64_t,
@@ -1932,8 +2574,8 @@ static int launch_batch_t(const Format& f, const DeviceInfo& di, const DevFormat
     int rc = prepare_kernel(kernel, smem);
     if (rc) return rc;
     int per_sm = 1;
-    HAC_CUDA(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kernel, warps * 32, smem));
-    per_sm = std::max(per_sm, 1);
+    rc = blocks_per_sm(reinterpret_cast<const void*>(kernel), warps * 32, smem, &per_sm);
+    if (rc) return rc;
     const uint64_t items = (uint64_t)d.units * batch_tiles;
     const unsigned grid = (unsigned)std::min<uint64_t>((items + warps - 1) / warps, (uint64_t)di.sms * per_sm);
     // up to 16 inputs: the smallest power of two that holds them, as lanes per entry
