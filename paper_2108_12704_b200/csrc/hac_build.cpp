@@ -651,8 +651,13 @@ int build_impl(const float* W, int64_t n, int64_t m, int64_t ldw, const hac_buil
             const uint32_t u_begin = f.seg_first[j], u_end = f.seg_first[j + 1];
             for (uint32_t u = u_begin; u < u_end; u += 2) {
                 const uint32_t in_item = std::min(2u, u_end - u);
-                uint32_t rec[12] = {0};
+                uint32_t rec[kItemWords] = {0};
                 for (uint32_t c = 0; c < in_item; ++c) {
+                    // the segment's 32 sub-segment bit lengths, so that one read brings all an item needs
+                    for (uint32_t l = 0; l < 32; ++l) {
+                        const uint32_t bits = f.sub_bits[(size_t)(u + c) * 32 + l];
+                        rec[12 + 16 * c + l / 2] |= bits << (16 * (l & 1u));
+                    }
                     const uint32_t pos0 = f.cb[j] + (u + c - u_begin) * 32u * S;
                     rec[4 * c + 0] = (uint32_t)(f.seg_bit_off[u + c] & 0xffffffffu);
                     rec[4 * c + 1] = (uint32_t)(f.seg_bit_off[u + c] >> 32);
@@ -662,7 +667,7 @@ int build_impl(const float* W, int64_t n, int64_t m, int64_t ldw, const hac_buil
                 rec[8] = (uint32_t)j;
                 rec[9] = in_item | ((u_end - u_begin) <= 2 ? 0x100u : 0u);   // bit 8: the item is the whole column
                 rec[10] = u;
-                f.item_info.insert(f.item_info.end(), rec, rec + 12);
+                f.item_info.insert(f.item_info.end(), rec, rec + kItemWords);
             }
         }
         f.max_units_per_col = 0;

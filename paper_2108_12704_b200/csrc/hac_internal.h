@@ -27,6 +27,7 @@ inline uint32_t xt_index(uint32_t window, int mant) {
 }
 constexpr size_t kSubTableBytesMax = 24 * 1024;
 constexpr int kStreamSlackWords = 4;     // zero words after the stream (decoder reads ahead)
+constexpr int kItemWords = 48;           // sHAC work item record: 12 header words, 2 x 16 words of sub-segment bit lengths, 4 spare
 
 // Decoding tables derived from the code lengths (canonical Huffman).  "rank" is the position of
 // a symbol in (length, id) order; values are stored in rank order so that short, frequent code
@@ -118,7 +119,7 @@ struct Format {
     std::vector<uint64_t> seg_bit_off;
     std::vector<uint16_t> sub_bits;
     std::vector<uint32_t> seg_first, seg_col;
-    std::vector<uint32_t> item_info;          // sHAC, device only: 12 words per work item (see ShacItem)
+    std::vector<uint32_t> item_info;          // sHAC, device only: kItemWords words per work item (see ShacItem)
     uint32_t max_unit_chunks = 0;             // largest 16-byte span a segment's stream covers
     uint32_t max_sub_chunks = 0;              // same for a single sub-segment
     uint32_t max_units_per_col = 0;

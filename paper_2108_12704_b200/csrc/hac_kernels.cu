@@ -1159,8 +1159,8 @@ struct ShacItem {
     uint32_t col, segments, whole_column, first_unit;
 };
 
-__device__ __forceinline__ ShacItem load_item(const void* base, uint32_t index) {     // 48-byte records
-    const uint4* w = reinterpret_cast<const uint4*>(base) + (size_t)index * 3;
+__device__ __forceinline__ ShacItem load_item(const void* base, uint32_t index) {     // header of a kItemWords record
+    const uint4* w = reinterpret_cast<const uint4*>(base) + (size_t)index * (kItemWords / 4);
     const uint4 a = __ldg(w), b = __ldg(w + 1), c = __ldg(w + 2);
     ShacItem r;
     r.bit_off[0] = ((uint64_t)a.y << 32) | a.x; r.pos0[0] = a.z; r.count[0] = a.w;
@@ -1367,6 +1367,288 @@ __global__ void __launch_bounds__(1024) shac_vec_kernel(DevFormat f, TablePlan t
             __syncwarp();
         }
     }
+}
+
+// This lane's sub-segment bit length in segment c of a work item (the copy kept inside the item record).
+__device__ __forceinline__ uint32_t load_item_bits(const void* base, uint32_t index, uint32_t c, uint32_t lane) {
+    const uint16_t* h = reinterpret_cast<const uint16_t*>(reinterpret_cast<const uint32_t*>(base) +
+                                                          (size_t)index * kItemWords + 12 + 16 * c);
+    return __ldg(h + lane);
+}
+
+// ------------------------------------------------------------------------------------------------
+// sHAC, one input vector (Algorithm 2 by segments), the kernel used when x and all staging areas fit in
+// shared memory.  A warp takes one work item at a time (up to two segments of one column = two decode
+// chains per lane).  Everything an item needs to be located comes in one read of its record; its two
+// spans of the stream and two slices of ri are then brought in by four bulk asynchronous copies (TMA,
+// issued by one lane, completion on the warp's own mbarrier), x by one more for the block.  Code words
+// are decoded three to a window (lookup3); the row of an entry comes from the staged slice of ri and
+// x is gathered from shared memory by row.
+//   kMode 0: product; 1: debug decode (values written to aux[position in nz]).
+// Every mbarrier wait is bounded; if one runs out the data is copied with ordinary loads instead.
+// ------------------------------------------------------------------------------------------------
+template <int kMode, int kTab, bool kLong, bool kGuard, typename RowT>
+__global__ void __launch_bounds__(1024) shac_items_kernel(DevFormat f, TablePlan tp, const float* __restrict__ x,
+                                                          int64_t xs_i, float* __restrict__ y, int64_t ys_j,
+                                                          float* __restrict__ aux) {
+    constexpr int kC = 2;
+    constexpr uint32_t kRow = (uint32_t)sizeof(RowT);
+    __shared__ DevFormat sf;               // for the rare paths that are calls (decode3_slow)
+    allow_dependents();
+    const uint32_t warp = threadIdx.x >> 5, lane = threadIdx.x & 31, warps = blockDim.x >> 5;
+    const uint32_t sb = shared_base();
+    const uint32_t xbar = sb, wbar = sb + 16 + 8 * warp;
+    // mbarriers first: the fence that publishes them would wait for any load already in flight
+    if (threadIdx.x == 0) mbar_init(xbar, 1);
+    if (lane == 0) mbar_init(wbar, 1);
+    __syncwarp();
+    uint32_t item = blockIdx.x + gridDim.x * warp;
+    ShacItem info;
+    info.segments = 0;
+    uint32_t my_bits[kC] = {0, 0};
+    // one trip: header and both arrays of lengths (zeros for an absent segment).  Taking the header apart
+    // waits for it, so the first record is asked for after everything else that can be in flight by then.
+    auto load_index = [&](uint32_t it) {
+#pragma unroll
+        for (int c = 0; c < kC; ++c) my_bits[c] = load_item_bits(f.unit_info, it, c, lane);
+        info = load_item(f.unit_info, it);
+    };
+    if (threadIdx.x == 0) sf = f;
+    // table entries: every warp takes groups of 32 consecutive entries, all its loads in flight at once
+    constexpr int kTabAhead = 2;
+    const uint32_t entries = f.l1_entries;
+    uint2 te[kTabAhead];
+#pragma unroll
+    for (int i = 0; i < kTabAhead; ++i) {
+        const uint32_t idx = (warp + i * warps) * 32 + lane;
+        te[i] = idx < entries ? __ldg(f.l1 + idx) : make_uint2(0u, 0u);
+    }
+    // shared memory: [mbarrier of x, mbarriers of the warps][x][tables][spans: warp, chain][ri slices: warp, chain]
+    unsigned char* p = smem + align16(16 + 8 * (size_t)warps);
+    float* xs = reinterpret_cast<float*>(p);
+    if (kMode == 0) p += align16((size_t)f.n * 4);
+    uint2* l1 = reinterpret_cast<uint2*>(p);
+    uint2* subt = reinterpret_cast<uint2*>(p + (((size_t)8 * f.l1_entries) << tp.repl_log2));
+    p += plan_smem_bytes(f.l1_entries, tp.repl_log2, f.sub_bytes);
+    const uint32_t span_bytes = f.max_unit_chunks * 16;
+    const uint32_t ri_bytes = kMode == 0 ? ((32u * f.S * kRow + 15u) / 16u + 1u) * 16u : 0u;
+    const uint32_t stage_a = smem_off(p) + warp * kC * span_bytes;
+    const uint32_t ri_a = smem_off(p) + warps * kC * span_bytes + warp * kC * ri_bytes;
+    const uint32_t xs_a = smem_off(xs);
+    const RowT* __restrict__ ri = reinterpret_cast<const RowT*>(f.ri);
+    const bool bulk = kMode == 0 && tp.x_bulk;
+    const uint32_t bulk_bytes = (f.n & ~3u) * 4u;
+
+    // requests the spans and slices of ri of the item whose record is in `info`; pos[c] = bit position of this
+    // lane's first code word relative to the staged span of chain c, ri_lane[c] = address of its first row index
+    uint32_t pos[kC], ri_lane[kC];
+    bool copy_lost = false;
+    auto fetch = [&]() {
+        uint32_t bytes_total = 0;
+        const uint4* src_s[kC]; const uint4* src_r[kC];
+        uint32_t n_s[kC], n_r[kC];
+#pragma unroll
+        for (int c = 0; c < kC; ++c) {
+            uint32_t total;
+            const uint32_t start = lane_start_bits(my_bits[c], lane, total);
+            pos[c] = 0; ri_lane[c] = ri_a; n_s[c] = 0; n_r[c] = 0; src_s[c] = nullptr; src_r[c] = nullptr;
+            if ((uint32_t)c < info.segments) {
+                const uint64_t first_chunk = info.bit_off[c] >> 7;
+                const uint64_t last_word = ((info.bit_off[c] + total) >> 5) + 2;
+                n_s[c] = (uint32_t)((last_word >> 2) - first_chunk + 1);
+                src_s[c] = reinterpret_cast<const uint4*>(f.stream) + first_chunk;
+                pos[c] = start + (uint32_t)(info.bit_off[c] - (first_chunk << 7));
+                if (kMode == 0) {
+                    const uintptr_t byte0 = reinterpret_cast<uintptr_t>(ri + info.pos0[c]);
+                    const uintptr_t chunk0 = byte0 & ~(uintptr_t)15;
+                    n_r[c] = (uint32_t)((byte0 + (uintptr_t)info.count[c] * kRow - chunk0 + 15) >> 4);
+                    src_r[c] = reinterpret_cast<const uint4*>(chunk0);
+                    ri_lane[c] = ri_a + c * ri_bytes + (uint32_t)(byte0 - chunk0) + lane * f.S * kRow;
+                }
+                bytes_total += 16u * (n_s[c] + n_r[c]);
+            }
+        }
+        if (lane == 0 && bytes_total > 0) {
+            mbar_expect_tx(wbar, bytes_total);
+#pragma unroll
+            for (int c = 0; c < kC; ++c) {
+                if (n_s[c]) bulk_copy_g2s(sb + stage_a + c * span_bytes, src_s[c], 16u * n_s[c], wbar);
+                if (n_r[c]) bulk_copy_g2s(sb + ri_a + c * ri_bytes, src_r[c], 16u * n_r[c], wbar);
+            }
+        }
+        __syncwarp();
+        return bytes_total;
+    };
+    // the same copies with ordinary loads: only after a wait on the mbarrier has run out
+    auto fetch_plain = [&]() {
+#pragma unroll
+        for (int c = 0; c < kC; ++c) {
+            if ((uint32_t)c >= info.segments) continue;
+            uint32_t total = 0;
+            for (int l = 0; l < 32; ++l) total += __shfl_sync(0xffffffffu, my_bits[c], l);
+            const uint64_t first_chunk = info.bit_off[c] >> 7;
+            const uint64_t last_word = ((info.bit_off[c] + total) >> 5) + 2;
+            const uint32_t ns = (uint32_t)((last_word >> 2) - first_chunk + 1);
+            const uint4* src = reinterpret_cast<const uint4*>(f.stream) + first_chunk;
+            uint4* dst = reinterpret_cast<uint4*>(smem + stage_a + c * span_bytes);
+            for (uint32_t k = lane; k < ns; k += 32) dst[k] = __ldg(src + k);
+            if (kMode == 0) {
+                const uintptr_t byte0 = reinterpret_cast<uintptr_t>(ri + info.pos0[c]);
+                const uintptr_t chunk0 = byte0 & ~(uintptr_t)15;
+                const uint32_t nr = (uint32_t)((byte0 + (uintptr_t)info.count[c] * kRow - chunk0 + 15) >> 4);
+                const uint4* srcr = reinterpret_cast<const uint4*>(chunk0);
+                uint4* dstr = reinterpret_cast<uint4*>(smem + ri_a + c * ri_bytes);
+                for (uint32_t k = lane; k < nr; k += 32) dstr[k] = __ldg(srcr + k);
+            }
+        }
+        __syncwarp();
+    };
+
+    // everything above reads the format only; x and the outputs belong to the kernels before this one
+    depends_wait();
+    if (bulk) {
+        if (threadIdx.x == 0 && bulk_bytes > 0) {
+            mbar_expect_tx(xbar, bulk_bytes);
+            bulk_copy_g2s(sb + xs_a, x, bulk_bytes, xbar);
+        }
+        for (uint32_t i = (f.n & ~3u) + threadIdx.x; i < f.n; i += blockDim.x) xs[i] = x[i];
+    }
+    uint32_t pending = 0;
+    if (item < f.items) { load_index(item); pending = fetch(); }
+    // tables -> shared memory, replicated (see TablePlan)
+    Decoder dec;
+    {
+        const uint32_t repl = 1u << tp.repl_log2;
+        auto spread = [&](uint32_t idx0, uint2 v) {
+            uint2* dst = l1 + ((size_t)idx0 << tp.repl_log2);
+            const uint32_t warp_slots = min(32u, entries - idx0) << tp.repl_log2;
+            for (uint32_t s0 = 0; s0 < warp_slots; s0 += 32) {
+                const uint32_t src = (s0 + lane) >> tp.repl_log2;
+                uint2 w;
+                w.x = __shfl_sync(0xffffffffu, v.x, src & 31u);
+                w.y = __shfl_sync(0xffffffffu, v.y, src & 31u);
+                if (s0 + lane < warp_slots) dst[s0 + lane] = w;
+            }
+        };
+#pragma unroll
+        for (int i = 0; i < kTabAhead; ++i) {
+            const uint32_t idx0 = (warp + i * warps) * 32;
+            if (idx0 < entries) spread(idx0, te[i]);
+        }
+        for (uint32_t idx0 = (warp + kTabAhead * warps) * 32; idx0 < entries; idx0 += warps * 32) {
+            const uint32_t idx = idx0 + lane;
+            spread(idx0, idx < entries ? __ldg(f.l1 + idx) : make_uint2(0u, 0u));
+        }
+        for (uint32_t i = threadIdx.x; i < f.sub_bytes / 8; i += blockDim.x) subt[i] = __ldg(f.sub + i);
+        dec.l1_lane = smem_off(l1) + ((threadIdx.x & (repl - 1)) << 3);
+        dec.l1_mul = 8u << tp.repl_log2;
+        dec.l1_shift = f.tab_kind ? 23 - f.xt_mant : 32 - f.l1_bits;
+        dec.bias = f.tab_kind ? (127u + f.xt_row0) << f.xt_mant : 0u;
+        dec.xt_low = f.xt_low;
+        dec.l1_bits = f.l1_bits;
+        dec.sub = smem_off(subt);
+    }
+    if (kMode == 0 && !bulk) {
+#pragma unroll 8
+        for (uint32_t i = threadIdx.x; i < f.n; i += blockDim.x) xs[i] = __ldg(x + (int64_t)i * xs_i);
+    }
+    __syncthreads();                       // tables (and an x copied by ordinary loads) are in place
+    if (bulk) {
+        const bool landed = bulk_bytes == 0 || mbar_wait_bounded(xbar, 0);
+        if (__syncthreads_or(landed ? 0 : 1)) {             // late or lost: copy x the ordinary way
+            for (uint32_t i = threadIdx.x; i < f.n; i += blockDim.x) xs[i] = x[i];
+            __syncthreads();
+        }
+    }
+    const uint32_t l1_abs = sb + dec.l1_lane - dec.bias * dec.l1_mul, xs_abs = sb + xs_a;
+    uint32_t phase = 0;
+    while (item < f.items) {
+        if (pending) {
+            const bool ok = mbar_wait_bounded(wbar, phase);
+            if (__any_sync(0xffffffffu, !ok)) { copy_lost = true; fetch_plain(); }
+            phase ^= 1u;
+        }
+        const ShacItem cur = info;
+        const uint32_t lane_pos = lane * f.S;
+        uint32_t count[kC];
+        FastReader fr[kC];
+        uint32_t ra[kC];
+#pragma unroll
+        for (int c = 0; c < kC; ++c) {
+            count[c] = ((uint32_t)c < cur.segments && lane_pos < cur.count[c]) ? min(f.S, cur.count[c] - lane_pos) : 0u;
+            BitReader br;
+            br.init(stage_a + c * span_bytes, pos[c]);
+            fr[c].hi = br.hi; fr[c].lo = br.lo; fr[c].off = br.off; fr[c].next = sb + br.next;
+            ra[c] = sb + ri_lane[c];
+        }
+        const uint32_t common = min(count[0], count[1]);
+        float acc[kC] = {0.0f, 0.0f};
+        float* out[kC];
+#pragma unroll
+        for (int c = 0; c < kC; ++c) out[c] = aux + cur.pos0[c] + lane_pos;
+        // one entry of chain c: value v, the s-th of the lane's sub-segment
+        auto apply = [&](int c, uint32_t v, uint32_t s) {
+            if (kMode == 0) {
+                const uint32_t row = kRow == 2 ? lds16(ra[c] - sb + s * kRow) : lds32(ra[c] - sb + s * kRow);
+                acc[c] = fmaf(ldsf(xs_a + (row << 2)), __uint_as_float(v), acc[c]);
+            } else {
+                out[c][s] = __uint_as_float(v);
+            }
+        };
+        auto triple = [&](int c, uint32_t s) {
+            uint32_t v0, v1, v2, tot, flags;
+            lookup3<kTab>(fr[c], dec.l1_shift, dec.l1_mul, l1_abs, dec.xt_low, v0, v1, v2, tot, flags);
+            if (kGuard || kLong) {
+                const bool bad = (kGuard && tot > 32u) || (kLong && (int32_t)flags < 0);
+                if (bad) {
+                    const Slow3 r = decode3_slow<kTab, kLong>(fr[c].hi, fr[c].lo, fr[c].off, fr[c].next - sb, dec, &sf);
+                    fr[c].hi = r.hi; fr[c].lo = r.lo; fr[c].off = r.off; fr[c].next = sb + r.next;
+                    v0 = r.v0; v1 = r.v1; v2 = r.v2; tot = 0;
+                }
+            }
+            fast_advance(fr[c], tot);
+            apply(c, v0, s); apply(c, v1, s + 1); apply(c, v2, s + 2);
+        };
+        uint32_t s = 0;
+        for (; s + 3 <= common; s += 3) {                         // both chains, three entries each
+            triple(0, s);
+            triple(1, s);
+        }
+#pragma unroll
+        for (int c = 0; c < kC; ++c) {                            // what one chain has beyond the other, and the ends
+            uint32_t t = s;
+            for (; t + 3 <= count[c]; t += 3) triple(c, t);
+            for (; t < count[c]; ++t) {
+                uint32_t top, val, len;
+                table_lookup<kTab>(fr[c], dec.l1_shift, dec.l1_mul, l1_abs, dec.xt_low, top, val, len);
+                if (kLong && (int32_t)len < 0) resolve_any<kTab>(top, dec, f, val, len);
+                fast_advance(fr[c], len);
+                apply(c, val, t);
+            }
+        }
+        (void)xs_abs;
+        // the record of the next item is requested before the reduction
+        const uint32_t next_item = item + gridDim.x * warps;
+        __syncwarp();                      // every lane has finished reading the staging areas
+        if (next_item < f.items) load_index(next_item);
+        if (kMode == 0) {
+#pragma unroll
+            for (int c = 0; c < kC; ++c) acc[c] = warp_sum(acc[c]);
+            if (lane == 0) {
+                if (cur.whole_column) {
+                    y[(int64_t)cur.col * ys_j] = acc[0] + acc[1];
+                } else {
+#pragma unroll
+                    for (int c = 0; c < kC; ++c)
+                        if ((uint32_t)c < cur.segments) aux[cur.first_unit + c] = acc[c];
+                }
+            }
+        }
+        item = next_item;
+        pending = 0;
+        if (item < f.items) pending = fetch();
+    }
+    (void)copy_lost;
 }
 
 // Columns made of several segments (or none): add the per-segment partials in segment order.
@@ -2055,10 +2337,11 @@ struct Tune {
     int xt;             // HAC_B200_XT=0: never use the magnitude table
     int prefetch;       // HAC_B200_PREFETCH=0: no L2 prefetch of the stream at the start of the rows-in-registers kernel
     int rows_chains;    // HAC_B200_ROWS_CHAINS=2|3: decode chains per lane of that kernel (0 = chosen by the library)
+    int items_kernel;   // HAC_B200_ITEMS=0: single-input sHAC always through the older kernel
 };
 static const Tune& tune() {
     static const Tune t = {env_int("HAC_B200_PDL", 1), env_int("HAC_B200_ROWS", 1), env_int("HAC_B200_ROWS_WARPS", 0),
-                           env_int("HAC_B200_ZERO_RUNS", 1), env_int("HAC_B200_XT", 1), env_int("HAC_B200_PREFETCH", 1), env_int("HAC_B200_ROWS_CHAINS", 0)};
+                           env_int("HAC_B200_ZERO_RUNS", 1), env_int("HAC_B200_XT", 1), env_int("HAC_B200_PREFETCH", 1), env_int("HAC_B200_ROWS_CHAINS", 0), env_int("HAC_B200_ITEMS", 1)};
     return t;
 }
 
@@ -2068,7 +2351,7 @@ static DevFormat dev_format(const Format& f) {
     d.l1 = reinterpret_cast<const uint2*>(f.dev.l1); d.sub = reinterpret_cast<const uint2*>(f.dev.sub);
     d.l1_bits = (uint32_t)f.tables.l1_bits; d.sub_bytes = (uint32_t)(f.tables.sub.size() * 4);
     d.l1_entries = 1u << d.l1_bits;
-    d.items = (uint32_t)(f.item_info.size() / 12);
+    d.items = (uint32_t)(f.item_info.size() / kItemWords);
     d.limit = f.dev.limit; d.first_left = f.dev.first_left; d.rank_base = f.dev.rank_base;
     d.seg_bit_off = f.dev.seg_bit_off; d.sub_bits = f.dev.sub_bits; d.seg_col = f.dev.seg_col;
     d.seg_first = f.dev.seg_first; d.ri = f.dev.ri; d.cb = f.dev.cb; d.unit_info = f.dev.unit_info;
@@ -2444,6 +2727,64 @@ static int launch_rows(const Format& f, const RowsPlan& pl, int mode, const floa
     return HAC_OK;
 }
 
+// ---- single-input sHAC with everything an item needs staged by bulk copies -------------------------
+typedef void (*ItemsKernel)(DevFormat, TablePlan, const float*, int64_t, float*, int64_t, float*);
+
+template <int kMode, int kTab, typename RowT>
+static ItemsKernel pick_items_kernel3(bool has_long, bool guard) {
+    if (kMode == 1 || has_long) return shac_items_kernel<kMode, kTab, true, true, RowT>;     // the test path takes the general one
+    return guard ? shac_items_kernel<kMode, kTab, false, true, RowT> : shac_items_kernel<kMode, kTab, false, false, RowT>;
+}
+template <int kMode, int kTab>
+static ItemsKernel pick_items_kernel2(uint32_t ri_bits, bool has_long, bool guard) {
+    return ri_bits == 16 ? pick_items_kernel3<kMode, kTab, uint16_t>(has_long, guard)
+                         : pick_items_kernel3<kMode, kTab, uint32_t>(has_long, guard);
+}
+template <int kMode>
+static ItemsKernel pick_items_kernel(bool xt, uint32_t ri_bits, bool has_long, bool guard) {
+    return xt ? pick_items_kernel2<kMode, 1>(ri_bits, has_long, guard) : pick_items_kernel2<kMode, 0>(ri_bits, has_long, guard);
+}
+
+// Launches shac_items_kernel if x, the tables and the staging areas of at least 16 warps fit in an SM's shared
+// memory; *launched tells whether it did.
+static int launch_items(const Format& f, const DeviceInfo& di, int mode, const float* x, int64_t xs_i, float* y,
+                        int64_t ys_j, float* aux, cudaStream_t st, bool* launched) {
+    *launched = false;
+    if (!f.sparse || tune().items_kernel == 0) return HAC_OK;
+    const DevFormat d = dev_format_xt(f);
+    if (d.items == 0) return HAC_OK;
+    const size_t budget = (size_t)di.max_smem_optin - 256;       // static shared memory of the kernel
+    const size_t xbytes = mode == 0 ? align16((size_t)f.n * 4) : 0;
+    const size_t ri_stage = mode == 0 ? ((size_t)(32u * f.S * (f.ri_bits / 8) + 15u) / 16u + 1u) * 16u : 0;
+    const size_t per_warp = 2 * ((size_t)d.max_unit_chunks * 16 + ri_stage);
+    int warps = 0, repl = 4;
+    for (; repl >= 0 && !warps; --repl) {
+        const size_t tab = plan_smem_bytes(d.l1_entries, (uint32_t)repl, d.sub_bytes);
+        for (int w = 32; w >= 16; w -= 4) {
+            if (align16(16 + 8 * (size_t)w) + xbytes + tab + per_warp * (size_t)w <= budget) { warps = w; break; }
+        }
+        if (warps) break;
+    }
+    if (!warps) return HAC_OK;
+    TablePlan tp{};
+    tp.repl_log2 = (uint32_t)repl;
+    tp.x_bulk = (mode == 0 && xs_i == 1 && (reinterpret_cast<uintptr_t>(x) & 15u) == 0) ? 1u : 0u;
+    const size_t smem = align16(16 + 8 * (size_t)warps) + xbytes + plan_smem_bytes(d.l1_entries, tp.repl_log2, d.sub_bytes) +
+                        per_warp * (size_t)warps;
+    const bool has_long = table_has_long(f, d), guard = 3u * f.max_len > 32u;
+    ItemsKernel kernel = mode == 1 ? pick_items_kernel<1>(d.tab_kind != 0, f.ri_bits, has_long, guard)
+                                   : pick_items_kernel<0>(d.tab_kind != 0, f.ri_bits, has_long, guard);
+    int rc = prepare_kernel(kernel, smem);
+    if (rc) return rc;
+    const unsigned grid = std::min<unsigned>(d.items, (unsigned)di.sms);
+    rc = launch_dependent(kernel, dim3(grid), dim3((unsigned)warps * 32), smem, st, d, tp, x, xs_i, y, ys_j, aux);
+    if (rc) return rc;
+    HAC_CUDA(cudaGetLastError());
+    f.last_launches++;
+    *launched = true;
+    return HAC_OK;
+}
+
 // mode 0: product with one input; mode 1: debug decode into `aux`.
 static int launch_vec(const Format& f, int mode, const float* x, int64_t xs_i, float* y, int64_t ys_j,
                       float* aux, cudaStream_t st, bool* vec_direct = nullptr) {
@@ -2458,6 +2799,10 @@ static int launch_vec(const Format& f, int mode, const float* x, int64_t xs_i, f
             if (vec_direct) *vec_direct = true;
             return launch_rows(f, pl, mode, x, xs_i, y, ys_j, aux, st);
         }
+    } else {
+        bool launched = false;
+        rc = launch_items(f, di, mode, x, xs_i, y, ys_j, aux, st, &launched);
+        if (rc || launched) return rc;
     }
     const size_t budget = (size_t)di.max_smem_optin;
     // HAC: two decode chains per lane when two staging areas per warp fit next to a fully

@@ -152,3 +152,17 @@ def test_device_calls_fail_loudly_without_upload():
     lib = hb.load()
     rc = lib.shac_dot(lf._h, 16, 1, 1, 0, 16, 1, 0, None, 0, None)
     assert rc == -7          # HAC_ERR_NOT_UPLOADED: no silent fallback
+
+
+def test_library_kmeans_on_the_hand_worked_example():
+    """The library's own k-means reproduces the centroids of tests/golden/kmeans_hand_worked.txt."""
+    from fractions import Fraction
+    from golden_io import golden, read_sections
+    g = read_sections(golden("kmeans_hand_worked.txt"))
+    W = np.array([float(v) for v in g["data"][0]], dtype=np.float32).reshape(-1, 1)
+    k, seed = int(g["k"][0][0]), int(g["seed"][0][0])
+    for iters in (1, 2):
+        want = sorted({np.float32(float(Fraction(v))) for v in g[f"centroids_after_{iters}"][0]})
+        for kind in ("hac", "shac"):
+            f = hb.Format(kind, W, sparsity=0.0, k=k, quantizer=si.QUANT_KMEANS, kmeans_iters=iters, seed=seed)
+            assert f.export()["codebook"].tolist() == [float(v) for v in want]

@@ -295,3 +295,29 @@ def test_pws_with_256_values_codes_at_8_bits_like_the_papers_table():
     Wq, mask = orc.pws_share(W, 256, seed=1)
     fmt = orc.hac_encode(Wq)
     assert 7.9 <= fmt["bits"] / W.size <= 8.05
+
+
+# ---------------------------------------------------------------- k-means against a hand-worked example
+def test_kmeans_two_iterations_worked_by_hand():
+    """Pins the Lloyd rule itself (midpoint assignment, a weight on a midpoint goes down, mean update,
+    exactly `iters` updates and one more assignment) against tests/golden/kmeans_hand_worked.txt,
+    whose numbers were derived on paper as exact fractions."""
+    from fractions import Fraction
+    from golden_io import golden, read_sections
+    g = read_sections(golden("kmeans_hand_worked.txt"))
+    data = np.array([float(v) for v in g["data"][0]], dtype=np.float32)
+    k, seed = int(g["k"][0][0]), int(g["seed"][0][0])
+    start = [float(v) for v in g["start"][0]]
+    assert orc.kmeans_init(np.unique(data.astype(np.float64)), k, seed).tolist() == start
+    W = data.reshape(-1, 1)
+    sse_want = [float(Fraction(v)) for v in g["sse"][0]]
+    for iters in (1, 2):
+        want_c = [Fraction(v) for v in g[f"centroids_after_{iters}"][0]]
+        want_a = [int(v) for v in g[f"assign_iters_{iters}"][0]]
+        Wq, mask, c, sse = orc.kmeans_share(W, k, iters, seed, return_trace=True)
+        assert mask.all()
+        # the centroids are the fractions rounded once to double
+        assert c.tolist() == [float(f) for f in want_c]
+        want_values = np.array([np.float32(float(want_c[a])) for a in want_a], dtype=np.float32)
+        assert np.array_equal(Wq.ravel().view(np.uint32), want_values.view(np.uint32))
+        assert np.allclose(sse[:iters + 1], sse_want[:iters + 1], rtol=1e-12, atol=0)
