@@ -397,23 +397,34 @@ def run_ours(args):
     gemm_s = median(t_gemm) * 1e-3 / K
 
     # ---- end to end through the host entry point: pinned host X / Y, copies inside the timed region ----------
-    xh1 = torch.from_numpy(si.inputs(wl, 1)).pin_memory()
-    yh1 = torch.empty((1, m), dtype=torch.float32).pin_memory()
-    xhB = torch.from_numpy(xb_host).pin_memory()
-    yhB = torch.empty((GEMM_BATCH, m), dtype=torch.float32).pin_memory()
-    scratch = torch.empty(max(fmt.dot_host_scratch_bytes(1), fmt.dot_host_scratch_bytes(GEMM_BATCH)),
-                          dtype=torch.uint8, device=dev)
-    for i in range(3):
-        fmt.attach(reps[i % R]); fmt.dot_host(xh1, yh1, scratch); fmt.dot_host(xhB, yhB, scratch)
+    # Two streams, each with its own pinned buffers and device staging area, take the steps in turn through the
+    # asynchronous host entry point, so that the copies of one step overlap the kernels of the other.
+    lanes = []
+    for _ in range(2):
+        lanes.append(dict(
+            stream=torch.cuda.Stream(device=dev),
+            xh1=torch.from_numpy(si.inputs(wl, 1)).pin_memory(), yh1=torch.empty((1, m), dtype=torch.float32).pin_memory(),
+            xhB=torch.from_numpy(xb_host).pin_memory(), yhB=torch.empty((GEMM_BATCH, m), dtype=torch.float32).pin_memory(),
+            scratch=torch.empty(max(fmt.dot_host_scratch_bytes(1), fmt.dot_host_scratch_bytes(GEMM_BATCH)),
+                                dtype=torch.uint8, device=dev)))
+
+    def e2e_step(i):
+        ln = lanes[i % 2]
+        with torch.cuda.stream(ln["stream"]):
+            fmt.attach(reps[i % R])
+            fmt.dot_host(ln["xh1"], ln["yh1"], ln["scratch"], wait=False)
+            fmt.dot_host(ln["xhB"], ln["yhB"], ln["scratch"], wait=False)
+
+    for i in range(4):
+        e2e_step(i)
     torch.cuda.synchronize()
+    check_against_host_decode(fmt, xb_host, lanes[0]["yhB"].numpy(), "HAC GEMM through the host entry point")
     if dist is not None:
         dist.barrier()
     Ke = 0
     t0 = time.perf_counter()
     while Ke < K or time.perf_counter() - t0 < 0.3:
-        fmt.attach(reps[Ke % R])
-        fmt.dot_host(xh1, yh1, scratch)
-        fmt.dot_host(xhB, yhB, scratch)
+        e2e_step(Ke)
         Ke += 1
         if Ke >= 20000:
             break
@@ -422,7 +433,7 @@ def run_ours(args):
     e2e_job_ms, e2e_units = reduce_job(e2e_ms, weights_per_step * Ke, dist)
     e2e_value = e2e_units / (e2e_job_ms * 1e-3) / 1e9
     hac_launches = leg_gemv.launches_per_product + leg_gemm.launches_per_product
-    del leg_gemv, leg_gemm, reps, x1, xB, y1, yB, scratch
+    del leg_gemv, leg_gemm, reps, x1, xB, y1, yB, lanes
     torch.cuda.empty_cache()
 
     # ---- the sHAC workload (large pruned fully connected layer), timed the same way, reported beside ----------
@@ -517,7 +528,7 @@ def run_ours(args):
                       for b, leg, t in zip(sbatches, slegB, st_legs[1:])},
         "roofline": roofline, "roofline_gemm": roofline_gemm, "roofline_shac": roofline_shac,
         "cpu_baseline": cpu_baseline,
-        "e2e": {"value": e2e_value, "unit": UNIT, "steps": Ke,
+        "e2e": {"value": e2e_value, "unit": UNIT, "steps": Ke, "how": "hac_dot_host_async on two alternating streams, pinned host X and Y, one synchronize at the end",
                 "h2d_bytes_per_step": 4 * n * (1 + GEMM_BATCH), "d2h_bytes_per_step": 4 * m * (1 + GEMM_BATCH)},
         "gpu_launches": repeats * K * hac_launches,
         "gpu_launches_shac": len(st_whole) * shac_launches,

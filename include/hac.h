@@ -139,16 +139,23 @@ typedef struct shac_host_view {
  *          duration of the call.  NaN / Inf -> HAC_ERR_NONFINITE_INPUT.  -0.0 counts as 0.
  *   params see hac_build_params.
  *   out    receives the new handle.
- * Steps: entries with |w| <= the floor(sparsity*n*m)-th smallest magnitude become 0; the others are
- * replaced by one of k shared values (k-means over them in column-major order, a uniform grid over
- * their range, or the zero-anchored grid delta * round(w / delta) whose delta is found by 70 halvings
- * of [0, 4 max|w|]: a trial delta that leaves at most k distinct values becomes the upper end, the
- * upper end is used; or probabilistic sharing between the two neighbouring i/(k-1) quantiles, the
- * i-th quantile being the order statistic floor(i (q-1)/(k-1)) of the q non-null weights and weight
- * p using the uniform number (SplitMix64(seed + (p+1) * 0x9E3779B97F4A7C15) >> 11) * 2^-53; weights
- * with at most k distinct values are kept as they are); distinct values sorted ascending form the codebook; a Huffman code over the
- * symbol counts (HAC: every entry, zeros included; sHAC: stored entries only) is made canonical;
- * code words are concatenated column by column, most significant bit first, into 32-bit words.
+ * Steps:
+ *   1. Pruning (Sect. III-B): entries with |w| <= the floor(sparsity*n*m)-th smallest magnitude become 0.
+ *   2. Weight sharing (Sect. III-C) of the others, taken in column-major order, by `quantizer`:
+ *        HAC_QUANT_KMEANS   k-means (Lloyd, kmeans_iters updates, start drawn from `seed`);
+ *        HAC_QUANT_UNIFORM  a uniform grid of k levels over [min, max];
+ *        HAC_QUANT_GRID     the zero-anchored grid delta * round(w / delta); delta is found by 70 halvings
+ *                           of [0, 4 max|w|]: a trial delta that leaves at most k distinct values becomes
+ *                           the upper end, and the upper end is used;
+ *        HAC_QUANT_PWS      probabilistic sharing between the two neighbouring i/(k-1) quantiles (the i-th
+ *                           quantile is the order statistic floor(i (q-1)/(k-1)) of the q non-null weights;
+ *                           weight p draws (SplitMix64(seed + (p+1) * 0x9E3779B97F4A7C15) >> 11) * 2^-53);
+ *        HAC_QUANT_NONE     none.
+ *      Weights with at most k distinct values are kept as they are.
+ *   3. The distinct values, sorted ascending, form the codebook.
+ *   4. A Huffman code over the symbol counts (HAC: every entry, zeros included; sHAC: stored entries
+ *      only), made canonical.
+ *   5. Code words concatenated column by column, most significant bit first, into 32-bit words.
  * Offset index (the column-offset vector suggested in the paper's conclusions, refined): each column
  * (HAC: its n entries; sHAC: its stored entries) is cut into sub-segments of S symbols, 32
  * consecutive sub-segments form a segment; seg_bit_off[u] is the bit where segment u starts and
@@ -183,7 +190,10 @@ int shac_device_bytes(const shac_format* f, size_t* out);
 int hac_upload (hac_format*  f, void* dev_buf, size_t dev_bytes, void* cuda_stream);
 int shac_upload(shac_format* f, void* dev_buf, size_t dev_bytes, void* cuda_stream);
 /* Point the handle at a device image that *_upload wrote earlier and that was then copied, byte
- * for byte, to `dev_buf` (same device).  No copy is made. */
+ * for byte, to `dev_buf` (same device).  No copy is made.  That copy must be COMPLETE (synchronised, or
+ * made by an earlier operation of the stream the products will run on whose kernels have finished) before
+ * the first product on it: the product kernels start reading the format ahead of stream order (see
+ * hac_dot). */
 int hac_attach (hac_format*  f, void* dev_buf, size_t dev_bytes);
 int shac_attach(shac_format* f, void* dev_buf, size_t dev_bytes);
 
@@ -220,13 +230,20 @@ int shac_dot(const shac_format* f, const float* x, int64_t batch, int64_t x_stri
 /* The same product for HOST inputs and outputs (Algorithm 3's calling convention: X is batch x n,
  * one input per row, Y is batch x m, both contiguous host fp32, ideally pinned).  The caller gives a
  * device staging buffer `dev_scratch` of at least *_dot_host_scratch_bytes(f, batch) bytes; the call
- * copies X to the device, runs the product, copies Y back and waits for cuda_stream. */
+ * copies X to the device, runs the product, copies Y back and waits for cuda_stream.
+ * *_dot_host_async enqueues the same three steps and returns without waiting: Y_host is valid, and
+ * X_host, Y_host and dev_scratch may be reused, once the caller has synchronised cuda_stream.  Two
+ * streams with a staging buffer each let the copies of one product overlap the kernels of another. */
 int hac_dot_host_scratch_bytes (const hac_format*  f, int64_t batch, size_t* out);
 int shac_dot_host_scratch_bytes(const shac_format* f, int64_t batch, size_t* out);
 int hac_dot_host (const hac_format*  f, const float* X_host, int64_t batch, float* Y_host,
                   void* dev_scratch, size_t dev_scratch_bytes, void* cuda_stream);
 int shac_dot_host(const shac_format* f, const float* X_host, int64_t batch, float* Y_host,
                   void* dev_scratch, size_t dev_scratch_bytes, void* cuda_stream);
+int hac_dot_host_async (const hac_format*  f, const float* X_host, int64_t batch, float* Y_host,
+                        void* dev_scratch, size_t dev_scratch_bytes, void* cuda_stream);
+int shac_dot_host_async(const shac_format* f, const float* X_host, int64_t batch, float* Y_host,
+                        void* dev_scratch, size_t dev_scratch_bytes, void* cuda_stream);
 
 /* ---------------------------------------------------------------------------------------------
  * hac_dot_noalloc - the HAC product of hac_dot for callers that cannot hand over a workspace.
@@ -267,6 +284,16 @@ int hac_dot_noalloc(const hac_format* f, const float* x, int64_t batch, int64_t 
 int hac_debug_decode (const hac_format*  f, float* W_colmajor_dev, void* cuda_stream);
 int shac_debug_decode(const shac_format* f, float* nz_dev, void* cuda_stream);
 
+/* TEST ONLY, host: what the kernels' first-level decoding table holds for a 32-bit window of the stream
+ * (most significant bit = next bit to decode): *length = 0 if the entry leaves the code word to the slower
+ * levels, else the code word's length and *value the shared value it stands for (Sect. IV-B: the inverse
+ * dictionary H^-1).  *kind = 0 for the table indexed by the leading bits, 1 for the one indexed by the
+ * magnitude of the inverted window; *never_unresolved = 1 if the kernels rely on every window being resolved. */
+int hac_debug_table_lookup (const hac_format*  f, uint32_t window, float* value, uint32_t* length, int* kind,
+                            int* never_unresolved);
+int shac_debug_table_lookup(const shac_format* f, uint32_t window, float* value, uint32_t* length, int* kind,
+                            int* never_unresolved);
+
 /* Number of kernels the last dot / debug call on this handle launched (for launch accounting). */
 int hac_last_launch_count (const hac_format*  f);
 int shac_last_launch_count(const shac_format* f);
@@ -277,6 +304,17 @@ void shac_free(shac_format* f);
 const char* hac_status_string(int status);
 /* Text of the last CUDA error seen by this library on the calling thread ("" if none). */
 const char* hac_last_cuda_error(void);
+
+/* Diagnostic switches.  Environment variables, read once when the first product is launched (changing
+ * them later has no effect); they select between code paths that all give the same results:
+ *   HAC_B200_PDL=0          launch without programmatic stream serialization
+ *   HAC_B200_ROWS=0         single-input HAC always through the kernel that keeps x in shared memory
+ *   HAC_B200_ROWS_WARPS=n   warps per block of the rows-in-registers kernel (default: chosen per format)
+ *   HAC_B200_ROWS_CHAINS=c  decode chains per lane of that kernel, 2 or 3 (default 2)
+ *   HAC_B200_PREFETCH=0     no request of the block's share of the stream into L2 at its start
+ *   HAC_B200_ITEMS=0        single-input sHAC always through the older kernel
+ *   HAC_B200_ZERO_RUNS=0    never use the zero-run table of mostly-zero HAC streams
+ *   HAC_B200_XT=0           never use the magnitude-indexed first-level table */
 
 #ifdef __cplusplus
 }

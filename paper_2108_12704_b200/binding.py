@@ -62,7 +62,8 @@ EXPORTS = (
     "hac_decode_host", "shac_decode_host", "hac_device_bytes", "shac_device_bytes", "hac_upload",
     "shac_upload", "hac_attach", "shac_attach", "hac_workspace_bytes", "shac_workspace_bytes", "hac_dot",
     "shac_dot", "hac_dot_noalloc", "hac_dot_host_scratch_bytes", "shac_dot_host_scratch_bytes", "hac_dot_host",
-    "shac_dot_host", "hac_debug_decode", "shac_debug_decode", "hac_last_launch_count",
+    "shac_dot_host", "hac_dot_host_async", "shac_dot_host_async", "hac_debug_decode", "shac_debug_decode",
+    "hac_debug_table_lookup", "shac_debug_table_lookup", "hac_last_launch_count",
     "shac_last_launch_count", "hac_free", "shac_free", "hac_status_string", "hac_last_cuda_error",
 )
 
@@ -94,7 +95,10 @@ def load():
         getattr(lib, f"{kind}_dot").argtypes = [vp, fp, i64, i64, i64, fp, i64, i64, vp, sz, vp]
         getattr(lib, f"{kind}_dot_host_scratch_bytes").argtypes = [vp, i64, C.POINTER(sz)]
         getattr(lib, f"{kind}_dot_host").argtypes = [vp, fp, i64, fp, vp, sz, vp]
+        getattr(lib, f"{kind}_dot_host_async").argtypes = [vp, fp, i64, fp, vp, sz, vp]
         getattr(lib, f"{kind}_debug_decode").argtypes = [vp, fp, vp]
+        getattr(lib, f"{kind}_debug_table_lookup").argtypes = [vp, C.c_uint32, C.POINTER(C.c_float), C.POINTER(C.c_uint32),
+                                                               C.POINTER(C.c_int), C.POINTER(C.c_int)]
         getattr(lib, f"{kind}_last_launch_count").argtypes = [vp]
         getattr(lib, f"{kind}_free").argtypes = [vp]
         getattr(lib, f"{kind}_free").restype = None
@@ -285,15 +289,17 @@ class Format:
         _check(self._fn("dot_host_scratch_bytes")(self._h, int(batch), C.byref(s)), "dot_host_scratch_bytes")
         return s.value
 
-    def dot_host(self, X_host, Y_host, scratch):
+    def dot_host(self, X_host, Y_host, scratch, wait=True):
         """Host-to-host product: X_host [B, n] and Y_host [B, m] are CPU float32 tensors (pinned for
-        speed) or numpy arrays, scratch a torch uint8 CUDA tensor.  Waits for completion."""
+        speed) or numpy arrays, scratch a torch uint8 CUDA tensor.  Waits for completion; with
+        wait=False (the *_dot_host_async entry points) the work is only enqueued on the current stream."""
         import torch
         B = X_host.shape[0] if X_host.ndim == 2 else 1
         xp = X_host.data_ptr() if hasattr(X_host, "data_ptr") else X_host.ctypes.data
         yp = Y_host.data_ptr() if hasattr(Y_host, "data_ptr") else Y_host.ctypes.data
         st = torch.cuda.current_stream().cuda_stream
-        _check(self._fn("dot_host")(self._h, xp, B, yp, scratch.data_ptr(), scratch.numel(), st), "dot_host")
+        name = "dot_host" if wait else "dot_host_async"
+        _check(self._fn(name)(self._h, xp, B, yp, scratch.data_ptr(), scratch.numel(), st), name)
         return Y_host
 
     def debug_decode(self):
@@ -305,6 +311,13 @@ class Format:
         _check(self._fn("debug_decode")(self._h, out.data_ptr(), st), "debug_decode")
         out = out[:count]
         return out.view(self.m, self.n) if self.kind == "hac" else out
+
+    def debug_table_lookup(self, window: int):
+        """TEST ONLY: (value, length, kind, never_unresolved) of the kernels' first-level table for a 32-bit window."""
+        v, l, k, nu = C.c_float(), C.c_uint32(), C.c_int(), C.c_int()
+        _check(self._fn("debug_table_lookup")(self._h, C.c_uint32(window & 0xffffffff), C.byref(v), C.byref(l),
+                                              C.byref(k), C.byref(nu)), "debug_table_lookup")
+        return v.value, l.value, k.value, bool(nu.value)
 
     def last_launch_count(self) -> int:
         return self._fn("last_launch_count")(self._h)

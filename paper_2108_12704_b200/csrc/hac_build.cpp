@@ -679,6 +679,23 @@ int build_impl(const float* W, int64_t n, int64_t m, int64_t ldw, const hac_buil
         }
     } else {
         f.max_units_per_col = f.G;
+        const uint64_t tasks = ((uint64_t)n + S - 1) / S;
+        f.task_off.clear();
+        if ((tasks + 1) * (uint64_t)m * 8 <= kTaskOffBytesMax) {
+            f.task_off.assign((size_t)((tasks + 1) * (uint64_t)m), 0);
+            for (int64_t j = 0; j < m; ++j) {
+                uint64_t t = 0;
+                for (uint32_t g = 0; g < f.G; ++g) {
+                    const size_t u = (size_t)j * f.G + g;
+                    uint64_t at = f.seg_bit_off[u];
+                    for (uint32_t l = 0; l < 32 && t < tasks; ++l, ++t) {
+                        f.task_off[(size_t)t * m + j] = at;
+                        at += f.sub_bits[u * 32 + l];
+                    }
+                    if (t == tasks) f.task_off[(size_t)tasks * m + j] = at;
+                }
+            }
+        }
     }
     make_decode_tables(f);
     return HAC_OK;
@@ -784,6 +801,7 @@ ImageLayout image_layout(const Format& f) {
     L.ri = take(f.ri_bits == 16 ? f.ri16.size() * 2 + 16 : f.ri32.size() * 4 + 16);
     L.cb = take(f.cb.size() * 4);
     L.unit_info = take(f.item_info.size() * 4);
+    L.task_off = take(f.task_off.size() * 8);
     L.total = o;
     return L;
 }
@@ -792,7 +810,40 @@ ImageLayout image_layout(const Format& f) {
 
 using hacb200::Format;
 
+// What the first-level decoding table of the kernels holds for a 32-bit window (test support).
+static int table_lookup_host(const Format& f, uint32_t window, float* value, uint32_t* length, int* kind,
+                             int* never_unresolved) {
+    if (!value || !length || !kind || !never_unresolved) return HAC_ERR_INVALID_ARG;
+    const hacb200::DecodeTables& t = f.tables;
+    uint32_t v = 0, meta = 0;
+    if (t.use_xt) {
+        const uint32_t low = f.max_len < 32u ? ((1u << (32u - f.max_len)) - 1u) | 1u : 1u;
+        const uint32_t idx = hacb200::xt_index(~(~window | low), t.xt_mant);     // the index the kernels form from ~window | low
+        v = t.xt[2 * (size_t)idx]; meta = t.xt[2 * (size_t)idx + 1];
+        *kind = 1;
+        *never_unresolved = t.xt_unresolved == 0.0;
+    } else {
+        if (t.l1.empty()) return HAC_ERR_INVALID_ARG;
+        const uint32_t idx = t.l1_bits >= 32 ? window : window >> (32 - t.l1_bits);
+        v = t.l1[2 * (size_t)idx]; meta = t.l1[2 * (size_t)idx + 1];
+        *kind = 0;
+        *never_unresolved = f.max_len <= (uint32_t)t.l1_bits;
+    }
+    if (meta & 0x80000000u) { *length = 0; *value = 0.0f; }
+    else { *length = meta; std::memcpy(value, &v, 4); }
+    return HAC_OK;
+}
+
 extern "C" {
+
+int hac_debug_table_lookup(const hac_format* f, uint32_t window, float* value, uint32_t* length, int* kind,
+                           int* never_unresolved) {
+    return f ? table_lookup_host(f->f, window, value, length, kind, never_unresolved) : HAC_ERR_INVALID_ARG;
+}
+int shac_debug_table_lookup(const shac_format* f, uint32_t window, float* value, uint32_t* length, int* kind,
+                            int* never_unresolved) {
+    return f ? table_lookup_host(f->f, window, value, length, kind, never_unresolved) : HAC_ERR_INVALID_ARG;
+}
 
 int hac_build(const float* W, int64_t n, int64_t m, int64_t ldw, const hac_build_params* params,
               hac_format** out) {

@@ -27,6 +27,7 @@ inline uint32_t xt_index(uint32_t window, int mant) {
 }
 constexpr size_t kSubTableBytesMax = 24 * 1024;
 constexpr int kStreamSlackWords = 4;     // zero words after the stream (decoder reads ahead)
+constexpr size_t kTaskOffBytesMax = (size_t)64 << 20;
 constexpr int kItemWords = 48;           // sHAC work item record: 12 header words, 2 x 16 words of sub-segment bit lengths, 4 spare
 
 // Decoding tables derived from the code lengths (canonical Huffman).  "rank" is the position of
@@ -92,6 +93,7 @@ struct DeviceImage {
     const void* ri = nullptr;
     const uint32_t* cb = nullptr;
     const void* unit_info = nullptr;
+    const uint64_t* task_off = nullptr;
 };
 
 struct Format {
@@ -120,6 +122,10 @@ struct Format {
     std::vector<uint16_t> sub_bits;
     std::vector<uint32_t> seg_first, seg_col;
     std::vector<uint32_t> item_info;          // sHAC, device only: kItemWords words per work item (see ShacItem)
+    // HAC, device only: start bit of every sub-segment of every column, [ceil(n/S) + 1][m] (the last row
+    // holds the columns' ends), for the batched kernel, whose lanes are columns.  Left empty, and then
+    // derived from the offset index on every call, when it would exceed kTaskOffBytesMax.
+    std::vector<uint64_t> task_off;
     uint32_t max_unit_chunks = 0;             // largest 16-byte span a segment's stream covers
     uint32_t max_sub_chunks = 0;              // same for a single sub-segment
     uint32_t max_units_per_col = 0;
@@ -139,7 +145,7 @@ void fill_size_report(const Format& f, hac_size_report* r);
 // device image layout: offsets of every section (256-byte aligned), total size
 struct ImageLayout {
     size_t stream, lut, l1, sub, l1_runs, xt, rank_value, limit, first_left, rank_base, seg_bit_off, sub_bits, seg_col,
-        seg_first, ri, cb, unit_info, total;
+        seg_first, ri, cb, unit_info, task_off, total;
 };
 ImageLayout image_layout(const Format& f);
 

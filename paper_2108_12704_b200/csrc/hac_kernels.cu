@@ -465,6 +465,15 @@ __device__ __forceinline__ float decode_value_any(BitReader& br, const Decoder& 
     return __uint_as_float(e.x);
 }
 
+// resolve_long_split for either kind of table.
+template <int kTab>
+__device__ __forceinline__ void resolve_split_any(uint32_t top, const Decoder& d, const DevFormat& f, uint32_t& lo,
+                                                  uint32_t& hi_len) {
+    if (kTab == 0) { resolve_long_split(top, d, f, lo, hi_len); return; }
+    const uint2 e = split_entry(decode_long(top, f.lut, f.lut_bits, f.rank_value, f.limit, f.first_left, f.rank_base, f.max_len));
+    lo = e.x; hi_len = e.y;
+}
+
 // One step of kChains chains: lookups first, then the consumes, so that the table loads overlap.
 template <bool kLong, int kChains, int kXOffset>
 __device__ __forceinline__ void fast_step(FastReader (&r)[kChains], const Decoder& d, const DevFormat& f,
@@ -1904,6 +1913,7 @@ __global__ void __launch_bounds__(256) hac_pack_x_kernel(DevFormat f, const floa
 // (tcgen05.commit once the MMAs that read the stage have finished).  The X tile of chunk k + 1 shares
 // its buffer with chunk k - 1 and is requested once that chunk's MMAs have been committed.
 // Every wait is bounded; if one runs out the block marks its outputs NaN and still terminates.
+template <int kTab, bool kLong>
 __global__ void __launch_bounds__(kGWarps * 32, 1) hac_gemm_tc_kernel(
     DevFormat f, TablePlan tp, const unsigned char* __restrict__ xpack, uint32_t batch, float* __restrict__ y,
     int64_t ys_j, int64_t ys_b, float* __restrict__ partial, const uint64_t* __restrict__ task_off,
@@ -2026,7 +2036,7 @@ __global__ void __launch_bounds__(kGWarps * 32, 1) hac_gemm_tc_kernel(
         const uint32_t buf_stride = 32 * slot_bytes;
         // this lane's buffers: [parity][chain], buf_stride apart
         const uint32_t my_buf = spans + warp * nbuf * kGChains * buf_stride + lane * slot_bytes;
-        const uint32_t l1_abs = sb + dec.l1_lane;
+        const uint32_t l1_abs = sb + dec.l1_lane - dec.bias * dec.l1_mul;
         const uint32_t a_base = tmem + ((q * 32u) << 16) + kGDCols + slot * kGStages * kGACols;
         const uint32_t full0 = bar_full + 8 * slot * kGStages, empty0 = bar_empty + 8 * slot * kGStages;
         // the copies of one round (the located sub-segment of every chain), as one cp.async group
@@ -2079,10 +2089,13 @@ __global__ void __launch_bounds__(kGWarps * 32, 1) hac_gemm_tc_kernel(
                     for (int s = 0; s < kGChainRows; ++s) {
                         uint32_t top[kGChains], wl[kGChains], wh[kGChains];
 #pragma unroll
-                        for (int c = 0; c < kGChains; ++c) fast_lookup(fr[c], dec.l1_shift, dec.l1_mul, l1_abs, top[c], wl[c], wh[c]);
-#pragma unroll
                         for (int c = 0; c < kGChains; ++c)
-                            if (wh[c] & kSplitLong) resolve_long_split(top[c], dec, f, wl[c], wh[c]);
+                            table_lookup<kTab>(fr[c], dec.l1_shift, dec.l1_mul, l1_abs, dec.xt_low, top[c], wl[c], wh[c]);
+                        if (kLong) {
+#pragma unroll
+                            for (int c = 0; c < kGChains; ++c)
+                                if (wh[c] & kSplitLong) resolve_split_any<kTab>(top[c], dec, f, wl[c], wh[c]);
+                        }
 #pragma unroll
                         for (int c = 0; c < kGChains; ++c) {
                             fast_consume_value(fr[c], wh[c] & 63u);
@@ -2097,8 +2110,8 @@ __global__ void __launch_bounds__(kGWarps * 32, 1) hac_gemm_tc_kernel(
                         for (int c = 0; c < kGChains; ++c) {
                             uint32_t top = 0, wl = 0, wh = 0;
                             if (valid && r + s < cnt[c]) {
-                                fast_lookup(fr[c], dec.l1_shift, dec.l1_mul, l1_abs, top, wl, wh);
-                                if (wh & kSplitLong) resolve_long_split(top, dec, f, wl, wh);
+                                table_lookup<kTab>(fr[c], dec.l1_shift, dec.l1_mul, l1_abs, dec.xt_low, top, wl, wh);
+                                if (kLong && (wh & kSplitLong)) resolve_split_any<kTab>(top, dec, f, wl, wh);
                                 fast_consume_value(fr[c], wh & 63u);
                             }
                             hi[c * kGChainRows + s] = wh & 0xffffe000u;
@@ -2409,6 +2422,7 @@ static void set_pointers(Format& f, void* dev_buf, size_t bytes) {
     f.dev.ri = b + L.ri;
     f.dev.cb = reinterpret_cast<const uint32_t*>(b + L.cb);
     f.dev.unit_info = b + L.unit_info;
+    f.dev.task_off = reinterpret_cast<const uint64_t*>(b + L.task_off);
 }
 
 static int upload(Format& f, void* dev_buf, size_t dev_bytes, void* stream_) {
@@ -2440,6 +2454,7 @@ static int upload(Format& f, void* dev_buf, size_t dev_bytes, void* stream_) {
     else HAC_CUDA(put(L.ri, f.ri32.data(), f.ri32.size() * 4));
     HAC_CUDA(put(L.cb, f.cb.data(), f.cb.size() * 4));
     HAC_CUDA(put(L.unit_info, f.item_info.data(), f.item_info.size() * 4));
+    HAC_CUDA(put(L.task_off, f.task_off.data(), f.task_off.size() * 8));
     // the source vectors are pageable host memory: wait so they may change or go away afterwards
     HAC_CUDA(cudaStreamSynchronize(st));
     set_pointers(f, dev_buf, dev_bytes);
@@ -2512,7 +2527,7 @@ static size_t xpack_bytes(const Format& f, int64_t batch) {
 
 // Batched HAC: start bit of every task of every column, [tasks + 1][m] (see hac_pack_x_kernel).
 static size_t task_off_bytes(const Format& f, int64_t batch) {
-    if (f.sparse || batch <= 1 || f.symbols == 0) return 0;
+    if (f.sparse || batch <= 1 || f.symbols == 0 || !f.task_off.empty()) return 0;    // kept in the device image
     return ((size_t)gemm_tasks(f) + 1) * (size_t)f.m * 8;
 }
 
@@ -2851,9 +2866,13 @@ static int launch_vec(const Format& f, int mode, const float* x, int64_t xs_i, f
 }
 
 // Batched HAC product: one block per (128 columns, row split, 64 inputs).
-static int launch_gemm_tc(const Format& f, const DeviceInfo& di, const DevFormat& d, const float* x, int64_t xs_i,
+static int launch_gemm_tc(const Format& f, const DeviceInfo& di, const DevFormat&, const float* x, int64_t xs_i,
                           int64_t xs_b, int64_t batch, float* y, int64_t ys_j, int64_t ys_b, float* partial,
                           unsigned char* xpack, cudaStream_t st, uint32_t* row_splits_out) {
+    const DevFormat d = dev_format_xt(f);
+    const bool has_long = table_has_long(f, d);
+    auto kernel = d.tab_kind ? (has_long ? hac_gemm_tc_kernel<1, true> : hac_gemm_tc_kernel<1, false>)
+                             : (has_long ? hac_gemm_tc_kernel<0, true> : hac_gemm_tc_kernel<0, false>);
     const size_t budget = (size_t)di.max_smem_optin;
     const uint32_t slot_bytes = d.max_sub_chunks * 16;
     // shared memory: double stream buffers if they still leave room for a level-1 table with 8 replicas,
@@ -2873,7 +2892,7 @@ static int launch_gemm_tc(const Format& f, const DeviceInfo& di, const DevFormat
     const TablePlan tp = plan_tables(d, budget - fixed);
     // the block allocates all of tensor memory: ask for enough shared memory that no second block shares the SM
     const size_t smem = std::max(fixed + plan_smem_bytes(d.l1_entries, tp.repl_log2, d.sub_bytes), budget / 2 + 1024);
-    int rc = prepare_kernel(hac_gemm_tc_kernel, smem);
+    int rc = prepare_kernel(kernel, smem);
     if (rc) return rc;
     const uint32_t col_blocks = (uint32_t)((f.m + kGCols - 1) / kGCols);
     const uint32_t batch_tiles = (uint32_t)((batch + kGBatch - 1) / kGBatch);
@@ -2885,14 +2904,16 @@ static int launch_gemm_tc(const Format& f, const DeviceInfo& di, const DevFormat
     const uint64_t pack_blocks = (uint64_t)batch_tiles * rs * kGSlots * max_rounds * cpr;
     if (pack_blocks > 0x7fffffffull) return HAC_ERR_OFFSET_OVERFLOW;
     // the B tiles are a multiple of 8 bytes, so the start bits that follow them are aligned
-    uint64_t* task_off = reinterpret_cast<uint64_t*>(xpack + xpack_bytes(f, batch));
-    const uint64_t off_blocks = ((uint64_t)d.G * d.m + 255) / 256;
+    const bool cached_off = !f.task_off.empty();
+    uint64_t* task_off = cached_off ? const_cast<uint64_t*>(f.dev.task_off)
+                                    : reinterpret_cast<uint64_t*>(xpack + xpack_bytes(f, batch));
+    const uint64_t off_blocks = cached_off ? 0 : ((uint64_t)d.G * d.m + 255) / 256;
     if (pack_blocks + off_blocks > 0x7fffffffull) return HAC_ERR_OFFSET_OVERFLOW;
     rc = launch_dependent(hac_pack_x_kernel, dim3((unsigned)(pack_blocks + off_blocks)), dim3(256), 0, st, d, x, xs_i, xs_b,
                           (uint32_t)batch, xpack, tasks, rs, max_rounds, cpr, (uint32_t)pack_blocks, task_off);
     if (rc) return rc;
     f.last_launches++;
-    rc = launch_dependent(hac_gemm_tc_kernel, dim3((unsigned)grid), dim3(kGWarps * 32), smem, st, d, tp,
+    rc = launch_dependent(kernel, dim3((unsigned)grid), dim3(kGWarps * 32), smem, st, d, tp,
                           (const unsigned char*)xpack, (uint32_t)batch, y, ys_j, ys_b, partial, (const uint64_t*)task_off,
                           col_blocks, rs, max_rounds, slot_bytes, nbuf);
     if (rc) return rc;
@@ -3016,12 +3037,12 @@ static int dot(const Format& f, const float* x, int64_t batch, int64_t xs_i, int
 static size_t host_scratch_bytes(const Format& f, int64_t batch) {
     const size_t xb = align16((size_t)batch * f.n * 4 + 240) ;
     const size_t yb = align16((size_t)batch * f.m * 4 + 240);
-    const size_t extra = batch > 1 ? xb : 0;               // transposed copy of X
+    const size_t extra = (batch > 1 && f.sparse) ? xb : 0;  // sHAC: transposed copy of X (its batched kernel gathers rows of X)
     return xb + extra + yb + align16(workspace_bytes(f, batch)) + 1024;
 }
 
 static int dot_host(const Format& f, const float* X, int64_t batch, float* Y, void* scratch, size_t scratch_bytes,
-                    void* stream_) {
+                    void* stream_, bool wait) {
     if (!f.dev.base) return HAC_ERR_NOT_UPLOADED;
     if (!X || !Y || !scratch || batch < 1) return HAC_ERR_INVALID_ARG;
     if (scratch_bytes < host_scratch_bytes(f, batch)) return HAC_ERR_BUFFER_TOO_SMALL;
@@ -3032,26 +3053,28 @@ static int dot_host(const Format& f, const float* X, int64_t batch, float* Y, vo
     float* xd = reinterpret_cast<float*>(b);
     b += up((size_t)batch * f.n * 4);
     float* xt = xd;
-    if (batch > 1) { xt = reinterpret_cast<float*>(b); b += up((size_t)batch * f.n * 4); }
+    const bool transpose = batch > 1 && f.sparse;
+    if (transpose) { xt = reinterpret_cast<float*>(b); b += up((size_t)batch * f.n * 4); }
     float* yd = reinterpret_cast<float*>(b);
     b += up((size_t)batch * f.m * 4);
     void* ws = b;
     HAC_CUDA(cudaMemcpyAsync(xd, X, (size_t)batch * f.n * 4, cudaMemcpyHostToDevice, st));
     int extra = 0;
     int rc;
-    if (batch > 1) {
+    if (transpose) {
         dim3 grid((unsigned)((f.n + 31) / 32), (unsigned)((batch + 31) / 32));
         transpose_kernel<<<grid, dim3(32, 8), 0, st>>>(xd, xt, (uint32_t)batch, (uint32_t)f.n);
         HAC_CUDA(cudaGetLastError());
         extra = 1;
         rc = dot(f, xt, batch, batch, 1, yd, 1, f.m, ws, workspace_bytes(f, batch), stream_);
     } else {
-        rc = dot(f, xd, 1, 1, f.n, yd, 1, f.m, ws, workspace_bytes(f, batch), stream_);
+        // X is used as it lies, one input per row: the kernels take element strides
+        rc = dot(f, xd, batch, 1, f.n, yd, 1, f.m, ws, workspace_bytes(f, batch), stream_);
     }
     if (rc) return rc;
     f.last_launches += extra;
     HAC_CUDA(cudaMemcpyAsync(Y, yd, (size_t)batch * f.m * 4, cudaMemcpyDeviceToHost, st));
-    HAC_CUDA(cudaStreamSynchronize(st));
+    if (wait) HAC_CUDA(cudaStreamSynchronize(st));
     return HAC_OK;
 }
 
@@ -3173,12 +3196,22 @@ int shac_dot_host_scratch_bytes(const shac_format* f, int64_t batch, size_t* out
 int hac_dot_host(const hac_format* f, const float* X_host, int64_t batch, float* Y_host, void* dev_scratch,
                  size_t dev_scratch_bytes, void* cuda_stream) {
     if (!f) return HAC_ERR_INVALID_ARG;
-    return dot_host(f->f, X_host, batch, Y_host, dev_scratch, dev_scratch_bytes, cuda_stream);
+    return dot_host(f->f, X_host, batch, Y_host, dev_scratch, dev_scratch_bytes, cuda_stream, true);
 }
 int shac_dot_host(const shac_format* f, const float* X_host, int64_t batch, float* Y_host, void* dev_scratch,
                   size_t dev_scratch_bytes, void* cuda_stream) {
     if (!f) return HAC_ERR_INVALID_ARG;
-    return dot_host(f->f, X_host, batch, Y_host, dev_scratch, dev_scratch_bytes, cuda_stream);
+    return dot_host(f->f, X_host, batch, Y_host, dev_scratch, dev_scratch_bytes, cuda_stream, true);
+}
+int hac_dot_host_async(const hac_format* f, const float* X_host, int64_t batch, float* Y_host, void* dev_scratch,
+                       size_t dev_scratch_bytes, void* cuda_stream) {
+    if (!f) return HAC_ERR_INVALID_ARG;
+    return dot_host(f->f, X_host, batch, Y_host, dev_scratch, dev_scratch_bytes, cuda_stream, false);
+}
+int shac_dot_host_async(const shac_format* f, const float* X_host, int64_t batch, float* Y_host, void* dev_scratch,
+                        size_t dev_scratch_bytes, void* cuda_stream) {
+    if (!f) return HAC_ERR_INVALID_ARG;
+    return dot_host(f->f, X_host, batch, Y_host, dev_scratch, dev_scratch_bytes, cuda_stream, false);
 }
 
 int hac_debug_decode(const hac_format* f, float* W_colmajor_dev, void* cuda_stream) {

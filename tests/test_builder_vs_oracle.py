@@ -166,3 +166,45 @@ def test_library_kmeans_on_the_hand_worked_example():
         for kind in ("hac", "shac"):
             f = hb.Format(kind, W, sparsity=0.0, k=k, quantizer=si.QUANT_KMEANS, kmeans_iters=iters, seed=seed)
             assert f.export()["codebook"].tolist() == [float(v) for v in want]
+
+
+def _geometric_matrix(rng, k, ratio, n=600, m=40):
+    p = ratio ** np.arange(k)
+    p /= p.sum()
+    values = np.sort(rng.standard_normal(k).astype(np.float32))
+    W = values[rng.choice(k, size=(n, m), p=p)].astype(np.float32)
+    W.ravel()[:k] = values                                   # every value occurs
+    return W
+
+
+@pytest.mark.parametrize("k,ratio", [(22, 0.5), (60, 0.8), (200, 0.95), (247, 0.985), (8, 0.3), (33, 1.0)])
+def test_first_level_table_of_the_kernels_decodes_every_window(k, ratio):
+    """The table the kernels look code words up in (indexed by leading bits, or by the magnitude of the
+    inverted window when code words are long) must give, for every code word followed by any bits,
+    that code word's value and length, or say that it leaves it to the slower levels; where the kernels
+    rely on it resolving everything, it must."""
+    rng = np.random.default_rng(k)
+    W = _geometric_matrix(rng, k, ratio)
+    for kind in ("hac", "shac"):
+        f = hb.Format(kind, W, sparsity=0.0, k=k, quantizer=si.QUANT_NONE)
+        e = f.export()
+        kinds = set()
+        for s in range(e["k_eff"]):
+            L = int(e["code_len"][s]); code = int(e["codes"][s])
+            tails = [0, (1 << (32 - L)) - 1] + [int(t) for t in rng.integers(0, 1 << (32 - L), size=40)] if L < 32 else [0]
+            for t in tails:
+                window = (code << (32 - L)) | t
+                value, length, tk, never = f.debug_table_lookup(window)
+                kinds.add(tk)
+                if length == 0:
+                    assert not never, "an unresolved window in a table the kernels treat as complete"
+                else:
+                    assert length == L and np.float32(value) == e["codebook"][s]
+        assert len(kinds) == 1
+
+
+def test_long_tailed_code_takes_the_magnitude_table():
+    rng = np.random.default_rng(3)
+    f = hb.Format("hac", _geometric_matrix(rng, 40, 0.6, n=3000), sparsity=0.0, k=40, quantizer=si.QUANT_NONE)
+    assert f.sizes()["max_code_len"] > 12
+    assert f.debug_table_lookup(0)[2] == 1

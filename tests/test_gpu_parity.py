@@ -170,46 +170,84 @@ def test_wide_row_index_and_large_n():
     check_outputs(run_dot(lf, X), y_ref, a)
 
 
-def _full_size(wl, kind, batches, ncols=48, S=0):
-    lf, Wq, mask = build_both(wl, kind, S)
+def _structured_sample(rng, m, B, ncols):
+    """Columns: `ncols` random ones plus one from every block of 128 columns (the unit a block of the batched
+    kernels owns; every column carries all row splits).  Inputs: all when there are at most 8, else 8 random
+    ones plus one from every tile of 64 inputs."""
+    cols = set(rng.choice(m, size=min(ncols, m), replace=False).tolist())
+    for c0 in range(0, m, 128):
+        cols.add(int(c0 + rng.integers(0, min(128, m - c0))))
+    if B <= 8:
+        rows = set(range(B))
+    else:
+        rows = set(rng.choice(B, size=8, replace=False).tolist())
+        for b0 in range(0, B, 64):
+            rows.add(int(b0 + rng.integers(0, min(64, B - b0))))
+    return np.array(sorted(cols)), np.array(sorted(rows))
+
+
+def _full_size(wl, kind, batches, ncols=48, S=0, quantized=None, all_outputs_up_to=1):
+    """Full-size parity.  One input: every output, against Algorithm 1 / 2 run literally.  A batch: every
+    output against the written-out definition when the batch is at most `all_outputs_up_to`, else a
+    structured sample.  `quantized` = (W, Wq, mask) lets several formats share one run of the oracle's
+    quantizer."""
+    if quantized is None:
+        lf, Wq, mask = build_both(wl, kind, S)
+    else:
+        W, Wq, mask = quantized
+        lf = hb.Format(kind, W, sparsity=wl.sparsity, k=wl.k, quantizer=wl.quantizer, kmeans_iters=wl.kmeans_iters,
+                       seed=wl.seed, seg_symbols=S).upload()
     check_decode(lf, Wq, mask)
     rng = np.random.default_rng(wl.seed)
-    cols = np.sort(rng.choice(wl.m, size=min(ncols, wl.m), replace=False))
     worst = 0.0
     for B in batches:
         X = si.inputs(wl, B)
         y = run_dot(lf, X)
-        rows = np.arange(B) if B <= 8 else np.sort(rng.choice(B, size=8, replace=False))
-        y_ref, a = orc.dot_definition(Wq, X[rows], cols=cols)
-        worst = max(worst, check_outputs(y[np.ix_(rows, cols)], y_ref, a))
         if B == 1:                                          # all outputs, via Algorithm 1 / 2
             ofmt = orc.hac_encode(Wq) if kind == "hac" else orc.shac_encode(Wq, mask)
             y_alg = (orc.dot_hac if kind == "hac" else orc.dot_shac)(ofmt, X[0])
+            cols = np.sort(rng.choice(wl.m, size=min(ncols, wl.m), replace=False))
+            y_ref, a = orc.dot_definition(Wq, X, cols=cols)
             assert np.array_equal(y_alg[cols], y_ref[0])
             a_all = np.abs(Wq.astype(np.float64)).T @ np.abs(X[0].astype(np.float64))
-            check_outputs(y[0], y_alg, a_all * (1 + 1e-9))
+            worst = max(worst, check_outputs(y[0], y_alg, a_all * (1 + 1e-9)))
+        elif B <= all_outputs_up_to:
+            y_ref, a = orc.dot_definition(Wq, X)
+            worst = max(worst, check_outputs(y, y_ref, a))
+        else:
+            cols, rows = _structured_sample(rng, wl.m, B, ncols)
+            y_ref, a = orc.dot_definition(Wq, X[rows], cols=cols)
+            worst = max(worst, check_outputs(y[np.ix_(rows, cols)], y_ref, a))
     return worst
 
 
 def test_config2_dense_hac_full_size():
-    _full_size(si.CFG2_DENSE_HAC, "hac", (1, 64))
+    _full_size(si.CFG2_DENSE_HAC, "hac", (1, 64), all_outputs_up_to=64)     # all 4096 x 64 outputs of the batch
 
 
 def test_config3_fc_shac_full_size():
-    _full_size(si.CFG3_FC_SHAC, "shac", (1, 16, 128))
+    _full_size(si.CFG3_FC_SHAC, "shac", (1, 16, 128), all_outputs_up_to=16)
 
 
 def test_config4_conv_full_size():
     wl = dataclasses.replace(si.CFG4_CONV, batches=(6272,))
-    _full_size(wl, "shac", (1, 6272))
-    _full_size(wl, "hac", (1, 6272))
+    W = si.weights(wl)
+    Wq, mask = orc.quantize(W, wl.sparsity, wl.k, wl.quantizer, wl.kmeans_iters, wl.seed)
+    _full_size(wl, "shac", (1, 6272), quantized=(W, Wq, mask))
+    _full_size(wl, "hac", (1, 6272), quantized=(W, Wq, mask))
 
 
-@pytest.mark.parametrize("sp,k", [(0.0, 2), (0.0, 1024), (0.5, 32), (0.9, 8), (0.99, 256), (0.95, 1024)])
+SWEEP = [(c.sparsity, c.k) for c in si.sweep_cells()]
+
+
+@pytest.mark.parametrize("sp,k", SWEEP, ids=[f"p{int(round(100 * sp))}-k{k}" for sp, k in SWEEP])
 def test_config5_sweep_cells_full_size(sp, k):
-    wl = dataclasses.replace(si.sweep_cells()[0], sparsity=sp, k=k)
+    """Every cell of the sparsity x k sweep, both formats on one run of the oracle's quantizer."""
+    cell = [c for c in si.sweep_cells() if c.sparsity == sp and c.k == k][0]
+    W = si.weights(cell)
+    Wq, mask = orc.quantize(W, cell.sparsity, cell.k, cell.quantizer, cell.kmeans_iters, cell.seed)
     for kind in ("hac", "shac"):
-        _full_size(wl, kind, (1, 32), ncols=32)
+        _full_size(cell, kind, (1, 32), ncols=32, quantized=(W, Wq, mask))
 
 
 def test_chained_products_keep_stream_order():
