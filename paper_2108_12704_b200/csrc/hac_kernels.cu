@@ -474,6 +474,44 @@ __device__ __forceinline__ void resolve_split_any(uint32_t top, const Decoder& d
     lo = e.x; hi_len = e.y;
 }
 
+// N (2 or 3) code words from one window, for tables in the split form {lo, hi | length} (see split_entry):
+// as lookup3, with the length taken from the low bits of the second word (the funnel shift only looks at
+// its low five bits).  tot = sum of the lengths, flags = kSplitLong if an entry does not hold its symbol.
+template <int kTab, int N>
+__device__ __forceinline__ void lookup_group_split(const FastReader& r, uint32_t l1_shift, uint32_t l1_mul, uint32_t l1_lane,
+                                                   uint32_t xt_low, uint32_t (&wl)[N], uint32_t (&wh)[N], uint32_t& tot,
+                                                   uint32_t& flags) {
+    uint32_t t;
+    const uint32_t zero = 0;
+    asm volatile("shf.l.wrap.b32 %0, %1, %2, %3;" : "=r"(t) : "r"(r.lo), "r"(r.hi), "r"(r.off));
+#pragma unroll
+    for (int i = 0; i < N; ++i) {
+        if (kTab == 0) {
+            asm volatile(
+                "{\n\t.reg .b32 i;\n\t"
+                "shr.u32 i, %2, %3;\n\t"
+                "mad.lo.u32 i, i, %4, %5;\n\t"
+                "ld.shared.v2.u32 {%0, %1}, [i];\n\t}"
+                : "=r"(wl[i]), "=r"(wh[i]) : "r"(t), "r"(l1_shift), "r"(l1_mul), "r"(l1_lane) : "memory");
+        } else {
+            asm volatile(
+                "{\n\t.reg .b32 i;\n\t"
+                "lop3.b32 i, %2, %6, 0, 0xCF;\n\t"
+                "cvt.rz.f32.u32 i, i;\n\t"
+                "shr.u32 i, i, %3;\n\t"
+                "mad.lo.u32 i, i, %4, %5;\n\t"
+                "ld.shared.v2.u32 {%0, %1}, [i];\n\t}"
+                : "=r"(wl[i]), "=r"(wh[i]) : "r"(t), "r"(l1_shift), "r"(l1_mul), "r"(l1_lane), "r"(xt_low) : "memory");
+        }
+        if (i + 1 < N) asm volatile("shf.l.wrap.b32 %0, %1, %0, %2;" : "+r"(t) : "r"(zero), "r"(wh[i]));
+    }
+    uint32_t sum = wh[0], any = wh[0];
+#pragma unroll
+    for (int i = 1; i < N; ++i) { sum += wh[i]; any |= wh[i]; }
+    tot = sum & 0xffu;
+    flags = any & kSplitLong;
+}
+
 // One step of kChains chains: lookups first, then the consumes, so that the table loads overlap.
 template <bool kLong, int kChains, int kXOffset>
 __device__ __forceinline__ void fast_step(FastReader (&r)[kChains], const Decoder& d, const DevFormat& f,
@@ -1917,12 +1955,14 @@ template <int kTab, bool kLong>
 __global__ void __launch_bounds__(kGWarps * 32, 1) hac_gemm_tc_kernel(
     DevFormat f, TablePlan tp, const unsigned char* __restrict__ xpack, uint32_t batch, float* __restrict__ y,
     int64_t ys_j, int64_t ys_b, float* __restrict__ partial, const uint64_t* __restrict__ task_off,
-    uint32_t col_blocks, uint32_t row_splits, uint32_t max_rounds, uint32_t slot_bytes, uint32_t nbuf) {
+    uint32_t col_blocks, uint32_t row_splits, uint32_t max_rounds, uint32_t slot_bytes, uint32_t nbuf,
+    uint32_t cluster_reduce) {
     allow_dependents();
     const uint32_t warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const uint32_t cblk = blockIdx.x % col_blocks;
-    const uint32_t rest = blockIdx.x / col_blocks;
-    const uint32_t rs = rest % row_splits, bt = rest / row_splits;
+    // the row splits of a column block are consecutive blocks (one thread-block cluster when cluster_reduce is set)
+    const uint32_t rs = blockIdx.x % row_splits;
+    const uint32_t rest = blockIdx.x / row_splits;
+    const uint32_t cblk = rest % col_blocks, bt = rest / col_blocks;
     const uint32_t tasks = (uint32_t)(((uint64_t)f.n + f.S - 1) / f.S);          // sub-segments of a column
     const uint32_t t_begin = gemm_split_begin(tasks, rs, row_splits);
     const uint32_t ntl = gemm_split_begin(tasks, rs + 1, row_splits) - t_begin;
@@ -2051,6 +2091,7 @@ __global__ void __launch_bounds__(kGWarps * 32, 1) hac_gemm_tc_kernel(
             asm volatile("cp.async.commit_group;" ::: "memory");
         };
         uint32_t par = 0, k = 0;
+        const bool guard = 3u * f.max_len > 32u;       // three code words may not fit one window
         if (rounds > 0) copy_round(loc_cur, 0);
         for (uint32_t pr = 0; pr < rounds; ++pr) {
             const bool more = pr + 1 < rounds;
@@ -2085,24 +2126,45 @@ __global__ void __launch_bounds__(kGWarps * 32, 1) hac_gemm_tc_kernel(
                 uint32_t hi[kGRows], lo[kGRows];
                 // the table entries are {lo, hi | length}: the symbol is ready for the tensor core as it is
                 if (all_valid && r + kGChainRows <= full_rows) {
-#pragma unroll
-                    for (int s = 0; s < kGChainRows; ++s) {
-                        uint32_t top[kGChains], wl[kGChains], wh[kGChains];
+                    // code words in groups of three (and a last group of two) per window
+                    auto one_by_one = [&](int c, int s0, int cntg) {
+                        for (int s = s0; s < s0 + cntg; ++s) {
+                            uint32_t top, wl1, wh1;
+                            table_lookup<kTab>(fr[c], dec.l1_shift, dec.l1_mul, l1_abs, dec.xt_low, top, wl1, wh1);
+                            if (kLong && (wh1 & kSplitLong)) resolve_split_any<kTab>(top, dec, f, wl1, wh1);
+                            fast_consume_value(fr[c], wh1 & 63u);
+                            hi[c * kGChainRows + s] = wh1 & 0xffffe000u;
+                            lo[c * kGChainRows + s] = wl1;
+                        }
+                    };
+                    auto group = [&](auto count, int s0) {
+                        constexpr int N = decltype(count)::value;
+                        uint32_t wl[kGChains][N], wh[kGChains][N], tot[kGChains], flags[kGChains];
 #pragma unroll
                         for (int c = 0; c < kGChains; ++c)
-                            table_lookup<kTab>(fr[c], dec.l1_shift, dec.l1_mul, l1_abs, dec.xt_low, top[c], wl[c], wh[c]);
-                        if (kLong) {
+                            lookup_group_split<kTab, N>(fr[c], dec.l1_shift, dec.l1_mul, l1_abs, dec.xt_low, wl[c], wh[c], tot[c], flags[c]);
+                        bool bad = false;
 #pragma unroll
-                            for (int c = 0; c < kGChains; ++c)
-                                if (wh[c] & kSplitLong) resolve_split_any<kTab>(top[c], dec, f, wl[c], wh[c]);
-                        }
+                        for (int c = 0; c < kGChains; ++c) bad = bad || (guard && tot[c] > 32u) || (kLong && flags[c] != 0u);
+                        if (bad) {
 #pragma unroll
-                        for (int c = 0; c < kGChains; ++c) {
-                            fast_consume_value(fr[c], wh[c] & 63u);
-                            hi[c * kGChainRows + s] = wh[c] & 0xffffe000u;
-                            lo[c * kGChainRows + s] = wl[c];
+                            for (int c = 0; c < kGChains; ++c) one_by_one(c, s0, N);
+                        } else {
+#pragma unroll
+                            for (int c = 0; c < kGChains; ++c) {
+                                fast_consume_value(fr[c], tot[c]);
+#pragma unroll
+                                for (int e = 0; e < N; ++e) {
+                                    hi[c * kGChainRows + s0 + e] = wh[c][e] & 0xffffe000u;
+                                    lo[c * kGChainRows + s0 + e] = wl[c][e];
+                                }
+                            }
                         }
-                    }
+                    };
+                    static_assert(kGChainRows == 8, "groups of 3 + 3 + 2 code words");
+                    group(std::integral_constant<int, 3>(), 0);
+                    group(std::integral_constant<int, 3>(), 3);
+                    group(std::integral_constant<int, 2>(), 6);
                 } else {
 #pragma unroll
                     for (int s = 0; s < kGChainRows; ++s) {
@@ -2169,7 +2231,17 @@ __global__ void __launch_bounds__(kGWarps * 32, 1) hac_gemm_tc_kernel(
             // when y_stride_j is 1; otherwise the 32 x 32 block goes through shared memory (the stream
             // buffers are free by now) and is stored with the lanes along the inputs.
             const uint32_t b0 = bt * kGBatch + half * 32;
-            if (row_splits > 1) {
+            if (row_splits > 1 && cluster_reduce) {
+                // this block's 128 x 64 tile of sums goes to its shared memory, in the orientation of y
+                float* tile = reinterpret_cast<float*>(smem + spans);
+                if (ys_b == 1 && ys_j != 1) {
+#pragma unroll
+                    for (int cc = 0; cc < 32; ++cc) tile[(warp * 32 + lane) * (kGBatch + 1) + half * 32 + cc] = acc[cc];
+                } else {
+#pragma unroll
+                    for (int cc = 0; cc < 32; ++cc) tile[(half * 32 + cc) * kGCols + warp * 32 + lane] = acc[cc];
+                }
+            } else if (row_splits > 1) {
                 if (j < f.m) {
 #pragma unroll
                     for (int cc = 0; cc < 32; ++cc)
@@ -2195,6 +2267,40 @@ __global__ void __launch_bounds__(kGWarps * 32, 1) hac_gemm_tc_kernel(
                 }
             }
         }
+    }
+    if (row_splits > 1 && cluster_reduce) {
+        // The blocks of the cluster hold the row splits of the same 128 columns: each adds, in split order, its
+        // share of the outputs from everybody's tile (distributed shared memory) and writes it to y.
+        asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
+        const uint32_t tile_a = sb + spans;
+        auto remote = [&](uint32_t byte_off, uint32_t rank) {
+            uint32_t a;
+            float v;
+            asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(a) : "r"(tile_a + byte_off), "r"(rank));
+            asm volatile("ld.shared::cluster.f32 %0, [%1];" : "=f"(v) : "r"(a) : "memory");
+            return v;
+        };
+        if (ys_b == 1 && ys_j != 1) {               // y is [column][input]: a share of the columns, inputs fastest
+            const uint32_t j0 = kGCols * rs / row_splits, j1 = kGCols * (rs + 1) / row_splits;
+            for (uint32_t idx = threadIdx.x; idx < (j1 - j0) * kGBatch; idx += blockDim.x) {
+                const uint32_t jl = j0 + idx / kGBatch, b = idx % kGBatch;
+                float sum = 0.0f;
+                for (uint32_t r = 0; r < row_splits; ++r) sum += remote((jl * (kGBatch + 1) + b) * 4u, r);
+                const uint32_t j = cblk * kGCols + jl, bb = bt * kGBatch + b;
+                if (j < f.m && bb < batch) y[(int64_t)j * ys_j + bb] = sum;
+            }
+        } else {                                     // a share of the inputs, columns fastest
+            const uint32_t b0 = kGBatch * rs / row_splits, b1 = kGBatch * (rs + 1) / row_splits;
+            for (uint32_t idx = threadIdx.x; idx < (b1 - b0) * kGCols; idx += blockDim.x) {
+                const uint32_t b = b0 + idx / kGCols, jl = idx % kGCols;
+                float sum = 0.0f;
+                for (uint32_t r = 0; r < row_splits; ++r) sum += remote((b * kGCols + jl) * 4u, r);
+                const uint32_t j = cblk * kGCols + jl, bb = bt * kGBatch + b;
+                if (j < f.m && bb < batch) y[(int64_t)j * ys_j + (int64_t)bb * ys_b] = sum;
+            }
+        }
+        // nobody leaves while its tile may still be read
+        asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
     }
     asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
     __syncthreads();
@@ -2351,10 +2457,11 @@ struct Tune {
     int prefetch;       // HAC_B200_PREFETCH=0: no L2 prefetch of the stream at the start of the rows-in-registers kernel
     int rows_chains;    // HAC_B200_ROWS_CHAINS=2|3: decode chains per lane of that kernel (0 = chosen by the library)
     int items_kernel;   // HAC_B200_ITEMS=0: single-input sHAC always through the older kernel
+    int gemm_cluster;   // HAC_B200_GEMM_CLUSTER=0: batched HAC adds its row splits in a finishing kernel, not in a cluster
 };
 static const Tune& tune() {
     static const Tune t = {env_int("HAC_B200_PDL", 1), env_int("HAC_B200_ROWS", 1), env_int("HAC_B200_ROWS_WARPS", 0),
-                           env_int("HAC_B200_ZERO_RUNS", 1), env_int("HAC_B200_XT", 1), env_int("HAC_B200_PREFETCH", 1), env_int("HAC_B200_ROWS_CHAINS", 0), env_int("HAC_B200_ITEMS", 1)};
+                           env_int("HAC_B200_ZERO_RUNS", 1), env_int("HAC_B200_XT", 1), env_int("HAC_B200_PREFETCH", 1), env_int("HAC_B200_ROWS_CHAINS", 0), env_int("HAC_B200_ITEMS", 1), env_int("HAC_B200_GEMM_CLUSTER", 1)};
     return t;
 }
 
@@ -2587,6 +2694,21 @@ static int launch_dependent(void (*kernel)(KArgs...), dim3 grid, dim3 block, siz
     cfg.attrs = attr; cfg.numAttrs = 1;
     HAC_CUDA(cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...));
     return HAC_OK;
+}
+
+// The same with `cluster_x` consecutive blocks forming a thread-block cluster.
+template <typename... KArgs, typename... Args>
+static cudaError_t launch_dependent_cluster(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st,
+                                            unsigned cluster_x, Args... args) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid; cfg.blockDim = block; cfg.dynamicSmemBytes = smem; cfg.stream = st;
+    cudaLaunchAttribute attr[2];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = tune().pdl != 0 ? 1 : 0;
+    attr[1].id = cudaLaunchAttributeClusterDimension;
+    attr[1].val.clusterDim.x = cluster_x; attr[1].val.clusterDim.y = 1; attr[1].val.clusterDim.z = 1;
+    cfg.attrs = attr; cfg.numAttrs = 2;
+    return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
 }
 
 // Largest number of warps per block (a multiple of `step`, at most `want`) whose shared memory
@@ -2882,8 +3004,10 @@ static int launch_gemm_tc(const Format& f, const DeviceInfo& di, const DevFormat
     for (uint32_t want_repl : {3u, 2u, 1u, 0u}) {
         for (uint32_t nb : {2u, 1u}) {
             // the stream buffers double as the epilogue's four 32 x 33 transpose tiles
+            // the stream buffers double as the epilogue's tiles (four 32 x 33 transposes, or the 128 x 65 sums)
             const size_t fx = 256 + 128 + (size_t)kGSlots * kGStages * kGXTileBytes +
-                              std::max<size_t>((size_t)kGDecodeWarps * nb * kGChains * 32 * slot_bytes, 4 * 32 * 33 * 4);
+                              std::max<size_t>((size_t)kGDecodeWarps * nb * kGChains * 32 * slot_bytes,
+                                               (size_t)kGCols * (kGBatch + 1) * 4);
             if (fx + plan_smem_bytes(d.l1_entries, want_repl, d.sub_bytes) <= budget) { nbuf = nb; fixed = fx; break; }
         }
         if (nbuf) break;
@@ -2913,12 +3037,24 @@ static int launch_gemm_tc(const Format& f, const DeviceInfo& di, const DevFormat
                           (uint32_t)batch, xpack, tasks, rs, max_rounds, cpr, (uint32_t)pack_blocks, task_off);
     if (rc) return rc;
     f.last_launches++;
-    rc = launch_dependent(kernel, dim3((unsigned)grid), dim3(kGWarps * 32), smem, st, d, tp,
-                          (const unsigned char*)xpack, (uint32_t)batch, y, ys_j, ys_b, partial, (const uint64_t*)task_off,
-                          col_blocks, rs, max_rounds, slot_bytes, nbuf);
-    if (rc) return rc;
+    // The row splits of a column block form a thread-block cluster that adds its sums through distributed
+    // shared memory; if the device refuses the cluster, they go to the workspace and a finishing kernel adds them.
+    bool clustered = false;
+    if (rs > 1 && tune().gemm_cluster != 0) {
+        const cudaError_t ce = launch_dependent_cluster(kernel, dim3((unsigned)grid), dim3(kGWarps * 32), smem, st, rs, d, tp,
+                                                        (const unsigned char*)xpack, (uint32_t)batch, y, ys_j, ys_b, partial,
+                                                        (const uint64_t*)task_off, col_blocks, rs, max_rounds, slot_bytes, nbuf, 1u);
+        if (ce == cudaSuccess) clustered = true;
+        else (void)cudaGetLastError();
+    }
+    if (!clustered) {
+        rc = launch_dependent(kernel, dim3((unsigned)grid), dim3(kGWarps * 32), smem, st, d, tp,
+                              (const unsigned char*)xpack, (uint32_t)batch, y, ys_j, ys_b, partial, (const uint64_t*)task_off,
+                              col_blocks, rs, max_rounds, slot_bytes, nbuf, 0u);
+        if (rc) return rc;
+    }
     f.last_launches++;
-    *row_splits_out = rs;
+    *row_splits_out = clustered ? 1u : rs;       // 1: the outputs are written, nothing to finish
     return HAC_OK;
 }
 
