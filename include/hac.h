@@ -227,6 +227,41 @@ int shac_dot(const shac_format* f, const float* x, int64_t batch, int64_t x_stri
              float* y, int64_t y_stride_j, int64_t y_stride_b,
              void* workspace, size_t workspace_bytes, void* cuda_stream);
 
+/* ---------------------------------------------------------------------------------------------
+ * Layer evaluation on the compressed format (Sect. V: the networks are evaluated with their fully
+ * connected layers kept in HAC / sHAC): the product of hac_dot / shac_dot with the layer's bias and
+ * activation applied to every output before it is stored, in the same kernels,
+ *       y[b][j] = act( sum_i W[i][j] x[b][i] + bias[j] ),   act = identity or max(., 0).
+ *   epilogue   NULL = plain product.  bias: device, m floats, or NULL; relu: 0 / 1; reserved: 0.
+ * Everything else as hac_dot.
+ * hac_chain evaluates a stack of such layers as one chained submission on cuda_stream (layer l + 1 may
+ * begin fetching its format while layer l finishes, see hac_dot): layers[l] names a HAC or an sHAC handle
+ * (exactly one non-NULL) and its epilogue; layer l's m must equal layer l + 1's n.  x is [n_0][batch] and y
+ * [m_last][batch] with the inputs of a batch contiguous (plain vectors for batch 1); act0 / act1 are two
+ * device buffers of act_floats floats each that take the intermediate activations in turn (act0 may be
+ * NULL for one layer, act1 for at most two); the workspace must satisfy every layer's *_workspace_bytes.
+ * After the call *_last_launch_count of the LAST layer's handle gives the launches of the whole chain.
+ * ------------------------------------------------------------------------------------------- */
+typedef struct hac_epilogue {
+    const float* bias;     /* device, one per output (column of W), or NULL                       */
+    uint32_t relu;         /* 1: negative results become 0                                        */
+    uint32_t reserved;     /* must be 0                                                           */
+} hac_epilogue;
+typedef struct hac_layer {
+    const hac_format*  hac;    /* the layer's weights as HAC ...                                   */
+    const shac_format* shac;   /* ... or as sHAC (exactly one of the two)                          */
+    hac_epilogue epilogue;
+} hac_layer;
+int hac_dot_layer (const hac_format* f, const float* x, int64_t batch, int64_t x_stride_i, int64_t x_stride_b,
+                   float* y, int64_t y_stride_j, int64_t y_stride_b, const hac_epilogue* epilogue,
+                   void* workspace, size_t workspace_bytes, void* cuda_stream);
+int shac_dot_layer(const shac_format* f, const float* x, int64_t batch, int64_t x_stride_i, int64_t x_stride_b,
+                   float* y, int64_t y_stride_j, int64_t y_stride_b, const hac_epilogue* epilogue,
+                   void* workspace, size_t workspace_bytes, void* cuda_stream);
+int hac_chain(const hac_layer* layers, int n_layers, const float* x, int64_t batch, float* y,
+              float* act0, float* act1, size_t act_floats, void* workspace, size_t workspace_bytes,
+              void* cuda_stream);
+
 /* The same product for HOST inputs and outputs (Algorithm 3's calling convention: X is batch x n,
  * one input per row, Y is batch x m, both contiguous host fp32, ideally pinned).  The caller gives a
  * device staging buffer `dev_scratch` of at least *_dot_host_scratch_bytes(f, batch) bytes; the call

@@ -644,3 +644,34 @@ def dot_definition(Wq: np.ndarray, X: np.ndarray, cols=None):
         if rc:
             raise RuntimeError("bad column index")
     return y, a
+
+
+def layer_definition(Wq: np.ndarray, X: np.ndarray, bias=None, relu: bool = False, cols=None):
+    """A fully connected layer evaluated on the compressed matrix, written out (Sect. V evaluates the
+    networks with their fully connected layers kept in HAC / sHAC; the layer itself is the ordinary
+    one): out[b, j] = act(sum_i Wq[i, j] X[b, i] + bias[j]) in fp64, act = identity or max(., 0).
+    Returns (out, a) with a[b, j] = sum_i |Wq[i, j] X[b, i]| + |bias[j]|, the scale of the output
+    tolerance (the activation does not enlarge an error)."""
+    y, a = dot_definition(Wq, X, cols=cols)
+    if bias is not None:
+        b = np.asarray(bias, dtype=np.float64)
+        if cols is not None:
+            b = b[np.asarray(cols)]
+        y = y + b[None, :]
+        a = a + np.abs(b)[None, :]
+    if relu:
+        y = np.where(y < 0.0, 0.0, y)
+    return y, a
+
+
+def chain_definition(layers, X: np.ndarray):
+    """A stack of such layers: `layers` is a list of (Wq, bias or None, relu); the input of layer l + 1 is
+    the output of layer l rounded to fp32 (activations are stored as fp32).  Returns the list of every
+    layer's (out, a)."""
+    outs = []
+    cur = np.atleast_2d(X)
+    for Wq, bias, relu in layers:
+        y, a = layer_definition(Wq, cur, bias, relu)
+        outs.append((y, a))
+        cur = y.astype(np.float32)
+    return outs

@@ -38,6 +38,14 @@ class SizeReport(C.Structure):
         return {n: getattr(self, n) for n, _ in self._fields_}
 
 
+class Epilogue(C.Structure):
+    _fields_ = [("bias", C.c_void_p), ("relu", C.c_uint32), ("reserved", C.c_uint32)]
+
+
+class Layer(C.Structure):
+    _fields_ = [("hac", C.c_void_p), ("shac", C.c_void_p), ("epilogue", Epilogue)]
+
+
 class HostView(C.Structure):
     _fields_ = [("n", C.c_int64), ("m", C.c_int64), ("k_eff", C.c_uint32), ("seg_symbols", C.c_uint32),
                 ("codebook", C.POINTER(C.c_float)), ("code_len", C.POINTER(C.c_uint8)),
@@ -61,7 +69,7 @@ EXPORTS = (
     "hac_build", "shac_build", "hac_sizes", "shac_sizes", "hac_export", "shac_export",
     "hac_decode_host", "shac_decode_host", "hac_device_bytes", "shac_device_bytes", "hac_upload",
     "shac_upload", "hac_attach", "shac_attach", "hac_workspace_bytes", "shac_workspace_bytes", "hac_dot",
-    "shac_dot", "hac_dot_noalloc", "hac_dot_host_scratch_bytes", "shac_dot_host_scratch_bytes", "hac_dot_host",
+    "shac_dot", "hac_dot_noalloc", "hac_dot_layer", "shac_dot_layer", "hac_chain", "hac_dot_host_scratch_bytes", "shac_dot_host_scratch_bytes", "hac_dot_host",
     "shac_dot_host", "hac_dot_host_async", "shac_dot_host_async", "hac_debug_decode", "shac_debug_decode",
     "hac_debug_table_lookup", "shac_debug_table_lookup", "hac_last_launch_count",
     "shac_last_launch_count", "hac_free", "shac_free", "hac_status_string", "hac_last_cuda_error",
@@ -93,6 +101,7 @@ def load():
         getattr(lib, f"{kind}_attach").argtypes = [vp, vp, sz]
         getattr(lib, f"{kind}_workspace_bytes").argtypes = [vp, i64, C.POINTER(sz)]
         getattr(lib, f"{kind}_dot").argtypes = [vp, fp, i64, i64, i64, fp, i64, i64, vp, sz, vp]
+        getattr(lib, f"{kind}_dot_layer").argtypes = [vp, fp, i64, i64, i64, fp, i64, i64, C.POINTER(Epilogue), vp, sz, vp]
         getattr(lib, f"{kind}_dot_host_scratch_bytes").argtypes = [vp, i64, C.POINTER(sz)]
         getattr(lib, f"{kind}_dot_host").argtypes = [vp, fp, i64, fp, vp, sz, vp]
         getattr(lib, f"{kind}_dot_host_async").argtypes = [vp, fp, i64, fp, vp, sz, vp]
@@ -103,6 +112,7 @@ def load():
         getattr(lib, f"{kind}_free").argtypes = [vp]
         getattr(lib, f"{kind}_free").restype = None
     lib.hac_dot_noalloc.argtypes = [vp, fp, i64, i64, i64, fp, i64, i64, vp]
+    lib.hac_chain.argtypes = [C.POINTER(Layer), C.c_int, fp, i64, fp, fp, fp, sz, vp, sz, vp]
     lib.hac_status_string.argtypes = [C.c_int]
     lib.hac_status_string.restype = C.c_char_p
     lib.hac_last_cuda_error.restype = C.c_char_p
@@ -227,9 +237,11 @@ class Format:
         _check(self._fn("workspace_bytes")(self._h, int(batch), C.byref(s)), "workspace_bytes")
         return s.value
 
-    def dot(self, x, y=None, workspace=None, layout="nb"):
+    def dot(self, x, y=None, workspace=None, layout="nb", bias=None, relu=False):
         """y = W^T x on the device.  x: torch float32 CUDA tensor, [n] or, for a batch, [n, B]
-        (layout 'nb') or [B, n] (layout 'bn').  Returns y shaped [m], [m, B] or [B, m] alike."""
+        (layout 'nb') or [B, n] (layout 'bn').  Returns y shaped [m], [m, B] or [B, m] alike.
+        With `bias` (torch float32 CUDA tensor [m]) and / or relu=True the call goes through *_dot_layer:
+        y = act(W^T x + bias)."""
         import torch
         assert x.is_cuda and x.dtype == torch.float32
         if x.dim() == 1:
@@ -255,7 +267,12 @@ class Format:
         wp = workspace.data_ptr() if workspace is not None else None
         wb = workspace.numel() * workspace.element_size() if workspace is not None else 0
         st = torch.cuda.current_stream().cuda_stream
-        _check(self._fn("dot")(self._h, x.data_ptr(), B, xs_i, xs_b, y.data_ptr(), ys_j, ys_b, wp, wb, st), "dot")
+        if bias is None and not relu:
+            _check(self._fn("dot")(self._h, x.data_ptr(), B, xs_i, xs_b, y.data_ptr(), ys_j, ys_b, wp, wb, st), "dot")
+        else:
+            epi = Epilogue(bias.data_ptr() if bias is not None else None, 1 if relu else 0, 0)
+            _check(self._fn("dot_layer")(self._h, x.data_ptr(), B, xs_i, xs_b, y.data_ptr(), ys_j, ys_b, C.byref(epi),
+                                         wp, wb, st), "dot_layer")
         return y
 
     def dot_noalloc(self, x, y=None, layout="nb"):
@@ -321,3 +338,30 @@ class Format:
 
     def last_launch_count(self) -> int:
         return self._fn("last_launch_count")(self._h)
+
+
+def chain(layers, x, y=None, workspace=None):
+    """hac_chain of the C ABI: `layers` is a list of (Format, bias or None, relu) evaluated one after the
+    other on the current stream; x is a torch float32 CUDA tensor [n0] or [n0, B] (inputs of a batch
+    contiguous), the result [m_last] or [m_last, B].  Returns (y, launches of the whole chain)."""
+    import torch
+    lib = load()
+    B = 1 if x.dim() == 1 else x.shape[1]
+    assert x.is_contiguous() and x.dtype == torch.float32
+    arr = (Layer * len(layers))()
+    for i, (fmt, bias, relu) in enumerate(layers):
+        arr[i].hac = fmt._h if fmt.kind == "hac" else None
+        arr[i].shac = fmt._h if fmt.kind == "shac" else None
+        arr[i].epilogue = Epilogue(bias.data_ptr() if bias is not None else None, 1 if relu else 0, 0)
+    last = layers[-1][0]
+    if y is None:
+        y = torch.empty((last.m,) if x.dim() == 1 else (last.m, B), dtype=torch.float32, device=x.device)
+    widest = max([f.m for f, _, _ in layers[:-1]] + [1]) * B
+    acts = torch.empty((2, widest), dtype=torch.float32, device=x.device)
+    need = max(f.workspace_bytes(B) for f, _, _ in layers)
+    if workspace is None or workspace.numel() < need:
+        workspace = torch.empty(max(need, 16), dtype=torch.uint8, device=x.device)
+    st = torch.cuda.current_stream().cuda_stream
+    _check(lib.hac_chain(arr, len(layers), x.data_ptr(), B, y.data_ptr(), acts[0].data_ptr(), acts[1].data_ptr(), widest,
+                         workspace.data_ptr(), workspace.numel(), st), "hac_chain")
+    return y, last.last_launch_count()

@@ -134,6 +134,9 @@ struct Format {
     DecodeTables tables;
     DeviceImage dev;
     mutable int last_launches = 0;
+    // epilogue of the product being launched (set by the *_dot_layer entry points for the duration of a call)
+    mutable const float* epi_bias = nullptr;
+    mutable uint32_t epi_relu = 0;
 };
 
 int build_impl(const float* W, int64_t n, int64_t m, int64_t ldw, const hac_build_params* p,

@@ -63,7 +63,20 @@ struct DevFormat {
     // leading ones than the longest code word has bits: xt_low, OR-ed into ~window, keeps the index out of them);
     // its unresolved cells go to the search over lengths (no sub-tables).
     uint32_t tab_kind, l1_entries, xt_mant, xt_row0, xt_low;
+    // what is done to an output before it is stored (layer evaluation): + bias[j], then max(., 0)
+    const float* epi_bias;
+    uint32_t epi_relu;
 };
+
+// The value stored for output j: the product, plus the layer's bias, through its activation.  (A NaN stays a NaN.)
+__device__ __forceinline__ float finish_output(const float* __restrict__ bias, uint32_t relu, float v, uint32_t j) {
+    if (bias) v += __ldg(bias + j);
+    if (relu && v < 0.0f) v = 0.0f;
+    return v;
+}
+__device__ __forceinline__ float finish_output(const DevFormat& f, float v, uint32_t j) {
+    return finish_output(f.epi_bias, f.epi_relu, v, j);
+}
 
 
 // ------------------------------------------------------------------------------------------------
@@ -773,13 +786,13 @@ __global__ void __launch_bounds__(1024) hac_vec_kernel(DevFormat f, TablePlan tp
             for (int c = 0; c < kChains; ++c) acc[c] = warp_sum(acc[c]);
             if (lane == 0) {
                 if (kChains == 2 && f.G == 2) {              // the item is one whole column
-                    y[(int64_t)item * ys_j] = acc[0] + acc[kChains - 1];
+                    y[(int64_t)item * ys_j] = finish_output(f, acc[0] + acc[kChains - 1], item);
                 } else {
 #pragma unroll
                     for (int c = 0; c < kChains; ++c) {
                         const uint32_t u = item * kChains + c;
                         if (u < f.units) {
-                            if (f.G == 1) y[(int64_t)u * ys_j] = acc[c];
+                            if (f.G == 1) y[(int64_t)u * ys_j] = finish_output(f, acc[c], u);
                             else aux[u] = acc[c];
                         }
                     }
@@ -1192,7 +1205,7 @@ __global__ void __launch_bounds__(kC <= 2 ? 512 : 384, 1) hac_rows_kernel(DevFor
         for (uint32_t t = threadIdx.x; t < ncol; t += blockDim.x) {
             float s = 0.0f;
             for (uint32_t g = 0; g < f.G; ++g) s += colsum[t * f.G + g];
-            y[(int64_t)(col0 + t) * ys_j] = s;
+            y[(int64_t)(col0 + t) * ys_j] = finish_output(f, s, col0 + t);
         }
     }
 }
@@ -1398,7 +1411,7 @@ __global__ void __launch_bounds__(1024) shac_vec_kernel(DevFormat f, TablePlan t
             for (int c = 0; c < kChains; ++c) acc[c] = warp_sum(acc[c]);
             if (lane == 0) {
                 if (cur.whole_column) {
-                    y[(int64_t)cur.col * ys_j] = acc[0] + acc[1];
+                    y[(int64_t)cur.col * ys_j] = finish_output(f, acc[0] + acc[1], cur.col);
                 } else {
 #pragma unroll
                     for (int c = 0; c < kChains; ++c)
@@ -1683,7 +1696,7 @@ __global__ void __launch_bounds__(1024) shac_items_kernel(DevFormat f, TablePlan
             for (int c = 0; c < kC; ++c) acc[c] = warp_sum(acc[c]);
             if (lane == 0) {
                 if (cur.whole_column) {
-                    y[(int64_t)cur.col * ys_j] = acc[0] + acc[1];
+                    y[(int64_t)cur.col * ys_j] = finish_output(f, acc[0] + acc[1], cur.col);
                 } else {
 #pragma unroll
                     for (int c = 0; c < kC; ++c)
@@ -1714,7 +1727,7 @@ __global__ void finalize_kernel(DevFormat f, bool sparse, const float* __restric
     if (u1 - u0 >= 1 && u1 - u0 <= direct_up_to) return;       // written by the product kernel itself
     float s = 0.0f;
     for (uint32_t u = u0; u < u1; ++u) s += partial[(size_t)u * batch + b];
-    y[(int64_t)j * ys_j + (int64_t)b * ys_b] = s;
+    y[(int64_t)j * ys_j + (int64_t)b * ys_b] = finish_output(f, s, j);
 }
 
 // Row splits of the batched HAC kernel: y[j][b] = sum over splits of partial[split][b][j], added in
@@ -1722,7 +1735,8 @@ __global__ void finalize_kernel(DevFormat f, bool sparse, const float* __restric
 // the partial sums) and writes along whichever of the two indices is contiguous in y.
 __global__ void __launch_bounds__(256) gemm_finalize_kernel(const float* __restrict__ partial, uint32_t splits,
                                                             uint32_t m, uint32_t batch, float* __restrict__ y,
-                                                            int64_t ys_j, int64_t ys_b) {
+                                                            int64_t ys_j, int64_t ys_b, const float* __restrict__ bias,
+                                                            uint32_t relu) {
     __shared__ float tile[32][33];
     allow_dependents();
     depends_wait();
@@ -1738,12 +1752,12 @@ __global__ void __launch_bounds__(256) gemm_finalize_kernel(const float* __restr
     if (ys_b == 1 && ys_j != 1) {
         for (uint32_t jj = threadIdx.y; jj < 32; jj += blockDim.y) {
             const uint32_t j = j0 + jj, b = b0 + threadIdx.x;
-            if (j < m && b < batch) y[(int64_t)j * ys_j + b] = tile[threadIdx.x][jj];
+            if (j < m && b < batch) y[(int64_t)j * ys_j + b] = finish_output(bias, relu, tile[threadIdx.x][jj], j);
         }
     } else {
         for (uint32_t bb = threadIdx.y; bb < 32; bb += blockDim.y) {
             const uint32_t j = j0 + threadIdx.x, b = b0 + bb;
-            if (j < m && b < batch) y[(int64_t)j * ys_j + (int64_t)b * ys_b] = tile[bb][threadIdx.x];
+            if (j < m && b < batch) y[(int64_t)j * ys_j + (int64_t)b * ys_b] = finish_output(bias, relu, tile[bb][threadIdx.x], j);
         }
     }
 }
@@ -2251,7 +2265,7 @@ __global__ void __launch_bounds__(kGWarps * 32, 1) hac_gemm_tc_kernel(
                 if (j < f.m) {
 #pragma unroll
                     for (int cc = 0; cc < 32; ++cc)
-                        if (b0 + cc < batch) y[(int64_t)j + (int64_t)(b0 + cc) * ys_b] = acc[cc];
+                        if (b0 + cc < batch) y[(int64_t)j + (int64_t)(b0 + cc) * ys_b] = finish_output(f, acc[cc], j);
                 }
             } else {
                 float* tile = reinterpret_cast<float*>(smem + spans) + warp * (32 * 33);
@@ -2263,7 +2277,7 @@ __global__ void __launch_bounds__(kGWarps * 32, 1) hac_gemm_tc_kernel(
                 if (b0 + lane < batch) {
                     float* yb = y + (int64_t)(b0 + lane) * ys_b;
                     const uint32_t jn = min(32u, f.m > jw ? f.m - jw : 0u);
-                    for (uint32_t jj = 0; jj < jn; ++jj) yb[(int64_t)(jw + jj) * ys_j] = tile[lane * 33 + jj];
+                    for (uint32_t jj = 0; jj < jn; ++jj) yb[(int64_t)(jw + jj) * ys_j] = finish_output(f, tile[lane * 33 + jj], jw + jj);
                 }
             }
         }
@@ -2287,7 +2301,7 @@ __global__ void __launch_bounds__(kGWarps * 32, 1) hac_gemm_tc_kernel(
                 float sum = 0.0f;
                 for (uint32_t r = 0; r < row_splits; ++r) sum += remote((jl * (kGBatch + 1) + b) * 4u, r);
                 const uint32_t j = cblk * kGCols + jl, bb = bt * kGBatch + b;
-                if (j < f.m && bb < batch) y[(int64_t)j * ys_j + bb] = sum;
+                if (j < f.m && bb < batch) y[(int64_t)j * ys_j + bb] = finish_output(f, sum, j);
             }
         } else {                                     // a share of the inputs, columns fastest
             const uint32_t b0 = kGBatch * rs / row_splits, b1 = kGBatch * (rs + 1) / row_splits;
@@ -2296,7 +2310,7 @@ __global__ void __launch_bounds__(kGWarps * 32, 1) hac_gemm_tc_kernel(
                 float sum = 0.0f;
                 for (uint32_t r = 0; r < row_splits; ++r) sum += remote((b * kGCols + jl) * 4u, r);
                 const uint32_t j = cblk * kGCols + jl, bb = bt * kGBatch + b;
-                if (j < f.m && bb < batch) y[(int64_t)j * ys_j + (int64_t)bb * ys_b] = sum;
+                if (j < f.m && bb < batch) y[(int64_t)j * ys_j + (int64_t)bb * ys_b] = finish_output(f, sum, j);
             }
         }
         // nobody leaves while its tile may still be read
@@ -2402,7 +2416,7 @@ __global__ void __launch_bounds__(1024) shac_batch_kernel(DevFormat f, TablePlan
         for (int a = 0; a < kAcc; ++a) {
             const uint32_t b = b0 + a * 32 + lane;
             if (writer && b < batch) {
-                if (single) y[(int64_t)j * ys_j + (int64_t)b * ys_b] = acc[a];
+                if (single) y[(int64_t)j * ys_j + (int64_t)b * ys_b] = finish_output(f, acc[a], j);
                 else partial[(size_t)u * batch + b] = acc[a];
             }
         }
@@ -2481,6 +2495,7 @@ static DevFormat dev_format(const Format& f) {
     d.max_unit_chunks = f.max_unit_chunks;
     d.max_sub_chunks = f.max_sub_chunks;
     d.tab_kind = 0;
+    d.epi_bias = f.epi_bias; d.epi_relu = f.epi_relu;
     return d;
 }
 
@@ -3090,8 +3105,16 @@ static int launch_batch_t(const Format& f, const DeviceInfo& di, const DevFormat
 }
 
 static int dot(const Format& f, const float* x, int64_t batch, int64_t xs_i, int64_t xs_b, float* y,
-               int64_t ys_j, int64_t ys_b, void* workspace, size_t workspace_bytes_given, void* stream_) {
+               int64_t ys_j, int64_t ys_b, void* workspace, size_t workspace_bytes_given, void* stream_,
+               const hac_epilogue* epi = nullptr) {
     if (!f.dev.base) return HAC_ERR_NOT_UPLOADED;
+    if (epi && epi->reserved != 0) return HAC_ERR_INVALID_ARG;
+    // the epilogue rides in the kernel-side view of the format for the duration of this call
+    struct EpilogueScope {
+        const Format& f;
+        EpilogueScope(const Format& f_, const hac_epilogue* e) : f(f_) { f.epi_bias = e ? e->bias : nullptr; f.epi_relu = e ? (e->relu != 0) : 0; }
+        ~EpilogueScope() { f.epi_bias = nullptr; f.epi_relu = 0; }
+    } scope(f, epi);
     if (!x || !y || batch < 1 || batch > ((int64_t)1 << 24)) return HAC_ERR_INVALID_ARG;
     const size_t need = workspace_bytes(f, batch);
     if (need > 0 && (!workspace || workspace_bytes_given < need)) return HAC_ERR_BUFFER_TOO_SMALL;
@@ -3153,7 +3176,7 @@ static int dot(const Format& f, const float* x, int64_t batch, int64_t xs_i, int
             // launched the ordinary way: started early, its blocks only took the idle SMs from the product
             // kernel's successor (measured: slower)
             gemm_finalize_kernel<<<grid, dim3(32, 8), 0, st>>>(partial, gemm_splits, (uint32_t)f.m, (uint32_t)batch, y,
-                                                               ys_j, ys_b);
+                                                               ys_j, ys_b, f.epi_bias, f.epi_relu);
             HAC_CUDA(cudaGetLastError());
             f.last_launches++;
         }
@@ -3311,6 +3334,55 @@ int shac_dot(const shac_format* f, const float* x, int64_t batch, int64_t x_stri
     if (!f) return HAC_ERR_INVALID_ARG;
     return dot(f->f, x, batch, x_stride_i, x_stride_b, y, y_stride_j, y_stride_b, workspace, workspace_bytes_,
                cuda_stream);
+}
+
+int hac_dot_layer(const hac_format* f, const float* x, int64_t batch, int64_t x_stride_i, int64_t x_stride_b, float* y,
+                  int64_t y_stride_j, int64_t y_stride_b, const hac_epilogue* epilogue, void* workspace,
+                  size_t workspace_bytes_, void* cuda_stream) {
+    if (!f) return HAC_ERR_INVALID_ARG;
+    return dot(f->f, x, batch, x_stride_i, x_stride_b, y, y_stride_j, y_stride_b, workspace, workspace_bytes_,
+               cuda_stream, epilogue);
+}
+int shac_dot_layer(const shac_format* f, const float* x, int64_t batch, int64_t x_stride_i, int64_t x_stride_b, float* y,
+                   int64_t y_stride_j, int64_t y_stride_b, const hac_epilogue* epilogue, void* workspace,
+                   size_t workspace_bytes_, void* cuda_stream) {
+    if (!f) return HAC_ERR_INVALID_ARG;
+    return dot(f->f, x, batch, x_stride_i, x_stride_b, y, y_stride_j, y_stride_b, workspace, workspace_bytes_,
+               cuda_stream, epilogue);
+}
+
+// A stack of layers as one chained submission: layer l reads the activations layer l - 1 wrote.
+int hac_chain(const hac_layer* layers, int n_layers, const float* x, int64_t batch, float* y, float* act0, float* act1,
+              size_t act_floats, void* workspace, size_t workspace_bytes_, void* cuda_stream) {
+    if (!layers || n_layers < 1 || !x || !y || batch < 1) return HAC_ERR_INVALID_ARG;
+    // shapes must chain, and the two activation buffers must hold the widest intermediate result
+    for (int l = 0; l < n_layers; ++l) {
+        if ((layers[l].hac != nullptr) == (layers[l].shac != nullptr)) return HAC_ERR_INVALID_ARG;
+        const Format& f = layers[l].hac ? layers[l].hac->f : layers[l].shac->f;
+        if (l > 0) {
+            const Format& p = layers[l - 1].hac ? layers[l - 1].hac->f : layers[l - 1].shac->f;
+            if (p.m != f.n) return HAC_ERR_INVALID_ARG;
+        }
+        if (l + 1 < n_layers) {
+            if (!act0 || (n_layers > 2 && !act1)) return HAC_ERR_INVALID_ARG;
+            if ((size_t)f.m * (size_t)batch > act_floats) return HAC_ERR_BUFFER_TOO_SMALL;
+        }
+        if (workspace_bytes(f, batch) > workspace_bytes_) return HAC_ERR_BUFFER_TOO_SMALL;
+    }
+    const float* in = x;
+    int launches = 0;
+    for (int l = 0; l < n_layers; ++l) {
+        const Format& f = layers[l].hac ? layers[l].hac->f : layers[l].shac->f;
+        float* out = l + 1 == n_layers ? y : ((l & 1) ? act1 : act0);
+        // activations are [features][batch], inputs of a batch contiguous (a plain vector for one input)
+        const int rc = dot(f, in, batch, batch, 1, out, batch, 1, workspace, workspace_bytes_, cuda_stream, &layers[l].epilogue);
+        if (rc) return rc;
+        launches += f.last_launches;
+        in = out;
+    }
+    const Format& last = layers[n_layers - 1].hac ? layers[n_layers - 1].hac->f : layers[n_layers - 1].shac->f;
+    last.last_launches = launches;               // the whole chain, reported through the last layer's handle
+    return HAC_OK;
 }
 
 int hac_dot_noalloc(const hac_format* f, const float* x, int64_t batch, int64_t x_stride_i, int64_t x_stride_b,

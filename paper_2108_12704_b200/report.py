@@ -134,11 +134,72 @@ def measure(wl, kind, batches, W=None, seg_symbols=0, max_check_batch=128, repla
     return rows
 
 
+def measure_chain(batches=(1, 64), replays=200):
+    """The fully connected stack of the paper's VGG19 (512 -> 4096 -> 4096 -> 10, Sect. V) evaluated on the
+    compressed formats with bias and ReLU applied in the product kernels: time of the three layers submitted as
+    one chain (hac_chain in one CUDA graph) against the three layers each submitted and waited for on its own."""
+    import torch
+    import paper_2108_12704_b200 as hb
+    specs = [(dataclasses.replace(si.CFG3_FC_SHAC, n=512, m=4096, sparsity=0.9, k=32, item=11), "shac", True),
+             (dataclasses.replace(si.CFG2_DENSE_HAC, n=4096, m=4096, k=64, item=12), "hac", True),
+             (dataclasses.replace(si.CFG2_DENSE_HAC, n=4096, m=10, k=32, quantizer=si.QUANT_KMEANS, item=13), "hac", False)]
+    layers = []
+    rng = np.random.default_rng(99)
+    for wl, kind, relu in specs:
+        fmt = hb.Format(kind, si.weights(wl), sparsity=wl.sparsity, k=wl.k, quantizer=wl.quantizer,
+                        kmeans_iters=wl.kmeans_iters, seed=wl.seed).upload()
+        bias = torch.from_numpy((rng.standard_normal(wl.m) * 0.1).astype(np.float32)).cuda()
+        layers.append((fmt, bias, relu))
+    rows = []
+    for B in batches:
+        X = np.maximum(np.random.default_rng(B).standard_normal((B, 512)), 0).astype(np.float32)
+        x = torch.from_numpy(X[0] if B == 1 else np.ascontiguousarray(X.T)).cuda()
+        ws = torch.empty(max(16, max(f.workspace_bytes(B) for f, _, _ in layers)), dtype=torch.uint8, device="cuda")
+        shape = lambda mm: (mm,) if B == 1 else (mm, B)
+        acts = [torch.empty(shape(f.m), device="cuda") for f, _, _ in layers]
+        ins = [x] + acts[:-1]
+        y_chain, launches = hb.hac_chain(layers, x, workspace=ws)
+        for (f, b, r), i, o in zip(layers, ins, acts):
+            f.dot(i, o, ws, bias=b, relu=r)
+        torch.cuda.synchronize()
+        same = bool(torch.equal(acts[-1], y_chain))
+        g_chain = _capture(torch, lambda: hb.hac_chain(layers, x, y_chain, ws))
+        g_layer = [_capture(torch, (lambda f=f, b=b, r=r, i=i, o=o: f.dot(i, o, ws, bias=b, relu=r)))
+                   for (f, b, r), i, o in zip(layers, ins, acts)]
+
+        def timed(graphs, wait_each):
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            torch.cuda.synchronize()
+            e0.record()
+            for _ in range(replays):
+                for g in graphs:
+                    g.replay()
+                    if wait_each:
+                        torch.cuda.synchronize()
+            e1.record()
+            torch.cuda.synchronize()
+            return e0.elapsed_time(e1) / replays * 1e3
+
+        timed([g_chain], False)
+        t_chain = min(timed([g_chain], False) for _ in range(3))
+        t_alone = [min(timed([g], True) for _ in range(3)) for g in g_layer]
+        rows.append(dict(report="layer_chain", stack="512-4096-4096-10 (sHAC 90 % pruned k=32, HAC k=64, HAC k=32), bias + ReLU",
+                         batch=B, launches_per_chain=launches, chain_us=round(t_chain, 2),
+                         per_layer_in_chain_us=round(t_chain / len(layers), 2),
+                         layers_alone_us=[round(t, 2) for t in t_alone], sum_alone_us=round(sum(t_alone), 2),
+                         chain_equals_layers=same,
+                         note="chain: one graph of the chained submission replayed back to back; alone: each layer's graph "
+                              "replayed and waited for by the host before the next (launch and wait latency included); "
+                              "the format stays in L2 here (no replica rotation)"))
+    return rows
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--configs", default="1,2,3,4")
     ap.add_argument("--sweep", action="store_true", help="configuration 5: sparsity x k grid, HAC and sHAC")
     ap.add_argument("--paper-shapes", action="store_true", help="the fully connected shapes of the paper's Sect. V-C")
+    ap.add_argument("--chain", action="store_true", help="the fully connected stack as a chain of layers")
     ap.add_argument("--out", default="")
     args = ap.parse_args()
     out = open(args.out, "w") if args.out else None
@@ -164,6 +225,8 @@ def main():
         for wl in cells:
             for kind in wl.formats:
                 emit(measure(wl, kind, wl.batches, W=W))
+    if args.chain:
+        emit(measure_chain())
     if args.paper_shapes:
         for wl in si.paper_shaped_cells():
             for kind in wl.formats:

@@ -98,3 +98,41 @@ def test_definition_column_subset():
     cols = np.array([0, 7, 15])
     ys, as_ = orc.dot_definition(Wq, X, cols=cols)
     assert np.array_equal(ys, y[:, cols]) and np.array_equal(as_, a[:, cols])
+
+
+# ---------------------------------------------------------------- layers (bias, activation, chains)
+def test_layer_definition_against_the_hand_worked_example():
+    from golden_io import golden, read_sections
+    g = read_sections(golden("layer_hand_worked.txt"))
+    num = lambda key: np.array([[float(v) for v in row] for row in g[key]])
+    W = num("W").astype(np.float32); x = num("x")[0].astype(np.float32); bias = num("bias")[0]
+    y, a = orc.layer_definition(W, x, bias, relu=False)
+    assert y[0].tolist() == num("linear")[0].tolist() and a[0].tolist() == num("scale")[0].tolist()
+    y, _ = orc.layer_definition(W, x, bias, relu=True)
+    assert y[0].tolist() == num("relu")[0].tolist()
+    V = num("V").astype(np.float32); bias2 = num("bias2")[0]
+    outs = orc.chain_definition([(W, bias, True), (V, bias2, False)], x)
+    assert outs[1][0][0].tolist() == num("chain_linear")[0].tolist()
+    outs = orc.chain_definition([(W, bias, True), (V, bias2, True)], x)
+    assert outs[1][0][0].tolist() == num("chain_relu")[0].tolist()
+
+
+def test_layer_definition_properties():
+    rng = np.random.default_rng(11)
+    W = rng.standard_normal((40, 9)).astype(np.float32); X = rng.standard_normal((3, 40)).astype(np.float32)
+    b = rng.standard_normal(9)
+    y0, a0 = orc.dot_definition(W, X)
+    y1, a1 = orc.layer_definition(W, X)                       # no bias, no activation: the product itself
+    assert np.array_equal(y0, y1) and np.array_equal(a0, a1)
+    yb, ab = orc.layer_definition(W, X, b)
+    assert np.array_equal(yb, y0 + b) and np.array_equal(ab, a0 + np.abs(b))
+    yr, _ = orc.layer_definition(W, X, b, relu=True)
+    assert np.array_equal(yr, np.maximum(yb, 0.0)) and (yr >= 0).all()
+    cols = np.array([1, 4, 8])
+    yc, ac = orc.layer_definition(W, X, b, relu=True, cols=cols)
+    assert np.array_equal(yc, yr[:, cols]) and np.array_equal(ac, ab[:, cols])
+    # a chain equals the layers applied one after the other with fp32 activations in between
+    V = rng.standard_normal((9, 4)).astype(np.float32)
+    outs = orc.chain_definition([(W, b, True), (V, None, False)], X)
+    want, _ = orc.dot_definition(V, yr.astype(np.float32))
+    assert np.array_equal(outs[1][0], want)
