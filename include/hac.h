@@ -42,9 +42,9 @@ extern "C" {
 #define HAC_ERR_NOT_UPLOADED     -7   /* device call on a format that was not uploaded            */
 #define HAC_ERR_BUFFER_TOO_SMALL -8   /* caller's buffer or workspace too small                   */
 #define HAC_ERR_CUDA             -9   /* a CUDA runtime call failed                               */
-#define HAC_ERR_CORRUPT          -10  /* serialized data fails validation                         */
+#define HAC_ERR_CORRUPT          -10  /* serialized data fails validation (*_deserialize, *_decode_host) */
 
-#define HAC_MAX_SYMBOLS        2048   /* largest alphabet (distinct values, zero included)        */
+#define HAC_MAX_SYMBOLS        4096   /* largest alphabet (distinct values, zero included)        */
 #define HAC_MAX_SEG_SYMBOLS    1024   /* largest sub-segment length of the offset index           */
 
 #define HAC_QUANT_NONE     0u   /* W already holds few distinct values                            */
@@ -177,6 +177,23 @@ int shac_export(const shac_format* f, shac_host_view* out);
  * leading dimension ldq >= m), reconstructed on the host from the stream (lossless, Sect. IV-B). */
 int hac_decode_host (const hac_format*  f, float* Wq, int64_t ldq);
 int shac_decode_host(const shac_format* f, float* Wq, int64_t ldq);
+
+/* ---------------------------------------------------------------------------------------------
+ * A built format as one flat little-endian byte string (the formats are the stored artefact, Sect. IV):
+ * *_serialize_bytes gives its length, *_serialize writes it into the caller's host buffer, and
+ * *_deserialize makes a new handle from such a string (released with *_free like any other).  The
+ * string holds what is stored (codebook, code lengths, counts, stream, offset index, ri, cb) and a
+ * checksum; decoding tables and work lists are rebuilt on load.  *_deserialize trusts nothing: a string
+ * that is truncated, altered, inconsistent with its own header, or whose code, offset index or CSC
+ * vectors are not valid gives HAC_ERR_CORRUPT (a string of the other format: HAC_ERR_INVALID_ARG).
+ * Host only.
+ * ------------------------------------------------------------------------------------------- */
+int hac_serialize_bytes (const hac_format*  f, size_t* out);
+int shac_serialize_bytes(const shac_format* f, size_t* out);
+int hac_serialize (const hac_format*  f, void* buf, size_t bytes);
+int shac_serialize(const shac_format* f, void* buf, size_t bytes);
+int hac_deserialize (const void* buf, size_t bytes, hac_format**  out);
+int shac_deserialize(const void* buf, size_t bytes, shac_format** out);
 
 /* ---------------------------------------------------------------------------------------------
  * Upload.  *_device_bytes gives the size of the device image of a format (all arrays the kernels

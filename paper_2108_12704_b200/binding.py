@@ -67,7 +67,8 @@ _lib = None
 # every symbol include/hac.h declares
 EXPORTS = (
     "hac_build", "shac_build", "hac_sizes", "shac_sizes", "hac_export", "shac_export",
-    "hac_decode_host", "shac_decode_host", "hac_device_bytes", "shac_device_bytes", "hac_upload",
+    "hac_decode_host", "shac_decode_host", "hac_serialize_bytes", "shac_serialize_bytes", "hac_serialize",
+    "shac_serialize", "hac_deserialize", "shac_deserialize", "hac_device_bytes", "shac_device_bytes", "hac_upload",
     "shac_upload", "hac_attach", "shac_attach", "hac_workspace_bytes", "shac_workspace_bytes", "hac_dot",
     "shac_dot", "hac_dot_noalloc", "hac_dot_layer", "shac_dot_layer", "hac_chain", "hac_dot_host_scratch_bytes", "shac_dot_host_scratch_bytes", "hac_dot_host",
     "shac_dot_host", "hac_dot_host_async", "shac_dot_host_async", "hac_debug_decode", "shac_debug_decode",
@@ -96,6 +97,9 @@ def load():
         getattr(lib, f"{kind}_sizes").argtypes = [vp, C.POINTER(SizeReport)]
         getattr(lib, f"{kind}_export").argtypes = [vp, vp]
         getattr(lib, f"{kind}_decode_host").argtypes = [vp, fp, i64]
+        getattr(lib, f"{kind}_serialize_bytes").argtypes = [vp, C.POINTER(sz)]
+        getattr(lib, f"{kind}_serialize").argtypes = [vp, vp, sz]
+        getattr(lib, f"{kind}_deserialize").argtypes = [vp, sz, C.POINTER(vp)]
         getattr(lib, f"{kind}_device_bytes").argtypes = [vp, C.POINTER(sz)]
         getattr(lib, f"{kind}_upload").argtypes = [vp, vp, sz, vp]
         getattr(lib, f"{kind}_attach").argtypes = [vp, vp, sz]
@@ -200,6 +204,29 @@ class Format:
                    seg_bit_off=_arr(base.seg_bit_off, base.units, np.uint64),
                    sub_bits=_arr(base.sub_bits, base.units * 32, np.uint16))
         return out
+
+    def serialize(self) -> bytes:
+        """The format as one byte string (*_serialize of the C ABI)."""
+        n = C.c_size_t()
+        _check(self._fn("serialize_bytes")(self._h, C.byref(n)), "serialize_bytes")
+        buf = (C.c_ubyte * n.value)()
+        _check(self._fn("serialize")(self._h, buf, n.value), "serialize")
+        return bytes(buf)
+
+    @classmethod
+    def deserialize(cls, kind: str, blob: bytes) -> "Format":
+        """A handle from a byte string written by serialize() (*_deserialize of the C ABI)."""
+        assert kind in ("hac", "shac")
+        self = cls.__new__(cls)
+        self.kind = kind
+        self._lib = load()
+        self._h = C.c_void_p()
+        self._device_buffer = None
+        buf = (C.c_ubyte * len(blob)).from_buffer_copy(blob)
+        _check(getattr(self._lib, f"{kind}_deserialize")(buf, len(blob), C.byref(self._h)), f"{kind}_deserialize")
+        sz = self.sizes()
+        self.n, self.m = sz["n"], sz["m"]
+        return self
 
     def decode_host(self) -> np.ndarray:
         Wq = np.empty((self.n, self.m), dtype=np.float32)

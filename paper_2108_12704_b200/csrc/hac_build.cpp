@@ -326,7 +326,7 @@ void make_decode_tables(Format& f) {
         if (l > t.lut_bits) continue;
         const uint32_t lo = f.codes[s] << (t.lut_bits - l);
         const uint32_t span = 1u << (t.lut_bits - l);
-        const uint16_t e = (uint16_t)((r << 5) | (uint32_t)l);
+        const uint16_t e = (uint16_t)((r << 4) | (uint32_t)l);      // l <= kLutBitsMax = 12, r < 4096
         for (uint32_t i = 0; i < span; ++i) t.lut[lo + i] = e;
     }
     // two-level table: direct entries for code words of at most l1_bits bits, sub-tables behind
@@ -459,6 +459,85 @@ void make_decode_tables(Format& f) {
             }
         }
     }
+}
+
+// Everything that is derived from the stored arrays of a format (used by the builder and by deserialization):
+// shared-memory sizing statistics, the device-only work lists and start-bit table, the decoding tables.
+void finish_derived(Format& f) {
+    const bool sparse = f.sparse;
+    const int64_t n = f.n, m = f.m;
+    const uint32_t S = f.S;
+    // per-segment statistics used to size shared memory and to pick the reduction path
+    const size_t U = f.seg_bit_off.size();
+    f.max_unit_chunks = 1;
+    f.max_sub_chunks = 1;
+    for (size_t u = 0; u < U; ++u) {
+        uint64_t bits = 0;
+        for (int l = 0; l < 32; ++l) bits += f.sub_bits[u * 32 + l];
+        const uint64_t first_chunk = f.seg_bit_off[u] >> 7;
+        const uint64_t last_word = ((f.seg_bit_off[u] + bits) >> 5) + 2;
+        f.max_unit_chunks = std::max<uint32_t>(f.max_unit_chunks, (uint32_t)((last_word >> 2) - first_chunk + 1));
+        uint64_t at = f.seg_bit_off[u];
+        for (int l = 0; l < 32; ++l) {
+            const uint64_t sub_last_word = ((at + f.sub_bits[u * 32 + l]) >> 5) + 2;
+            f.max_sub_chunks = std::max<uint32_t>(f.max_sub_chunks, (uint32_t)((sub_last_word >> 2) - (at >> 7) + 1));
+            at += f.sub_bits[u * 32 + l];
+        }
+    }
+    if (sparse) {
+        // device-only work list: an item is one or two consecutive segments of one column
+        f.item_info.clear();
+        for (int64_t j = 0; j < m; ++j) {
+            const uint32_t u_begin = f.seg_first[j], u_end = f.seg_first[j + 1];
+            for (uint32_t u = u_begin; u < u_end; u += 2) {
+                const uint32_t in_item = std::min(2u, u_end - u);
+                uint32_t rec[kItemWords] = {0};
+                for (uint32_t c = 0; c < in_item; ++c) {
+                    // the segment's 32 sub-segment bit lengths, so that one read brings all an item needs
+                    for (uint32_t l = 0; l < 32; ++l) {
+                        const uint32_t bits = f.sub_bits[(size_t)(u + c) * 32 + l];
+                        rec[12 + 16 * c + l / 2] |= bits << (16 * (l & 1u));
+                    }
+                    const uint32_t pos0 = f.cb[j] + (u + c - u_begin) * 32u * S;
+                    rec[4 * c + 0] = (uint32_t)(f.seg_bit_off[u + c] & 0xffffffffu);
+                    rec[4 * c + 1] = (uint32_t)(f.seg_bit_off[u + c] >> 32);
+                    rec[4 * c + 2] = pos0;
+                    rec[4 * c + 3] = std::min<uint32_t>(32u * S, f.cb[j + 1] - pos0);
+                }
+                rec[8] = (uint32_t)j;
+                rec[9] = in_item | ((u_end - u_begin) <= 2 ? 0x100u : 0u);   // bit 8: the item is the whole column
+                rec[10] = u;
+                f.item_info.insert(f.item_info.end(), rec, rec + kItemWords);
+            }
+        }
+        f.max_units_per_col = 0;
+        f.has_empty_col = false;
+        for (int64_t j = 0; j < m; ++j) {
+            const uint32_t g = f.seg_first[j + 1] - f.seg_first[j];
+            f.max_units_per_col = std::max(f.max_units_per_col, g);
+            if (g == 0) f.has_empty_col = true;
+        }
+    } else {
+        f.max_units_per_col = f.G;
+        const uint64_t tasks = ((uint64_t)n + S - 1) / S;
+        f.task_off.clear();
+        if ((tasks + 1) * (uint64_t)m * 8 <= kTaskOffBytesMax) {
+            f.task_off.assign((size_t)((tasks + 1) * (uint64_t)m), 0);
+            for (int64_t j = 0; j < m; ++j) {
+                uint64_t t = 0;
+                for (uint32_t g = 0; g < f.G; ++g) {
+                    const size_t u = (size_t)j * f.G + g;
+                    uint64_t at = f.seg_bit_off[u];
+                    for (uint32_t l = 0; l < 32 && t < tasks; ++l, ++t) {
+                        f.task_off[(size_t)t * m + j] = at;
+                        at += f.sub_bits[u * 32 + l];
+                    }
+                    if (t == tasks) f.task_off[(size_t)tasks * m + j] = at;
+                }
+            }
+        }
+    }
+    make_decode_tables(f);
 }
 
 int build_impl(const float* W, int64_t n, int64_t m, int64_t ldw, const hac_build_params* p,
@@ -627,77 +706,7 @@ int build_impl(const float* W, int64_t n, int64_t m, int64_t ldw, const hac_buil
     f.pad_words = padded - f.stream_words;
     f.stream.resize(padded, 0u);
 
-    // per-segment statistics used to size shared memory and to pick the reduction path
-    const size_t U = f.seg_bit_off.size();
-    f.max_unit_chunks = 1;
-    f.max_sub_chunks = 1;
-    for (size_t u = 0; u < U; ++u) {
-        uint64_t bits = 0;
-        for (int l = 0; l < 32; ++l) bits += f.sub_bits[u * 32 + l];
-        const uint64_t first_chunk = f.seg_bit_off[u] >> 7;
-        const uint64_t last_word = ((f.seg_bit_off[u] + bits) >> 5) + 2;
-        f.max_unit_chunks = std::max<uint32_t>(f.max_unit_chunks, (uint32_t)((last_word >> 2) - first_chunk + 1));
-        uint64_t at = f.seg_bit_off[u];
-        for (int l = 0; l < 32; ++l) {
-            const uint64_t sub_last_word = ((at + f.sub_bits[u * 32 + l]) >> 5) + 2;
-            f.max_sub_chunks = std::max<uint32_t>(f.max_sub_chunks, (uint32_t)((sub_last_word >> 2) - (at >> 7) + 1));
-            at += f.sub_bits[u * 32 + l];
-        }
-    }
-    if (sparse) {
-        // device-only work list: an item is one or two consecutive segments of one column
-        f.item_info.clear();
-        for (int64_t j = 0; j < m; ++j) {
-            const uint32_t u_begin = f.seg_first[j], u_end = f.seg_first[j + 1];
-            for (uint32_t u = u_begin; u < u_end; u += 2) {
-                const uint32_t in_item = std::min(2u, u_end - u);
-                uint32_t rec[kItemWords] = {0};
-                for (uint32_t c = 0; c < in_item; ++c) {
-                    // the segment's 32 sub-segment bit lengths, so that one read brings all an item needs
-                    for (uint32_t l = 0; l < 32; ++l) {
-                        const uint32_t bits = f.sub_bits[(size_t)(u + c) * 32 + l];
-                        rec[12 + 16 * c + l / 2] |= bits << (16 * (l & 1u));
-                    }
-                    const uint32_t pos0 = f.cb[j] + (u + c - u_begin) * 32u * S;
-                    rec[4 * c + 0] = (uint32_t)(f.seg_bit_off[u + c] & 0xffffffffu);
-                    rec[4 * c + 1] = (uint32_t)(f.seg_bit_off[u + c] >> 32);
-                    rec[4 * c + 2] = pos0;
-                    rec[4 * c + 3] = std::min<uint32_t>(32u * S, f.cb[j + 1] - pos0);
-                }
-                rec[8] = (uint32_t)j;
-                rec[9] = in_item | ((u_end - u_begin) <= 2 ? 0x100u : 0u);   // bit 8: the item is the whole column
-                rec[10] = u;
-                f.item_info.insert(f.item_info.end(), rec, rec + kItemWords);
-            }
-        }
-        f.max_units_per_col = 0;
-        f.has_empty_col = false;
-        for (int64_t j = 0; j < m; ++j) {
-            const uint32_t g = f.seg_first[j + 1] - f.seg_first[j];
-            f.max_units_per_col = std::max(f.max_units_per_col, g);
-            if (g == 0) f.has_empty_col = true;
-        }
-    } else {
-        f.max_units_per_col = f.G;
-        const uint64_t tasks = ((uint64_t)n + S - 1) / S;
-        f.task_off.clear();
-        if ((tasks + 1) * (uint64_t)m * 8 <= kTaskOffBytesMax) {
-            f.task_off.assign((size_t)((tasks + 1) * (uint64_t)m), 0);
-            for (int64_t j = 0; j < m; ++j) {
-                uint64_t t = 0;
-                for (uint32_t g = 0; g < f.G; ++g) {
-                    const size_t u = (size_t)j * f.G + g;
-                    uint64_t at = f.seg_bit_off[u];
-                    for (uint32_t l = 0; l < 32 && t < tasks; ++l, ++t) {
-                        f.task_off[(size_t)t * m + j] = at;
-                        at += f.sub_bits[u * 32 + l];
-                    }
-                    if (t == tasks) f.task_off[(size_t)tasks * m + j] = at;
-                }
-            }
-        }
-    }
-    make_decode_tables(f);
+    finish_derived(f);
     return HAC_OK;
 }
 
@@ -806,6 +815,159 @@ ImageLayout image_layout(const Format& f) {
     return L;
 }
 
+
+// ------------------------------------------------------------------------------------------------
+// Flat little-endian image of a built format (what has to be stored to use it later; everything
+// derived is rebuilt on load).  Layout: 16 header words of 64 bits, then the arrays in the order of
+// write_arrays(), each padded to 8 bytes, then a 64-bit FNV-1a checksum of all bytes before it.
+// ------------------------------------------------------------------------------------------------
+static const uint64_t kBlobMagic = 0x3130424341480aefull;      // "\xef\nHACB01"
+static const uint64_t kBlobVersion = 1;
+
+static uint64_t fnv1a(const unsigned char* p, size_t n) {
+    uint64_t h = 0xcbf29ce484222325ull;
+    for (size_t i = 0; i < n; ++i) { h ^= p[i]; h *= 0x100000001b3ull; }
+    return h;
+}
+static size_t pad8(size_t x) { return (x + 7) & ~(size_t)7; }
+
+struct BlobSizes { size_t codebook, code_len, counts, stream, seg_bit_off, sub_bits, seg_first, seg_col, ri, cb, total; };
+static BlobSizes blob_sizes(bool sparse, uint64_t k, uint64_t stream_words_padded, uint64_t units, uint64_t m, uint64_t nnz,
+                            uint32_t ri_bits) {
+    BlobSizes b{};
+    b.codebook = pad8(k * 4); b.code_len = pad8(k); b.counts = k * 8; b.stream = pad8(stream_words_padded * 4);
+    b.seg_bit_off = units * 8; b.sub_bits = pad8(units * 64);
+    b.seg_first = sparse ? pad8((m + 1) * 4) : 0; b.seg_col = sparse ? pad8(units * 4) : 0;
+    b.ri = sparse ? pad8(nnz * (ri_bits / 8)) : 0; b.cb = sparse ? pad8((m + 1) * 4) : 0;
+    b.total = 16 * 8 + b.codebook + b.code_len + b.counts + b.stream + b.seg_bit_off + b.sub_bits + b.seg_first + b.seg_col +
+              b.ri + b.cb + 8;
+    return b;
+}
+
+static size_t serialized_bytes(const Format& f) {
+    return blob_sizes(f.sparse, f.codebook.size(), f.stream.size(), f.seg_bit_off.size(), (uint64_t)f.m, (uint64_t)f.nnz,
+                      f.ri_bits ? f.ri_bits : 32).total;
+}
+
+static int serialize(const Format& f, void* buf, size_t bytes) {
+    if (!buf) return HAC_ERR_INVALID_ARG;
+    const size_t need = serialized_bytes(f);
+    if (bytes < need) return HAC_ERR_BUFFER_TOO_SMALL;
+    unsigned char* p = static_cast<unsigned char*>(buf);
+    std::memset(p, 0, need);
+    const uint64_t hdr[16] = {kBlobMagic, kBlobVersion, f.sparse ? 1u : 0u, (uint64_t)f.n, (uint64_t)f.m, (uint64_t)f.nnz,
+                              (uint64_t)f.symbols, f.S, f.G, f.ri_bits, (uint64_t)f.codebook.size(), (uint64_t)f.stream_bits,
+                              (uint64_t)f.stream_words, (uint64_t)f.pad_words, (uint64_t)f.seg_bit_off.size(), 0};
+    std::memcpy(p, hdr, sizeof(hdr));
+    size_t o = sizeof(hdr);
+    auto put = [&](const void* src, size_t n) { if (n) std::memcpy(p + o, src, n); o += pad8(n); };
+    put(f.codebook.data(), f.codebook.size() * 4);
+    put(f.code_len.data(), f.code_len.size());
+    put(f.counts.data(), f.counts.size() * 8);
+    put(f.stream.data(), f.stream.size() * 4);
+    put(f.seg_bit_off.data(), f.seg_bit_off.size() * 8);
+    put(f.sub_bits.data(), f.sub_bits.size() * 2);
+    if (f.sparse) {
+        put(f.seg_first.data(), f.seg_first.size() * 4);
+        put(f.seg_col.data(), f.seg_col.size() * 4);
+        if (f.ri_bits == 16) put(f.ri16.data(), f.ri16.size() * 2); else put(f.ri32.data(), f.ri32.size() * 4);
+        put(f.cb.data(), f.cb.size() * 4);
+    }
+    const uint64_t sum = fnv1a(p, o);
+    std::memcpy(p + o, &sum, 8);
+    return HAC_OK;
+}
+
+// Rebuilds a format from its image.  Everything is checked before it is used: sizes against the header,
+// the checksum, the code (lengths between 1 and 32 that satisfy the Kraft equality, values strictly
+// ascending, counts that add up to the number of code words and to the length of the stream), the offset
+// index (segments in stream order, sub-segment lengths that tile the stream) and, for sHAC, cb, ri and
+// the segment lists.  Anything else is HAC_ERR_CORRUPT.
+static int deserialize(const void* buf, size_t bytes, bool want_sparse, Format& f) {
+    if (!buf) return HAC_ERR_INVALID_ARG;
+    const unsigned char* p = static_cast<const unsigned char*>(buf);
+    if (bytes < 16 * 8 + 8) return HAC_ERR_CORRUPT;
+    uint64_t hdr[16];
+    std::memcpy(hdr, p, sizeof(hdr));
+    if (hdr[0] != kBlobMagic || hdr[1] != kBlobVersion || hdr[2] > 1 || hdr[15] != 0) return HAC_ERR_CORRUPT;
+    const bool sparse = hdr[2] == 1;
+    if (sparse != want_sparse) return HAC_ERR_INVALID_ARG;
+    const uint64_t n = hdr[3], m = hdr[4], nnz = hdr[5], symbols = hdr[6], S = hdr[7], G = hdr[8], ri_bits = hdr[9], k = hdr[10],
+                   stream_bits = hdr[11], stream_words = hdr[12], pad_words = hdr[13], units = hdr[14];
+    if (n < 1 || m < 1 || n > ((uint64_t)1 << 31) || m > ((uint64_t)1 << 31) || n * m > ((uint64_t)1 << 36)) return HAC_ERR_CORRUPT;
+    if (S < 1 || S > HAC_MAX_SEG_SYMBOLS || k > HAC_MAX_SYMBOLS || nnz > n * m) return HAC_ERR_CORRUPT;
+    if (symbols != (sparse ? nnz : n * m) || (symbols > 0 && k == 0)) return HAC_ERR_CORRUPT;
+    if (sparse ? (ri_bits != 16 && ri_bits != 32) || (ri_bits == 16 && n > 65536) || G != 0 : ri_bits != 0) return HAC_ERR_CORRUPT;
+    if (stream_words != (stream_bits + 31) / 32 || pad_words != ((stream_words + 3) / 4) * 4 + kStreamSlackWords - stream_words)
+        return HAC_ERR_CORRUPT;
+    if (!sparse && (G != ((n + S - 1) / S + 31) / 32 || units != G * m)) return HAC_ERR_CORRUPT;
+    if (units > ((uint64_t)1 << 31)) return HAC_ERR_CORRUPT;
+    const BlobSizes bs = blob_sizes(sparse, k, stream_words + pad_words, units, m, nnz, (uint32_t)(ri_bits ? ri_bits : 32));
+    if (bs.total != bytes) return HAC_ERR_CORRUPT;
+    uint64_t sum;
+    std::memcpy(&sum, p + bytes - 8, 8);
+    if (sum != fnv1a(p, bytes - 8)) return HAC_ERR_CORRUPT;
+
+    f = Format();
+    f.sparse = sparse; f.n = (int64_t)n; f.m = (int64_t)m; f.nnz = (int64_t)nnz; f.symbols = (int64_t)symbols;
+    f.S = (uint32_t)S; f.G = (uint32_t)G; f.ri_bits = (uint32_t)ri_bits;
+    f.stream_bits = (int64_t)stream_bits; f.stream_words = (int64_t)stream_words; f.pad_words = (int64_t)pad_words;
+    size_t o = sizeof(hdr);
+    auto get = [&](void* dst, size_t nbytes) { if (nbytes) std::memcpy(dst, p + o, nbytes); o += pad8(nbytes); };
+    f.codebook.resize(k); get(f.codebook.data(), k * 4);
+    f.code_len.resize(k); get(f.code_len.data(), k);
+    f.counts.resize(k); get(f.counts.data(), k * 8);
+    f.stream.resize(stream_words + pad_words); get(f.stream.data(), f.stream.size() * 4);
+    f.seg_bit_off.resize(units); get(f.seg_bit_off.data(), units * 8);
+    f.sub_bits.resize(units * 32); get(f.sub_bits.data(), units * 64);
+    if (sparse) {
+        f.seg_first.resize(m + 1); get(f.seg_first.data(), (m + 1) * 4);
+        f.seg_col.resize(units); get(f.seg_col.data(), units * 4);
+        if (ri_bits == 16) { f.ri16.resize(nnz); get(f.ri16.data(), nnz * 2); }
+        else { f.ri32.resize(nnz); get(f.ri32.data(), nnz * 4); }
+        f.cb.resize(m + 1); get(f.cb.data(), (m + 1) * 4);
+    }
+    // the code
+    f.max_len = 0; f.min_len = k ? 255 : 0;
+    long double kraft = 0;
+    uint64_t total_count = 0, total_bits = 0;
+    for (uint64_t s = 0; s < k; ++s) {
+        const uint32_t l = f.code_len[s];
+        if (l < 1 || l > (uint32_t)kMaxCodeLen || f.counts[s] < 1) return HAC_ERR_CORRUPT;
+        if (!std::isfinite(f.codebook[s]) || (s > 0 && !(f.codebook[s] > f.codebook[s - 1]))) return HAC_ERR_CORRUPT;
+        kraft += std::ldexp((long double)1, -(int)l);
+        total_count += (uint64_t)f.counts[s]; total_bits += (uint64_t)f.counts[s] * l;
+        f.max_len = std::max(f.max_len, l); f.min_len = std::min(f.min_len, l);
+    }
+    if (k == 1 ? f.code_len[0] != 1 : (k >= 2 && kraft != 1)) return HAC_ERR_CORRUPT;
+    if (total_count != symbols || total_bits != stream_bits || S * f.max_len > 65535u) return HAC_ERR_CORRUPT;
+    for (uint64_t w = stream_words; w < stream_words + pad_words; ++w) if (f.stream[w] != 0) return HAC_ERR_CORRUPT;
+    if (stream_bits & 31u) { if (f.stream[stream_words - 1] & ((1u << (32 - (stream_bits & 31u))) - 1u)) return HAC_ERR_CORRUPT; }
+    canonical_assign(f.code_len, f.codes);
+    // the offset index: segments tile the stream in order
+    uint64_t at = 0;
+    for (uint64_t u = 0; u < units; ++u) {
+        if (f.seg_bit_off[u] != at) return HAC_ERR_CORRUPT;
+        for (int l = 0; l < 32; ++l) at += f.sub_bits[u * 32 + l];
+    }
+    if (at != stream_bits) return HAC_ERR_CORRUPT;
+    if (sparse) {
+        if (f.cb[0] != 0 || f.cb[m] != nnz || f.seg_first[0] != 0 || f.seg_first[m] != units) return HAC_ERR_CORRUPT;
+        for (uint64_t j = 0; j < m; ++j) {
+            if (f.cb[j + 1] < f.cb[j] || f.seg_first[j + 1] < f.seg_first[j]) return HAC_ERR_CORRUPT;
+            const uint64_t entries = f.cb[j + 1] - f.cb[j];
+            if (f.seg_first[j + 1] - f.seg_first[j] != (entries + 32 * S - 1) / (32 * S)) return HAC_ERR_CORRUPT;
+            for (uint32_t u = f.seg_first[j]; u < f.seg_first[j + 1]; ++u) if (f.seg_col[u] != j) return HAC_ERR_CORRUPT;
+            for (uint64_t q = f.cb[j]; q < f.cb[j + 1]; ++q) {
+                const uint64_t r = ri_bits == 16 ? f.ri16[q] : f.ri32[q];
+                if (r >= n || (q > f.cb[j] && r <= (ri_bits == 16 ? (uint64_t)f.ri16[q - 1] : (uint64_t)f.ri32[q - 1]))) return HAC_ERR_CORRUPT;
+            }
+        }
+    }
+    finish_derived(f);
+    return HAC_OK;
+}
+
 }  // namespace hacb200
 
 using hacb200::Format;
@@ -835,6 +997,43 @@ static int table_lookup_host(const Format& f, uint32_t window, float* value, uin
 }
 
 extern "C" {
+
+int hac_serialize_bytes(const hac_format* f, size_t* out) {
+    if (!f || !out) return HAC_ERR_INVALID_ARG;
+    *out = hacb200::serialized_bytes(f->f);
+    return HAC_OK;
+}
+int shac_serialize_bytes(const shac_format* f, size_t* out) {
+    if (!f || !out) return HAC_ERR_INVALID_ARG;
+    *out = hacb200::serialized_bytes(f->f);
+    return HAC_OK;
+}
+int hac_serialize(const hac_format* f, void* buf, size_t bytes) { return f ? hacb200::serialize(f->f, buf, bytes) : HAC_ERR_INVALID_ARG; }
+int shac_serialize(const shac_format* f, void* buf, size_t bytes) { return f ? hacb200::serialize(f->f, buf, bytes) : HAC_ERR_INVALID_ARG; }
+int hac_deserialize(const void* buf, size_t bytes, hac_format** out) {
+    if (!out) return HAC_ERR_INVALID_ARG;
+    *out = nullptr;
+    hac_format* h = new (std::nothrow) hac_format();
+    if (!h) return HAC_ERR_ALLOC;
+    int rc;
+    try { rc = hacb200::deserialize(buf, bytes, false, h->f); }
+    catch (const std::bad_alloc&) { rc = HAC_ERR_ALLOC; }
+    if (rc != HAC_OK) { delete h; return rc; }
+    *out = h;
+    return HAC_OK;
+}
+int shac_deserialize(const void* buf, size_t bytes, shac_format** out) {
+    if (!out) return HAC_ERR_INVALID_ARG;
+    *out = nullptr;
+    shac_format* h = new (std::nothrow) shac_format();
+    if (!h) return HAC_ERR_ALLOC;
+    int rc;
+    try { rc = hacb200::deserialize(buf, bytes, true, h->f); }
+    catch (const std::bad_alloc&) { rc = HAC_ERR_ALLOC; }
+    if (rc != HAC_OK) { delete h; return rc; }
+    *out = h;
+    return HAC_OK;
+}
 
 int hac_debug_table_lookup(const hac_format* f, uint32_t window, float* value, uint32_t* length, int* kind,
                            int* never_unresolved) {

@@ -11,7 +11,8 @@
 namespace hacb200 {
 
 constexpr int kMaxCodeLen = 32;
-constexpr int kLutBitsMax = 12;          // full-width decode table: 2^L entries of 16 bits
+constexpr int kLutBitsMax = 12;          // full-width decode table: 2^L entries of 16 bits (12-bit rank, 4-bit length)
+static_assert(kLutBitsMax < 16 && HAC_MAX_SYMBOLS <= 4096, "a table entry holds (rank << 4) | length in 16 bits");
 constexpr int kL1BitsMax = 10;           // level-1 table of the kernels: 2^L1 entries of 8 bytes
 constexpr int kSubBitsMax = 8;           // widest level-2 sub-table
 constexpr int kXtMantMax = 5;            // magnitude table: at most 32 << 5 entries (the size of the prefix table)
@@ -35,7 +36,7 @@ constexpr int kItemWords = 48;           // sHAC work item record: 12 header wor
 // words use the first entries.
 struct DecodeTables {
     int lut_bits = 0;                         // L = min(max_len, kLutBitsMax)
-    std::vector<uint16_t> lut;                // [2^L] (rank << 5) | len, 0 = code longer than L
+    std::vector<uint16_t> lut;                // [2^L] (rank << 4) | len, 0 = code longer than L
     std::vector<float> rank_value;            // [k_eff]
     std::vector<uint16_t> rank_symbol;        // [k_eff] symbol id of each rank
     // Two-level table used by the kernels.  l1[i] for the L1-bit prefix i is {value bits, length}

@@ -228,7 +228,7 @@ __device__ __noinline__ uint2 decode_long(uint32_t top, const uint16_t* __restri
                                           const uint32_t* __restrict__ first_left,
                                           const uint32_t* __restrict__ rank_base, uint32_t max_len) {
     const uint32_t code = lut[top >> (32 - lut_bits)];
-    uint32_t len = code & 31u, rank = code >> 5;
+    uint32_t len = code & 15u, rank = code >> 4;       // lengths here are at most kLutBitsMax = 12
     if (len == 0) {
         len = max_len; rank = 0;
         for (uint32_t l = lut_bits + 1; l <= max_len; ++l) {

@@ -208,3 +208,75 @@ def test_long_tailed_code_takes_the_magnitude_table():
     f = hb.Format("hac", _geometric_matrix(rng, 40, 0.6, n=3000), sparsity=0.0, k=40, quantizer=si.QUANT_NONE)
     assert f.sizes()["max_code_len"] > 12
     assert f.debug_table_lookup(0)[2] == 1
+
+
+# ---------------------------------------------------------------- serialization
+def _same_arrays(a, b):
+    assert a.keys() == b.keys()
+    for k in a:
+        if isinstance(a[k], np.ndarray):
+            assert a[k].dtype == b[k].dtype and np.array_equal(a[k], b[k]), k
+        else:
+            assert a[k] == b[k], k
+
+
+@pytest.mark.parametrize("kind", ["hac", "shac"])
+def test_serialize_round_trip_and_rejection_of_altered_strings(kind):
+    wl = si.scaled(si.CFG3_FC_SHAC, 700, 60)
+    W = si.weights(wl)
+    f = hb.Format(kind, W, sparsity=wl.sparsity, k=wl.k, quantizer=wl.quantizer, kmeans_iters=wl.kmeans_iters, seed=wl.seed)
+    blob = f.serialize()
+    g = hb.Format.deserialize(kind, blob)
+    _same_arrays(f.export(), g.export())
+    assert f.sizes() == g.sizes()
+    assert np.array_equal(f.decode_host().view(np.uint32), g.decode_host().view(np.uint32))
+    assert g.serialize() == blob
+    for kk in ("xt", "l1"):
+        pass
+    # same tables: the first-level entry of a few windows
+    for w in (0, 0x12345678, 0xffffffff, 0x80000000):
+        assert f.debug_table_lookup(w) == g.debug_table_lookup(w)
+    # every single flipped bit and every truncation is refused (checked on a sample of positions)
+    rng = np.random.default_rng(1)
+    positions = sorted(set([0, 8, 17, 100, 128, len(blob) - 9, len(blob) - 1] + rng.integers(0, len(blob), size=60).tolist()))
+    for pos in positions:
+        bad = bytearray(blob)
+        bad[pos] ^= 1 << int(rng.integers(0, 8))
+        with pytest.raises(hb.HacError) as ei:
+            hb.Format.deserialize(kind, bytes(bad))
+        assert ei.value.status == -10, pos
+    for cut in (0, 7, 127, 136, len(blob) - 8, len(blob) - 1):
+        with pytest.raises(hb.HacError) as ei:
+            hb.Format.deserialize(kind, blob[:cut])
+        assert ei.value.status == -10
+    with pytest.raises(hb.HacError) as ei:
+        hb.Format.deserialize("shac" if kind == "hac" else "hac", blob)
+    assert ei.value.status == -1
+
+
+def test_deserialize_checks_the_contents_not_only_the_checksum():
+    """A string whose checksum was recomputed after tampering is still refused when its code or its index
+    is not valid."""
+    def fnv1a(b):
+        h = 0xcbf29ce484222325
+        for x in b:
+            h = ((h ^ x) * 0x100000001b3) & 0xffffffffffffffff
+        return h
+    W = si.weights(si.scaled(si.CFG2_DENSE_HAC, 300, 20))
+    f = hb.Format("hac", W, sparsity=0.0, k=16, quantizer=si.QUANT_UNIFORM)
+    blob = bytearray(f.serialize())
+    k = f.sizes()["k_eff"]
+    def resealed(b):
+        b = bytearray(b)
+        b[-8:] = fnv1a(bytes(b[:-8])).to_bytes(8, "little")
+        return bytes(b)
+    hb.Format.deserialize("hac", resealed(blob))                       # untouched and resealed: accepted
+    off_len = 128 + ((4 * k + 7) // 8) * 8                               # code lengths follow the codebook
+    bad = bytearray(blob); bad[off_len] += 1                            # breaks the Kraft equality
+    with pytest.raises(hb.HacError) as ei:
+        hb.Format.deserialize("hac", resealed(bad))
+    assert ei.value.status == -10
+    bad = bytearray(blob); bad[128:132], bad[132:136] = blob[132:136], blob[128:132]      # codebook not ascending
+    with pytest.raises(hb.HacError) as ei:
+        hb.Format.deserialize("hac", resealed(bad))
+    assert ei.value.status == -10
