@@ -363,7 +363,7 @@ const char* hac_last_cuda_error(void);
  *   HAC_B200_ROWS=0         single-input HAC always through the kernel that keeps x in shared memory
  *   HAC_B200_ROWS_WARPS=n   warps per block of the rows-in-registers kernel (default: chosen per format)
  *   HAC_B200_ROWS_CHAINS=c  decode chains per lane of that kernel, 2 or 3 (default 2)
- *   HAC_B200_PREFETCH=0     no request of the block's share of the stream into L2 at its start
+ *   HAC_B200_PREFETCH=1     that kernel requests its block's share of the stream into L2 at its start (default off)
  *   HAC_B200_ITEMS=0        single-input sHAC always through the older kernel
  *   HAC_B200_GEMM_CLUSTER=0 batched HAC adds its row splits in a finishing kernel instead of a thread-block cluster
  *   HAC_B200_ZERO_RUNS=0    never use the zero-run table of mostly-zero HAC streams

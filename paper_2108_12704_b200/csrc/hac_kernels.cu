@@ -2468,14 +2468,15 @@ struct Tune {
     int rows_warps;     // HAC_B200_ROWS_WARPS=n: warps per block of the rows-in-registers kernel (0 = chosen by the library)
     int zero_runs;      // HAC_B200_ZERO_RUNS=0: never use the zero-run table
     int xt;             // HAC_B200_XT=0: never use the magnitude table
-    int prefetch;       // HAC_B200_PREFETCH=0: no L2 prefetch of the stream at the start of the rows-in-registers kernel
+    int prefetch;       // HAC_B200_PREFETCH=1: the rows-in-registers kernel asks for its share of the stream into L2 at its start
+                        // (measured slightly slower: the requests compete with the index entries; off by default)
     int rows_chains;    // HAC_B200_ROWS_CHAINS=2|3: decode chains per lane of that kernel (0 = chosen by the library)
     int items_kernel;   // HAC_B200_ITEMS=0: single-input sHAC always through the older kernel
     int gemm_cluster;   // HAC_B200_GEMM_CLUSTER=0: batched HAC adds its row splits in a finishing kernel, not in a cluster
 };
 static const Tune& tune() {
     static const Tune t = {env_int("HAC_B200_PDL", 1), env_int("HAC_B200_ROWS", 1), env_int("HAC_B200_ROWS_WARPS", 0),
-                           env_int("HAC_B200_ZERO_RUNS", 1), env_int("HAC_B200_XT", 1), env_int("HAC_B200_PREFETCH", 1), env_int("HAC_B200_ROWS_CHAINS", 0), env_int("HAC_B200_ITEMS", 1), env_int("HAC_B200_GEMM_CLUSTER", 1)};
+                           env_int("HAC_B200_ZERO_RUNS", 1), env_int("HAC_B200_XT", 1), env_int("HAC_B200_PREFETCH", 0), env_int("HAC_B200_ROWS_CHAINS", 0), env_int("HAC_B200_ITEMS", 1), env_int("HAC_B200_GEMM_CLUSTER", 1)};
     return t;
 }
 
@@ -2522,6 +2523,12 @@ static DevFormat dev_format_xt(const Format& f) {
 static bool table_has_long(const Format& f, const DevFormat& d) {
     return d.tab_kind ? f.tables.xt_unresolved > 0.0 : d.max_len > d.l1_bits;
 }
+// Share of the symbols whose first-level entry does not hold them.  The kernels that decode three code words
+// per window pay a call for every group with such a symbol, so they only take formats where those are rare.
+static double table_unresolved_share(const Format& f, const DevFormat& d) {
+    return d.tab_kind ? f.tables.xt_unresolved : f.tables.l1_unresolved;
+}
+constexpr double kGroupedDecodeMaxUnresolved = 1e-4;      // about 2 % of the groups of a warp (2 chains x 3 symbols x 32 lanes)
 
 static void set_pointers(Format& f, void* dev_buf, size_t bytes) {
     const ImageLayout L = image_layout(f);
@@ -2820,6 +2827,7 @@ static RowsPlan plan_rows(const Format& f, const DeviceInfo& di, int mode) {
     if ((uint64_t)f.m * 2 < (uint64_t)di.sms) return pl;
     pl.d = dev_format_xt(f);
     pl.has_long = table_has_long(f, pl.d);
+    if (table_unresolved_share(f, pl.d) > kGroupedDecodeMaxUnresolved) return pl;
     pl.grid = (unsigned)std::min<int64_t>(di.sms, f.m);
     const uint32_t max_cols = (uint32_t)((f.m + pl.grid - 1) / pl.grid);
     pl.colsum_bytes = (uint32_t)align16((size_t)max_cols * f.G * 4);
@@ -2849,6 +2857,9 @@ static RowsPlan plan_rows(const Format& f, const DeviceInfo& di, int mode) {
                 }
             }
         }
+        // more than two rounds of items per warp: the kernel with x in shared memory, which runs twice the
+        // warps, is the faster one
+        if (best_w > 0 && best_cost > 2ull * 60 && tune().rows_warps == 0) { if (repl == 4) return pl; continue; }
         if (best_w * best_c >= std::min<int>(16, (int)(f.G * 2)) || (repl == 0 && best_w > 0)) {
             pl.tp = TablePlan{};
             pl.tp.repl_log2 = (uint32_t)repl;
@@ -2904,7 +2915,7 @@ static int launch_items(const Format& f, const DeviceInfo& di, int mode, const f
     *launched = false;
     if (!f.sparse || tune().items_kernel == 0) return HAC_OK;
     const DevFormat d = dev_format_xt(f);
-    if (d.items == 0) return HAC_OK;
+    if (d.items == 0 || table_unresolved_share(f, d) > kGroupedDecodeMaxUnresolved) return HAC_OK;
     const size_t budget = (size_t)di.max_smem_optin - 256;       // static shared memory of the kernel
     const size_t xbytes = mode == 0 ? align16((size_t)f.n * 4) : 0;
     const size_t ri_stage = mode == 0 ? ((size_t)(32u * f.S * (f.ri_bits / 8) + 15u) / 16u + 1u) * 16u : 0;
