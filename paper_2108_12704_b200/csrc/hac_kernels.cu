@@ -595,17 +595,108 @@ __device__ __forceinline__ float warp_sum(float v) {
 }
 
 // ------------------------------------------------------------------------------------------------
+// Three code words from one 32-bit window.  The window holds 32 valid bits from the current position,
+// so after a code word of length l the next one starts at window << l, and a third one after that,
+// as long as the three lengths add up to at most 32; the caller checks `tot` (and `flags`, the OR of
+// the three length words, whose top bit marks an entry that does not hold its symbol) before it uses
+// the values, and otherwise decodes the three code words one at a time.  The reader is not advanced.
+// ------------------------------------------------------------------------------------------------
+template <int kTab>
+__device__ __forceinline__ void lookup3(const FastReader& r, uint32_t l1_shift, uint32_t l1_mul, uint32_t l1_lane,
+                                        uint32_t xt_low, uint32_t& v1, uint32_t& v2, uint32_t& v3, uint32_t& tot,
+                                        uint32_t& flags) {
+    if (kTab == 0) {
+        asm volatile(
+            "{\n\t"
+            ".reg .b32 t, i, a, b, c;\n\t"
+            "shf.l.wrap.b32 t, %5, %6, %7;\n\t"
+            "shr.u32 i, t, %8;\n\t"
+            "mad.lo.u32 i, i, %9, %10;\n\t"
+            "ld.shared.v2.u32 {%0, a}, [i];\n\t"
+            "shl.b32 t, t, a;\n\t"
+            "shr.u32 i, t, %8;\n\t"
+            "mad.lo.u32 i, i, %9, %10;\n\t"
+            "ld.shared.v2.u32 {%1, b}, [i];\n\t"
+            "shl.b32 t, t, b;\n\t"
+            "shr.u32 i, t, %8;\n\t"
+            "mad.lo.u32 i, i, %9, %10;\n\t"
+            "ld.shared.v2.u32 {%2, c}, [i];\n\t"
+            "add.u32 %3, a, b;\n\t"
+            "add.u32 %3, %3, c;\n\t"
+            "lop3.b32 %4, a, b, c, 0xFE;\n\t"
+            "}"
+            : "=r"(v1), "=r"(v2), "=r"(v3), "=r"(tot), "=r"(flags)
+            : "r"(r.lo), "r"(r.hi), "r"(r.off), "r"(l1_shift), "r"(l1_mul), "r"(l1_lane)
+            : "memory");
+    } else {
+        asm volatile(
+            "{\n\t"
+            ".reg .b32 t, i, a, b, c;\n\t"
+            "shf.l.wrap.b32 t, %5, %6, %7;\n\t"
+            "lop3.b32 i, t, %11, 0, 0xCF;\n\t"
+            "cvt.rz.f32.u32 i, i;\n\t"
+            "shr.u32 i, i, %8;\n\t"
+            "mad.lo.u32 i, i, %9, %10;\n\t"
+            "ld.shared.v2.u32 {%0, a}, [i];\n\t"
+            "shl.b32 t, t, a;\n\t"
+            "lop3.b32 i, t, %11, 0, 0xCF;\n\t"
+            "cvt.rz.f32.u32 i, i;\n\t"
+            "shr.u32 i, i, %8;\n\t"
+            "mad.lo.u32 i, i, %9, %10;\n\t"
+            "ld.shared.v2.u32 {%1, b}, [i];\n\t"
+            "shl.b32 t, t, b;\n\t"
+            "lop3.b32 i, t, %11, 0, 0xCF;\n\t"
+            "cvt.rz.f32.u32 i, i;\n\t"
+            "shr.u32 i, i, %8;\n\t"
+            "mad.lo.u32 i, i, %9, %10;\n\t"
+            "ld.shared.v2.u32 {%2, c}, [i];\n\t"
+            "add.u32 %3, a, b;\n\t"
+            "add.u32 %3, %3, c;\n\t"
+            "lop3.b32 %4, a, b, c, 0xFE;\n\t"
+            "}"
+            : "=r"(v1), "=r"(v2), "=r"(v3), "=r"(tot), "=r"(flags)
+            : "r"(r.lo), "r"(r.hi), "r"(r.off), "r"(l1_shift), "r"(l1_mul), "r"(l1_lane), "r"(xt_low)
+            : "memory");
+    }
+}
+
+// The three code words of lookup3 one at a time (refills in between, entries without a symbol resolved):
+// where a lane's three lengths exceed the window, or one of its entries does not hold its symbol.  Rare,
+// so it is a call, which keeps the unrolled code around it small.  `sf` is the block's copy of the format
+// descriptor in shared memory.
+struct Slow3 { uint32_t hi, lo, off, next, v0, v1, v2; };
+template <int kTab, bool kLong>
+__device__ __noinline__ Slow3 decode3_slow(uint32_t hi, uint32_t lo, uint32_t off, uint32_t next_rel, Decoder dec,
+                                           const DevFormat* sf) {
+    BitReader br;
+    br.hi = hi; br.lo = lo; br.off = off; br.next = next_rel;
+    Slow3 r;
+    r.v0 = __float_as_uint(decode_value_any<kTab, kLong>(br, dec, *sf));
+    r.v1 = __float_as_uint(decode_value_any<kTab, kLong>(br, dec, *sf));
+    r.v2 = __float_as_uint(decode_value_any<kTab, kLong>(br, dec, *sf));
+    r.hi = br.hi; r.lo = br.lo; r.off = br.off; r.next = br.next;
+    return r;
+}
+
+// Advance the reader by up to 32 bits (one refill at most).
+__device__ __forceinline__ void fast_advance(FastReader& r, uint32_t bits) { fast_consume_value(r, bits); }
+
+// ------------------------------------------------------------------------------------------------
 // HAC, one input vector (Algorithm 1 by segments).  x is staged in shared memory; a lane's rows
 // are consecutive, lanes are S rows apart, so one padding word per sub-segment (when S is even)
 // keeps the 32 lanes on distinct banks.
 //   kMode 0: product; 1: debug decode (values written to out[j*n + i]).
 // ------------------------------------------------------------------------------------------------
-template <int kMode, bool kXShared, bool kLong, int kChains, bool kRuns>
+//   kGroup: code words are decoded three to a window (lookup3), from either kind of first-level table (kTab);
+//           kGuard: three lengths can exceed the window.  Without kGroup the table is the prefix table.
+template <int kMode, bool kXShared, bool kLong, int kChains, bool kRuns, bool kGroup = false, int kTab = 0, bool kGuard = false>
 __global__ void __launch_bounds__(1024) hac_vec_kernel(DevFormat f, TablePlan tp, const float* __restrict__ x,
                                                        int64_t xs_i, float* __restrict__ y, int64_t ys_j,
                                                        float* __restrict__ aux) {
     // A warp works on kChains consecutive segments at a time (an "item"); every lane then runs
     // kChains independent decode chains, which hides the latency of the dependent table lookups.
+    __shared__ DevFormat sf;               // for the rare paths that are calls (decode3_slow)
+    if (kGroup && threadIdx.x == 0) sf = f;
     allow_dependents();
     const uint32_t warp = threadIdx.x >> 5, lane = threadIdx.x & 31, warps = blockDim.x >> 5;
     const uint32_t items = (f.units + kChains - 1) / kChains;
@@ -731,6 +822,53 @@ __global__ void __launch_bounds__(1024) hac_vec_kernel(DevFormat f, TablePlan tp
                     left -= covered;
                 }
             }
+        } else if (kMode == 0 && kXShared && kGroup) {
+            const uint32_t sb = shared_base();
+            FastReader fr[kChains];
+#pragma unroll
+            for (int c = 0; c < kChains; ++c) {
+                fr[c].hi = br[c].hi; fr[c].lo = br[c].lo; fr[c].off = br[c].off; fr[c].next = sb + br[c].next;
+            }
+            const uint32_t l1_abs = sb + dec.l1_lane - dec.bias * dec.l1_mul;
+            uint32_t s = 0;
+            for (; s + 3 <= common; s += 3) {
+                uint32_t v[kChains][3], tot[kChains], flags[kChains];
+#pragma unroll
+                for (int c = 0; c < kChains; ++c)
+                    lookup3<kTab>(fr[c], dec.l1_shift, dec.l1_mul, l1_abs, dec.xt_low, v[c][0], v[c][1], v[c][2], tot[c], flags[c]);
+                if (kGuard || kLong) {
+                    bool bad = false;
+#pragma unroll
+                    for (int c = 0; c < kChains; ++c) bad = bad || (kGuard && tot[c] > 32u) || (kLong && (int32_t)flags[c] < 0);
+                    if (__any_sync(__activemask(), bad)) {
+                        if (bad) {
+#pragma unroll
+                            for (int c = 0; c < kChains; ++c) {
+                                const Slow3 r = decode3_slow<kTab, kLong>(fr[c].hi, fr[c].lo, fr[c].off, fr[c].next - sb, dec, &sf);
+                                fr[c].hi = r.hi; fr[c].lo = r.lo; fr[c].off = r.off; fr[c].next = sb + r.next;
+                                v[c][0] = r.v0; v[c][1] = r.v1; v[c][2] = r.v2;
+                                tot[c] = 0;
+                            }
+                        }
+                    }
+                }
+#pragma unroll
+                for (int c = 0; c < kChains; ++c) {
+                    fast_advance(fr[c], tot[c]);
+#pragma unroll
+                    for (int e = 0; e < 3; ++e) acc[c] = fmaf(ldsf(xa[c] + 4 * e), __uint_as_float(v[c][e]), acc[c]);
+                    xa[c] += 12;
+                }
+            }
+#pragma unroll
+            for (int c = 0; c < kChains; ++c) {              // what is left of each chain, one code word at a time
+                br[c].hi = fr[c].hi; br[c].lo = fr[c].lo; br[c].off = fr[c].off; br[c].next = fr[c].next - sb;
+                for (uint32_t t = s; t < count[c]; ++t) {
+                    const float w = decode_value_any<kTab, kLong>(br[c], dec, f);
+                    acc[c] = fmaf(ldsf(xa[c]), w, acc[c]);
+                    xa[c] += 4;
+                }
+            }
         } else if (kMode == 0 && kXShared) {
             const uint32_t sb = shared_base();
             FastReader fr[kChains];
@@ -808,93 +946,6 @@ __global__ void __launch_bounds__(1024) hac_vec_kernel(DevFormat f, TablePlan tp
         }
     }
 }
-
-// ------------------------------------------------------------------------------------------------
-// Three code words from one 32-bit window.  The window holds 32 valid bits from the current position,
-// so after a code word of length l the next one starts at window << l, and a third one after that,
-// as long as the three lengths add up to at most 32; the caller checks `tot` (and `flags`, the OR of
-// the three length words, whose top bit marks an entry that does not hold its symbol) before it uses
-// the values, and otherwise decodes the three code words one at a time.  The reader is not advanced.
-// ------------------------------------------------------------------------------------------------
-template <int kTab>
-__device__ __forceinline__ void lookup3(const FastReader& r, uint32_t l1_shift, uint32_t l1_mul, uint32_t l1_lane,
-                                        uint32_t xt_low, uint32_t& v1, uint32_t& v2, uint32_t& v3, uint32_t& tot,
-                                        uint32_t& flags) {
-    if (kTab == 0) {
-        asm volatile(
-            "{\n\t"
-            ".reg .b32 t, i, a, b, c;\n\t"
-            "shf.l.wrap.b32 t, %5, %6, %7;\n\t"
-            "shr.u32 i, t, %8;\n\t"
-            "mad.lo.u32 i, i, %9, %10;\n\t"
-            "ld.shared.v2.u32 {%0, a}, [i];\n\t"
-            "shl.b32 t, t, a;\n\t"
-            "shr.u32 i, t, %8;\n\t"
-            "mad.lo.u32 i, i, %9, %10;\n\t"
-            "ld.shared.v2.u32 {%1, b}, [i];\n\t"
-            "shl.b32 t, t, b;\n\t"
-            "shr.u32 i, t, %8;\n\t"
-            "mad.lo.u32 i, i, %9, %10;\n\t"
-            "ld.shared.v2.u32 {%2, c}, [i];\n\t"
-            "add.u32 %3, a, b;\n\t"
-            "add.u32 %3, %3, c;\n\t"
-            "lop3.b32 %4, a, b, c, 0xFE;\n\t"
-            "}"
-            : "=r"(v1), "=r"(v2), "=r"(v3), "=r"(tot), "=r"(flags)
-            : "r"(r.lo), "r"(r.hi), "r"(r.off), "r"(l1_shift), "r"(l1_mul), "r"(l1_lane)
-            : "memory");
-    } else {
-        asm volatile(
-            "{\n\t"
-            ".reg .b32 t, i, a, b, c;\n\t"
-            "shf.l.wrap.b32 t, %5, %6, %7;\n\t"
-            "lop3.b32 i, t, %11, 0, 0xCF;\n\t"
-            "cvt.rz.f32.u32 i, i;\n\t"
-            "shr.u32 i, i, %8;\n\t"
-            "mad.lo.u32 i, i, %9, %10;\n\t"
-            "ld.shared.v2.u32 {%0, a}, [i];\n\t"
-            "shl.b32 t, t, a;\n\t"
-            "lop3.b32 i, t, %11, 0, 0xCF;\n\t"
-            "cvt.rz.f32.u32 i, i;\n\t"
-            "shr.u32 i, i, %8;\n\t"
-            "mad.lo.u32 i, i, %9, %10;\n\t"
-            "ld.shared.v2.u32 {%1, b}, [i];\n\t"
-            "shl.b32 t, t, b;\n\t"
-            "lop3.b32 i, t, %11, 0, 0xCF;\n\t"
-            "cvt.rz.f32.u32 i, i;\n\t"
-            "shr.u32 i, i, %8;\n\t"
-            "mad.lo.u32 i, i, %9, %10;\n\t"
-            "ld.shared.v2.u32 {%2, c}, [i];\n\t"
-            "add.u32 %3, a, b;\n\t"
-            "add.u32 %3, %3, c;\n\t"
-            "lop3.b32 %4, a, b, c, 0xFE;\n\t"
-            "}"
-            : "=r"(v1), "=r"(v2), "=r"(v3), "=r"(tot), "=r"(flags)
-            : "r"(r.lo), "r"(r.hi), "r"(r.off), "r"(l1_shift), "r"(l1_mul), "r"(l1_lane), "r"(xt_low)
-            : "memory");
-    }
-}
-
-// The three code words of lookup3 one at a time (refills in between, entries without a symbol resolved):
-// where a lane's three lengths exceed the window, or one of its entries does not hold its symbol.  Rare,
-// so it is a call, which keeps the unrolled code around it small.  `sf` is the block's copy of the format
-// descriptor in shared memory.
-struct Slow3 { uint32_t hi, lo, off, next, v0, v1, v2; };
-template <int kTab, bool kLong>
-__device__ __noinline__ Slow3 decode3_slow(uint32_t hi, uint32_t lo, uint32_t off, uint32_t next_rel, Decoder dec,
-                                           const DevFormat* sf) {
-    BitReader br;
-    br.hi = hi; br.lo = lo; br.off = off; br.next = next_rel;
-    Slow3 r;
-    r.v0 = __float_as_uint(decode_value_any<kTab, kLong>(br, dec, *sf));
-    r.v1 = __float_as_uint(decode_value_any<kTab, kLong>(br, dec, *sf));
-    r.v2 = __float_as_uint(decode_value_any<kTab, kLong>(br, dec, *sf));
-    r.hi = br.hi; r.lo = br.lo; r.off = br.off; r.next = br.next;
-    return r;
-}
-
-// Advance the reader by up to 32 bits (one refill at most).
-__device__ __forceinline__ void fast_advance(FastReader& r, uint32_t bits) { fast_consume_value(r, bits); }
 
 // ------------------------------------------------------------------------------------------------
 // HAC, one input vector, rows held in registers (Algorithm 1 by segments).
@@ -2472,11 +2523,13 @@ struct Tune {
                         // (measured slightly slower: the requests compete with the index entries; off by default)
     int rows_chains;    // HAC_B200_ROWS_CHAINS=2|3: decode chains per lane of that kernel (0 = chosen by the library)
     int items_kernel;   // HAC_B200_ITEMS=0: single-input sHAC always through the older kernel
+    int vec_warps;      // HAC_B200_VEC_WARPS=n: warps per block of the shared-memory-x kernels (0 = chosen by the library)
+    int vec_group;      // HAC_B200_VEC_GROUP=0: the shared-memory-x HAC kernel decodes one code word per lookup
     int gemm_cluster;   // HAC_B200_GEMM_CLUSTER=0: batched HAC adds its row splits in a finishing kernel, not in a cluster
 };
 static const Tune& tune() {
     static const Tune t = {env_int("HAC_B200_PDL", 1), env_int("HAC_B200_ROWS", 1), env_int("HAC_B200_ROWS_WARPS", 0),
-                           env_int("HAC_B200_ZERO_RUNS", 1), env_int("HAC_B200_XT", 1), env_int("HAC_B200_PREFETCH", 0), env_int("HAC_B200_ROWS_CHAINS", 0), env_int("HAC_B200_ITEMS", 1), env_int("HAC_B200_GEMM_CLUSTER", 1)};
+                           env_int("HAC_B200_ZERO_RUNS", 1), env_int("HAC_B200_XT", 1), env_int("HAC_B200_PREFETCH", 0), env_int("HAC_B200_ROWS_CHAINS", 0), env_int("HAC_B200_ITEMS", 1), env_int("HAC_B200_VEC_WARPS", 0), env_int("HAC_B200_VEC_GROUP", 1), env_int("HAC_B200_GEMM_CLUSTER", 1)};
     return t;
 }
 
@@ -2948,6 +3001,10 @@ static int launch_items(const Format& f, const DeviceInfo& di, int mode, const f
     return HAC_OK;
 }
 
+static int launch_vec_shared_x(const Format& f, const DeviceInfo& di, const DevFormat& d_plain, int mode, const float* x,
+                               int64_t xs_i, float* y, int64_t ys_j, float* aux, cudaStream_t st, bool* vec_direct,
+                               bool allow_group = true);
+
 // mode 0: product with one input; mode 1: debug decode into `aux`.
 static int launch_vec(const Format& f, int mode, const float* x, int64_t xs_i, float* y, int64_t ys_j,
                       float* aux, cudaStream_t st, bool* vec_direct = nullptr) {
@@ -2967,17 +3024,39 @@ static int launch_vec(const Format& f, int mode, const float* x, int64_t xs_i, f
         rc = launch_items(f, di, mode, x, xs_i, y, ys_j, aux, st, &launched);
         if (rc || launched) return rc;
     }
-    const size_t budget = (size_t)di.max_smem_optin;
+    return launch_vec_shared_x(f, di, d, mode, x, xs_i, y, ys_j, aux, st, vec_direct);
+}
+
+// The single-input kernels that keep x in shared memory (the general ones).
+static int launch_vec_shared_x(const Format& f, const DeviceInfo& di, const DevFormat& d_plain, int mode, const float* x,
+                               int64_t xs_i, float* y, int64_t ys_j, float* aux, cudaStream_t st, bool* vec_direct,
+                               bool allow_group) {
+    int rc = HAC_OK;
+    const size_t budget = (size_t)di.max_smem_optin - 256;   // static shared memory of the kernels
     // HAC: two decode chains per lane when two staging areas per warp fit next to a fully
     // replicated table; sHAC: one
-    const int chains = f.sparse ? 2 : (d.units > 1 ? 2 : 1);
+    const int chains = f.sparse ? 2 : (d_plain.units > 1 ? 2 : 1);
+    // HAC with a first-level table that resolves (nearly) every code word: three code words per window
+    bool group = false;
+    DevFormat d = d_plain;
+    if (allow_group && !f.sparse && mode == 0 && chains == 2 && (f.tables.l1_runs.empty() || tune().zero_runs == 0) &&
+        tune().vec_group != 0) {
+        const DevFormat dx = dev_format_xt(f);
+        if (table_unresolved_share(f, dx) <= kGroupedDecodeMaxUnresolved) { group = true; d = dx; }
+    }
     size_t per_warp = (size_t)d.max_unit_chunks * 16 * chains;
     if (f.sparse && mode == 0) per_warp += ((size_t)(32u * f.S * (f.ri_bits / 8) + 15u) / 16u + 1u) * 16u * chains;
     size_t xbytes = 0;
     if (mode == 0) xbytes = f.sparse ? align16((size_t)f.n * 4) : align16(((size_t)f.n + (f.n / f.S + 1)) * 4);
-    const int want = 32;
+    int want = 32;
     // shared memory: tables + x + per-warp staging.  Prefer keeping x and all warps; give up
-    // replicas of the level-1 table before giving up warps.
+    // replicas of the level-1 table before giving up warps (the grouped decoder, whose lookups are most of
+    // its shared-memory traffic, gives up to a quarter of the warps first).
+    if (group) {
+        for (int w = 32; w >= 24; w -= 2)
+            if (plan_smem_bytes(d.l1_entries, 4, d.sub_bytes) + xbytes + per_warp * (size_t)w <= budget) { want = w; break; }
+    }
+    if (tune().vec_warps > 0) want = std::min(32, tune().vec_warps);
     bool x_shared = mode == 0;
     const size_t min_tables = plan_smem_bytes(d.l1_entries, 0, d.sub_bytes) + 16;
     if (x_shared && xbytes + min_tables + per_warp * std::min(want, 8) > budget) { x_shared = false; xbytes = 0; }
@@ -2989,7 +3068,7 @@ static int launch_vec(const Format& f, int mode, const float* x, int64_t xs_i, f
     tp.x_bulk = (f.sparse && mode == 0 && x_shared && xs_i == 1 && (reinterpret_cast<uintptr_t>(x) & 15u) == 0) ? 1u : 0u;
     const size_t smem = fixed + plan_smem_bytes(d.l1_entries, tp.repl_log2, d.sub_bytes) + xbytes + per_warp * warps;
     if (smem > budget) return HAC_ERR_BUFFER_TOO_SMALL;
-    const bool has_long = d.max_len > d.l1_bits;
+    const bool has_long = group ? table_has_long(f, d) : d.max_len > d.l1_bits;
     const int threads = warps * 32;
     // HAC with a short code word for zero: the zero-run table replaces the level-1 table
     const bool runs = !f.sparse && mode == 0 && x_shared && !f.tables.l1_runs.empty() && tune().zero_runs != 0;
@@ -2997,6 +3076,18 @@ static int launch_vec(const Format& f, int mode, const float* x, int64_t xs_i, f
     if (runs) { dk.l1 = reinterpret_cast<const uint2*>(f.dev.l1_runs); tp.zero_len = f.tables.zero_len; }
     VecKernel kernel = has_long ? pick_vec_kernel<true>(f, mode, x_shared, chains, runs)
                                 : pick_vec_kernel<false>(f, mode, x_shared, chains, runs);
+    if (group && x_shared && !runs) {
+        const bool guard = 3u * f.max_len > 32u;
+        if (d.tab_kind)
+            kernel = has_long ? hac_vec_kernel<0, true, true, 2, false, true, 1, true>
+                              : (guard ? hac_vec_kernel<0, true, false, 2, false, true, 1, true> : hac_vec_kernel<0, true, false, 2, false, true, 1, false>);
+        else
+            kernel = has_long ? hac_vec_kernel<0, true, true, 2, false, true, 0, true>
+                              : (guard ? hac_vec_kernel<0, true, false, 2, false, true, 0, true> : hac_vec_kernel<0, true, false, 2, false, true, 0, false>);
+    } else if (group) {
+        // x does not fit in shared memory: the plain decoder, which can read it from global memory
+        return launch_vec_shared_x(f, di, d_plain, mode, x, xs_i, y, ys_j, aux, st, vec_direct, false);
+    }
     rc = prepare_kernel(kernel, smem);
     if (rc) return rc;
     int per_sm = 1;
