@@ -467,6 +467,7 @@ void finish_derived(Format& f) {
     const bool sparse = f.sparse;
     const int64_t n = f.n, m = f.m;
     const uint32_t S = f.S;
+    make_decode_tables(f);
     // per-segment statistics used to size shared memory and to pick the reduction path
     const size_t U = f.seg_bit_off.size();
     f.max_unit_chunks = 1;
@@ -517,6 +518,62 @@ void finish_derived(Format& f) {
             f.max_units_per_col = std::max(f.max_units_per_col, g);
             if (g == 0) f.has_empty_col = true;
         }
+        // Row tasks of the batched tensor-core kernel.  Every lane of that kernel keeps a private copy of its
+        // column's span of the stream and slice of ri for the task at hand, so the task length is the largest
+        // power of two (16 .. 1024 rows) for which the fullest task of any column fits 128 bytes of such buffers.
+        f.task_off.clear(); f.task_pos.clear(); f.tc_rows = 0;
+        f.max_task_chunks = 1; f.max_task_ri_chunks = 1;
+        if (f.nnz > 0) {
+            // code word length of every stored entry (canonical code: first length whose range holds the window)
+            std::vector<uint8_t> entry_len((size_t)f.nnz);
+            {
+                const DecodeTables& tb = f.tables;
+                uint64_t bit = 0;
+                for (int64_t q = 0; q < f.nnz; ++q) {
+                    const uint64_t wi = bit >> 5;
+                    const uint32_t sh = (uint32_t)(bit & 31);
+                    const uint64_t two = ((uint64_t)f.stream[wi] << 32) | f.stream[wi + 1];
+                    const uint32_t top = (uint32_t)((two << sh) >> 32);
+                    uint32_t len = f.max_len;
+                    for (uint32_t l = f.min_len; l <= f.max_len; ++l)
+                        if ((uint64_t)top < tb.limit[l]) { len = l; break; }
+                    entry_len[(size_t)q] = (uint8_t)len;
+                    bit += len;
+                }
+            }
+            const uint32_t row_bytes = f.ri_bits / 8;
+            for (uint32_t T = 1024; T >= 16; T /= 2) {
+                const uint64_t tasks = ((uint64_t)n + T - 1) / T;
+                if ((tasks + 1) * (uint64_t)m * 12 > kTaskOffBytesMax) break;      // smaller tasks only need more
+                std::vector<uint64_t> off((size_t)((tasks + 1) * (uint64_t)m), 0);
+                std::vector<uint32_t> pos((size_t)((tasks + 1) * (uint64_t)m), 0);
+                uint32_t max_s = 1, max_r = 1;
+                uint64_t bit = 0;
+                for (int64_t j = 0; j < m; ++j) {
+                    uint64_t t = 0;                       // next task whose start has not been recorded yet
+                    auto record = [&](uint32_t p) { off[(size_t)t * m + j] = bit; pos[(size_t)t * m + j] = p; ++t; };
+                    for (uint32_t q = f.cb[j]; q < f.cb[j + 1]; ++q) {
+                        const uint64_t row = f.ri_bits == 16 ? f.ri16[q] : f.ri32[q];
+                        while (t <= tasks && t * T <= row) record(q);
+                        bit += entry_len[q];
+                    }
+                    while (t <= tasks) record(f.cb[j + 1]);
+                    for (uint64_t tt = 0; tt < tasks; ++tt) {
+                        const uint64_t b0 = off[(size_t)tt * m + j], b1 = off[(size_t)(tt + 1) * m + j];
+                        const uint64_t last_word = (b1 >> 5) + 2;
+                        max_s = std::max<uint32_t>(max_s, (uint32_t)((last_word >> 2) - (b0 >> 7) + 1));
+                        const uint64_t p0 = (uint64_t)pos[(size_t)tt * m + j] * row_bytes;
+                        const uint64_t p1 = (uint64_t)pos[(size_t)(tt + 1) * m + j] * row_bytes;
+                        max_r = std::max<uint32_t>(max_r, (uint32_t)(((p1 + 15) >> 4) - (p0 >> 4) + 1));
+                    }
+                }
+                if (max_s + max_r <= 8 || T == 16) {
+                    f.tc_rows = T; f.task_off.swap(off); f.task_pos.swap(pos);
+                    f.max_task_chunks = max_s; f.max_task_ri_chunks = max_r;
+                    break;
+                }
+            }
+        }
     } else {
         f.max_units_per_col = f.G;
         const uint64_t tasks = ((uint64_t)n + S - 1) / S;
@@ -537,7 +594,6 @@ void finish_derived(Format& f) {
             }
         }
     }
-    make_decode_tables(f);
 }
 
 int build_impl(const float* W, int64_t n, int64_t m, int64_t ldw, const hac_build_params* p,
@@ -811,6 +867,7 @@ ImageLayout image_layout(const Format& f) {
     L.cb = take(f.cb.size() * 4);
     L.unit_info = take(f.item_info.size() * 4);
     L.task_off = take(f.task_off.size() * 8);
+    L.task_pos = take(f.task_pos.size() * 4);
     L.total = o;
     return L;
 }

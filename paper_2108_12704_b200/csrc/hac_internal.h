@@ -95,6 +95,7 @@ struct DeviceImage {
     const uint32_t* cb = nullptr;
     const void* unit_info = nullptr;
     const uint64_t* task_off = nullptr;
+    const uint32_t* task_pos = nullptr;
 };
 
 struct Format {
@@ -127,6 +128,15 @@ struct Format {
     // holds the columns' ends), for the batched kernel, whose lanes are columns.  Left empty, and then
     // derived from the offset index on every call, when it would exceed kTaskOffBytesMax.
     std::vector<uint64_t> task_off;
+    // sHAC, device only, for the batched tensor-core kernel: the rows are cut into tasks of tc_rows rows (a
+    // power of two chosen so that a task of a column holds a few dozen stored entries); task_off[t][j] is
+    // the bit where the first entry of column j with row >= t * tc_rows starts and task_pos[t][j] its
+    // position in nz / ri ([tasks + 1][m]; the last row holds the columns' ends).  Empty (no tensor-core
+    // path) when the tables would exceed kTaskOffBytesMax.
+    std::vector<uint32_t> task_pos;
+    uint32_t tc_rows = 0;
+    uint32_t max_task_chunks = 1;             // largest 16-byte span of the stream a task of a column covers
+    uint32_t max_task_ri_chunks = 1;          // the same for its slice of ri
     uint32_t max_unit_chunks = 0;             // largest 16-byte span a segment's stream covers
     uint32_t max_sub_chunks = 0;              // same for a single sub-segment
     uint32_t max_units_per_col = 0;
@@ -149,7 +159,7 @@ void fill_size_report(const Format& f, hac_size_report* r);
 // device image layout: offsets of every section (256-byte aligned), total size
 struct ImageLayout {
     size_t stream, lut, l1, sub, l1_runs, xt, rank_value, limit, first_left, rank_base, seg_bit_off, sub_bits, seg_col,
-        seg_first, ri, cb, unit_info, task_off, total;
+        seg_first, ri, cb, unit_info, task_off, task_pos, total;
 };
 ImageLayout image_layout(const Format& f);
 

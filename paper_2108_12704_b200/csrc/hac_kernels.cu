@@ -2016,12 +2016,17 @@ __global__ void __launch_bounds__(256) hac_pack_x_kernel(DevFormat f, const floa
 // (tcgen05.commit once the MMAs that read the stage have finished).  The X tile of chunk k + 1 shares
 // its buffer with chunk k - 1 and is requested once that chunk's MMAs have been committed.
 // Every wait is bounded; if one runs out the block marks its outputs NaN and still terminates.
-template <int kTab, bool kLong>
+// kSp = 0: HAC (a task is a sub-segment: f.S consecutive rows, one code word per row).  kSp = 2 or 4: sHAC with
+// row indices of that many bytes: a task is f.S consecutive rows as well (the caller passes the row-task length
+// there), but a column stores code words only for some of them: task_off / task_pos give where the first entry at
+// or after the task's first row starts in the stream and in ri, the lane copies that slice of ri next to its span
+// of the stream, and a row without an entry contributes a zero to the tile.
+template <int kTab, bool kLong, int kSp>
 __global__ void __launch_bounds__(kGWarps * 32, 1) hac_gemm_tc_kernel(
     DevFormat f, TablePlan tp, const unsigned char* __restrict__ xpack, uint32_t batch, float* __restrict__ y,
     int64_t ys_j, int64_t ys_b, float* __restrict__ partial, const uint64_t* __restrict__ task_off,
     uint32_t col_blocks, uint32_t row_splits, uint32_t max_rounds, uint32_t slot_bytes, uint32_t nbuf,
-    uint32_t cluster_reduce) {
+    uint32_t cluster_reduce, const uint32_t* __restrict__ task_pos, uint32_t rslot_bytes) {
     allow_dependents();
     const uint32_t warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     // the row splits of a column block are consecutive blocks (one thread-block cluster when cluster_reduce is set)
@@ -2057,13 +2062,21 @@ __global__ void __launch_bounds__(kGWarps * 32, 1) hac_gemm_tc_kernel(
     const uint32_t rounds = warp < kGDecodeWarps ? gemm_slot_rounds(ntl, dslot) : 0u;
     // first 16-byte chunk of the stream that holds a sub-segment, and (chunks it spans << 7) | bit
     // position of its first code word inside the first chunk
-    struct Loc { uint32_t chunk, span; };
+    struct Loc { uint32_t chunk, span, rchunk, rspan, entries; };
     auto locate = [&](uint32_t pr, Loc (&loc)[kGChains]) {
 #pragma unroll
         for (int c = 0; c < kGChains; ++c) {
-            loc[c].chunk = 0; loc[c].span = 0;
+            loc[c].chunk = 0; loc[c].span = 0; loc[c].rchunk = 0; loc[c].rspan = 0; loc[c].entries = 0;
             const uint32_t tl = (pr * kGChains + c) * kGSlots + dslot;
             if (!dvalid || pr >= rounds || tl >= ntl) continue;
+            if (kSp) {
+                const uint32_t* pa = task_pos + (size_t)(t_begin + tl) * f.m + dj;
+                const uint32_t p0 = __ldg(pa), p1 = __ldg(pa + f.m);
+                const uint64_t byte0 = (uint64_t)p0 * kSp, byte1 = (uint64_t)p1 * kSp;
+                loc[c].entries = p1 - p0;
+                loc[c].rchunk = (uint32_t)(byte0 >> 4);
+                loc[c].rspan = (p1 > p0 ? (uint32_t)(((byte1 + 15) >> 4) - (byte0 >> 4)) << 7 : 0u) | (uint32_t)(byte0 & 15u);
+            }
             const uint64_t* at = task_off + (size_t)(t_begin + tl) * f.m + dj;
             const uint64_t start = __ldg(at);
             const uint32_t mine = (uint32_t)(__ldg(at + f.m) - start);
@@ -2139,8 +2152,11 @@ __global__ void __launch_bounds__(kGWarps * 32, 1) hac_gemm_tc_kernel(
         const bool valid = dvalid;
         const bool all_valid = __all_sync(0xffffffffu, valid);
         const uint32_t buf_stride = 32 * slot_bytes;
-        // this lane's buffers: [parity][chain], buf_stride apart
+        // this lane's buffers: [parity][chain], buf_stride apart; the slices of ri (sHAC) lie behind all of them
         const uint32_t my_buf = spans + warp * nbuf * kGChains * buf_stride + lane * slot_bytes;
+        const uint32_t rbuf_stride = 32 * rslot_bytes;
+        const uint32_t my_rbuf = spans + kGDecodeWarps * nbuf * kGChains * buf_stride + warp * nbuf * kGChains * rbuf_stride +
+                                 lane * rslot_bytes;
         const uint32_t l1_abs = sb + dec.l1_lane - dec.bias * dec.l1_mul;
         const uint32_t a_base = tmem + ((q * 32u) << 16) + kGDCols + slot * kGStages * kGACols;
         const uint32_t full0 = bar_full + 8 * slot * kGStages, empty0 = bar_empty + 8 * slot * kGStages;
@@ -2152,6 +2168,11 @@ __global__ void __launch_bounds__(kGWarps * 32, 1) hac_gemm_tc_kernel(
                 const uint4* src = stream4 + loc[c].chunk;
                 const uint32_t dst = sb + my_buf + (par * kGChains + c) * buf_stride, nch = loc[c].span >> 7;
                 for (uint32_t i = 0; i < nch; ++i) cp_async16(dst + 16 * i, src + i);
+                if (kSp) {
+                    const uint4* rsrc = reinterpret_cast<const uint4*>(f.ri) + loc[c].rchunk;
+                    const uint32_t rdst = sb + my_rbuf + (par * kGChains + c) * rbuf_stride, rn = loc[c].rspan >> 7;
+                    for (uint32_t i = 0; i < rn; ++i) cp_async16(rdst + 16 * i, rsrc + i);
+                }
             }
             asm volatile("cp.async.commit_group;" ::: "memory");
         };
@@ -2174,6 +2195,7 @@ __global__ void __launch_bounds__(kGWarps * 32, 1) hac_gemm_tc_kernel(
             for (int c = 0; c < kGChains; ++c) bitpos[c] = loc_cur[c].span & 127u;
             FastReader fr[kGChains];
             uint32_t cnt[kGChains];
+            uint32_t left[kGChains], nrow[kGChains], rp[kGChains], rowbase[kGChains];    // sHAC: entries left, row of the next, where it is read
             uint32_t full_rows = f.S;                 // rows every chain of the round has
 #pragma unroll
             for (int c = 0; c < kGChains; ++c) {
@@ -2181,6 +2203,12 @@ __global__ void __launch_bounds__(kGWarps * 32, 1) hac_gemm_tc_kernel(
                 cnt[c] = tl < ntl ? (uint32_t)min((uint64_t)f.S, (uint64_t)f.n - (uint64_t)(t_begin + tl) * f.S) : 0u;
                 full_rows = min(full_rows, cnt[c]);
                 fr[c].hi = fr[c].lo = fr[c].off = 0; fr[c].next = sb + my_buf;
+                left[c] = 0; nrow[c] = 0xffffffffu; rp[c] = 0; rowbase[c] = (t_begin + tl) * f.S;
+                if (kSp && valid && cnt[c] > 0 && loc_cur[c].entries > 0) {
+                    left[c] = loc_cur[c].entries;
+                    rp[c] = my_rbuf + (par * kGChains + c) * rbuf_stride + (loc_cur[c].rspan & 127u);
+                    nrow[c] = kSp == 2 ? lds16(rp[c]) : lds32(rp[c]);
+                }
                 if (valid && cnt[c] > 0) {
                     BitReader br;
                     br.init(my_buf + (par * kGChains + c) * buf_stride, bitpos[c]);
@@ -2190,7 +2218,27 @@ __global__ void __launch_bounds__(kGWarps * 32, 1) hac_gemm_tc_kernel(
             for (uint32_t r = 0; r < cpr * kGChainRows; r += kGChainRows, ++k) {
                 uint32_t hi[kGRows], lo[kGRows];
                 // the table entries are {lo, hi | length}: the symbol is ready for the tensor core as it is
-                if (all_valid && r + kGChainRows <= full_rows) {
+                if (kSp) {
+                    // sHAC: a row of the tile is the column's next stored entry if that entry lies in this row, else zero
+                    // (a variant that looks every row up and only selects was measured: 4 % faster at 60 % zeros, 16 %
+                    // slower at 96 %)
+#pragma unroll
+                    for (int s = 0; s < kGChainRows; ++s) {
+#pragma unroll
+                        for (int c = 0; c < kGChains; ++c) {
+                            uint32_t top = 0, wl = 0, wh = 0;
+                            if (nrow[c] == rowbase[c] + r + s) {
+                                table_lookup<kTab>(fr[c], dec.l1_shift, dec.l1_mul, l1_abs, dec.xt_low, top, wl, wh);
+                                if (kLong && (wh & kSplitLong)) resolve_split_any<kTab>(top, dec, f, wl, wh);
+                                fast_consume_value(fr[c], wh & 63u);
+                                rp[c] += kSp;
+                                nrow[c] = --left[c] ? (kSp == 2 ? lds16(rp[c]) : lds32(rp[c])) : 0xffffffffu;
+                            }
+                            hi[c * kGChainRows + s] = wh & 0xffffe000u;
+                            lo[c * kGChainRows + s] = wl;
+                        }
+                    }
+                } else if (all_valid && r + kGChainRows <= full_rows) {
                     // code words in groups of three (and a last group of two) per window
                     auto one_by_one = [&](int c, int s0, int cntg) {
                         for (int s = s0; s < s0 + cntg; ++s) {
@@ -2523,13 +2571,14 @@ struct Tune {
                         // (measured slightly slower: the requests compete with the index entries; off by default)
     int rows_chains;    // HAC_B200_ROWS_CHAINS=2|3: decode chains per lane of that kernel (0 = chosen by the library)
     int items_kernel;   // HAC_B200_ITEMS=0: single-input sHAC always through the older kernel
+    int shac_tc;        // HAC_B200_SHAC_TC=0: batched sHAC never on the tensor cores; 2: always (1 = chosen by estimated cost)
     int vec_warps;      // HAC_B200_VEC_WARPS=n: warps per block of the shared-memory-x kernels (0 = chosen by the library)
     int vec_group;      // HAC_B200_VEC_GROUP=0: the shared-memory-x HAC kernel decodes one code word per lookup
     int gemm_cluster;   // HAC_B200_GEMM_CLUSTER=0: batched HAC adds its row splits in a finishing kernel, not in a cluster
 };
 static const Tune& tune() {
     static const Tune t = {env_int("HAC_B200_PDL", 1), env_int("HAC_B200_ROWS", 1), env_int("HAC_B200_ROWS_WARPS", 0),
-                           env_int("HAC_B200_ZERO_RUNS", 1), env_int("HAC_B200_XT", 1), env_int("HAC_B200_PREFETCH", 0), env_int("HAC_B200_ROWS_CHAINS", 0), env_int("HAC_B200_ITEMS", 1), env_int("HAC_B200_VEC_WARPS", 0), env_int("HAC_B200_VEC_GROUP", 1), env_int("HAC_B200_GEMM_CLUSTER", 1)};
+                           env_int("HAC_B200_ZERO_RUNS", 1), env_int("HAC_B200_XT", 1), env_int("HAC_B200_PREFETCH", 0), env_int("HAC_B200_ROWS_CHAINS", 0), env_int("HAC_B200_ITEMS", 1), env_int("HAC_B200_SHAC_TC", 1), env_int("HAC_B200_VEC_WARPS", 0), env_int("HAC_B200_VEC_GROUP", 1), env_int("HAC_B200_GEMM_CLUSTER", 1)};
     return t;
 }
 
@@ -2605,6 +2654,7 @@ static void set_pointers(Format& f, void* dev_buf, size_t bytes) {
     f.dev.cb = reinterpret_cast<const uint32_t*>(b + L.cb);
     f.dev.unit_info = b + L.unit_info;
     f.dev.task_off = reinterpret_cast<const uint64_t*>(b + L.task_off);
+    f.dev.task_pos = reinterpret_cast<const uint32_t*>(b + L.task_pos);
 }
 
 static int upload(Format& f, void* dev_buf, size_t dev_bytes, void* stream_) {
@@ -2637,6 +2687,7 @@ static int upload(Format& f, void* dev_buf, size_t dev_bytes, void* stream_) {
     HAC_CUDA(put(L.cb, f.cb.data(), f.cb.size() * 4));
     HAC_CUDA(put(L.unit_info, f.item_info.data(), f.item_info.size() * 4));
     HAC_CUDA(put(L.task_off, f.task_off.data(), f.task_off.size() * 8));
+    HAC_CUDA(put(L.task_pos, f.task_pos.data(), f.task_pos.size() * 4));
     // the source vectors are pageable host memory: wait so they may change or go away afterwards
     HAC_CUDA(cudaStreamSynchronize(st));
     set_pointers(f, dev_buf, dev_bytes);
@@ -2650,8 +2701,22 @@ static int attach(Format& f, void* dev_buf, size_t dev_bytes) {
     return HAC_OK;
 }
 
-// Tasks of the batched HAC kernel: sub-segments (S rows) of a column.
-static uint32_t gemm_tasks(const Format& f) { return f.S ? (uint32_t)((f.n + f.S - 1) / f.S) : 0u; }
+// Tasks of the tensor-core kernel: runs of consecutive rows of a column (HAC: a sub-segment, S rows; sHAC:
+// tc_rows rows, see Format::task_pos).
+static uint32_t gemm_task_rows(const Format& f) { return f.sparse ? f.tc_rows : f.S; }
+static uint32_t gemm_tasks(const Format& f) {
+    const uint32_t t = gemm_task_rows(f);
+    return t ? (uint32_t)((f.n + t - 1) / t) : 0u;
+}
+// Whether a batched sHAC product goes to the tensor-core kernel (zero-filled tiles) rather than to the kernel
+// that gathers rows of X: the first costs the dense product, the second nnz * batch * 4 bytes from L2.
+static bool shac_tc_wanted(const Format& f, int64_t batch) {
+    if (!f.sparse || batch < 2 || f.task_pos.empty() || tune().shac_tc == 0) return false;
+    const double tiles = (double)((batch + kGBatch - 1) / kGBatch);
+    const double dense_s = (double)f.n * (double)f.m * tiles * kGBatch * 6.0 / 200e12;
+    const double gather_s = (double)f.nnz * (double)batch * 4.0 / 5e12;
+    return tune().shac_tc == 2 || dense_s < gather_s;
+}
 
 // Whether the single-input sHAC kernel can hold the format: it stages two segments' spans and slices of
 // ri per warp, which a very large S with 32-bit row indices can push past the shared memory of an SM
@@ -2662,15 +2727,17 @@ static bool shac_vec_fits(const Format& f) {
 }
 
 static size_t partial_bytes(const Format& f, int64_t batch) {
-    // batched HAC: one partial per row split of the product kernel
-    if (!f.sparse && batch > 1) {
+    // tensor-core kernel: one partial per row split of the product kernel
+    size_t tc = 0;
+    if (batch > 1 && (!f.sparse || shac_tc_wanted(f, batch))) {
         const uint32_t t = gemm_tasks(f);
-        return t > 1 ? (size_t)std::min<uint32_t>(t, kGMaxSplits) * (size_t)f.m * (size_t)batch * 4 : 0;
+        tc = t > 1 ? (size_t)std::min<uint32_t>(t, kGMaxSplits) * (size_t)f.m * (size_t)batch * 4 : 0;
+        if (!f.sparse) return tc;
     }
     // sHAC with one input handles up to two segments of a column in one warp; the batched sHAC kernel
     // and HAC with one input keep one partial per segment
     const bool partials = f.sparse ? f.max_units_per_col > ((batch == 1 && shac_vec_fits(f)) ? 2u : 1u) : f.G > 1;
-    return partials ? f.seg_bit_off.size() * (size_t)batch * 4 : 0;
+    return std::max(tc, partials ? f.seg_bit_off.size() * (size_t)batch * 4 : (size_t)0);
 }
 
 // Row splits of the tensor-core HAC kernel: 1 (a block owns whole columns and writes y itself)
@@ -2693,8 +2760,8 @@ static uint32_t gemm_max_rounds(const Format& f, uint32_t row_splits) {
     return (max_ntl + kGChains * kGSlots - 1) / (kGChains * kGSlots);
 }
 static size_t xpack_bytes(const Format& f, int64_t batch) {
-    if (f.sparse || batch <= 1 || f.symbols == 0) return 0;
-    const size_t cpr = (f.S + kGChainRows - 1) / kGChainRows;
+    if (batch <= 1 || f.symbols == 0 || (f.sparse && !shac_tc_wanted(f, batch))) return 0;
+    const size_t cpr = (gemm_task_rows(f) + kGChainRows - 1) / kGChainRows;
     size_t tiles = 0;
     DeviceInfo di;
     if (device_info(di) == HAC_OK) {
@@ -3108,12 +3175,20 @@ static int launch_vec_shared_x(const Format& f, const DeviceInfo& di, const DevF
 static int launch_gemm_tc(const Format& f, const DeviceInfo& di, const DevFormat&, const float* x, int64_t xs_i,
                           int64_t xs_b, int64_t batch, float* y, int64_t ys_j, int64_t ys_b, float* partial,
                           unsigned char* xpack, cudaStream_t st, uint32_t* row_splits_out) {
-    const DevFormat d = dev_format_xt(f);
+    DevFormat d = dev_format_xt(f);
     const bool has_long = table_has_long(f, d);
-    auto kernel = d.tab_kind ? (has_long ? hac_gemm_tc_kernel<1, true> : hac_gemm_tc_kernel<1, false>)
-                             : (has_long ? hac_gemm_tc_kernel<0, true> : hac_gemm_tc_kernel<0, false>);
+    const int sp = f.sparse ? (int)(f.ri_bits / 8) : 0;
+    if (f.sparse) d.S = f.tc_rows;               // the kernels' task length
+    auto pick = [&](auto tab, auto lng) {
+        constexpr int kTab = decltype(tab)::value;
+        constexpr bool kLng = decltype(lng)::value;
+        return sp == 0 ? hac_gemm_tc_kernel<kTab, kLng, 0> : (sp == 2 ? hac_gemm_tc_kernel<kTab, kLng, 2> : hac_gemm_tc_kernel<kTab, kLng, 4>);
+    };
+    auto kernel = d.tab_kind ? (has_long ? pick(std::integral_constant<int, 1>(), std::true_type()) : pick(std::integral_constant<int, 1>(), std::false_type()))
+                             : (has_long ? pick(std::integral_constant<int, 0>(), std::true_type()) : pick(std::integral_constant<int, 0>(), std::false_type()));
     const size_t budget = (size_t)di.max_smem_optin;
-    const uint32_t slot_bytes = d.max_sub_chunks * 16;
+    const uint32_t slot_bytes = (f.sparse ? f.max_task_chunks : d.max_sub_chunks) * 16;
+    const uint32_t rslot_bytes = f.sparse ? f.max_task_ri_chunks * 16 : 0;
     // shared memory: double stream buffers if they still leave room for a level-1 table with 8 replicas,
     // else single ones with the widest table that fits
     uint32_t nbuf = 0;
@@ -3123,7 +3198,7 @@ static int launch_gemm_tc(const Format& f, const DeviceInfo& di, const DevFormat
             // the stream buffers double as the epilogue's four 32 x 33 transpose tiles
             // the stream buffers double as the epilogue's tiles (four 32 x 33 transposes, or the 128 x 65 sums)
             const size_t fx = 256 + 128 + (size_t)kGSlots * kGStages * kGXTileBytes +
-                              std::max<size_t>((size_t)kGDecodeWarps * nb * kGChains * 32 * slot_bytes,
+                              std::max<size_t>((size_t)kGDecodeWarps * nb * kGChains * 32 * (slot_bytes + rslot_bytes),
                                                (size_t)kGCols * (kGBatch + 1) * 4);
             if (fx + plan_smem_bytes(d.l1_entries, want_repl, d.sub_bytes) <= budget) { nbuf = nb; fixed = fx; break; }
         }
@@ -3145,6 +3220,7 @@ static int launch_gemm_tc(const Format& f, const DeviceInfo& di, const DevFormat
     const uint64_t pack_blocks = (uint64_t)batch_tiles * rs * kGSlots * max_rounds * cpr;
     if (pack_blocks > 0x7fffffffull) return HAC_ERR_OFFSET_OVERFLOW;
     // the B tiles are a multiple of 8 bytes, so the start bits that follow them are aligned
+    if (f.sparse && f.task_off.empty()) return HAC_ERR_BUFFER_TOO_SMALL;
     const bool cached_off = !f.task_off.empty();
     uint64_t* task_off = cached_off ? const_cast<uint64_t*>(f.dev.task_off)
                                     : reinterpret_cast<uint64_t*>(xpack + xpack_bytes(f, batch));
@@ -3160,14 +3236,15 @@ static int launch_gemm_tc(const Format& f, const DeviceInfo& di, const DevFormat
     if (rs > 1 && tune().gemm_cluster != 0) {
         const cudaError_t ce = launch_dependent_cluster(kernel, dim3((unsigned)grid), dim3(kGWarps * 32), smem, st, rs, d, tp,
                                                         (const unsigned char*)xpack, (uint32_t)batch, y, ys_j, ys_b, partial,
-                                                        (const uint64_t*)task_off, col_blocks, rs, max_rounds, slot_bytes, nbuf, 1u);
+                                                        (const uint64_t*)task_off, col_blocks, rs, max_rounds, slot_bytes, nbuf, 1u,
+                                                        f.dev.task_pos, rslot_bytes);
         if (ce == cudaSuccess) clustered = true;
         else (void)cudaGetLastError();
     }
     if (!clustered) {
         rc = launch_dependent(kernel, dim3((unsigned)grid), dim3(kGWarps * 32), smem, st, d, tp,
                               (const unsigned char*)xpack, (uint32_t)batch, y, ys_j, ys_b, partial, (const uint64_t*)task_off,
-                              col_blocks, rs, max_rounds, slot_bytes, nbuf, 0u);
+                              col_blocks, rs, max_rounds, slot_bytes, nbuf, 0u, f.dev.task_pos, rslot_bytes);
         if (rc) return rc;
     }
     f.last_launches++;
@@ -3229,6 +3306,7 @@ static int dot(const Format& f, const float* x, int64_t batch, int64_t xs_i, int
     bool direct = false;                     // the product kernel wrote every output itself
     uint32_t gemm_splits = 0;                // batched HAC: row splits used (1 = outputs written directly)
     bool wide_single = false;                // sHAC, one input, through the batched kernel (see shac_vec_fits)
+    bool shac_tc = false;                    // sHAC batch through the tensor-core kernel
     if (d.units > 0) {
         if (batch == 1 && (!f.sparse || shac_vec_fits(f))) {
             rc = launch_vec(f, 0, x, xs_i, y, ys_j, partial, st, &direct);
@@ -3256,6 +3334,14 @@ static int dot(const Format& f, const float* x, int64_t batch, int64_t xs_i, int
                             rc = launch_finalize(f, d, partial, 1, y + b * ys_b, ys_j, 0, st, 1);
                     }
                 }
+            } else if (shac_tc_wanted(f, batch) && [&]() {
+                           // moderately sparse, or a large batch: the tensor-core kernel with zero-filled tiles
+                           unsigned char* xpack = static_cast<unsigned char*>(workspace) + ((partial_bytes(f, batch) + 255) & ~(size_t)255);
+                           rc = launch_gemm_tc(f, di, d, x, xs_i, xs_b, batch, y, ys_j, ys_b, partial, xpack, st, &gemm_splits);
+                           if (rc == HAC_ERR_BUFFER_TOO_SMALL) { rc = HAC_OK; gemm_splits = 0; return false; }
+                           shac_tc = true;
+                           return true;
+                       }()) {
             } else {
                 const int acc = (int)std::min<int64_t>(kAccMax, (batch + 31) / 32);
                 switch (acc) {
@@ -3272,7 +3358,7 @@ static int dot(const Format& f, const float* x, int64_t batch, int64_t xs_i, int
     uint32_t direct_up_to = 1;
     bool finish;
     DevFormat dfin = d;
-    if (!f.sparse && batch > 1) {
+    if ((!f.sparse && batch > 1) || shac_tc) {
         if (gemm_splits > 1) {               // partial[split][b][j]
             dim3 grid((unsigned)((f.m + 31) / 32), (unsigned)((batch + 31) / 32));
             // launched the ordinary way: started early, its blocks only took the idle SMs from the product
