@@ -224,11 +224,15 @@ int shac_attach(shac_format* f, void* dev_buf, size_t dev_bytes);
  * fly; the uncompressed weights are never written to global memory.  Products and sums are fp32.
  *   workspace  device scratch of at least *_workspace_bytes(f, batch) bytes, 16-byte aligned (may be
  *              NULL when that is 0).  It holds partial sums of columns that span several segments
- *              and, for a batched HAC product, the inputs split into two TF32 parts and arranged
- *              in the tiles the tensor-core kernel reads, plus the start bit of every sub-segment
- *              of every column (rebuilt from the offset index on each call); its contents need not
- *              be initialised and are undefined afterwards.  Two dot calls that run concurrently
- *              must not share it.
+ *              and, for a batched product on the tensor cores (HAC always; sHAC when that is estimated
+ *              to be faster than gathering rows of X), the inputs split into two TF32 parts and
+ *              arranged in the tiles that kernel reads (for very large HAC matrices also the start bit
+ *              of every sub-segment of every column, which is otherwise kept in the device image); its
+ *              contents need not be initialised and are undefined afterwards.  Two dot calls that run
+ *              concurrently must not share it.
+ *   results    A batched product on the tensor cores rounds every weight and input to two TF32 parts
+ *              (three partial products, error about 1e-7 of sum |w x|).  If a bounded wait inside
+ *              that kernel ever ran out (it never has), the outputs of the affected block are NaN.
  * Asynchronous on cuda_stream.  The kernels are launched with programmatic stream serialization:
  * they may begin fetching the uploaded format while the kernel before them in the stream is still
  * finishing, but read x and the workspace and write y only once that kernel has completed, so the
@@ -364,7 +368,10 @@ const char* hac_last_cuda_error(void);
  *   HAC_B200_ROWS_WARPS=n   warps per block of the rows-in-registers kernel (default: chosen per format)
  *   HAC_B200_ROWS_CHAINS=c  decode chains per lane of that kernel, 2 or 3 (default 2)
  *   HAC_B200_PREFETCH=1     that kernel requests its block's share of the stream into L2 at its start (default off)
+ *   HAC_B200_VEC_GROUP=0    the kernel that keeps x in shared memory decodes one code word per table lookup
+ *   HAC_B200_VEC_WARPS=n    warps per block of the kernels that keep x in shared memory (default: as many as fit)
  *   HAC_B200_ITEMS=0        single-input sHAC always through the older kernel
+ *   HAC_B200_SHAC_TC=0|2    batched sHAC never / always on the tensor cores (default 1: by estimated cost)
  *   HAC_B200_GEMM_CLUSTER=0 batched HAC adds its row splits in a finishing kernel instead of a thread-block cluster
  *   HAC_B200_ZERO_RUNS=0    never use the zero-run table of mostly-zero HAC streams
  *   HAC_B200_XT=0           never use the magnitude-indexed first-level table */
