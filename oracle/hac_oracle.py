@@ -675,3 +675,62 @@ def chain_definition(layers, X: np.ndarray):
         outs.append((y, a))
         cur = y.astype(np.float32)
     return outs
+
+
+# ----------------------------------------------------------------------------
+# Sect. III-C.1 / IV-A  the formats HAC and sHAC are compared with (Sect. V, comparison of the formats):
+# the index map and plain CSC
+# ----------------------------------------------------------------------------
+def index_map_encode(Wq: np.ndarray) -> dict:
+    """Index map of Sect. III-C.1: the distinct values of Wq (zero included when it occurs) in a vector c,
+    ascending, and the matrix Pi of pointers into it, pi_ij = position of Wq[i, j] in c, stored with
+    b_bar = 8 bits when there are at most 256 values, else 16 (the paper's example), else 32."""
+    Wq = _c32(Wq)
+    c, inverse = np.unique(Wq, return_inverse=True)
+    k = len(c)
+    b_bar = 8 if k <= 256 else (16 if k <= 65536 else 32)
+    dtype = {8: np.uint8, 16: np.uint16, 32: np.uint32}[b_bar]
+    return {"n": Wq.shape[0], "m": Wq.shape[1], "codebook": c.astype(np.float32),
+            "index": inverse.reshape(Wq.shape).astype(dtype), "b_bar": b_bar}
+
+
+def index_map_bits(fmt: dict) -> int:
+    """Size as the paper counts it: b_bar * n * m + k * b."""
+    return fmt["b_bar"] * fmt["n"] * fmt["m"] + len(fmt["codebook"]) * B_WORD
+
+
+def index_map_decode(fmt: dict) -> np.ndarray:
+    return fmt["codebook"][fmt["index"].astype(np.int64)]
+
+
+def dot_index_map(fmt: dict, X: np.ndarray):
+    """x^T W with every weight fetched through its pointer, fp64, rows ascending; (y, a) as dot_definition."""
+    X = np.atleast_2d(_c32(X)).astype(np.float64)
+    n, m = fmt["n"], fmt["m"]
+    c = fmt["codebook"].astype(np.float64)
+    y = np.zeros((X.shape[0], m)); a = np.zeros((X.shape[0], m))
+    idx = fmt["index"]
+    for i in range(n):
+        w = c[idx[i].astype(np.int64)]                  # row i of W through the map
+        t = X[:, i:i + 1] * w[None, :]
+        y += t; a += np.abs(t)
+    return y, a
+
+
+def csc_bits(nz, ri, cb) -> int:
+    """Size of CSC as the paper counts it: (2 q + m + 1) b."""
+    return (2 * len(nz) + len(cb)) * B_WORD
+
+
+def dot_csc(nz, ri, cb, n: int, X: np.ndarray):
+    """x^T W from the CSC vectors (Sect. IV-A): out[j] = sum over the stored entries p of column j of
+    nz[p] * x[ri[p]], fp64, in storage order; (y, a) as dot_definition."""
+    X = np.atleast_2d(_c32(X)).astype(np.float64)
+    m = len(cb) - 1
+    y = np.zeros((X.shape[0], m)); a = np.zeros((X.shape[0], m))
+    nz64 = np.asarray(nz, dtype=np.float64)
+    for j in range(m):
+        for p in range(int(cb[j]), int(cb[j + 1])):
+            t = X[:, int(ri[p])] * nz64[p]
+            y[:, j] += t; a[:, j] += np.abs(t)
+    return y, a

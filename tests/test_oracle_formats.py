@@ -183,3 +183,51 @@ def test_crossover_formula_consistent_with_bounds():
         shac_b = orc.cor2_bound_bits(n, m, q, k) - 6 * k * 32
         hac_b = orc.cor1_bound_bits(n, m, k) - 6 * k * 32
         assert (shac_b < hac_b) == (s < s_star)
+
+
+# ---------------------------------------------------------------- index map and plain CSC (the comparison formats)
+def test_index_map_on_the_papers_example_and_its_occupancy():
+    W = example2_matrix() if "example2_matrix" in globals() else None
+    if W is None:
+        from golden_io import golden, read_sections
+        g = read_sections(golden("layer_hand_worked.txt"))
+        W = np.array([[float(v) for v in row] for row in g["W"]], dtype=np.float32)
+    im = orc.index_map_encode(W)
+    assert im["codebook"].tolist() == [0, 1, 2, 3, 4, 5, 6, 10] and im["b_bar"] == 8
+    assert np.array_equal(orc.index_map_decode(im), W)
+    # pi_ij points at the value: row 1 of the example holds 10 in column 1
+    assert im["codebook"][im["index"][1, 1]] == 10 and im["index"][3].tolist() == [0] * 5
+    # occupancy b_bar / b + k / (n m) (Sect. III-C.1): 8/32 + 8/25 here; about 1/4 for a large matrix with k <= 256
+    assert orc.index_map_bits(im) == 8 * 25 + 8 * 32
+    big = orc.index_map_encode((np.arange(300 * 200) % 256).reshape(300, 200).astype(np.float32))
+    assert abs(orc.index_map_bits(big) / (32.0 * 300 * 200) - (0.25 + 256 / 60000)) < 1e-12
+    wide = orc.index_map_encode(np.arange(400, dtype=np.float32).reshape(20, 20))
+    assert wide["b_bar"] == 16                              # more than 256 values: two bytes per pointer
+    x = np.array([1, 2, 3, 4, 5], dtype=np.float32)
+    y, a = orc.dot_index_map(im, x)
+    assert y[0].tolist() == [7, 29, 4, 0, 45] and a[0].tolist() == [7, 29, 4, 0, 45]
+
+
+def test_csc_dot_and_size_on_the_papers_example():
+    from golden_io import golden, read_sections
+    g = read_sections(golden("layer_hand_worked.txt"))
+    W = np.array([[float(v) for v in row] for row in g["W"]], dtype=np.float32)
+    nz, ri, cb = orc.csc(W, W != 0)
+    assert orc.csc_bits(nz, ri, cb) == (2 * 7 + 5 + 1) * 32       # (2q + m + 1) b, Sect. IV-A
+    x = np.array([1, 2, 3, 4, 5], dtype=np.float32)
+    y, a = orc.dot_csc(nz, ri, cb, 5, x)
+    assert y[0].tolist() == [7, 29, 4, 0, 45]
+
+
+def test_comparison_formats_agree_with_the_definition():
+    rng = np.random.default_rng(21)
+    W = rng.standard_normal((60, 17)).astype(np.float32)
+    W[np.abs(W) < 0.8] = 0
+    W = np.round(W * 4) / 4                                   # few distinct values
+    X = rng.standard_normal((3, 60)).astype(np.float32)
+    y_ref, a_ref = orc.dot_definition(W, X)
+    y, a = orc.dot_index_map(orc.index_map_encode(W), X)
+    assert np.array_equal(y, y_ref) and np.array_equal(a, a_ref)
+    nz, ri, cb = orc.csc(W, W != 0)
+    y, a = orc.dot_csc(nz, ri, cb, 60, X)
+    assert np.array_equal(y, y_ref) and np.array_equal(a, a_ref)
