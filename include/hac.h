@@ -332,6 +332,45 @@ int hac_dot_noalloc(const hac_format* f, const float* x, int64_t batch, int64_t 
                     float* y, int64_t y_stride_j, int64_t y_stride_b, void* cuda_stream);
 
 /* ---------------------------------------------------------------------------------------------
+ * The two formats HAC and sHAC are compared with: the index map (Sect. III-C.1) and plain CSC
+ * (Sect. IV-A), each with its encoder on the host and its product on the device.  They take no handle:
+ * the caller owns every array.
+ *
+ * hac_index_map_encode - the k distinct values of Wq (row-major, leading dimension ldw; zero is a
+ *   value like any other; -0.0 counts as 0) ascending into codebook (room for 2^index_bits floats),
+ *   their number into *k, and for every weight the position of its value into index_colmajor
+ *   (index_colmajor[j*n + i] points at Wq[i][j]; uint8_t for index_bits == 8, uint16_t for 16; n*m
+ *   entries).  All host memory.  Occupancy as the paper counts it: index_bits / 32 + k / (n m).
+ *   Errors: HAC_ERR_INVALID_ARG, HAC_ERR_NONFINITE_INPUT, HAC_ERR_K_TOO_LARGE (more than 2^index_bits
+ *   values), HAC_ERR_ALLOC.
+ * hac_index_map_dot - y = x^T W with W[i][j] = codebook[index[j*n + i]], all pointers device memory,
+ *   x and y with the strides of hac_dot, fp32 products and sums, asynchronous on cuda_stream.  A
+ *   pointer at or beyond k reads the last codebook entry (two-byte pointers) or 0 (one-byte pointers).
+ *   128-bit loads of the pointers are used when n is a multiple of 16 / index_bits * 8 and index_dev is
+ *   16-byte aligned; otherwise element loads.  Needs no workspace.
+ *
+ * shac_csc_encode - CSC of Wq: the nonzero weights column by column, rows ascending, into nz, their rows
+ *   into ri, and the m+1 column boundaries into cb; their number into *q.  With nz, ri and cb all NULL
+ *   only *q is written (size query); otherwise capacity is the room in nz and ri (entries).  Occupancy
+ *   as the paper counts it: (2 q + m + 1) / (n m).  Errors: HAC_ERR_INVALID_ARG, HAC_ERR_NONFINITE_INPUT,
+ *   HAC_ERR_BUFFER_TOO_SMALL, HAC_ERR_OFFSET_OVERFLOW (2^32 entries or more).
+ * shac_csc_dot - y[j] = sum over p in [cb[j], cb[j+1]) of nz[p] * x[ri[p]], device pointers, strides as
+ *   hac_dot, asynchronous on cuda_stream; a row at or beyond n contributes nothing.  nz_dev and ri_dev may
+ *   be NULL when nothing is stored.
+ * Both products: HAC_ERR_INVALID_ARG (null pointers, sizes below 1), HAC_ERR_CUDA (launch failure).
+ * ------------------------------------------------------------------------------------------- */
+int hac_index_map_encode(const float* Wq, int64_t n, int64_t m, int64_t ldw, int index_bits, void* index_colmajor,
+                         float* codebook, int* k);
+int hac_index_map_dot(const void* index_dev, int index_bits, const float* codebook_dev, int k, int64_t n, int64_t m,
+                      const float* x, int64_t batch, int64_t x_stride_i, int64_t x_stride_b, float* y,
+                      int64_t y_stride_j, int64_t y_stride_b, void* cuda_stream);
+int shac_csc_encode(const float* Wq, int64_t n, int64_t m, int64_t ldw, float* nz, uint32_t* ri, uint32_t* cb,
+                    int64_t capacity, int64_t* q);
+int shac_csc_dot(const float* nz_dev, const uint32_t* ri_dev, const uint32_t* cb_dev, int64_t n, int64_t m, const float* x,
+                 int64_t batch, int64_t x_stride_i, int64_t x_stride_b, float* y, int64_t y_stride_j, int64_t y_stride_b,
+                 void* cuda_stream);
+
+/* ---------------------------------------------------------------------------------------------
  * TEST ONLY: decode on the device into a caller's device buffer, to show that the kernels' decoder
  * reproduces the quantized weights bit for bit (the formats are lossless, Sect. IV-B).  The product
  * path never does this.  hac: W_colmajor[j*n + i] = Wq[i][j] (n*m floats).  shac: nz[p] for the nnz

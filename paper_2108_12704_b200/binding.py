@@ -74,6 +74,7 @@ EXPORTS = (
     "shac_dot_host", "hac_dot_host_async", "shac_dot_host_async", "hac_debug_decode", "shac_debug_decode",
     "hac_debug_table_lookup", "shac_debug_table_lookup", "hac_last_launch_count",
     "shac_last_launch_count", "hac_free", "shac_free", "hac_status_string", "hac_last_cuda_error",
+    "hac_index_map_encode", "hac_index_map_dot", "shac_csc_encode", "shac_csc_dot",
 )
 
 
@@ -117,6 +118,10 @@ def load():
         getattr(lib, f"{kind}_free").restype = None
     lib.hac_dot_noalloc.argtypes = [vp, fp, i64, i64, i64, fp, i64, i64, vp]
     lib.hac_chain.argtypes = [C.POINTER(Layer), C.c_int, fp, i64, fp, fp, fp, sz, vp, sz, vp]
+    lib.hac_index_map_encode.argtypes = [fp, i64, i64, i64, C.c_int, vp, fp, C.POINTER(C.c_int)]
+    lib.hac_index_map_dot.argtypes = [vp, C.c_int, fp, C.c_int, i64, i64, fp, i64, i64, i64, fp, i64, i64, vp]
+    lib.shac_csc_encode.argtypes = [fp, i64, i64, i64, fp, vp, vp, i64, C.POINTER(i64)]
+    lib.shac_csc_dot.argtypes = [fp, vp, vp, i64, i64, fp, i64, i64, i64, fp, i64, i64, vp]
     lib.hac_status_string.argtypes = [C.c_int]
     lib.hac_status_string.restype = C.c_char_p
     lib.hac_last_cuda_error.restype = C.c_char_p
@@ -392,3 +397,99 @@ def chain(layers, x, y=None, workspace=None):
     _check(lib.hac_chain(arr, len(layers), x.data_ptr(), B, y.data_ptr(), acts[0].data_ptr(), acts[1].data_ptr(), widest,
                          workspace.data_ptr(), workspace.numel(), st), "hac_chain")
     return y, last.last_launch_count()
+
+
+def _dot_strides(x, y, m, layout):
+    """(B, x_stride_i, x_stride_b, y, y_stride_j, y_stride_b) for the x / y conventions of Format.dot."""
+    import torch
+    assert x.is_cuda and x.dtype == torch.float32
+    if x.dim() == 1:
+        B, xs_i, xs_b, yshape = 1, x.stride(0), 0, (m,)
+    elif layout == "nb":
+        B, xs_i, xs_b, yshape = x.shape[1], x.stride(0), x.stride(1), (m, x.shape[1])
+    else:
+        B, xs_i, xs_b, yshape = x.shape[0], x.stride(1), x.stride(0), (x.shape[0], m)
+    if y is None:
+        y = torch.empty(yshape, dtype=torch.float32, device=x.device)
+    if y.dim() == 1:
+        ys_j, ys_b = y.stride(0), 0
+    elif layout == "nb":
+        ys_j, ys_b = y.stride(0), y.stride(1)
+    else:
+        ys_j, ys_b = y.stride(1), y.stride(0)
+    return B, xs_i, xs_b, y, ys_j, ys_b
+
+
+class IndexMap:
+    """hac_index_map_* of the C ABI (Sect. III-C.1): encode on the host, keep the arrays in device tensors, multiply."""
+
+    def __init__(self, Wq: np.ndarray, index_bits: int = 8):
+        lib = load()
+        Wq = np.ascontiguousarray(Wq, dtype=np.float32)
+        self.n, self.m, self.index_bits = Wq.shape[0], Wq.shape[1], int(index_bits)
+        self.index = np.empty(self.n * self.m, dtype=np.uint8 if index_bits == 8 else np.uint16)
+        codebook = np.zeros(1 << index_bits, dtype=np.float32)
+        k = C.c_int()
+        _check(lib.hac_index_map_encode(Wq.ctypes.data, self.n, self.m, Wq.strides[0] // 4, self.index_bits,
+                                        self.index.ctypes.data, codebook.ctypes.data, C.byref(k)), "index_map_encode")
+        self.k = k.value
+        self.codebook = codebook[:self.k].copy()
+        self._dev = None
+
+    def psi(self) -> float:
+        return self.index_bits / 32.0 + self.k / (self.n * self.m)
+
+    def upload(self, device="cuda"):
+        import torch
+        self._dev = (torch.from_numpy(self.index.view(np.uint8)).to(device), torch.from_numpy(self.codebook).to(device))
+        return self
+
+    def dot(self, x, y=None, layout="nb"):
+        import torch
+        if self._dev is None:
+            raise HacError(-7, "index_map_dot", "not uploaded")
+        B, xs_i, xs_b, y, ys_j, ys_b = _dot_strides(x, y, self.m, layout)
+        _check(load().hac_index_map_dot(self._dev[0].data_ptr(), self.index_bits, self._dev[1].data_ptr(), self.k, self.n,
+                                        self.m, x.data_ptr(), B, xs_i, xs_b, y.data_ptr(), ys_j, ys_b,
+                                        torch.cuda.current_stream().cuda_stream), "index_map_dot")
+        return y
+
+
+class Csc:
+    """shac_csc_* of the C ABI (Sect. IV-A): nz, ri, cb built on the host, kept in device tensors, multiplied."""
+
+    def __init__(self, Wq: np.ndarray):
+        lib = load()
+        Wq = np.ascontiguousarray(Wq, dtype=np.float32)
+        self.n, self.m = Wq.shape
+        q = C.c_int64()
+        ld = Wq.strides[0] // 4
+        _check(lib.shac_csc_encode(Wq.ctypes.data, self.n, self.m, ld, None, None, None, 0, C.byref(q)), "csc_encode")
+        self.q = q.value
+        self.nz = np.empty(max(self.q, 1), dtype=np.float32)
+        self.ri = np.empty(max(self.q, 1), dtype=np.uint32)
+        self.cb = np.empty(self.m + 1, dtype=np.uint32)
+        _check(lib.shac_csc_encode(Wq.ctypes.data, self.n, self.m, ld, self.nz.ctypes.data, self.ri.ctypes.data,
+                                   self.cb.ctypes.data, self.q, C.byref(q)), "csc_encode")
+        self.nz, self.ri = self.nz[:self.q], self.ri[:self.q]
+        self._dev = None
+
+    def psi(self) -> float:
+        return (2 * self.q + self.m + 1) / (self.n * self.m)
+
+    def upload(self, device="cuda"):
+        import torch
+        as_i32 = lambda a: torch.from_numpy(np.ascontiguousarray(a).view(np.int32)).to(device)
+        self._dev = (torch.from_numpy(np.ascontiguousarray(self.nz)).to(device), as_i32(self.ri), as_i32(self.cb))
+        return self
+
+    def dot(self, x, y=None, layout="nb"):
+        import torch
+        if self._dev is None:
+            raise HacError(-7, "csc_dot", "not uploaded")
+        B, xs_i, xs_b, y, ys_j, ys_b = _dot_strides(x, y, self.m, layout)
+        nz, ri, cb = self._dev
+        _check(load().shac_csc_dot(nz.data_ptr() if self.q else None, ri.data_ptr() if self.q else None, cb.data_ptr(),
+                                   self.n, self.m, x.data_ptr(), B, xs_i, xs_b, y.data_ptr(), ys_j, ys_b,
+                                   torch.cuda.current_stream().cuda_stream), "csc_dot")
+        return y

@@ -8,7 +8,7 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(_HERE)
 CSRC = os.path.join(_HERE, "csrc")
 LIB = os.path.join(_HERE, "libhac_b200.so")
-SOURCES = ("hac_build.cpp", "hac_kernels.cu")
+SOURCES = ("hac_build.cpp", "hac_kernels.cu", "compare_kernels.cu")
 HEADERS = (os.path.join(CSRC, "hac_internal.h"), os.path.join(ROOT, "include", "hac.h"))
 
 

@@ -4,6 +4,7 @@
 
 #include <cstddef>
 #include <cstdint>
+#include <string>
 #include <vector>
 
 #include "hac.h"
@@ -162,6 +163,9 @@ struct ImageLayout {
         seg_first, ri, cb, unit_info, task_off, task_pos, total;
 };
 ImageLayout image_layout(const Format& f);
+
+// Text that hac_last_cuda_error() returns on this thread (set by every file that makes CUDA calls).
+void set_last_cuda_error(const std::string& text);
 
 }  // namespace hacb200
 

@@ -2537,6 +2537,8 @@ __global__ void transpose_kernel(const float* __restrict__ in, float* __restrict
 // ------------------------------------------------------------------------------------------------
 // Host side
 // ------------------------------------------------------------------------------------------------
+void set_last_cuda_error(const std::string& text) { g_last_cuda_error = text; }
+
 struct DeviceInfo {
     int sms = 0;
     int max_smem_optin = 0;

@@ -2,7 +2,7 @@
 kernel times against the HBM roofline on the compressed bytes, for the benchmark configurations
 and the sparsity x k sweep.  One JSON line per (configuration, format, batch).
 
-    python -m paper_2108_12704_b200.report [--configs 1,2,3,4] [--sweep] [--paper-shapes] [--out FILE]
+    python -m paper_2108_12704_b200.report [--configs 1,2,3,4] [--sweep] [--paper-shapes] [--chain] [--compare] [--out FILE]
 
 Timing protocol as in bench.py: device images replicated to more than three times the L2 size and
 rotated per launch, launches captured in CUDA graphs, CUDA events on the launching stream, best of
@@ -194,12 +194,106 @@ def measure_chain(batches=(1, 64), replays=200):
     return rows
 
 
+def measure_compare(wl, replays=5):
+    """One-input product of the same quantized matrix in the formats the paper compares (Sect. V): dense fp32
+    (the library's matrix-vector product, for context), index map, CSC, and HAC / sHAC; psi as the paper counts it."""
+    import torch
+    import paper_2108_12704_b200 as hb
+    from paper_2108_12704_b200.binding import Csc, IndexMap
+    W = si.weights(wl)
+    peak, peak_kind = _peaks()
+    ours = {kind: hb.Format(kind, W, sparsity=wl.sparsity, k=wl.k, quantizer=wl.quantizer, kmeans_iters=wl.kmeans_iters,
+                            seed=wl.seed) for kind in ("hac", "shac")}
+    Wq = ours["hac"].decode_host()
+    Xh = si.inputs(wl, 1)
+    ref = Xh.astype(np.float64) @ Wq.astype(np.float64)
+    tol = 1e-5 * (np.abs(Xh.astype(np.float64)) @ np.abs(Wq.astype(np.float64))) + 1e-7
+    x = torch.from_numpy(Xh[0]).cuda()
+    rows = []
+
+    def timed(name, psi, nbytes, make_step, R):
+        steps = [make_step(r) for r in range(R)]
+        y = steps[0]()
+        torch.cuda.synchronize()
+        ok = bool(np.all(np.abs(y.cpu().numpy().astype(np.float64)[None] - ref) <= (tol if name != "dense_fp32" else 10 * tol)))
+        for st in steps[:3]:
+            st()
+        g = _capture(torch, lambda: [st() for st in steps])
+        g.replay()
+        torch.cuda.synchronize()
+        best = float("inf")
+        for _ in range(replays):
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record(); g.replay(); e1.record()
+            torch.cuda.synchronize()
+            best = min(best, e0.elapsed_time(e1) / R * 1e3)
+        rows.append(dict(report="format_comparison", workload=wl.name, n=wl.n, m=wl.m, sparsity=wl.sparsity, k=wl.k,
+                         format=name, psi=round(psi, 5), bytes=int(nbytes), us=round(best, 2), within_tolerance=ok,
+                         gb_per_s=round(nbytes / best / 1e3, 1), frac_of_hbm=round(nbytes / best / 1e3 / peak, 4),
+                         hbm_peak=f"{peak} GB/s ({peak_kind})"))
+
+    def replicas(nbytes):
+        return min(64, max(2, math.ceil(3 * L2_BYTES / max(1, nbytes))))
+
+    # dense fp32, [m, n] row-major so that the library reads every column of W contiguously
+    dense_bytes = 4 * wl.n * wl.m
+    R = replicas(dense_bytes)
+    Wd = [torch.from_numpy(np.ascontiguousarray(Wq.T)).cuda() for _ in range(R)]
+    yd = torch.empty(wl.m, device="cuda")
+    timed("dense_fp32", 1.0, dense_bytes, lambda r: (lambda: torch.mv(Wd[r], x, out=yd)), R)
+    del Wd
+    im = IndexMap(Wq, 8 if len(np.unique(Wq)) <= 256 else 16)
+    nbytes = im.index.nbytes + 4 * im.k
+    R = replicas(nbytes)
+    ims = [IndexMap.__new__(IndexMap) for _ in range(R)]
+    for o in ims:
+        o.__dict__.update(im.__dict__)
+        o.upload()
+    yi = torch.empty(wl.m, device="cuda")
+    timed(f"index_map{im.index_bits}", im.psi(), nbytes, lambda r: (lambda: ims[r].dot(x, yi)), R)
+    del ims
+    c = Csc(Wq)
+    nbytes = 8 * c.q + 4 * (wl.m + 1)
+    R = replicas(nbytes)
+    cs = [Csc.__new__(Csc) for _ in range(R)]
+    for o in cs:
+        o.__dict__.update(c.__dict__)
+        o.upload()
+    yc = torch.empty(wl.m, device="cuda")
+    timed("csc", c.psi(), nbytes, lambda r: (lambda: cs[r].dot(x, yc)), R)
+    del cs
+    for kind, fmt in ours.items():
+        fmt.upload()
+        sizes = fmt.sizes()
+        nbytes = fmt.device_bytes()
+        R = replicas(nbytes)
+        reps = []
+        for _ in range(R):
+            buf = torch.empty(nbytes + 256, dtype=torch.uint8, device="cuda")
+            off = (-buf.data_ptr()) % 256
+            view = buf[off:off + nbytes]
+            view.copy_(fmt.image())
+            reps.append(view)
+        yo = torch.empty(wl.m, device="cuda")
+        ws = torch.empty(max(16, fmt.workspace_bytes(1)), dtype=torch.uint8, device="cuda")
+
+        def make(r, fmt=fmt, reps=reps, yo=yo, ws=ws):
+            def step():
+                fmt.attach(reps[r])
+                return fmt.dot(x, yo, ws)
+            return step
+        timed(kind, sizes["paper_bits"] / (32.0 * wl.n * wl.m), algorithmic_bytes(sizes), make, R)
+        del reps
+    return rows
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--configs", default="1,2,3,4")
     ap.add_argument("--sweep", action="store_true", help="configuration 5: sparsity x k grid, HAC and sHAC")
     ap.add_argument("--paper-shapes", action="store_true", help="the fully connected shapes of the paper's Sect. V-C")
     ap.add_argument("--chain", action="store_true", help="the fully connected stack as a chain of layers")
+    ap.add_argument("--compare", action="store_true", help="dense, index map, CSC, HAC and sHAC on configurations 2 and 3")
     ap.add_argument("--out", default="")
     args = ap.parse_args()
     out = open(args.out, "w") if args.out else None
@@ -227,6 +321,9 @@ def main():
                 emit(measure(wl, kind, wl.batches, W=W))
     if args.chain:
         emit(measure_chain())
+    if args.compare:
+        for wl in (si.CFG2_DENSE_HAC, si.CFG3_FC_SHAC):
+            emit(measure_compare(wl))
     if args.paper_shapes:
         for wl in si.paper_shaped_cells():
             for kind in wl.formats:

@@ -280,3 +280,41 @@ def test_deserialize_checks_the_contents_not_only_the_checksum():
     with pytest.raises(hb.HacError) as ei:
         hb.Format.deserialize("hac", resealed(bad))
     assert ei.value.status == -10
+
+
+# ---------------------------------------------------------------- the comparison formats' encoders (host only)
+def test_index_map_and_csc_encoders_against_the_oracle():
+    from paper_2108_12704_b200.binding import IndexMap, Csc
+    wl = si.scaled(si.CFG3_FC_SHAC, 300, 37)
+    W = si.weights(wl)
+    Wq, mask = orc.quantize(W, wl.sparsity, wl.k, wl.quantizer, wl.kmeans_iters, wl.seed)
+    ref = orc.index_map_encode(Wq)
+    im = IndexMap(Wq, 8)
+    assert im.k == len(ref["codebook"]) and np.array_equal(im.codebook.view(np.uint32), ref["codebook"].view(np.uint32))
+    assert np.array_equal(im.index.reshape(wl.m, wl.n), ref["index"].T)             # column-major pointers
+    assert abs(im.psi() - orc.index_map_bits(ref) / (32.0 * wl.n * wl.m)) < 1e-12
+    im16 = IndexMap(Wq, 16)
+    assert im16.index.dtype == np.uint16 and np.array_equal(im16.index.reshape(wl.m, wl.n), ref["index"].T)
+    nz, ri, cb = orc.csc(Wq, Wq != 0)
+    c = Csc(Wq)
+    assert c.q == len(nz) and np.array_equal(c.nz.view(np.uint32), np.asarray(nz, np.float32).view(np.uint32))
+    assert np.array_equal(c.ri.astype(np.int64), np.asarray(ri, np.int64)) and np.array_equal(c.cb.astype(np.int64), cb)
+    assert abs(c.psi() - orc.csc_bits(nz, ri, cb) / (32.0 * wl.n * wl.m)) < 1e-12
+
+
+def test_comparison_encoders_reject_bad_input():
+    from paper_2108_12704_b200.binding import IndexMap, Csc
+    many = np.arange(300, dtype=np.float32).reshape(20, 15)
+    with pytest.raises(hb.HacError) as e:
+        IndexMap(many, 8)                                    # 300 values do not fit one byte
+    assert e.value.status == -4
+    assert IndexMap(many, 16).k == 300
+    bad = many.copy(); bad[3, 3] = np.nan
+    for cls in (lambda w: IndexMap(w, 8), Csc):
+        with pytest.raises(hb.HacError) as e:
+            cls(bad)
+        assert e.value.status == -3
+    z = Csc(np.zeros((4, 3), dtype=np.float32))
+    assert z.q == 0 and z.cb.tolist() == [0, 0, 0, 0]
+    neg = IndexMap(np.array([[-0.0, 0.0], [1.0, 0.0]], dtype=np.float32), 8)
+    assert neg.k == 2                                        # -0.0 and 0.0 are one value
