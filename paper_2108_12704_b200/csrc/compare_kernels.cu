@@ -85,6 +85,85 @@ index_map8_kernel(const uint8_t* __restrict__ index, const float* __restrict__ c
     }
 }
 
+// One input, x contiguous and small enough for shared memory: x is staged once per block, a lane takes four consecutive
+// pointers (one 32-bit load) and the four matching elements of x (one 128-bit load, lanes on disjoint banks), four such
+// groups in flight per step.
+constexpr int kVecThreads = 512;
+constexpr int kVecWarps = kVecThreads / 32;
+
+__global__ void __launch_bounds__(kVecThreads)
+index_map8_vec_kernel(const uint8_t* __restrict__ index, const float* __restrict__ codebook, int k, int64_t n, int64_t m,
+                      const float* __restrict__ x, float* __restrict__ y, int64_t y_stride_j) {
+    extern __shared__ __align__(16) float smem[];
+    float* cb_s = smem;                                   // [256][32]
+    float* x_s = smem + 256 * kCodebookCopies;            // [n rounded up to 4]
+    for (int e = threadIdx.x; e < 256 * kCodebookCopies; e += kVecThreads) {
+        const int entry = e / kCodebookCopies;
+        cb_s[e] = entry < k ? codebook[entry] : 0.0f;
+    }
+    for (int64_t i = threadIdx.x; i < n; i += kVecThreads) x_s[i] = __ldg(x + i);
+    __syncthreads();
+    const int lane = threadIdx.x & 31;
+    const float* mine = cb_s + lane;
+    const int64_t warp = (int64_t)blockIdx.x * kVecWarps + (threadIdx.x >> 5);
+    const int64_t warps = (int64_t)gridDim.x * kVecWarps;
+    const int64_t groups = n / 4;                         // n is a multiple of 4 here
+    for (int64_t j = warp; j < m; j += warps) {
+        const uint32_t* col = reinterpret_cast<const uint32_t*>(index + j * n);
+        float acc0 = 0.0f, acc1 = 0.0f;
+        for (int64_t g0 = lane; g0 < groups; g0 += 4 * 32) {
+            uint32_t p[4];
+#pragma unroll
+            for (int u = 0; u < 4; ++u) p[u] = g0 + 32 * u < groups ? __ldg(col + g0 + 32 * u) : 0u;
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+                if (g0 + 32 * u < groups) {
+                    const float4 xv = *reinterpret_cast<const float4*>(x_s + 4 * (g0 + 32 * u));
+                    acc0 = fmaf(mine[(p[u] & 0xffu) * kCodebookCopies], xv.x, acc0);
+                    acc1 = fmaf(mine[((p[u] >> 8) & 0xffu) * kCodebookCopies], xv.y, acc1);
+                    acc0 = fmaf(mine[((p[u] >> 16) & 0xffu) * kCodebookCopies], xv.z, acc0);
+                    acc1 = fmaf(mine[(p[u] >> 24) * kCodebookCopies], xv.w, acc1);
+                }
+            }
+        }
+        const float s = warp_sum(acc0 + acc1);
+        if (lane == 0) y[j * y_stride_j] = s;
+    }
+}
+
+// CSC, one input, x staged in shared memory and gathered from there.
+__global__ void __launch_bounds__(kVecThreads)
+csc_vec_kernel(const float* __restrict__ nz, const uint32_t* __restrict__ ri, const uint32_t* __restrict__ cb, int64_t n,
+               int64_t m, const float* __restrict__ x, float* __restrict__ y, int64_t y_stride_j) {
+    extern __shared__ __align__(16) float smem[];
+    for (int64_t i = threadIdx.x; i < n; i += kVecThreads) smem[i] = __ldg(x + i);
+    __syncthreads();
+    const int lane = threadIdx.x & 31;
+    const int64_t warp = (int64_t)blockIdx.x * kVecWarps + (threadIdx.x >> 5);
+    const int64_t warps = (int64_t)gridDim.x * kVecWarps;
+    for (int64_t j = warp; j < m; j += warps) {
+        const uint32_t lo = __ldg(cb + j), hi = __ldg(cb + j + 1);
+        float acc0 = 0.0f, acc1 = 0.0f;
+        for (uint32_t p0 = lo + lane; p0 < hi; p0 += 4 * 32) {
+            float w[4];
+            uint32_t r[4];
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+                const bool in = p0 + 32 * u < hi;
+                w[u] = in ? __ldg(nz + p0 + 32 * u) : 0.0f;
+                r[u] = in ? __ldg(ri + p0 + 32 * u) : 0u;
+            }
+#pragma unroll
+            for (int u = 0; u < 4; u += 2) {
+                acc0 = fmaf(w[u], r[u] < n ? smem[r[u]] : 0.0f, acc0);
+                acc1 = fmaf(w[u + 1], r[u + 1] < n ? smem[r[u + 1]] : 0.0f, acc1);
+            }
+        }
+        const float s = warp_sum(acc0 + acc1);
+        if (lane == 0) y[j * y_stride_j] = s;
+    }
+}
+
 // Index map with two bytes per weight (more than 256 values): the codebook stays in global memory and is
 // read through the read-only cache.  A pointer at or beyond k reads the last entry.
 template <int kB>
@@ -171,14 +250,30 @@ int cuda_error(cudaError_t e, const char* what) {
 }
 
 // Enough blocks to fill the device a few times over, never more than there are columns to hand out.
-int grid_for(int64_t m, int* out) {
-    int dev = 0, sms = 0;
+int device_limits(int* sms, int* smem_optin) {
+    int dev = 0;
     cudaError_t e = cudaGetDevice(&dev);
-    if (e == cudaSuccess) e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
-    if (e != cudaSuccess) return cuda_error(e, "cudaDeviceGetAttribute");
+    if (e == cudaSuccess) e = cudaDeviceGetAttribute(sms, cudaDevAttrMultiProcessorCount, dev);
+    if (e == cudaSuccess) e = cudaDeviceGetAttribute(smem_optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev);
+    return e == cudaSuccess ? HAC_OK : cuda_error(e, "cudaDeviceGetAttribute");
+}
+
+int grid_for(int64_t m, int* out) {
+    int sms = 0, smem = 0;
+    if (int rc = device_limits(&sms, &smem)) return rc;
     const int64_t want = (m + kCmpWarps - 1) / kCmpWarps;
     *out = (int)std::max<int64_t>(1, std::min<int64_t>(want, (int64_t)sms * 8));
     return HAC_OK;
+}
+
+// Launch shape of the kernels that stage x: as many blocks per SM as the shared memory allows (at most 4), the columns dealt
+// to their warps.  Returns false when x does not fit.
+bool staged_x_shape(int64_t m, size_t smem_bytes, int sms, int smem_optin, int* grid) {
+    if (smem_bytes > (size_t)smem_optin) return false;
+    const int per_sm = (int)std::max<size_t>(1, std::min<size_t>(4, ((size_t)228 * 1024) / (smem_bytes + 1024)));
+    const int64_t want = (m + kVecWarps - 1) / kVecWarps;
+    *grid = (int)std::max<int64_t>(1, std::min<int64_t>(want, (int64_t)sms * per_sm));
+    return true;
 }
 
 bool finite_and_normal_zero(float& v) {
@@ -237,6 +332,19 @@ int hac_index_map_dot(const void* index_dev, int index_bits, const float* codebo
     if (int rc = grid_for(m, &grid)) return rc;
     cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
     const Strides st{x_stride_i, x_stride_b, y_stride_j, y_stride_b};
+    if (index_bits == 8 && batch == 1 && x_stride_i == 1 && n % 4 == 0 && reinterpret_cast<uintptr_t>(index_dev) % 4 == 0) {
+        int sms = 0, optin = 0, vgrid = 0;
+        if (int rc = device_limits(&sms, &optin)) return rc;
+        const size_t smem = ((size_t)256 * kCodebookCopies + (size_t)n) * sizeof(float);
+        if (staged_x_shape(m, smem, sms, optin, &vgrid)) {
+            cudaError_t e = cudaFuncSetAttribute(index_map8_vec_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+            if (e != cudaSuccess) return cuda_error(e, "cudaFuncSetAttribute");
+            index_map8_vec_kernel<<<vgrid, kVecThreads, smem, s>>>(static_cast<const uint8_t*>(index_dev), codebook_dev, k, n, m, x,
+                                                                    y, y_stride_j);
+            e = cudaGetLastError();
+            return e == cudaSuccess ? HAC_OK : cuda_error(e, "index map kernel launch");
+        }
+    }
     if (index_bits == 8) {
         const size_t smem = (size_t)256 * kCodebookCopies * sizeof(float);
         auto launch = [&](auto kern) -> int {
@@ -294,6 +402,18 @@ int shac_csc_dot(const float* nz_dev, const uint32_t* ri_dev, const uint32_t* cb
     if (int rc = grid_for(m, &grid)) return rc;
     cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
     const Strides st{x_stride_i, x_stride_b, y_stride_j, y_stride_b};
+    if (batch == 1 && x_stride_i == 1) {
+        int sms = 0, optin = 0, vgrid = 0;
+        if (int rc = device_limits(&sms, &optin)) return rc;
+        const size_t smem = (size_t)n * sizeof(float);
+        if (staged_x_shape(m, smem, sms, optin, &vgrid)) {
+            cudaError_t e = cudaFuncSetAttribute(csc_vec_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+            if (e != cudaSuccess) return cuda_error(e, "cudaFuncSetAttribute");
+            csc_vec_kernel<<<vgrid, kVecThreads, smem, s>>>(nz_dev, ri_dev, cb_dev, n, m, x, y, y_stride_j);
+            e = cudaGetLastError();
+            return e == cudaSuccess ? HAC_OK : cuda_error(e, "CSC kernel launch");
+        }
+    }
     if (batch == 1) csc_kernel<1><<<grid, kCmpThreads, 0, s>>>(nz_dev, ri_dev, cb_dev, n, m, x, (int)batch, st, y);
     else csc_kernel<kCmpBatchTile><<<grid, kCmpThreads, 0, s>>>(nz_dev, ri_dev, cb_dev, n, m, x, (int)batch, st, y);
     const cudaError_t e = cudaGetLastError();

@@ -250,6 +250,25 @@ def test_config5_sweep_cells_full_size(sp, k):
         _full_size(cell, kind, (1, 32), ncols=32, quantized=(W, Wq, mask))
 
 
+PAPER_CELLS = si.paper_shaped_cells()
+
+
+@pytest.mark.parametrize("cell", PAPER_CELLS, ids=[c.name for c in PAPER_CELLS])
+def test_paper_shaped_cells_all_formats(cell):
+    """The fully connected shapes of the paper's comparison of formats (Sect. V-C), one input and its eight inputs: HAC and
+    sHAC on every output, and the index map and CSC of the same quantized matrix, all against the oracle."""
+    from paper_2108_12704_b200.binding import Csc, IndexMap
+    W = si.weights(cell)
+    Wq, mask = orc.quantize(W, cell.sparsity, cell.k, cell.quantizer, cell.kmeans_iters, cell.seed)
+    for kind in ("hac", "shac"):
+        _full_size(cell, kind, (1, 8), ncols=min(32, cell.m), quantized=(W, Wq, mask), all_outputs_up_to=8)
+    X = si.inputs(cell, 8)
+    y_ref, a = orc.dot_definition(Wq, X)
+    for fmt in (IndexMap(Wq, 8 if len(np.unique(Wq)) <= 256 else 16).upload(), Csc(Wq).upload()):
+        check_outputs(run_dot(fmt, X), y_ref, a)
+        check_outputs(run_dot(fmt, X[:1]), y_ref[:1], a[:1])
+
+
 def test_chained_products_keep_stream_order():
     """Two layers back to back on one stream, the second reading what the first wrote, then the same
     buffers reused at once for another input: the kernels may start early (they are launched with
