@@ -167,6 +167,31 @@ int hac_build (const float* W, int64_t n, int64_t m, int64_t ldw, const hac_buil
 int shac_build(const float* W, int64_t n, int64_t m, int64_t ldw, const hac_build_params* params,
                shac_format** out);
 
+/* ---------------------------------------------------------------------------------------------
+ * hac_build_unified - several matrices quantized at the same time with one k and coded with one dictionary
+ * (the "unified" quantization of Sect. V-D: uCWS, uPWS, uUQ).  Host only.
+ *   1. Every matrix is pruned on its own (step 1 of hac_build, the same sparsity for all).
+ *   2. The non-null weights of all matrices, matrix after matrix in the order given and column-major inside
+ *      each, go through the weight sharing of params->quantizer together: one set of at most k shared values.
+ *   3. One codebook (the distinct shared values of all matrices, plus 0 when a HAC matrix has a null entry) and
+ *      one Huffman code on the symbol counts of all the streams together.
+ *   4. Every matrix is emitted with that code as a format of its own (out[i] is a hac_format* when
+ *      layers[i].sparse == 0, a shac_format* when it is 1), to be used, serialized and freed like any other.
+ *      Each keeps the whole shared codebook and code (a symbol that does not occur in it has count 0), so
+ *      hac_sizes counts the dictionary once per matrix; as the paper counts a unified model the dictionary
+ *      term 6 k b of paper_bits is paid once for all of them.
+ * With one matrix the result equals hac_build / shac_build.  On error no handle is returned.
+ * Errors as hac_build; HAC_ERR_INVALID_ARG also for n_layers outside [1, HAC_MAX_UNIFIED_LAYERS].
+ * ------------------------------------------------------------------------------------------- */
+#define HAC_MAX_UNIFIED_LAYERS 1024
+typedef struct {
+    const float* W;           /* host, row-major, borrowed for the call */
+    int64_t      n, m, ldw;
+    int32_t      sparse;      /* 0: HAC, 1: sHAC */
+    int32_t      reserved;
+} hac_unified_layer;
+int hac_build_unified(const hac_unified_layer* layers, int n_layers, const hac_build_params* params, void** out);
+
 /* Sizes (Corollaries 1 and 2 for bound_bits) and borrowed views of the built arrays. Host only. */
 int hac_sizes  (const hac_format*  f, hac_size_report* out);
 int shac_sizes (const shac_format* f, hac_size_report* out);

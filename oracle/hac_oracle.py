@@ -734,3 +734,75 @@ def dot_csc(nz, ri, cb, n: int, X: np.ndarray):
             t = X[:, int(ri[p])] * nz64[p]
             y[:, j] += t; a[:, j] += np.abs(t)
     return y, a
+
+
+# ----------------------------------------------------------------------------
+# Sect. V-D  unified quantization: all matrices quantized together, one dictionary
+# ----------------------------------------------------------------------------
+def quantize_unified(Ws, sparsity: float, k: int, quantizer: int, iters: int = 20, seed: int = 0):
+    """Every matrix pruned on its own (Sect. III-B), then ONE run of the weight sharing over the non-null weights of all
+    of them, listed matrix after matrix and column-major inside each (reading: the paper says the matrices are quantized
+    "at the same time using a unique value of k"; the order only matters for the seeded start of k-means and the random
+    draws of PWS).  Returns a list of (Wq, mask)."""
+    pruned = [prune(W, sparsity) for W in Ws]
+    parts = [_nonnull_colmajor(Wp) for Wp in pruned]
+    if sum(d.size for d, _ in parts) == 0:
+        return [(np.zeros_like(Wp), mask) for Wp, (_, mask) in zip(pruned, parts)]
+    # the concatenated weights as one column: its column-major list of non-null weights is that concatenation
+    column = np.concatenate([d for d, _ in parts]).astype(np.float32).reshape(-1, 1)
+    if quantizer == 0:
+        shared, _ = share_none(column)
+    elif quantizer == 1:
+        shared, _ = kmeans_share(column, k, iters, seed)
+    elif quantizer == 2:
+        shared, _ = uniform_share(column, k)
+    elif quantizer == 3:
+        shared, _ = grid_share(column, k)
+    elif quantizer == 4:
+        shared, _ = pws_share(column, k, seed)
+    else:
+        raise ValueError("unknown quantizer")
+    out, at = [], 0
+    for data, mask in parts:
+        out.append((_scatter_colmajor(mask, shared[at:at + data.size, 0]), mask))
+        at += data.size
+    return out
+
+
+def unified_encode(layers):
+    """layers: list of (kind, Wq, mask).  One alphabet and one Huffman code on the symbol counts of all the streams together
+    (HAC: every entry of the matrix, zeros included; sHAC: the stored entries), then each matrix coded with it.  Returns one
+    format dict per layer (as hac_encode / shac_encode; `counts` are the layer's own, `shared_counts` those of the code)."""
+    seqs = []
+    for kind, Wq, mask in layers:
+        seqs.append(np.ascontiguousarray(Wq.T).ravel() if kind == "hac" else csc(Wq, mask)[0])
+    codebook, sym_all, counts = _alphabet(np.concatenate(seqs))
+    lengths = huffman_lengths(counts)
+    codes = canonical_codes(lengths)
+    out, at = [], 0
+    for (kind, Wq, mask), seq in zip(layers, seqs):
+        sym = sym_all[at:at + seq.size]
+        at += seq.size
+        if seq.size:
+            words, bits = _pack(sym, codes, lengths)
+        else:
+            words, bits = np.zeros(0, np.uint32), 0
+        fmt = dict(kind=kind, n=Wq.shape[0], m=Wq.shape[1], codebook=codebook, code_len=lengths, codes=codes,
+                   counts=np.bincount(sym, minlength=len(codebook)).astype(np.int64), shared_counts=counts, sym=sym,
+                   words=words, bits=bits)
+        if kind == "shac":
+            nz, ri, cb = csc(Wq, mask)
+            fmt.update(nz=nz, ri=ri, cb=cb)
+        out.append(fmt)
+    return out
+
+
+def unified_paper_bits(fmts) -> int:
+    """Size of a unified model as the paper counts it: every stream (and ri, cb of the sHAC ones), one dictionary."""
+    k = len(fmts[0]["codebook"])
+    total = 6 * k * B_WORD
+    for f in fmts:
+        total += len(f["words"]) * B_WORD
+        if f["kind"] == "shac":
+            total += B_WORD * (int(f["cb"][-1]) + f["m"] + 1)
+    return total

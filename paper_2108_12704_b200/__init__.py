@@ -1,7 +1,7 @@
 """HAC / sHAC compressed-domain products on NVIDIA B200: Python binding of libhac_b200.so.
 
 The functions carry the names of the C ABI (include/hac.h) and only marshal arguments."""
-from .binding import (Format, HacError, chain as hac_chain, QUANT_GRID, QUANT_KMEANS, QUANT_NONE, QUANT_PWS, QUANT_UNIFORM, EXPORTS, load,
+from .binding import (Format, HacError, chain as hac_chain, build_unified as hac_build_unified, QUANT_GRID, QUANT_KMEANS, QUANT_NONE, QUANT_PWS, QUANT_UNIFORM, EXPORTS, load,
                       library_path)
 
 
@@ -28,4 +28,4 @@ def shac_dot(fmt: Format, x, y=None, workspace=None, layout="nb"):
 
 
 __all__ = ["Format", "HacError", "QUANT_NONE", "QUANT_KMEANS", "QUANT_UNIFORM", "QUANT_GRID", "QUANT_PWS", "EXPORTS", "load",
-           "library_path", "hac_build", "shac_build", "hac_dot", "shac_dot", "hac_chain"]
+           "library_path", "hac_build", "shac_build", "hac_dot", "shac_dot", "hac_chain", "hac_build_unified"]

@@ -46,6 +46,11 @@ class Layer(C.Structure):
     _fields_ = [("hac", C.c_void_p), ("shac", C.c_void_p), ("epilogue", Epilogue)]
 
 
+class UnifiedLayer(C.Structure):
+    _fields_ = [("W", C.c_void_p), ("n", C.c_int64), ("m", C.c_int64), ("ldw", C.c_int64), ("sparse", C.c_int32),
+                ("reserved", C.c_int32)]
+
+
 class HostView(C.Structure):
     _fields_ = [("n", C.c_int64), ("m", C.c_int64), ("k_eff", C.c_uint32), ("seg_symbols", C.c_uint32),
                 ("codebook", C.POINTER(C.c_float)), ("code_len", C.POINTER(C.c_uint8)),
@@ -74,7 +79,7 @@ EXPORTS = (
     "shac_dot_host", "hac_dot_host_async", "shac_dot_host_async", "hac_debug_decode", "shac_debug_decode",
     "hac_debug_table_lookup", "shac_debug_table_lookup", "hac_last_launch_count",
     "shac_last_launch_count", "hac_free", "shac_free", "hac_status_string", "hac_last_cuda_error",
-    "hac_index_map_encode", "hac_index_map_dot", "shac_csc_encode", "shac_csc_dot",
+    "hac_index_map_encode", "hac_index_map_dot", "shac_csc_encode", "shac_csc_dot", "hac_build_unified",
 )
 
 
@@ -122,6 +127,7 @@ def load():
     lib.hac_index_map_dot.argtypes = [vp, C.c_int, fp, C.c_int, i64, i64, fp, i64, i64, i64, fp, i64, i64, vp]
     lib.shac_csc_encode.argtypes = [fp, i64, i64, i64, fp, vp, vp, i64, C.POINTER(i64)]
     lib.shac_csc_dot.argtypes = [fp, vp, vp, i64, i64, fp, i64, i64, i64, fp, i64, i64, vp]
+    lib.hac_build_unified.argtypes = [C.POINTER(UnifiedLayer), C.c_int, C.POINTER(BuildParams), C.POINTER(vp)]
     lib.hac_status_string.argtypes = [C.c_int]
     lib.hac_status_string.restype = C.c_char_p
     lib.hac_last_cuda_error.restype = C.c_char_p
@@ -397,6 +403,27 @@ def chain(layers, x, y=None, workspace=None):
     _check(lib.hac_chain(arr, len(layers), x.data_ptr(), B, y.data_ptr(), acts[0].data_ptr(), acts[1].data_ptr(), widest,
                          workspace.data_ptr(), workspace.numel(), st), "hac_chain")
     return y, last.last_launch_count()
+
+
+def build_unified(layers, sparsity=0.0, k=32, quantizer=QUANT_KMEANS, kmeans_iters=20, seed=0, seg_symbols=0, ri_bits=0):
+    """hac_build_unified of the C ABI: `layers` is a list of (kind, W); all matrices are quantized together and share one
+    code.  Returns one Format per layer."""
+    lib = load()
+    mats = [np.ascontiguousarray(W, dtype=np.float32) for _, W in layers]
+    arr = (UnifiedLayer * len(layers))()
+    for i, ((kind, _), W) in enumerate(zip(layers, mats)):
+        assert kind in ("hac", "shac") and W.ndim == 2
+        arr[i] = UnifiedLayer(W.ctypes.data, W.shape[0], W.shape[1], W.shape[1], 1 if kind == "shac" else 0, 0)
+    p = BuildParams(float(sparsity), int(k), int(quantizer), int(kmeans_iters), int(seg_symbols), int(seed), int(ri_bits), 0)
+    out = (C.c_void_p * len(layers))()
+    _check(lib.hac_build_unified(arr, len(layers), C.byref(p), out), "hac_build_unified")
+    fmts = []
+    for (kind, _), W, h in zip(layers, mats, out):
+        f = Format.__new__(Format)
+        f.kind, f._lib, f._h, f._device_buffer = kind, lib, C.c_void_p(h), None
+        f.n, f.m = W.shape
+        fmts.append(f)
+    return fmts
 
 
 def _dot_strides(x, y, m, layout):

@@ -596,15 +596,28 @@ void finish_derived(Format& f) {
     }
 }
 
-int build_impl(const float* W, int64_t n, int64_t m, int64_t ldw, const hac_build_params* p,
-                      bool sparse, Format& f) {
-    if (!W || !p || n < 1 || m < 1 || ldw < m) return HAC_ERR_INVALID_ARG;
+// One matrix on its way through the builder: checked, copied column-major and pruned (Sect. III-B).
+struct Layer {
+    Format* f = nullptr;
+    std::vector<float> col;          // pruned weights, column-major
+    int64_t first = 0;               // position of its first non-null weight among those of all layers
+};
+
+static int check_params(const hac_build_params* p) {
+    if (!p) return HAC_ERR_INVALID_ARG;
     if (!(p->sparsity >= 0.0 && p->sparsity < 1.0) || p->reserved != 0) return HAC_ERR_INVALID_ARG;
     if (p->quantizer > HAC_QUANT_PWS) return HAC_ERR_INVALID_ARG;
     if (p->quantizer == HAC_QUANT_KMEANS && p->k < 1) return HAC_ERR_INVALID_ARG;
     if (p->quantizer >= HAC_QUANT_UNIFORM && p->k < 2) return HAC_ERR_INVALID_ARG;
     if (p->seg_symbols > HAC_MAX_SEG_SYMBOLS) return HAC_ERR_INVALID_ARG;
     if (p->ri_bits != 0 && p->ri_bits != 16 && p->ri_bits != 32) return HAC_ERR_INVALID_ARG;
+    return HAC_OK;
+}
+
+static int prepare_layer(const float* W, int64_t n, int64_t m, int64_t ldw, const hac_build_params* p, bool sparse,
+                         Layer& L) {
+    Format& f = *L.f;
+    if (!W || n < 1 || m < 1 || ldw < m) return HAC_ERR_INVALID_ARG;
     if (n > (int64_t)1 << 31 || m > (int64_t)1 << 31 || n * m > ((int64_t)1 << 36))
         return HAC_ERR_OFFSET_OVERFLOW;
     f.sparse = sparse;
@@ -615,7 +628,8 @@ int build_impl(const float* W, int64_t n, int64_t m, int64_t ldw, const hac_buil
     const int64_t total = n * m;
 
     // column-major copy, input checks
-    std::vector<float> col(total);
+    std::vector<float>& col = L.col;
+    col.resize(total);
     for (int64_t i = 0; i < n; ++i) {
         const float* row = W + i * ldw;
         for (int64_t j = 0; j < m; ++j) {
@@ -653,64 +667,29 @@ int build_impl(const float* W, int64_t n, int64_t m, int64_t ldw, const hac_buil
         if (f.ri_bits == 16) { while (S % 4 != 2) ++S; } else { S |= 1u; }
         f.S = S;
     }
-    std::vector<double> data;
-    data.reserve(q);
-    for (int64_t t = 0; t < total; ++t)
-        if (col[t] != 0.0f) data.push_back((double)col[t]);
+    return HAC_OK;
+}
 
-    Shared sh;
-    if (q > 0) {
-        int rc = HAC_OK;
-        if (p->quantizer == HAC_QUANT_KMEANS) rc = share_kmeans(data, p->k, p->kmeans_iters, p->seed, sh);
-        else if (p->quantizer == HAC_QUANT_UNIFORM) rc = share_uniform(data, p->k, sh);
-        else if (p->quantizer == HAC_QUANT_GRID) rc = share_grid(data, p->k, sh);
-        else if (p->quantizer == HAC_QUANT_PWS) rc = share_pws(data, p->k, p->seed, sh);
-        else rc = share_none(data, sh);
-        if (rc != HAC_OK) return rc;
-    }
-    std::vector<double>().swap(data);
-    for (float& v : sh.level_value) if (v == 0.0f) v = 0.0f;           // -0.0 -> +0.0
-
-    // alphabet: occupied levels (plus zero for HAC when a null entry exists), merged by value
-    const size_t nlev = sh.level_value.size();
-    std::vector<int64_t> level_count(nlev, 0);
-    for (int64_t t = 0; t < q; ++t) level_count[sh.level_of[t]]++;
-    std::vector<float> values;
-    for (size_t l = 0; l < nlev; ++l) if (level_count[l] > 0) values.push_back(sh.level_value[l]);
-    const int64_t nulls = total - q;
-    if (!sparse && nulls > 0) values.push_back(0.0f);
-    std::sort(values.begin(), values.end());
-    values.erase(std::unique(values.begin(), values.end()), values.end());
-    if (values.size() > HAC_MAX_SYMBOLS) return HAC_ERR_K_TOO_LARGE;
-    f.codebook = values;
+// Sect. IV-B / IV-C: emit the code words of one matrix column by column with the given code, recording the
+// offset index on the way.  level_of: the shared level of each of its non-null weights, in column-major order.
+static int emit_layer(Layer& L, const uint32_t* level_of, const std::vector<uint32_t>& level_symbol, uint32_t zero_symbol,
+                      const std::vector<float>& values, const std::vector<uint8_t>& code_len, const std::vector<uint32_t>& codes) {
+    Format& f = *L.f;
+    const std::vector<float>& col = L.col;
+    const bool sparse = f.sparse;
+    const int64_t n = f.n, m = f.m, total = n * m, q = f.nnz;
     const uint32_t k_eff = (uint32_t)values.size();
-    std::vector<uint32_t> level_symbol(nlev, 0);
-    for (size_t l = 0; l < nlev; ++l)
-        level_symbol[l] = (uint32_t)(std::lower_bound(values.begin(), values.end(), sh.level_value[l]) -
-                                     values.begin());
-    uint32_t zero_symbol = 0;
-    if (!sparse && nulls > 0)
-        zero_symbol = (uint32_t)(std::lower_bound(values.begin(), values.end(), 0.0f) - values.begin());
+    f.codebook = values;
+    f.code_len = code_len;
+    f.codes = codes;
     f.counts.assign(k_eff, 0);
-    for (size_t l = 0; l < nlev; ++l) if (level_count[l] > 0) f.counts[level_symbol[l]] += level_count[l];
-    if (!sparse && nulls > 0) f.counts[zero_symbol] += nulls;
-
-    int rc = huffman_code_lengths(f.counts, f.code_len);
-    if (rc != HAC_OK) return rc;
-    canonical_assign(f.code_len, f.codes);
     f.max_len = 0; f.min_len = k_eff ? 255 : 0;
     for (uint8_t l : f.code_len) { f.max_len = std::max<uint32_t>(f.max_len, l); f.min_len = std::min<uint32_t>(f.min_len, l); }
     if ((uint64_t)f.S * f.max_len > 65535u) return HAC_ERR_OFFSET_OVERFLOW;   // sub_bits is 16 bit
 
-    // Sect. IV-B / IV-C: emit the code words column by column, recording the offset index on the way
     const uint32_t S = f.S;
     BitWriter bw(f.stream);
     f.symbols = sparse ? q : total;
-    {
-        double expect = 0;
-        for (uint32_t s = 0; s < k_eff; ++s) expect += (double)f.counts[s] * f.code_len[s];
-        f.stream.reserve((size_t)(expect / 32) + 16);
-    }
     if (sparse) {
         f.cb.assign(m + 1, 0);
         f.seg_first.assign(m + 1, 0);
@@ -741,11 +720,12 @@ int build_impl(const float* W, int64_t n, int64_t m, int64_t ldw, const hac_buil
         for (int64_t i = 0; i < n; ++i) {
             const bool stored = (c[i] != 0.0f);
             uint32_t s;
-            if (stored) s = level_symbol[sh.level_of[w++]];
+            if (stored) s = level_symbol[level_of[w++]];
             else if (sparse) continue;
             else s = zero_symbol;
             open_segment_if_needed();
             bw.put(f.codes[s], f.code_len[s]);
+            f.counts[s]++;
             if (sparse) { if (f.ri_bits == 16) f.ri16.push_back((uint16_t)i); else f.ri32.push_back((uint32_t)i); }
             if (++in_sub == S) close_sub();
         }
@@ -764,6 +744,81 @@ int build_impl(const float* W, int64_t n, int64_t m, int64_t ldw, const hac_buil
 
     finish_derived(f);
     return HAC_OK;
+}
+
+// Weight sharing over the non-null weights of all the layers at once (one layer: Sect. III-C; several: the unified
+// quantization of Sect. V-D, one k and one dictionary for all of them), one Huffman code on the symbol counts of all the
+// streams together, then every layer emitted with that code.  A layer keeps the whole shared codebook and code and its
+// own symbol counts.
+int build_layers(std::vector<Layer>& layers, const hac_build_params* p) {
+    std::vector<double> data;
+    int64_t q_all = 0, nulls_in_hac = 0;
+    for (Layer& L : layers) {
+        L.first = q_all;
+        q_all += L.f->nnz;
+        if (!L.f->sparse) nulls_in_hac += L.f->n * L.f->m - L.f->nnz;
+    }
+    data.reserve(q_all);
+    for (const Layer& L : layers)
+        for (float v : L.col)
+            if (v != 0.0f) data.push_back((double)v);
+
+    Shared sh;
+    if (q_all > 0) {
+        int rc = HAC_OK;
+        if (p->quantizer == HAC_QUANT_KMEANS) rc = share_kmeans(data, p->k, p->kmeans_iters, p->seed, sh);
+        else if (p->quantizer == HAC_QUANT_UNIFORM) rc = share_uniform(data, p->k, sh);
+        else if (p->quantizer == HAC_QUANT_GRID) rc = share_grid(data, p->k, sh);
+        else if (p->quantizer == HAC_QUANT_PWS) rc = share_pws(data, p->k, p->seed, sh);
+        else rc = share_none(data, sh);
+        if (rc != HAC_OK) return rc;
+    }
+    std::vector<double>().swap(data);
+    for (float& v : sh.level_value) if (v == 0.0f) v = 0.0f;           // -0.0 -> +0.0
+
+    // alphabet: occupied levels (plus zero when a HAC layer has a null entry), merged by value.  A stored entry of an
+    // sHAC layer is counted like any other occurrence of its value.
+    const size_t nlev = sh.level_value.size();
+    std::vector<int64_t> level_count(nlev, 0);
+    for (int64_t t = 0; t < q_all; ++t) level_count[sh.level_of[t]]++;
+    std::vector<float> values;
+    for (size_t l = 0; l < nlev; ++l) if (level_count[l] > 0) values.push_back(sh.level_value[l]);
+    if (nulls_in_hac > 0) values.push_back(0.0f);
+    std::sort(values.begin(), values.end());
+    values.erase(std::unique(values.begin(), values.end()), values.end());
+    if (values.size() > HAC_MAX_SYMBOLS) return HAC_ERR_K_TOO_LARGE;
+    const uint32_t k_eff = (uint32_t)values.size();
+    std::vector<uint32_t> level_symbol(nlev, 0);
+    for (size_t l = 0; l < nlev; ++l)
+        level_symbol[l] = (uint32_t)(std::lower_bound(values.begin(), values.end(), sh.level_value[l]) -
+                                     values.begin());
+    uint32_t zero_symbol = 0;
+    if (nulls_in_hac > 0)
+        zero_symbol = (uint32_t)(std::lower_bound(values.begin(), values.end(), 0.0f) - values.begin());
+    std::vector<int64_t> counts(k_eff, 0);
+    for (size_t l = 0; l < nlev; ++l) if (level_count[l] > 0) counts[level_symbol[l]] += level_count[l];
+    if (nulls_in_hac > 0) counts[zero_symbol] += nulls_in_hac;
+
+    std::vector<uint8_t> code_len;
+    std::vector<uint32_t> codes;
+    int rc = huffman_code_lengths(counts, code_len);
+    if (rc != HAC_OK) return rc;
+    canonical_assign(code_len, codes);
+    for (Layer& L : layers) {
+        rc = emit_layer(L, sh.level_of.data() + L.first, level_symbol, zero_symbol, values, code_len, codes);
+        if (rc != HAC_OK) return rc;
+        std::vector<float>().swap(L.col);
+    }
+    return HAC_OK;
+}
+
+int build_impl(const float* W, int64_t n, int64_t m, int64_t ldw, const hac_build_params* p,
+                      bool sparse, Format& f) {
+    if (int rc = check_params(p)) return rc;
+    std::vector<Layer> layers(1);
+    layers[0].f = &f;
+    if (int rc = prepare_layer(W, n, m, ldw, p, sparse, layers[0])) return rc;
+    return build_layers(layers, p);
 }
 
 // Host decoder (canonical decoding by lengths, one symbol at a time); used by *_decode_host.
@@ -990,7 +1045,7 @@ static int deserialize(const void* buf, size_t bytes, bool want_sparse, Format& 
     uint64_t total_count = 0, total_bits = 0;
     for (uint64_t s = 0; s < k; ++s) {
         const uint32_t l = f.code_len[s];
-        if (l < 1 || l > (uint32_t)kMaxCodeLen || f.counts[s] < 1) return HAC_ERR_CORRUPT;
+        if (l < 1 || l > (uint32_t)kMaxCodeLen || f.counts[s] < 0) return HAC_ERR_CORRUPT;   // 0: a symbol of a shared code that this matrix lacks
         if (!std::isfinite(f.codebook[s]) || (s > 0 && !(f.codebook[s] > f.codebook[s - 1]))) return HAC_ERR_CORRUPT;
         kraft += std::ldexp((long double)1, -(int)l);
         total_count += (uint64_t)f.counts[s]; total_bits += (uint64_t)f.counts[s] * l;
@@ -1127,6 +1182,29 @@ int shac_build(const float* W, int64_t n, int64_t m, int64_t ldw, const hac_buil
     if (rc != HAC_OK) { delete h; return rc; }
     *out = h;
     return HAC_OK;
+}
+
+int hac_build_unified(const hac_unified_layer* layers, int n_layers, const hac_build_params* params, void** out) {
+    if (!layers || !out || n_layers < 1 || n_layers > HAC_MAX_UNIFIED_LAYERS) return HAC_ERR_INVALID_ARG;
+    for (int i = 0; i < n_layers; ++i) out[i] = nullptr;
+    if (int rc = hacb200::check_params(params)) return rc;
+    // hac_format and shac_format hold the same thing; which one a layer's handle is follows its `sparse` field
+    std::vector<hac_format*> hs;
+    std::vector<shac_format*> ss;
+    auto drop = [&]() { for (auto* h : hs) delete h; for (auto* h : ss) delete h; for (int i = 0; i < n_layers; ++i) out[i] = nullptr; };
+    int rc = HAC_OK;
+    try {
+        std::vector<hacb200::Layer> ls((size_t)n_layers);
+        for (int i = 0; i < n_layers && rc == HAC_OK; ++i) {
+            if (layers[i].sparse != 0 && layers[i].sparse != 1) { rc = HAC_ERR_INVALID_ARG; break; }
+            if (layers[i].sparse) { ss.push_back(new shac_format()); ls[i].f = &ss.back()->f; out[i] = ss.back(); }
+            else { hs.push_back(new hac_format()); ls[i].f = &hs.back()->f; out[i] = hs.back(); }
+            rc = hacb200::prepare_layer(layers[i].W, layers[i].n, layers[i].m, layers[i].ldw, params, layers[i].sparse != 0, ls[i]);
+        }
+        if (rc == HAC_OK) rc = hacb200::build_layers(ls, params);
+    } catch (const std::bad_alloc&) { rc = HAC_ERR_ALLOC; }
+    if (rc != HAC_OK) drop();
+    return rc;
 }
 
 int hac_sizes(const hac_format* f, hac_size_report* out) {

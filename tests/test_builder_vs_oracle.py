@@ -318,3 +318,49 @@ def test_comparison_encoders_reject_bad_input():
     assert z.q == 0 and z.cb.tolist() == [0, 0, 0, 0]
     neg = IndexMap(np.array([[-0.0, 0.0], [1.0, 0.0]], dtype=np.float32), 8)
     assert neg.k == 2                                        # -0.0 and 0.0 are one value
+
+
+# ---------------------------------------------------------------- unified quantization (Sect. V-D)
+@pytest.mark.parametrize("quantizer,k", [(si.QUANT_KMEANS, 12), (si.QUANT_UNIFORM, 40), (si.QUANT_PWS, 9), (si.QUANT_GRID, 16)])
+def test_unified_build_bit_exact(quantizer, k):
+    """Three matrices of different shapes, HAC and sHAC mixed, quantized together: every array of every format against
+    the oracle, and every format usable on its own (host decode, serialization)."""
+    shapes = [("hac", si.scaled(si.CFG2_DENSE_HAC, 300, 40)), ("shac", si.scaled(si.CFG3_FC_SHAC, 900, 30)),
+              ("hac", si.scaled(si.CFG4_CONV, 200, 10))]
+    Ws = [si.weights(wl) for _, wl in shapes]
+    sparsity, iters, seed = 0.7, 6, 11
+    parts = orc.quantize_unified(Ws, sparsity, k, quantizer, iters, seed)
+    ofmts = orc.unified_encode([(kind, Wq, mask) for (kind, _), (Wq, mask) in zip(shapes, parts)])
+    lfs = hb.hac_build_unified([(kind, W) for (kind, _), W in zip(shapes, Ws)], sparsity=sparsity, k=k, quantizer=quantizer,
+                               kmeans_iters=iters, seed=seed)
+    for lf, ofmt, (Wq, mask) in zip(lfs, ofmts, parts):
+        S_eff = lf.sizes()["seg_symbols"]
+        oidx = orc.hac_offset_index(ofmt, S_eff) if lf.kind == "hac" else orc.shac_offset_index(ofmt, S_eff)
+        assert_same_format(lf, ofmt, oidx, Wq)
+        back = hb.Format.deserialize(lf.kind, lf.serialize())
+        assert np.array_equal(back.decode_host().view(np.uint32), Wq.view(np.uint32))
+    # the dictionary is one for all: the same codebook and code in every format
+    e = [lf.export() for lf in lfs]
+    assert all(np.array_equal(x["codebook"], e[0]["codebook"]) and np.array_equal(x["codes"], e[0]["codes"]) for x in e)
+    total = sum(x["counts"] for x in e)
+    assert np.array_equal(total, ofmts[0]["shared_counts"]) and (total > 0).all()
+
+
+def test_unified_build_on_the_hand_worked_example_and_bad_arguments():
+    from golden_io import golden, read_sections
+    g = read_sections(golden("unified_hand_worked.txt"))
+    mat = lambda key: np.array([[float(v) for v in row] for row in g[key]], dtype=np.float32)
+    lfs = hb.hac_build_unified([("hac", mat("A")), ("hac", mat("B")), ("shac", mat("C"))], quantizer=si.QUANT_NONE)
+    words = [int(v, 0) for v in g["words"][0]]
+    for lf, word, bits, own in zip(lfs, words, g["bits"][0], g["own_counts"]):
+        e = lf.export()
+        assert e["stream"][0] == word and e["stream_bits"] == int(bits) and e["counts"].tolist() == [int(v) for v in own]
+        assert e["code_len"].tolist() == [int(v) for v in g["lengths"][0]]
+    one = hb.hac_build_unified([("hac", mat("A"))], quantizer=si.QUANT_NONE)[0].export()
+    assert one["stream_bits"] == int(g["A_alone_bits"][0][0])
+    with pytest.raises(hb.HacError):
+        hb.hac_build_unified([], quantizer=si.QUANT_NONE)
+    bad = mat("A").copy(); bad[0, 0] = np.inf
+    with pytest.raises(hb.HacError) as err:
+        hb.hac_build_unified([("hac", mat("B")), ("hac", bad)], quantizer=si.QUANT_NONE)
+    assert err.value.status == -3

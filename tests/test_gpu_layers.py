@@ -134,3 +134,42 @@ def test_chain_of_layers(scale, batches):
             _check(g[None] if B == 1 else g.T, y_ref, a)
             cur = got
         assert torch.equal(cur, y), "the chained submission must give what the layers give one by one"
+
+
+def test_chain_of_layers_with_one_dictionary():
+    """The same stack (scaled down) quantized together (unified quantization, Sect. V-D): one codebook and one code for the
+    three layers, every layer multiplied from its own stream, layer by layer against the oracle."""
+    specs = fc_stack(4)
+    Ws = [si.weights(wl) for wl, _, _ in specs]
+    sparsity, k, iters, seed = 0.8, 48, 8, 5
+    parts = orc.quantize_unified(Ws, sparsity, k, si.QUANT_KMEANS, iters, seed)
+    lfs = hb.hac_build_unified([(kind, W) for (_, kind, _), W in zip(specs, Ws)], sparsity=sparsity, k=k,
+                               quantizer=si.QUANT_KMEANS, kmeans_iters=iters, seed=seed)
+    cb0 = lfs[0].export()["codebook"]
+    rng = np.random.default_rng(98)
+    layers, oracle_layers = [], []
+    for lf, (wl, _, relu), (Wq, _) in zip(lfs, specs, parts):
+        assert np.array_equal(lf.export()["codebook"], cb0)
+        lf.upload()
+        assert np.array_equal(lf.decode_host().view(np.uint32), Wq.view(np.uint32))
+        if lf.kind == "hac":                                  # the kernels' decoder with a code that has unused symbols
+            got = lf.debug_decode().cpu().numpy()
+            assert np.array_equal(got.view(np.uint32), np.ascontiguousarray(Wq.T).view(np.uint32))
+        bias = (rng.standard_normal(wl.m) * 0.1).astype(np.float32)
+        layers.append((lf, torch.from_numpy(bias).cuda(), relu))
+        oracle_layers.append((Wq, bias, relu))
+    n0 = Ws[0].shape[0]
+    for B in (1, 8):
+        X = np.maximum(np.random.default_rng(B).standard_normal((B, n0)), 0).astype(np.float32)
+        xin = torch.from_numpy(X[0] if B == 1 else np.ascontiguousarray(X.T)).cuda()
+        y, _ = hb.hac_chain(layers, xin)
+        cur = xin
+        for (lf, bias_d, relu), (Wq, bias, _) in zip(layers, oracle_layers):
+            got = lf.dot(cur, bias=bias_d, relu=relu)
+            inp = cur.cpu().numpy()
+            inp = inp[None] if B == 1 else inp.T
+            y_ref, a = orc.layer_definition(Wq, inp, bias, relu)
+            g = got.cpu().numpy()
+            _check(g[None] if B == 1 else g.T, y_ref, a)
+            cur = got
+        assert torch.equal(cur, y)

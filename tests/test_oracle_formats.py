@@ -231,3 +231,71 @@ def test_comparison_formats_agree_with_the_definition():
     nz, ri, cb = orc.csc(W, W != 0)
     y, a = orc.dot_csc(nz, ri, cb, 60, X)
     assert np.array_equal(y, y_ref) and np.array_equal(a, a_ref)
+
+
+# ---------------------------------------------------------------- unified quantization (Sect. V-D)
+def _unified_golden():
+    from golden_io import golden, read_sections
+    g = read_sections(golden("unified_hand_worked.txt"))
+    mat = lambda key: np.array([[float(v) for v in row] for row in g[key]], dtype=np.float32)
+    ints = lambda key: [[int(v, 0) for v in row] for row in g[key]]
+    return g, mat, ints
+
+
+def test_unified_code_on_the_hand_worked_example():
+    g, mat, ints = _unified_golden()
+    A, B, Cm = mat("A"), mat("B"), mat("C")
+    fmts = orc.unified_encode([("hac", A, A != 0), ("hac", B, B != 0), ("shac", Cm, Cm != 0)])
+    for f, bits, word, own in zip(fmts, ints("bits")[0], ints("words")[0], ints("own_counts")):
+        assert f["codebook"].tolist() == [float(v) for v in g["codebook"][0]]
+        assert f["shared_counts"].tolist() == ints("counts")[0]
+        assert f["code_len"].tolist() == ints("lengths")[0] and f["codes"].tolist() == ints("codes")[0]
+        assert f["bits"] == bits and f["words"].tolist() == [word] and f["counts"].tolist() == own
+    assert fmts[2]["ri"].tolist() == ints("ri")[0] and fmts[2]["cb"].tolist() == ints("cb")[0]
+    assert orc.hac_encode(A)["bits"] == ints("A_alone_bits")[0][0]        # its own code would be shorter for A
+    assert orc.unified_paper_bits(fmts) == ints("unified_paper_bits")[0][0]
+    # every stream decodes back with the shared code
+    assert np.array_equal(orc.hac_decode(fmts[0]), A) and np.array_equal(orc.hac_decode(fmts[1]), B)
+    assert np.array_equal(orc.shac_decode(fmts[2]), Cm)
+
+
+def test_unified_of_one_matrix_is_the_ordinary_format():
+    rng = np.random.default_rng(3)
+    W = rng.standard_normal((40, 12)).astype(np.float32)
+    for quantizer in (1, 2, 3, 4):
+        (Wq, mask), = orc.quantize_unified([W], 0.5, 8, quantizer, 5, 7)
+        Wq1, mask1 = orc.quantize(W, 0.5, 8, quantizer, 5, 7)
+        assert np.array_equal(Wq.view(np.uint32), Wq1.view(np.uint32)) and np.array_equal(mask, mask1)
+    for kind in ("hac", "shac"):
+        u, = orc.unified_encode([(kind, Wq1, mask1)])
+        o = orc.hac_encode(Wq1) if kind == "hac" else orc.shac_encode(Wq1, mask1)
+        for key in ("codebook", "code_len", "codes", "counts", "words"):
+            assert np.array_equal(u[key], o[key]), key
+        assert u["bits"] == o["bits"]
+
+
+def test_unified_over_the_column_halves_of_a_matrix_is_the_matrix():
+    """Cutting a matrix between two columns and quantizing the halves together must change nothing: the weights reach the
+    sharing in the same order, the counts add up to the same code, and the two streams are the whole stream cut in two."""
+    rng = np.random.default_rng(4)
+    W = rng.standard_normal((30, 10)).astype(np.float32)
+    W[np.abs(W) < 0.4] = 0                                   # already sparse: pruning (per matrix) stays off
+    for quantizer in (1, 2, 4):
+        whole, mask = orc.quantize(W, 0.0, 6, quantizer, 4, 9)
+        (L, mL), (R, mR) = orc.quantize_unified([W[:, :4], W[:, 4:]], 0.0, 6, quantizer, 4, 9)
+        assert np.array_equal(np.hstack([L, R]).view(np.uint32), whole.view(np.uint32))
+        fw = orc.hac_encode(whole)
+        fl, fr = orc.unified_encode([("hac", L, mL), ("hac", R, mR)])
+        assert np.array_equal(fl["code_len"], fw["code_len"]) and np.array_equal(fl["codes"], fw["codes"])
+        assert np.array_equal(np.concatenate([fl["sym"], fr["sym"]]), fw["sym"]) and fl["bits"] + fr["bits"] == fw["bits"]
+        assert np.array_equal(fl["counts"] + fr["counts"], fw["counts"])
+
+
+def test_unified_sharing_uses_one_set_of_values():
+    rng = np.random.default_rng(5)
+    Ws = [rng.standard_normal((20, 8)).astype(np.float32), (3 * rng.standard_normal((16, 5))).astype(np.float32)]
+    parts = orc.quantize_unified(Ws, 0.25, 4, 1, 10, 1)
+    values = np.unique(np.concatenate([Wq[mask] for Wq, mask in parts]))
+    assert len(values) <= 4                                   # k values for all matrices together, not per matrix
+    for (Wq, mask), W in zip(parts, Ws):
+        assert abs((~mask).mean() - 0.25) < 0.02             # each matrix pruned on its own
