@@ -741,9 +741,9 @@ def dot_csc(nz, ri, cb, n: int, X: np.ndarray):
 # ----------------------------------------------------------------------------
 def quantize_unified(Ws, sparsity: float, k: int, quantizer: int, iters: int = 20, seed: int = 0):
     """Every matrix pruned on its own (Sect. III-B), then ONE run of the weight sharing over the non-null weights of all
-    of them, listed matrix after matrix and column-major inside each (reading: the paper says the matrices are quantized
-    "at the same time using a unique value of k"; the order only matters for the seeded start of k-means and the random
-    draws of PWS).  Returns a list of (Wq, mask)."""
+    of them, listed matrix after matrix and column-major inside each (reading: the paper only says that the matrices are
+    quantized together with a single k; the order only matters for the seeded start of k-means and the random draws of
+    PWS).  Returns a list of (Wq, mask)."""
     pruned = [prune(W, sparsity) for W in Ws]
     parts = [_nonnull_colmajor(Wp) for Wp in pruned]
     if sum(d.size for d, _ in parts) == 0:
