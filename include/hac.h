@@ -258,6 +258,10 @@ int shac_attach(shac_format* f, void* dev_buf, size_t dev_bytes);
  *   results    A batched product on the tensor cores rounds every weight and input to two TF32 parts
  *              (three partial products, error about 1e-7 of sum |w x|).  If a bounded wait inside
  *              that kernel ever ran out (it never has), the outputs of the affected block are NaN.
+ *              x is expected to be finite.  A NaN or Inf in x[i] reaches every output whose column stores row i,
+ *              as the definition says, and may also reach outputs whose column has a zero there: HAC multiplies
+ *              its coded zeros (except where a run of them is skipped), the tensor-core tiles and the batched sHAC
+ *              kernel pad with zero weights, and 0 * Inf is NaN.
  * Asynchronous on cuda_stream.  The kernels are launched with programmatic stream serialization:
  * they may begin fetching the uploaded format while the kernel before them in the stream is still
  * finishing, but read x and the workspace and write y only once that kernel has completed, so the
