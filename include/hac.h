@@ -375,8 +375,8 @@ int hac_dot_noalloc(const hac_format* f, const float* x, int64_t batch, int64_t 
  * hac_index_map_dot - y = x^T W with W[i][j] = codebook[index[j*n + i]], all pointers device memory,
  *   x and y with the strides of hac_dot, fp32 products and sums, asynchronous on cuda_stream.  A
  *   pointer at or beyond k reads the last codebook entry (two-byte pointers) or 0 (one-byte pointers).
- *   128-bit loads of the pointers are used when n is a multiple of 16 / index_bits * 8 and index_dev is
- *   16-byte aligned; otherwise element loads.  Needs no workspace.
+ *   128-bit loads of the pointers are used when n is a multiple of 16 (one-byte pointers) or 8 (two-byte)
+ *   and index_dev is 16-byte aligned; otherwise element loads.  Needs no workspace.
  *
  * shac_csc_encode - CSC of Wq: the nonzero weights column by column, rows ascending, into nz, their rows
  *   into ri, and the m+1 column boundaries into cb; their number into *q.  With nz, ri and cb all NULL

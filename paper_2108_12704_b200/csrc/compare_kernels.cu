@@ -85,44 +85,51 @@ index_map8_kernel(const uint8_t* __restrict__ index, const float* __restrict__ c
     }
 }
 
-// One input, x contiguous and small enough for shared memory: x is staged once per block, a lane takes four consecutive
-// pointers (one 32-bit load) and the four matching elements of x (one 128-bit load, lanes on disjoint banks), four such
-// groups in flight per step.
+// One input, x contiguous and small enough for shared memory: x is staged once per block, a lane takes sixteen consecutive
+// pointers (one 128-bit load, two of them in flight) and the sixteen matching elements of x.  x is stored with four padding
+// words after every sixteen, so that the 128-bit reads of the eight lanes of a quarter-warp, 16 elements apart, fall on
+// disjoint banks.
 constexpr int kVecThreads = 512;
 constexpr int kVecWarps = kVecThreads / 32;
+__host__ __device__ constexpr int64_t padded_x(int64_t i) { return i + (i >> 4) * 4; }
 
 __global__ void __launch_bounds__(kVecThreads)
 index_map8_vec_kernel(const uint8_t* __restrict__ index, const float* __restrict__ codebook, int k, int64_t n, int64_t m,
                       const float* __restrict__ x, float* __restrict__ y, int64_t y_stride_j) {
     extern __shared__ __align__(16) float smem[];
     float* cb_s = smem;                                   // [256][32]
-    float* x_s = smem + 256 * kCodebookCopies;            // [n rounded up to 4]
+    float* x_s = smem + 256 * kCodebookCopies;            // [padded_x(n)]
     for (int e = threadIdx.x; e < 256 * kCodebookCopies; e += kVecThreads) {
         const int entry = e / kCodebookCopies;
         cb_s[e] = entry < k ? codebook[entry] : 0.0f;
     }
-    for (int64_t i = threadIdx.x; i < n; i += kVecThreads) x_s[i] = __ldg(x + i);
+    for (int64_t i = threadIdx.x; i < n; i += kVecThreads) x_s[padded_x(i)] = __ldg(x + i);
     __syncthreads();
     const int lane = threadIdx.x & 31;
     const float* mine = cb_s + lane;
     const int64_t warp = (int64_t)blockIdx.x * kVecWarps + (threadIdx.x >> 5);
     const int64_t warps = (int64_t)gridDim.x * kVecWarps;
-    const int64_t groups = n / 4;                         // n is a multiple of 4 here
+    const int64_t groups = n / 16;                        // n is a multiple of 16 here
     for (int64_t j = warp; j < m; j += warps) {
-        const uint32_t* col = reinterpret_cast<const uint32_t*>(index + j * n);
+        const uint4* col = reinterpret_cast<const uint4*>(index + j * n);
         float acc0 = 0.0f, acc1 = 0.0f;
-        for (int64_t g0 = lane; g0 < groups; g0 += 4 * 32) {
-            uint32_t p[4];
+        for (int64_t g0 = lane; g0 < groups; g0 += 2 * 32) {
+            uint4 p[2];
 #pragma unroll
-            for (int u = 0; u < 4; ++u) p[u] = g0 + 32 * u < groups ? __ldg(col + g0 + 32 * u) : 0u;
+            for (int u = 0; u < 2; ++u) p[u] = g0 + 32 * u < groups ? __ldg(col + g0 + 32 * u) : make_uint4(0u, 0u, 0u, 0u);
 #pragma unroll
-            for (int u = 0; u < 4; ++u) {
+            for (int u = 0; u < 2; ++u) {
                 if (g0 + 32 * u < groups) {
-                    const float4 xv = *reinterpret_cast<const float4*>(x_s + 4 * (g0 + 32 * u));
-                    acc0 = fmaf(mine[(p[u] & 0xffu) * kCodebookCopies], xv.x, acc0);
-                    acc1 = fmaf(mine[((p[u] >> 8) & 0xffu) * kCodebookCopies], xv.y, acc1);
-                    acc0 = fmaf(mine[((p[u] >> 16) & 0xffu) * kCodebookCopies], xv.z, acc0);
-                    acc1 = fmaf(mine[(p[u] >> 24) * kCodebookCopies], xv.w, acc1);
+                    const float* xg = x_s + 20 * (g0 + 32 * u);
+                    const uint32_t w4[4] = {p[u].x, p[u].y, p[u].z, p[u].w};
+#pragma unroll
+                    for (int t = 0; t < 4; ++t) {
+                        const float4 xv = *reinterpret_cast<const float4*>(xg + 4 * t);
+                        acc0 = fmaf(mine[(w4[t] & 0xffu) * kCodebookCopies], xv.x, acc0);
+                        acc1 = fmaf(mine[((w4[t] >> 8) & 0xffu) * kCodebookCopies], xv.y, acc1);
+                        acc0 = fmaf(mine[((w4[t] >> 16) & 0xffu) * kCodebookCopies], xv.z, acc0);
+                        acc1 = fmaf(mine[(w4[t] >> 24) * kCodebookCopies], xv.w, acc1);
+                    }
                 }
             }
         }
@@ -332,10 +339,10 @@ int hac_index_map_dot(const void* index_dev, int index_bits, const float* codebo
     if (int rc = grid_for(m, &grid)) return rc;
     cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
     const Strides st{x_stride_i, x_stride_b, y_stride_j, y_stride_b};
-    if (index_bits == 8 && batch == 1 && x_stride_i == 1 && n % 4 == 0 && reinterpret_cast<uintptr_t>(index_dev) % 4 == 0) {
+    if (index_bits == 8 && batch == 1 && x_stride_i == 1 && n % 16 == 0 && reinterpret_cast<uintptr_t>(index_dev) % 16 == 0) {
         int sms = 0, optin = 0, vgrid = 0;
         if (int rc = device_limits(&sms, &optin)) return rc;
-        const size_t smem = ((size_t)256 * kCodebookCopies + (size_t)n) * sizeof(float);
+        const size_t smem = ((size_t)256 * kCodebookCopies + (size_t)padded_x(n)) * sizeof(float);
         if (staged_x_shape(m, smem, sms, optin, &vgrid)) {
             cudaError_t e = cudaFuncSetAttribute(index_map8_vec_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
             if (e != cudaSuccess) return cuda_error(e, "cudaFuncSetAttribute");

@@ -351,3 +351,24 @@ print("ok")
     root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
     out = subprocess.run([sys.executable, "-c", code], cwd=root, env=env, capture_output=True, text=True, timeout=600)
     assert out.returncode == 0 and "ok" in out.stdout, out.stdout + out.stderr
+
+
+def test_column_shards_give_the_whole_product():
+    """Column sharding (one product split over several GPUs) on one GPU: the shards of two and three ranks are multiplied one
+    after the other and their slices put side by side; the exchange itself is covered by the two-rank CPU test."""
+    from paper_2108_12704_b200.sharded import ColumnSharded
+    wl = si.scaled(si.CFG3_FC_SHAC, 3000, 101)
+    W = si.weights(wl)
+    Wq, mask = orc.quantize(W, wl.sparsity, wl.k, wl.quantizer, wl.kmeans_iters, wl.seed)
+    quant = dict(sparsity=wl.sparsity, k=wl.k, quantizer=wl.quantizer, kmeans_iters=wl.kmeans_iters, seed=wl.seed)
+    X = si.inputs(wl, 5)
+    y_ref, a = orc.dot_definition(Wq, X)
+    for kind in ("shac", "hac"):
+        for world in (1, 2, 3):
+            slices = []
+            for rank in range(world):
+                sh = ColumnSharded(kind, W, rank, world, **quant).upload()
+                slices.append(sh.format.dot(torch.from_numpy(np.ascontiguousarray(X.T)).cuda()).cpu().numpy().T)
+            check_outputs(np.concatenate(slices, axis=1), y_ref, a)
+    one = ColumnSharded("shac", W, 0, 1, **quant).upload()
+    check_outputs(one.dot(torch.from_numpy(X[0]).cuda()).cpu().numpy()[None], y_ref[:1], a[:1])
