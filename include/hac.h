@@ -429,6 +429,12 @@ const char* hac_status_string(int status);
 /* Text of the last CUDA error seen by this library on the calling thread ("" if none). */
 const char* hac_last_cuda_error(void);
 
+/* Number of thread blocks of the batched tensor-core kernel, on the current device since the library was loaded, in which
+ * a bounded wait ran out (the affected outputs were set to NaN, see hac_dot).  0 is the only value ever observed; a caller that
+ * finds NaN in y can tell a lost wait from NaN inputs with it.  Synchronous: a cudaMemcpyFromSymbol, which waits for the
+ * device work submitted before it on blocking streams.  Errors: HAC_ERR_INVALID_ARG, HAC_ERR_CUDA. */
+int hac_lost_waits(unsigned int* count);
+
 /* Diagnostic switches.  Environment variables, read once when the first product is launched (changing
  * them later has no effect); they select between code paths that all give the same results:
  *   HAC_B200_PDL=0          launch without programmatic stream serialization

@@ -79,7 +79,7 @@ EXPORTS = (
     "shac_dot_host", "hac_dot_host_async", "shac_dot_host_async", "hac_debug_decode", "shac_debug_decode",
     "hac_debug_table_lookup", "shac_debug_table_lookup", "hac_last_launch_count",
     "shac_last_launch_count", "hac_free", "shac_free", "hac_status_string", "hac_last_cuda_error",
-    "hac_index_map_encode", "hac_index_map_dot", "shac_csc_encode", "shac_csc_dot", "hac_build_unified",
+    "hac_index_map_encode", "hac_index_map_dot", "shac_csc_encode", "shac_csc_dot", "hac_build_unified", "hac_lost_waits",
 )
 
 
@@ -128,6 +128,7 @@ def load():
     lib.shac_csc_encode.argtypes = [fp, i64, i64, i64, fp, vp, vp, i64, C.POINTER(i64)]
     lib.shac_csc_dot.argtypes = [fp, vp, vp, i64, i64, fp, i64, i64, i64, fp, i64, i64, vp]
     lib.hac_build_unified.argtypes = [C.POINTER(UnifiedLayer), C.c_int, C.POINTER(BuildParams), C.POINTER(vp)]
+    lib.hac_lost_waits.argtypes = [C.POINTER(C.c_uint)]
     lib.hac_status_string.argtypes = [C.c_int]
     lib.hac_status_string.restype = C.c_char_p
     lib.hac_last_cuda_error.restype = C.c_char_p
@@ -403,6 +404,13 @@ def chain(layers, x, y=None, workspace=None):
     _check(lib.hac_chain(arr, len(layers), x.data_ptr(), B, y.data_ptr(), acts[0].data_ptr(), acts[1].data_ptr(), widest,
                          workspace.data_ptr(), workspace.numel(), st), "hac_chain")
     return y, last.last_launch_count()
+
+
+def lost_waits() -> int:
+    """hac_lost_waits of the C ABI."""
+    n = C.c_uint()
+    _check(load().hac_lost_waits(C.byref(n)), "hac_lost_waits")
+    return n.value
 
 
 def build_unified(layers, sparsity=0.0, k=32, quantizer=QUANT_KMEANS, kmeans_iters=20, seed=0, seg_symbols=0, ri_bits=0):

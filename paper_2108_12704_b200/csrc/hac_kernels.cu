@@ -2004,6 +2004,10 @@ __global__ void __launch_bounds__(256) hac_pack_x_kernel(DevFormat f, const floa
     *reinterpret_cast<float4*>(at + kGXLoRows) = make_float4(lo[0], lo[1], lo[2], lo[3]);
 }
 
+// Blocks of the tensor-core kernel whose bounded waits ran out since the library was loaded on this device (their
+// outputs are NaN); read by hac_lost_waits.
+static __device__ unsigned int g_lost_waits;
+
 // Warps 0..15 decode: warp w serves lane quarter q = w % 4 (columns 32q..32q+31 of the block) in
 // slot w / 4.  In every round a lane works on kGChains tasks of its column at once (independent decode
 // chains, interleaved instruction by instruction, which hides the latency of the dependent table
@@ -2319,6 +2323,7 @@ __global__ void __launch_bounds__(kGWarps * 32, 1) hac_gemm_tc_kernel(
     // one lane waits for the last commits; everyone else sleeps in the block barrier below
     if (warp == kGDecodeWarps && lane == 0 && !tc_wait_idle(bar_done, 0)) lost = true;
     const bool any_lost = __syncthreads_or((lost || *lost_flag) ? 1 : 0) != 0;
+    if (any_lost && threadIdx.x == 0) atomicAdd(&g_lost_waits, 1u);
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
     if (warp < 4) {
         // lane l of warp q holds column 32q + l; slot s accumulated its tasks in columns 64s..64s+63
@@ -3626,5 +3631,11 @@ void hac_free(hac_format* f) { delete f; }
 void shac_free(shac_format* f) { delete f; }
 
 const char* hac_last_cuda_error(void) { return g_last_cuda_error.c_str(); }
+
+int hac_lost_waits(unsigned int* count) {
+    if (!count) return HAC_ERR_INVALID_ARG;
+    HAC_CUDA(cudaMemcpyFromSymbol(count, g_lost_waits, sizeof(unsigned int)));
+    return HAC_OK;
+}
 
 }  // extern "C"

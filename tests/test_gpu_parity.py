@@ -372,3 +372,14 @@ def test_column_shards_give_the_whole_product():
             check_outputs(np.concatenate(slices, axis=1), y_ref, a)
     one = ColumnSharded("shac", W, 0, 1, **quant).upload()
     check_outputs(one.dot(torch.from_numpy(X[0]).cuda()).cpu().numpy()[None], y_ref[:1], a[:1])
+
+
+def test_no_bounded_wait_ran_out():
+    """The batched kernel marks outputs NaN and counts the block when one of its bounded waits runs out; after batched products
+    of both formats the count must still be zero and the outputs finite."""
+    from paper_2108_12704_b200.binding import lost_waits
+    for wl, kind in ((si.scaled(si.CFG2_DENSE_HAC, 2100, 300), "hac"), (si.scaled(si.CFG4_CONV, 1152, 128), "shac")):
+        lf, Wq, mask = build_both(wl, kind)
+        y = run_dot(lf, si.inputs(wl, 70))
+        assert np.isfinite(y).all()
+    assert lost_waits() == 0
