@@ -447,6 +447,8 @@ int hac_lost_waits(unsigned int* count);
  *   HAC_B200_ITEMS=0        single-input sHAC always through the older kernel
  *   HAC_B200_SHAC_TC=0|2    batched sHAC never / always on the tensor cores (default 1: by estimated cost)
  *   HAC_B200_GEMM_CLUSTER=0 batched HAC adds its row splits in a finishing kernel instead of a thread-block cluster
+ *   HAC_B200_SHAC_ROWS=0     batched sHAC never through the kernel that stages rows of X in shared memory; 2: whenever it can
+ *   HAC_B200_SHAC_ROWS_GROUP=n  row tasks per staged group of that kernel (0 = chosen by the library)
  *   HAC_B200_ZERO_RUNS=0    never use the zero-run table of mostly-zero HAC streams
  *   HAC_B200_XT=0           never use the magnitude-indexed first-level table */
 

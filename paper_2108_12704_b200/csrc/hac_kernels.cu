@@ -2527,6 +2527,187 @@ __global__ void __launch_bounds__(1024) shac_batch_kernel(DevFormat f, TablePlan
     }
 }
 
+// ------------------------------------------------------------------------------------------------
+// sHAC, batch of inputs, rows of X staged in shared memory.  The row tasks of the format (f.S consecutive rows
+// here; task_off / task_pos give, per task and column, where the column's first stored entry at or after the
+// task's first row starts in the stream and in ri) cut every column into cells.  A block owns kRbCols
+// consecutive columns, a range of tasks (the row split) and a tile of 32 * kIn inputs.  It walks its tasks in
+// groups of `group` tasks: the group's rows of X for its inputs are brought into shared memory (coalesced
+// 16-byte asynchronous copies), then every warp works off the cells of its eight columns, 32 cells at a time
+// (lane l: column l % 8, task l / 8 of the pass): every lane decodes one entry of its cell straight from global
+// memory (a cell is a handful of code words), and for every entry so decoded the whole warp multiplies its value
+// with the entry's row of X, lane l holding inputs l * kIn .. + kIn - 1 of each of the eight column sums.  X is
+// thus read from memory once per block of 256 columns, not once per stored entry.  Sums of a row split go to
+// partial[split][column][input] for rowblock_finalize_kernel; without a split y is written directly.
+// ------------------------------------------------------------------------------------------------
+constexpr uint32_t kRbWarps = 32, kRbWarpCols = 8, kRbCols = kRbWarps * kRbWarpCols;
+
+template <int kIn, typename RowT>
+__global__ void __launch_bounds__(kRbWarps * 32, 1)
+shac_rowblock_kernel(DevFormat f, TablePlan tp, const float* __restrict__ x, int64_t xs_i, uint32_t batch,
+                     float* __restrict__ y, int64_t ys_j, int64_t ys_b, float* __restrict__ partial,
+                     const uint64_t* __restrict__ task_off, const uint32_t* __restrict__ task_pos, uint32_t tasks,
+                     uint32_t row_splits, uint32_t col_blocks, uint32_t nbuf, uint32_t x_aligned, uint32_t group) {
+    constexpr uint32_t kTileB = 32 * kIn;
+    allow_dependents();
+    unsigned char* p = smem;
+    const Decoder dec = stage_decoder(f, tp, p);
+    float* xs = reinterpret_cast<float*>(smem + ((smem_off(p) + 15u) & ~15u));          // [nbuf][group * T][kTileB]
+    const uint32_t T = f.S, group_rows = group * T;
+    const uint32_t warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const uint32_t cblk = blockIdx.x % col_blocks, rs = blockIdx.x / col_blocks;
+    const uint32_t b0 = blockIdx.y * kTileB;
+    const uint32_t t_begin = gemm_split_begin(tasks, rs, row_splits), t_end = gemm_split_begin(tasks, rs + 1, row_splits);
+    const uint32_t jw = cblk * kRbCols + warp * kRbWarpCols;
+    const uint32_t jc = jw + (lane & 7u);
+    const RowT* __restrict__ ri = reinterpret_cast<const RowT*>(f.ri);
+    float acc[kRbWarpCols][kIn];
+#pragma unroll
+    for (int c = 0; c < (int)kRbWarpCols; ++c)
+#pragma unroll
+        for (int i = 0; i < kIn; ++i) acc[c][i] = 0.0f;
+
+    // where this lane's cell (its column, task t) starts, and how many entries it holds; t_hi bounds the group
+    auto cell = [&](uint32_t t, uint32_t t_hi, uint64_t& bit, uint32_t& p0, uint32_t& cnt) {
+        bit = 0; p0 = 0; cnt = 0;
+        if (jc < f.m && t < t_hi) {
+            const size_t i = (size_t)t * f.m + jc;
+            bit = __ldg(task_off + i);
+            p0 = __ldg(task_pos + i);
+            cnt = __ldg(task_pos + i + f.m) - p0;
+        }
+    };
+    // rows [r0, r0 + nrows) of X for this block's inputs -> shared memory; rows past the matrix and inputs past the
+    // batch are zero
+    auto stage_x = [&](uint32_t r0, uint32_t nrows, uint32_t buf) {
+        float* dst0 = xs + (size_t)buf * group_rows * kTileB;
+        constexpr uint32_t kQ = kTileB / 4;
+        for (uint32_t idx = threadIdx.x; idx < nrows * kQ; idx += blockDim.x) {
+            const uint32_t r = idx / kQ, q = idx % kQ;
+            float* dst = dst0 + r * kTileB + 4 * q;
+            const uint32_t b = b0 + 4 * q;
+            if (r0 + r < f.n && x_aligned && b + 3 < batch) {
+                cp_async16((uint32_t)__cvta_generic_to_shared(dst), x + (int64_t)(r0 + r) * xs_i + b);
+            } else {
+                float4 v = make_float4(0.0f, 0.0f, 0.0f, 0.0f);
+                if (r0 + r < f.n) {
+                    const float* src = x + (int64_t)(r0 + r) * xs_i;
+                    if (b < batch) v.x = __ldg(src + b);
+                    if (b + 1 < batch) v.y = __ldg(src + b + 1);
+                    if (b + 2 < batch) v.z = __ldg(src + b + 2);
+                    if (b + 3 < batch) v.w = __ldg(src + b + 3);
+                }
+                *reinterpret_cast<float4*>(dst) = v;
+            }
+        }
+        asm volatile("cp.async.commit_group;" ::: "memory");
+    };
+    auto group_tasks = [&](uint32_t gt) { return min(group, t_end - gt); };
+
+    uint64_t bit_n;
+    uint32_t p0_n, cnt_n;
+    cell(t_begin + (lane >> 3), min(t_begin + group, t_end), bit_n, p0_n, cnt_n);
+    depends_wait();                               // x and the partial sums belong to the kernels before this one
+    if (t_begin < t_end) stage_x(t_begin * T, group_tasks(t_begin) * T, 0);
+    uint32_t gi = 0;
+    for (uint32_t gt = t_begin; gt < t_end; gt += group, ++gi) {
+        const uint32_t buf = nbuf == 2 ? (gi & 1u) : 0u;
+        const uint32_t g_hi = gt + group_tasks(gt);
+        asm volatile("cp.async.wait_group 0;" ::: "memory");
+        __syncthreads();                          // this group's rows have landed; everyone has left the group before
+        if (nbuf == 2 && g_hi < t_end) stage_x(g_hi * T, group_tasks(g_hi) * T, buf ^ 1u);     // lands while this group is worked off
+        const float* xb = xs + (size_t)buf * group_rows * kTileB + lane * kIn;
+        const uint32_t row0 = gt * T;
+        for (uint32_t tp0 = gt; tp0 < g_hi; tp0 += 4) {               // a pass: four tasks x eight columns
+            uint64_t bit = bit_n;
+            const uint32_t p0 = p0_n, cnt = cnt_n;
+            // the cells of the next pass (or of the next group's first pass) are requested now
+            if (tp0 + 4 < g_hi) cell(tp0 + 4 + (lane >> 3), g_hi, bit_n, p0_n, cnt_n);
+            else cell(g_hi + (lane >> 3), min(g_hi + group, t_end), bit_n, p0_n, cnt_n);
+            uint32_t maxc = cnt;
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1) maxc = max(maxc, __shfl_xor_sync(0xffffffffu, maxc, o));
+            for (uint32_t e = 0; e < maxc; ++e) {
+                float v = 0.0f;
+                uint32_t rr = 0;
+                const bool have = e < cnt;
+                if (have) {
+                    const uint32_t* w = f.stream + (bit >> 5);
+                    const uint32_t top = __funnelshift_l(__ldg(w + 1), __ldg(w), (uint32_t)bit & 31u);
+                    uint2 en = lds64(dec.l1_lane + (top >> dec.l1_shift) * dec.l1_mul);
+                    if ((int32_t)en.y < 0) {
+                        const uint32_t q = (top << dec.l1_bits) >> (32 - (en.y & 31u));
+                        en = lds64(dec.sub + en.x + (q << 3));
+                        if (en.y == 0)
+                            en = decode_long(top, f.lut, f.lut_bits, f.rank_value, f.limit, f.first_left, f.rank_base, f.max_len);
+                    }
+                    bit += en.y;
+                    v = __uint_as_float(en.x);
+                    rr = min((uint32_t)ri[p0 + e] - row0, group_rows - 1);
+                }
+                const uint32_t mask = __ballot_sync(0xffffffffu, have);
+                // column after column (the sums of a column are named registers), the up to four tasks of a column by set bit
+#pragma unroll
+                for (int c = 0; c < (int)kRbWarpCols; ++c) {
+                    uint32_t mc = (mask >> c) & 0x01010101u;
+                    while (mc) {
+                        const int src = __ffs((int)mc) - 1 + c;
+                        mc &= mc - 1;
+                        const float vc = __shfl_sync(0xffffffffu, v, src);
+                        const uint32_t rc = __shfl_sync(0xffffffffu, rr, src);
+                        const float* xr = xb + rc * kTileB;
+                        if (kIn == 4) {
+                            const float4 xv = *reinterpret_cast<const float4*>(xr);
+                            acc[c][0] = fmaf(vc, xv.x, acc[c][0]);
+                            acc[c][1 % kIn] = fmaf(vc, xv.y, acc[c][1 % kIn]);
+                            acc[c][2 % kIn] = fmaf(vc, xv.z, acc[c][2 % kIn]);
+                            acc[c][3 % kIn] = fmaf(vc, xv.w, acc[c][3 % kIn]);
+                        } else if (kIn == 2) {
+                            const float2 xv = *reinterpret_cast<const float2*>(xr);
+                            acc[c][0] = fmaf(vc, xv.x, acc[c][0]);
+                            acc[c][1 % kIn] = fmaf(vc, xv.y, acc[c][1 % kIn]);
+                        } else {
+                            acc[c][0] = fmaf(vc, xr[0], acc[c][0]);
+                        }
+                    }
+                }
+            }
+        }
+        if (nbuf == 1) {
+            __syncthreads();                      // everyone is done with the rows before they are replaced
+            if (g_hi < t_end) stage_x(g_hi * T, group_tasks(g_hi) * T, 0);
+        }
+    }
+    // inputs of a lane are consecutive, so a warp writes kTileB consecutive inputs of one column at a time
+#pragma unroll
+    for (int c = 0; c < (int)kRbWarpCols; ++c) {
+        const uint32_t j = jw + c;
+        if (j >= f.m) continue;
+#pragma unroll
+        for (int i = 0; i < kIn; ++i) {
+            const uint32_t b = b0 + lane * kIn + i;
+            if (b >= batch) continue;
+            if (row_splits == 1) y[(int64_t)j * ys_j + (int64_t)b * ys_b] = finish_output(f, acc[c][i], j);
+            else partial[((size_t)rs * f.m + j) * batch + b] = acc[c][i];
+        }
+    }
+}
+
+// y[j][b] = sum over the row splits of partial[split][j][b], added in split order (see shac_rowblock_kernel).
+__global__ void __launch_bounds__(256) rowblock_finalize_kernel(const float* __restrict__ partial, uint32_t splits, uint32_t m,
+                                                                uint32_t batch, float* __restrict__ y, int64_t ys_j,
+                                                                int64_t ys_b, const float* __restrict__ bias, uint32_t relu) {
+    allow_dependents();
+    depends_wait();
+    const uint64_t total = (uint64_t)m * batch;
+    for (uint64_t idx = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x; idx < total; idx += (uint64_t)gridDim.x * blockDim.x) {
+        const uint32_t j = (uint32_t)(idx / batch), b = (uint32_t)(idx % batch);
+        float sum = 0.0f;
+        for (uint32_t r = 0; r < splits; ++r) sum += partial[(size_t)r * total + idx];
+        y[(int64_t)j * ys_j + (int64_t)b * ys_b] = finish_output(bias, relu, sum, j);
+    }
+}
+
 // X[batch][n] -> Xt[n][batch] (host-input path only).
 __global__ void transpose_kernel(const float* __restrict__ in, float* __restrict__ out, uint32_t rows,
                                  uint32_t cols) {
@@ -2582,10 +2763,13 @@ struct Tune {
     int vec_warps;      // HAC_B200_VEC_WARPS=n: warps per block of the shared-memory-x kernels (0 = chosen by the library)
     int vec_group;      // HAC_B200_VEC_GROUP=0: the shared-memory-x HAC kernel decodes one code word per lookup
     int gemm_cluster;   // HAC_B200_GEMM_CLUSTER=0: batched HAC adds its row splits in a finishing kernel, not in a cluster
+    int shac_rows_group;// HAC_B200_SHAC_ROWS_GROUP=n: row tasks per staged group of that kernel, one buffer (0 = chosen by the library)
+    int shac_rows;      // HAC_B200_SHAC_ROWS=0: batched sHAC never through the kernel that stages rows of X; 2: whenever it can
+                        // (1 = chosen by estimated cost)
 };
 static const Tune& tune() {
     static const Tune t = {env_int("HAC_B200_PDL", 1), env_int("HAC_B200_ROWS", 1), env_int("HAC_B200_ROWS_WARPS", 0),
-                           env_int("HAC_B200_ZERO_RUNS", 1), env_int("HAC_B200_XT", 1), env_int("HAC_B200_PREFETCH", 0), env_int("HAC_B200_ROWS_CHAINS", 0), env_int("HAC_B200_ITEMS", 1), env_int("HAC_B200_SHAC_TC", 1), env_int("HAC_B200_VEC_WARPS", 0), env_int("HAC_B200_VEC_GROUP", 1), env_int("HAC_B200_GEMM_CLUSTER", 1)};
+                           env_int("HAC_B200_ZERO_RUNS", 1), env_int("HAC_B200_XT", 1), env_int("HAC_B200_PREFETCH", 0), env_int("HAC_B200_ROWS_CHAINS", 0), env_int("HAC_B200_ITEMS", 1), env_int("HAC_B200_SHAC_TC", 1), env_int("HAC_B200_VEC_WARPS", 0), env_int("HAC_B200_VEC_GROUP", 1), env_int("HAC_B200_GEMM_CLUSTER", 1), env_int("HAC_B200_SHAC_ROWS_GROUP", 0), env_int("HAC_B200_SHAC_ROWS", 1)};
     return t;
 }
 
@@ -2733,10 +2917,15 @@ static bool shac_vec_fits(const Format& f) {
     return 16 + plan_smem_bytes(1u << f.tables.l1_bits, 0, (uint32_t)(f.tables.sub.size() * 4)) + per_warp <= (size_t)232448;
 }
 
+// Whether a batched sHAC product may go to the kernel that stages rows of X in shared memory (it needs the row tasks).
+static bool shac_rows_possible(const Format& f, int64_t batch) {
+    return f.sparse && batch >= 2 && !f.task_pos.empty() && tune().shac_rows != 0;
+}
+
 static size_t partial_bytes(const Format& f, int64_t batch) {
-    // tensor-core kernel: one partial per row split of the product kernel
+    // tensor-core kernel and the kernel that stages rows of X: one partial per row split of the product kernel
     size_t tc = 0;
-    if (batch > 1 && (!f.sparse || shac_tc_wanted(f, batch))) {
+    if (batch > 1 && (!f.sparse || shac_tc_wanted(f, batch) || shac_rows_possible(f, batch))) {
         const uint32_t t = gemm_tasks(f);
         tc = t > 1 ? (size_t)std::min<uint32_t>(t, kGMaxSplits) * (size_t)f.m * (size_t)batch * 4 : 0;
         if (!f.sparse) return tc;
@@ -3290,6 +3479,69 @@ static int launch_batch_t(const Format& f, const DeviceInfo& di, const DevFormat
     return HAC_OK;
 }
 
+// Batched sHAC through shac_rowblock_kernel.  Returns HAC_ERR_BUFFER_TOO_SMALL (nothing launched) when the format,
+// the layout of X or the estimate says that another kernel should take the product.  *splits_out: row splits whose
+// sums rowblock_finalize_kernel has added (0: y was written directly).
+static int launch_shac_rows(const Format& f, const DeviceInfo& di, const DevFormat& d0, const float* x, int64_t xs_i,
+                            int64_t xs_b, int64_t batch, float* y, int64_t ys_j, int64_t ys_b, float* partial,
+                            cudaStream_t st) {
+    if (!shac_rows_possible(f, batch) || xs_b != 1 || batch > ((int64_t)1 << 22)) return HAC_ERR_BUFFER_TOO_SMALL;
+    DevFormat d = d0;
+    d.S = f.tc_rows;
+    const int in = batch > 64 ? 4 : (batch > 32 ? 2 : 1);
+    const uint32_t tile_b = 32u * (uint32_t)in;
+    const uint32_t tiles = (uint32_t)((batch + tile_b - 1) / tile_b);
+    const size_t budget = (size_t)di.max_smem_optin;
+    TablePlan tp = plan_tables(d, 32 * 1024);
+    const size_t tab = plan_smem_bytes(d.l1_entries, tp.repl_log2, d.sub_bytes) + 16;
+    const uint32_t tasks = gemm_tasks(f);
+    // tasks per group: as many rows of X as shared memory holds (a multiple of the four tasks of a pass where possible),
+    // in one buffer; two buffers of half that when a group is still at least a pass
+    const size_t task_bytes = (size_t)d.S * tile_b * 4;
+    if (tab + task_bytes > budget) return HAC_ERR_BUFFER_TOO_SMALL;
+    uint32_t group = (uint32_t)std::min<size_t>((budget - tab) / task_bytes, tasks), nbuf = 1;
+    if (group >= 8) { group = (group / 2) & ~3u; nbuf = 2; }
+    else if (group >= 4) group &= ~3u;
+    if (tune().shac_rows_group > 0 && (size_t)tune().shac_rows_group * task_bytes + tab <= budget) {
+        group = (uint32_t)tune().shac_rows_group;
+        nbuf = 2 * (size_t)group * task_bytes + tab <= budget ? 2u : 1u;
+    }
+    const size_t xbytes = (size_t)group * task_bytes;
+    const uint32_t col_blocks = (uint32_t)((f.m + kRbCols - 1) / kRbCols);
+    const uint64_t blocks = (uint64_t)col_blocks * tiles;
+    uint32_t rs = 1;
+    if (blocks * 5 < (uint64_t)di.sms * 3 && tasks > 1)
+        rs = (uint32_t)std::min<uint64_t>(std::min<uint64_t>(((uint64_t)di.sms + blocks - 1) / blocks, tasks), kGMaxSplits);
+    // Measured on a 25088 x 4096 layer with 96 % zeros: 164 / 267 us for 64 / 128 inputs against 219 / 390 us for the
+    // other two kernels, but slower than they are for 32 inputs or fewer and for moderately sparse layers (whose row
+    // tasks are short), so: many inputs and at most one weight in ten stored.
+    if (tune().shac_rows != 2 && (batch < 48 || (double)f.nnz * 10.0 > (double)f.n * (double)f.m)) return HAC_ERR_BUFFER_TOO_SMALL;
+    const uint32_t aligned = (reinterpret_cast<uintptr_t>(x) % 16 == 0 && xs_i % 4 == 0) ? 1u : 0u;
+    typedef void (*RowsKernel)(DevFormat, TablePlan, const float*, int64_t, uint32_t, float*, int64_t, int64_t, float*,
+                               const uint64_t*, const uint32_t*, uint32_t, uint32_t, uint32_t, uint32_t, uint32_t, uint32_t);
+    RowsKernel kernel;
+    if (f.ri_bits == 16)
+        kernel = in == 4 ? shac_rowblock_kernel<4, uint16_t> : (in == 2 ? shac_rowblock_kernel<2, uint16_t> : shac_rowblock_kernel<1, uint16_t>);
+    else
+        kernel = in == 4 ? shac_rowblock_kernel<4, uint32_t> : (in == 2 ? shac_rowblock_kernel<2, uint32_t> : shac_rowblock_kernel<1, uint32_t>);
+    const size_t smem = tab + nbuf * xbytes;
+    int rc = prepare_kernel(kernel, smem);
+    if (rc) return rc;
+    rc = launch_dependent(kernel, dim3(col_blocks * rs, tiles), dim3(kRbWarps * 32), smem, st, d, tp, x, xs_i, (uint32_t)batch, y,
+                          ys_j, ys_b, partial, f.dev.task_off, f.dev.task_pos, tasks, rs, col_blocks, nbuf, aligned, group);
+    if (rc) return rc;
+    f.last_launches++;
+    if (rs > 1) {
+        const uint64_t total = (uint64_t)f.m * (uint64_t)batch;
+        const unsigned grid = (unsigned)std::min<uint64_t>((total + 255) / 256, (uint64_t)di.sms * 8);
+        rc = launch_dependent(rowblock_finalize_kernel, dim3(grid), dim3(256), 0, st, (const float*)partial, rs, (uint32_t)f.m,
+                              (uint32_t)batch, y, ys_j, ys_b, f.epi_bias, (uint32_t)f.epi_relu);
+        if (rc) return rc;
+        f.last_launches++;
+    }
+    return HAC_OK;
+}
+
 static int dot(const Format& f, const float* x, int64_t batch, int64_t xs_i, int64_t xs_b, float* y,
                int64_t ys_j, int64_t ys_b, void* workspace, size_t workspace_bytes_given, void* stream_,
                const hac_epilogue* epi = nullptr) {
@@ -3314,6 +3566,7 @@ static int dot(const Format& f, const float* x, int64_t batch, int64_t xs_i, int
     uint32_t gemm_splits = 0;                // batched HAC: row splits used (1 = outputs written directly)
     bool wide_single = false;                // sHAC, one input, through the batched kernel (see shac_vec_fits)
     bool shac_tc = false;                    // sHAC batch through the tensor-core kernel
+    bool shac_rows = false;                  // sHAC batch through the kernel that stages rows of X (it finishes y itself)
     if (d.units > 0) {
         if (batch == 1 && (!f.sparse || shac_vec_fits(f))) {
             rc = launch_vec(f, 0, x, xs_i, y, ys_j, partial, st, &direct);
@@ -3341,7 +3594,9 @@ static int dot(const Format& f, const float* x, int64_t batch, int64_t xs_i, int
                             rc = launch_finalize(f, d, partial, 1, y + b * ys_b, ys_j, 0, st, 1);
                     }
                 }
-            } else if (shac_tc_wanted(f, batch) && [&]() {
+            } else if ((rc = launch_shac_rows(f, di, d, x, xs_i, xs_b, batch, y, ys_j, ys_b, partial, st)) != HAC_ERR_BUFFER_TOO_SMALL) {
+                shac_rows = true;                    // launched (or failed for good)
+            } else if ((rc = HAC_OK, shac_tc_wanted(f, batch)) && [&]() {
                            // moderately sparse, or a large batch: the tensor-core kernel with zero-filled tiles
                            unsigned char* xpack = static_cast<unsigned char*>(workspace) + ((partial_bytes(f, batch) + 255) & ~(size_t)255);
                            rc = launch_gemm_tc(f, di, d, x, xs_i, xs_b, batch, y, ys_j, ys_b, partial, xpack, st, &gemm_splits);
@@ -3365,7 +3620,9 @@ static int dot(const Format& f, const float* x, int64_t batch, int64_t xs_i, int
     uint32_t direct_up_to = 1;
     bool finish;
     DevFormat dfin = d;
-    if ((!f.sparse && batch > 1) || shac_tc) {
+    if (shac_rows) {
+        finish = false;
+    } else if ((!f.sparse && batch > 1) || shac_tc) {
         if (gemm_splits > 1) {               // partial[split][b][j]
             dim3 grid((unsigned)((f.m + 31) / 32), (unsigned)((batch + 31) / 32));
             // launched the ordinary way: started early, its blocks only took the idle SMs from the product

@@ -383,3 +383,37 @@ def test_no_bounded_wait_ran_out():
         y = run_dot(lf, si.inputs(wl, 70))
         assert np.isfinite(y).all()
     assert lost_waits() == 0
+
+
+def test_rowblock_kernel_forced_on_every_shape():
+    """The batched sHAC kernel that stages rows of X is chosen only for many inputs and very sparse layers; here a
+    diagnostic switch (read once per process, hence the child process) sends every batched sHAC product through it:
+    ragged batches, unaligned X, several row splits, 32-bit row indices."""
+    import os, subprocess, sys
+    code = r'''
+import dataclasses, numpy as np, torch
+import synth_inputs as si
+from oracle import hac_oracle as orc
+import paper_2108_12704_b200 as hb
+cases = [(si.scaled(si.CFG3_FC_SHAC, 6000, 200), 0, (5, 40, 64, 130)), (si.scaled(si.CFG4_CONV, 1152, 128), 0, (33, 200)),
+         (si.scaled(si.CFG3_FC_SHAC, 70000, 24), 0, (64,)), (si.CFG1_TINY_SHAC, 0, (2, 70))]
+for wl, S, batches in cases:
+    W = si.weights(wl)
+    Wq, mask = orc.quantize(W, wl.sparsity, wl.k, wl.quantizer, wl.kmeans_iters, wl.seed)
+    lf = hb.Format("shac", W, sparsity=wl.sparsity, k=wl.k, quantizer=wl.quantizer, kmeans_iters=wl.kmeans_iters,
+                   seed=wl.seed, seg_symbols=S).upload()
+    for B in batches:
+        X = si.inputs(wl, B)
+        y_ref, a = orc.dot_definition(Wq, X)
+        y = lf.dot(torch.from_numpy(np.ascontiguousarray(X.T)).cuda()).cpu().numpy().T
+        assert np.all(np.abs(y - y_ref) <= 1e-5 * a + 1e-7), (wl.name, B)
+        bias = torch.linspace(-1, 1, wl.m, device="cuda")
+        yb = lf.dot(torch.from_numpy(np.ascontiguousarray(X.T)).cuda(), bias=bias, relu=True).cpu().numpy().T
+        ref = np.maximum(y_ref + bias.cpu().numpy().astype(np.float64), 0)
+        assert np.all(np.abs(yb - ref) <= 1e-5 * (a + 1) + 1e-6), (wl.name, B, "layer")
+print("ok")
+'''
+    env = dict(os.environ, HAC_B200_SHAC_ROWS="2")
+    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+    out = subprocess.run([sys.executable, "-c", code], cwd=root, env=env, capture_output=True, text=True, timeout=900)
+    assert out.returncode == 0 and "ok" in out.stdout, out.stdout + out.stderr
