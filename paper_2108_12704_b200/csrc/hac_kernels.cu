@@ -2540,30 +2540,37 @@ __global__ void __launch_bounds__(1024) shac_batch_kernel(DevFormat f, TablePlan
 // thus read from memory once per block of 256 columns, not once per stored entry.  Sums of a row split go to
 // partial[split][column][input] for rowblock_finalize_kernel; without a split y is written directly.
 // ------------------------------------------------------------------------------------------------
-constexpr uint32_t kRbWarps = 32, kRbWarpCols = 8, kRbCols = kRbWarps * kRbWarpCols;
+// A warp has kWC columns (8, or 4 when the tile is 128 inputs wide and eight columns' sums would not fit the registers) and
+// 32 / kWC tasks per pass, so 32 cells either way; a column collects up to kRbChunk entries of each of those tasks.
+constexpr uint32_t kRbWarps = 32, kRbChunk = 4;
+constexpr size_t kRbListBytes = (size_t)kRbWarps * 32 * kRbChunk * 8;
 
-template <int kIn, typename RowT>
+template <int kIn, int kWC, typename RowT>
 __global__ void __launch_bounds__(kRbWarps * 32, 1)
 shac_rowblock_kernel(DevFormat f, TablePlan tp, const float* __restrict__ x, int64_t xs_i, uint32_t batch,
                      float* __restrict__ y, int64_t ys_j, int64_t ys_b, float* __restrict__ partial,
                      const uint64_t* __restrict__ task_off, const uint32_t* __restrict__ task_pos, uint32_t tasks,
                      uint32_t row_splits, uint32_t col_blocks, uint32_t nbuf, uint32_t x_aligned, uint32_t group) {
     constexpr uint32_t kTileB = 32 * kIn;
+    constexpr uint32_t kPassTasks = 32 / kWC, kListLen = kPassTasks * kRbChunk;
+    constexpr uint32_t kTaskBits = kWC == 8 ? 0x01010101u : 0x11111111u;      // ballot bits of one column: one per task of the pass
     allow_dependents();
     unsigned char* p = smem;
     const Decoder dec = stage_decoder(f, tp, p);
-    float* xs = reinterpret_cast<float*>(smem + ((smem_off(p) + 15u) & ~15u));          // [nbuf][group * T][kTileB]
+    // decoded entries of the pass at hand, per warp and column: kRbChunk steps x four tasks of {value, row in the group}
+    uint2* lists = reinterpret_cast<uint2*>(smem + ((smem_off(p) + 15u) & ~15u));
+    float* xs = reinterpret_cast<float*>(lists + (size_t)kRbWarps * kWC * kListLen);      // [nbuf][group * T][kTileB]
     const uint32_t T = f.S, group_rows = group * T;
     const uint32_t warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const uint32_t cblk = blockIdx.x % col_blocks, rs = blockIdx.x / col_blocks;
     const uint32_t b0 = blockIdx.y * kTileB;
     const uint32_t t_begin = gemm_split_begin(tasks, rs, row_splits), t_end = gemm_split_begin(tasks, rs + 1, row_splits);
-    const uint32_t jw = cblk * kRbCols + warp * kRbWarpCols;
-    const uint32_t jc = jw + (lane & 7u);
+    const uint32_t jw = cblk * (kRbWarps * kWC) + warp * kWC;
+    const uint32_t jc = jw + (lane & (kWC - 1u));
     const RowT* __restrict__ ri = reinterpret_cast<const RowT*>(f.ri);
-    float acc[kRbWarpCols][kIn];
+    float acc[kWC][kIn];
 #pragma unroll
-    for (int c = 0; c < (int)kRbWarpCols; ++c)
+    for (int c = 0; c < (int)kWC; ++c)
 #pragma unroll
         for (int i = 0; i < kIn; ++i) acc[c][i] = 0.0f;
 
@@ -2606,7 +2613,7 @@ shac_rowblock_kernel(DevFormat f, TablePlan tp, const float* __restrict__ x, int
 
     uint64_t bit_n;
     uint32_t p0_n, cnt_n;
-    cell(t_begin + (lane >> 3), min(t_begin + group, t_end), bit_n, p0_n, cnt_n);
+    cell(t_begin + (lane / kWC), min(t_begin + group, t_end), bit_n, p0_n, cnt_n);
     depends_wait();                               // x and the partial sums belong to the kernels before this one
     if (t_begin < t_end) stage_x(t_begin * T, group_tasks(t_begin) * T, 0);
     uint32_t gi = 0;
@@ -2618,58 +2625,119 @@ shac_rowblock_kernel(DevFormat f, TablePlan tp, const float* __restrict__ x, int
         if (nbuf == 2 && g_hi < t_end) stage_x(g_hi * T, group_tasks(g_hi) * T, buf ^ 1u);     // lands while this group is worked off
         const float* xb = xs + (size_t)buf * group_rows * kTileB + lane * kIn;
         const uint32_t row0 = gt * T;
-        for (uint32_t tp0 = gt; tp0 < g_hi; tp0 += 4) {               // a pass: four tasks x eight columns
+        for (uint32_t tp0 = gt; tp0 < g_hi; tp0 += kPassTasks) {               // a pass: 32 cells
             uint64_t bit = bit_n;
             const uint32_t p0 = p0_n, cnt = cnt_n;
             // the cells of the next pass (or of the next group's first pass) are requested now
-            if (tp0 + 4 < g_hi) cell(tp0 + 4 + (lane >> 3), g_hi, bit_n, p0_n, cnt_n);
-            else cell(g_hi + (lane >> 3), min(g_hi + group, t_end), bit_n, p0_n, cnt_n);
+            if (tp0 + kPassTasks < g_hi) cell(tp0 + kPassTasks + (lane / kWC), g_hi, bit_n, p0_n, cnt_n);
+            else cell(g_hi + (lane / kWC), min(g_hi + group, t_end), bit_n, p0_n, cnt_n);
             uint32_t maxc = cnt;
 #pragma unroll
             for (int o = 16; o > 0; o >>= 1) maxc = max(maxc, __shfl_xor_sync(0xffffffffu, maxc, o));
-            for (uint32_t e = 0; e < maxc; ++e) {
-                float v = 0.0f;
-                uint32_t rr = 0;
-                const bool have = e < cnt;
-                if (have) {
-                    const uint32_t* w = f.stream + (bit >> 5);
-                    const uint32_t top = __funnelshift_l(__ldg(w + 1), __ldg(w), (uint32_t)bit & 31u);
-                    uint2 en = lds64(dec.l1_lane + (top >> dec.l1_shift) * dec.l1_mul);
-                    if ((int32_t)en.y < 0) {
-                        const uint32_t q = (top << dec.l1_bits) >> (32 - (en.y & 31u));
-                        en = lds64(dec.sub + en.x + (q << 3));
-                        if (en.y == 0)
-                            en = decode_long(top, f.lut, f.lut_bits, f.rank_value, f.limit, f.first_left, f.rank_base, f.max_len);
+            if (kIn == 4) {
+                // 128 inputs: the eight columns' sums leave no registers for the lists' bookkeeping; every decoded entry is
+                // handed to the warp by shuffle instead
+                for (uint32_t e = 0; e < maxc; ++e) {
+                    float v = 0.0f;
+                    uint32_t rr = 0;
+                    const bool have = e < cnt;
+                    if (have) {
+                        const uint32_t* w = f.stream + (bit >> 5);
+                        const uint32_t top = __funnelshift_l(__ldg(w + 1), __ldg(w), (uint32_t)bit & 31u);
+                        uint2 en = lds64(dec.l1_lane + (top >> dec.l1_shift) * dec.l1_mul);
+                        if ((int32_t)en.y < 0) {
+                            const uint32_t q = (top << dec.l1_bits) >> (32 - (en.y & 31u));
+                            en = lds64(dec.sub + en.x + (q << 3));
+                            if (en.y == 0)
+                                en = decode_long(top, f.lut, f.lut_bits, f.rank_value, f.limit, f.first_left, f.rank_base, f.max_len);
+                        }
+                        bit += en.y;
+                        v = __uint_as_float(en.x);
+                        rr = min((uint32_t)ri[p0 + e] - row0, group_rows - 1);
                     }
-                    bit += en.y;
-                    v = __uint_as_float(en.x);
-                    rr = min((uint32_t)ri[p0 + e] - row0, group_rows - 1);
-                }
-                const uint32_t mask = __ballot_sync(0xffffffffu, have);
-                // column after column (the sums of a column are named registers), the up to four tasks of a column by set bit
-#pragma unroll
-                for (int c = 0; c < (int)kRbWarpCols; ++c) {
-                    uint32_t mc = (mask >> c) & 0x01010101u;
-                    while (mc) {
-                        const int src = __ffs((int)mc) - 1 + c;
-                        mc &= mc - 1;
-                        const float vc = __shfl_sync(0xffffffffu, v, src);
-                        const uint32_t rc = __shfl_sync(0xffffffffu, rr, src);
-                        const float* xr = xb + rc * kTileB;
-                        if (kIn == 4) {
-                            const float4 xv = *reinterpret_cast<const float4*>(xr);
-                            acc[c][0] = fmaf(vc, xv.x, acc[c][0]);
-                            acc[c][1 % kIn] = fmaf(vc, xv.y, acc[c][1 % kIn]);
-                            acc[c][2 % kIn] = fmaf(vc, xv.z, acc[c][2 % kIn]);
-                            acc[c][3 % kIn] = fmaf(vc, xv.w, acc[c][3 % kIn]);
-                        } else if (kIn == 2) {
-                            const float2 xv = *reinterpret_cast<const float2*>(xr);
-                            acc[c][0] = fmaf(vc, xv.x, acc[c][0]);
-                            acc[c][1 % kIn] = fmaf(vc, xv.y, acc[c][1 % kIn]);
-                        } else {
-                            acc[c][0] = fmaf(vc, xr[0], acc[c][0]);
+                    const uint32_t mask = __ballot_sync(0xffffffffu, have);
+                    // column after column (the sums of a column are named registers), the up to four tasks of a column by set bit
+    #pragma unroll
+                    for (int c = 0; c < (int)kWC; ++c) {
+                        uint32_t mc = (mask >> c) & kTaskBits;
+                        while (mc) {
+                            const int src = __ffs((int)mc) - 1 + c;
+                            mc &= mc - 1;
+                            const float vc = __shfl_sync(0xffffffffu, v, src);
+                            const uint32_t rc = __shfl_sync(0xffffffffu, rr, src);
+                            const float* xr = xb + rc * kTileB;
+                            if (kIn == 4) {
+                                const float4 xv = *reinterpret_cast<const float4*>(xr);
+                                acc[c][0] = fmaf(vc, xv.x, acc[c][0]);
+                                acc[c][1 % kIn] = fmaf(vc, xv.y, acc[c][1 % kIn]);
+                                acc[c][2 % kIn] = fmaf(vc, xv.z, acc[c][2 % kIn]);
+                                acc[c][3 % kIn] = fmaf(vc, xv.w, acc[c][3 % kIn]);
+                            } else if (kIn == 2) {
+                                const float2 xv = *reinterpret_cast<const float2*>(xr);
+                                acc[c][0] = fmaf(vc, xv.x, acc[c][0]);
+                                acc[c][1 % kIn] = fmaf(vc, xv.y, acc[c][1 % kIn]);
+                            } else {
+                                acc[c][0] = fmaf(vc, xr[0], acc[c][0]);
+                            }
                         }
                     }
+                }
+            } else {
+                uint2* mylist = lists + ((size_t)warp * kWC + (lane & (kWC - 1u))) * kListLen;
+                const uint32_t below = (1u << (kWC * (lane / kWC))) - 1u;         // the tasks of my column that come before mine
+                for (uint32_t e0 = 0; e0 < maxc; e0 += kRbChunk) {
+                    // decode: every lane one entry of its cell per step, appended to its column's list in (step, task) order
+                    uint32_t mine = 0;                                           // entries my column has collected (same in its four lanes)
+    #pragma unroll 1
+                    for (uint32_t de = 0; de < kRbChunk; ++de) {
+                        const uint32_t e = e0 + de;
+                        const bool have = e < cnt;
+                        float v = 0.0f;
+                        uint32_t rr = 0;
+                        if (have) {
+                            const uint32_t* w = f.stream + (bit >> 5);
+                            const uint32_t top = __funnelshift_l(__ldg(w + 1), __ldg(w), (uint32_t)bit & 31u);
+                            uint2 en = lds64(dec.l1_lane + (top >> dec.l1_shift) * dec.l1_mul);
+                            if ((int32_t)en.y < 0) {
+                                const uint32_t q = (top << dec.l1_bits) >> (32 - (en.y & 31u));
+                                en = lds64(dec.sub + en.x + (q << 3));
+                                if (en.y == 0)
+                                    en = decode_long(top, f.lut, f.lut_bits, f.rank_value, f.limit, f.first_left, f.rank_base, f.max_len);
+                            }
+                            bit += en.y;
+                            v = __uint_as_float(en.x);
+                            rr = min((uint32_t)ri[p0 + e] - row0, group_rows - 1);
+                        }
+                        const uint32_t mc = (__ballot_sync(0xffffffffu, have) >> (lane & (kWC - 1u))) & kTaskBits;
+                        if (have) mylist[mine + __popc(mc & below)] = make_uint2(__float_as_uint(v), rr);
+                        mine += __popc(mc);
+                    }
+                    __syncwarp();
+                    // multiply: column after column (the sums of a column are named registers), every lane its inputs
+    #pragma unroll
+                    for (int c = 0; c < (int)kWC; ++c) {
+                        const uint32_t nc = __shfl_sync(0xffffffffu, mine, c);
+                        const uint2* lc = lists + ((size_t)warp * kWC + c) * kListLen;
+                        for (uint32_t i = 0; i < nc; ++i) {
+                            const uint2 en = lc[i];
+                            const float vc = __uint_as_float(en.x);
+                            const float* xr = xb + en.y * kTileB;
+                            if (kIn == 4) {
+                                const float4 xv = *reinterpret_cast<const float4*>(xr);
+                                acc[c][0] = fmaf(vc, xv.x, acc[c][0]);
+                                acc[c][1 % kIn] = fmaf(vc, xv.y, acc[c][1 % kIn]);
+                                acc[c][2 % kIn] = fmaf(vc, xv.z, acc[c][2 % kIn]);
+                                acc[c][3 % kIn] = fmaf(vc, xv.w, acc[c][3 % kIn]);
+                            } else if (kIn == 2) {
+                                const float2 xv = *reinterpret_cast<const float2*>(xr);
+                                acc[c][0] = fmaf(vc, xv.x, acc[c][0]);
+                                acc[c][1 % kIn] = fmaf(vc, xv.y, acc[c][1 % kIn]);
+                            } else {
+                                acc[c][0] = fmaf(vc, xr[0], acc[c][0]);
+                            }
+                        }
+                    }
+                    __syncwarp();
                 }
             }
         }
@@ -2680,7 +2748,7 @@ shac_rowblock_kernel(DevFormat f, TablePlan tp, const float* __restrict__ x, int
     }
     // inputs of a lane are consecutive, so a warp writes kTileB consecutive inputs of one column at a time
 #pragma unroll
-    for (int c = 0; c < (int)kRbWarpCols; ++c) {
+    for (int c = 0; c < (int)kWC; ++c) {
         const uint32_t j = jw + c;
         if (j >= f.m) continue;
 #pragma unroll
@@ -3493,37 +3561,38 @@ static int launch_shac_rows(const Format& f, const DeviceInfo& di, const DevForm
     const uint32_t tiles = (uint32_t)((batch + tile_b - 1) / tile_b);
     const size_t budget = (size_t)di.max_smem_optin;
     TablePlan tp = plan_tables(d, 32 * 1024);
-    const size_t tab = plan_smem_bytes(d.l1_entries, tp.repl_log2, d.sub_bytes) + 16;
+    const size_t tab = plan_smem_bytes(d.l1_entries, tp.repl_log2, d.sub_bytes) + 16 + kRbListBytes;
     const uint32_t tasks = gemm_tasks(f);
     // tasks per group: as many rows of X as shared memory holds (a multiple of the four tasks of a pass where possible),
     // in one buffer; two buffers of half that when a group is still at least a pass
     const size_t task_bytes = (size_t)d.S * tile_b * 4;
     if (tab + task_bytes > budget) return HAC_ERR_BUFFER_TOO_SMALL;
     uint32_t group = (uint32_t)std::min<size_t>((budget - tab) / task_bytes, tasks), nbuf = 1;
-    if (group >= 8) { group = (group / 2) & ~3u; nbuf = 2; }
-    else if (group >= 4) group &= ~3u;
+    const uint32_t wc = 8u, pass = 32u / wc;      // columns per warp, tasks per pass
+    if (group >= 2 * pass) { group = (group / 2) / pass * pass; nbuf = 2; }
+    else if (group >= pass) group = group / pass * pass;
     if (tune().shac_rows_group > 0 && (size_t)tune().shac_rows_group * task_bytes + tab <= budget) {
         group = (uint32_t)tune().shac_rows_group;
         nbuf = 2 * (size_t)group * task_bytes + tab <= budget ? 2u : 1u;
     }
     const size_t xbytes = (size_t)group * task_bytes;
-    const uint32_t col_blocks = (uint32_t)((f.m + kRbCols - 1) / kRbCols);
+    const uint32_t col_blocks = (uint32_t)((f.m + kRbWarps * wc - 1) / (kRbWarps * wc));
     const uint64_t blocks = (uint64_t)col_blocks * tiles;
     uint32_t rs = 1;
     if (blocks * 5 < (uint64_t)di.sms * 3 && tasks > 1)
-        rs = (uint32_t)std::min<uint64_t>(std::min<uint64_t>(((uint64_t)di.sms + blocks - 1) / blocks, tasks), kGMaxSplits);
-    // Measured on a 25088 x 4096 layer with 96 % zeros: 164 / 267 us for 64 / 128 inputs against 219 / 390 us for the
-    // other two kernels, but slower than they are for 32 inputs or fewer and for moderately sparse layers (whose row
-    // tasks are short), so: many inputs and at most one weight in ten stored.
-    if (tune().shac_rows != 2 && (batch < 48 || (double)f.nnz * 10.0 > (double)f.n * (double)f.m)) return HAC_ERR_BUFFER_TOO_SMALL;
+        rs = (uint32_t)std::min<uint64_t>(std::min<uint64_t>(std::max<uint64_t>(1, (uint64_t)di.sms / blocks), tasks), kGMaxSplits);      // one wave
+    // Measured on a 25088 x 4096 layer with 96 % zeros: 99 / 157 / 282 us for 32 / 64 / 128 inputs against 127 / 219 / 390 us
+    // for the other two kernels, but slower than they are for 16 inputs (102 against 77 us) and for moderately sparse layers
+    // (whose row tasks are short), so: a tile's worth of inputs and at most one weight in eight stored.
+    if (tune().shac_rows != 2 && (batch < 28 || (double)f.nnz * 8.0 > (double)f.n * (double)f.m)) return HAC_ERR_BUFFER_TOO_SMALL;
     const uint32_t aligned = (reinterpret_cast<uintptr_t>(x) % 16 == 0 && xs_i % 4 == 0) ? 1u : 0u;
     typedef void (*RowsKernel)(DevFormat, TablePlan, const float*, int64_t, uint32_t, float*, int64_t, int64_t, float*,
                                const uint64_t*, const uint32_t*, uint32_t, uint32_t, uint32_t, uint32_t, uint32_t, uint32_t);
     RowsKernel kernel;
     if (f.ri_bits == 16)
-        kernel = in == 4 ? shac_rowblock_kernel<4, uint16_t> : (in == 2 ? shac_rowblock_kernel<2, uint16_t> : shac_rowblock_kernel<1, uint16_t>);
+        kernel = in == 4 ? shac_rowblock_kernel<4, 8, uint16_t> : (in == 2 ? shac_rowblock_kernel<2, 8, uint16_t> : shac_rowblock_kernel<1, 8, uint16_t>);
     else
-        kernel = in == 4 ? shac_rowblock_kernel<4, uint32_t> : (in == 2 ? shac_rowblock_kernel<2, uint32_t> : shac_rowblock_kernel<1, uint32_t>);
+        kernel = in == 4 ? shac_rowblock_kernel<4, 8, uint32_t> : (in == 2 ? shac_rowblock_kernel<2, 8, uint32_t> : shac_rowblock_kernel<1, 8, uint32_t>);
     const size_t smem = tab + nbuf * xbytes;
     int rc = prepare_kernel(kernel, smem);
     if (rc) return rc;
