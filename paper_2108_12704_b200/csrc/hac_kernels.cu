@@ -600,64 +600,63 @@ __device__ __forceinline__ float warp_sum(float v) {
 // as long as the three lengths add up to at most 32; the caller checks `tot` (and `flags`, the OR of
 // the three length words, whose top bit marks an entry that does not hold its symbol) before it uses
 // the values, and otherwise decodes the three code words one at a time.  The reader is not advanced.
+// The asm block hands back the three length words; their sum and OR are formed outside it, so that the
+// compiler picks the instructions (one three-input add) and drops `flags` where it is not used.
 // ------------------------------------------------------------------------------------------------
 template <int kTab>
 __device__ __forceinline__ void lookup3(const FastReader& r, uint32_t l1_shift, uint32_t l1_mul, uint32_t l1_lane,
                                         uint32_t xt_low, uint32_t& v1, uint32_t& v2, uint32_t& v3, uint32_t& tot,
                                         uint32_t& flags) {
+    uint32_t la, lb, lc;
     if (kTab == 0) {
         asm volatile(
             "{\n\t"
-            ".reg .b32 t, i, a, b, c;\n\t"
-            "shf.l.wrap.b32 t, %5, %6, %7;\n\t"
-            "shr.u32 i, t, %8;\n\t"
-            "mad.lo.u32 i, i, %9, %10;\n\t"
-            "ld.shared.v2.u32 {%0, a}, [i];\n\t"
-            "shl.b32 t, t, a;\n\t"
-            "shr.u32 i, t, %8;\n\t"
-            "mad.lo.u32 i, i, %9, %10;\n\t"
-            "ld.shared.v2.u32 {%1, b}, [i];\n\t"
-            "shl.b32 t, t, b;\n\t"
-            "shr.u32 i, t, %8;\n\t"
-            "mad.lo.u32 i, i, %9, %10;\n\t"
-            "ld.shared.v2.u32 {%2, c}, [i];\n\t"
-            "add.u32 %3, a, b;\n\t"
-            "add.u32 %3, %3, c;\n\t"
-            "lop3.b32 %4, a, b, c, 0xFE;\n\t"
+            ".reg .b32 t, i;\n\t"
+            "shf.l.wrap.b32 t, %6, %7, %8;\n\t"
+            "shr.u32 i, t, %9;\n\t"
+            "mad.lo.u32 i, i, %10, %11;\n\t"
+            "ld.shared.v2.u32 {%0, %3}, [i];\n\t"
+            "shl.b32 t, t, %3;\n\t"
+            "shr.u32 i, t, %9;\n\t"
+            "mad.lo.u32 i, i, %10, %11;\n\t"
+            "ld.shared.v2.u32 {%1, %4}, [i];\n\t"
+            "shl.b32 t, t, %4;\n\t"
+            "shr.u32 i, t, %9;\n\t"
+            "mad.lo.u32 i, i, %10, %11;\n\t"
+            "ld.shared.v2.u32 {%2, %5}, [i];\n\t"
             "}"
-            : "=r"(v1), "=r"(v2), "=r"(v3), "=r"(tot), "=r"(flags)
+            : "=r"(v1), "=r"(v2), "=r"(v3), "=r"(la), "=r"(lb), "=r"(lc)
             : "r"(r.lo), "r"(r.hi), "r"(r.off), "r"(l1_shift), "r"(l1_mul), "r"(l1_lane)
             : "memory");
     } else {
         asm volatile(
             "{\n\t"
-            ".reg .b32 t, i, a, b, c;\n\t"
-            "shf.l.wrap.b32 t, %5, %6, %7;\n\t"
-            "lop3.b32 i, t, %11, 0, 0xCF;\n\t"
+            ".reg .b32 t, i;\n\t"
+            "shf.l.wrap.b32 t, %6, %7, %8;\n\t"
+            "lop3.b32 i, t, %12, 0, 0xCF;\n\t"
             "cvt.rz.f32.u32 i, i;\n\t"
-            "shr.u32 i, i, %8;\n\t"
-            "mad.lo.u32 i, i, %9, %10;\n\t"
-            "ld.shared.v2.u32 {%0, a}, [i];\n\t"
-            "shl.b32 t, t, a;\n\t"
-            "lop3.b32 i, t, %11, 0, 0xCF;\n\t"
+            "shr.u32 i, i, %9;\n\t"
+            "mad.lo.u32 i, i, %10, %11;\n\t"
+            "ld.shared.v2.u32 {%0, %3}, [i];\n\t"
+            "shl.b32 t, t, %3;\n\t"
+            "lop3.b32 i, t, %12, 0, 0xCF;\n\t"
             "cvt.rz.f32.u32 i, i;\n\t"
-            "shr.u32 i, i, %8;\n\t"
-            "mad.lo.u32 i, i, %9, %10;\n\t"
-            "ld.shared.v2.u32 {%1, b}, [i];\n\t"
-            "shl.b32 t, t, b;\n\t"
-            "lop3.b32 i, t, %11, 0, 0xCF;\n\t"
+            "shr.u32 i, i, %9;\n\t"
+            "mad.lo.u32 i, i, %10, %11;\n\t"
+            "ld.shared.v2.u32 {%1, %4}, [i];\n\t"
+            "shl.b32 t, t, %4;\n\t"
+            "lop3.b32 i, t, %12, 0, 0xCF;\n\t"
             "cvt.rz.f32.u32 i, i;\n\t"
-            "shr.u32 i, i, %8;\n\t"
-            "mad.lo.u32 i, i, %9, %10;\n\t"
-            "ld.shared.v2.u32 {%2, c}, [i];\n\t"
-            "add.u32 %3, a, b;\n\t"
-            "add.u32 %3, %3, c;\n\t"
-            "lop3.b32 %4, a, b, c, 0xFE;\n\t"
+            "shr.u32 i, i, %9;\n\t"
+            "mad.lo.u32 i, i, %10, %11;\n\t"
+            "ld.shared.v2.u32 {%2, %5}, [i];\n\t"
             "}"
-            : "=r"(v1), "=r"(v2), "=r"(v3), "=r"(tot), "=r"(flags)
+            : "=r"(v1), "=r"(v2), "=r"(v3), "=r"(la), "=r"(lb), "=r"(lc)
             : "r"(r.lo), "r"(r.hi), "r"(r.off), "r"(l1_shift), "r"(l1_mul), "r"(l1_lane), "r"(xt_low)
             : "memory");
     }
+    tot = la + lb + lc;
+    flags = la | lb | lc;
 }
 
 // The three code words of lookup3 one at a time (refills in between, entries without a symbol resolved):
@@ -734,7 +733,8 @@ __global__ void __launch_bounds__(1024) hac_vec_kernel(DevFormat f, TablePlan tp
         }
     };
     if (item < items) fetch();
-    // everything above reads the format only; x and the outputs belong to the kernels before this one
+    // everything above (index, spans of the first item, tables) reads the format only; x and the outputs
+    // belong to the kernels before this one
     depends_wait();
     // the first elements of x are requested together with the tables (one trip to memory for both)
     constexpr int kXAhead = 4;
@@ -964,11 +964,11 @@ __global__ void __launch_bounds__(1024) hac_vec_kernel(DevFormat f, TablePlan tp
 // three symbols.  A lane whose three lengths exceed the window, or that meets an entry without its
 // symbol, leaves the unrolled code and finishes its sub-segment one code word at a time.
 //
-// Order in a block: the whole range of the stream that the block's columns occupy is requested into L2
-// (its position is estimated from the column numbers, all columns holding the same number of code
-// words); index entries of the first two items, table entries and x are requested together (one trip to
-// memory); the spans of a warp's next item are copied to shared memory (cp.async, second buffer set)
-// while the current item is decoded.
+// Order in a block: index entries of the first two items and the table entries are requested together
+// (optionally also the block's range of the stream into L2); the spans of the first item are requested
+// and the tables staged BEFORE the dependency wait, since all of that is format data; x follows the
+// wait; the spans of a warp's next item are copied to shared memory (cp.async, second buffer set) while
+// the current item is decoded.
 //   kMode 0: product; 1: debug decode (values written to aux[j*n + i]).
 //   kTab  0: prefix table; 1: magnitude table.   kGuard: three lengths can exceed 32 bits.
 // ------------------------------------------------------------------------------------------------
@@ -1062,41 +1062,7 @@ __global__ void __launch_bounds__(kC <= 2 ? 512 : 384, 1) hac_rows_kernel(DevFor
                          : "memory");
         }
     }
-    // everything above reads the format only; x and the outputs belong to the kernels before this one
-    depends_wait();
-    float xr[kS];
-    constexpr int kXAhead = 8;
-    const uint32_t rows = f.G * 32u * kS;
-    float xv[kXAhead];
-    if (kMode == 0) {                      // the first elements of x are requested before the index entries are waited for
-#pragma unroll
-        for (int i = 0; i < kXAhead; ++i) {
-            const uint32_t r = threadIdx.x + i * blockDim.x;
-            xv[i] = r < f.n ? __ldg(x + (int64_t)r * xs_i) : 0.0f;
-        }
-    }
     fetch(0, 0, ix0, pos_cur);
-    if (kMode == 0) {
-        // x -> shared memory (coalesced; one padding word per sub-segment keeps the lanes of a warp, which
-        // are kS rows apart, on distinct banks; rows past the end of x are zeros) -> registers
-        for (uint32_t r0 = 0; r0 < rows; r0 += kXAhead * blockDim.x) {
-            if (r0 > 0) {
-#pragma unroll
-                for (int i = 0; i < kXAhead; ++i) {
-                    const uint32_t r = r0 + threadIdx.x + i * blockDim.x;
-                    xv[i] = r < f.n ? __ldg(x + (int64_t)r * xs_i) : 0.0f;
-                }
-            }
-#pragma unroll
-            for (int i = 0; i < kXAhead; ++i) {
-                const uint32_t r = r0 + threadIdx.x + i * blockDim.x;
-                if (r < rows) xs[r + r / kS] = xv[i];
-            }
-        }
-        __syncthreads();
-#pragma unroll
-        for (int s = 0; s < kS; ++s) xr[s] = xs[row0 + sub + s];
-    }
     // tables -> shared memory, replicated (see TablePlan): the warp writes its 32 entries' replicas slot by
     // slot, the value for a slot fetched from the lane that holds it (consecutive lanes write consecutive slots)
     Decoder dec;
@@ -1132,6 +1098,41 @@ __global__ void __launch_bounds__(kC <= 2 ? 512 : 384, 1) hac_rows_kernel(DevFor
         dec.xt_low = f.xt_low;
         dec.l1_bits = f.l1_bits;
         dec.sub = smem_off(subt);
+    }
+    // everything above (index, spans of the first item, tables) reads the format only; x and the outputs
+    // belong to the kernels before this one
+    depends_wait();
+    float xr[kS];
+    constexpr int kXAhead = 8;
+    const uint32_t rows = f.G * 32u * kS;
+    float xv[kXAhead];
+    if (kMode == 0) {                      // the first elements of x, all requests in flight at once
+#pragma unroll
+        for (int i = 0; i < kXAhead; ++i) {
+            const uint32_t r = threadIdx.x + i * blockDim.x;
+            xv[i] = r < f.n ? __ldg(x + (int64_t)r * xs_i) : 0.0f;
+        }
+    }
+    if (kMode == 0) {
+        // x -> shared memory (coalesced; one padding word per sub-segment keeps the lanes of a warp, which
+        // are kS rows apart, on distinct banks; rows past the end of x are zeros) -> registers
+        for (uint32_t r0 = 0; r0 < rows; r0 += kXAhead * blockDim.x) {
+            if (r0 > 0) {
+#pragma unroll
+                for (int i = 0; i < kXAhead; ++i) {
+                    const uint32_t r = r0 + threadIdx.x + i * blockDim.x;
+                    xv[i] = r < f.n ? __ldg(x + (int64_t)r * xs_i) : 0.0f;
+                }
+            }
+#pragma unroll
+            for (int i = 0; i < kXAhead; ++i) {
+                const uint32_t r = r0 + threadIdx.x + i * blockDim.x;
+                if (r < rows) xs[r + r / kS] = xv[i];
+            }
+        }
+        __syncthreads();
+#pragma unroll
+        for (int s = 0; s < kS; ++s) xr[s] = xs[row0 + sub + s];
     }
     __syncthreads();                       // tables are in place; x has left the second buffer set
     fetch(1, 1, ix1, pos_nxt);
@@ -1176,10 +1177,14 @@ __global__ void __launch_bounds__(kC <= 2 ? 512 : 384, 1) hac_rows_kernel(DevFor
                     for (int c = 0; c < kC; ++c)
                         lookup3<kTab>(fr[c], dec.l1_shift, dec.l1_mul, l1_abs, dec.xt_low, v[c][0], v[c][1], v[c][2], tot[c], flags[c]);
                     if (kGuard || kLong) {
-                        bool bad = false;
+                        // one test for all chains: the OR of the sums is above 32 if one of them is (and, rarely,
+                        // when one is exactly 32: the slow path is right for any group); only the lanes concerned
+                        // leave the unrolled code
+                        uint32_t tall = 0, fall = 0;
 #pragma unroll
-                        for (int c = 0; c < kC; ++c) bad = bad || (kGuard && tot[c] > 32u) || (kLong && (int32_t)flags[c] < 0);
-                        if (__any_sync(__activemask(), bad)) {              // uniform for the lanes in the unrolled code
+                        for (int c = 0; c < kC; ++c) { tall |= tot[c]; fall |= flags[c]; }
+                        const bool bad = (kGuard && tall > 32u) || (kLong && (int32_t)fall < 0);
+                        {
                             if (bad) {
 #pragma unroll
                                 for (int c = 0; c < kC; ++c) {
@@ -1351,7 +1356,8 @@ __global__ void __launch_bounds__(1024) shac_vec_kernel(DevFormat f, TablePlan t
         }
     };
     if (item < f.items) fetch();
-    // everything above reads the format only; x and the outputs belong to the kernels before this one
+    // everything above (index, spans of the first item, tables) reads the format only; x and the outputs
+    // belong to the kernels before this one
     depends_wait();
     if (bulk) {
         __syncthreads();                   // the mbarrier is initialised
@@ -1615,7 +1621,8 @@ __global__ void __launch_bounds__(1024) shac_items_kernel(DevFormat f, TablePlan
         __syncwarp();
     };
 
-    // everything above reads the format only; x and the outputs belong to the kernels before this one
+    // everything above (index, spans of the first item, tables) reads the format only; x and the outputs
+    // belong to the kernels before this one
     depends_wait();
     if (bulk) {
         if (threadIdx.x == 0 && bulk_bytes > 0) {
